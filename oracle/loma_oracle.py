@@ -1,0 +1,430 @@
+"""Plain fp64 NumPy oracle for LoMA's attention hot path.
+
+TEST INFRASTRUCTURE ONLY.  Nothing here is tuned, tiled, fused or reordered:
+each function takes the paper's definition and writes it out, so a reader can
+hold it against the paper by eye.  Floating point is float64 throughout
+(inputs are upcast exactly from whatever precision they were stored in).
+
+Notation (Section 3.1, Section 4.3):
+    c   compression ratio
+    t   memory-zone length (number of <m> tokens per chunk)
+    tc  = t*c, reading-zone length = repetition-zone length
+    s   = t*(2c+1) = 2*tc + t, length of one training chunk
+    n   number of complete chunks
+    tail_read  extra reading rows after the last complete chunk (the
+        uncompressed tail of an unfinished chunk; with t == 0 the whole
+        sequence is such a tail, i.e. ordinary causal attention)
+
+Readings of the paper taken here (each is listed with its evidence in the
+repository's design notes):
+  * a mask value of 0 removes the key from the softmax (weight exactly 0),
+    following the Fig. 5 caption rather than the literal product of Eq. 6;
+  * the softmax scale that Section 4.4 drops "without loss of generality" is an
+    explicit argument, default 1/sqrt(D);
+  * memory rows see only their own reading zone and their own memory zone
+    (Eq. 3 has zero memory rows; criterion 2 of Section 4.3; Appendix A slices
+    the last read_len cache entries).  FLAG_MEM_SEES_PRIOR_MEM switches on the
+    other reading, in which memory rows also see every earlier memory zone;
+  * memory position ids of chunk y are y*tc + (j+1)*c - 1 (Eq. 14 read together
+    with the generator listing, whose chunk start is y*tc);
+  * repetition-zone position ids repeat those of the reading token each row
+    reproduces.  The paper is silent on this one: PARITY UNPINNED for that
+    single output column of layout_index (pos_id on repetition rows).
+"""
+
+from __future__ import annotations
+
+import numpy as np
+
+FLAG_MEM_SEES_PRIOR_MEM = 1
+
+ZONE_READ = 0
+ZONE_MEM = 1
+ZONE_REP = 2
+
+
+# --------------------------------------------------------------------------
+# Layout (Section 4.1) and index maps (Eq. 14, Appendix A)
+# --------------------------------------------------------------------------
+
+def chunk_len(c: int, t: int) -> int:
+    """s = t(2c+1): reading zone + memory zone + repetition zone (Section 4.3)."""
+    return t * (2 * c + 1)
+
+
+def seq_len(n_chunks: int, c: int, t: int, tail_read: int = 0) -> int:
+    """Length of the laid-out sequence: n complete chunks plus a reading tail."""
+    return n_chunks * chunk_len(c, t) + tail_read
+
+
+def decompose(i: int, n_chunks: int, c: int, t: int):
+    """Row index -> (chunk y, zone z, offset o inside the zone) (Section 4.1).
+
+    Rows past the last complete chunk form the reading zone of chunk n_chunks.
+    """
+    tc = t * c
+    s = chunk_len(c, t)
+    if s == 0 or i >= n_chunks * s:
+        return n_chunks, ZONE_READ, i - n_chunks * s
+    y, r = divmod(i, s)
+    if r < tc:
+        return y, ZONE_READ, r
+    if r < tc + t:
+        return y, ZONE_MEM, r - tc
+    return y, ZONE_REP, r - tc - t
+
+
+def layout_index(n_chunks: int, c: int, t: int, tail_read: int = 0):
+    """Integer maps over the rows of the laid-out sequence.
+
+    Returns int32 arrays (chunk, zone, offset, src_token, pos_id), each [S].
+      src_token: index into the original token sequence that the row carries
+                 (reading rows) or must reproduce (repetition rows); -1 for <m>
+                 rows (Section 4.1, Eq. 13).
+      pos_id:    reading rows keep their original position y*tc+o; memory row j
+                 of chunk y gets y*tc+(j+1)c-1 (Eq. 14); repetition rows repeat
+                 the reading position (paper silent, unpinned).
+    """
+    tc = t * c
+    S = seq_len(n_chunks, c, t, tail_read)
+    chunk = np.zeros(S, np.int32)
+    zone = np.zeros(S, np.int32)
+    offset = np.zeros(S, np.int32)
+    src = np.zeros(S, np.int32)
+    pos = np.zeros(S, np.int32)
+    for i in range(S):
+        y, z, o = decompose(i, n_chunks, c, t)
+        chunk[i], zone[i], offset[i] = y, z, o
+        if z == ZONE_MEM:
+            src[i] = -1
+            pos[i] = y * tc + (o + 1) * c - 1
+        else:
+            src[i] = y * tc + o
+            pos[i] = y * tc + o
+    return chunk, zone, offset, src, pos
+
+
+def generation_index(n_tokens: int, c: int, t: int):
+    """Per generated token g: where its KV lands and what the cache looks like.
+
+    Section 3.1 steps 1-3 with the Appendix A bookkeeping: the cache holds
+    compressed_chunks*t memory entries followed by the uncompressed tail, and a
+    compress pass fires as soon as the tail reaches tc entries.
+
+    Returns int32 arrays [n_tokens]:
+      slot            cache index the token's K/V is appended at
+                      (= entries in the cache before the token)
+      pos_id          the generator's `cursor` value for the token (= g)
+      compress_after  1 if a compress pass runs right after this token
+    With t == 0 nothing is ever compressed (`while self.mem_len > 0`).
+    """
+    tc = t * c
+    slot = np.zeros(n_tokens, np.int32)
+    pos = np.zeros(n_tokens, np.int32)
+    comp = np.zeros(n_tokens, np.int32)
+    compressed_chunks = 0
+    tail = 0
+    for g in range(n_tokens):
+        slot[g] = compressed_chunks * t + tail
+        pos[g] = g
+        tail += 1
+        if t > 0 and tail == tc:
+            comp[g] = 1
+            compressed_chunks += 1
+            tail = 0
+    return slot, pos, comp
+
+
+# --------------------------------------------------------------------------
+# Mask (Eq. 1-3)
+# --------------------------------------------------------------------------
+
+def chunk_mask(c: int, t: int) -> np.ndarray:
+    """Eq. 1: the s x s mask of one training chunk, as a boolean array.
+
+        [ L  0  0 ]   reading rows: causal inside the reading zone
+        [ 1  1  0 ]   memory rows: whole reading zone + whole memory zone
+        [ 0  1  I ]   repetition rows: whole memory zone + the row itself
+    """
+    tc = t * c
+    L = np.tril(np.ones((tc, tc), bool))
+    I = np.eye(tc, dtype=bool)
+    Z = lambda a, b: np.zeros((a, b), bool)
+    O = lambda a, b: np.ones((a, b), bool)
+    return np.block([
+        [L,         Z(tc, t), Z(tc, tc)],
+        [O(t, tc),  O(t, t),  Z(t, tc)],
+        [Z(tc, tc), O(tc, t), I],
+    ])
+
+
+def cross_chunk_block(c: int, t: int, flags: int = 0) -> np.ndarray:
+    """Eq. 3: the s x s block linking a chunk (rows) to an EARLIER chunk (cols).
+
+    Only reading rows x memory columns are 1.  Under FLAG_MEM_SEES_PRIOR_MEM the
+    memory rows x memory columns block is 1 as well.
+    """
+    tc = t * c
+    s = chunk_len(c, t)
+    S = np.zeros((s, s), bool)
+    S[0:tc, tc:tc + t] = True
+    if flags & FLAG_MEM_SEES_PRIOR_MEM:
+        S[tc:tc + t, tc:tc + t] = True
+    return S
+
+
+def dense_mask(n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0) -> np.ndarray:
+    """Eq. 2: the whole-sample mask, block lower triangular in chunks.
+
+    Diagonal blocks are Eq. 1, blocks below the diagonal are Eq. 3, blocks above
+    are zero.  A reading tail (an unfinished chunk) contributes the leading
+    tail_read rows/cols of one more chunk row: reading rows of Eq. 3 towards
+    every earlier chunk and the leading corner of L on the diagonal.
+    """
+    s = chunk_len(c, t)
+    S = seq_len(n_chunks, c, t, tail_read)
+    M = np.zeros((S, S), bool)
+    if n_chunks > 0:
+        Mc = chunk_mask(c, t)
+        Sc = cross_chunk_block(c, t, flags)
+        for y in range(n_chunks):
+            for x in range(y):
+                M[y * s:(y + 1) * s, x * s:(x + 1) * s] = Sc
+            M[y * s:(y + 1) * s, y * s:(y + 1) * s] = Mc
+        if tail_read:
+            for x in range(n_chunks):
+                M[n_chunks * s:, x * s:(x + 1) * s] = Sc[:tail_read, :]
+    if tail_read:
+        M[n_chunks * s:, n_chunks * s:] = np.tril(np.ones((tail_read, tail_read), bool))
+    return M
+
+
+def allowed(i: int, j: int, n_chunks: int, c: int, t: int, flags: int = 0) -> bool:
+    """May row i attend to column j?  Eq. 1-3 read entry by entry."""
+    yi, zi, oi = decompose(i, n_chunks, c, t)
+    yj, zj, oj = decompose(j, n_chunks, c, t)
+    if yj > yi:
+        return False                       # Eq. 2: zero above the block diagonal
+    if yj == yi:                           # Eq. 1
+        if zi == ZONE_READ:
+            return zj == ZONE_READ and oj <= oi
+        if zi == ZONE_MEM:
+            return zj in (ZONE_READ, ZONE_MEM)
+        return zj == ZONE_MEM or j == i
+    # yj < yi: Eq. 3
+    if zi == ZONE_READ and zj == ZONE_MEM:
+        return True
+    if (flags & FLAG_MEM_SEES_PRIOR_MEM) and zi == ZONE_MEM and zj == ZONE_MEM:
+        return True
+    return False
+
+
+def mask_rows(rows, n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0) -> np.ndarray:
+    """Selected rows of the Eq. 2 mask, built from the entry-wise rule.
+
+    For sequences whose full S x S mask does not fit in memory.  Returns a
+    boolean [len(rows), S].
+    """
+    S = seq_len(n_chunks, c, t, tail_read)
+    ch, zn, of, _, _ = layout_index(n_chunks, c, t, tail_read)
+    cols = np.arange(S)
+    out = np.zeros((len(rows), S), bool)
+    for r, i in enumerate(rows):
+        yi, zi, oi = int(ch[i]), int(zn[i]), int(of[i])
+        same = ch == yi
+        earlier = ch < yi
+        if zi == ZONE_READ:
+            row = (same & (zn == ZONE_READ) & (of <= oi)) | (earlier & (zn == ZONE_MEM))
+        elif zi == ZONE_MEM:
+            row = same & ((zn == ZONE_READ) | (zn == ZONE_MEM))
+            if flags & FLAG_MEM_SEES_PRIOR_MEM:
+                row = row | (earlier & (zn == ZONE_MEM))
+        else:
+            row = (same & (zn == ZONE_MEM)) | (cols == i)
+        out[r] = row
+    return out
+
+
+# --------------------------------------------------------------------------
+# Attention (Eq. 5-7)
+# --------------------------------------------------------------------------
+
+def _f64(x) -> np.ndarray:
+    return np.asarray(x, dtype=np.float64)
+
+
+def masked_softmax_attention(q, k, v, mask, scale=None):
+    """O = Softmax(A) V with A = scale * Q K^T restricted to mask (Eq. 5-7).
+
+    q [R, D], k [C, D], v [C, Dv], mask boolean [R, C] (True = attend).
+    Masked keys get weight exactly 0.  Every row must have at least one True.
+    Returns (O [R, Dv], P [R, C], lse [R]) in float64; lse is the natural-log
+    normaliser log(sum_j exp(A_ij)) over the allowed keys.
+    """
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    if scale is None:
+        scale = 1.0 / np.sqrt(q.shape[-1])
+    A = scale * (q @ k.T)
+    A = np.where(mask, A, -np.inf)
+    m = A.max(axis=1, keepdims=True)
+    E = np.exp(A - m)
+    l = E.sum(axis=1, keepdims=True)
+    P = E / l
+    O = P @ v
+    lse = (m + np.log(l))[:, 0]
+    return O, P, lse
+
+
+def masked_attn_fwd(q, k, v, n_chunks, c, t, tail_read=0, flags=0, scale=None,
+                    rows=None, return_p=False):
+    """Zone-masked attention over the laid-out sequence.
+
+    q, k, v: [B, H, S, D] with S = n_chunks*s + tail_read.
+    rows: optional list of row indices; if given only those rows are computed
+          (against all S keys) and the outputs have len(rows) in place of S.
+    Returns (O [B,H,R,D], lse [B,H,R]) and, with return_p, also P [B,H,R,S].
+    """
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    B, H, S, D = q.shape
+    assert S == seq_len(n_chunks, c, t, tail_read)
+    if rows is None:
+        rows = np.arange(S)
+        M = dense_mask(n_chunks, c, t, tail_read, flags)
+    else:
+        rows = np.asarray(rows)
+        M = mask_rows(rows, n_chunks, c, t, tail_read, flags)
+    R = len(rows)
+    O = np.zeros((B, H, R, v.shape[-1]))
+    LSE = np.zeros((B, H, R))
+    P = np.zeros((B, H, R, S)) if return_p else None
+    for b in range(B):
+        for h in range(H):
+            o, p, lse = masked_softmax_attention(q[b, h][rows], k[b, h], v[b, h], M, scale)
+            O[b, h], LSE[b, h] = o, lse
+            if return_p:
+                P[b, h] = p
+    if return_p:
+        return O, LSE, P
+    return O, LSE
+
+
+# --------------------------------------------------------------------------
+# Generation (Section 3.1, Appendix A)
+# --------------------------------------------------------------------------
+
+def decode_attn(q, k_new, v_new, k_cache, v_cache, cache_len, scale=None):
+    """One decode step: a single new token over the whole cache plus itself.
+
+    Appendix A `inference_input` with one input token: the mask row is all ones
+    over the cache_len cached entries and the token's own column
+    (tril(..., diagonal=cache_len)), and the token's K/V is appended.
+
+    q, k_new, v_new: [B, H, 1, D]; k_cache, v_cache: [B, H, cap, D] of which the
+    first cache_len entries are valid.
+    Returns (o [B,H,1,D], lse [B,H,1], k_cache', v_cache') where the primed
+    caches are copies with entry cache_len filled in.
+    """
+    q = _f64(q)
+    B, H, _, D = q.shape
+    kc = np.array(k_cache, copy=True)
+    vc = np.array(v_cache, copy=True)
+    kc[:, :, cache_len, :] = np.asarray(k_new)[:, :, 0, :]
+    vc[:, :, cache_len, :] = np.asarray(v_new)[:, :, 0, :]
+    o = np.zeros((B, H, 1, D))
+    lse = np.zeros((B, H, 1))
+    ones = np.ones((1, cache_len + 1), bool)
+    for b in range(B):
+        for h in range(H):
+            keys = kc[b, h, :cache_len + 1]
+            vals = vc[b, h, :cache_len + 1]
+            o[b, h], _, lse[b, h] = masked_softmax_attention(q[b, h], keys, vals, ones, scale)
+    return o, lse, kc, vc
+
+
+def compress_step(q_mem, k_mem, v_mem, k_cache, v_cache, mem_len, c, t, flags=0, scale=None):
+    """Compress pass + compaction (Section 3.1 steps 2-3; Appendix A
+    `compress_last_chunk`).
+
+    Before: the cache holds mem_len memory entries followed by exactly tc tail
+    entries (the listing asserts this).  The t <m> queries attend, with an
+    all-ones mask, to the tc tail entries and to their own t keys.  Under
+    FLAG_MEM_SEES_PRIOR_MEM the mem_len earlier memory entries are visible too.
+    After: cache' = concatenate(cache[:mem_len], k_mem), valid length mem_len+t.
+
+    q_mem, k_mem, v_mem: [B, H, t, D]; caches [B, H, cap, D].
+    Returns (o_mem [B,H,t,D], lse [B,H,t], k_cache' [B,H,mem_len+t,D], v_cache').
+    """
+    tc = t * c
+    q_mem = _f64(q_mem)
+    k_cache = np.asarray(k_cache)
+    v_cache = np.asarray(v_cache)
+    k_mem_a = np.asarray(k_mem)
+    v_mem_a = np.asarray(v_mem)
+    B, H, _, D = q_mem.shape
+    lo = 0 if (flags & FLAG_MEM_SEES_PRIOR_MEM) else mem_len
+    o = np.zeros((B, H, t, D))
+    lse = np.zeros((B, H, t))
+    for b in range(B):
+        for h in range(H):
+            keys = np.concatenate([_f64(k_cache[b, h, lo:mem_len + tc]), _f64(k_mem_a[b, h])], axis=0)
+            vals = np.concatenate([_f64(v_cache[b, h, lo:mem_len + tc]), _f64(v_mem_a[b, h])], axis=0)
+            ones = np.ones((t, keys.shape[0]), bool)
+            o[b, h], _, lse[b, h] = masked_softmax_attention(q_mem[b, h], keys, vals, ones, scale)
+    # Compaction by explicit copies into fresh arrays.
+    new_k = np.empty((B, H, mem_len + t, D), dtype=k_cache.dtype)
+    new_v = np.empty((B, H, mem_len + t, D), dtype=v_cache.dtype)
+    for b in range(B):
+        for h in range(H):
+            for e in range(mem_len):
+                new_k[b, h, e] = k_cache[b, h, e]
+                new_v[b, h, e] = v_cache[b, h, e]
+            for j in range(t):
+                new_k[b, h, mem_len + j] = k_mem_a[b, h, j]
+                new_v[b, h, mem_len + j] = v_mem_a[b, h, j]
+    return o, lse, new_k, new_v
+
+
+def replay_generation(q, k, v, n_chunks, c, t, tail_read=0, flags=0, scale=None):
+    """Run the laid-out sequence through the generation path chunk by chunk.
+
+    For chunk y: the tc reading rows are decoded one token at a time, then the t
+    memory rows run as one compress pass and the cache is compacted.  Repetition
+    rows have no counterpart at generation time and are left as NaN.  A reading
+    tail is decoded after the last compress.
+
+    Returns (O [B,H,S,D] with NaN on repetition rows, k_cache, v_cache, length):
+    the final cache arrays [B,H,cap,D] and their valid length.
+    """
+    q, k, v = np.asarray(q), np.asarray(k), np.asarray(v)
+    B, H, S, D = q.shape
+    tc = t * c
+    s = chunk_len(c, t)
+    cap = n_chunks * t + max(tc, tail_read) + 1
+    kc = np.zeros((B, H, cap, D), dtype=k.dtype)
+    vc = np.zeros((B, H, cap, D), dtype=v.dtype)
+    O = np.full((B, H, S, D), np.nan)
+    length = 0
+    for y in range(n_chunks):
+        base = y * s
+        for o_ in range(tc):
+            i = base + o_
+            out, _, kc, vc = decode_attn(q[:, :, i:i + 1], k[:, :, i:i + 1], v[:, :, i:i + 1],
+                                         kc, vc, length, scale)
+            O[:, :, i] = out[:, :, 0]
+            length += 1
+        m0 = base + tc
+        mem_len = y * t
+        assert length == mem_len + tc
+        out, _, nk, nv = compress_step(q[:, :, m0:m0 + t], k[:, :, m0:m0 + t], v[:, :, m0:m0 + t],
+                                       kc, vc, mem_len, c, t, flags, scale)
+        O[:, :, m0:m0 + t] = out
+        length = mem_len + t
+        kc[:, :, :length] = nk
+        vc[:, :, :length] = nv
+    for o_ in range(tail_read):
+        i = n_chunks * s + o_
+        out, _, kc, vc = decode_attn(q[:, :, i:i + 1], k[:, :, i:i + 1], v[:, :, i:i + 1],
+                                     kc, vc, length, scale)
+        O[:, :, i] = out[:, :, 0]
+        length += 1
+    return O, kc, vc, length
