@@ -1,0 +1,241 @@
+/*
+ * loma.h -- C ABI of the LoMA (Lossless Compressed Memory Attention,
+ * arxiv 2401.09486) attention hot path for NVIDIA B200 (sm_100a).
+ *
+ * Three device operations and two integer index maps:
+ *
+ *   loma_masked_attn_fwd   zone-masked attention over the training layout
+ *                          (Section 4.3, Eq. 1-3; Section 4.4, Eq. 5-7)
+ *   loma_decode_attn       one generated token over the compressed cache
+ *                          (Section 3.1 steps 1 and 3; Appendix A, inference_input)
+ *   loma_compress_step     the t <m> queries over the uncompressed tail, fused
+ *                          with the in-place compaction of the cache
+ *                          (Section 3.1 steps 2-3; Appendix A, compress_last_chunk)
+ *   loma_layout_index      row -> (chunk, zone, offset, source token, position id)
+ *                          (Section 4.1; Section 4.5, Eq. 14)
+ *   loma_generation_index  generated token -> cache slot / position / compress flag
+ *                          (Section 3.1; Appendix A, add_token_ids)
+ *
+ * Notation (Section 3.1, Section 4.3):  c = compression ratio, t = memory-zone
+ * length, tc = t*c = reading-zone length = repetition-zone length,
+ * s = t*(2c+1) = chunk length.  A laid-out sequence is n_chunks chunks
+ * [tc reading | t memory | tc repetition] followed by tail_read extra reading
+ * rows (an unfinished chunk); S = n_chunks*s + tail_read.
+ *
+ * Conventions common to every entry point
+ *   - Return value: LOMA_OK (0) or a negative loma_status.  Nothing throws,
+ *     aborts or traps the device.  Arguments are validated on the host before
+ *     anything is launched; on error nothing has been launched.
+ *   - Pointers marked [device] are CUDA device pointers on the current device;
+ *     [host] are ordinary host pointers.  The caller owns every buffer before
+ *     and after the call; the library allocates no device memory and keeps no
+ *     pointer beyond the call.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
+ *     work is enqueued on it and the call returns without synchronising.
+ *   - Tensors are row-major with the head dimension D contiguous.  D is 64 or
+ *     128.  dtype is LOMA_F32 or LOMA_BF16 for every tensor of the call;
+ *     accumulation and softmax are always fp32; bf16 outputs are rounded to
+ *     nearest even.  Log-sum-exp outputs are fp32, natural log, and may be NULL.
+ *   - softmax_scale <= 0 selects 1/sqrt(D) (the factor Section 4.4 drops
+ *     "without loss of generality").
+ *   - A mask value of 0 removes the key from the softmax (its weight is exactly
+ *     zero), as the Fig. 5 caption describes.
+ *   - Results are bitwise repeatable for fixed arguments.
+ *   - Kernels that wait (on an mbarrier) do so with an iteration limit; on
+ *     expiry they record LOMA_ERR_TIMEOUT in a device status word and return.
+ *     loma_device_status() reads that word.
+ */
+#ifndef LOMA_H_
+#define LOMA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define LOMA_API __attribute__((visibility("default")))
+#else
+#define LOMA_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LOMA_OK = 0,
+    LOMA_ERR_INVALID_ARG = -1, /* NULL pointer, negative size, tc != c*t, ...        */
+    LOMA_ERR_UNSUPPORTED = -2, /* D not in {64,128}, unknown dtype, device not sm_100 */
+    LOMA_ERR_ALIGNMENT = -3,   /* pointer or stride not 16-byte aligned              */
+    LOMA_ERR_CAPACITY = -4,    /* cache capacity too small for the request           */
+    LOMA_ERR_WORKSPACE = -5,   /* workspace NULL or smaller than *_workspace_bytes    */
+    LOMA_ERR_CUDA = -6,        /* a CUDA runtime/driver call failed                  */
+    LOMA_ERR_TIMEOUT = -7      /* a bounded device-side wait expired                 */
+} loma_status;
+
+typedef enum { LOMA_F32 = 0, LOMA_BF16 = 1 } loma_dtype;
+
+enum {
+    /* Section 4.3 criterion 2 and Eq. 3 (memory rows all zero) say that memory
+     * rows see only their own reading zone and their own memory zone, and
+     * Appendix A hands the compress pass only the last tc cache entries.  That
+     * is the default.  With this flag memory rows additionally see every earlier
+     * memory zone (masked forward) and the compress pass additionally attends to
+     * the mem_len memory entries already in the cache; both change together so
+     * that incremental generation still equals the one-shot forward. */
+    LOMA_FLAG_MEM_SEES_PRIOR_MEM = 1u,
+    /* Run the plain CUDA-core kernel even where a tensor-core kernel exists
+     * (second opinion for tests; always used for LOMA_F32). */
+    LOMA_FLAG_FORCE_GENERIC = 1u << 8
+};
+
+/* Zone codes written by loma_layout_index. */
+enum { LOMA_ZONE_READ = 0, LOMA_ZONE_MEM = 1, LOMA_ZONE_REP = 2 };
+
+/* ---------------------------------------------------------------------------
+ * loma_layout_index -- Section 4.1 (chunk layout) and Eq. 14 (position ids).
+ *
+ * For every row i of a laid-out sequence of S = n_chunks*t*(2c+1) + tail_read
+ * rows writes
+ *   chunk[i]      y = i div s                       (tail rows: n_chunks)
+ *   zone[i]       LOMA_ZONE_READ / _MEM / _REP
+ *   offset[i]     position inside the zone
+ *   src_token[i]  y*tc + offset for reading rows (the original token carried)
+ *                 and repetition rows (the token to reproduce, Eq. 13);
+ *                 -1 for <m> rows
+ *   pos_id[i]     reading rows: y*tc + offset (original ids are preserved);
+ *                 memory row j: y*tc + (j+1)*c - 1 (Eq. 14, chunk start y*tc as
+ *                 in the Appendix A listing); repetition rows: y*tc + offset
+ *                 (the paper does not say; same id as the token reproduced).
+ * Each output is int32[S]; any of them may be NULL (skipped).  on_device != 0:
+ * outputs are [device] and filled by a kernel on `stream`; on_device == 0:
+ * outputs are [host], filled synchronously, no CUDA call is made.
+ * t == 0 requires n_chunks == 0 (the sequence is one reading zone).
+ * Errors: INVALID_ARG (negative sizes, c < 1, t == 0 with n_chunks > 0,
+ * t > 0 with tail_read > tc, S > INT32_MAX), CUDA.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_layout_index(int n_chunks, int c, int t, int tail_read,
+                               int32_t* chunk, int32_t* zone, int32_t* offset,
+                               int32_t* src_token, int32_t* pos_id,
+                               int on_device, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * loma_generation_index -- Section 3.1 steps 1-3, Appendix A add_token_ids.
+ *
+ * For generated token g = 0..n_tokens-1 (no prompt), with the cache holding
+ * compressed_chunks*t memory entries followed by the uncompressed tail:
+ *   slot[g]            cache index the token's K/V is appended at
+ *                      = (g div tc)*t + g mod tc   (= g when t == 0)
+ *   pos_id[g]          g (the generator's cursor)
+ *   compress_after[g]  1 if the tail reaches tc with this token, i.e. a compress
+ *                      pass follows it; always 0 when t == 0
+ * Outputs int32[n_tokens], NULL = skipped; on_device as above.
+ * Errors: INVALID_ARG, CUDA.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_generation_index(int n_tokens, int c, int t,
+                                   int32_t* slot, int32_t* pos_id, int32_t* compress_after,
+                                   int on_device, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * loma_masked_attn_fwd -- O = Softmax(A) V with A = scale * Q K^T restricted to
+ * the mask M of Eq. 2 (diagonal blocks Eq. 1, sub-diagonal blocks Eq. 3),
+ * evaluated row by row as in Eq. 7.  The mask is never stored: it is computed
+ * from (chunk, zone, offset) of the row and the key, and tiles with no allowed
+ * entry are skipped.
+ *
+ *   q, k, v [device, in]   [B, H, S, D], element (b,h,i,d) at
+ *                          b*stride_b + h*stride_h + i*stride_s + d  (elements)
+ *   o       [device, out]  same shape and strides as q
+ *   lse     [device, out]  fp32 [B, H, S] contiguous, or NULL
+ *   n_chunks, c, t, tc, tail_read   layout; tc must equal c*t; t == 0 requires
+ *                          n_chunks == 0 and gives plain causal attention over
+ *                          tail_read rows; t > 0 requires tail_read <= tc
+ *   flags                  LOMA_FLAG_* bits
+ * o must not alias q, k or v.  Rows are independent; every row has at least one
+ * allowed key (itself), so no output is undefined.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT (pointers and byte strides must be
+ * multiples of 16), CUDA.  S == 0 or B*H == 0 is a successful no-op.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_masked_attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse,
+                                  int B, int H, int D,
+                                  int n_chunks, int c, int t, int tc, int tail_read,
+                                  int64_t stride_b, int64_t stride_h, int64_t stride_s,
+                                  loma_dtype dtype, float softmax_scale, unsigned flags, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * loma_decode_attn -- one new token per (batch, head) attends to the cache_len
+ * entries already in the cache (all memory entries, then the uncompressed tail)
+ * and to itself: the mask row tril(ones(1, 1+k), diagonal=k) of Appendix A with
+ * k = cache_len.  Its key and value are appended at slot cache_len.
+ *
+ *   q               [device, in]      [B, H, 1, D] contiguous
+ *   k_new, v_new    [device, in]      [B, H, 1, D] contiguous; both NULL means the
+ *                                     token's K/V already sit at slot cache_len
+ *   k_cache, v_cache [device, in/out] [B, H, cap, D] contiguous; entries
+ *                                     [0, cache_len) are read, entry cache_len is
+ *                                     written (when k_new is given); nothing else
+ *                                     is touched
+ *   o               [device, out]     [B, H, 1, D] contiguous
+ *   lse             [device, out]     fp32 [B, H], or NULL
+ *   cache_len       entries before this token, the same for every (b,h);
+ *                   requires 0 <= cache_len < cap
+ *   workspace       [device] scratch of at least
+ *                   loma_decode_workspace_bytes(B,H,D,cache_len) bytes, 16-byte
+ *                   aligned; contents on entry and exit are unspecified
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CAPACITY (cache_len >= cap),
+ * WORKSPACE, CUDA.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_decode_attn(const void* q, const void* k_new, const void* v_new,
+                              void* k_cache, void* v_cache, void* o, float* lse,
+                              int B, int H, int D, int cap, int cache_len,
+                              loma_dtype dtype, float softmax_scale, unsigned flags,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
+LOMA_API size_t loma_decode_workspace_bytes(int B, int H, int D, int cache_len);
+
+/* ---------------------------------------------------------------------------
+ * loma_compress_step -- Section 3.1 step 2 (one pass of t <m> tokens over
+ * KV_Read) and step 3 (KV_Read is discarded), fused.
+ *
+ * Precondition (asserted by the Appendix A listing): the cache holds mem_len
+ * memory entries followed by exactly tc tail entries.  The t memory queries
+ * attend with an all-ones t x (tc+t) mask to the tail and to their own keys
+ * (with LOMA_FLAG_MEM_SEES_PRIOR_MEM also to entries [0, mem_len)).  Then the
+ * cache becomes cat(cache[:mem_len], k_mem): k_mem / v_mem are copied, bit for
+ * bit, into slots [mem_len, mem_len+t), overwriting the first tail entries
+ * only after every read of them has completed.
+ *
+ *   q_mem, k_mem, v_mem [device, in]  [B, H, t, D] contiguous
+ *   k_cache, v_cache [device, in/out] [B, H, cap, D] contiguous, cap >= mem_len+tc
+ *   o_mem            [device, out]    [B, H, t, D] contiguous
+ *   lse              [device, out]    fp32 [B, H, t], or NULL
+ * Postcondition: the valid cache length is mem_len + t; entries [0, mem_len) are
+ * untouched; entries at and beyond mem_len + t are unspecified.
+ * Requires t >= 1, c >= 1, tc == c*t, mem_len >= 0.
+ *   workspace  [device] at least loma_compress_workspace_bytes(...) bytes
+ *              (NULL is accepted when that is 0)
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CAPACITY, WORKSPACE, CUDA.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_compress_step(const void* q_mem, const void* k_mem, const void* v_mem,
+                                void* k_cache, void* v_cache, void* o_mem, float* lse,
+                                int B, int H, int D, int cap, int mem_len, int c, int t, int tc,
+                                loma_dtype dtype, float softmax_scale, unsigned flags,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
+LOMA_API size_t loma_compress_workspace_bytes(int B, int H, int D, int t, int mem_len, unsigned flags);
+
+/* Synchronises `stream`, then returns the device status word of the current
+ * device: LOMA_OK, or LOMA_ERR_TIMEOUT if a bounded wait inside a kernel has
+ * expired since the last call (the word is cleared by the call).
+ * LOMA_ERR_CUDA if the synchronisation or the read fails. */
+LOMA_API int loma_device_status(void* stream);
+
+/* Static, human-readable name of a status code. */
+LOMA_API const char* loma_status_string(int status);
+
+/* Library version: major*10000 + minor*100 + patch. */
+LOMA_API int loma_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOMA_H_ */

@@ -1,0 +1,185 @@
+"""ctypes binding of libloma (declared in ``include/loma.h``).
+
+Argument marshalling only: every function here has the name of the C entry
+point it calls, takes torch tensors (device memory) or plain ints, pulls out
+pointers, shapes and strides, and raises :class:`LomaError` on a negative
+status.  No arithmetic of the method happens in Python, and there is no
+fallback: if the library has not been built, loading fails with an error.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+LOMA_F32 = 0
+LOMA_BF16 = 1
+LOMA_FLAG_MEM_SEES_PRIOR_MEM = 1
+LOMA_FLAG_FORCE_GENERIC = 1 << 8
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libloma.so")
+_lib = None
+
+_i, _i64, _f, _u, _p, _sz = (ctypes.c_int, ctypes.c_int64, ctypes.c_float, ctypes.c_uint, ctypes.c_void_p,
+                             ctypes.c_size_t)
+
+# name -> (restype, argtypes); mirrors include/loma.h
+SIGNATURES = {
+    "loma_layout_index": (_i, [_i, _i, _i, _i, _p, _p, _p, _p, _p, _i, _p]),
+    "loma_generation_index": (_i, [_i, _i, _i, _p, _p, _p, _i, _p]),
+    "loma_masked_attn_fwd": (_i, [_p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i, _f,
+                                  _u, _p]),
+    "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
+    "loma_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
+    "loma_compress_step": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz,
+                                _p]),
+    "loma_compress_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _u]),
+    "loma_device_status": (_i, [_p]),
+    "loma_status_string": (ctypes.c_char_p, [_i]),
+    "loma_version": (_i, []),
+}
+
+
+class LomaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def lib() -> ctypes.CDLL:
+    """Load libloma.so once.  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2401_09486_b200.build` "
+                "(there is no fallback path)")
+        handle = ctypes.CDLL(_LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = handle
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().loma_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise LomaError(status, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return LOMA_F32
+    if t.dtype == torch.bfloat16:
+        return LOMA_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    elif isinstance(stream, torch.cuda.Stream):
+        stream = stream.cuda_stream
+    return ctypes.c_void_p(int(stream))
+
+
+def loma_version() -> int:
+    return lib().loma_version()
+
+
+def loma_device_status(stream=None) -> int:
+    return lib().loma_device_status(_stream(stream))
+
+
+def loma_layout_index(n_chunks: int, c: int, t: int, tail_read: int = 0, device="cpu", stream=None):
+    """Returns int32 tensors (chunk, zone, offset, src_token, pos_id) on `device`."""
+    tc = c * t
+    S = n_chunks * (2 * tc + t) + tail_read
+    on_device = torch.device(device).type == "cuda"
+    outs = [torch.empty(max(S, 0), dtype=torch.int32, device=device) for _ in range(5)]
+    st = _stream(stream) if on_device else None
+    rc = lib().loma_layout_index(n_chunks, c, t, tail_read, *[_ptr(x) for x in outs], int(on_device), st)
+    _check(rc, "loma_layout_index")
+    return tuple(outs)
+
+
+def loma_generation_index(n_tokens: int, c: int, t: int, device="cpu", stream=None):
+    """Returns int32 tensors (slot, pos_id, compress_after) on `device`."""
+    on_device = torch.device(device).type == "cuda"
+    outs = [torch.empty(max(n_tokens, 0), dtype=torch.int32, device=device) for _ in range(3)]
+    st = _stream(stream) if on_device else None
+    rc = lib().loma_generation_index(n_tokens, c, t, *[_ptr(x) for x in outs], int(on_device), st)
+    _check(rc, "loma_generation_index")
+    return tuple(outs)
+
+
+def loma_masked_attn_fwd(q, k, v, o, lse, n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0,
+                         softmax_scale: float = 0.0, stream=None) -> None:
+    """q, k, v, o: [B, H, S, D] device tensors with identical strides, D contiguous;
+    lse: fp32 [B, H, S] contiguous or None."""
+    B, H, S, D = q.shape
+    for x in (k, v, o):
+        if x.shape != q.shape or x.stride() != q.stride() or x.dtype != q.dtype:
+            raise ValueError("q, k, v, o must share shape, strides and dtype")
+    if q.stride(3) != 1:
+        raise ValueError("head dimension must be contiguous")
+    if lse is not None and (lse.dtype != torch.float32 or not lse.is_contiguous()):
+        raise ValueError("lse must be contiguous fp32")
+    rc = lib().loma_masked_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), B, H, D, n_chunks, c, t, c * t,
+                                    tail_read, q.stride(0), q.stride(1), q.stride(2), _dtype_code(q),
+                                    float(softmax_scale), int(flags), _stream(stream))
+    _check(rc, "loma_masked_attn_fwd")
+
+
+def loma_decode_workspace_bytes(B: int, H: int, D: int, cache_len: int) -> int:
+    return int(lib().loma_decode_workspace_bytes(B, H, D, cache_len))
+
+
+def loma_decode_attn(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len: int, workspace=None, flags: int = 0,
+                     softmax_scale: float = 0.0, stream=None) -> None:
+    """q, k_new, v_new, o: [B, H, 1, D]; caches [B, H, cap, D]; all contiguous."""
+    B, H, cap, D = k_cache.shape
+    for x in (q, k_new, v_new, k_cache, v_cache, o):
+        if x is not None and not x.is_contiguous():
+            raise ValueError("decode tensors must be contiguous")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().loma_decode_attn(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(o),
+                                _ptr(lse), B, H, D, cap, cache_len, _dtype_code(q), float(softmax_scale),
+                                int(flags), _ptr(workspace), ws_bytes, _stream(stream))
+    _check(rc, "loma_decode_attn")
+
+
+def loma_compress_workspace_bytes(B: int, H: int, D: int, t: int, mem_len: int, flags: int = 0) -> int:
+    return int(lib().loma_compress_workspace_bytes(B, H, D, t, mem_len, int(flags)))
+
+
+def loma_compress_step(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, mem_len: int, c: int, t: int,
+                       workspace=None, flags: int = 0, softmax_scale: float = 0.0, stream=None) -> None:
+    """q_mem, k_mem, v_mem, o_mem: [B, H, t, D]; caches [B, H, cap, D]; all contiguous."""
+    B, H, cap, D = k_cache.shape
+    for x in (q_mem, k_mem, v_mem, k_cache, v_cache, o_mem):
+        if not x.is_contiguous():
+            raise ValueError("compress tensors must be contiguous")
+    if q_mem.shape[2] != t:
+        raise ValueError("q_mem must have t rows")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().loma_compress_step(_ptr(q_mem), _ptr(k_mem), _ptr(v_mem), _ptr(k_cache), _ptr(v_cache),
+                                  _ptr(o_mem), _ptr(lse), B, H, D, cap, mem_len, c, t, c * t, _dtype_code(q_mem),
+                                  float(softmax_scale), int(flags), _ptr(workspace), ws_bytes, _stream(stream))
+    _check(rc, "loma_compress_step")

@@ -1,0 +1,394 @@
+// Plain CUDA-core attention kernels: one warp per query row, fp32 arithmetic.
+//
+// These serve three purposes: the fp32 path (tensor cores would cost mantissa
+// bits the 1e-5 bar does not allow), geometries the tensor-core kernels do not
+// cover, and an on-GPU second opinion (LOMA_FLAG_FORCE_GENERIC).
+//
+// Every row of Eq. 7 is an independent softmax over the keys its mask row
+// allows.  For each kind of row those keys form a short list of contiguous
+// ranges, so a row is described by a count of visible keys and a map from a
+// "visible index" to a key pointer -- the mask of Eq. 1-3 is never stored:
+//   reading row (y, o):    memory zones of chunks 0..y-1, then own reading
+//                          zone up to and including o            (Eq. 1 L, Eq. 3)
+//   memory row (y, j):     own reading zone and own memory zone  (Eq. 1 row 2)
+//                          [+ earlier memory zones with the prior-memory flag]
+//   repetition row (y, o): own memory zone, then itself          (Eq. 1 row 3)
+//   decode:                cache[0, len) then the new token      (Appendix A)
+//   compress:              cache tail (tc) then the t own keys   (Appendix A)
+#include <math.h>
+
+#include "loma_internal.cuh"
+
+namespace loma {
+
+// ---------------------------------------------------------------- element IO
+template <typename T>
+struct Io;
+
+template <>
+struct Io<float> {
+    // dot of a D-float row in shared memory with a D-element global row
+    template <int D>
+    static __device__ __forceinline__ float dot(const float* __restrict__ qs, const float* __restrict__ kp) {
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        const float4* k4 = reinterpret_cast<const float4*>(kp);
+        const float4* q4 = reinterpret_cast<const float4*>(qs);
+#pragma unroll
+        for (int i = 0; i < D / 4; ++i) {
+            const float4 kv = __ldg(k4 + i);
+            const float4 qv = q4[i];
+            a0 = fmaf(qv.x, kv.x, a0);
+            a1 = fmaf(qv.y, kv.y, a1);
+            a2 = fmaf(qv.z, kv.z, a2);
+            a3 = fmaf(qv.w, kv.w, a3);
+        }
+        return (a0 + a1) + (a2 + a3);
+    }
+    template <int N>
+    static __device__ __forceinline__ void load(const float* p, float (&x)[N]) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) x[i] = __ldg(p + i);
+    }
+    template <int N>
+    static __device__ __forceinline__ void store(float* p, const float (&x)[N]) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) p[i] = x[i];
+    }
+};
+
+template <>
+struct Io<__nv_bfloat16> {
+    template <int D>
+    static __device__ __forceinline__ float dot(const float* __restrict__ qs,
+                                                const __nv_bfloat16* __restrict__ kp) {
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        const uint4* k8 = reinterpret_cast<const uint4*>(kp);
+        const float4* q4 = reinterpret_cast<const float4*>(qs);
+#pragma unroll
+        for (int i = 0; i < D / 8; ++i) {
+            const uint4 kv = __ldg(k8 + i);
+            const float4 qa = q4[2 * i], qb = q4[2 * i + 1];
+            a0 = fmaf(qa.x, bf16lo(kv.x), a0);
+            a1 = fmaf(qa.y, bf16hi(kv.x), a1);
+            a2 = fmaf(qa.z, bf16lo(kv.y), a2);
+            a3 = fmaf(qa.w, bf16hi(kv.y), a3);
+            a0 = fmaf(qb.x, bf16lo(kv.z), a0);
+            a1 = fmaf(qb.y, bf16hi(kv.z), a1);
+            a2 = fmaf(qb.z, bf16lo(kv.w), a2);
+            a3 = fmaf(qb.w, bf16hi(kv.w), a3);
+        }
+        return (a0 + a1) + (a2 + a3);
+    }
+    template <int N>
+    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&x)[N]) {
+        static_assert(N % 2 == 0, "pairs");
+        const uint32_t* u = reinterpret_cast<const uint32_t*>(p);
+#pragma unroll
+        for (int i = 0; i < N / 2; ++i) {
+            const uint32_t w = __ldg(u + i);
+            x[2 * i] = bf16lo(w);
+            x[2 * i + 1] = bf16hi(w);
+        }
+    }
+    template <int N>
+    static __device__ __forceinline__ void store(__nv_bfloat16* p, const float (&x)[N]) {
+        uint32_t* u = reinterpret_cast<uint32_t*>(p);
+#pragma unroll
+        for (int i = 0; i < N / 2; ++i) u[i] = pack_bf16(x[2 * i], x[2 * i + 1]);
+    }
+};
+
+// ------------------------------------------------------------ one query row
+// qs: the row's query as D floats in shared memory (this warp's slice).
+// map.kptr(v) / map.vptr(v): pointer to the D-element key / value row of
+// visible index v, 0 <= v < nkeys.  Online softmax over blocks of 32 keys:
+// lane = key for the scores, lane = slice of D for the output.
+template <typename T, int D, typename Map>
+__device__ __forceinline__ void attend_row(const float* qs, const Map& map, int nkeys, float scale,
+                                           T* o_out, float* lse_out, int lane) {
+    constexpr int DPL = D / 32;
+    float o[DPL];
+#pragma unroll
+    for (int d = 0; d < DPL; ++d) o[d] = 0.f;
+    float m = -INFINITY, l = 0.f;
+    for (int base = 0; base < nkeys; base += 32) {
+        const int v = base + lane;
+        const bool valid = v < nkeys;
+        float sc = -INFINITY;
+        if (valid) sc = Io<T>::template dot<D>(qs, map.kptr(v)) * scale;
+        const float m_new = fmaxf(m, warp_max(sc));
+        const float p = valid ? expf(sc - m_new) : 0.f;
+        const float alpha = expf(m - m_new);   // first block: exp(-inf) = 0
+        l = l * alpha + warp_sum(p);
+#pragma unroll
+        for (int d = 0; d < DPL; ++d) o[d] *= alpha;
+        const int cnt = min(32, nkeys - base);
+        for (int jj = 0; jj < cnt; ++jj) {
+            const float pj = __shfl_sync(0xffffffffu, p, jj);
+            float vv[DPL];
+            Io<T>::template load<DPL>(map.vptr(base + jj) + lane * DPL, vv);
+#pragma unroll
+            for (int d = 0; d < DPL; ++d) o[d] = fmaf(pj, vv[d], o[d]);
+        }
+        m = m_new;
+    }
+    const float inv = 1.f / l;
+#pragma unroll
+    for (int d = 0; d < DPL; ++d) o[d] *= inv;
+    Io<T>::template store<DPL>(o_out + lane * DPL, o);
+    if (lse_out && lane == 0) *lse_out = m + logf(l);
+}
+
+template <typename T, int D>
+__device__ __forceinline__ void stage_query(float* qs, const T* qrow, int lane) {
+    constexpr int DPL = D / 32;
+    float x[DPL];
+    Io<T>::template load<DPL>(qrow + lane * DPL, x);
+#pragma unroll
+    for (int d = 0; d < DPL; ++d) qs[lane * DPL + d] = x[d];
+    __syncwarp();
+}
+
+// ------------------------------------------------------- masked forward map
+template <typename T>
+struct TrainMap {
+    const T* k;
+    const T* v;
+    int64_t ss;       // row stride (elements)
+    int s, tc, t;
+    int kind;         // 0: memory zones of chunks < y then rows [lo, ...)   1: rows [lo, lo+n_range) then row `self`
+    int n_prior;      // visible memory keys of earlier chunks (kind 0)
+    int lo;           // first row of the contiguous range
+    int n_range;      // length of the contiguous range (kind 1)
+    int self;         // row index of the trailing self key (kind 1)
+    __device__ __forceinline__ int64_t row(int vi) const {
+        if (kind == 0) {
+            if (vi < n_prior) {
+                const int x = vi / t;
+                return (int64_t)x * s + tc + (vi - x * t);
+            }
+            return lo + (vi - n_prior);
+        }
+        return vi < n_range ? lo + vi : self;
+    }
+    __device__ __forceinline__ const T* kptr(int vi) const { return k + row(vi) * ss; }
+    __device__ __forceinline__ const T* vptr(int vi) const { return v + row(vi) * ss; }
+};
+
+constexpr int GENERIC_WARPS = 8;
+
+template <typename T, int D>
+__global__ void __launch_bounds__(GENERIC_WARPS * 32)
+masked_attn_generic_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                           T* __restrict__ o, float* __restrict__ lse, int H, Layout L, int64_t sb,
+                           int64_t sh, int64_t ss, float scale) {
+    __shared__ __align__(16) float q_sh[GENERIC_WARPS][D];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int i = blockIdx.x * GENERIC_WARPS + warp;
+    if (i >= L.S) return;
+    const int bh = blockIdx.y;
+    const int b = bh / H, h = bh - b * H;
+    const int64_t base = (int64_t)b * sb + (int64_t)h * sh;
+
+    // (chunk, zone, offset) of the row, as in Section 4.1
+    int y, zone, off;
+    if (L.s == 0 || i >= L.n_chunks * L.s) {
+        y = L.n_chunks; zone = LOMA_ZONE_READ; off = i - L.n_chunks * L.s;
+    } else {
+        y = i / L.s;
+        const int r = i - y * L.s;
+        if (r < L.tc) { zone = LOMA_ZONE_READ; off = r; }
+        else if (r < L.tc + L.t) { zone = LOMA_ZONE_MEM; off = r - L.tc; }
+        else { zone = LOMA_ZONE_REP; off = r - L.tc - L.t; }
+    }
+
+    TrainMap<T> map;
+    map.k = k + base; map.v = v + base; map.ss = ss; map.s = L.s; map.tc = L.tc; map.t = L.t;
+    map.n_range = 0; map.self = 0;
+    int nkeys;
+    if (zone == LOMA_ZONE_READ) {                 // Eq. 3 reading rows + L of Eq. 1
+        map.kind = 0; map.n_prior = y * L.t; map.lo = y * L.s;
+        nkeys = map.n_prior + off + 1;
+    } else if (zone == LOMA_ZONE_MEM) {           // Eq. 1 second block row
+        map.kind = 0; map.lo = y * L.s;
+        map.n_prior = (L.flags & LOMA_FLAG_MEM_SEES_PRIOR_MEM) ? y * L.t : 0;
+        nkeys = map.n_prior + L.tc + L.t;
+    } else {                                      // Eq. 1 third block row
+        map.kind = 1; map.n_prior = 0; map.lo = y * L.s + L.tc; map.n_range = L.t; map.self = i;
+        nkeys = L.t + 1;
+    }
+    stage_query<T, D>(q_sh[warp], q + base + (int64_t)i * ss, lane);
+    attend_row<T, D>(q_sh[warp], map, nkeys, scale, o + base + (int64_t)i * ss,
+                     lse ? lse + (int64_t)bh * L.S + i : nullptr, lane);
+}
+
+// --------------------------------------------------------------- decode map
+template <typename T>
+struct DecodeMap {
+    const T* kc;
+    const T* vc;
+    const T* kn;
+    const T* vn;
+    int len, D;
+    __device__ __forceinline__ const T* kptr(int vi) const { return vi < len ? kc + (int64_t)vi * D : kn; }
+    __device__ __forceinline__ const T* vptr(int vi) const { return vi < len ? vc + (int64_t)vi * D : vn; }
+};
+
+template <typename T, int D>
+__global__ void __launch_bounds__(32)
+decode_generic_kernel(const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
+                      T* __restrict__ k_cache, T* __restrict__ v_cache, T* __restrict__ o,
+                      float* __restrict__ lse, int cap, int cache_len, float scale) {
+    __shared__ __align__(16) float q_sh[D];
+    const int bh = blockIdx.x, lane = threadIdx.x;
+    T* kc = k_cache + (int64_t)bh * cap * D;
+    T* vc = v_cache + (int64_t)bh * cap * D;
+    DecodeMap<T> map;
+    map.kc = kc; map.vc = vc; map.len = cache_len; map.D = D;
+    map.kn = k_new ? k_new + (int64_t)bh * D : kc + (int64_t)cache_len * D;
+    map.vn = v_new ? v_new + (int64_t)bh * D : vc + (int64_t)cache_len * D;
+    stage_query<T, D>(q_sh, q + (int64_t)bh * D, lane);
+    attend_row<T, D>(q_sh, map, cache_len + 1, scale, o + (int64_t)bh * D, lse ? lse + bh : nullptr, lane);
+    if (k_new) {      // append: the slot is read by nobody in this launch
+        constexpr int DPL = D / 32;
+#pragma unroll
+        for (int d = 0; d < DPL; ++d) {
+            kc[(int64_t)cache_len * D + lane * DPL + d] = k_new[(int64_t)bh * D + lane * DPL + d];
+            vc[(int64_t)cache_len * D + lane * DPL + d] = v_new[(int64_t)bh * D + lane * DPL + d];
+        }
+    }
+}
+
+// ------------------------------------------------------------- compress map
+template <typename T>
+struct CompressMap {
+    const T* kc;   // cache row `lo`
+    const T* vc;
+    const T* km;   // this (b,h)'s t memory keys
+    const T* vm;
+    int n_cache, D;
+    __device__ __forceinline__ const T* kptr(int vi) const {
+        return vi < n_cache ? kc + (int64_t)vi * D : km + (int64_t)(vi - n_cache) * D;
+    }
+    __device__ __forceinline__ const T* vptr(int vi) const {
+        return vi < n_cache ? vc + (int64_t)vi * D : vm + (int64_t)(vi - n_cache) * D;
+    }
+};
+
+// One CTA per (b,h): its warps take the t memory rows in turn; after a block
+// barrier (every read of the tail by this (b,h) is done, and no other CTA reads
+// it) the t memory K/V rows are copied over slots [mem_len, mem_len+t).
+template <typename T, int D>
+__global__ void __launch_bounds__(GENERIC_WARPS * 32)
+compress_generic_kernel(const T* __restrict__ q_mem, const T* __restrict__ k_mem,
+                        const T* __restrict__ v_mem, T* __restrict__ k_cache, T* __restrict__ v_cache,
+                        T* __restrict__ o_mem, float* __restrict__ lse, int cap, int mem_len, int t, int tc,
+                        unsigned flags, float scale) {
+    __shared__ __align__(16) float q_sh[GENERIC_WARPS][D];
+    const int bh = blockIdx.x;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    T* kc = k_cache + (int64_t)bh * cap * D;
+    T* vc = v_cache + (int64_t)bh * cap * D;
+    const int lo = (flags & LOMA_FLAG_MEM_SEES_PRIOR_MEM) ? 0 : mem_len;
+    CompressMap<T> map;
+    map.kc = kc + (int64_t)lo * D; map.vc = vc + (int64_t)lo * D;
+    map.km = k_mem + (int64_t)bh * t * D; map.vm = v_mem + (int64_t)bh * t * D;
+    map.n_cache = mem_len + tc - lo; map.D = D;
+    for (int j = warp; j < t; j += GENERIC_WARPS) {
+        stage_query<T, D>(q_sh[warp], q_mem + ((int64_t)bh * t + j) * D, lane);
+        attend_row<T, D>(q_sh[warp], map, map.n_cache + t, scale, o_mem + ((int64_t)bh * t + j) * D,
+                         lse ? lse + (int64_t)bh * t + j : nullptr, lane);
+        __syncwarp();
+    }
+    __syncthreads();
+    // compaction: 16-byte vector copies, bit for bit
+    constexpr int VEC = 16 / sizeof(T);
+    const int nvec = t * D / VEC;
+    const uint4* ksrc = reinterpret_cast<const uint4*>(map.km);
+    const uint4* vsrc = reinterpret_cast<const uint4*>(map.vm);
+    uint4* kdst = reinterpret_cast<uint4*>(kc + (int64_t)mem_len * D);
+    uint4* vdst = reinterpret_cast<uint4*>(vc + (int64_t)mem_len * D);
+    for (int e = threadIdx.x; e < nvec; e += blockDim.x) {
+        kdst[e] = ksrc[e];
+        vdst[e] = vsrc[e];
+    }
+}
+
+// ------------------------------------------------------------------ launchers
+template <typename T, int D>
+static cudaError_t masked_generic_t(const void* q, const void* k, const void* v, void* o, float* lse, int B,
+                                    int H, const Layout& L, int64_t sb, int64_t sh, int64_t ss, float scale,
+                                    cudaStream_t st) {
+    dim3 grid((L.S + GENERIC_WARPS - 1) / GENERIC_WARPS, B * H);
+    masked_attn_generic_kernel<T, D><<<grid, GENERIC_WARPS * 32, 0, st>>>(
+        static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), static_cast<T*>(o), lse,
+        H, L, sb, sh, ss, scale);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_masked_attn_generic(const void* q, const void* k, const void* v, void* o, float* lse,
+                                       int B, int H, int D, const Layout& L, int64_t sb, int64_t sh,
+                                       int64_t ss, loma_dtype dt, float scale, cudaStream_t st) {
+    if (dt == LOMA_F32) {
+        return D == 64 ? masked_generic_t<float, 64>(q, k, v, o, lse, B, H, L, sb, sh, ss, scale, st)
+                       : masked_generic_t<float, 128>(q, k, v, o, lse, B, H, L, sb, sh, ss, scale, st);
+    }
+    return D == 64 ? masked_generic_t<__nv_bfloat16, 64>(q, k, v, o, lse, B, H, L, sb, sh, ss, scale, st)
+                   : masked_generic_t<__nv_bfloat16, 128>(q, k, v, o, lse, B, H, L, sb, sh, ss, scale, st);
+}
+
+template <typename T, int D>
+static cudaError_t decode_generic_t(const void* q, const void* kn, const void* vn, void* kc, void* vc,
+                                    void* o, float* lse, int BH, int cap, int cache_len, float scale,
+                                    cudaStream_t st) {
+    decode_generic_kernel<T, D><<<BH, 32, 0, st>>>(static_cast<const T*>(q), static_cast<const T*>(kn),
+                                                   static_cast<const T*>(vn), static_cast<T*>(kc),
+                                                   static_cast<T*>(vc), static_cast<T*>(o), lse, cap,
+                                                   cache_len, scale);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode_generic(const void* q, const void* k_new, const void* v_new, void* k_cache,
+                                  void* v_cache, void* o, float* lse, int B, int H, int D, int cap,
+                                  int cache_len, loma_dtype dt, float scale, cudaStream_t st) {
+    const int BH = B * H;
+    if (dt == LOMA_F32) {
+        return D == 64 ? decode_generic_t<float, 64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
+                                                     cache_len, scale, st)
+                       : decode_generic_t<float, 128>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
+                                                      cache_len, scale, st);
+    }
+    return D == 64 ? decode_generic_t<__nv_bfloat16, 64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
+                                                         cache_len, scale, st)
+                   : decode_generic_t<__nv_bfloat16, 128>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
+                                                          cache_len, scale, st);
+}
+
+template <typename T, int D>
+static cudaError_t compress_generic_t(const void* qm, const void* km, const void* vm, void* kc, void* vc,
+                                      void* om, float* lse, int BH, int cap, int mem_len, int t, int tc,
+                                      unsigned flags, float scale, cudaStream_t st) {
+    compress_generic_kernel<T, D><<<BH, GENERIC_WARPS * 32, 0, st>>>(
+        static_cast<const T*>(qm), static_cast<const T*>(km), static_cast<const T*>(vm), static_cast<T*>(kc),
+        static_cast<T*>(vc), static_cast<T*>(om), lse, cap, mem_len, t, tc, flags, scale);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache,
+                                    void* v_cache, void* o_mem, float* lse, int B, int H, int D, int cap,
+                                    int mem_len, int c, int t, loma_dtype dt, float scale, unsigned flags,
+                                    cudaStream_t st) {
+    const int BH = B * H, tc = c * t;
+    if (dt == LOMA_F32) {
+        return D == 64 ? compress_generic_t<float, 64>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH,
+                                                       cap, mem_len, t, tc, flags, scale, st)
+                       : compress_generic_t<float, 128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH,
+                                                        cap, mem_len, t, tc, flags, scale, st);
+    }
+    return D == 64 ? compress_generic_t<__nv_bfloat16, 64>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse,
+                                                           BH, cap, mem_len, t, tc, flags, scale, st)
+                   : compress_generic_t<__nv_bfloat16, 128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse,
+                                                            BH, cap, mem_len, t, tc, flags, scale, st);
+}
+
+}  // namespace loma

@@ -1,0 +1,129 @@
+// Integer index maps of the LoMA layout (Section 4.1, Eq. 14) and of the
+// generation-time cache (Section 3.1, Appendix A).  Pure integer work; the host
+// and device versions use the same inline row functions.
+#include "loma_internal.cuh"
+
+namespace loma {
+
+struct RowInfo {
+    int chunk, zone, offset, src, pos;
+};
+
+// Row i of the laid-out sequence -> its chunk, zone, offset, source token and
+// position id.  Rows beyond the last complete chunk are reading rows of chunk
+// n_chunks.  Memory position ids follow Eq. 14 with the chunk start at y*tc.
+__host__ __device__ inline RowInfo layout_row(int i, int n_chunks, int c, int t) {
+    const int tc = c * t;
+    const int s = 2 * tc + t;
+    RowInfo r;
+    if (s == 0 || i >= n_chunks * s) {
+        r.chunk = n_chunks;
+        r.zone = LOMA_ZONE_READ;
+        r.offset = i - n_chunks * s;
+    } else {
+        r.chunk = i / s;
+        const int rem = i - r.chunk * s;
+        if (rem < tc) {
+            r.zone = LOMA_ZONE_READ;
+            r.offset = rem;
+        } else if (rem < tc + t) {
+            r.zone = LOMA_ZONE_MEM;
+            r.offset = rem - tc;
+        } else {
+            r.zone = LOMA_ZONE_REP;
+            r.offset = rem - tc - t;
+        }
+    }
+    if (r.zone == LOMA_ZONE_MEM) {
+        r.src = -1;
+        r.pos = r.chunk * tc + (r.offset + 1) * c - 1;
+    } else {
+        r.src = r.chunk * tc + r.offset;
+        r.pos = r.src;
+    }
+    return r;
+}
+
+struct GenInfo {
+    int slot, pos, comp;
+};
+
+// Generated token g -> cache slot it is appended at, its position id, and
+// whether the tail is full (tc entries) once it has been appended.
+__host__ __device__ inline GenInfo generation_row(int g, int c, int t) {
+    GenInfo r;
+    r.pos = g;
+    if (t == 0) {
+        r.slot = g;
+        r.comp = 0;
+    } else {
+        const int tc = c * t;
+        const int y = g / tc;
+        const int o = g - y * tc;
+        r.slot = y * t + o;
+        r.comp = (o == tc - 1) ? 1 : 0;
+    }
+    return r;
+}
+
+__global__ void layout_index_kernel(int S, int n_chunks, int c, int t, int32_t* chunk, int32_t* zone,
+                                    int32_t* offset, int32_t* src, int32_t* pos) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= S) return;
+    const RowInfo r = layout_row(i, n_chunks, c, t);
+    if (chunk) chunk[i] = r.chunk;
+    if (zone) zone[i] = r.zone;
+    if (offset) offset[i] = r.offset;
+    if (src) src[i] = r.src;
+    if (pos) pos[i] = r.pos;
+}
+
+__global__ void generation_index_kernel(int n, int c, int t, int32_t* slot, int32_t* pos, int32_t* comp) {
+    const int g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= n) return;
+    const GenInfo r = generation_row(g, c, t);
+    if (slot) slot[g] = r.slot;
+    if (pos) pos[g] = r.pos;
+    if (comp) comp[g] = r.comp;
+}
+
+cudaError_t launch_layout_index(const Layout& L, int32_t* chunk, int32_t* zone, int32_t* offset,
+                                int32_t* src, int32_t* pos, cudaStream_t st) {
+    if (L.S == 0) return cudaSuccess;
+    const int threads = 256;
+    layout_index_kernel<<<(L.S + threads - 1) / threads, threads, 0, st>>>(L.S, L.n_chunks, L.c, L.t, chunk,
+                                                                         zone, offset, src, pos);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_generation_index(int n_tokens, int c, int t, int32_t* slot, int32_t* pos,
+                                    int32_t* comp, cudaStream_t st) {
+    if (n_tokens == 0) return cudaSuccess;
+    const int threads = 256;
+    generation_index_kernel<<<(n_tokens + threads - 1) / threads, threads, 0, st>>>(n_tokens, c, t, slot, pos,
+                                                                                  comp);
+    return cudaGetLastError();
+}
+
+void host_layout_index(const Layout& L, int32_t* chunk, int32_t* zone, int32_t* offset, int32_t* src,
+                       int32_t* pos) {
+    for (int i = 0; i < L.S; ++i) {
+        const RowInfo r = layout_row(i, L.n_chunks, L.c, L.t);
+        if (chunk) chunk[i] = r.chunk;
+        if (zone) zone[i] = r.zone;
+        if (offset) offset[i] = r.offset;
+        if (src) src[i] = r.src;
+        if (pos) pos[i] = r.pos;
+    }
+}
+
+void host_generation_index(int n_tokens, int c, int t, int32_t* slot, int32_t* pos, int32_t* comp) {
+    for (int g = 0; g < n_tokens; ++g) {
+        const GenInfo r = generation_row(g, c, t);
+        if (slot) slot[g] = r.slot;
+        if (pos) pos[g] = r.pos;
+        if (comp) comp[g] = r.comp;
+    }
+}
+
+}  // namespace loma

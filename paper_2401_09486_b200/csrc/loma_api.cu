@@ -1,0 +1,215 @@
+// extern "C" boundary of libloma: argument validation and kernel selection.
+// Every check happens on the host before anything is enqueued.
+#include <limits.h>
+#include <math.h>
+
+#include "loma_internal.cuh"
+
+namespace loma {
+
+__device__ int g_status_word = 0;
+
+int* device_status_word() {
+    // one address per device; looked up on first use with that device current
+    static int* addr[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+        addr[dev] = static_cast<int*>(p);
+    }
+    return addr[dev];
+}
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline size_t elt_size(loma_dtype dt) { return dt == LOMA_F32 ? 4 : 2; }
+
+// B200 check, cached per device.  Returns LOMA_OK / LOMA_ERR_UNSUPPORTED / LOMA_ERR_CUDA.
+static int check_device() {
+    static int cached[64];
+    static bool have[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return LOMA_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return LOMA_ERR_UNSUPPORTED;
+    if (!have[dev]) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+            return LOMA_ERR_CUDA;
+        cached[dev] = (major == 10) ? LOMA_OK : LOMA_ERR_UNSUPPORTED;
+        have[dev] = true;
+    }
+    return cached[dev];
+}
+
+static int make_layout(int n_chunks, int c, int t, int tail_read, unsigned flags, Layout* L) {
+    if (n_chunks < 0 || c < 1 || t < 0 || tail_read < 0) return LOMA_ERR_INVALID_ARG;
+    if (t == 0 && n_chunks != 0) return LOMA_ERR_INVALID_ARG;
+    const int64_t tc = (int64_t)c * t;
+    if (t > 0 && tail_read > tc) return LOMA_ERR_INVALID_ARG;
+    const int64_t s = 2 * tc + t;
+    const int64_t S = (int64_t)n_chunks * s + tail_read;
+    if (tc > INT_MAX / 4 || S > INT_MAX) return LOMA_ERR_INVALID_ARG;
+    L->n_chunks = n_chunks; L->c = c; L->t = t; L->tc = (int)tc; L->s = (int)s;
+    L->tail_read = tail_read; L->S = (int)S; L->flags = flags;
+    return LOMA_OK;
+}
+
+}  // namespace loma
+
+using namespace loma;
+
+extern "C" {
+
+int loma_version(void) { return 100; }
+
+const char* loma_status_string(int status) {
+    switch (status) {
+        case LOMA_OK: return "LOMA_OK";
+        case LOMA_ERR_INVALID_ARG: return "LOMA_ERR_INVALID_ARG: invalid argument";
+        case LOMA_ERR_UNSUPPORTED: return "LOMA_ERR_UNSUPPORTED: unsupported head dimension, dtype or device";
+        case LOMA_ERR_ALIGNMENT: return "LOMA_ERR_ALIGNMENT: pointer or stride not 16-byte aligned";
+        case LOMA_ERR_CAPACITY: return "LOMA_ERR_CAPACITY: cache capacity too small";
+        case LOMA_ERR_WORKSPACE: return "LOMA_ERR_WORKSPACE: workspace missing or too small";
+        case LOMA_ERR_CUDA: return "LOMA_ERR_CUDA: a CUDA call failed";
+        case LOMA_ERR_TIMEOUT: return "LOMA_ERR_TIMEOUT: a bounded device-side wait expired";
+        default: return "unknown loma status";
+    }
+}
+
+int loma_layout_index(int n_chunks, int c, int t, int tail_read, int32_t* chunk, int32_t* zone,
+                      int32_t* offset, int32_t* src_token, int32_t* pos_id, int on_device, void* stream) {
+    Layout L;
+    const int rc = make_layout(n_chunks, c, t, tail_read, 0, &L);
+    if (rc != LOMA_OK) return rc;
+    if (!on_device) {
+        host_layout_index(L, chunk, zone, offset, src_token, pos_id);
+        return LOMA_OK;
+    }
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    return launch_layout_index(L, chunk, zone, offset, src_token, pos_id, static_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess
+               ? LOMA_OK
+               : LOMA_ERR_CUDA;
+}
+
+int loma_generation_index(int n_tokens, int c, int t, int32_t* slot, int32_t* pos_id, int32_t* compress_after,
+                          int on_device, void* stream) {
+    if (n_tokens < 0 || c < 1 || t < 0) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)c * t > INT_MAX / 4) return LOMA_ERR_INVALID_ARG;
+    if (!on_device) {
+        host_generation_index(n_tokens, c, t, slot, pos_id, compress_after);
+        return LOMA_OK;
+    }
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    return launch_generation_index(n_tokens, c, t, slot, pos_id, compress_after,
+                                   static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? LOMA_OK
+               : LOMA_ERR_CUDA;
+}
+
+int loma_masked_attn_fwd(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int D,
+                         int n_chunks, int c, int t, int tc, int tail_read, int64_t stride_b, int64_t stride_h,
+                         int64_t stride_s, loma_dtype dtype, float softmax_scale, unsigned flags,
+                         void* stream) {
+    if (B < 0 || H < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    Layout L;
+    const int rc = make_layout(n_chunks, c, t, tail_read, flags, &L);
+    if (rc != LOMA_OK) return rc;
+    if (tc != L.tc) return LOMA_ERR_INVALID_ARG;
+    if (L.S == 0 || B == 0 || H == 0) return LOMA_OK;
+    if (!q || !k || !v || !o) return LOMA_ERR_INVALID_ARG;
+    if (o == q || o == k || o == v) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
+    if (stride_s < D || stride_b < 0 || stride_h < 0) return LOMA_ERR_INVALID_ARG;
+    const size_t es = elt_size(dtype);
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return LOMA_ERR_ALIGNMENT;
+    if ((stride_b * es) % 16 || (stride_h * es) % 16 || (stride_s * es) % 16) return LOMA_ERR_ALIGNMENT;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_masked_attn_generic(q, k, v, o, lse, B, H, D, L, stride_b, stride_h, stride_s, dtype,
+                                               scale, st);
+    return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
+size_t loma_decode_workspace_bytes(int B, int H, int D, int cache_len) {
+    (void)B; (void)H; (void)D; (void)cache_len;
+    return 0;
+}
+
+int loma_decode_attn(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
+                     float* lse, int B, int H, int D, int cap, int cache_len, loma_dtype dtype,
+                     float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes,
+                     void* stream) {
+    (void)flags;
+    if (B < 0 || H < 0 || cap < 0 || cache_len < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    if ((k_new == nullptr) != (v_new == nullptr)) return LOMA_ERR_INVALID_ARG;
+    if (cache_len >= cap) return LOMA_ERR_CAPACITY;
+    if (B == 0 || H == 0) return LOMA_OK;
+    if (!q || !k_cache || !v_cache || !o) return LOMA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) || !aligned16(k_new) ||
+        !aligned16(v_new) || !aligned16(workspace))
+        return LOMA_ERR_ALIGNMENT;
+    const size_t need = loma_decode_workspace_bytes(B, H, D, cache_len);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return LOMA_ERR_WORKSPACE;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_decode_generic(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len,
+                                          dtype, scale, st);
+    return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
+size_t loma_compress_workspace_bytes(int B, int H, int D, int t, int mem_len, unsigned flags) {
+    (void)B; (void)H; (void)D; (void)t; (void)mem_len; (void)flags;
+    return 0;
+}
+
+int loma_compress_step(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
+                       void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len, int c, int t, int tc,
+                       loma_dtype dtype, float softmax_scale, unsigned flags, void* workspace,
+                       size_t workspace_bytes, void* stream) {
+    if (B < 0 || H < 0 || cap < 0 || mem_len < 0 || c < 1 || t < 1) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)c * t != (int64_t)tc) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    if ((int64_t)mem_len + tc > (int64_t)cap) return LOMA_ERR_CAPACITY;
+    if (B == 0 || H == 0) return LOMA_OK;
+    if (!q_mem || !k_mem || !v_mem || !k_cache || !v_cache || !o_mem) return LOMA_ERR_INVALID_ARG;
+    if (!aligned16(q_mem) || !aligned16(k_mem) || !aligned16(v_mem) || !aligned16(k_cache) ||
+        !aligned16(v_cache) || !aligned16(o_mem) || !aligned16(workspace))
+        return LOMA_ERR_ALIGNMENT;
+    const size_t need = loma_compress_workspace_bytes(B, H, D, t, mem_len, flags);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return LOMA_ERR_WORKSPACE;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_compress_generic(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap,
+                                            mem_len, c, t, dtype, scale, flags, st);
+    return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
+int loma_device_status(void* stream) {
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return LOMA_ERR_CUDA;
+    int* w = device_status_word();
+    if (!w) return LOMA_ERR_CUDA;
+    int val = 0;
+    if (cudaMemcpy(&val, w, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return LOMA_ERR_CUDA;
+    if (val != 0) {
+        const int zero = 0;
+        if (cudaMemcpy(w, &zero, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return LOMA_ERR_CUDA;
+    }
+    return val;
+}
+
+}  // extern "C"

@@ -1,0 +1,70 @@
+// Internal declarations shared by the translation units of libloma.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "loma.h"
+
+namespace loma {
+
+// ---- layout parameters handed to kernels ---------------------------------
+struct Layout {
+    int n_chunks;   // complete chunks
+    int c, t, tc;   // tc = c*t
+    int s;          // chunk length 2*tc + t (0 when t == 0)
+    int tail_read;  // trailing reading rows
+    int S;          // n_chunks*s + tail_read
+    unsigned flags;
+};
+
+// ---- launchers (each defined in its own .cu) ------------------------------
+cudaError_t launch_layout_index(const Layout& L, int32_t* chunk, int32_t* zone, int32_t* offset,
+                                int32_t* src, int32_t* pos, cudaStream_t st);
+cudaError_t launch_generation_index(int n_tokens, int c, int t, int32_t* slot, int32_t* pos,
+                                    int32_t* comp, cudaStream_t st);
+void host_layout_index(const Layout& L, int32_t* chunk, int32_t* zone, int32_t* offset, int32_t* src,
+                       int32_t* pos);
+void host_generation_index(int n_tokens, int c, int t, int32_t* slot, int32_t* pos, int32_t* comp);
+
+cudaError_t launch_masked_attn_generic(const void* q, const void* k, const void* v, void* o, float* lse,
+                                       int B, int H, int D, const Layout& L,
+                                       int64_t sb, int64_t sh, int64_t ss,
+                                       loma_dtype dt, float scale, cudaStream_t st);
+
+cudaError_t launch_decode_generic(const void* q, const void* k_new, const void* v_new,
+                                  void* k_cache, void* v_cache, void* o, float* lse,
+                                  int B, int H, int D, int cap, int cache_len,
+                                  loma_dtype dt, float scale, cudaStream_t st);
+
+cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const void* v_mem,
+                                    void* k_cache, void* v_cache, void* o_mem, float* lse,
+                                    int B, int H, int D, int cap, int mem_len, int c, int t,
+                                    loma_dtype dt, float scale, unsigned flags, cudaStream_t st);
+
+// ---- device status word (bounded waits report here) ------------------------
+int* device_status_word();   // device address of the status word of the current device (NULL on failure)
+
+// ---- small device helpers ---------------------------------------------------
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+    return x;
+}
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+// two packed bf16 -> two floats (exact)
+__device__ __forceinline__ float bf16lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 p = __floats2bfloat162_rn(lo, hi);   // .x = lo (low half), .y = hi
+    return *reinterpret_cast<uint32_t*>(&p);
+}
+
+}  // namespace loma

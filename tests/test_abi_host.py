@@ -1,0 +1,133 @@
+"""Host-side checks of the C-ABI library that need no GPU: it builds and loads,
+exports everything include/loma.h declares, rejects bad arguments before any
+CUDA call, and its host index maps agree bit for bit with the oracle."""
+
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2401_09486_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+INVALID, UNSUPPORTED, ALIGNMENT, CAPACITY, WORKSPACE = -1, -2, -3, -4, -5
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return binding.lib()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "loma.h")).read()
+    return sorted(set(re.findall(r"LOMA_API\s+[\w\s\*]+?\b(loma_\w+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = _declared_symbols()
+    assert len(names) >= 10
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in loma.h but not exported"
+        assert n in binding.SIGNATURES, f"{n} has no binding signature"
+    assert sorted(binding.SIGNATURES) == names
+    assert lib.loma_version() >= 100
+    assert b"LOMA_OK" in lib.loma_status_string(0)
+    for code in range(-7, 0):
+        assert b"LOMA_ERR" in lib.loma_status_string(code)
+
+
+@pytest.mark.parametrize("n,c,t,tail", [(0, 4, 0, 9), (1, 1, 1, 0), (3, 2, 2, 0), (2, 4, 4, 3), (32, 4, 16, 0),
+                                        (5, 3, 7, 21), (128, 8, 32, 0), (0, 2, 3, 0)])
+def test_host_layout_index_bit_exact(lib, n, c, t, tail):
+    got = binding.loma_layout_index(n, c, t, tail, device="cpu")
+    want = oracle.layout_index(n, c, t, tail)
+    for g, w in zip(got, want):
+        assert g.dtype == torch.int32
+        assert np.array_equal(g.numpy(), w)
+
+
+@pytest.mark.parametrize("n_tok,c,t", [(0, 4, 4), (1, 4, 4), (100, 4, 4), (257, 8, 16), (50, 3, 0), (64, 1, 5)])
+def test_host_generation_index_bit_exact(lib, n_tok, c, t):
+    got = binding.loma_generation_index(n_tok, c, t, device="cpu")
+    want = oracle.generation_index(n_tok, c, t)
+    for g, w in zip(got, want):
+        assert np.array_equal(g.numpy(), w)
+
+
+def test_layout_index_null_outputs_are_skipped(lib):
+    S = oracle.seq_len(2, 2, 2)
+    pos = (ctypes.c_int32 * S)()
+    assert lib.loma_layout_index(2, 2, 2, 0, None, None, None, None, pos, 0, None) == 0
+    assert list(pos) == oracle.layout_index(2, 2, 2)[4].tolist()
+
+
+def test_layout_index_rejects_bad_geometry(lib):
+    buf = (ctypes.c_int32 * 64)()
+    bad = [(-1, 2, 2, 0), (1, 0, 2, 0), (1, 2, -1, 0), (1, 2, 0, 0), (1, 2, 2, 5), (1, 2, 2, -1),
+           (1 << 20, 64, 64, 0)]
+    for n, c, t, tail in bad:
+        assert lib.loma_layout_index(n, c, t, tail, buf, None, None, None, None, 0, None) == INVALID
+
+
+def _fwd(lib, q=0x1000, k=0x2000, v=0x3000, o=0x4000, lse=None, B=1, H=1, D=64, n=1, c=2, t=2, tc=4, tail=0,
+         sb=640, sh=640, ss=64, dt=1, scale=0.0, flags=0):
+    return lib.loma_masked_attn_fwd(q, k, v, o, lse, B, H, D, n, c, t, tc, tail, sb, sh, ss, dt, scale, flags,
+                                    None)
+
+
+def test_masked_attn_fwd_validation_precedes_any_cuda_call(lib):
+    # pointers are never dereferenced: every call below must fail on the host
+    assert _fwd(lib, tc=5) == INVALID                   # tc != c*t
+    assert _fwd(lib, D=96) == UNSUPPORTED
+    assert _fwd(lib, dt=7) == UNSUPPORTED
+    assert _fwd(lib, B=-1) == INVALID
+    assert _fwd(lib, q=None) == INVALID
+    assert _fwd(lib, o=0x1000) == INVALID               # o aliases q
+    assert _fwd(lib, q=0x1008) == ALIGNMENT
+    assert _fwd(lib, ss=68, dt=1) == ALIGNMENT          # 136-byte row stride
+    assert _fwd(lib, ss=32) == INVALID                  # rows overlap
+    assert _fwd(lib, t=0, tc=0, n=1) == INVALID         # t == 0 needs n_chunks == 0
+    assert _fwd(lib, tail=5) == INVALID                 # tail longer than a reading zone
+    assert _fwd(lib, n=0, t=2, tc=4, tail=0) == 0       # empty sequence: no-op
+    assert _fwd(lib, B=0) == 0
+
+
+def test_decode_validation(lib):
+    def call(q=0x1000, kn=0x2000, vn=0x3000, kc=0x4000, vc=0x5000, o=0x6000, B=1, H=1, D=128, cap=8, ln=3, dt=1,
+             ws=None, wsb=0):
+        return lib.loma_decode_attn(q, kn, vn, kc, vc, o, None, B, H, D, cap, ln, dt, 0.0, 0, ws, wsb, None)
+    assert call(ln=8) == CAPACITY
+    assert call(ln=-1) == INVALID
+    assert call(D=100) == UNSUPPORTED
+    assert call(kn=None) == INVALID                     # k_new and v_new must come together
+    assert call(kc=None) == INVALID
+    assert call(o=0x6004) == ALIGNMENT
+    assert call(B=0) == 0
+    # a workspace is required whenever the size query says so
+    need = lib.loma_decode_workspace_bytes(32, 32, 128, 8192)
+    if need:
+        assert lib.loma_decode_attn(0x1000, 0x2000, 0x3000, 0x4000, 0x5000, 0x6000, None, 32, 32, 128, 9000,
+                                    8192, 1, 0.0, 0, None, 0, None) == WORKSPACE
+        assert lib.loma_decode_attn(0x1000, 0x2000, 0x3000, 0x4000, 0x5000, 0x6000, None, 32, 32, 128, 9000,
+                                    8192, 1, 0.0, 0, 0x7000, need - 1, None) == WORKSPACE
+
+
+def test_compress_validation(lib):
+    def call(qm=0x1000, km=0x2000, vm=0x3000, kc=0x4000, vc=0x5000, om=0x6000, B=1, H=1, D=128, cap=100,
+             mem_len=16, c=4, t=16, tc=64, dt=1, flags=0):
+        return lib.loma_compress_step(qm, km, vm, kc, vc, om, None, B, H, D, cap, mem_len, c, t, tc, dt, 0.0,
+                                      flags, None, 0, None)
+    assert call(cap=79) == CAPACITY                     # needs mem_len + tc entries
+    assert call(tc=63) == INVALID
+    assert call(t=0, tc=0) == INVALID
+    assert call(mem_len=-16) == INVALID
+    assert call(D=32) == UNSUPPORTED
+    assert call(vm=None) == INVALID
+    assert call(vc=0x5002) == ALIGNMENT
+    assert call(H=0) == 0
