@@ -1,0 +1,381 @@
+"""Parity of the CUDA library (through the C ABI) with the CPU oracle, element by
+element on the same seeded inputs.
+
+Tolerances: integer maps and cache contents are bit-exact.  fp32 attention
+outputs: max |delta| <= 1e-5.  bf16 (fp32 accumulation) on N(0,1) inputs:
+max |delta| <= 2e-2 and mean |delta| <= 2e-3.
+"""
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2401_09486_b200 import binding as L
+from paper_2401_09486_b200 import build, synthetic
+
+pytestmark = pytest.mark.gpu
+
+PRIOR = L.LOMA_FLAG_MEM_SEES_PRIOR_MEM
+GENERIC = L.LOMA_FLAG_FORCE_GENERIC
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _library():
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    build.build_library()
+    L.lib()
+    torch.cuda.set_device(0)
+    yield
+    assert L.loma_device_status() == 0
+
+
+def npf(x: torch.Tensor) -> np.ndarray:
+    return x.detach().to("cpu").to(torch.float64).numpy()
+
+
+def bits(x: torch.Tensor) -> np.ndarray:
+    return x.detach().cpu().contiguous().view(torch.int16 if x.dtype == torch.bfloat16 else torch.int32).numpy()
+
+
+def check_close(got: torch.Tensor, want: np.ndarray, dtype):
+    g = npf(got)
+    assert g.shape == want.shape
+    assert np.isfinite(g).all()
+    d = np.abs(g - want)
+    if dtype == torch.float32:
+        assert d.max() <= 1e-5, f"fp32 max |delta| {d.max():.3e}"
+    else:
+        assert d.max() <= 2e-2, f"bf16 max |delta| {d.max():.3e}"
+        assert d.mean() <= 2e-3, f"bf16 mean |delta| {d.mean():.3e}"
+
+
+def run_fwd(q, k, v, n, c, t, tail=0, flags=0, scale=0.0, want_lse=True):
+    o = torch.full_like(q, float("nan"))
+    lse = torch.full(q.shape[:3], float("nan"), dtype=torch.float32, device=q.device) if want_lse else None
+    L.loma_masked_attn_fwd(q, k, v, o, lse, n, c, t, tail, flags, scale)
+    torch.cuda.synchronize()
+    return o, lse
+
+
+def workspace(nbytes):
+    return torch.empty(max(16, nbytes), dtype=torch.uint8, device=DEV)
+
+
+# ----------------------------------------------------------------- index maps
+
+@pytest.mark.parametrize("n,c,t,tail", [(0, 4, 0, 9), (3, 2, 2, 0), (2, 4, 4, 3), (32, 4, 16, 0), (128, 8, 32, 0),
+                                        (5, 3, 7, 21)])
+def test_device_layout_index_bit_exact(n, c, t, tail):
+    got = L.loma_layout_index(n, c, t, tail, device=DEV)
+    torch.cuda.synchronize()
+    for g, w in zip(got, oracle.layout_index(n, c, t, tail)):
+        assert np.array_equal(g.cpu().numpy(), w)
+
+
+@pytest.mark.parametrize("n_tok,c,t", [(1, 4, 4), (1000, 4, 16), (777, 8, 16), (50, 3, 0)])
+def test_device_generation_index_bit_exact(n_tok, c, t):
+    got = L.loma_generation_index(n_tok, c, t, device=DEV)
+    torch.cuda.synchronize()
+    for g, w in zip(got, oracle.generation_index(n_tok, c, t)):
+        assert np.array_equal(g.cpu().numpy(), w)
+
+
+# ------------------------------------------------------- masked forward, small
+
+FWD_CASES = [
+    # B, H, D, n, c, t, tail
+    (1, 1, 64, 2, 4, 4, 0),       # the tiny configuration (72 rows)
+    (2, 3, 64, 3, 2, 2, 3),
+    (1, 2, 128, 2, 4, 16, 0),     # one 64|16|64 chunk pair
+    (2, 2, 128, 5, 4, 16, 37),    # several tiles and a ragged reading tail
+    (1, 2, 128, 3, 8, 16, 0),     # tc = 128
+    (1, 1, 128, 3, 8, 32, 200),   # tc = 256 with a tail
+    (1, 2, 64, 4, 1, 5, 2),       # c = 1, odd t
+    (1, 1, 128, 2, 3, 7, 0),      # nothing is a power of two
+    (1, 2, 128, 0, 4, 0, 301),    # t = 0: plain causal attention
+    (1, 1, 64, 1, 2, 64, 0),      # t = 64
+    (1, 1, 128, 9, 2, 8, 16),     # t = 8
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, PRIOR, GENERIC, GENERIC | PRIOR])
+@pytest.mark.parametrize("B,H,D,n,c,t,tail", FWD_CASES)
+def test_masked_fwd_matches_oracle(B, H, D, n, c, t, tail, flags, dtype):
+    S = oracle.seq_len(n, c, t, tail)
+    q, k, v = synthetic.qkv(B, H, S, D, seed=7, std=1.0, dtype=dtype)
+    want_o, want_lse = oracle.masked_attn_fwd(npf(q), npf(k), npf(v), n, c, t, tail, flags & PRIOR)
+    o, lse = run_fwd(q.to(DEV), k.to(DEV), v.to(DEV), n, c, t, tail, flags)
+    check_close(o, want_o, dtype)
+    lse_tol = 1e-5 if dtype == torch.float32 else 2e-2
+    assert np.abs(npf(lse) - want_lse).max() <= lse_tol
+
+
+def test_masked_fwd_strided_views_and_explicit_scale():
+    """Q/K/V/O given as views into a packed [B, S, 3+1, H, D]-style buffer."""
+    B, H, D, n, c, t = 2, 3, 128, 3, 4, 16
+    S = oracle.seq_len(n, c, t)
+    buf = synthetic.normal_tensor((B, S, 4, H, D), 9, 1.0, torch.bfloat16).to(DEV)
+    q, k, v, o = (buf[:, :, i].permute(0, 2, 1, 3) for i in range(4))      # [B, H, S, D] strided
+    want_o, _ = oracle.masked_attn_fwd(npf(q), npf(k), npf(v), n, c, t, scale=0.05)
+    L.loma_masked_attn_fwd(q, k, v, o, None, n, c, t, 0, 0, 0.05)
+    torch.cuda.synchronize()
+    check_close(o, want_o, torch.bfloat16)
+
+
+def replay_on_gpu(q, k, v, n, c, t, tail, flags):
+    """Drive loma_decode_attn / loma_compress_step over a laid-out sequence the
+    way the generator would (host logic only; all arithmetic in the library)."""
+    B, H, S, D = q.shape
+    tc, s = c * t, oracle.chunk_len(c, t)
+    cap = n * t + max(tc, tail) + 1
+    kc = torch.zeros(B, H, cap, D, dtype=q.dtype, device=q.device)
+    vc = torch.zeros_like(kc)
+    out = torch.full_like(q, float("nan"))
+    ws = workspace(max(L.loma_decode_workspace_bytes(B, H, D, cap),
+                       L.loma_compress_workspace_bytes(B, H, D, max(t, 1), n * t, flags)))
+    length = 0
+
+    def decode(i):
+        nonlocal length
+        o1 = torch.empty(B, H, 1, D, dtype=q.dtype, device=q.device)
+        L.loma_decode_attn(q[:, :, i:i + 1].contiguous(), k[:, :, i:i + 1].contiguous(),
+                           v[:, :, i:i + 1].contiguous(), kc, vc, o1, None, length, ws, flags)
+        out[:, :, i] = o1[:, :, 0]
+        length += 1
+
+    for y in range(n):
+        for o_ in range(tc):
+            decode(y * s + o_)
+        m0 = y * s + tc
+        om = torch.empty(B, H, t, D, dtype=q.dtype, device=q.device)
+        L.loma_compress_step(q[:, :, m0:m0 + t].contiguous(), k[:, :, m0:m0 + t].contiguous(),
+                             v[:, :, m0:m0 + t].contiguous(), kc, vc, om, None, y * t, c, t, ws, flags)
+        out[:, :, m0:m0 + t] = om
+        length = y * t + t
+    for o_ in range(tail):
+        decode(n * s + o_)
+    torch.cuda.synchronize()
+    return out, kc, vc, length
+
+
+def test_tiny_config_fp32_forward_then_incremental_replay():
+    """B1 H1 D64 fp32, c=4, t=4, two chunks [16|4|16] = 72 rows, N(0,1) from
+    seed 0.  Forward, then the same rows replayed as generation with one compress
+    step per chunk; caches compared bit for bit."""
+    B, H, D, n, c, t = 1, 1, 64, 2, 4, 4
+    tc, s = c * t, oracle.chunk_len(c, t)
+    S = n * s
+    q, k, v = synthetic.qkv(B, H, S, D, seed=0, std=1.0, dtype=torch.float32)
+    want_o, _ = oracle.masked_attn_fwd(npf(q), npf(k), npf(v), n, c, t)
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    o, _ = run_fwd(qd, kd, vd, n, c, t)
+    check_close(o, want_o, torch.float32)
+
+    got_o, kc, vc, length = replay_on_gpu(qd, kd, vd, n, c, t, 0, 0)
+    zone = oracle.layout_index(n, c, t)[1]
+    live = zone != oracle.ZONE_REP
+    assert np.abs(npf(got_o)[:, :, live] - want_o[:, :, live]).max() <= 1e-5      # invariant (c)
+    ref_o, ref_k, ref_v, ref_len = oracle.replay_generation(q.numpy(), k.numpy(), v.numpy(), n, c, t)
+    assert length == ref_len == n * t
+    assert np.array_equal(kc[:, :, :length].cpu().numpy(), ref_k[:, :, :length])
+    assert np.array_equal(vc[:, :, :length].cpu().numpy(), ref_v[:, :, :length])
+    slot, _, comp = L.loma_generation_index(n * tc, c, t, device="cpu")
+    assert comp.sum().item() == n
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, PRIOR, GENERIC, GENERIC | PRIOR])
+@pytest.mark.parametrize("B,H,D,n,c,t,tail", [(1, 2, 64, 3, 2, 4, 3), (2, 2, 128, 3, 4, 16, 10),
+                                              (1, 1, 128, 2, 8, 16, 0), (1, 2, 128, 2, 3, 5, 1)])
+def test_incremental_generation_equals_one_shot(B, H, D, n, c, t, tail, flags, dtype):
+    """Invariant (c) on the GPU path, and bit-exact compaction."""
+    S = oracle.seq_len(n, c, t, tail)
+    q, k, v = synthetic.qkv(B, H, S, D, seed=11, std=1.0, dtype=dtype)
+    want_o, _ = oracle.masked_attn_fwd(npf(q), npf(k), npf(v), n, c, t, tail, flags & PRIOR)
+    got_o, kc, vc, length = replay_on_gpu(q.to(DEV), k.to(DEV), v.to(DEV), n, c, t, tail, flags)
+    zone = oracle.layout_index(n, c, t, tail)[1]
+    live = zone != oracle.ZONE_REP
+    check_close(got_o[:, :, torch.from_numpy(live).to(DEV)], want_o[:, :, live], dtype)
+    tc, s = c * t, oracle.chunk_len(c, t)
+    rows = [y * s + tc + j for y in range(n) for j in range(t)] + list(range(n * s, S))
+    assert length == len(rows)
+    assert torch.equal(kc[:, :, :length].cpu(), k[:, :, rows])        # bit for bit
+    assert torch.equal(vc[:, :, :length].cpu(), v[:, :, rows])
+
+
+# ------------------------------------------------------------- decode, compress
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, GENERIC])
+@pytest.mark.parametrize("B,H,D,cap,cache_len", [(1, 1, 64, 4, 0), (2, 3, 128, 40, 1), (2, 2, 128, 700, 613),
+                                                 (1, 4, 128, 3000, 2999), (3, 2, 64, 1100, 1024),
+                                                 (2, 2, 128, 5000, 4133)])
+def test_decode_matches_oracle(B, H, D, cap, cache_len, flags, dtype):
+    kc = synthetic.normal_tensor((B, H, cap, D), 21, 1.0, dtype)
+    vc = synthetic.normal_tensor((B, H, cap, D), 22, 1.0, dtype)
+    q, kn, vn = synthetic.qkv(B, H, 1, D, seed=23, std=1.0, dtype=dtype)
+    want_o, want_lse, _, _ = oracle.decode_attn(npf(q), npf(kn), npf(vn), npf(kc), npf(vc), cache_len)
+    kcd, vcd = kc.to(DEV), vc.to(DEV)
+    o = torch.full((B, H, 1, D), float("nan"), dtype=dtype, device=DEV)
+    lse = torch.full((B, H), float("nan"), dtype=torch.float32, device=DEV)
+    ws = workspace(L.loma_decode_workspace_bytes(B, H, D, cache_len))
+    L.loma_decode_attn(q.to(DEV), kn.to(DEV), vn.to(DEV), kcd, vcd, o, lse, cache_len, ws, flags)
+    torch.cuda.synchronize()
+    check_close(o, want_o, dtype)
+    assert np.abs(npf(lse) - want_lse[:, :, 0]).max() <= (1e-5 if dtype == torch.float32 else 2e-2)
+    # append is a bit-exact copy into slot cache_len and touches nothing else
+    exp_k, exp_v = kc.clone(), vc.clone()
+    exp_k[:, :, cache_len] = kn[:, :, 0]
+    exp_v[:, :, cache_len] = vn[:, :, 0]
+    assert np.array_equal(bits(kcd), bits(exp_k)) and np.array_equal(bits(vcd), bits(exp_v))
+    # the same step with the token already in the cache (k_new = v_new = NULL)
+    o2 = torch.empty_like(o)
+    L.loma_decode_attn(q.to(DEV), None, None, kcd, vcd, o2, None, cache_len, ws, flags)
+    torch.cuda.synchronize()
+    assert torch.equal(o2, o)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, PRIOR, GENERIC, GENERIC | PRIOR])
+@pytest.mark.parametrize("B,H,D,c,t,mem_len,extra", [(1, 1, 64, 4, 4, 0, 0), (2, 2, 128, 4, 16, 48, 5),
+                                                     (2, 3, 128, 8, 16, 1024, 0), (1, 2, 128, 3, 5, 35, 2),
+                                                     (1, 2, 128, 8, 32, 640, 7), (1, 1, 64, 1, 1, 3, 0),
+                                                     (2, 2, 128, 4, 16, 2000, 1)])
+def test_compress_matches_oracle_and_compacts_bit_exact(B, H, D, c, t, mem_len, extra, flags, dtype):
+    tc = c * t
+    cap = mem_len + tc + extra
+    kc = synthetic.normal_tensor((B, H, cap, D), 31, 1.0, dtype)
+    vc = synthetic.normal_tensor((B, H, cap, D), 32, 1.0, dtype)
+    qm, km, vm = synthetic.qkv(B, H, t, D, seed=33, std=1.0, dtype=dtype)
+    want_o, want_lse, _, _ = oracle.compress_step(npf(qm), npf(km), npf(vm), npf(kc), npf(vc), mem_len, c, t,
+                                                  flags & PRIOR)
+    kcd, vcd = kc.to(DEV), vc.to(DEV)
+    om = torch.full((B, H, t, D), float("nan"), dtype=dtype, device=DEV)
+    lse = torch.full((B, H, t), float("nan"), dtype=torch.float32, device=DEV)
+    ws = workspace(L.loma_compress_workspace_bytes(B, H, D, t, mem_len, flags))
+    L.loma_compress_step(qm.to(DEV), km.to(DEV), vm.to(DEV), kcd, vcd, om, lse, mem_len, c, t, ws, flags)
+    torch.cuda.synchronize()
+    check_close(om, want_o, dtype)
+    assert np.abs(npf(lse) - want_lse).max() <= (1e-5 if dtype == torch.float32 else 2e-2)
+    # compaction == cat(cache[:mem_len], k_mem): the oracle's explicit copies run on the raw bit patterns
+    _, _, nk, nv = oracle.compress_step(np.zeros((B, H, t, D)), bits(km), bits(vm), bits(kc), bits(vc), mem_len,
+                                        c, t, flags & PRIOR, scale=0.0)
+    assert np.array_equal(bits(kcd[:, :, :mem_len + t]), nk)
+    assert np.array_equal(bits(vcd[:, :, :mem_len + t]), nv)
+    assert np.array_equal(bits(kcd[:, :, :mem_len]), bits(kc[:, :, :mem_len]))
+
+
+# ----------------------------------------------------------- repeatability
+
+def test_results_are_bitwise_repeatable():
+    B, H, D, n, c, t = 1, 2, 128, 4, 4, 16
+    S = oracle.seq_len(n, c, t)
+    q, k, v = (x.to(DEV) for x in synthetic.qkv(B, H, S, D, seed=5, dtype=torch.bfloat16))
+    o1, l1 = run_fwd(q, k, v, n, c, t)
+    o2, l2 = run_fwd(q, k, v, n, c, t)
+    assert torch.equal(o1, o2) and torch.equal(l1, l2)
+    kc = synthetic.normal_tensor((2, 4, 3000, 128), 1, 1.0, torch.bfloat16).to(DEV)
+    vc = synthetic.normal_tensor((2, 4, 3000, 128), 2, 1.0, torch.bfloat16).to(DEV)
+    q1 = synthetic.normal_tensor((2, 4, 1, 128), 3, 1.0, torch.bfloat16).to(DEV)
+    ws = workspace(L.loma_decode_workspace_bytes(2, 4, 128, 2900))
+    outs = []
+    for _ in range(2):
+        o = torch.empty_like(q1)
+        L.loma_decode_attn(q1, None, None, kc, vc, o, None, 2900, ws)
+        torch.cuda.synchronize()
+        outs.append(o)
+    assert torch.equal(outs[0], outs[1])
+
+
+# ------------------------------------- named workloads at full size (sampled)
+
+def test_training_layout_4608_tokens_sampled_heads():
+    """B4 H32 D128 bf16, c=4, t=16, 32 chunks of [64|16|64] = 4608 rows, N(0,1):
+    the launch covers the full tensor, the oracle checks two (b,h) pairs in full."""
+    B, H, D, n, c, t = 4, 32, 128, 32, 4, 16
+    S = oracle.seq_len(n, c, t)
+    assert S == 4608
+    q = synthetic.big_normal_(torch.empty(B, H, S, D, dtype=torch.bfloat16, device=DEV), 100)
+    k = synthetic.big_normal_(torch.empty(B, H, S, D, dtype=torch.bfloat16, device=DEV), 101)
+    v = synthetic.big_normal_(torch.empty(B, H, S, D, dtype=torch.bfloat16, device=DEV), 102)
+    for flags in (0, PRIOR):
+        o, lse = run_fwd(q, k, v, n, c, t, 0, flags)
+        for b, h in [(0, 0), (3, 17)]:
+            want_o, want_lse = oracle.masked_attn_fwd(npf(q[b:b + 1, h:h + 1]), npf(k[b:b + 1, h:h + 1]),
+                                                      npf(v[b:b + 1, h:h + 1]), n, c, t, 0, flags)
+            check_close(o[b:b + 1, h:h + 1], want_o, torch.bfloat16)
+            assert np.abs(npf(lse[b:b + 1, h:h + 1]) - want_lse).max() <= 2e-2
+        assert torch.isfinite(o.float()).all()
+
+
+def test_long_training_layout_69632_tokens_sampled_rows():
+    """B1 H32 D128 bf16, c=8, t=32, 128 chunks of [256|32|256] = 69632 rows: the
+    full launch, checked on a seeded sample of rows of every zone type."""
+    B, H, D, n, c, t = 1, 32, 128, 128, 8, 32
+    S = oracle.seq_len(n, c, t)
+    assert S == 69632
+    q = synthetic.big_normal_(torch.empty(B, H, S, D, dtype=torch.bfloat16, device=DEV), 110)
+    k = synthetic.big_normal_(torch.empty(B, H, S, D, dtype=torch.bfloat16, device=DEV), 111)
+    v = synthetic.big_normal_(torch.empty(B, H, S, D, dtype=torch.bfloat16, device=DEV), 112)
+    o, lse = run_fwd(q, k, v, n, c, t)
+    zone = oracle.layout_index(n, c, t)[1]
+    rng = np.random.default_rng(0)
+    rows = np.concatenate([rng.choice(np.nonzero(zone == z)[0], 96, replace=False) for z in (0, 1, 2)]
+                          + [np.array([0, 255, 256, 287, 288, 543, 544, S - 1, S - 257, S - 545])])
+    rows = np.unique(rows)
+    idx = torch.from_numpy(rows).to(DEV)
+    for h in (0, 13, 31):
+        want_o, want_lse = oracle.masked_attn_fwd(npf(q[:, h:h + 1]), npf(k[:, h:h + 1]), npf(v[:, h:h + 1]),
+                                                  n, c, t, rows=rows)
+        check_close(o[:, h:h + 1][:, :, idx], want_o, torch.bfloat16)
+        assert np.abs(npf(lse[:, h:h + 1][:, :, idx]) - want_lse).max() <= 2e-2
+    assert torch.isfinite(o.float()).all()
+
+
+@pytest.mark.parametrize("B,H,c,t,mem_len,steps", [(32, 32, 4, 16, 8192, (0, 1, 37, 63)),
+                                                   (8, 32, 8, 16, 16384, (0, 127))])
+def test_generation_workloads_sampled_heads(B, H, c, t, mem_len, steps):
+    """Generation shapes (D128 bf16): a cache of mem_len memory entries plus a
+    growing tail; decode at several tail lengths, then the compress step.  The
+    launch covers every (b,h); the oracle checks three of them in full."""
+    D, tc = 128, c * t
+    cap = mem_len + tc + t
+    kc = synthetic.big_normal_(torch.empty(B, H, cap, D, dtype=torch.bfloat16, device=DEV), 120)
+    vc = synthetic.big_normal_(torch.empty(B, H, cap, D, dtype=torch.bfloat16, device=DEV), 121)
+    ws = workspace(max(L.loma_decode_workspace_bytes(B, H, D, cap),
+                       L.loma_compress_workspace_bytes(B, H, D, t, mem_len, PRIOR)))
+    picks = [(0, 0), (B // 2, 5), (B - 1, H - 1)]
+    for j in steps:
+        cache_len = mem_len + j
+        q, kn, vn = (x.to(DEV) for x in synthetic.qkv(B, H, 1, D, seed=200 + j, dtype=torch.bfloat16))
+        before_k = [kc[b, h].clone() for b, h in picks]
+        before_v = [vc[b, h].clone() for b, h in picks]
+        o = torch.empty(B, H, 1, D, dtype=torch.bfloat16, device=DEV)
+        lse = torch.empty(B, H, dtype=torch.float32, device=DEV)
+        L.loma_decode_attn(q, kn, vn, kc, vc, o, lse, cache_len, ws)
+        torch.cuda.synchronize()
+        for (b, h), bk, bv in zip(picks, before_k, before_v):
+            want_o, want_lse, wk, wv = oracle.decode_attn(npf(q[b:b + 1, h:h + 1]), npf(kn[b:b + 1, h:h + 1]),
+                                                          npf(vn[b:b + 1, h:h + 1]), npf(bk[None, None]),
+                                                          npf(bv[None, None]), cache_len)
+            check_close(o[b:b + 1, h:h + 1], want_o, torch.bfloat16)
+            assert abs(float(lse[b, h]) - want_lse[0, 0, 0]) <= 2e-2
+            assert np.array_equal(npf(kc[b, h]), wk[0, 0]) and np.array_equal(npf(vc[b, h]), wv[0, 0])
+    for flags in (0, PRIOR):
+        kc2, vc2 = kc.clone(), vc.clone()
+        qm, km, vm = (x.to(DEV) for x in synthetic.qkv(B, H, t, D, seed=300, dtype=torch.bfloat16))
+        om = torch.empty(B, H, t, D, dtype=torch.bfloat16, device=DEV)
+        L.loma_compress_step(qm, km, vm, kc2, vc2, om, None, mem_len, c, t, ws, flags)
+        torch.cuda.synchronize()
+        for b, h in picks:
+            want_o, _, nk, nv = oracle.compress_step(npf(qm[b:b + 1, h:h + 1]), npf(km[b:b + 1, h:h + 1]),
+                                                     npf(vm[b:b + 1, h:h + 1]), npf(kc[b:b + 1, h:h + 1]),
+                                                     npf(vc[b:b + 1, h:h + 1]), mem_len, c, t, flags)
+            check_close(om[b:b + 1, h:h + 1], want_o, torch.bfloat16)
+            assert np.array_equal(npf(kc2[b, h, :mem_len + t]), nk[0, 0])
+            assert np.array_equal(npf(vc2[b, h, :mem_len + t]), nv[0, 0])
+        del kc2, vc2
