@@ -1,0 +1,447 @@
+#!/usr/bin/env python
+"""Benchmark of the LoMA attention hot path on B200.
+
+One step = one pass of the whole hot path over one batch of synthetic input:
+  1. index maps (loma_layout_index, loma_generation_index) on the device
+  2. loma_masked_attn_fwd on the 4608-token training layout
+     (B4 H32 D128 bf16, c=4, t=16, 32 chunks of [64|16|64])
+  3. one generation cycle on the compressed cache (B32 H32 D128 bf16, 8192
+     memory entries): tc = 64 x loma_decode_attn with the tail growing from 0 to
+     63, then one loma_compress_step (16 memory queries + in-place compaction)
+
+`value` is the masked-attention useful TFLOP/s (4*D FLOPs per allowed
+(query, key) pair; allowed pairs counted from Eq. 1-3 in closed form); the
+decode GB/s (the other half of the metric) is in `decode_attn`, and the
+roofline object describes the decode kernel, which dominates the step's time.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With --gpus N > 1 (launched under torch.distributed.run, one rank per GPU) every
+rank runs the same per-GPU workload on its own (batch, head) shard: no
+collective is on the data path, scaling is weak, and times are the max over
+ranks.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "LoMA masked-attn useful TFLOP/s; compressed decode-attn HBM GB/s vs roofline"
+
+# workload: training-layout forward (configs[1]) + generation cycle (configs[2])
+FWD = dict(B=4, H=32, D=128, n=32, c=4, t=16)
+GEN = dict(B=32, H=32, D=128, c=4, t=16, mem_len=8192)
+
+
+def allowed_pairs(n: int, c: int, t: int, prior_mem: bool = False) -> int:
+    """Ones in the Eq. 2 mask of n chunks, counted block by block (Eq. 1, Eq. 3)."""
+    tc = t * c
+    per_chunk = tc * (tc + 1) // 2 + t * (tc + t) + tc * (t + 1)
+    cross = tc * t + (t * t if prior_mem else 0)
+    return n * per_chunk + cross * n * (n - 1) // 2
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); smax.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for nme, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nme)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
+        return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), power_w_max=max(power),
+                    samples=len(sm), reasons=sorted(reasons))
+
+
+# --------------------------------------------------------------------------- ours
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2401_09486_b200 import binding as L
+    from paper_2401_09486_b200 import build, synthetic
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        if world == 1 and args.gpus > 1:
+            raise SystemExit("--gpus N > 1 must be launched with torch.distributed.run, one rank per GPU")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        build.build_library()
+    if world > 1:
+        dist.barrier()
+    L.lib()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------- inputs (seeded, synthetic; rank-dependent seeds) ----------------
+    f, g = FWD, GEN
+    tc_f = f["c"] * f["t"]
+    S = f["n"] * (2 * tc_f + f["t"])
+    std = 1.0 / math.sqrt(f["D"])
+    bf = torch.bfloat16
+    q, k, v = (synthetic.big_normal_(torch.empty(f["B"], f["H"], S, f["D"], dtype=bf, device=dev), 1000 + 10 * rank + i,
+                                     std) for i in range(3))
+    o = torch.empty_like(q)
+    tc_g = g["c"] * g["t"]
+    cap = g["mem_len"] + tc_g + g["t"]
+    kc = synthetic.big_normal_(torch.empty(g["B"], g["H"], cap, g["D"], dtype=bf, device=dev), 2000 + 10 * rank, std)
+    vc = synthetic.big_normal_(torch.empty(g["B"], g["H"], cap, g["D"], dtype=bf, device=dev), 2001 + 10 * rank, std)
+    # one (q, k_new, v_new) triple per decode step of the cycle, and the memory-token triple
+    dq, dk, dv = (synthetic.big_normal_(torch.empty(tc_g, g["B"], g["H"], 1, g["D"], dtype=bf, device=dev),
+                                        2100 + 10 * rank + i, std) for i in range(3))
+    do = torch.empty_like(dq)
+    qm, km, vm = (synthetic.big_normal_(torch.empty(g["B"], g["H"], g["t"], g["D"], dtype=bf, device=dev),
+                                        2200 + 10 * rank + i, std) for i in range(3))
+    om = torch.empty_like(qm)
+    ws_bytes = max(16, L.loma_decode_workspace_bytes(g["B"], g["H"], g["D"], cap),
+                   L.loma_compress_workspace_bytes(g["B"], g["H"], g["D"], g["t"], g["mem_len"], 0))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    idx_fwd = [torch.empty(S, dtype=torch.int32, device=dev) for _ in range(5)]
+    idx_gen = [torch.empty(tc_g, dtype=torch.int32, device=dev) for _ in range(3)]
+    stream = torch.cuda.current_stream()
+    st = stream.cuda_stream
+    lib = L.lib()
+    import ctypes
+    P = lambda x: ctypes.c_void_p(x.data_ptr())
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def step(marks=None):
+        """All hot-path calls of one step, on the current stream, through the C ABI."""
+        def mark(name):
+            if marks is not None:
+                e = ev(); e.record(stream); marks.append((name, e))
+        mark("start")
+        rc = lib.loma_layout_index(f["n"], f["c"], f["t"], 0, *[P(x) for x in idx_fwd], 1, st)
+        rc |= lib.loma_generation_index(tc_g, g["c"], g["t"], *[P(x) for x in idx_gen], 1, st)
+        mark("index")
+        L.loma_masked_attn_fwd(q, k, v, o, None, f["n"], f["c"], f["t"], 0, 0, 0.0, stream)
+        mark("masked_fwd")
+        for j in range(tc_g):
+            L.loma_decode_attn(dq[j], dk[j], dv[j], kc, vc, do[j], None, g["mem_len"] + j, ws, 0, 0.0, stream)
+        mark("decode")
+        L.loma_compress_step(qm, km, vm, kc, vc, om, None, g["mem_len"], g["c"], g["t"], ws, 0, 0.0, stream)
+        mark("compress")
+        if rc != 0:
+            raise RuntimeError("index map call failed")
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = L.loma_launch_count()
+    all_marks = []
+    e0, e1 = ev(), ev()
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        marks = []
+        step(marks)
+        all_marks.append(marks)
+    e1.record(stream)
+    barrier()
+    total_ms = e0.elapsed_time(e1)
+    launches = L.loma_launch_count() - launches0
+    clocks = sampler.stop()
+    assert L.loma_device_status() == 0
+
+    phase_ms = {}
+    for marks in all_marks:
+        for (n0, a), (n1, b) in zip(marks[:-1], marks[1:]):
+            phase_ms[n1] = phase_ms.get(n1, 0.0) + a.elapsed_time(b)
+    phase_ms = {kk: vv / args.steps for kk, vv in phase_ms.items()}
+
+    # max over ranks of every time
+    times = torch.tensor([total_ms] + [phase_ms[x] for x in ("index", "masked_fwd", "decode", "compress")],
+                         dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, t_index, t_fwd, t_dec, t_cmp = times.tolist()
+    ms_per_step = total_ms / args.steps
+
+    # ---------------- e2e: host buffers, copies inside the timed region ----------------
+    pin = lambda x: torch.empty(x.shape, dtype=x.dtype, device="cpu", pin_memory=True).copy_(x)
+    hq, hk, hv = pin(q), pin(k), pin(v)
+    ho = torch.empty(o.shape, dtype=o.dtype, device="cpu", pin_memory=True)
+    hdq, hdk, hdv = pin(dq), pin(dk), pin(dv)
+    hdo = torch.empty(do.shape, dtype=do.dtype, device="cpu", pin_memory=True)
+    hqm, hkm, hvm = pin(qm), pin(km), pin(vm)
+    hom = torch.empty(om.shape, dtype=om.dtype, device="cpu", pin_memory=True)
+    nbytes = lambda *xs: sum(x.numel() * x.element_size() for x in xs)
+    h2d = nbytes(hq, hk, hv, hdq, hdk, hdv, hqm, hkm, hvm)
+    d2h = nbytes(ho, hdo, hom)
+
+    def e2e_step(marks):
+        def mark(name):
+            e = ev(); e.record(stream); marks.append((name, e))
+        mark("start")
+        q.copy_(hq, non_blocking=True); k.copy_(hk, non_blocking=True); v.copy_(hv, non_blocking=True)
+        L.loma_masked_attn_fwd(q, k, v, o, None, f["n"], f["c"], f["t"], 0, 0, 0.0, stream)
+        ho.copy_(o, non_blocking=True)
+        mark("masked_fwd")
+        for j in range(tc_g):
+            dq[j].copy_(hdq[j], non_blocking=True); dk[j].copy_(hdk[j], non_blocking=True)
+            dv[j].copy_(hdv[j], non_blocking=True)
+            L.loma_decode_attn(dq[j], dk[j], dv[j], kc, vc, do[j], None, g["mem_len"] + j, ws, 0, 0.0, stream)
+            hdo[j].copy_(do[j], non_blocking=True)
+        mark("decode")
+        qm.copy_(hqm, non_blocking=True); km.copy_(hkm, non_blocking=True); vm.copy_(hvm, non_blocking=True)
+        L.loma_compress_step(qm, km, vm, kc, vc, om, None, g["mem_len"], g["c"], g["t"], ws, 0, 0.0, stream)
+        hom.copy_(om, non_blocking=True)
+        mark("compress")
+
+    e2e_step([])
+    barrier()
+    e2e_steps = max(1, min(args.steps, 3))
+    e2e_fwd = e2e_dec = e2e_tot = 0.0
+    for _ in range(e2e_steps):
+        marks = []
+        e2e_step(marks)
+        torch.cuda.synchronize()
+        e2e_fwd += marks[0][1].elapsed_time(marks[1][1])
+        e2e_dec += marks[1][1].elapsed_time(marks[2][1])
+        e2e_tot += marks[0][1].elapsed_time(marks[3][1])
+    et = torch.tensor([e2e_fwd / e2e_steps, e2e_dec / e2e_steps, e2e_tot / e2e_steps], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(et, op=dist.ReduceOp.MAX)
+    e2e_fwd, e2e_dec, e2e_tot = et.tolist()
+
+    # ---------------- figures ----------------
+    peaks = load_peaks()
+    pairs = allowed_pairs(f["n"], f["c"], f["t"])
+    fwd_flops = 4.0 * f["D"] * pairs * f["B"] * f["H"]                 # per GPU
+    fwd_bytes = 4.0 * q.numel() * 2                                    # Q, K, V read + O written once
+    fwd_tflops = world * fwd_flops / (t_fwd * 1e-3) / 1e12
+    # decode: algorithmic bytes = every visible K and V row read once (cache_len + 1 rows per (b,h))
+    dec_rows = sum(g["mem_len"] + j + 1 for j in range(tc_g))
+    dec_bytes_cycle = 2.0 * dec_rows * g["B"] * g["H"] * g["D"] * 2
+    dec_bytes_launch = dec_bytes_cycle / tc_g
+    dec_ms_launch = t_dec / tc_g
+    dec_gbs = dec_bytes_launch / (dec_ms_launch * 1e-3) / 1e9          # per GPU
+    # compress (paper variant): tail K,V read + q,k,v_mem read + o_mem written + compaction written
+    bh = g["B"] * g["H"]
+    cmp_bytes = bh * g["D"] * 2.0 * (2 * tc_g + 3 * g["t"] + g["t"] + 2 * g["t"])
+    cmp_gbs = cmp_bytes / (t_cmp * 1e-3) / 1e9
+
+    out = {
+        "metric": METRIC,
+        "value": fwd_tflops,
+        "unit": "TFLOP/s",
+        "n_gpus": world,
+        "steps": args.steps,
+        "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step,
+        "higher_is_better": True,
+        "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": "bf16",
+        "data": "synthetic",
+        "config": {
+            "workload": ("masked fwd B4 H32 D128 c4 t16 n32 S4608 + generation cycle B32 H32 D128 c4 t16 "
+                         "mem 8192: 64 decode + 1 compress"),
+            "masked_fwd": dict(f, S=S, std="1/sqrt(D)"),
+            "generation": dict(g, cap=cap, decode_steps=tc_g),
+            "l2": "inputs larger than L2 (604 MB forward tensors, 4.3 GB cache streamed by every decode)",
+            "per_gpu_batch": "fixed (weak scaling over (batch, head) shards, no collective)",
+        },
+        "phases_ms": {"index_maps": t_index, "masked_attn_fwd": t_fwd, "decode_cycle": t_dec, "compress_step": t_cmp},
+        "decode_attn": {"value": world * dec_gbs, "unit": "GB/s", "ms_per_call": dec_ms_launch,
+                        "bytes_per_call": dec_bytes_launch, "frac_of_measured_hbm": dec_gbs / peaks["hbm_gbs"],
+                        "frac_of_8tbs": dec_gbs / 8000.0},
+        "masked_attn": {"useful_tflops": fwd_tflops, "ms": t_fwd, "useful_flops": fwd_flops,
+                        "compulsory_bytes": fwd_bytes, "gbs": fwd_bytes / (t_fwd * 1e-3) / 1e9,
+                        "frac_of_measured_hbm": fwd_bytes / (t_fwd * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                        "frac_of_measured_bf16": fwd_tflops / world / peaks["bf16_tflops"]},
+        "compress": {"ms": t_cmp, "bytes": cmp_bytes, "gbs": cmp_gbs,
+                     "frac_of_measured_hbm": cmp_gbs / peaks["hbm_gbs"],
+                     "note": "timed in place after the 64 decodes of the cycle"},
+        "roofline": {"kernel": "decode_splitkv_kernel<128> (+ merge), per loma_decode_attn call", "bound": "hbm",
+                     "achieved": dec_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": dec_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None},
+        "e2e": {"value": world * fwd_flops / (e2e_fwd * 1e-3) / 1e12, "unit": "TFLOP/s",
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_tot,
+                "masked_fwd_ms": e2e_fwd, "decode_cycle_ms": e2e_dec,
+                "decode_gbs": world * dec_bytes_cycle / (e2e_dec * 1e-3) / 1e9},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    if rank == 0:
+        out["cpu_baseline"] = cpu_baseline()
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------ oracle timing
+
+def _oracle_sample(n_heads_fwd: int, n_heads_dec: int, seed: int = 0):
+    """Times the oracle, as it stands, on a bounded sample of the bench workload:
+    the masked forward for n_heads_fwd (b,h) pairs of the 4608-token layout and
+    one decode step (tail 32) for n_heads_dec (b,h) pairs of the generation cache."""
+    import numpy as np
+    import torch
+
+    import oracle
+    from paper_2401_09486_b200 import synthetic
+
+    f, g = FWD, GEN
+    tc_f = f["c"] * f["t"]
+    S = f["n"] * (2 * tc_f + f["t"])
+    std = 1.0 / math.sqrt(f["D"])
+    q, k, v = (x.to(torch.float64).numpy() for x in synthetic.qkv(1, n_heads_fwd, S, f["D"], seed, std, torch.bfloat16))
+    t0 = time.perf_counter()
+    oracle.masked_attn_fwd(q, k, v, f["n"], f["c"], f["t"])
+    t_fwd = time.perf_counter() - t0
+    cache_len = g["mem_len"] + 32
+    kc = synthetic.normal_tensor((1, n_heads_dec, cache_len + 1, g["D"]), seed + 1, std, torch.bfloat16).to(torch.float64).numpy()
+    vc = synthetic.normal_tensor((1, n_heads_dec, cache_len + 1, g["D"]), seed + 2, std, torch.bfloat16).to(torch.float64).numpy()
+    q1, k1, v1 = (x.to(torch.float64).numpy() for x in synthetic.qkv(1, n_heads_dec, 1, g["D"], seed + 3, std, torch.bfloat16))
+    t0 = time.perf_counter()
+    oracle.decode_attn(q1, k1, v1, kc, vc, cache_len)
+    t_dec = time.perf_counter() - t0
+    pairs = allowed_pairs(f["n"], f["c"], f["t"])
+    tflops = 4.0 * f["D"] * pairs * n_heads_fwd / t_fwd / 1e12
+    dec_gbs = 2.0 * (cache_len + 1) * g["D"] * 2 * n_heads_dec / t_dec / 1e9
+    return tflops, dec_gbs, t_fwd, t_dec
+
+
+def _threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        return int(n)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline():
+    tflops, dec_gbs, t_fwd, t_dec = _oracle_sample(n_heads_fwd=16, n_heads_dec=64)
+    return {"value": tflops, "unit": "TFLOP/s", "cores": _threads(), "kind": "oracle",
+            "sample": ("masked fwd: 16 of 128 (b,h) pairs of the 4608-token layout, dense fp64 NumPy, "
+                       f"{t_fwd:.2f} s; decode: 64 of 1024 (b,h) pairs, one step at cache length 8224, {t_dec:.2f} s"),
+            "decode_gbs": dec_gbs, "host_cores": os.cpu_count()}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals, decs, times = [], [], []
+    for i in range(max(args.warmup, 1) + args.steps):
+        t0 = time.perf_counter()
+        tf, dg, _, _ = _oracle_sample(n_heads_fwd=1, n_heads_dec=4, seed=i)
+        if i >= max(args.warmup, 1):
+            vals.append(tf); decs.append(dg); times.append(time.perf_counter() - t0)
+    val = statistics.mean(vals)
+    cores = _threads()
+    sample = "per step: masked fwd of 1 of 128 (b,h) pairs (4608 tokens) + one decode step for 4 of 1024 (b,h) pairs"
+    out = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": max(args.warmup, 1), "ms_per_step": 1e3 * statistics.mean(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "CPU oracle on a bounded sample of the same workload", "masked_fwd": FWD,
+                   "generation": GEN},
+        "decode_attn": {"value": statistics.mean(decs), "unit": "GB/s"},
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -229,6 +229,10 @@ LOMA_API size_t loma_compress_workspace_bytes(int B, int H, int D, int t, int me
  * LOMA_ERR_CUDA if the synchronisation or the read fails. */
 LOMA_API int loma_device_status(void* stream);
 
+/* Number of kernels this library has enqueued in the calling process since it
+ * was loaded (all devices, all streams).  Host-side counter; never fails. */
+LOMA_API uint64_t loma_launch_count(void);
+
 /* Static, human-readable name of a status code. */
 LOMA_API const char* loma_status_string(int status);
 

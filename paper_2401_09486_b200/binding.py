@@ -38,6 +38,7 @@ SIGNATURES = {
                                 _p]),
     "loma_compress_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _u]),
     "loma_device_status": (_i, [_p]),
+    "loma_launch_count": (ctypes.c_uint64, []),
     "loma_status_string": (ctypes.c_char_p, [_i]),
     "loma_version": (_i, []),
 }
@@ -101,6 +102,10 @@ def _stream(stream) -> ctypes.c_void_p:
 
 def loma_version() -> int:
     return lib().loma_version()
+
+
+def loma_launch_count() -> int:
+    return int(lib().loma_launch_count())
 
 
 def loma_device_status(stream=None) -> int:

@@ -323,6 +323,7 @@ static cudaError_t masked_generic_t(const void* q, const void* k, const void* v,
     masked_attn_generic_kernel<T, D><<<grid, GENERIC_WARPS * 32, 0, st>>>(
         static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), static_cast<T*>(o), lse,
         H, L, sb, sh, ss, scale);
+    count_launches(1);
     return cudaGetLastError();
 }
 
@@ -345,6 +346,7 @@ static cudaError_t decode_generic_t(const void* q, const void* kn, const void* v
                                                    static_cast<const T*>(vn), static_cast<T*>(kc),
                                                    static_cast<T*>(vc), static_cast<T*>(o), lse, cap,
                                                    cache_len, scale);
+    count_launches(1);
     return cudaGetLastError();
 }
 
@@ -371,6 +373,7 @@ static cudaError_t compress_generic_t(const void* qm, const void* km, const void
     compress_generic_kernel<T, D><<<BH, GENERIC_WARPS * 32, 0, st>>>(
         static_cast<const T*>(qm), static_cast<const T*>(km), static_cast<const T*>(vm), static_cast<T*>(kc),
         static_cast<T*>(vc), static_cast<T*>(om), lse, cap, mem_len, t, tc, flags, scale);
+    count_launches(1);
     return cudaGetLastError();
 }
 

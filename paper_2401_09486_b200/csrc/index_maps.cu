@@ -93,6 +93,7 @@ cudaError_t launch_layout_index(const Layout& L, int32_t* chunk, int32_t* zone, 
     const int threads = 256;
     layout_index_kernel<<<(L.S + threads - 1) / threads, threads, 0, st>>>(L.S, L.n_chunks, L.c, L.t, chunk,
                                                                          zone, offset, src, pos);
+    count_launches(1);
     return cudaGetLastError();
 }
 
@@ -102,6 +103,7 @@ cudaError_t launch_generation_index(int n_tokens, int c, int t, int32_t* slot, i
     const int threads = 256;
     generation_index_kernel<<<(n_tokens + threads - 1) / threads, threads, 0, st>>>(n_tokens, c, t, slot, pos,
                                                                                   comp);
+    count_launches(1);
     return cudaGetLastError();
 }
 

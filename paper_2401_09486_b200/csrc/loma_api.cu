@@ -3,9 +3,14 @@
 #include <limits.h>
 #include <math.h>
 
+#include <atomic>
+
 #include "loma_internal.cuh"
 
 namespace loma {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
 __device__ int g_status_word = 0;
 
@@ -62,6 +67,8 @@ using namespace loma;
 extern "C" {
 
 int loma_version(void) { return 100; }
+
+uint64_t loma_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* loma_status_string(int status) {
     switch (status) {
@@ -139,15 +146,14 @@ int loma_masked_attn_fwd(const void* q, const void* k, const void* v, void* o, f
 }
 
 size_t loma_decode_workspace_bytes(int B, int H, int D, int cache_len) {
-    (void)B; (void)H; (void)D; (void)cache_len;
-    return 0;
+    if (B <= 0 || H <= 0 || D <= 0 || cache_len < 0) return 0;
+    return decode_workspace_bytes(B * H, D, cache_len + 1);
 }
 
 int loma_decode_attn(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
                      float* lse, int B, int H, int D, int cap, int cache_len, loma_dtype dtype,
                      float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes,
                      void* stream) {
-    (void)flags;
     if (B < 0 || H < 0 || cap < 0 || cache_len < 0) return LOMA_ERR_INVALID_ARG;
     if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
     if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
@@ -164,8 +170,14 @@ int loma_decode_attn(const void* q, const void* k_new, const void* v_new, void* 
     if (dc != LOMA_OK) return dc;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = launch_decode_generic(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len,
-                                          dtype, scale, st);
+    if ((int64_t)B * H * 128 > INT_MAX) return LOMA_ERR_INVALID_ARG;
+    cudaError_t e;
+    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC))
+        e = launch_decode_bf16(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, scale,
+                               workspace, st);
+    else
+        e = launch_decode_generic(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, dtype,
+                                  scale, st);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 

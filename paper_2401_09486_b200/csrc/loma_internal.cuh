@@ -38,10 +38,19 @@ cudaError_t launch_decode_generic(const void* q, const void* k_new, const void* 
                                   int B, int H, int D, int cap, int cache_len,
                                   loma_dtype dt, float scale, cudaStream_t st);
 
+// bf16 split-KV decode (decode_splitkv.cu)
+size_t decode_workspace_bytes(int BH, int D, int total_keys);
+cudaError_t launch_decode_bf16(const void* q, const void* k_new, const void* v_new, void* k_cache,
+                               void* v_cache, void* o, float* lse, int B, int H, int D, int cap, int cache_len,
+                               float scale, void* ws, cudaStream_t st);
+
 cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const void* v_mem,
                                     void* k_cache, void* v_cache, void* o_mem, float* lse,
                                     int B, int H, int D, int cap, int mem_len, int c, int t,
                                     loma_dtype dt, float scale, unsigned flags, cudaStream_t st);
+
+// ---- launch accounting -------------------------------------------------------
+void count_launches(int n);   // called by every launcher with the number of kernels it enqueued
 
 // ---- device status word (bounded waits report here) ------------------------
 int* device_status_word();   // device address of the status word of the current device (NULL on failure)
