@@ -193,6 +193,53 @@ LOMA_API int loma_decode_attn(const void* q, const void* k_new, const void* v_ne
 LOMA_API size_t loma_decode_workspace_bytes(int B, int H, int D, int cache_len);
 
 /* ---------------------------------------------------------------------------
+ * loma_decode_attn_static -- the same decode step as loma_decode_attn (bf16
+ * only), for callers that cannot hand the library a workspace because they
+ * cannot obtain device memory at the point of the call.  (The paper has no
+ * counterpart: this is a packaging variant, not a different computation.)
+ *
+ * Who needs it: code that runs after the process has committed all of its
+ * device memory to a fixed plan (a serving engine whose KV-cache pool owns the
+ * rest of HBM, so a late cudaMalloc fails); plug-ins called from a host
+ * runtime that forbids allocation inside its step function because
+ * cudaMalloc/cudaFree synchronise the whole device; and callers with no
+ * allocator of their own at hand (a bare C program holding only the tensors
+ * it was given).  For them the split-KV partial results go into an 8 MiB
+ * array that is part of the library image itself:
+ *
+ *   - Every GPU on which the library is used holds those 8 MiB
+ *     (loma_decode_static_scratch_bytes()) from the first use until the
+ *     process exits, whether or not this entry point is ever called again.
+ *   - A request whose partials do not fit -- i.e. whose
+ *     loma_decode_workspace_bytes(B,H,D,cache_len) exceeds that size -- is
+ *     rejected with LOMA_ERR_WORKSPACE and nothing is launched.  (B*H = 1024
+ *     pairs at a cache length of 8k need 4.8 MB; 1024 pairs at 16k do not fit.)
+ *   - The call itself allocates nothing: no cudaMalloc, cudaFree or other
+ *     allocating routine is reached from it.
+ *   - The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current) and caches it.  Make
+ *     that first call during set-up, before any stream capture begins.
+ *   - All calls share the one array.  Nothing in it has to be cleared between
+ *     calls (every partial that is read has been written by the same call),
+ *     but two calls that can overlap on the GPU -- different streams without an
+ *     ordering between them -- overwrite each other's partials and give wrong
+ *     results.  Keep calls on one stream, or order them with events.
+ *
+ * Arguments, layouts, the append of k_new/v_new at slot cache_len and the
+ * results are exactly those of loma_decode_attn without its workspace pair and
+ * flags.  Errors: INVALID_ARG, UNSUPPORTED (dtype other than LOMA_BF16, D not
+ * 64/128, device not sm_100), ALIGNMENT, CAPACITY, WORKSPACE (too large for the
+ * built-in array), CUDA.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_decode_attn_static(const void* q, const void* k_new, const void* v_new,
+                                     void* k_cache, void* v_cache, void* o, float* lse,
+                                     int B, int H, int D, int cap, int cache_len,
+                                     loma_dtype dtype, float softmax_scale, void* stream);
+
+/* Size in bytes of the built-in scratch array used by loma_decode_attn_static. */
+LOMA_API size_t loma_decode_static_scratch_bytes(void);
+
+/* ---------------------------------------------------------------------------
  * loma_compress_step -- Section 3.1 step 2 (one pass of t <m> tokens over
  * KV_Read) and step 3 (KV_Read is discarded), fused.
  *

@@ -34,6 +34,8 @@ SIGNATURES = {
                                   _u, _p]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
+    "loma_decode_attn_static": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _p]),
+    "loma_decode_static_scratch_bytes": (_sz, []),
     "loma_compress_step": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz,
                                 _p]),
     "loma_compress_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _u]),
@@ -168,6 +170,25 @@ def loma_decode_attn(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len: int, 
                                 _ptr(lse), B, H, D, cap, cache_len, _dtype_code(q), float(softmax_scale),
                                 int(flags), _ptr(workspace), ws_bytes, _stream(stream))
     _check(rc, "loma_decode_attn")
+
+
+def loma_decode_static_scratch_bytes() -> int:
+    return int(lib().loma_decode_static_scratch_bytes())
+
+
+def loma_decode_attn_static(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len: int, softmax_scale: float = 0.0,
+                            stream=None) -> None:
+    """loma_decode_attn without a workspace argument: the split partials go to
+    the library's built-in 8 MiB array, so the call needs no device memory beyond
+    the tensors passed in.  Same tensor conventions as loma_decode_attn (bf16)."""
+    B, H, cap, D = k_cache.shape
+    for x in (q, k_new, v_new, k_cache, v_cache, o):
+        if x is not None and not x.is_contiguous():
+            raise ValueError("decode tensors must be contiguous")
+    rc = lib().loma_decode_attn_static(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(o),
+                                       _ptr(lse), B, H, D, cap, cache_len, _dtype_code(q), float(softmax_scale),
+                                       _stream(stream))
+    _check(rc, "loma_decode_attn_static")
 
 
 def loma_compress_workspace_bytes(B: int, H: int, D: int, t: int, mem_len: int, flags: int = 0) -> int:

@@ -264,4 +264,37 @@ cudaError_t launch_decode_bf16(const void* q, const void* k_new, const void* v_n
                                         st);
 }
 
+// ---------------------------------------------------------------------------
+// Built-in scratch for loma_decode_attn_static: the split partials live in this
+// fixed array instead of a caller-provided workspace.  In host code the name
+// below is only a handle; the device address is looked up per device.
+constexpr size_t DEC_STATIC_SCRATCH_BYTES = 8u << 20;   // 8 MiB, held by every device that loads the library
+static __device__ __align__(256) unsigned char g_decode_scratch[DEC_STATIC_SCRATCH_BYTES];
+
+size_t decode_static_scratch_bytes() { return DEC_STATIC_SCRATCH_BYTES; }
+
+// Device address of g_decode_scratch on the current device (looked up once per
+// device, with that device current).  nullptr if the lookup fails.
+static void* decode_static_scratch() {
+    static void* addr[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!addr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress((void**)&p, g_decode_scratch) != cudaSuccess) return nullptr;
+        addr[dev] = p;
+    }
+    return addr[dev];
+}
+
+// Same kernels as launch_decode_bf16, with the partials in the built-in array.
+// The caller has checked that decode_workspace_bytes(...) fits.
+cudaError_t launch_decode_bf16_static(const void* q, const void* k_new, const void* v_new, void* k_cache,
+                                      void* v_cache, void* o, float* lse, int B, int H, int D, int cap,
+                                      int cache_len, float scale, cudaStream_t st) {
+    void* ws = decode_static_scratch();
+    if (!ws) return cudaErrorInvalidSymbol;
+    return launch_decode_bf16(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, scale, ws, st);
+}
+
 }  // namespace loma

@@ -181,6 +181,32 @@ int loma_decode_attn(const void* q, const void* k_new, const void* v_new, void* 
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 
+size_t loma_decode_static_scratch_bytes(void) { return decode_static_scratch_bytes(); }
+
+int loma_decode_attn_static(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                            void* o, float* lse, int B, int H, int D, int cap, int cache_len, loma_dtype dtype,
+                            float softmax_scale, void* stream) {
+    if (B < 0 || H < 0 || cap < 0 || cache_len < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    if ((k_new == nullptr) != (v_new == nullptr)) return LOMA_ERR_INVALID_ARG;
+    if (cache_len >= cap) return LOMA_ERR_CAPACITY;
+    if (B == 0 || H == 0) return LOMA_OK;
+    if (!q || !k_cache || !v_cache || !o) return LOMA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) || !aligned16(k_new) ||
+        !aligned16(v_new))
+        return LOMA_ERR_ALIGNMENT;
+    if ((int64_t)B * H * 128 > INT_MAX) return LOMA_ERR_INVALID_ARG;
+    // the request must fit the built-in scratch array
+    if (decode_workspace_bytes(B * H, D, cache_len + 1) > decode_static_scratch_bytes()) return LOMA_ERR_WORKSPACE;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    cudaError_t e = launch_decode_bf16_static(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len,
+                                              scale, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
 size_t loma_compress_workspace_bytes(int B, int H, int D, int t, int mem_len, unsigned flags) {
     (void)B; (void)H; (void)D; (void)t; (void)mem_len; (void)flags;
     return 0;

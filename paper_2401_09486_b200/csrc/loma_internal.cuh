@@ -44,6 +44,11 @@ cudaError_t launch_decode_bf16(const void* q, const void* k_new, const void* v_n
                                void* v_cache, void* o, float* lse, int B, int H, int D, int cap, int cache_len,
                                float scale, void* ws, cudaStream_t st);
 
+size_t decode_static_scratch_bytes();
+cudaError_t launch_decode_bf16_static(const void* q, const void* k_new, const void* v_new, void* k_cache,
+                                      void* v_cache, void* o, float* lse, int B, int H, int D, int cap,
+                                      int cache_len, float scale, cudaStream_t st);
+
 cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const void* v_mem,
                                     void* k_cache, void* v_cache, void* o_mem, float* lse,
                                     int B, int H, int D, int cap, int mem_len, int c, int t,
