@@ -162,6 +162,20 @@ LOMA_API int loma_masked_attn_fwd(const void* q, const void* k, const void* v, v
                                   loma_dtype dtype, float softmax_scale, unsigned flags, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * loma_masked_attn_plan_coverage -- host-only introspection of the tensor-core
+ * kernel's tile plan for loma_masked_attn_fwd (Eq. 1-3).  The kernel never
+ * stores the mask: it visits, per 128-row query tile, only the key tiles that
+ * hold an allowed entry, and inside a visited tile lets each row attend to one
+ * interval of columns.  This routine replays that plan on the host and writes
+ *   counts[i*S + j] = how many visits let row i attend to column j  (saturating)
+ * into a [host] uint8 buffer of S*S bytes, S = n_chunks*t*(2c+1) + tail_read.
+ * A correct plan reproduces the mask M of Eq. 2 exactly (every count 0 or 1).
+ * No CUDA call is made.  Errors: INVALID_ARG (bad geometry, NULL, S*S > 2^32).
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_masked_attn_plan_coverage(int n_chunks, int c, int t, int tail_read, unsigned flags,
+                                            uint8_t* counts);
+
+/* ---------------------------------------------------------------------------
  * loma_decode_attn -- one new token per (batch, head) attends to the cache_len
  * entries already in the cache (all memory entries, then the uncompressed tail)
  * and to itself: the mask row tril(ones(1, 1+k), diagonal=k) of Appendix A with

@@ -32,6 +32,7 @@ SIGNATURES = {
     "loma_generation_index": (_i, [_i, _i, _i, _p, _p, _p, _i, _p]),
     "loma_masked_attn_fwd": (_i, [_p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i, _f,
                                   _u, _p]),
+    "loma_masked_attn_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "loma_decode_attn_static": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _p]),
@@ -152,6 +153,15 @@ def loma_masked_attn_fwd(q, k, v, o, lse, n_chunks: int, c: int, t: int, tail_re
                                     tail_read, q.stride(0), q.stride(1), q.stride(2), _dtype_code(q),
                                     float(softmax_scale), int(flags), _stream(stream))
     _check(rc, "loma_masked_attn_fwd")
+
+
+def loma_masked_attn_plan_coverage(n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0) -> torch.Tensor:
+    """Host replay of the tensor-core kernel's tile plan: uint8 [S, S] visit counts."""
+    S = n_chunks * (2 * c * t + t) + tail_read
+    counts = torch.empty((S, S), dtype=torch.uint8)
+    rc = lib().loma_masked_attn_plan_coverage(n_chunks, c, t, tail_read, int(flags), _ptr(counts))
+    _check(rc, "loma_masked_attn_plan_coverage")
+    return counts
 
 
 def loma_decode_workspace_bytes(B: int, H: int, D: int, cache_len: int) -> int:

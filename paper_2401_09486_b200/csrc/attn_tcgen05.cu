@@ -1,0 +1,588 @@
+// Zone-masked attention forward on the 5th-generation tensor cores (sm_100a):
+// tcgen05.mma with TMEM accumulators, operands staged by TMA.
+//
+// The mask of Eq. 1-3 is never stored and never evaluated entry by entry.  The
+// sequence is seen through four "zone views" -- reading, memory and repetition
+// zones of the complete chunks, and the reading tail -- each a 5-D tensor
+// (d, row in zone, chunk, head, batch) over the caller's Q/K/V/O.  A tile is
+// 128 rows of one view: 128 consecutive rows of a zone when the zone is at
+// least that long, otherwise the whole zone of as many consecutive chunks as
+// fit (one TMA box gathers them into a dense tile).  For a query tile only the
+// key tiles that hold an allowed entry are visited (everything else is
+// skipped), and inside a visited tile the allowed columns of a row always form
+// one interval [lo, hi), so the mask costs two compares per score at most:
+//
+//   reading rows    x memory tiles of earlier chunks   key chunk <  row chunk  (Eq. 3)
+//   reading rows    x own reading zone                 causal                   (L of Eq. 1)
+//   memory rows     x own reading and memory zone      key chunk == row chunk   (Eq. 1, row 2)
+//   memory rows     x earlier memory zones             key chunk <= row chunk   (prior-memory flag)
+//   repetition rows x own memory zone                  key chunk == row chunk   (Eq. 1, row 3)
+//   repetition rows x themselves                       diagonal                 (I of Eq. 1)
+//
+// One CTA (192 threads) per SM, persistent over a statically ordered tile list
+// (longest tiles first, (batch, head) fastest).  Roles:
+//   warps 0-3  softmax: thread = query row = TMEM lane; two passes over the
+//              score tile in TMEM (row max, then exp2 / row sum / bf16 P written
+//              back over the scores), output accumulated in registers from the
+//              per-step P.V products, final O staged in shared memory for a TMA store
+//   warp 4     TMA producer: Q per tile, K and V rings of two stages each
+//   warp 5     MMA issuer: S = Q K^T (both operands in shared memory), then
+//              P.V with P read from TMEM and V as an MN-major shared operand
+// TMEM (512 columns): two score buffers and two P.V buffers of 128 columns, so
+// the tensor pipe computes S(j+1) and P.V(j-1) while the softmax warps work on
+// S(j).  Every mbarrier wait is bounded: on expiry the CTA records
+// LOMA_ERR_TIMEOUT, all roles leave their loops, TMEM is freed and the kernel
+// returns.
+#include <cuda.h>
+#include <math.h>
+
+#include <mutex>
+
+#include "loma_internal.cuh"
+#include "tile_plan.cuh"
+
+namespace loma {
+
+struct TmaMaps {
+    CUtensorMap q[4], k[4], v[4], o[4];
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s: far beyond any legitimate wait
+
+// Bounded wait.  Returns false if the CTA is aborting (this or another thread's wait expired).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+                *abort_flag = 1;
+                atomicExch(status, (int)LOMA_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, "
+        "%7}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3,
+                                             int c4) {
+    asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];" ::"l"(
+                     reinterpret_cast<uint64_t>(map)),
+                 "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.u32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.u32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+// 16 consecutive 32-bit columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+
+__device__ __forceinline__ float fast_ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// ------------------------------------------------------------------ the kernel
+constexpr int TC_THREADS = 192;
+constexpr int TMEM_COLS = 512;
+
+template <int D>
+struct TcSmem {
+    static constexpr int PANELS = D / 64;
+    static constexpr int PANEL_BYTES = 128 * 128;           // 128 rows x 64 bf16
+    static constexpr int TILE_BYTES = PANELS * PANEL_BYTES; // one 128 x D tile
+    static constexpr int Q_OFF = 0;
+    static constexpr int K_OFF = TILE_BYTES;
+    static constexpr int V_OFF = 3 * TILE_BYTES;
+    static constexpr int O_OFF = 5 * TILE_BYTES;
+    static constexpr int TOTAL = 6 * TILE_BYTES;
+};
+
+template <int D>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
+    using SM = TcSmem<D>;
+    constexpr int PANELS = SM::PANELS;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bars[16];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // barrier ids
+    enum { B_QF = 0, B_QE = 1, B_KF = 2, B_KE = 4, B_VF = 6, B_VE = 8, B_SF = 10, B_PF = 12, B_PVF = 14 };
+    auto bar = [&](int i) { return smem_u32(&bars[i]); };
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(bar(B_QF), 1); mbar_init(bar(B_QE), 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar(B_KF + i), 1); mbar_init(bar(B_KE + i), 1);
+            mbar_init(bar(B_VF + i), 1); mbar_init(bar(B_VE + i), 1);
+            mbar_init(bar(B_SF + i), 1); mbar_init(bar(B_PF + i), 128);
+            mbar_init(bar(B_PVF + i), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // zero the operand buffers once: rows a TMA box does not cover keep finite contents
+    for (int i = threadIdx.x; i < SM::TOTAL / 16; i += TC_THREADS) reinterpret_cast<uint4*>(smem_gen)[i] = make_uint4(0, 0, 0, 0);
+    fence_async_smem();
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
+                     "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+    volatile int* abortp = &abort_flag;
+
+    const int total_work = p.total_tiles * p.BH;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t gs = 0, tcount = 0;
+            bool ok = true;
+            for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++tcount) {
+                const int rank = w / p.BH, bh = w - rank * p.BH;
+                const int bi = bh / p.H, hi = bh - bi * p.H;
+                TileDesc td;
+                decode_tile(p, rank, td);
+                const View& qv = p.view[td.view];
+                if (tcount > 0) ok = mbar_wait(bar(B_QE), (tcount - 1) & 1, abortp, p.status);
+                if (!ok) break;
+                mbar_expect_tx(bar(B_QF), qv.R * qv.CH * 128 * PANELS);
+                for (int pn = 0; pn < PANELS; ++pn)
+                    tma_load_5d(smem_base + SM::Q_OFF + pn * SM::PANEL_BYTES, &maps.q[td.view], bar(B_QF), pn * 64, td.r0,
+                                td.c0, hi, bi);
+                for (int j = 0; j < td.nsteps; ++j, ++gs) {
+                    KTile kt;
+                    step_ktile(p, td, j, kt);
+                    const View& kv = p.view[kt.view];
+                    const uint32_t b = gs & 1, ph = (gs >> 1) & 1;
+                    const uint32_t bytes = kv.R * kv.CH * 128 * PANELS;
+                    ok = mbar_wait(bar(B_KE + b), ph ^ 1, abortp, p.status);
+                    if (!ok) break;
+                    mbar_expect_tx(bar(B_KF + b), bytes);
+                    for (int pn = 0; pn < PANELS; ++pn)
+                        tma_load_5d(smem_base + SM::K_OFF + b * SM::TILE_BYTES + pn * SM::PANEL_BYTES, &maps.k[kt.view],
+                                    bar(B_KF + b), pn * 64, kt.r0, kt.c0, hi, bi);
+                    ok = mbar_wait(bar(B_VE + b), ph ^ 1, abortp, p.status);
+                    if (!ok) break;
+                    mbar_expect_tx(bar(B_VF + b), bytes);
+                    for (int pn = 0; pn < PANELS; ++pn)
+                        tma_load_5d(smem_base + SM::V_OFF + b * SM::TILE_BYTES + pn * SM::PANEL_BYTES, &maps.v[kt.view],
+                                    bar(B_VF + b), pn * 64, kt.r0, kt.c0, hi, bi);
+                }
+            }
+            if (!ok) {
+                // leaving early: give copies already in flight a bounded time to land in this CTA's shared memory
+                const long long t0 = clock64();
+                while (clock64() - t0 < 2000000ll) {}
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            // instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128
+            constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+            constexpr uint32_t IDESC_PV =
+                (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
+            uint32_t gs = 0, tcount = 0;
+            bool ok = true;
+            auto issue_s = [&](uint32_t g) -> bool {
+                const uint32_t b = g & 1, ph = (g >> 1) & 1;
+                if (!mbar_wait(bar(B_KF + b), ph, abortp, p.status)) return false;
+                tc_fence_after();
+                const uint32_t qa = smem_base + SM::Q_OFF, ka = smem_base + SM::K_OFF + b * SM::TILE_BYTES;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32;
+                    mma_ss(tmem + b * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), IDESC_S, kk > 0);
+                }
+                tc_commit(bar(B_SF + b));
+                tc_commit(bar(B_KE + b));
+                return true;
+            };
+            for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++tcount) {
+                const int rank = w / p.BH;
+                TileDesc td;
+                decode_tile(p, rank, td);
+                ok = mbar_wait(bar(B_QF), tcount & 1, abortp, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                ok = issue_s(gs);
+                for (int j = 0; j < td.nsteps && ok; ++j, ++gs) {
+                    const uint32_t b = gs & 1, ph = (gs >> 1) & 1;
+                    if (j + 1 < td.nsteps) { ok = issue_s(gs + 1); if (!ok) break; }
+                    else tc_commit(bar(B_QE));
+                    ok = mbar_wait(bar(B_PF + b), ph, abortp, p.status) && mbar_wait(bar(B_VF + b), ph, abortp, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t va = smem_base + SM::V_OFF + b * SM::TILE_BYTES;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)   // 16 keys per instruction
+                        mma_ts(tmem + 256 + b * 128, tmem + b * 128 + kk * 8,
+                               smem_desc(va + kk * 2048, SM::PANEL_BYTES, 1024), IDESC_PV, kk > 0);
+                    tc_commit(bar(B_PVF + b));
+                    tc_commit(bar(B_VE + b));
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ softmax + epilogue (128 threads)
+        const int rr = threadIdx.x;
+        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        uint32_t gs = 0;
+        bool ok = true;
+        bool store_pending = false;
+        for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+            const int rank = w / p.BH, bh = w - rank * p.BH;
+            const int bi = bh / p.H, hi = bh - bi * p.H;
+            TileDesc td;
+            decode_tile(p, rank, td);
+            const View& qv = p.view[td.view];
+            const int rsub = rr / qv.R;
+            const int ro = td.r0 + (rr - rsub * qv.R);
+            const int rc = td.a0 + rsub;
+            const bool row_valid = (rr < qv.R * qv.CH) && (rc <= td.a1) && (ro < qv.Z);
+
+            float m = -INFINITY, l = 0.f, alpha_prev = 0.f;
+            float o[D];
+#pragma unroll
+            for (int d = 0; d < D; ++d) o[d] = 0.f;
+
+            auto accumulate_pv = [&](uint32_t g, float alpha) -> bool {
+                const uint32_t b = g & 1, ph = (g >> 1) & 1;
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(B_PVF + b), ph, abortp, p.status))) return false;
+                tc_fence_after();
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(lane_addr + 256 + b * 128 + c * 32, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) o[c * 32 + e] = fmaf(o[c * 32 + e], alpha, __uint_as_float(r[e]));
+                }
+                return true;
+            };
+
+            for (int j = 0; j < td.nsteps; ++j, ++gs) {
+                const uint32_t b = gs & 1, ph = (gs >> 1) & 1;
+                KTile kt;
+                step_ktile(p, td, j, kt);
+                int lo, hi2;
+                row_interval(p.view[kt.view], kt, rc, ro, rr, row_valid, lo, hi2);
+                const bool full = __all_sync(0xffffffffu, lo <= 0 && hi2 >= 128);
+                const uint32_t span = (uint32_t)(hi2 - lo);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF + b), ph, abortp, p.status));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t s_addr = lane_addr + b * 128;
+                // pass 1: row maximum over the allowed columns
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(s_addr + c * 32, r);
+                    tmem_wait_ld();
+                    if (full) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) {
+                            const bool in = (uint32_t)(c * 32 + e - lo) < span;
+                            mx = fmaxf(mx, in ? __uint_as_float(r[e]) : -INFINITY);
+                        }
+                    }
+                }
+                const float m_new = fmaxf(m, mx * p.scale_log2);
+                const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
+                const float alpha = fast_ex2(m - m_safe);
+                // pass 2: probabilities (bf16, written over the scores) and row sum
+                float lsum = 0.f;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(s_addr + c * 32, r);
+                    tmem_wait_ld();
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        float s0 = __uint_as_float(r[e]), s1 = __uint_as_float(r[e + 1]);
+                        if (!full) {
+                            s0 = ((uint32_t)(c * 32 + e - lo) < span) ? s0 : -INFINITY;
+                            s1 = ((uint32_t)(c * 32 + e + 1 - lo) < span) ? s1 : -INFINITY;
+                        }
+                        const float p0 = fast_ex2(fmaf(s0, p.scale_log2, -m_safe));
+                        const float p1 = fast_ex2(fmaf(s1, p.scale_log2, -m_safe));
+                        lsum += p0 + p1;
+                        pk[e >> 1] = pack_bf16(p0, p1);
+                    }
+                    tmem_st16(s_addr + c * 16, pk);
+                }
+                l = fmaf(l, alpha, lsum);
+                m = m_new;
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(B_PF + b));
+                if (j > 0) { ok = accumulate_pv(gs - 1, alpha_prev); if (!ok) break; }
+                alpha_prev = alpha;
+            }
+            if (ok) ok = accumulate_pv(gs - 1, alpha_prev);
+
+            // epilogue: normalise, round to bf16, stage the tile in shared memory, TMA store.
+            // Every thread reaches this barrier for every tile it started; the barrier also
+            // makes the decision to give up uniform across the four warps.
+            if (threadIdx.x == 0 && store_pending) tma_store_wait_read();
+            {
+                uint32_t any_bad;
+                asm volatile(
+                    "{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, 1, 128, p;\nselp.u32 %0, 1, 0, q;\n}"
+                    : "=r"(any_bad)
+                    : "r"((uint32_t)(ok ? 0 : 1))
+                    : "memory");
+                if (any_bad) { ok = false; break; }
+            }
+            const float inv = 1.f / l;
+            uint8_t* orow = smem_gen + SM::O_OFF + rr * 128;
+#pragma unroll
+            for (int ci = 0; ci < D / 8; ++ci) {
+                uint4 u;
+                u.x = pack_bf16(o[ci * 8 + 0] * inv, o[ci * 8 + 1] * inv);
+                u.y = pack_bf16(o[ci * 8 + 2] * inv, o[ci * 8 + 3] * inv);
+                u.z = pack_bf16(o[ci * 8 + 4] * inv, o[ci * 8 + 5] * inv);
+                u.w = pack_bf16(o[ci * 8 + 6] * inv, o[ci * 8 + 7] * inv);
+                *reinterpret_cast<uint4*>(orow + (ci >> 3) * SM::PANEL_BYTES + (((ci & 7) ^ (rr & 7)) << 4)) = u;
+            }
+            if (p.lse && row_valid) {
+                const int64_t grow = (int64_t)rc * p.s + qv.zone_row0 + ro;
+                p.lse[(int64_t)bh * p.S + grow] = (m + log2f(l)) * 0.6931471805599453f;
+            }
+            fence_async_smem();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (threadIdx.x == 0) {
+                for (int pn = 0; pn < PANELS; ++pn)
+                    tma_store_5d(&maps.o[td.view], smem_base + SM::O_OFF + pn * SM::PANEL_BYTES, pn * 64, td.r0, td.c0, hi,
+                                 bi);
+                tma_store_commit();
+                store_pending = true;
+            }
+        }
+        if (threadIdx.x == 0 && store_pending) tma_store_wait_all();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(f);
+    });
+    return fn;
+}
+
+// 5-D map (d, row in zone, chunk, head, batch) over one zone view of one tensor.
+static bool encode_view(CUtensorMap* map, const void* base, const View& v, int D, int B, int H, int64_t row0,
+                        int64_t sb, int64_t sh, int64_t ss, int64_t chunk_stride_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const uint64_t es = 2;
+    cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)v.Z, (cuuint64_t)v.nch, (cuuint64_t)H, (cuuint64_t)B};
+    cuuint64_t chunk_stride = (v.nch > 1 ? (uint64_t)chunk_stride_rows : (uint64_t)v.Z) * ss * es;
+    cuuint64_t hstride = (uint64_t)(sh > 0 ? sh : ss * v.Z) * es;
+    cuuint64_t bstride = (uint64_t)(sb > 0 ? sb : ss * v.Z) * es;
+    cuuint64_t strides[4] = {(cuuint64_t)ss * es, chunk_stride, hstride, bstride};
+    cuuint32_t box[5] = {64, (cuuint32_t)v.R, (cuuint32_t)v.CH, 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    void* addr = const_cast<uint8_t*>(static_cast<const uint8_t*>(base)) + row0 * ss * es;
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, addr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct MapCacheKey {
+    const void *q, *k, *v, *o;
+    int B, H, D, n, c, t, tail;
+    int64_t sb, sh, ss;
+    bool operator==(const MapCacheKey& r) const {
+        return q == r.q && k == r.k && v == r.v && o == r.o && B == r.B && H == r.H && D == r.D && n == r.n && c == r.c &&
+               t == r.t && tail == r.tail && sb == r.sb && sh == r.sh && ss == r.ss;
+    }
+};
+
+// Returns cudaErrorNotSupported when the tensor-core path cannot take the call
+// (the caller then uses the CUDA-core kernel).
+cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int D,
+                                  const Layout& L, int64_t sb, int64_t sh, int64_t ss, float scale, cudaStream_t st) {
+    if (!encode_fn()) return cudaErrorNotSupported;
+    if (L.t > 256 * 128 || L.tc > (1 << 24)) return cudaErrorNotSupported;
+
+    FwdParams p{};
+    make_plan(L, B, H, &p);
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.lse = lse;
+    p.status = device_status_word();
+    if (!p.status) return cudaErrorUnknown;
+    if ((int64_t)p.total_tiles * p.BH > 0x7fffffffll) return cudaErrorNotSupported;
+
+    // tensor maps, cached for repeated calls on the same tensors
+    static std::mutex mu;
+    static MapCacheKey cached_key{};
+    static TmaMaps cached_maps;
+    static bool have_cache = false;
+    TmaMaps maps;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        MapCacheKey key{q, k, v, o, B, H, D, L.n_chunks, L.c, L.t, L.tail_read, sb, sh, ss};
+        if (!(have_cache && key == cached_key)) {
+            TmaMaps mnew{};
+            const void* bases[4] = {q, k, v, o};
+            CUtensorMap* arrs[4] = {mnew.q, mnew.k, mnew.v, mnew.o};
+            for (int ti = 0; ti < 4; ++ti) {
+                for (int vi = 0; vi < 4; ++vi) {
+                    const View& vw = p.view[vi];
+                    if (vw.ntiles == 0) continue;
+                    const int64_t row0 = (vi == V_TAIL) ? (int64_t)L.n_chunks * L.s : vw.zone_row0;
+                    if (!encode_view(&arrs[ti][vi], bases[ti], vw, D, B, H, row0, sb, sh, ss, L.s))
+                        return cudaErrorNotSupported;
+                }
+            }
+            cached_maps = mnew;
+            cached_key = key;
+            have_cache = true;
+        }
+        maps = cached_maps;
+    }
+
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int64_t work = (int64_t)p.total_tiles * p.BH;
+    const int grid = (int)(work < sms ? work : sms);
+    cudaError_t e;
+    if (D == 128) {
+        const int smem = TcSmem<128>::TOTAL + 1024;
+        e = cudaFuncSetAttribute(masked_attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        masked_attn_tc_kernel<128><<<grid, TC_THREADS, smem, st>>>(maps, p);
+    } else {
+        // the shared-memory footprint also keeps one CTA per SM (each allocates all 512 TMEM columns)
+        const int smem = 120 * 1024;
+        e = cudaFuncSetAttribute(masked_attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        masked_attn_tc_kernel<64><<<grid, TC_THREADS, smem, st>>>(maps, p);
+    }
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+}  // namespace loma

@@ -140,9 +140,22 @@ int loma_masked_attn_fwd(const void* q, const void* k, const void* v, void* o, f
     if (dc != LOMA_OK) return dc;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = launch_masked_attn_generic(q, k, v, o, lse, B, H, D, L, stride_b, stride_h, stride_s, dtype,
-                                               scale, st);
+    cudaError_t e = cudaErrorNotSupported;
+    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC))
+        e = launch_masked_attn_tc(q, k, v, o, lse, B, H, D, L, stride_b, stride_h, stride_s, scale, st);
+    if (e == cudaErrorNotSupported)
+        e = launch_masked_attn_generic(q, k, v, o, lse, B, H, D, L, stride_b, stride_h, stride_s, dtype, scale, st);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
+int loma_masked_attn_plan_coverage(int n_chunks, int c, int t, int tail_read, unsigned flags, uint8_t* counts) {
+    Layout L;
+    const int rc = make_layout(n_chunks, c, t, tail_read, flags, &L);
+    if (rc != LOMA_OK) return rc;
+    if (L.S > 0 && !counts) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)L.S * L.S > (1ll << 32)) return LOMA_ERR_INVALID_ARG;
+    if (L.S > 0) plan_coverage_host(L, counts);
+    return LOMA_OK;
 }
 
 size_t loma_decode_workspace_bytes(int B, int H, int D, int cache_len) {

@@ -33,6 +33,12 @@ cudaError_t launch_masked_attn_generic(const void* q, const void* k, const void*
                                        int64_t sb, int64_t sh, int64_t ss,
                                        loma_dtype dt, float scale, cudaStream_t st);
 
+// tcgen05 / TMEM / TMA masked forward (attn_tcgen05.cu); cudaErrorNotSupported = use the generic kernel
+cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int D,
+                                  const Layout& L, int64_t sb, int64_t sh, int64_t ss, float scale, cudaStream_t st);
+
+void plan_coverage_host(const Layout& L, uint8_t* counts);   // tile_plan_host.cu
+
 cudaError_t launch_decode_generic(const void* q, const void* k_new, const void* v_new,
                                   void* k_cache, void* v_cache, void* o, float* lse,
                                   int B, int H, int D, int cap, int cache_len,

@@ -1,0 +1,147 @@
+// Tile plan of the tensor-core masked forward: how the laid-out sequence is cut
+// into 128-row tiles of the four zone views, which key tiles each query tile
+// visits, and which columns of a visited tile a row may attend to (Eq. 1-3).
+// Plain integer logic shared by the kernel (device) and by the host-side
+// reconstruction of the mask that the tests compare with the oracle's.
+#pragma once
+
+#include "loma_internal.cuh"
+
+namespace loma {
+
+__host__ __device__ __forceinline__ int plan_min(int a, int b) { return a < b ? a : b; }
+__host__ __device__ __forceinline__ int plan_max(int a, int b) { return a > b ? a : b; }
+
+enum { V_READ = 0, V_MEM = 1, V_REP = 2, V_TAIL = 3 };
+enum { M_LT = 0, M_LE = 1, M_EQ = 2, M_CAUSAL = 3, M_DIAG = 4 };
+
+struct View {
+    int Z;           // zone length (rows per chunk in this view)
+    int R;           // rows of one chunk inside a tile: min(Z, 128)
+    int CH;          // chunks per tile: 1 if Z >= 128 else 128 / Z
+    int tpc;         // tiles per chunk (Z >= 128) else 0
+    int ntiles;      // tiles in the view
+    int nch;         // chunks in the view
+    int chunk_base;  // absolute chunk number of the view's chunk 0 (n_chunks for the tail)
+    int zone_row0;   // first row of the zone inside its chunk
+};
+
+struct FwdParams {
+    View view[4];
+    int n_chunks, s, S, H, BH;
+    int total_tiles;
+    int n_tail, n_read, n_mem, n_rep;   // tiles per view, in scheduling order
+    unsigned flags;
+    float scale_log2;
+    float* lse;
+    int* status;
+};
+
+
+struct Seg {
+    int view, mode, first, count;
+};
+struct TileDesc {
+    int view, qi, c0, r0;   // view, tile index, first chunk (view-relative), first row in zone
+    int a0, a1;             // absolute first / last chunk covered
+    Seg seg[2];
+    int nsteps;
+};
+struct KTile {
+    int view, mode, c0, r0, a0;   // view-relative chunk, first row, absolute chunk
+};
+
+// ------------------------------------------------------------------ tile lists
+__host__ __device__ __forceinline__ int tile_of_chunk(const View& v, int c) { return v.Z >= 128 ? c * v.tpc : c / v.CH; }
+__host__ __device__ __forceinline__ int tiles_covering(const View& v, int nchunks) {
+    return v.Z >= 128 ? nchunks * v.tpc : (nchunks + v.CH - 1) / v.CH;
+}
+
+__host__ __device__ __forceinline__ void decode_tile(const FwdParams& p, int rank, TileDesc& td) {
+    int view, qi;
+    if (rank < p.n_tail) { view = V_TAIL; qi = p.n_tail - 1 - rank; }
+    else if ((rank -= p.n_tail) < p.n_read) { view = V_READ; qi = p.n_read - 1 - rank; }
+    else if ((rank -= p.n_read) < p.n_mem) { view = V_MEM; qi = p.n_mem - 1 - rank; }
+    else { view = V_REP; qi = rank - p.n_mem; }
+    const View& g = p.view[view];
+    td.view = view; td.qi = qi;
+    int c1;
+    if (g.Z >= 128) { td.c0 = qi / g.tpc; td.r0 = (qi - td.c0 * g.tpc) * 128; c1 = td.c0; }
+    else { td.c0 = qi * g.CH; td.r0 = 0; c1 = plan_min(td.c0 + g.CH, g.nch) - 1; }
+    td.a0 = g.chunk_base + td.c0;
+    td.a1 = g.chunk_base + c1;
+    const View& vm = p.view[V_MEM];
+    const View& vr = p.view[V_READ];
+    const int sub = (g.Z >= 128) ? qi - td.c0 * g.tpc : 0;   // tile index inside its chunk
+    if (view == V_READ || view == V_TAIL) {
+        // memory zones of every earlier chunk, then the own reading zone up to this tile
+        td.seg[0] = Seg{V_MEM, M_LT, 0, tiles_covering(vm, td.a1)};
+        td.seg[1] = Seg{view, M_CAUSAL, (g.Z >= 128) ? td.c0 * g.tpc : qi, sub + 1};
+    } else if (view == V_MEM) {
+        if (p.flags & LOMA_FLAG_MEM_SEES_PRIOR_MEM)
+            td.seg[0] = Seg{V_MEM, M_LE, 0, (g.Z >= 128) ? (td.a0 + 1) * g.tpc : qi + 1};
+        else
+            td.seg[0] = Seg{V_MEM, M_EQ, (g.Z >= 128) ? td.c0 * g.tpc : qi, (g.Z >= 128) ? g.tpc : 1};
+        const int f = tile_of_chunk(vr, td.a0);
+        td.seg[1] = Seg{V_READ, M_EQ, f, (vr.Z >= 128) ? (td.a1 - td.a0 + 1) * vr.tpc : tile_of_chunk(vr, td.a1) - f + 1};
+    } else {
+        const int f = tile_of_chunk(vm, td.a0);
+        td.seg[0] = Seg{V_MEM, M_EQ, f, (vm.Z >= 128) ? (td.a1 - td.a0 + 1) * vm.tpc : tile_of_chunk(vm, td.a1) - f + 1};
+        td.seg[1] = Seg{V_REP, M_DIAG, qi, 1};
+    }
+    td.nsteps = td.seg[0].count + td.seg[1].count;
+}
+
+__host__ __device__ __forceinline__ void step_ktile(const FwdParams& p, const TileDesc& td, int j, KTile& kt) {
+    const Seg& sg = (j < td.seg[0].count) ? td.seg[0] : td.seg[1];
+    const int t = sg.first + ((j < td.seg[0].count) ? j : j - td.seg[0].count);
+    const View& g = p.view[sg.view];
+    kt.view = sg.view; kt.mode = sg.mode;
+    if (g.Z >= 128) { kt.c0 = t / g.tpc; kt.r0 = (t - kt.c0 * g.tpc) * 128; }
+    else { kt.c0 = t * g.CH; kt.r0 = 0; }
+    kt.a0 = g.chunk_base + kt.c0;
+}
+
+// Allowed columns [lo, hi) of a key tile for a row at (chunk rc, offset ro), tile-local row rr.
+__host__ __device__ __forceinline__ void row_interval(const View& kv, const KTile& kt, int rc, int ro, int rr, bool row_valid,
+                                             int& lo, int& hi) {
+    const int vcols = plan_min(kv.R, kv.Z - kt.r0);   // valid columns per chunk of this tile
+    const int d = rc - kt.a0;
+    lo = 0; hi = 0;
+    if (kt.mode == M_LT || kt.mode == M_LE) {
+        const int nch = plan_min(plan_max(d + (kt.mode == M_LE ? 1 : 0), 0), kv.CH);
+        hi = nch > 0 ? (nch - 1) * kv.R + vcols : 0;
+    } else if (kt.mode == M_DIAG) {
+        lo = rr; hi = rr + 1;
+    } else if (d >= 0 && d < kv.CH) {
+        lo = d * kv.R;
+        hi = lo + (kt.mode == M_EQ ? vcols : plan_min(plan_max(ro - kt.r0 + 1, 0), vcols));
+    }
+    if (!row_valid) { lo = 0; hi = 0; }
+}
+
+// Fills the geometry part of FwdParams (views, tile counts) from the layout.
+inline View make_view(int Z, int nch, int chunk_base, int zone_row0) {
+    View v{};
+    v.Z = Z; v.nch = nch; v.chunk_base = chunk_base; v.zone_row0 = zone_row0;
+    if (Z <= 0 || nch <= 0) { v.R = 1; v.CH = 1; v.tpc = 0; v.ntiles = 0; v.Z = (Z > 0 ? Z : 1); v.nch = 0; return v; }
+    v.R = Z < 128 ? Z : 128;
+    v.CH = Z >= 128 ? 1 : 128 / Z;
+    v.tpc = Z >= 128 ? (Z + 127) / 128 : 0;
+    v.ntiles = Z >= 128 ? nch * v.tpc : (nch + v.CH - 1) / v.CH;
+    return v;
+}
+
+inline void make_plan(const Layout& L, int B, int H, FwdParams* p) {
+    p->view[V_READ] = make_view(L.tc, L.n_chunks, 0, 0);
+    p->view[V_MEM] = make_view(L.t, L.n_chunks, 0, L.tc);
+    p->view[V_REP] = make_view(L.tc, L.n_chunks, 0, L.tc + L.t);
+    p->view[V_TAIL] = make_view(L.tail_read, L.tail_read > 0 ? 1 : 0, L.n_chunks, 0);
+    p->n_chunks = L.n_chunks; p->s = L.s; p->S = L.S; p->H = H; p->BH = B * H;
+    p->n_tail = p->view[V_TAIL].ntiles; p->n_read = p->view[V_READ].ntiles;
+    p->n_mem = p->view[V_MEM].ntiles; p->n_rep = p->view[V_REP].ntiles;
+    p->total_tiles = p->n_tail + p->n_read + p->n_mem + p->n_rep;
+    p->flags = L.flags;
+}
+
+}  // namespace loma

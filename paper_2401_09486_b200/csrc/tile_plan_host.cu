@@ -1,0 +1,47 @@
+// Host-side replay of the tensor-core kernel's tile plan.
+#include <string.h>
+
+#include "tile_plan.cuh"
+
+namespace loma {
+
+// counts[i*S + j] = number of (query tile, key tile) visits in which row i
+// attends to column j.  A correct plan gives exactly the 0/1 mask of Eq. 2.
+void plan_coverage_host(const Layout& L, uint8_t* counts) {
+    FwdParams p{};
+    make_plan(L, 1, 1, &p);
+    memset(counts, 0, (size_t)L.S * L.S);
+    for (int rank = 0; rank < p.total_tiles; ++rank) {
+        TileDesc td;
+        decode_tile(p, rank, td);
+        const View& qv = p.view[td.view];
+        for (int j = 0; j < td.nsteps; ++j) {
+            KTile kt;
+            step_ktile(p, td, j, kt);
+            const View& kv = p.view[kt.view];
+            for (int rr = 0; rr < 128; ++rr) {
+                const int rsub = rr / qv.R;
+                const int ro = td.r0 + (rr - rsub * qv.R);
+                const int rc = td.a0 + rsub;
+                const bool row_valid = (rr < qv.R * qv.CH) && (rc <= td.a1) && (ro < qv.Z);
+                int lo, hi;
+                row_interval(kv, kt, rc, ro, rr, row_valid, lo, hi);
+                if (!row_valid || hi <= lo) continue;
+                const int64_t grow = (int64_t)rc * L.s + qv.zone_row0 + ro;
+                for (int col = lo; col < hi; ++col) {
+                    // column of the key tile -> row of the laid-out sequence, the way the TMA box gathers it
+                    const int ksub = col / kv.R;
+                    const int ko = kt.r0 + (col - ksub * kv.R);
+                    const int kc = kt.a0 + ksub;
+                    const int64_t gcol = (int64_t)kc * L.s + kv.zone_row0 + ko;
+                    if (grow < L.S && gcol >= 0 && gcol < L.S) {
+                        uint8_t& c = counts[grow * L.S + gcol];
+                        if (c < 255) ++c;
+                    }
+                }
+            }
+        }
+    }
+}
+
+}  // namespace loma

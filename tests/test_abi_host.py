@@ -131,3 +131,19 @@ def test_compress_validation(lib):
     assert call(vm=None) == INVALID
     assert call(vc=0x5002) == ALIGNMENT
     assert call(H=0) == 0
+
+
+PLAN_GEOMS = [(3, 2, 2, 0), (2, 4, 4, 3), (5, 4, 16, 37), (9, 4, 16, 0), (3, 8, 16, 0), (3, 8, 16, 100), (3, 8, 32, 200),
+              (2, 8, 32, 256), (4, 1, 5, 2), (2, 3, 7, 0), (0, 4, 0, 301), (0, 1, 0, 128), (1, 2, 64, 0), (9, 2, 8, 16),
+              (2, 1, 128, 5), (2, 2, 130, 17), (2, 3, 100, 300), (3, 1, 1, 1), (17, 2, 8, 0), (2, 1, 200, 0)]
+
+
+@pytest.mark.parametrize("n,c,t,tail", PLAN_GEOMS)
+@pytest.mark.parametrize("flags", [0, 1])
+def test_tensor_core_tile_plan_reproduces_the_mask_exactly(lib, n, c, t, tail, flags):
+    """Every allowed (row, key) pair of Eq. 2 is visited exactly once by the
+    tensor-core kernel's tile plan, and no blocked pair is visited at all."""
+    got = binding.loma_masked_attn_plan_coverage(n, c, t, tail, flags).numpy()
+    want = oracle.dense_mask(n, c, t, tail, flags).astype(np.uint8)
+    assert got.shape == want.shape
+    assert np.array_equal(got, want), f"{int((got != want).sum())} entries differ"
