@@ -1,0 +1,369 @@
+// Compress step for bf16: the t <m> queries of one (batch, head) over the
+// uncompressed tail and their own keys (Section 3.1 step 2, all-ones mask of
+// Appendix A), fused with the in-place compaction of the cache (step 3).
+//
+// With t = 16 query rows per key row the step has ~16 flop per byte: it is bound
+// by HBM (or, for the short default variant, by launch latency), but too heavy
+// for the CUDA cores when the prior-memory variant streams the whole cache.  The
+// 16 queries are exactly one M = 16 tile of the warp-level tensor-core
+// instruction (mma.sync.m16n8k16); the 128-row tcgen05 tile would idle 7/8 of
+// the array here, so this kernel uses the warp-level path on purpose.
+//
+//   CTA (4 warps) = one key range of one (b,h).  The last range of a (b,h) is
+//   always [tail (tc rows) ; k_mem (t rows)]; with the prior-memory flag the
+//   earlier ranges cut cache[0, mem_len) into pieces.
+//   K and V rows are staged 64 at a time in shared memory with 16-byte
+//   cp.async copies (double buffered), padded rows so ldmatrix is conflict free.
+//   Each warp takes 16 of the 64 staged keys: S = Q K^T (16 x 16), online
+//   softmax in registers, O += P V with P straight from the accumulator
+//   registers.  Warps are merged in shared memory; ranges through the workspace
+//   and a small merge kernel (fixed order: bitwise repeatable).
+//   Compaction: the CTA that owns the tail is the only reader of the slots
+//   [mem_len, mem_len + t) in this launch; after a block barrier it overwrites
+//   them with k_mem / v_mem using 16-byte vector stores.
+#include <math.h>
+
+#include "loma_internal.cuh"
+
+namespace loma {
+
+constexpr int CMP_WARPS = 4;
+constexpr int CMP_CHUNK = 64;          // keys staged per pipeline stage
+constexpr int CMP_PRIOR_LEN = 1024;    // keys per prior-memory range (when there are many (b,h))
+
+int compress_num_prior(int BH, int mem_len, unsigned flags) {
+    if (!(flags & LOMA_FLAG_MEM_SEES_PRIOR_MEM) || mem_len <= 0) return 0;
+    int by_len = (mem_len + CMP_PRIOR_LEN - 1) / CMP_PRIOR_LEN;
+    int by_fill = (4 * 148 + BH - 1) / BH - 1;
+    int n = by_len > by_fill ? by_len : by_fill;
+    int cap = (mem_len + 255) / 256;
+    if (n > cap) n = cap;
+    if (n > 255) n = 255;
+    if (n < 1) n = 1;
+    return n;
+}
+
+size_t compress_workspace_bytes(int BH, int D, int t, int mem_len, unsigned flags) {
+    if (t > 16) return 0;   // handled by the CUDA-core kernel, which needs none
+    const int np = compress_num_prior(BH, mem_len, flags);
+    if (np == 0) return 0;
+    return (size_t)BH * (np + 1) * 16 * (D + 2) * sizeof(float);
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+    const int sz = valid ? 16 : 0;   // 0 source bytes = zero fill
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2f(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+template <int D>
+struct CmpSmem {
+    static constexpr int ROWB = D * 2 + 16;                  // padded row: conflict-free ldmatrix
+    static constexpr int STAGE = 2 * CMP_CHUNK * ROWB;       // K then V
+    static constexpr int Q_OFF = 2 * STAGE;
+    static constexpr int TOTAL = Q_OFF + 16 * ROWB;
+    static constexpr int MERGE_BYTES = CMP_WARPS * 16 * (D + 2) * 4;   // reuses the stages
+    static_assert(MERGE_BYTES <= 2 * STAGE, "merge buffer must fit in the stage buffers");
+};
+
+template <int D>
+__global__ void __launch_bounds__(CMP_WARPS * 32)
+compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16* __restrict__ k_mem,
+                    const __nv_bfloat16* __restrict__ v_mem, __nv_bfloat16* __restrict__ k_cache,
+                    __nv_bfloat16* __restrict__ v_cache, __nv_bfloat16* __restrict__ o_mem, float* __restrict__ lse,
+                    float* __restrict__ ws, int BH, int cap, int mem_len, int t, int tc, int nprior, int prior_len,
+                    float scale_log2) {
+    using SM = CmpSmem<D>;
+    constexpr int ROWB = SM::ROWB;
+    constexpr int VPR = D / 8;                 // 16-byte vectors per row
+    extern __shared__ __align__(16) uint8_t smem[];
+    const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(smem);
+    const int nsp = nprior + 1;
+    const int bh = blockIdx.x / nsp, split = blockIdx.x - bh * nsp;
+    const bool is_tail = split == nprior;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;
+
+    const __nv_bfloat16* kc = k_cache + (int64_t)bh * cap * D;
+    const __nv_bfloat16* vc = v_cache + (int64_t)bh * cap * D;
+    const __nv_bfloat16* km = k_mem + (int64_t)bh * t * D;
+    const __nv_bfloat16* vm = v_mem + (int64_t)bh * t * D;
+    // key i of this CTA's range -> source row
+    const int k0 = is_tail ? mem_len : split * prior_len;
+    const int n_cache_rows = is_tail ? tc : min(prior_len, mem_len - k0);
+    const int nkeys = is_tail ? tc + t : n_cache_rows;
+
+    auto stage_chunk = [&](int ci, int st) {
+        const uint32_t kdst = sbase + st * SM::STAGE, vdst = kdst + CMP_CHUNK * ROWB;
+        for (int e = threadIdx.x; e < CMP_CHUNK * VPR; e += CMP_WARPS * 32) {
+            const int r = e / VPR, cv = e - r * VPR;
+            const int i = ci * CMP_CHUNK + r;
+            const bool valid = i < nkeys;
+            const int ic = valid ? i : 0;
+            const __nv_bfloat16 *ksrc, *vsrc;
+            if (ic < n_cache_rows) { ksrc = kc + (int64_t)(k0 + ic) * D; vsrc = vc + (int64_t)(k0 + ic) * D; }
+            else { ksrc = km + (int64_t)(ic - n_cache_rows) * D; vsrc = vm + (int64_t)(ic - n_cache_rows) * D; }
+            cp_async16(kdst + r * ROWB + cv * 16, ksrc + cv * 8, valid);
+            cp_async16(vdst + r * ROWB + cv * 16, vsrc + cv * 8, valid);
+        }
+    };
+
+    const int nchunks = (nkeys + CMP_CHUNK - 1) / CMP_CHUNK;
+    if (nchunks > 0) stage_chunk(0, 0);
+    cp_async_commit();
+
+    // queries: 16 rows (rows >= t are zero), staged once, then kept as A fragments
+    for (int e = threadIdx.x; e < 16 * VPR; e += CMP_WARPS * 32) {
+        const int r = e / VPR, cv = e - r * VPR;
+        uint4 val = make_uint4(0, 0, 0, 0);
+        if (r < t) val = __ldg(reinterpret_cast<const uint4*>(q_mem + ((int64_t)bh * t + r) * D) + cv);
+        *reinterpret_cast<uint4*>(smem + SM::Q_OFF + r * ROWB + cv * 16) = val;
+    }
+    __syncthreads();
+    uint32_t qa[D / 16][4];
+    {
+        const int mi = lane >> 3;
+        const uint32_t row_addr = sbase + SM::Q_OFF + ((mi & 1) * 8 + (lane & 7)) * ROWB + (mi >> 1) * 16;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) ldsm_x4(row_addr + kk * 32, qa[kk]);
+    }
+
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // rows g and g+8
+    float oacc[D / 8][4];
+#pragma unroll
+    for (int j = 0; j < D / 8; ++j) { oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f; }
+
+    for (int ci = 0; ci < nchunks; ++ci) {
+        if (ci + 1 < nchunks) stage_chunk(ci + 1, (ci + 1) & 1);
+        cp_async_commit();
+        cp_async_wait<1>();
+        __syncthreads();
+        const int kb = ci * CMP_CHUNK + warp * 16;        // this warp's 16 keys
+        if (kb < nkeys) {
+            const uint32_t kst = sbase + (ci & 1) * SM::STAGE + warp * 16 * ROWB;
+            const uint32_t vst = kst + CMP_CHUNK * ROWB;
+            float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+            {
+                const int mi = lane >> 3;
+                const uint32_t addr = kst + ((mi >> 1) * 8 + (lane & 7)) * ROWB + (mi & 1) * 16;
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    uint32_t kf[4];
+                    ldsm_x4(addr + kk * 32, kf);
+                    mma_bf16_16816(sc[0], qa[kk], kf[0], kf[1]);
+                    mma_bf16_16816(sc[1], qa[kk], kf[2], kf[3]);
+                }
+            }
+            // mask keys beyond the range, then online softmax (exp2 domain)
+            float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const bool valid = kb + 8 * j + 2 * tq + e < nkeys;
+                    sc[j][e] = valid ? sc[j][e] * scale_log2 : -INFINITY;
+                    sc[j][2 + e] = valid ? sc[j][2 + e] * scale_log2 : -INFINITY;
+                    mx0 = fmaxf(mx0, sc[j][e]);
+                    mx1 = fmaxf(mx1, sc[j][2 + e]);
+                }
+            }
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+            const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);   // finite: key kb is valid for every row
+            const float a0 = ex2f(m0 - mn0), a1 = ex2f(m1 - mn1);
+            m0 = mn0; m1 = mn1;
+            uint32_t pa[4];
+            {
+                const float p00 = ex2f(sc[0][0] - mn0), p01 = ex2f(sc[0][1] - mn0);
+                const float p02 = ex2f(sc[0][2] - mn1), p03 = ex2f(sc[0][3] - mn1);
+                const float p10 = ex2f(sc[1][0] - mn0), p11 = ex2f(sc[1][1] - mn0);
+                const float p12 = ex2f(sc[1][2] - mn1), p13 = ex2f(sc[1][3] - mn1);
+                l0 = l0 * a0 + (p00 + p01) + (p10 + p11);
+                l1 = l1 * a1 + (p02 + p03) + (p12 + p13);
+                pa[0] = pack_bf16(p00, p01);   // (row g,   keys 2t, 2t+1)
+                pa[1] = pack_bf16(p02, p03);   // (row g+8, keys 2t, 2t+1)
+                pa[2] = pack_bf16(p10, p11);   // (row g,   keys 8+2t, ..)
+                pa[3] = pack_bf16(p12, p13);   // (row g+8, keys 8+2t, ..)
+            }
+#pragma unroll
+            for (int j = 0; j < D / 8; ++j) {
+                oacc[j][0] *= a0; oacc[j][1] *= a0; oacc[j][2] *= a1; oacc[j][3] *= a1;
+            }
+            {
+                const int mi = lane >> 3;
+                const uint32_t addr = vst + ((mi & 1) * 8 + (lane & 7)) * ROWB + (mi >> 1) * 16;
+#pragma unroll
+                for (int jd = 0; jd < D / 8; jd += 2) {
+                    uint32_t vf[4];
+                    ldsm_x4_trans(addr + jd * 16, vf);
+                    mma_bf16_16816(oacc[jd], pa, vf[0], vf[1]);
+                    mma_bf16_16816(oacc[jd + 1], pa, vf[2], vf[3]);
+                }
+            }
+        }
+        __syncthreads();   // the stage is refilled two iterations later
+    }
+    cp_async_wait<0>();
+    // row sums live in the four lanes of a quad
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+
+    // merge the warps through shared memory (stage buffers are free now)
+    float* mg_o = reinterpret_cast<float*>(smem);                          // [warp][16][D]
+    float* mg_ml = mg_o + CMP_WARPS * 16 * D;                              // [warp][16][2]
+#pragma unroll
+    for (int j = 0; j < D / 8; ++j) {
+        float* r0 = mg_o + ((warp * 16 + g) * D) + 8 * j + 2 * tq;
+        float* r1 = mg_o + ((warp * 16 + g + 8) * D) + 8 * j + 2 * tq;
+        r0[0] = oacc[j][0]; r0[1] = oacc[j][1];
+        r1[0] = oacc[j][2]; r1[1] = oacc[j][3];
+    }
+    if (tq == 0) {
+        mg_ml[(warp * 16 + g) * 2] = m0; mg_ml[(warp * 16 + g) * 2 + 1] = l0;
+        mg_ml[(warp * 16 + g + 8) * 2] = m1; mg_ml[(warp * 16 + g + 8) * 2 + 1] = l1;
+    }
+    __syncthreads();
+    {
+        constexpr int SEG = D / 8;               // 8 threads per row, SEG columns each
+        const int r = threadIdx.x >> 3, d0 = (threadIdx.x & 7) * SEG;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < CMP_WARPS; ++w) M = fmaxf(M, mg_ml[(w * 16 + r) * 2]);
+        float f[CMP_WARPS], lt = 0.f;
+#pragma unroll
+        for (int w = 0; w < CMP_WARPS; ++w) {
+            const float mw = mg_ml[(w * 16 + r) * 2];
+            f[w] = (mw > -INFINITY) ? ex2f(mw - M) : 0.f;
+            lt = fmaf(mg_ml[(w * 16 + r) * 2 + 1], f[w], lt);
+        }
+        if (r < t) {
+            if (nsp == 1) {
+                const float inv = 1.f / lt;
+                __nv_bfloat16* dst = o_mem + ((int64_t)bh * t + r) * D + d0;
+#pragma unroll
+                for (int d = 0; d < SEG; d += 2) {
+                    float x0 = 0.f, x1 = 0.f;
+#pragma unroll
+                    for (int w = 0; w < CMP_WARPS; ++w) {
+                        x0 = fmaf(mg_o[(w * 16 + r) * D + d0 + d], f[w], x0);
+                        x1 = fmaf(mg_o[(w * 16 + r) * D + d0 + d + 1], f[w], x1);
+                    }
+                    *reinterpret_cast<uint32_t*>(dst + d) = pack_bf16(x0 * inv, x1 * inv);
+                }
+                if (lse && d0 == 0) lse[(int64_t)bh * t + r] = (M + log2f(lt)) * 0.6931471805599453f;
+            } else {
+                float* po = ws + (((int64_t)bh * nsp + split) * 16 + r) * D + d0;
+#pragma unroll
+                for (int d = 0; d < SEG; ++d) {
+                    float x = 0.f;
+#pragma unroll
+                    for (int w = 0; w < CMP_WARPS; ++w) x = fmaf(mg_o[(w * 16 + r) * D + d0 + d], f[w], x);
+                    po[d] = x;
+                }
+                if (d0 == 0) {
+                    float* pml = ws + (int64_t)BH * nsp * 16 * D + (((int64_t)bh * nsp + split) * 16 + r) * 2;
+                    pml[0] = M; pml[1] = lt;
+                }
+            }
+        }
+    }
+    // compaction (Section 3.1 step 3): every read of the tail by this launch happened in this CTA, above
+    if (is_tail) {
+        __syncthreads();
+        const uint4* ksrc = reinterpret_cast<const uint4*>(km);
+        const uint4* vsrc = reinterpret_cast<const uint4*>(vm);
+        uint4* kdst = reinterpret_cast<uint4*>(k_cache + ((int64_t)bh * cap + mem_len) * D);
+        uint4* vdst = reinterpret_cast<uint4*>(v_cache + ((int64_t)bh * cap + mem_len) * D);
+        for (int e = threadIdx.x; e < t * VPR; e += CMP_WARPS * 32) {
+            kdst[e] = __ldg(ksrc + e);
+            vdst[e] = __ldg(vsrc + e);
+        }
+    }
+}
+
+template <int D>
+__global__ void __launch_bounds__(D)
+compress_merge_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ o_mem, float* __restrict__ lse,
+                      int BH, int t, int nsp) {
+    const int bh = blockIdx.x / t, r = blockIdx.x - bh * t, d = threadIdx.x;
+    const float* pml = ws + (int64_t)BH * nsp * 16 * D;
+    float M = -INFINITY;
+    for (int s = 0; s < nsp; ++s) M = fmaxf(M, pml[(((int64_t)bh * nsp + s) * 16 + r) * 2]);
+    float lt = 0.f, ot = 0.f;
+    for (int s = 0; s < nsp; ++s) {
+        const float ms = pml[(((int64_t)bh * nsp + s) * 16 + r) * 2];
+        if (ms > -INFINITY) {
+            const float f = exp2f(ms - M);
+            lt = fmaf(pml[(((int64_t)bh * nsp + s) * 16 + r) * 2 + 1], f, lt);
+            ot = fmaf(ws[(((int64_t)bh * nsp + s) * 16 + r) * D + d], f, ot);
+        }
+    }
+    o_mem[((int64_t)bh * t + r) * D + d] = __float2bfloat16_rn(ot / lt);
+    if (lse && d == 0) lse[(int64_t)bh * t + r] = (M + log2f(lt)) * 0.6931471805599453f;
+}
+
+template <int D>
+static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* vm, void* kc, void* vc, void* om,
+                                   float* lse, int BH, int cap, int mem_len, int t, int tc, unsigned flags, float scale,
+                                   void* ws, cudaStream_t st) {
+    const int nprior = compress_num_prior(BH, mem_len, flags);
+    int prior_len = 0;
+    if (nprior > 0) prior_len = ((mem_len + nprior - 1) / nprior + 15) / 16 * 16;
+    const int nsp = nprior + 1;
+    const int smem = CmpSmem<D>::TOTAL;
+    cudaError_t e = cudaFuncSetAttribute(compress_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    compress_mma_kernel<D><<<BH * nsp, CMP_WARPS * 32, smem, st>>>(
+        static_cast<const __nv_bfloat16*>(qm), static_cast<const __nv_bfloat16*>(km),
+        static_cast<const __nv_bfloat16*>(vm), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
+        static_cast<__nv_bfloat16*>(om), lse, static_cast<float*>(ws), BH, cap, mem_len, t, tc, nprior, prior_len,
+        scale * 1.4426950408889634f);
+    count_launches(1);
+    e = cudaGetLastError();
+    if (e != cudaSuccess || nsp == 1) return e;
+    compress_merge_kernel<D><<<BH * t, D, 0, st>>>(static_cast<const float*>(ws), static_cast<__nv_bfloat16*>(om), lse,
+                                                   BH, t, nsp);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+// t <= 16 only; the caller falls back to the CUDA-core kernel otherwise.
+cudaError_t launch_compress_bf16(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
+                                 void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len, int c, int t,
+                                 unsigned flags, float scale, void* ws, cudaStream_t st) {
+    const int BH = B * H, tc = c * t;
+    return D == 64 ? compress_bf16_t<64>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH, cap, mem_len, t, tc,
+                                         flags, scale, ws, st)
+                   : compress_bf16_t<128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH, cap, mem_len, t, tc,
+                                          flags, scale, ws, st);
+}
+
+}  // namespace loma

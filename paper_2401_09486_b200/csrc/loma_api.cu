@@ -221,8 +221,8 @@ int loma_decode_attn_static(const void* q, const void* k_new, const void* v_new,
 }
 
 size_t loma_compress_workspace_bytes(int B, int H, int D, int t, int mem_len, unsigned flags) {
-    (void)B; (void)H; (void)D; (void)t; (void)mem_len; (void)flags;
-    return 0;
+    if (B <= 0 || H <= 0 || D <= 0 || t <= 0 || mem_len < 0) return 0;
+    return compress_workspace_bytes(B * H, D, t, mem_len, flags);
 }
 
 int loma_compress_step(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
@@ -245,8 +245,14 @@ int loma_compress_step(const void* q_mem, const void* k_mem, const void* v_mem, 
     if (dc != LOMA_OK) return dc;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = launch_compress_generic(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap,
-                                            mem_len, c, t, dtype, scale, flags, st);
+    if ((int64_t)B * H * 256 > INT_MAX) return LOMA_ERR_INVALID_ARG;
+    cudaError_t e;
+    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC) && t <= 16)
+        e = launch_compress_bf16(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, mem_len, c, t, flags,
+                                 scale, workspace, st);
+    else
+        e = launch_compress_generic(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, mem_len, c, t,
+                                    dtype, scale, flags, st);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 

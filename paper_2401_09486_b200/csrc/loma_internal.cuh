@@ -55,6 +55,12 @@ cudaError_t launch_decode_bf16_static(const void* q, const void* k_new, const vo
                                       void* v_cache, void* o, float* lse, int B, int H, int D, int cap,
                                       int cache_len, float scale, cudaStream_t st);
 
+// bf16 compress step on warp-level tensor cores (compress_mma.cu); t <= 16
+size_t compress_workspace_bytes(int BH, int D, int t, int mem_len, unsigned flags);
+cudaError_t launch_compress_bf16(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
+                                 void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len, int c, int t,
+                                 unsigned flags, float scale, void* ws, cudaStream_t st);
+
 cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const void* v_mem,
                                     void* k_cache, void* v_cache, void* o_mem, float* lse,
                                     int B, int H, int D, int cap, int mem_len, int c, int t,
