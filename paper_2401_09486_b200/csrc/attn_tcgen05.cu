@@ -21,16 +21,17 @@
 //
 // One CTA (192 threads) per SM, persistent over a statically ordered tile list
 // (longest tiles first, (batch, head) fastest).  Roles:
-//   warps 0-3  softmax: thread = query row = TMEM lane; two passes over the
-//              score tile in TMEM (row max, then exp2 / row sum / bf16 P written
-//              back over the scores), output accumulated in registers from the
-//              per-step P.V products, final O staged in shared memory for a TMA store
+//   warps 0-3  softmax: thread = query row = TMEM lane; one pass over the score
+//              tile (row max, exp2, row sum, bf16 P written back over the scores);
+//              the output accumulates in TMEM and is rescaled only when a row
+//              maximum has grown by more than 2^8; final O is staged in shared
+//              memory for a TMA store
 //   warp 4     TMA producer: Q per tile, K and V rings of two stages each
 //   warp 5     MMA issuer: S = Q K^T (both operands in shared memory), then
 //              P.V with P read from TMEM and V as an MN-major shared operand
-// TMEM (512 columns): two score buffers and two P.V buffers of 128 columns, so
-// the tensor pipe computes S(j+1) and P.V(j-1) while the softmax warps work on
-// S(j).  Every mbarrier wait is bounded: on expiry the CTA records
+// TMEM (512 columns allocated): two score buffers of 128 columns and one output
+// accumulator, so the tensor pipe computes S(j+1) and P.V(j-1) while the softmax
+// warps work on S(j).  Every mbarrier wait is bounded: on expiry the CTA records
 // LOMA_ERR_TIMEOUT, all roles leave their loops, TMEM is freed and the kernel
 // returns.
 #include <cuda.h>
@@ -132,8 +133,8 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// 32 consecutive fp32 columns of this thread's TMEM lane
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+// 32 consecutive 32-bit columns of this thread's TMEM lane -> r[0..31]
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -145,8 +146,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+        "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
 // 16 consecutive 32-bit columns of this thread's TMEM lane
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
         "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
@@ -198,7 +210,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     // barrier ids
-    enum { B_QF = 0, B_QE = 1, B_KF = 2, B_KE = 4, B_VF = 6, B_VE = 8, B_SF = 10, B_PF = 12, B_PVF = 14 };
+    enum { B_QF = 0, B_QE = 1, B_KF = 2, B_KE = 4, B_VF = 6, B_VE = 8, B_SF = 10, B_PF = 12, B_OF = 14 };
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
 
     if (threadIdx.x == 0) {
@@ -208,8 +220,8 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             mbar_init(bar(B_KF + i), 1); mbar_init(bar(B_KE + i), 1);
             mbar_init(bar(B_VF + i), 1); mbar_init(bar(B_VE + i), 1);
             mbar_init(bar(B_SF + i), 1); mbar_init(bar(B_PF + i), 128);
-            mbar_init(bar(B_PVF + i), 1);
         }
+        mbar_init(bar(B_OF), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // zero the operand buffers once: rows a TMA box does not cover keep finite contents
@@ -313,9 +325,9 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     const uint32_t va = smem_base + SM::V_OFF + b * SM::TILE_BYTES;
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)   // 16 keys per instruction
-                        mma_ts(tmem + 256 + b * 128, tmem + b * 128 + kk * 8,
-                               smem_desc(va + kk * 2048, SM::PANEL_BYTES, 1024), IDESC_PV, kk > 0);
-                    tc_commit(bar(B_PVF + b));
+                        mma_ts(tmem + 256, tmem + b * 128 + kk * 8, smem_desc(va + kk * 2048, SM::PANEL_BYTES, 1024),
+                               IDESC_PV, (j > 0) || (kk > 0));
+                    tc_commit(bar(B_OF));
                     tc_commit(bar(B_VE + b));
                 }
             }
@@ -338,25 +350,11 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             const int rc = td.a0 + rsub;
             const bool row_valid = (rr < qv.R * qv.CH) && (rc <= td.a1) && (ro < qv.Z);
 
-            float m = -INFINITY, l = 0.f, alpha_prev = 0.f;
-            float o[D];
-#pragma unroll
-            for (int d = 0; d < D; ++d) o[d] = 0.f;
-
-            auto accumulate_pv = [&](uint32_t g, float alpha) -> bool {
-                const uint32_t b = g & 1, ph = (g >> 1) & 1;
-                if (!__all_sync(0xffffffffu, mbar_wait(bar(B_PVF + b), ph, abortp, p.status))) return false;
-                tc_fence_after();
-#pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(lane_addr + 256 + b * 128 + c * 32, r);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) o[c * 32 + e] = fmaf(o[c * 32 + e], alpha, __uint_as_float(r[e]));
-                }
-                return true;
-            };
+            // Running reference maximum (exp2 domain) and row sum.  The reference only moves
+            // when the row maximum has grown by more than 2^8 since it was set; then the
+            // output accumulator in TMEM is rescaled once.  Probabilities stay below 2^8.
+            float m_used = -INFINITY, l = 0.f;
+            const uint32_t o_addr = lane_addr + 256;
 
             for (int j = 0; j < td.nsteps; ++j, ++gs) {
                 const uint32_t b = gs & 1, ph = (gs >> 1) & 1;
@@ -370,58 +368,67 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t s_addr = lane_addr + b * 128;
-                // pass 1: row maximum over the allowed columns
-                float mx = -INFINITY;
+                uint32_t s[128];
+                tmem_ld32(s_addr, s);
+                tmem_ld32(s_addr + 32, s + 32);
+                tmem_ld32(s_addr + 64, s + 64);
+                tmem_ld32(s_addr + 96, s + 96);
+                tmem_wait_ld();
+                if (!full) {
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(s_addr + c * 32, r);
-                    tmem_wait_ld();
-                    if (full) {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) {
-                            const bool in = (uint32_t)(c * 32 + e - lo) < span;
-                            mx = fmaxf(mx, in ? __uint_as_float(r[e]) : -INFINITY);
-                        }
-                    }
+                    for (int e = 0; e < 128; ++e)
+                        if ((uint32_t)(e - lo) >= span) s[e] = 0xff800000u;   // -inf
                 }
-                const float m_new = fmaxf(m, mx * p.scale_log2);
-                const float m_safe = (m_new == -INFINITY) ? 0.f : m_new;
-                const float alpha = fast_ex2(m - m_safe);
-                // pass 2: probabilities (bf16, written over the scores) and row sum
-                float lsum = 0.f;
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int e = 0; e < 128; e += 4) {
+                    mx0 = fmaxf(mx0, __uint_as_float(s[e]));
+                    mx1 = fmaxf(mx1, __uint_as_float(s[e + 1]));
+                    mx2 = fmaxf(mx2, __uint_as_float(s[e + 2]));
+                    mx3 = fmaxf(mx3, __uint_as_float(s[e + 3]));
+                }
+                const float mrow = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
+                const bool need = mrow > m_used + 8.f;
+                if (j > 0 && __any_sync(0xffffffffu, need)) {
+                    // rescale the accumulated output: wait until P.V(j-1) has landed in TMEM
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF), (gs - 1) & 1, abortp, p.status));
+                    if (!ok) break;
+                    tc_fence_after();
+                    const float alpha = need ? fast_ex2(m_used - mrow) : 1.f;
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(o_addr + c * 32, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+                        tmem_st32(o_addr + c * 32, r);
+                    }
+                    l *= alpha;
+                }
+                if (need) m_used = mrow;
+                const float neg_ref = (m_used == -INFINITY) ? 0.f : -m_used;
+                float ls0 = 0.f, ls1 = 0.f;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(s_addr + c * 32, r);
-                    tmem_wait_ld();
                     uint32_t pk[16];
 #pragma unroll
                     for (int e = 0; e < 32; e += 2) {
-                        float s0 = __uint_as_float(r[e]), s1 = __uint_as_float(r[e + 1]);
-                        if (!full) {
-                            s0 = ((uint32_t)(c * 32 + e - lo) < span) ? s0 : -INFINITY;
-                            s1 = ((uint32_t)(c * 32 + e + 1 - lo) < span) ? s1 : -INFINITY;
-                        }
-                        const float p0 = fast_ex2(fmaf(s0, p.scale_log2, -m_safe));
-                        const float p1 = fast_ex2(fmaf(s1, p.scale_log2, -m_safe));
-                        lsum += p0 + p1;
+                        const float p0 = fast_ex2(fmaf(__uint_as_float(s[c * 32 + e]), p.scale_log2, neg_ref));
+                        const float p1 = fast_ex2(fmaf(__uint_as_float(s[c * 32 + e + 1]), p.scale_log2, neg_ref));
+                        ls0 += p0;
+                        ls1 += p1;
                         pk[e >> 1] = pack_bf16(p0, p1);
                     }
                     tmem_st16(s_addr + c * 16, pk);
                 }
-                l = fmaf(l, alpha, lsum);
-                m = m_new;
+                l += ls0 + ls1;
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(B_PF + b));
-                if (j > 0) { ok = accumulate_pv(gs - 1, alpha_prev); if (!ok) break; }
-                alpha_prev = alpha;
             }
-            if (ok) ok = accumulate_pv(gs - 1, alpha_prev);
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF), (gs - 1) & 1, abortp, p.status));
+            if (ok) tc_fence_after();
 
             // epilogue: normalise, round to bf16, stage the tile in shared memory, TMA store.
             // Every thread reaches this barrier for every tile it started; the barrier also
@@ -439,17 +446,25 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             const float inv = 1.f / l;
             uint8_t* orow = smem_gen + SM::O_OFF + rr * 128;
 #pragma unroll
-            for (int ci = 0; ci < D / 8; ++ci) {
-                uint4 u;
-                u.x = pack_bf16(o[ci * 8 + 0] * inv, o[ci * 8 + 1] * inv);
-                u.y = pack_bf16(o[ci * 8 + 2] * inv, o[ci * 8 + 3] * inv);
-                u.z = pack_bf16(o[ci * 8 + 4] * inv, o[ci * 8 + 5] * inv);
-                u.w = pack_bf16(o[ci * 8 + 6] * inv, o[ci * 8 + 7] * inv);
-                *reinterpret_cast<uint4*>(orow + (ci >> 3) * SM::PANEL_BYTES + (((ci & 7) ^ (rr & 7)) << 4)) = u;
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(o_addr + c * 32, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const int ci = c * 4 + q4;       // 16-byte chunk of the row
+                    uint4 u;
+                    u.x = pack_bf16(__uint_as_float(r[q4 * 8 + 0]) * inv, __uint_as_float(r[q4 * 8 + 1]) * inv);
+                    u.y = pack_bf16(__uint_as_float(r[q4 * 8 + 2]) * inv, __uint_as_float(r[q4 * 8 + 3]) * inv);
+                    u.z = pack_bf16(__uint_as_float(r[q4 * 8 + 4]) * inv, __uint_as_float(r[q4 * 8 + 5]) * inv);
+                    u.w = pack_bf16(__uint_as_float(r[q4 * 8 + 6]) * inv, __uint_as_float(r[q4 * 8 + 7]) * inv);
+                    *reinterpret_cast<uint4*>(orow + (ci >> 3) * SM::PANEL_BYTES + (((ci & 7) ^ (rr & 7)) << 4)) = u;
+                }
             }
+            tc_fence_before();
             if (p.lse && row_valid) {
                 const int64_t grow = (int64_t)rc * p.s + qv.zone_row0 + ro;
-                p.lse[(int64_t)bh * p.S + grow] = (m + log2f(l)) * 0.6931471805599453f;
+                p.lse[(int64_t)bh * p.S + grow] = (m_used + log2f(l)) * 0.6931471805599453f;
             }
             fence_async_smem();
             asm volatile("bar.sync 1, 128;" ::: "memory");
