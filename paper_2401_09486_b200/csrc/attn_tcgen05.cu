@@ -19,18 +19,20 @@
 //   repetition rows x own memory zone                  key chunk == row chunk   (Eq. 1, row 3)
 //   repetition rows x themselves                       diagonal                 (I of Eq. 1)
 //
-// One CTA (192 threads) per SM, persistent over a statically ordered tile list
+// One CTA (320 threads) per SM, persistent over a statically ordered tile list
 // (longest tiles first, (batch, head) fastest).  Roles:
-//   warps 0-3  softmax: thread = query row = TMEM lane; one pass over the score
-//              tile (row max, exp2, row sum, bf16 P written back over the scores);
-//              the output accumulates in TMEM and is rescaled only when a row
-//              maximum has grown by more than 2^8; final O is staged in shared
+//   warps 0-7  two softmax warpgroups, thread = query row = TMEM lane; warpgroup g
+//              takes every other key tile (score buffer g): one pass over the
+//              scores (row max, exp2, row sum, bf16 P written back over the
+//              scores); its output accumulates in TMEM buffer g and is rescaled
+//              only when a row maximum has grown by more than 2^8; the two
+//              partial outputs are merged in the epilogue and staged in shared
 //              memory for a TMA store
-//   warp 4     TMA producer: Q per tile, K and V rings of two stages each
-//   warp 5     MMA issuer: S = Q K^T (both operands in shared memory), then
+//   warp 8     TMA producer: Q per tile, K and V rings of two stages each
+//   warp 9     MMA issuer: S = Q K^T (both operands in shared memory), then
 //              P.V with P read from TMEM and V as an MN-major shared operand
-// TMEM (512 columns allocated): two score buffers of 128 columns and one output
-// accumulator, so the tensor pipe computes S(j+1) and P.V(j-1) while the softmax
+// TMEM (512 columns): two score buffers and two output accumulators of 128
+// columns, so the tensor pipe computes S(j+1) and P.V(j-1) while the softmax
 // warps work on S(j).  Every mbarrier wait is bounded: on expiry the CTA records
 // LOMA_ERR_TIMEOUT, all roles leave their loops, TMEM is freed and the kernel
 // returns.
@@ -179,8 +181,49 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
            ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
 }
 
+// ---- softmax helpers on one 64-column half of a score row (registers only) ----
+__device__ __forceinline__ void half_load(uint32_t addr, uint32_t (&a)[64], bool full, int col0, int lo, uint32_t span) {
+    tmem_ld32(addr, a);
+    tmem_ld32(addr + 32, a + 32);
+    tmem_wait_ld();
+    if (!full) {
+#pragma unroll
+        for (int e = 0; e < 64; ++e)
+            if ((uint32_t)(col0 + e - lo) >= span) a[e] = 0xff800000u;   // -inf: the key is blocked for this row
+    }
+}
+__device__ __forceinline__ float half_max(const uint32_t (&a)[64]) {
+    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+    for (int e = 0; e < 64; e += 4) {
+        mx0 = fmaxf(mx0, __uint_as_float(a[e]));
+        mx1 = fmaxf(mx1, __uint_as_float(a[e + 1]));
+        mx2 = fmaxf(mx2, __uint_as_float(a[e + 2]));
+        mx3 = fmaxf(mx3, __uint_as_float(a[e + 3]));
+    }
+    return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+}
+// p = 2^(s*scale - ref) for 64 scores, packed to bf16 pairs and written to 32 TMEM columns at p_addr
+__device__ __forceinline__ void half_exp(const uint32_t (&a)[64], uint32_t p_addr, float scale_log2, float neg_ref,
+                                         float& ls0, float& ls1) {
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+            const float p0 = fast_ex2(fmaf(__uint_as_float(a[c * 32 + e]), scale_log2, neg_ref));
+            const float p1 = fast_ex2(fmaf(__uint_as_float(a[c * 32 + e + 1]), scale_log2, neg_ref));
+            ls0 += p0;
+            ls1 += p1;
+            pk[e >> 1] = pack_bf16(p0, p1);
+        }
+        tmem_st16(p_addr + c * 16, pk);
+    }
+}
+
 // ------------------------------------------------------------------ the kernel
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 320;   // 2 softmax warpgroups + TMA warp + MMA warp
+constexpr int W_TMA = 8, W_MMA = 9;
 constexpr int TMEM_COLS = 512;
 
 template <int D>
@@ -204,6 +247,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     __shared__ __align__(8) uint64_t bars[16];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ float2 xch[2][128];   // (reference max, row sum) of each softmax warpgroup, per row
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -221,13 +265,13 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             mbar_init(bar(B_VF + i), 1); mbar_init(bar(B_VE + i), 1);
             mbar_init(bar(B_SF + i), 1); mbar_init(bar(B_PF + i), 128);
         }
-        mbar_init(bar(B_OF), 1);
+        mbar_init(bar(B_OF), 1); mbar_init(bar(B_OF + 1), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // zero the operand buffers once: rows a TMA box does not cover keep finite contents
     for (int i = threadIdx.x; i < SM::TOTAL / 16; i += TC_THREADS) reinterpret_cast<uint4*>(smem_gen)[i] = make_uint4(0, 0, 0, 0);
     fence_async_smem();
-    if (warp == 5) {
+    if (warp == W_MMA) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
                      "r"(TMEM_COLS)
                      : "memory");
@@ -241,7 +285,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
 
     const int total_work = p.total_tiles * p.BH;
 
-    if (warp == 4) {
+    if (warp == W_TMA) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t gs = 0, tcount = 0;
@@ -284,7 +328,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 while (clock64() - t0 < 2000000ll) {}
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == W_MMA) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             // instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128
@@ -325,18 +369,24 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     const uint32_t va = smem_base + SM::V_OFF + b * SM::TILE_BYTES;
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)   // 16 keys per instruction
-                        mma_ts(tmem + 256, tmem + b * 128 + kk * 8, smem_desc(va + kk * 2048, SM::PANEL_BYTES, 1024),
-                               IDESC_PV, (j > 0) || (kk > 0));
-                    tc_commit(bar(B_OF));
+                        mma_ts(tmem + 256 + b * 128, tmem + b * 128 + (kk < 4 ? kk * 8 : 32 + kk * 8),
+                               smem_desc(va + kk * 2048, SM::PANEL_BYTES, 1024), IDESC_PV, (j > 1) || (kk > 0));
+                    tc_commit(bar(B_OF + b));
                     tc_commit(bar(B_VE + b));
                 }
             }
         }
     } else {
-        // ------------------------------------------------------------ softmax + epilogue (128 threads)
-        const int rr = threadIdx.x;
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
-        uint32_t gs = 0;
+        // ------------------------------------------------------------ softmax + epilogue (2 x 128 threads)
+        // Warpgroup wg takes the steps whose score buffer is wg (every other key tile) and
+        // keeps its own reference maximum, row sum and output accumulator; the two partial
+        // results of a query tile are merged in the epilogue.
+        const int wg = warp >> 2;
+        const int rr = threadIdx.x & 127;
+        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        const uint32_t s_addr = lane_addr + wg * 128;
+        const uint32_t o_addr = lane_addr + 256 + wg * 128;
+        uint32_t gs0 = 0;            // global step number of the tile's first step
         bool ok = true;
         bool store_pending = false;
         for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
@@ -354,44 +404,33 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             // when the row maximum has grown by more than 2^8 since it was set; then the
             // output accumulator in TMEM is rescaled once.  Probabilities stay below 2^8.
             float m_used = -INFINITY, l = 0.f;
-            const uint32_t o_addr = lane_addr + 256;
+            const int jfirst = (int)((gs0 ^ (uint32_t)wg) & 1u);   // first step of this tile that is ours
+            int jlast = -1;
 
-            for (int j = 0; j < td.nsteps; ++j, ++gs) {
-                const uint32_t b = gs & 1, ph = (gs >> 1) & 1;
+            for (int j = jfirst; j < td.nsteps; j += 2) {
+                const uint32_t gs = gs0 + j, ph = (gs >> 1) & 1;
                 KTile kt;
                 step_ktile(p, td, j, kt);
                 int lo, hi2;
                 row_interval(p.view[kt.view], kt, rc, ro, rr, row_valid, lo, hi2);
                 const bool full = __all_sync(0xffffffffu, lo <= 0 && hi2 >= 128);
                 const uint32_t span = (uint32_t)(hi2 - lo);
-                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF + b), ph, abortp, p.status));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF + wg), ph, abortp, p.status));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t s_addr = lane_addr + b * 128;
-                uint32_t s[128];
-                tmem_ld32(s_addr, s);
-                tmem_ld32(s_addr + 32, s + 32);
-                tmem_ld32(s_addr + 64, s + 64);
-                tmem_ld32(s_addr + 96, s + 96);
-                tmem_wait_ld();
-                if (!full) {
-#pragma unroll
-                    for (int e = 0; e < 128; ++e)
-                        if ((uint32_t)(e - lo) >= span) s[e] = 0xff800000u;   // -inf
-                }
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-                for (int e = 0; e < 128; e += 4) {
-                    mx0 = fmaxf(mx0, __uint_as_float(s[e]));
-                    mx1 = fmaxf(mx1, __uint_as_float(s[e + 1]));
-                    mx2 = fmaxf(mx2, __uint_as_float(s[e + 2]));
-                    mx3 = fmaxf(mx3, __uint_as_float(s[e + 3]));
-                }
-                const float mrow = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
+                // Scores of keys 0..63 sit in columns 0..63, keys 64..127 in columns 64..127.  Only 64
+                // of them are held in registers at a time: the first half is read twice (once for the
+                // row maximum, once for the exponentials).  P (bf16 pairs) goes to columns 0..31
+                // (keys 0..63) and 64..95 (keys 64..127), i.e. over scores already consumed.
+                uint32_t a[64];
+                half_load(s_addr, a, full, 0, lo, span);
+                float mrow = half_max(a);
+                half_load(s_addr + 64, a, full, 64, lo, span);
+                mrow = fmaxf(mrow, half_max(a)) * p.scale_log2;
                 const bool need = mrow > m_used + 8.f;
-                if (j > 0 && __any_sync(0xffffffffu, need)) {
-                    // rescale the accumulated output: wait until P.V(j-1) has landed in TMEM
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF), (gs - 1) & 1, abortp, p.status));
+                if (jlast >= 0 && __any_sync(0xffffffffu, need)) {
+                    // rescale the accumulated output: wait until our previous P.V has landed in TMEM
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + wg), ((gs - 2) >> 1) & 1, abortp, p.status));
                     if (!ok) break;
                     tc_fence_after();
                     const float alpha = need ? fast_ex2(m_used - mrow) : 1.f;
@@ -409,65 +448,84 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 if (need) m_used = mrow;
                 const float neg_ref = (m_used == -INFINITY) ? 0.f : -m_used;
                 float ls0 = 0.f, ls1 = 0.f;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        const float p0 = fast_ex2(fmaf(__uint_as_float(s[c * 32 + e]), p.scale_log2, neg_ref));
-                        const float p1 = fast_ex2(fmaf(__uint_as_float(s[c * 32 + e + 1]), p.scale_log2, neg_ref));
-                        ls0 += p0;
-                        ls1 += p1;
-                        pk[e >> 1] = pack_bf16(p0, p1);
-                    }
-                    tmem_st16(s_addr + c * 16, pk);
-                }
+                half_exp(a, s_addr + 64, p.scale_log2, neg_ref, ls0, ls1);   // the second half is still in registers
+                half_load(s_addr, a, full, 0, lo, span);
+                half_exp(a, s_addr, p.scale_log2, neg_ref, ls0, ls1);
                 l += ls0 + ls1;
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar(B_PF + b));
+                mbar_arrive(bar(B_PF + wg));
+                jlast = j;
             }
-            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF), (gs - 1) & 1, abortp, p.status));
+            if (ok && jlast >= 0)
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + wg), ((gs0 + jlast) >> 1) & 1, abortp, p.status));
             if (ok) tc_fence_after();
 
-            // epilogue: normalise, round to bf16, stage the tile in shared memory, TMA store.
-            // Every thread reaches this barrier for every tile it started; the barrier also
-            // makes the decision to give up uniform across the four warps.
+            // epilogue: merge the two warpgroups' partial results, normalise, round to bf16,
+            // stage the tile in shared memory, TMA store.  All 256 threads reach the first
+            // barrier for every tile they started; it also makes giving up a uniform decision.
+            xch[wg][rr] = make_float2(m_used, l);
             if (threadIdx.x == 0 && store_pending) tma_store_wait_read();
             {
                 uint32_t any_bad;
                 asm volatile(
-                    "{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, 1, 128, p;\nselp.u32 %0, 1, 0, q;\n}"
+                    "{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, 1, 256, p;\nselp.u32 %0, 1, 0, q;\n}"
                     : "=r"(any_bad)
                     : "r"((uint32_t)(ok ? 0 : 1))
                     : "memory");
                 if (any_bad) { ok = false; break; }
             }
-            const float inv = 1.f / l;
+            const float2 mine = xch[wg][rr], other = xch[wg ^ 1][rr];
+            const float2 a = wg == 0 ? mine : other, b2 = wg == 0 ? other : mine;   // warpgroup 0's and 1's state
+            // a warpgroup without a step in this tile has nothing valid in its accumulator
+            const bool has0 = ((gs0 & 1u) == 0u) || td.nsteps > 1;
+            const bool has1 = ((gs0 & 1u) == 1u) || td.nsteps > 1;
+            const float M = fmaxf(a.x, b2.x);
+            const float w0 = (has0 && a.x > -INFINITY) ? fast_ex2(a.x - M) : 0.f;
+            const float w1 = (has1 && b2.x > -INFINITY) ? fast_ex2(b2.x - M) : 0.f;
+            const float L = a.y * w0 + b2.y * w1;
+            const float inv = 1.f / L;
+            const float f0 = w0 * inv, f1 = w1 * inv;
             uint8_t* orow = smem_gen + SM::O_OFF + rr * 128;
+            // this warpgroup finishes output columns [wg*D/2, (wg+1)*D/2)
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld32(o_addr + c * 32, r);
-                tmem_wait_ld();
+            for (int cc = 0; cc < D / 64; ++cc) {
+                const int c = wg * (D / 64) + cc;
+                float x[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) x[e] = 0.f;
+                if (has0) {
+                    uint32_t r[32];
+                    tmem_ld32(lane_addr + 256 + c * 32, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) x[e] = __uint_as_float(r[e]) * f0;
+                }
+                if (has1) {
+                    uint32_t r[32];
+                    tmem_ld32(lane_addr + 384 + c * 32, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) x[e] = fmaf(__uint_as_float(r[e]), f1, x[e]);
+                }
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
                     const int ci = c * 4 + q4;       // 16-byte chunk of the row
                     uint4 u;
-                    u.x = pack_bf16(__uint_as_float(r[q4 * 8 + 0]) * inv, __uint_as_float(r[q4 * 8 + 1]) * inv);
-                    u.y = pack_bf16(__uint_as_float(r[q4 * 8 + 2]) * inv, __uint_as_float(r[q4 * 8 + 3]) * inv);
-                    u.z = pack_bf16(__uint_as_float(r[q4 * 8 + 4]) * inv, __uint_as_float(r[q4 * 8 + 5]) * inv);
-                    u.w = pack_bf16(__uint_as_float(r[q4 * 8 + 6]) * inv, __uint_as_float(r[q4 * 8 + 7]) * inv);
+                    u.x = pack_bf16(x[q4 * 8 + 0], x[q4 * 8 + 1]);
+                    u.y = pack_bf16(x[q4 * 8 + 2], x[q4 * 8 + 3]);
+                    u.z = pack_bf16(x[q4 * 8 + 4], x[q4 * 8 + 5]);
+                    u.w = pack_bf16(x[q4 * 8 + 6], x[q4 * 8 + 7]);
                     *reinterpret_cast<uint4*>(orow + (ci >> 3) * SM::PANEL_BYTES + (((ci & 7) ^ (rr & 7)) << 4)) = u;
                 }
             }
             tc_fence_before();
-            if (p.lse && row_valid) {
+            if (wg == 0 && p.lse && row_valid) {
                 const int64_t grow = (int64_t)rc * p.s + qv.zone_row0 + ro;
-                p.lse[(int64_t)bh * p.S + grow] = (m_used + log2f(l)) * 0.6931471805599453f;
+                p.lse[(int64_t)bh * p.S + grow] = (M + log2f(L)) * 0.6931471805599453f;
             }
             fence_async_smem();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             if (threadIdx.x == 0) {
                 for (int pn = 0; pn < PANELS; ++pn)
                     tma_store_5d(&maps.o[td.view], smem_base + SM::O_OFF + pn * SM::PANEL_BYTES, pn * 64, td.r0, td.c0, hi,
@@ -475,13 +533,14 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 tma_store_commit();
                 store_pending = true;
             }
+            gs0 += td.nsteps;
         }
         if (threadIdx.x == 0 && store_pending) tma_store_wait_all();
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == W_MMA) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
     }

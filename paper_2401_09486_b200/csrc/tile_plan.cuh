@@ -93,10 +93,12 @@ __host__ __device__ __forceinline__ void decode_tile(const FwdParams& p, int ran
 }
 
 __host__ __device__ __forceinline__ void step_ktile(const FwdParams& p, const TileDesc& td, int j, KTile& kt) {
-    const Seg& sg = (j < td.seg[0].count) ? td.seg[0] : td.seg[1];
-    const int t = sg.first + ((j < td.seg[0].count) ? j : j - td.seg[0].count);
-    const View& g = p.view[sg.view];
-    kt.view = sg.view; kt.mode = sg.mode;
+    const bool first = j < td.seg[0].count;
+    const int view = first ? td.seg[0].view : td.seg[1].view;
+    const int mode = first ? td.seg[0].mode : td.seg[1].mode;
+    const int t = first ? td.seg[0].first + j : td.seg[1].first + (j - td.seg[0].count);
+    const View& g = p.view[view];
+    kt.view = view; kt.mode = mode;
     if (g.Z >= 128) { kt.c0 = t / g.tpc; kt.r0 = (t - kt.c0 * g.tpc) * 128; }
     else { kt.c0 = t * g.CH; kt.r0 = 0; }
     kt.a0 = g.chunk_base + kt.c0;
