@@ -222,10 +222,11 @@ __device__ __forceinline__ void half_exp(const uint32_t (&a)[64], uint32_t p_add
 }
 
 // ------------------------------------------------------------------ the kernel
-constexpr int TC_THREADS = 320;   // 2 softmax warpgroups + TMA warp + MMA warp
-constexpr int W_TMA = 8, W_MMA = 9;
+constexpr int TC_THREADS = 384;   // 2 softmax warpgroups + 1 warpgroup with 2 TMA warps and 2 MMA warps
 constexpr int TMEM_COLS = 512;
+constexpr int NBAR = 9;           // mbarriers per stream
 
+// Shared memory of one stream: Q tile, one K tile, one V tile, and a 64-column output staging panel.
 template <int D>
 struct TcSmem {
     static constexpr int PANELS = D / 64;
@@ -233,9 +234,10 @@ struct TcSmem {
     static constexpr int TILE_BYTES = PANELS * PANEL_BYTES; // one 128 x D tile
     static constexpr int Q_OFF = 0;
     static constexpr int K_OFF = TILE_BYTES;
-    static constexpr int V_OFF = 3 * TILE_BYTES;
-    static constexpr int O_OFF = 5 * TILE_BYTES;
-    static constexpr int TOTAL = 6 * TILE_BYTES;
+    static constexpr int V_OFF = 2 * TILE_BYTES;
+    static constexpr int O_OFF = 3 * TILE_BYTES;
+    static constexpr int STREAM_BYTES = 3 * TILE_BYTES + PANEL_BYTES;
+    static constexpr int TOTAL = 2 * STREAM_BYTES;
 };
 
 template <int D>
@@ -244,34 +246,32 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     using SM = TcSmem<D>;
     constexpr int PANELS = SM::PANELS;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[16];
+    __shared__ __align__(8) uint64_t bars[2 * NBAR];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ float2 xch[2][128];   // (reference max, row sum) of each softmax warpgroup, per row
 
-    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // which of the CTA's two independent streams this warp serves
+    const int st = warp < 8 ? (warp >> 2) : (warp & 1);
+    const uint32_t smem_base0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen0 = smem_raw + (smem_base0 - smem_u32(smem_raw));
+    const uint32_t smem_base = smem_base0 + st * SM::STREAM_BYTES;
+    uint8_t* smem_gen = smem_gen0 + st * SM::STREAM_BYTES;
 
-    // barrier ids
-    enum { B_QF = 0, B_QE = 1, B_KF = 2, B_KE = 4, B_VF = 6, B_VE = 8, B_SF = 10, B_PF = 12, B_OF = 14 };
-    auto bar = [&](int i) { return smem_u32(&bars[i]); };
+    enum { B_QF = 0, B_QE = 1, B_KF = 2, B_KE = 3, B_VF = 4, B_VE = 5, B_SF = 6, B_PF = 7, B_OF = 8 };
+    auto bar = [&](int i) { return smem_u32(&bars[st * NBAR + i]); };
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        mbar_init(bar(B_QF), 1); mbar_init(bar(B_QE), 1);
-        for (int i = 0; i < 2; ++i) {
-            mbar_init(bar(B_KF + i), 1); mbar_init(bar(B_KE + i), 1);
-            mbar_init(bar(B_VF + i), 1); mbar_init(bar(B_VE + i), 1);
-            mbar_init(bar(B_SF + i), 1); mbar_init(bar(B_PF + i), 128);
-        }
-        mbar_init(bar(B_OF), 1); mbar_init(bar(B_OF + 1), 1);
+        for (int s2 = 0; s2 < 2; ++s2)
+            for (int i = 0; i < NBAR; ++i) mbar_init(smem_u32(&bars[s2 * NBAR + i]), i == B_PF ? 128 : 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // zero the operand buffers once: rows a TMA box does not cover keep finite contents
-    for (int i = threadIdx.x; i < SM::TOTAL / 16; i += TC_THREADS) reinterpret_cast<uint4*>(smem_gen)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = threadIdx.x; i < SM::TOTAL / 16; i += TC_THREADS)
+        reinterpret_cast<uint4*>(smem_gen0)[i] = make_uint4(0, 0, 0, 0);
     fence_async_smem();
-    if (warp == W_MMA) {
+    if (warp == 10) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
                      "r"(TMEM_COLS)
                      : "memory");
@@ -280,17 +280,21 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = tmem_slot;
+    const uint32_t tmem = tmem_slot + st * 256;   // this stream's scores at +0, output accumulator at +128
     volatile int* abortp = &abort_flag;
 
+    // tiles are dealt to the 2*gridDim.x streams round robin, longest first
     const int total_work = p.total_tiles * p.BH;
+    const int nstreams = 2 * gridDim.x;
+    const int w0 = blockIdx.x + st * gridDim.x;
 
-    if (warp == W_TMA) {
-        // ------------------------------------------------------------ TMA producer
+    if (warp == 8 || warp == 9) {
+        // ------------------------------------------------------------ TMA producer of stream st
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
         if (lane == 0) {
             uint32_t gs = 0, tcount = 0;
             bool ok = true;
-            for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++tcount) {
+            for (int w = w0; w < total_work && ok; w += nstreams, ++tcount) {
                 const int rank = w / p.BH, bh = w - rank * p.BH;
                 const int bi = bh / p.H, hi = bh - bi * p.H;
                 TileDesc td;
@@ -306,20 +310,20 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     KTile kt;
                     step_ktile(p, td, j, kt);
                     const View& kv = p.view[kt.view];
-                    const uint32_t b = gs & 1, ph = (gs >> 1) & 1;
+                    const uint32_t ph = gs & 1;
                     const uint32_t bytes = kv.R * kv.CH * 128 * PANELS;
-                    ok = mbar_wait(bar(B_KE + b), ph ^ 1, abortp, p.status);
+                    ok = mbar_wait(bar(B_KE), ph ^ 1, abortp, p.status);
                     if (!ok) break;
-                    mbar_expect_tx(bar(B_KF + b), bytes);
+                    mbar_expect_tx(bar(B_KF), bytes);
                     for (int pn = 0; pn < PANELS; ++pn)
-                        tma_load_5d(smem_base + SM::K_OFF + b * SM::TILE_BYTES + pn * SM::PANEL_BYTES, &maps.k[kt.view],
-                                    bar(B_KF + b), pn * 64, kt.r0, kt.c0, hi, bi);
-                    ok = mbar_wait(bar(B_VE + b), ph ^ 1, abortp, p.status);
+                        tma_load_5d(smem_base + SM::K_OFF + pn * SM::PANEL_BYTES, &maps.k[kt.view], bar(B_KF), pn * 64,
+                                    kt.r0, kt.c0, hi, bi);
+                    ok = mbar_wait(bar(B_VE), ph ^ 1, abortp, p.status);
                     if (!ok) break;
-                    mbar_expect_tx(bar(B_VF + b), bytes);
+                    mbar_expect_tx(bar(B_VF), bytes);
                     for (int pn = 0; pn < PANELS; ++pn)
-                        tma_load_5d(smem_base + SM::V_OFF + b * SM::TILE_BYTES + pn * SM::PANEL_BYTES, &maps.v[kt.view],
-                                    bar(B_VF + b), pn * 64, kt.r0, kt.c0, hi, bi);
+                        tma_load_5d(smem_base + SM::V_OFF + pn * SM::PANEL_BYTES, &maps.v[kt.view], bar(B_VF), pn * 64,
+                                    kt.r0, kt.c0, hi, bi);
                 }
             }
             if (!ok) {
@@ -328,8 +332,9 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 while (clock64() - t0 < 2000000ll) {}
             }
         }
-    } else if (warp == W_MMA) {
-        // ------------------------------------------------------------ MMA issuer
+    } else if (warp >= 10) {
+        // ------------------------------------------------------------ MMA issuer of stream st
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
         if (lane == 0) {
             // instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128
             constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
@@ -337,21 +342,20 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
             uint32_t gs = 0, tcount = 0;
             bool ok = true;
+            const uint32_t qa = smem_base + SM::Q_OFF, ka = smem_base + SM::K_OFF, va = smem_base + SM::V_OFF;
             auto issue_s = [&](uint32_t g) -> bool {
-                const uint32_t b = g & 1, ph = (g >> 1) & 1;
-                if (!mbar_wait(bar(B_KF + b), ph, abortp, p.status)) return false;
+                if (!mbar_wait(bar(B_KF), g & 1, abortp, p.status)) return false;
                 tc_fence_after();
-                const uint32_t qa = smem_base + SM::Q_OFF, ka = smem_base + SM::K_OFF + b * SM::TILE_BYTES;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = (kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32;
-                    mma_ss(tmem + b * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), IDESC_S, kk > 0);
+                    mma_ss(tmem, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), IDESC_S, kk > 0);
                 }
-                tc_commit(bar(B_SF + b));
-                tc_commit(bar(B_KE + b));
+                tc_commit(bar(B_SF));
+                tc_commit(bar(B_KE));
                 return true;
             };
-            for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x, ++tcount) {
+            for (int w = w0; w < total_work && ok; w += nstreams, ++tcount) {
                 const int rank = w / p.BH;
                 TileDesc td;
                 decode_tile(p, rank, td);
@@ -360,36 +364,31 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 tc_fence_after();
                 ok = issue_s(gs);
                 for (int j = 0; j < td.nsteps && ok; ++j, ++gs) {
-                    const uint32_t b = gs & 1, ph = (gs >> 1) & 1;
-                    if (j + 1 < td.nsteps) { ok = issue_s(gs + 1); if (!ok) break; }
-                    else tc_commit(bar(B_QE));
-                    ok = mbar_wait(bar(B_PF + b), ph, abortp, p.status) && mbar_wait(bar(B_VF + b), ph, abortp, p.status);
+                    const uint32_t ph = gs & 1;
+                    ok = mbar_wait(bar(B_PF), ph, abortp, p.status) && mbar_wait(bar(B_VF), ph, abortp, p.status);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t va = smem_base + SM::V_OFF + b * SM::TILE_BYTES;
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)   // 16 keys per instruction
-                        mma_ts(tmem + 256 + b * 128, tmem + b * 128 + (kk < 4 ? kk * 8 : 32 + kk * 8),
-                               smem_desc(va + kk * 2048, SM::PANEL_BYTES, 1024), IDESC_PV, (j > 1) || (kk > 0));
-                    tc_commit(bar(B_OF + b));
-                    tc_commit(bar(B_VE + b));
+                    for (int kk = 0; kk < 8; ++kk)   // 16 keys per instruction, P read from TMEM
+                        mma_ts(tmem + 128, tmem + kk * 8, smem_desc(va + kk * 2048, SM::PANEL_BYTES, 1024), IDESC_PV,
+                               (j > 0) || (kk > 0));
+                    tc_commit(bar(B_OF));
+                    tc_commit(bar(B_VE));
+                    if (j + 1 < td.nsteps) ok = issue_s(gs + 1);
+                    else tc_commit(bar(B_QE));
                 }
             }
         }
     } else {
-        // ------------------------------------------------------------ softmax + epilogue (2 x 128 threads)
-        // Warpgroup wg takes the steps whose score buffer is wg (every other key tile) and
-        // keeps its own reference maximum, row sum and output accumulator; the two partial
-        // results of a query tile are merged in the epilogue.
-        const int wg = warp >> 2;
+        // ------------------------------------------------------------ softmax + epilogue of stream st (128 threads)
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 232;" ::: "memory");
         const int rr = threadIdx.x & 127;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-        const uint32_t s_addr = lane_addr + wg * 128;
-        const uint32_t o_addr = lane_addr + 256 + wg * 128;
-        uint32_t gs0 = 0;            // global step number of the tile's first step
+        const uint32_t s_addr = lane_addr, o_addr = lane_addr + 128;
+        uint32_t gs = 0;
         bool ok = true;
         bool store_pending = false;
-        for (int w = blockIdx.x; w < total_work && ok; w += gridDim.x) {
+        for (int w = w0; w < total_work && ok; w += nstreams) {
             const int rank = w / p.BH, bh = w - rank * p.BH;
             const int bi = bh / p.H, hi = bh - bi * p.H;
             TileDesc td;
@@ -404,33 +403,41 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             // when the row maximum has grown by more than 2^8 since it was set; then the
             // output accumulator in TMEM is rescaled once.  Probabilities stay below 2^8.
             float m_used = -INFINITY, l = 0.f;
-            const int jfirst = (int)((gs0 ^ (uint32_t)wg) & 1u);   // first step of this tile that is ours
-            int jlast = -1;
 
-            for (int j = jfirst; j < td.nsteps; j += 2) {
-                const uint32_t gs = gs0 + j, ph = (gs >> 1) & 1;
+            for (int j = 0; j < td.nsteps; ++j, ++gs) {
                 KTile kt;
                 step_ktile(p, td, j, kt);
                 int lo, hi2;
                 row_interval(p.view[kt.view], kt, rc, ro, rr, row_valid, lo, hi2);
                 const bool full = __all_sync(0xffffffffu, lo <= 0 && hi2 >= 128);
                 const uint32_t span = (uint32_t)(hi2 - lo);
-                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF + wg), ph, abortp, p.status));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF), gs & 1, abortp, p.status));
                 if (!ok) break;
                 tc_fence_after();
-                // Scores of keys 0..63 sit in columns 0..63, keys 64..127 in columns 64..127.  Only 64
-                // of them are held in registers at a time: the first half is read twice (once for the
-                // row maximum, once for the exponentials).  P (bf16 pairs) goes to columns 0..31
-                // (keys 0..63) and 64..95 (keys 64..127), i.e. over scores already consumed.
-                uint32_t a[64];
-                half_load(s_addr, a, full, 0, lo, span);
-                float mrow = half_max(a);
-                half_load(s_addr + 64, a, full, 64, lo, span);
-                mrow = fmaxf(mrow, half_max(a)) * p.scale_log2;
+                uint32_t s[128];
+                tmem_ld32(s_addr, s);
+                tmem_ld32(s_addr + 32, s + 32);
+                tmem_ld32(s_addr + 64, s + 64);
+                tmem_ld32(s_addr + 96, s + 96);
+                tmem_wait_ld();
+                if (!full) {
+#pragma unroll
+                    for (int e = 0; e < 128; ++e)
+                        if ((uint32_t)(e - lo) >= span) s[e] = 0xff800000u;   // -inf: the key is blocked for this row
+                }
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int e = 0; e < 128; e += 4) {
+                    mx0 = fmaxf(mx0, __uint_as_float(s[e]));
+                    mx1 = fmaxf(mx1, __uint_as_float(s[e + 1]));
+                    mx2 = fmaxf(mx2, __uint_as_float(s[e + 2]));
+                    mx3 = fmaxf(mx3, __uint_as_float(s[e + 3]));
+                }
+                const float mrow = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
                 const bool need = mrow > m_used + 8.f;
-                if (jlast >= 0 && __any_sync(0xffffffffu, need)) {
-                    // rescale the accumulated output: wait until our previous P.V has landed in TMEM
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + wg), ((gs - 2) >> 1) & 1, abortp, p.status));
+                if (j > 0 && __any_sync(0xffffffffu, need)) {
+                    // rescale the accumulated output: wait until P.V(j-1) has landed in TMEM
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF), (gs - 1) & 1, abortp, p.status));
                     if (!ok) break;
                     tc_fence_after();
                     const float alpha = need ? fast_ex2(m_used - mrow) : 1.f;
@@ -448,101 +455,86 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 if (need) m_used = mrow;
                 const float neg_ref = (m_used == -INFINITY) ? 0.f : -m_used;
                 float ls0 = 0.f, ls1 = 0.f;
-                half_exp(a, s_addr + 64, p.scale_log2, neg_ref, ls0, ls1);   // the second half is still in registers
-                half_load(s_addr, a, full, 0, lo, span);
-                half_exp(a, s_addr, p.scale_log2, neg_ref, ls0, ls1);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        const float p0 = fast_ex2(fmaf(__uint_as_float(s[c * 32 + e]), p.scale_log2, neg_ref));
+                        const float p1 = fast_ex2(fmaf(__uint_as_float(s[c * 32 + e + 1]), p.scale_log2, neg_ref));
+                        ls0 += p0;
+                        ls1 += p1;
+                        pk[e >> 1] = pack_bf16(p0, p1);
+                    }
+                    tmem_st16(s_addr + c * 16, pk);   // P over the scores: keys 32c..32c+31 -> columns 16c..16c+15
+                }
                 l += ls0 + ls1;
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar(B_PF + wg));
-                jlast = j;
+                mbar_arrive(bar(B_PF));
             }
-            if (ok && jlast >= 0)
-                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + wg), ((gs0 + jlast) >> 1) & 1, abortp, p.status));
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF), (gs - 1) & 1, abortp, p.status));
             if (ok) tc_fence_after();
 
-            // epilogue: merge the two warpgroups' partial results, normalise, round to bf16,
-            // stage the tile in shared memory, TMA store.  All 256 threads reach the first
-            // barrier for every tile they started; it also makes giving up a uniform decision.
-            xch[wg][rr] = make_float2(m_used, l);
-            if (threadIdx.x == 0 && store_pending) tma_store_wait_read();
-            {
-                uint32_t any_bad;
-                asm volatile(
-                    "{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, 1, 256, p;\nselp.u32 %0, 1, 0, q;\n}"
-                    : "=r"(any_bad)
-                    : "r"((uint32_t)(ok ? 0 : 1))
-                    : "memory");
-                if (any_bad) { ok = false; break; }
-            }
-            const float2 mine = xch[wg][rr], other = xch[wg ^ 1][rr];
-            const float2 a = wg == 0 ? mine : other, b2 = wg == 0 ? other : mine;   // warpgroup 0's and 1's state
-            // a warpgroup without a step in this tile has nothing valid in its accumulator
-            const bool has0 = ((gs0 & 1u) == 0u) || td.nsteps > 1;
-            const bool has1 = ((gs0 & 1u) == 1u) || td.nsteps > 1;
-            const float M = fmaxf(a.x, b2.x);
-            const float w0 = (has0 && a.x > -INFINITY) ? fast_ex2(a.x - M) : 0.f;
-            const float w1 = (has1 && b2.x > -INFINITY) ? fast_ex2(b2.x - M) : 0.f;
-            const float L = a.y * w0 + b2.y * w1;
-            const float inv = 1.f / L;
-            const float f0 = w0 * inv, f1 = w1 * inv;
+            // epilogue: normalise, round to bf16, stage 64 output columns at a time in shared
+            // memory, TMA store.  Every thread of the warpgroup reaches the first barrier for
+            // every tile it started; it also makes giving up a uniform decision.
+            const float inv = 1.f / l;
             uint8_t* orow = smem_gen + SM::O_OFF + rr * 128;
-            // this warpgroup finishes output columns [wg*D/2, (wg+1)*D/2)
+            bool give_up = false;
 #pragma unroll
-            for (int cc = 0; cc < D / 64; ++cc) {
-                const int c = wg * (D / 64) + cc;
-                float x[32];
-#pragma unroll
-                for (int e = 0; e < 32; ++e) x[e] = 0.f;
-                if (has0) {
-                    uint32_t r[32];
-                    tmem_ld32(lane_addr + 256 + c * 32, r);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) x[e] = __uint_as_float(r[e]) * f0;
-                }
-                if (has1) {
-                    uint32_t r[32];
-                    tmem_ld32(lane_addr + 384 + c * 32, r);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) x[e] = fmaf(__uint_as_float(r[e]), f1, x[e]);
+            for (int pn = 0; pn < PANELS; ++pn) {
+                if (rr == 0 && store_pending) tma_store_wait_read();   // the staging panel is free again
+                if (pn == 0) {
+                    uint32_t any_bad;
+                    asm volatile(
+                        "{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, %2, 128, p;\nselp.u32 %0, 1, 0, q;\n}"
+                        : "=r"(any_bad)
+                        : "r"((uint32_t)(ok ? 0 : 1)), "r"(1 + st)
+                        : "memory");
+                    if (any_bad) { give_up = true; break; }
+                } else {
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + st) : "memory");
                 }
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const int ci = c * 4 + q4;       // 16-byte chunk of the row
-                    uint4 u;
-                    u.x = pack_bf16(x[q4 * 8 + 0], x[q4 * 8 + 1]);
-                    u.y = pack_bf16(x[q4 * 8 + 2], x[q4 * 8 + 3]);
-                    u.z = pack_bf16(x[q4 * 8 + 4], x[q4 * 8 + 5]);
-                    u.w = pack_bf16(x[q4 * 8 + 6], x[q4 * 8 + 7]);
-                    *reinterpret_cast<uint4*>(orow + (ci >> 3) * SM::PANEL_BYTES + (((ci & 7) ^ (rr & 7)) << 4)) = u;
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(o_addr + pn * 64 + c * 32, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const int ci = c * 4 + q4;       // 16-byte chunk of the 128-byte panel row
+                        uint4 u;
+                        u.x = pack_bf16(__uint_as_float(r[q4 * 8 + 0]) * inv, __uint_as_float(r[q4 * 8 + 1]) * inv);
+                        u.y = pack_bf16(__uint_as_float(r[q4 * 8 + 2]) * inv, __uint_as_float(r[q4 * 8 + 3]) * inv);
+                        u.z = pack_bf16(__uint_as_float(r[q4 * 8 + 4]) * inv, __uint_as_float(r[q4 * 8 + 5]) * inv);
+                        u.w = pack_bf16(__uint_as_float(r[q4 * 8 + 6]) * inv, __uint_as_float(r[q4 * 8 + 7]) * inv);
+                        *reinterpret_cast<uint4*>(orow + ((ci ^ (rr & 7)) << 4)) = u;
+                    }
+                }
+                fence_async_smem();
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + st) : "memory");
+                if (rr == 0) {
+                    tma_store_5d(&maps.o[td.view], smem_base + SM::O_OFF, pn * 64, td.r0, td.c0, hi, bi);
+                    tma_store_commit();
+                    store_pending = true;
                 }
             }
+            if (give_up) { ok = false; break; }
             tc_fence_before();
-            if (wg == 0 && p.lse && row_valid) {
+            if (p.lse && row_valid) {
                 const int64_t grow = (int64_t)rc * p.s + qv.zone_row0 + ro;
-                p.lse[(int64_t)bh * p.S + grow] = (M + log2f(L)) * 0.6931471805599453f;
+                p.lse[(int64_t)bh * p.S + grow] = (m_used + log2f(l)) * 0.6931471805599453f;
             }
-            fence_async_smem();
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (threadIdx.x == 0) {
-                for (int pn = 0; pn < PANELS; ++pn)
-                    tma_store_5d(&maps.o[td.view], smem_base + SM::O_OFF + pn * SM::PANEL_BYTES, pn * 64, td.r0, td.c0, hi,
-                                 bi);
-                tma_store_commit();
-                store_pending = true;
-            }
-            gs0 += td.nsteps;
         }
-        if (threadIdx.x == 0 && store_pending) tma_store_wait_all();
+        if (rr == 0 && store_pending) tma_store_wait_all();
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == W_MMA) {
+    if (warp == 10) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_slot), "r"(TMEM_COLS) : "memory");
     }
 }
 
@@ -641,16 +633,17 @@ cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, v
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int64_t work = (int64_t)p.total_tiles * p.BH;
-    const int grid = (int)(work < sms ? work : sms);
+    const int64_t want = (work + 1) / 2;            // two streams (query tiles in flight) per CTA
+    const int grid = (int)(want < sms ? want : sms);
     cudaError_t e;
+    // the shared-memory footprint also keeps one CTA per SM (each allocates all 512 TMEM columns)
     if (D == 128) {
         const int smem = TcSmem<128>::TOTAL + 1024;
         e = cudaFuncSetAttribute(masked_attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         masked_attn_tc_kernel<128><<<grid, TC_THREADS, smem, st>>>(maps, p);
     } else {
-        // the shared-memory footprint also keeps one CTA per SM (each allocates all 512 TMEM columns)
-        const int smem = 120 * 1024;
+        const int smem = TcSmem<64>::TOTAL + 1024;
         e = cudaFuncSetAttribute(masked_attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         masked_attn_tc_kernel<64><<<grid, TC_THREADS, smem, st>>>(maps, p);
