@@ -175,6 +175,14 @@ __device__ __forceinline__ float fast_ex2(float x) {
     return y;
 }
 
+// One lane of a converged warp.  The MMA and TMA roles keep their control flow warp-uniform and
+// predicate only the issuing instruction, so descriptors and addresses can live in uniform registers.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n.reg .pred P;\nelect.sync _|P, 0xffffffff;\nselp.u32 %0, 1, 0, P;\n}" : "=r"(pred)::"memory");
+    return pred != 0;
+}
+
 // Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
     return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
@@ -250,7 +258,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
     // which of the CTA's two independent streams this warp serves
     const int st = warp < 8 ? (warp >> 2) : (warp & 1);
     const uint32_t smem_base0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -334,48 +342,62 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         }
     } else if (warp >= 10) {
         // ------------------------------------------------------------ MMA issuer of stream st
+        // All 32 lanes run the loops (warp-uniform); one elected lane issues the instructions.
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
-        if (lane == 0) {
+        {
             // instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128
             constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
             constexpr uint32_t IDESC_PV =
                 (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
             uint32_t gs = 0, tcount = 0;
             bool ok = true;
-            const uint32_t qa = smem_base + SM::Q_OFF, ka = smem_base + SM::K_OFF, va = smem_base + SM::V_OFF;
+            const uint64_t qd = smem_desc(smem_base + SM::Q_OFF, 16, 1024);
+            const uint64_t kd = smem_desc(smem_base + SM::K_OFF, 16, 1024);
+            const uint64_t vd = smem_desc(smem_base + SM::V_OFF, SM::PANEL_BYTES, 1024);
             auto issue_s = [&](uint32_t g) -> bool {
-                if (!mbar_wait(bar(B_KF), g & 1, abortp, p.status)) return false;
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(B_KF), g & 1, abortp, p.status))) return false;
                 tc_fence_after();
+                if (elect_one()) {
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32;
-                    mma_ss(tmem, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), IDESC_S, kk > 0);
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        // descriptor start addresses are in 16-byte units
+                        const uint64_t off = (uint64_t)(((kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32) >> 4);
+                        mma_ss(tmem, qd + off, kd + off, IDESC_S, kk > 0);
+                    }
+                    tc_commit(bar(B_SF));
+                    tc_commit(bar(B_KE));
                 }
-                tc_commit(bar(B_SF));
-                tc_commit(bar(B_KE));
+                __syncwarp();
                 return true;
             };
             for (int w = w0; w < total_work && ok; w += nstreams, ++tcount) {
                 const int rank = w / p.BH;
                 TileDesc td;
                 decode_tile(p, rank, td);
-                ok = mbar_wait(bar(B_QF), tcount & 1, abortp, p.status);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_QF), tcount & 1, abortp, p.status));
                 if (!ok) break;
                 tc_fence_after();
                 ok = issue_s(gs);
                 for (int j = 0; j < td.nsteps && ok; ++j, ++gs) {
                     const uint32_t ph = gs & 1;
-                    ok = mbar_wait(bar(B_PF), ph, abortp, p.status) && mbar_wait(bar(B_VF), ph, abortp, p.status);
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_PF), ph, abortp, p.status) &&
+                                                     mbar_wait(bar(B_VF), ph, abortp, p.status));
                     if (!ok) break;
                     tc_fence_after();
+                    if (elect_one()) {
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)   // 16 keys per instruction, P read from TMEM
-                        mma_ts(tmem + 128, tmem + kk * 8, smem_desc(va + kk * 2048, SM::PANEL_BYTES, 1024), IDESC_PV,
-                               (j > 0) || (kk > 0));
-                    tc_commit(bar(B_OF));
-                    tc_commit(bar(B_VE));
+                        for (int kk = 0; kk < 8; ++kk)   // 16 keys per instruction, P read from TMEM
+                            mma_ts(tmem + 128, tmem + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), IDESC_PV,
+                                   (j > 0) || (kk > 0));
+                        tc_commit(bar(B_OF));
+                        tc_commit(bar(B_VE));
+                    }
+                    __syncwarp();
                     if (j + 1 < td.nsteps) ok = issue_s(gs + 1);
-                    else tc_commit(bar(B_QE));
+                    else {
+                        if (elect_one()) tc_commit(bar(B_QE));
+                        __syncwarp();
+                    }
                 }
             }
         }
