@@ -175,6 +175,32 @@ __device__ __forceinline__ float fast_ex2(float x) {
     return y;
 }
 
+// Packed pairs of fp32 (sm_100 has two-wide fp32 FMA and ADD) and the three-input maximum: the
+// softmax warps are bound by instruction issue, so fewer instructions per score matter.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
 // One lane of a converged warp.  The MMA and TMA roles keep their control flow warp-uniform and
 // predicate only the issuing instruction, so descriptors and addresses can live in uniform registers.
 __device__ __forceinline__ bool elect_one() {
@@ -449,11 +475,11 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 }
                 float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                for (int e = 0; e < 128; e += 4) {
-                    mx0 = fmaxf(mx0, __uint_as_float(s[e]));
-                    mx1 = fmaxf(mx1, __uint_as_float(s[e + 1]));
-                    mx2 = fmaxf(mx2, __uint_as_float(s[e + 2]));
-                    mx3 = fmaxf(mx3, __uint_as_float(s[e + 3]));
+                for (int e = 0; e < 128; e += 8) {
+                    mx0 = max3(mx0, __uint_as_float(s[e]), __uint_as_float(s[e + 1]));
+                    mx1 = max3(mx1, __uint_as_float(s[e + 2]), __uint_as_float(s[e + 3]));
+                    mx2 = max3(mx2, __uint_as_float(s[e + 4]), __uint_as_float(s[e + 5]));
+                    mx3 = max3(mx3, __uint_as_float(s[e + 6]), __uint_as_float(s[e + 7]));
                 }
                 const float mrow = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
                 const bool need = mrow > m_used + 8.f;
@@ -476,21 +502,30 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 }
                 if (need) m_used = mrow;
                 const float neg_ref = (m_used == -INFINITY) ? 0.f : -m_used;
-                float ls0 = 0.f, ls1 = 0.f;
+                const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nr2 = pack2(neg_ref, neg_ref);
+                uint64_t lsa = pack2(0.f, 0.f), lsb = lsa;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     uint32_t pk[16];
 #pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        const float p0 = fast_ex2(fmaf(__uint_as_float(s[c * 32 + e]), p.scale_log2, neg_ref));
-                        const float p1 = fast_ex2(fmaf(__uint_as_float(s[c * 32 + e + 1]), p.scale_log2, neg_ref));
-                        ls0 += p0;
-                        ls1 += p1;
+                    for (int e = 0; e < 32; e += 4) {
+                        float x0, x1, x2, x3;
+                        unpack2(fma2(pack2(__uint_as_float(s[c * 32 + e]), __uint_as_float(s[c * 32 + e + 1])), sc2, nr2), x0, x1);
+                        unpack2(fma2(pack2(__uint_as_float(s[c * 32 + e + 2]), __uint_as_float(s[c * 32 + e + 3])), sc2, nr2), x2, x3);
+                        const float p0 = fast_ex2(x0), p1 = fast_ex2(x1), p2 = fast_ex2(x2), p3 = fast_ex2(x3);
+                        lsa = add2(lsa, pack2(p0, p1));
+                        lsb = add2(lsb, pack2(p2, p3));
                         pk[e >> 1] = pack_bf16(p0, p1);
+                        pk[(e >> 1) + 1] = pack_bf16(p2, p3);
                     }
                     tmem_st16(s_addr + c * 16, pk);   // P over the scores: keys 32c..32c+31 -> columns 16c..16c+15
                 }
-                l += ls0 + ls1;
+                {
+                    float a0, a1, b0, b1;
+                    unpack2(lsa, a0, a1);
+                    unpack2(lsb, b0, b1);
+                    l += (a0 + a1) + (b0 + b1);
+                }
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(B_PF));
