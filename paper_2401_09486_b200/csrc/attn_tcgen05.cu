@@ -258,7 +258,7 @@ __device__ __forceinline__ void half_exp(const uint32_t (&a)[64], uint32_t p_add
 // ------------------------------------------------------------------ the kernel
 constexpr int TC_THREADS = 384;   // 2 softmax warpgroups + 1 warpgroup with 2 TMA warps and 2 MMA warps
 constexpr int TMEM_COLS = 512;
-constexpr int NBAR = 9;           // mbarriers per stream
+constexpr int NBAR = 11;          // mbarriers per stream
 
 // Shared memory of one stream: Q tile, one K tile, one V tile, and a 64-column output staging panel.
 template <int D>
@@ -292,13 +292,13 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     const uint32_t smem_base = smem_base0 + st * SM::STREAM_BYTES;
     uint8_t* smem_gen = smem_gen0 + st * SM::STREAM_BYTES;
 
-    enum { B_QF = 0, B_QE = 1, B_KF = 2, B_KE = 3, B_VF = 4, B_VE = 5, B_SF = 6, B_PF = 7, B_OF = 8 };
+    enum { B_QF = 0, B_QE = 1, B_KF = 2, B_KE = 3, B_VF = 4, B_VE = 5, B_SF = 6, B_PF = 8, B_OF = 10 };
     auto bar = [&](int i) { return smem_u32(&bars[st * NBAR + i]); };
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
         for (int s2 = 0; s2 < 2; ++s2)
-            for (int i = 0; i < NBAR; ++i) mbar_init(smem_u32(&bars[s2 * NBAR + i]), i == B_PF ? 128 : 1);
+            for (int i = 0; i < NBAR; ++i) mbar_init(smem_u32(&bars[s2 * NBAR + i]), (i == B_PF || i == B_PF + 1) ? 128 : 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // zero the operand buffers once: rows a TMA box does not cover keep finite contents
@@ -372,7 +372,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
         {
             // instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128
-            constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+            constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
             constexpr uint32_t IDESC_PV =
                 (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
             uint32_t gs = 0, tcount = 0;
@@ -380,46 +380,61 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             const uint64_t qd = smem_desc(smem_base + SM::Q_OFF, 16, 1024);
             const uint64_t kd = smem_desc(smem_base + SM::K_OFF, 16, 1024);
             const uint64_t vd = smem_desc(smem_base + SM::V_OFF, SM::PANEL_BYTES, 1024);
-            auto issue_s = [&](uint32_t g) -> bool {
-                if (!__all_sync(0xffffffffu, mbar_wait(bar(B_KF), g & 1, abortp, p.status))) return false;
-                tc_fence_after();
+            // scores of keys [64h, 64h+64) of the staged key tile -> score buffer h (64 columns)
+            auto issue_s = [&](int h, bool last) {
                 if (elect_one()) {
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
-                        // descriptor start addresses are in 16-byte units
+                        // descriptor start addresses are in 16-byte units; 64 key rows are 8192 bytes further
                         const uint64_t off = (uint64_t)(((kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32) >> 4);
-                        mma_ss(tmem, qd + off, kd + off, IDESC_S, kk > 0);
+                        mma_ss(tmem + h * 64, qd + off, kd + off + (uint64_t)((h * 8192) >> 4), IDESC_S, kk > 0);
                     }
-                    tc_commit(bar(B_SF));
-                    tc_commit(bar(B_KE));
+                    tc_commit(bar(B_SF + h));
+                    if (last) tc_commit(bar(B_KE));
                 }
                 __syncwarp();
-                return true;
+            };
+            // O += P_h V[64h .. 64h+63]: four instructions of 16 keys, P read from TMEM over score buffer h
+            auto issue_pv = [&](int h, bool first) {
+                if (elect_one()) {
+#pragma unroll
+                    for (int k4 = 0; k4 < 4; ++k4)
+                        mma_ts(tmem + 128, tmem + h * 64 + k4 * 8, vd + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_PV,
+                               !first || (k4 > 0));
+                    tc_commit(bar(B_OF));
+                    if (h == 1) tc_commit(bar(B_VE));
+                }
+                __syncwarp();
             };
             for (int w = w0; w < total_work && ok; w += nstreams, ++tcount) {
                 const int rank = w / p.BH;
                 TileDesc td;
                 decode_tile(p, rank, td);
-                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_QF), tcount & 1, abortp, p.status));
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_QF), tcount & 1, abortp, p.status) &&
+                                                 mbar_wait(bar(B_KF), gs & 1, abortp, p.status));
                 if (!ok) break;
                 tc_fence_after();
-                ok = issue_s(gs);
+                issue_s(0, false);
+                issue_s(1, true);
                 for (int j = 0; j < td.nsteps && ok; ++j, ++gs) {
                     const uint32_t ph = gs & 1;
+                    const bool more = j + 1 < td.nsteps;
                     ok = __all_sync(0xffffffffu, mbar_wait(bar(B_PF), ph, abortp, p.status) &&
                                                      mbar_wait(bar(B_VF), ph, abortp, p.status));
                     if (!ok) break;
                     tc_fence_after();
-                    if (elect_one()) {
-#pragma unroll
-                        for (int kk = 0; kk < 8; ++kk)   // 16 keys per instruction, P read from TMEM
-                            mma_ts(tmem + 128, tmem + kk * 8, vd + (uint64_t)((kk * 2048) >> 4), IDESC_PV,
-                                   (j > 0) || (kk > 0));
-                        tc_commit(bar(B_OF));
-                        tc_commit(bar(B_VE));
+                    issue_pv(0, j == 0);
+                    if (more) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar(B_KF), (gs + 1) & 1, abortp, p.status));
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_s(0, false);
                     }
-                    __syncwarp();
-                    if (j + 1 < td.nsteps) ok = issue_s(gs + 1);
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_PF + 1), ph, abortp, p.status));
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(1, false);
+                    if (more) issue_s(1, true);
                     else {
                         if (elect_one()) tc_commit(bar(B_QE));
                         __syncwarp();
@@ -452,85 +467,90 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             // output accumulator in TMEM is rescaled once.  Probabilities stay below 2^8.
             float m_used = -INFINITY, l = 0.f;
 
-            for (int j = 0; j < td.nsteps; ++j, ++gs) {
+            for (int j = 0; j < td.nsteps && ok; ++j, ++gs) {
                 KTile kt;
                 step_ktile(p, td, j, kt);
                 int lo, hi2;
                 row_interval(p.view[kt.view], kt, rc, ro, rr, row_valid, lo, hi2);
-                const bool full = __all_sync(0xffffffffu, lo <= 0 && hi2 >= 128);
                 const uint32_t span = (uint32_t)(hi2 - lo);
-                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF), gs & 1, abortp, p.status));
-                if (!ok) break;
-                tc_fence_after();
-                uint32_t s[128];
-                tmem_ld32(s_addr, s);
-                tmem_ld32(s_addr + 32, s + 32);
-                tmem_ld32(s_addr + 64, s + 64);
-                tmem_ld32(s_addr + 96, s + 96);
-                tmem_wait_ld();
-                if (!full) {
+                // the 128 keys of the step are handled as two halves of 64, each with its own score buffer,
+                // so the tensor pipe works on one half while this warpgroup works on the other
 #pragma unroll
-                    for (int e = 0; e < 128; ++e)
-                        if ((uint32_t)(e - lo) >= span) s[e] = 0xff800000u;   // -inf: the key is blocked for this row
-                }
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-                for (int e = 0; e < 128; e += 8) {
-                    mx0 = max3(mx0, __uint_as_float(s[e]), __uint_as_float(s[e + 1]));
-                    mx1 = max3(mx1, __uint_as_float(s[e + 2]), __uint_as_float(s[e + 3]));
-                    mx2 = max3(mx2, __uint_as_float(s[e + 4]), __uint_as_float(s[e + 5]));
-                    mx3 = max3(mx3, __uint_as_float(s[e + 6]), __uint_as_float(s[e + 7]));
-                }
-                const float mrow = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
-                const bool need = mrow > m_used + 8.f;
-                if (j > 0 && __any_sync(0xffffffffu, need)) {
-                    // rescale the accumulated output: wait until P.V(j-1) has landed in TMEM
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF), (gs - 1) & 1, abortp, p.status));
+                for (int h = 0; h < 2; ++h) {
+                    const bool full = __all_sync(0xffffffffu, lo <= 64 * h && hi2 >= 64 * h + 64);
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF + h), gs & 1, abortp, p.status));
                     if (!ok) break;
                     tc_fence_after();
-                    const float alpha = need ? fast_ex2(m_used - mrow) : 1.f;
+                    const uint32_t sh_addr = s_addr + h * 64;
+                    uint32_t s[64];
+                    tmem_ld32(sh_addr, s);
+                    tmem_ld32(sh_addr + 32, s + 32);
+                    tmem_wait_ld();
+                    if (!full) {
 #pragma unroll
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t r[32];
-                        tmem_ld32(o_addr + c * 32, r);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-                        tmem_st32(o_addr + c * 32, r);
+                        for (int e = 0; e < 64; ++e)
+                            if ((uint32_t)(64 * h + e - lo) >= span) s[e] = 0xff800000u;   // -inf: blocked for this row
                     }
-                    l *= alpha;
-                }
-                if (need) m_used = mrow;
-                const float neg_ref = (m_used == -INFINITY) ? 0.f : -m_used;
-                const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nr2 = pack2(neg_ref, neg_ref);
-                uint64_t lsa = pack2(0.f, 0.f), lsb = lsa;
+                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int e = 0; e < 32; e += 4) {
-                        float x0, x1, x2, x3;
-                        unpack2(fma2(pack2(__uint_as_float(s[c * 32 + e]), __uint_as_float(s[c * 32 + e + 1])), sc2, nr2), x0, x1);
-                        unpack2(fma2(pack2(__uint_as_float(s[c * 32 + e + 2]), __uint_as_float(s[c * 32 + e + 3])), sc2, nr2), x2, x3);
-                        const float p0 = fast_ex2(x0), p1 = fast_ex2(x1), p2 = fast_ex2(x2), p3 = fast_ex2(x3);
-                        lsa = add2(lsa, pack2(p0, p1));
-                        lsb = add2(lsb, pack2(p2, p3));
-                        pk[e >> 1] = pack_bf16(p0, p1);
-                        pk[(e >> 1) + 1] = pack_bf16(p2, p3);
+                    for (int e = 0; e < 64; e += 8) {
+                        mx0 = max3(mx0, __uint_as_float(s[e]), __uint_as_float(s[e + 1]));
+                        mx1 = max3(mx1, __uint_as_float(s[e + 2]), __uint_as_float(s[e + 3]));
+                        mx2 = max3(mx2, __uint_as_float(s[e + 4]), __uint_as_float(s[e + 5]));
+                        mx3 = max3(mx3, __uint_as_float(s[e + 6]), __uint_as_float(s[e + 7]));
                     }
-                    tmem_st16(s_addr + c * 16, pk);   // P over the scores: keys 32c..32c+31 -> columns 16c..16c+15
+                    const float mrow = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
+                    const bool need = mrow > m_used + 8.f;
+                    if ((j > 0 || h > 0) && __any_sync(0xffffffffu, need)) {
+                        // rescale the accumulated output: wait until the previous P.V has landed in TMEM
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF), (2 * gs + h - 1) & 1, abortp, p.status));
+                        if (!ok) break;
+                        tc_fence_after();
+                        const float alpha = need ? fast_ex2(m_used - mrow) : 1.f;
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t r[32];
+                            tmem_ld32(o_addr + c * 32, r);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+                            tmem_st32(o_addr + c * 32, r);
+                        }
+                        l *= alpha;
+                    }
+                    if (need) m_used = mrow;
+                    const float neg_ref = (m_used == -INFINITY) ? 0.f : -m_used;
+                    const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nr2 = pack2(neg_ref, neg_ref);
+                    uint64_t lsa = pack2(0.f, 0.f), lsb = lsa;
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4) {
+                            float x0, x1, x2, x3;
+                            unpack2(fma2(pack2(__uint_as_float(s[c * 32 + e]), __uint_as_float(s[c * 32 + e + 1])), sc2, nr2), x0, x1);
+                            unpack2(fma2(pack2(__uint_as_float(s[c * 32 + e + 2]), __uint_as_float(s[c * 32 + e + 3])), sc2, nr2), x2, x3);
+                            const float p0 = fast_ex2(x0), p1 = fast_ex2(x1), p2 = fast_ex2(x2), p3 = fast_ex2(x3);
+                            lsa = add2(lsa, pack2(p0, p1));
+                            lsb = add2(lsb, pack2(p2, p3));
+                            pk[e >> 1] = pack_bf16(p0, p1);
+                            pk[(e >> 1) + 1] = pack_bf16(p2, p3);
+                        }
+                        tmem_st16(sh_addr + c * 16, pk);   // P over the scores: 32 keys -> 16 columns
+                    }
+                    {
+                        float a0, a1, b0, b1;
+                        unpack2(lsa, a0, a1);
+                        unpack2(lsb, b0, b1);
+                        l += (a0 + a1) + (b0 + b1);
+                    }
+                    tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(bar(B_PF + h));
                 }
-                {
-                    float a0, a1, b0, b1;
-                    unpack2(lsa, a0, a1);
-                    unpack2(lsb, b0, b1);
-                    l += (a0 + a1) + (b0 + b1);
-                }
-                tmem_wait_st();
-                tc_fence_before();
-                mbar_arrive(bar(B_PF));
             }
-            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF), (gs - 1) & 1, abortp, p.status));
+            // the last P.V of the tile is half-step 2*gs - 1
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF), (2 * gs - 1) & 1, abortp, p.status));
             if (ok) tc_fence_after();
 
             // epilogue: normalise, round to bf16, stage 64 output columns at a time in shared
