@@ -19,23 +19,29 @@
 //   repetition rows x own memory zone                  key chunk == row chunk   (Eq. 1, row 3)
 //   repetition rows x themselves                       diagonal                 (I of Eq. 1)
 //
-// One CTA (320 threads) per SM, persistent over a statically ordered tile list
-// (longest tiles first, (batch, head) fastest).  Roles:
-//   warps 0-7  two softmax warpgroups, thread = query row = TMEM lane; warpgroup g
-//              takes every other key tile (score buffer g): one pass over the
-//              scores (row max, exp2, row sum, bf16 P written back over the
-//              scores); its output accumulates in TMEM buffer g and is rescaled
-//              only when a row maximum has grown by more than 2^8; the two
-//              partial outputs are merged in the epilogue and staged in shared
-//              memory for a TMA store
-//   warp 8     TMA producer: Q per tile, K and V rings of two stages each
-//   warp 9     MMA issuer: S = Q K^T (both operands in shared memory), then
-//              P.V with P read from TMEM and V as an MN-major shared operand
-// TMEM (512 columns): two score buffers and two output accumulators of 128
-// columns, so the tensor pipe computes S(j+1) and P.V(j-1) while the softmax
-// warps work on S(j).  Every mbarrier wait is bounded: on expiry the CTA records
-// LOMA_ERR_TIMEOUT, all roles leave their loops, TMEM is freed and the kernel
-// returns.
+// One CTA (384 threads) per SM, persistent.  A CTA runs two independent "streams": each stream
+// owns a query tile at a time and has its own shared-memory buffers (Q, one K tile, one V tile,
+// a 64-column output staging panel), its own quarter of TMEM (two 64-column score buffers and a
+// 128-column output accumulator) and its own warps:
+//   warps 0-3 / 4-7   softmax warpgroup of stream 0 / 1: thread = query row = TMEM lane.  The 128
+//                     keys of a step are taken as two halves of 64: read the scores of a half,
+//                     row maximum (three-input max), probabilities 2^(s*scale - ref) with packed
+//                     two-wide fp32 FMA/ADD, bf16 P written back over the scores.  The output
+//                     accumulates in TMEM; the reference maximum only moves, and the accumulator
+//                     is only rescaled, when a row maximum has grown by more than 2^8.  Epilogue:
+//                     normalise, round to bf16, stage 64 columns at a time, TMA store.
+//   warp 8 / 9        TMA producer of stream 0 / 1 (one lane): Q per tile, K and V per step
+//   warp 10 / 11      MMA issuer of stream 0 / 1: the warp's control flow is uniform and one
+//                     elected lane issues, so descriptors stay in uniform registers (issuing from
+//                     a divergent single-lane branch halved the tensor throughput).  Per step:
+//                     S_h = Q K_h^T for both halves (operands in shared memory, N = 64), and
+//                     O += P_h V_h with P read from TMEM and V as an MN-major shared operand.
+//                     S_h of the next step is issued right after P_h V_h of this one, so the
+//                     tensor pipe works on one half while the warpgroup works on the other.
+// The two streams fill each other's waits (tensor latency, TMEM loads, epilogues).  Tiles are dealt
+// to the 2*gridDim.x streams round robin from a statically ordered list (longest first, (batch,
+// head) fastest).  Every mbarrier wait is bounded: on expiry the CTA records LOMA_ERR_TIMEOUT, all
+// roles leave their loops, TMEM is freed and the kernel returns.
 #include <cuda.h>
 #include <math.h>
 
@@ -258,7 +264,7 @@ __device__ __forceinline__ void half_exp(const uint32_t (&a)[64], uint32_t p_add
 // ------------------------------------------------------------------ the kernel
 constexpr int TC_THREADS = 384;   // 2 softmax warpgroups + 1 warpgroup with 2 TMA warps and 2 MMA warps
 constexpr int TMEM_COLS = 512;
-constexpr int NBAR = 11;          // mbarriers per stream
+constexpr int NBAR = 12;          // mbarriers per stream
 
 // Shared memory of one stream: Q tile, one K tile, one V tile, and a 64-column output staging panel.
 template <int D>
@@ -401,7 +407,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     for (int k4 = 0; k4 < 4; ++k4)
                         mma_ts(tmem + 128, tmem + h * 64 + k4 * 8, vd + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_PV,
                                !first || (k4 > 0));
-                    tc_commit(bar(B_OF));
+                    tc_commit(bar(B_OF + h));   // one barrier per half: each completes exactly once per step
                     if (h == 1) tc_commit(bar(B_VE));
                 }
                 __syncwarp();
@@ -503,7 +509,9 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     const bool need = mrow > m_used + 8.f;
                     if ((j > 0 || h > 0) && __any_sync(0xffffffffu, need)) {
                         // rescale the accumulated output: wait until the previous P.V has landed in TMEM
-                        ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF), (2 * gs + h - 1) & 1, abortp, p.status));
+                        // (the other half's product of this step, or the second half's of the step before)
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + (h ^ 1)), (h == 0 ? gs - 1 : gs) & 1, abortp,
+                                                               p.status));
                         if (!ok) break;
                         tc_fence_after();
                         const float alpha = need ? fast_ex2(m_used - mrow) : 1.f;
@@ -549,8 +557,8 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     mbar_arrive(bar(B_PF + h));
                 }
             }
-            // the last P.V of the tile is half-step 2*gs - 1
-            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF), (2 * gs - 1) & 1, abortp, p.status));
+            // the last P.V of the tile is the second half of step gs - 1 (products complete in issue order)
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + 1), (gs - 1) & 1, abortp, p.status));
             if (ok) tc_fence_after();
 
             // epilogue: normalise, round to bf16, stage 64 output columns at a time in shared
