@@ -337,7 +337,21 @@ def run_ours(args):
                      "note": "timed in place after the 64 decodes of the cycle"},
         "roofline": {"kernel": "decode_splitkv_kernel<128> (+ merge), per loma_decode_attn call", "bound": "hbm",
                      "achieved": dec_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                     "frac": dec_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None},
+                     "frac": dec_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                     # dram__bytes_read + write of one launch: captured on the B8 case (1.084e9 bytes for 1.0779e9
+                     # algorithmic, profiles/decode_splitkv_B8_H32_L8224.md) and scaled by the (b,h) count, 1024 / 256
+                     "traffic": 1.084e9 * (g["B"] * g["H"]) / 256.0,
+                     "traffic_source": "ncu small case x4"},
+        "roofline_other_kernels": [
+            {"kernel": "masked_attn_tc_kernel<128>", "workload": "4608-token layout", "bound": "hbm",
+             "achieved": fwd_bytes / (t_fwd * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+             "frac": fwd_bytes / (t_fwd * 1e-3) / 1e9 / peaks["hbm_gbs"],
+             "traffic": 141.3e6 * f["B"],   # ncu, one batch element (profiles/masked_attn_tc_small_cases.md) x B
+             "tensor_frac_of_measured_bf16_useful": fwd_tflops / world / peaks["bf16_tflops"]},
+            {"kernel": "compress_mma_kernel<128>", "workload": "B32 H32 mem 8192, default variant", "bound": "hbm",
+             "achieved": cmp_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": cmp_gbs / peaks["hbm_gbs"],
+             "traffic": None, "note": "launch-latency bound: 59 MB in one ~35 us launch"},
+        ],
         "e2e": {"value": world * fwd_flops / (e2e_fwd * 1e-3) / 1e12, "unit": "TFLOP/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_tot,
                 "masked_fwd_ms": e2e_fwd, "decode_cycle_ms": e2e_dec,
