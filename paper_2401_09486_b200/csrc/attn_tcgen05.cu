@@ -323,10 +323,12 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     const uint32_t tmem = tmem_slot + st * 256;   // this stream's scores at +0, output accumulator at +128
     volatile int* abortp = &abort_flag;
 
-    // tiles are dealt to the 2*gridDim.x streams round robin, longest first
+    // Tiles (longest first) are dealt to the 2*gridDim.x streams in rounds, forwards in even rounds
+    // and backwards in odd ones, so no stream always receives the longest tile of a round.
     const int total_work = p.total_tiles * p.BH;
     const int nstreams = 2 * gridDim.x;
-    const int w0 = blockIdx.x + st * gridDim.x;
+    const int sid = blockIdx.x + st * gridDim.x;
+    auto tile_of_round = [&](int r) { return r * nstreams + ((r & 1) ? nstreams - 1 - sid : sid); };
 
     if (warp == 8 || warp == 9) {
         // ------------------------------------------------------------ TMA producer of stream st
@@ -334,7 +336,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         if (lane == 0) {
             uint32_t gs = 0, tcount = 0;
             bool ok = true;
-            for (int w = w0; w < total_work && ok; w += nstreams, ++tcount) {
+            for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
                 const int rank = w / p.BH, bh = w - rank * p.BH;
                 const int bi = bh / p.H, hi = bh - bi * p.H;
                 TileDesc td;
@@ -412,7 +414,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 }
                 __syncwarp();
             };
-            for (int w = w0; w < total_work && ok; w += nstreams, ++tcount) {
+            for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
                 const int rank = w / p.BH;
                 TileDesc td;
                 decode_tile(p, rank, td);
@@ -457,7 +459,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         uint32_t gs = 0;
         bool ok = true;
         bool store_pending = false;
-        for (int w = w0; w < total_work && ok; w += nstreams) {
+        for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r)) {
             const int rank = w / p.BH, bh = w - rank * p.BH;
             const int bi = bh / p.H, hi = bh - bi * p.H;
             TileDesc td;
