@@ -127,7 +127,7 @@ def run_ours(args):
     import torch.distributed as dist
 
     from paper_2401_09486_b200 import binding as L
-    from paper_2401_09486_b200 import build, synthetic
+    from paper_2401_09486_b200 import build, multi_gpu, synthetic
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -156,19 +156,19 @@ def run_ours(args):
     S = f["n"] * (2 * tc_f + f["t"])
     std = 1.0 / math.sqrt(f["D"])
     bf = torch.bfloat16
-    q, k, v = (synthetic.big_normal_(torch.empty(f["B"], f["H"], S, f["D"], dtype=bf, device=dev), 1000 + 10 * rank + i,
+    q, k, v = (synthetic.big_normal_(torch.empty(f["B"], f["H"], S, f["D"], dtype=bf, device=dev), multi_gpu.rank_seed(1000, rank, i),
                                      std) for i in range(3))
     o = torch.empty_like(q)
     tc_g = g["c"] * g["t"]
     cap = g["mem_len"] + tc_g + g["t"]
-    kc = synthetic.big_normal_(torch.empty(g["B"], g["H"], cap, g["D"], dtype=bf, device=dev), 2000 + 10 * rank, std)
-    vc = synthetic.big_normal_(torch.empty(g["B"], g["H"], cap, g["D"], dtype=bf, device=dev), 2001 + 10 * rank, std)
+    kc = synthetic.big_normal_(torch.empty(g["B"], g["H"], cap, g["D"], dtype=bf, device=dev), multi_gpu.rank_seed(2000, rank), std)
+    vc = synthetic.big_normal_(torch.empty(g["B"], g["H"], cap, g["D"], dtype=bf, device=dev), multi_gpu.rank_seed(2001, rank), std)
     # one (q, k_new, v_new) triple per decode step of the cycle, and the memory-token triple
     dq, dk, dv = (synthetic.big_normal_(torch.empty(tc_g, g["B"], g["H"], 1, g["D"], dtype=bf, device=dev),
-                                        2100 + 10 * rank + i, std) for i in range(3))
+                                        multi_gpu.rank_seed(2100, rank, i), std) for i in range(3))
     do = torch.empty_like(dq)
     qm, km, vm = (synthetic.big_normal_(torch.empty(g["B"], g["H"], g["t"], g["D"], dtype=bf, device=dev),
-                                        2200 + 10 * rank + i, std) for i in range(3))
+                                        multi_gpu.rank_seed(2200, rank, i), std) for i in range(3))
     om = torch.empty_like(qm)
     ws_bytes = max(16, L.loma_decode_workspace_bytes(g["B"], g["H"], g["D"], cap),
                    L.loma_compress_workspace_bytes(g["B"], g["H"], g["D"], g["t"], g["mem_len"], 0))
@@ -232,11 +232,8 @@ def run_ours(args):
     phase_ms = {kk: vv / args.steps for kk, vv in phase_ms.items()}
 
     # max over ranks of every time
-    times = torch.tensor([total_ms] + [phase_ms[x] for x in ("index", "masked_fwd", "decode", "compress")],
-                         dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, t_index, t_fwd, t_dec, t_cmp = times.tolist()
+    total_ms, t_index, t_fwd, t_dec, t_cmp = multi_gpu.max_over_ranks(
+        [total_ms] + [phase_ms[x] for x in ("index", "masked_fwd", "decode", "compress")], dev)
     ms_per_step = total_ms / args.steps
 
     # ---------------- e2e: host buffers, copies inside the timed region ----------------
@@ -281,17 +278,15 @@ def run_ours(args):
         e2e_fwd += marks[0][1].elapsed_time(marks[1][1])
         e2e_dec += marks[1][1].elapsed_time(marks[2][1])
         e2e_tot += marks[0][1].elapsed_time(marks[3][1])
-    et = torch.tensor([e2e_fwd / e2e_steps, e2e_dec / e2e_steps, e2e_tot / e2e_steps], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(et, op=dist.ReduceOp.MAX)
-    e2e_fwd, e2e_dec, e2e_tot = et.tolist()
+    e2e_fwd, e2e_dec, e2e_tot = multi_gpu.max_over_ranks(
+        [e2e_fwd / e2e_steps, e2e_dec / e2e_steps, e2e_tot / e2e_steps], dev)
 
     # ---------------- figures ----------------
     peaks = load_peaks()
     pairs = allowed_pairs(f["n"], f["c"], f["t"])
     fwd_flops = 4.0 * f["D"] * pairs * f["B"] * f["H"]                 # per GPU
     fwd_bytes = 4.0 * q.numel() * 2                                    # Q, K, V read + O written once
-    fwd_tflops = world * fwd_flops / (t_fwd * 1e-3) / 1e12
+    fwd_tflops = multi_gpu.job_throughput(fwd_flops, world, t_fwd) / 1e12
     # decode: algorithmic bytes = every visible K and V row read once (cache_len + 1 rows per (b,h))
     dec_rows = sum(g["mem_len"] + j + 1 for j in range(tc_g))
     dec_bytes_cycle = 2.0 * dec_rows * g["B"] * g["H"] * g["D"] * 2

@@ -8,4 +8,4 @@ the library; the first call through the binding does, and fails loudly if the
 library has not been built.
 """
 
-__all__ = ["binding", "synthetic", "build"]
+__all__ = ["binding", "synthetic", "build", "multi_gpu"]
