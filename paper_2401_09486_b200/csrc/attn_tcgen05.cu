@@ -716,25 +716,31 @@ cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, v
         maps = cached_maps;
     }
 
-    int dev = 0, sms = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    // per-device set-up, done once: SM count and the opt-in to large dynamic shared memory
+    static int sm_count[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (sm_count[dev] == 0) {
+        int sms = 0;
+        cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(masked_attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TcSmem<128>::TOTAL + 1024);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(masked_attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TcSmem<64>::TOTAL + 1024);
+        if (e != cudaSuccess) return e;
+        sm_count[dev] = sms;
+    }
+    const int sms = sm_count[dev];
     const int64_t work = (int64_t)p.total_tiles * p.BH;
     const int64_t want = (work + 1) / 2;            // two streams (query tiles in flight) per CTA
     const int grid = (int)(want < sms ? want : sms);
-    cudaError_t e;
     // the shared-memory footprint also keeps one CTA per SM (each allocates all 512 TMEM columns)
-    if (D == 128) {
-        const int smem = TcSmem<128>::TOTAL + 1024;
-        e = cudaFuncSetAttribute(masked_attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-        masked_attn_tc_kernel<128><<<grid, TC_THREADS, smem, st>>>(maps, p);
-    } else {
-        const int smem = TcSmem<64>::TOTAL + 1024;
-        e = cudaFuncSetAttribute(masked_attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-        masked_attn_tc_kernel<64><<<grid, TC_THREADS, smem, st>>>(maps, p);
-    }
+    if (D == 128)
+        masked_attn_tc_kernel<128><<<grid, TC_THREADS, TcSmem<128>::TOTAL + 1024, st>>>(maps, p);
+    else
+        masked_attn_tc_kernel<64><<<grid, TC_THREADS, TcSmem<64>::TOTAL + 1024, st>>>(maps, p);
     count_launches(1);
     return cudaGetLastError();
 }

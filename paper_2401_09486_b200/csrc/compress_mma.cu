@@ -339,8 +339,15 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
     if (nprior > 0) prior_len = ((mem_len + nprior - 1) / nprior + 15) / 16 * 16;
     const int nsp = nprior + 1;
     const int smem = CmpSmem<D>::TOTAL;
-    cudaError_t e = cudaFuncSetAttribute(compress_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
+    cudaError_t e;
+    static bool attr_set[64] = {false};   // per device, per template instance
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
+        e = cudaFuncSetAttribute(compress_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
     compress_mma_kernel<D><<<BH * nsp, CMP_WARPS * 32, smem, st>>>(
         static_cast<const __nv_bfloat16*>(qm), static_cast<const __nv_bfloat16*>(km),
         static_cast<const __nv_bfloat16*>(vm), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
