@@ -290,6 +290,13 @@ LOMA_API size_t loma_compress_workspace_bytes(int B, int H, int D, int t, int me
  * LOMA_ERR_CUDA if the synchronisation or the read fails. */
 LOMA_API int loma_device_status(void* stream);
 
+/* Failure-detection self test: enqueues a one-thread kernel that waits, with the library's bounded
+ * wait, on a barrier nobody ever signals.  After about a millisecond the wait gives up, the kernel
+ * records LOMA_ERR_TIMEOUT in the device status word and returns normally (no trap, the context
+ * stays usable); the next loma_device_status() then returns LOMA_ERR_TIMEOUT once.
+ * Errors: UNSUPPORTED (device), CUDA. */
+LOMA_API int loma_selftest_bounded_wait(void* stream);
+
 /* Number of kernels this library has enqueued in the calling process since it
  * was loaded (all devices, all streams).  Host-side counter; never fails. */
 LOMA_API uint64_t loma_launch_count(void);

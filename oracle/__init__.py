@@ -11,6 +11,7 @@ CUDA path never calls it.
 
 from .loma_oracle import (  # noqa: F401
     FLAG_MEM_SEES_PRIOR_MEM,
+    FLAG_NO_REP_ZONE,
     ZONE_READ,
     ZONE_MEM,
     ZONE_REP,

@@ -37,6 +37,10 @@ from __future__ import annotations
 import numpy as np
 
 FLAG_MEM_SEES_PRIOR_MEM = 1
+# Inference layout: chunks are [tc reading | t memory] with no repetition zone, i.e. the sequence the
+# generator of Section 3.1 / Appendix A actually feeds the model (the <r> rows exist only for the
+# training loss, Section 4.2).  The mask is Eq. 2 with the repetition rows and columns deleted.
+FLAG_NO_REP_ZONE = 2
 
 ZONE_READ = 0
 ZONE_MEM = 1
@@ -47,23 +51,26 @@ ZONE_REP = 2
 # Layout (Section 4.1) and index maps (Eq. 14, Appendix A)
 # --------------------------------------------------------------------------
 
-def chunk_len(c: int, t: int) -> int:
-    """s = t(2c+1): reading zone + memory zone + repetition zone (Section 4.3)."""
+def chunk_len(c: int, t: int, flags: int = 0) -> int:
+    """s = t(2c+1): reading zone + memory zone + repetition zone (Section 4.3);
+    t(c+1) in the inference layout, which has no repetition zone."""
+    if flags & FLAG_NO_REP_ZONE:
+        return t * (c + 1)
     return t * (2 * c + 1)
 
 
-def seq_len(n_chunks: int, c: int, t: int, tail_read: int = 0) -> int:
+def seq_len(n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0) -> int:
     """Length of the laid-out sequence: n complete chunks plus a reading tail."""
-    return n_chunks * chunk_len(c, t) + tail_read
+    return n_chunks * chunk_len(c, t, flags) + tail_read
 
 
-def decompose(i: int, n_chunks: int, c: int, t: int):
+def decompose(i: int, n_chunks: int, c: int, t: int, flags: int = 0):
     """Row index -> (chunk y, zone z, offset o inside the zone) (Section 4.1).
 
     Rows past the last complete chunk form the reading zone of chunk n_chunks.
     """
     tc = t * c
-    s = chunk_len(c, t)
+    s = chunk_len(c, t, flags)
     if s == 0 or i >= n_chunks * s:
         return n_chunks, ZONE_READ, i - n_chunks * s
     y, r = divmod(i, s)
@@ -74,7 +81,7 @@ def decompose(i: int, n_chunks: int, c: int, t: int):
     return y, ZONE_REP, r - tc - t
 
 
-def layout_index(n_chunks: int, c: int, t: int, tail_read: int = 0):
+def layout_index(n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0):
     """Integer maps over the rows of the laid-out sequence.
 
     Returns int32 arrays (chunk, zone, offset, src_token, pos_id), each [S].
@@ -86,14 +93,14 @@ def layout_index(n_chunks: int, c: int, t: int, tail_read: int = 0):
                  the reading position (paper silent, unpinned).
     """
     tc = t * c
-    S = seq_len(n_chunks, c, t, tail_read)
+    S = seq_len(n_chunks, c, t, tail_read, flags)
     chunk = np.zeros(S, np.int32)
     zone = np.zeros(S, np.int32)
     offset = np.zeros(S, np.int32)
     src = np.zeros(S, np.int32)
     pos = np.zeros(S, np.int32)
     for i in range(S):
-        y, z, o = decompose(i, n_chunks, c, t)
+        y, z, o = decompose(i, n_chunks, c, t, flags)
         chunk[i], zone[i], offset[i] = y, z, o
         if z == ZONE_MEM:
             src[i] = -1
@@ -139,7 +146,7 @@ def generation_index(n_tokens: int, c: int, t: int):
 # Mask (Eq. 1-3)
 # --------------------------------------------------------------------------
 
-def chunk_mask(c: int, t: int) -> np.ndarray:
+def chunk_mask(c: int, t: int, flags: int = 0) -> np.ndarray:
     """Eq. 1: the s x s mask of one training chunk, as a boolean array.
 
         [ L  0  0 ]   reading rows: causal inside the reading zone
@@ -151,11 +158,14 @@ def chunk_mask(c: int, t: int) -> np.ndarray:
     I = np.eye(tc, dtype=bool)
     Z = lambda a, b: np.zeros((a, b), bool)
     O = lambda a, b: np.ones((a, b), bool)
-    return np.block([
+    M = np.block([
         [L,         Z(tc, t), Z(tc, tc)],
         [O(t, tc),  O(t, t),  Z(t, tc)],
         [Z(tc, tc), O(tc, t), I],
     ])
+    if flags & FLAG_NO_REP_ZONE:      # inference layout: the third block row and column do not exist
+        M = M[:tc + t, :tc + t]
+    return M
 
 
 def cross_chunk_block(c: int, t: int, flags: int = 0) -> np.ndarray:
@@ -170,6 +180,8 @@ def cross_chunk_block(c: int, t: int, flags: int = 0) -> np.ndarray:
     S[0:tc, tc:tc + t] = True
     if flags & FLAG_MEM_SEES_PRIOR_MEM:
         S[tc:tc + t, tc:tc + t] = True
+    if flags & FLAG_NO_REP_ZONE:
+        S = S[:tc + t, :tc + t]
     return S
 
 
@@ -181,11 +193,11 @@ def dense_mask(n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0
     tail_read rows/cols of one more chunk row: reading rows of Eq. 3 towards
     every earlier chunk and the leading corner of L on the diagonal.
     """
-    s = chunk_len(c, t)
-    S = seq_len(n_chunks, c, t, tail_read)
+    s = chunk_len(c, t, flags)
+    S = seq_len(n_chunks, c, t, tail_read, flags)
     M = np.zeros((S, S), bool)
     if n_chunks > 0:
-        Mc = chunk_mask(c, t)
+        Mc = chunk_mask(c, t, flags)
         Sc = cross_chunk_block(c, t, flags)
         for y in range(n_chunks):
             for x in range(y):
@@ -201,8 +213,8 @@ def dense_mask(n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0
 
 def allowed(i: int, j: int, n_chunks: int, c: int, t: int, flags: int = 0) -> bool:
     """May row i attend to column j?  Eq. 1-3 read entry by entry."""
-    yi, zi, oi = decompose(i, n_chunks, c, t)
-    yj, zj, oj = decompose(j, n_chunks, c, t)
+    yi, zi, oi = decompose(i, n_chunks, c, t, flags)
+    yj, zj, oj = decompose(j, n_chunks, c, t, flags)
     if yj > yi:
         return False                       # Eq. 2: zero above the block diagonal
     if yj == yi:                           # Eq. 1
@@ -225,8 +237,8 @@ def mask_rows(rows, n_chunks: int, c: int, t: int, tail_read: int = 0, flags: in
     For sequences whose full S x S mask does not fit in memory.  Returns a
     boolean [len(rows), S].
     """
-    S = seq_len(n_chunks, c, t, tail_read)
-    ch, zn, of, _, _ = layout_index(n_chunks, c, t, tail_read)
+    S = seq_len(n_chunks, c, t, tail_read, flags)
+    ch, zn, of, _, _ = layout_index(n_chunks, c, t, tail_read, flags)
     cols = np.arange(S)
     out = np.zeros((len(rows), S), bool)
     for r, i in enumerate(rows):
@@ -286,7 +298,7 @@ def masked_attn_fwd(q, k, v, n_chunks, c, t, tail_read=0, flags=0, scale=None,
     """
     q, k, v = _f64(q), _f64(k), _f64(v)
     B, H, S, D = q.shape
-    assert S == seq_len(n_chunks, c, t, tail_read)
+    assert S == seq_len(n_chunks, c, t, tail_read, flags)
     if rows is None:
         rows = np.arange(S)
         M = dense_mask(n_chunks, c, t, tail_read, flags)
@@ -398,7 +410,7 @@ def replay_generation(q, k, v, n_chunks, c, t, tail_read=0, flags=0, scale=None)
     q, k, v = np.asarray(q), np.asarray(k), np.asarray(v)
     B, H, S, D = q.shape
     tc = t * c
-    s = chunk_len(c, t)
+    s = chunk_len(c, t, flags)
     cap = n_chunks * t + max(tc, tail_read) + 1
     kc = np.zeros((B, H, cap, D), dtype=k.dtype)
     vc = np.zeros((B, H, cap, D), dtype=v.dtype)

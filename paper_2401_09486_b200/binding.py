@@ -41,6 +41,7 @@ SIGNATURES = {
                                 _p]),
     "loma_compress_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _u]),
     "loma_device_status": (_i, [_p]),
+    "loma_selftest_bounded_wait": (_i, [_p]),
     "loma_launch_count": (ctypes.c_uint64, []),
     "loma_status_string": (ctypes.c_char_p, [_i]),
     "loma_version": (_i, []),
@@ -109,6 +110,10 @@ def loma_version() -> int:
 
 def loma_launch_count() -> int:
     return int(lib().loma_launch_count())
+
+
+def loma_selftest_bounded_wait(stream=None) -> None:
+    _check(lib().loma_selftest_bounded_wait(_stream(stream)), "loma_selftest_bounded_wait")
 
 
 def loma_device_status(stream=None) -> int:

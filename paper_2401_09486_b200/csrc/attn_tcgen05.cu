@@ -625,6 +625,36 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     }
 }
 
+// ------------------------------------------------------------------ bounded-wait self test
+// One thread waits on an mbarrier that nobody ever arrives on, with the same wait routine as the
+// attention kernel but a limit of about a millisecond; it must give up, record LOMA_ERR_TIMEOUT in the
+// status word and return, leaving the context usable.
+__global__ void bounded_wait_selftest_kernel(int* status, long long limit_cycles) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const long long t0 = clock64();
+    const uint32_t b = smem_u32(&bar);
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(b, 0)) return;            // cannot happen: no arrival is ever made
+        if ((it & 63u) == 0 && clock64() - t0 > limit_cycles) {
+            abort_flag = 1;
+            atomicExch(status, (int)LOMA_ERR_TIMEOUT);
+            return;
+        }
+    }
+}
+
+cudaError_t launch_bounded_wait_selftest(cudaStream_t st) {
+    int* status = device_status_word();
+    if (!status) return cudaErrorUnknown;
+    bounded_wait_selftest_kernel<<<1, 1, 0, st>>>(status, 2000000ll);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,

@@ -256,6 +256,12 @@ int loma_compress_step(const void* q_mem, const void* k_mem, const void* v_mem, 
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 
+int loma_selftest_bounded_wait(void* stream) {
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    return launch_bounded_wait_selftest(static_cast<cudaStream_t>(stream)) == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
 int loma_device_status(void* stream) {
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return LOMA_ERR_CUDA;
     int* w = device_status_word();

@@ -39,6 +39,8 @@ cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, v
 
 void plan_coverage_host(const Layout& L, uint8_t* counts);   // tile_plan_host.cu
 
+cudaError_t launch_bounded_wait_selftest(cudaStream_t st);   // attn_tcgen05.cu
+
 cudaError_t launch_decode_generic(const void* q, const void* k_new, const void* v_new,
                                   void* k_cache, void* v_cache, void* o, float* lse,
                                   int B, int H, int D, int cap, int cache_len,

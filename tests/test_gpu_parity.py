@@ -269,6 +269,21 @@ def test_compress_matches_oracle_and_compacts_bit_exact(B, H, D, c, t, mem_len, 
     assert np.array_equal(bits(kcd[:, :, :mem_len]), bits(kc[:, :, :mem_len]))
 
 
+# ------------------------------------------------------- failure detection
+
+def test_bounded_wait_times_out_and_leaves_the_context_usable():
+    """A device-side wait that can never be satisfied gives up after its limit,
+    reports LOMA_ERR_TIMEOUT through the status word, and later launches work."""
+    assert L.loma_device_status() == 0
+    L.loma_selftest_bounded_wait()
+    assert L.loma_device_status() == -7          # LOMA_ERR_TIMEOUT, reported once
+    assert L.loma_device_status() == 0           # cleared by the read
+    q, k, v = (x.to(DEV) for x in synthetic.qkv(1, 1, 144, 128, seed=3, dtype=torch.bfloat16))
+    o, _ = run_fwd(q, k, v, 1, 4, 16)
+    want, _ = oracle.masked_attn_fwd(npf(q), npf(k), npf(v), 1, 4, 16)
+    check_close(o, want, torch.bfloat16)
+
+
 # ----------------------------------------------------------- repeatability
 
 def test_results_are_bitwise_repeatable():

@@ -444,6 +444,60 @@ def test_t0_generation_never_compresses_and_is_causal():
     assert length == S and np.allclose(Og, ref, atol=1e-13)
 
 
+# ------------------------------------------------ inference layout (no <r> zone)
+
+NOREP = oracle.FLAG_NO_REP_ZONE
+
+
+def test_inference_layout_mask_is_fig5_mask_without_repetition_rows_and_columns(golden_dir):
+    """Section 3.1 generates over [reading | memory] chunks only; the <r> rows exist for the training
+    loss (Section 4.2).  Deleting the repetition rows and columns from the hand-typed Fig. 5 mask must
+    give the inference-layout mask."""
+    full = _load_mask(os.path.join(golden_dir, "fig5_mask_t2_c2_n3.txt"))
+    keep = [i for i in range(30) if i % 10 < 6]
+    want = full[np.ix_(keep, keep)]
+    got = oracle.dense_mask(3, 2, 2, 0, NOREP)
+    assert got.shape == (18, 18) and np.array_equal(got, want)
+    ent = np.array([[oracle.allowed(i, j, 3, 2, 2, NOREP) for j in range(18)] for i in range(18)])
+    assert np.array_equal(ent, want)
+    assert np.array_equal(oracle.mask_rows(list(range(18)), 3, 2, 2, 0, NOREP), want)
+    full_p = _load_mask(os.path.join(golden_dir, "fig5_mask_t2_c2_n3_prior_mem.txt"))
+    assert np.array_equal(oracle.dense_mask(3, 2, 2, 0, NOREP | 1), full_p[np.ix_(keep, keep)])
+
+
+@pytest.mark.parametrize("n,c,t,tail", [(2, 4, 4, 0), (3, 2, 2, 3), (2, 3, 5, 1), (4, 1, 3, 0)])
+@pytest.mark.parametrize("prior", [0, 1])
+def test_inference_layout_equals_training_layout_on_shared_rows_and_replays(n, c, t, tail, prior):
+    """Reading and memory rows never see a repetition key, so their outputs over the inference layout
+    equal their outputs over the training layout built from the same rows; and incremental generation
+    (decode per token, compress per chunk) reproduces every row of the one-shot inference-layout pass."""
+    flags = NOREP | prior
+    S2 = oracle.seq_len(n, c, t, tail, flags)
+    assert S2 == n * t * (c + 1) + tail
+    D = 8
+    q2, k2, v2 = (_rand((1, 2, S2, D), sd) for sd in (190, 191, 192))
+    O2, lse2 = oracle.masked_attn_fwd(q2, k2, v2, n, c, t, tail, flags)
+    # embed into the training layout: repetition rows get unrelated values
+    S = oracle.seq_len(n, c, t, tail)
+    zone = oracle.layout_index(n, c, t, tail)[1]
+    live = np.nonzero(zone != oracle.ZONE_REP)[0]
+    q, k, v = (_rand((1, 2, S, D), sd) for sd in (193, 194, 195))
+    q[:, :, live], k[:, :, live], v[:, :, live] = q2, k2, v2
+    O, lse = oracle.masked_attn_fwd(q, k, v, n, c, t, tail, prior)
+    assert np.allclose(O[:, :, live], O2, atol=1e-13) and np.allclose(lse[:, :, live], lse2, atol=1e-13)
+    Og, kc, vc, length = oracle.replay_generation(q2, k2, v2, n, c, t, tail, flags)
+    assert not np.isnan(Og).any()
+    assert np.allclose(Og, O2, atol=1e-13)
+    ch2, zn2, of2, src2, pos2 = oracle.layout_index(n, c, t, tail, flags)
+    assert set(zn2.tolist()) <= {oracle.ZONE_READ, oracle.ZONE_MEM}
+    mem_rows = np.nonzero(zn2 == oracle.ZONE_MEM)[0].tolist()
+    tail_rows = list(range(n * t * (c + 1), S2))
+    assert length == len(mem_rows) + tail
+    assert np.array_equal(kc[:, :, :length], k2[:, :, mem_rows + tail_rows])
+    # positions of the shared rows agree with the training layout (Eq. 14)
+    assert pos2.tolist() == oracle.layout_index(n, c, t, tail)[4][live].tolist()
+
+
 # ------------------------------------------ planted mistakes must be caught
 
 def _run_core_pins(golden_dir):
@@ -462,14 +516,14 @@ def test_planted_mistakes_in_the_oracle_are_caught(monkeypatch, golden_dir):
     """Break the oracle (on the CPU) in plausible ways; the pins above must fail each time."""
     _run_core_pins(golden_dir)   # sanity: intact oracle passes
 
-    def broken_chunk_mask_no_identity(c, t):
-        M = orig_chunk_mask(c, t)
+    def broken_chunk_mask_no_identity(c, t, flags=0):
+        M = orig_chunk_mask(c, t, flags)
         tc = t * c
         M[tc + t:, tc + t:] = False            # dropped I block
         return M
 
-    def broken_chunk_mask_mem_causal(c, t):
-        M = orig_chunk_mask(c, t)
+    def broken_chunk_mask_mem_causal(c, t, flags=0):
+        M = orig_chunk_mask(c, t, flags)
         tc = t * c
         M[tc:tc + t, tc:tc + t] = np.tril(np.ones((t, t), bool))   # memory zone made causal
         return M
@@ -510,8 +564,8 @@ def test_planted_mistakes_in_the_oracle_are_caught(monkeypatch, golden_dir):
                 _run_core_pins(golden_dir)
 
     # index-map and cache plants
-    def broken_layout(n, c, t, tail_read=0):
-        ch, zn, of, src, pos = orig_layout(n, c, t, tail_read)
+    def broken_layout(n, c, t, tail_read=0, flags=0):
+        ch, zn, of, src, pos = orig_layout(n, c, t, tail_read, flags)
         pos = pos.copy()
         pos[zn == 1] -= c - 1                  # memory ids start at the chunk start instead of +c-1
         return ch, zn, of, src, pos
