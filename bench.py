@@ -190,7 +190,7 @@ def run_ours(args):
             if marks is not None:
                 e = ev(); e.record(stream); marks.append((name, e))
         mark("start")
-        rc = lib.loma_layout_index(f["n"], f["c"], f["t"], 0, *[P(x) for x in idx_fwd], 1, st)
+        rc = lib.loma_layout_index(f["n"], f["c"], f["t"], 0, 0, *[P(x) for x in idx_fwd], 1, st)
         rc |= lib.loma_generation_index(tc_g, g["c"], g["t"], *[P(x) for x in idx_gen], 1, st)
         mark("index")
         L.loma_masked_attn_fwd(q, k, v, o, None, f["n"], f["c"], f["t"], 0, 0, 0.0, stream)

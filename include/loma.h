@@ -83,6 +83,12 @@ enum {
      * the mem_len memory entries already in the cache; both change together so
      * that incremental generation still equals the one-shot forward. */
     LOMA_FLAG_MEM_SEES_PRIOR_MEM = 1u,
+    /* Inference layout: chunks are [tc reading | t memory] with no repetition zone (s = tc + t), the
+     * sequence Section 3.1 / Appendix A actually feed the model -- the <r> rows exist only for the
+     * training loss (Section 4.2).  The mask is Eq. 2 with the repetition rows and columns deleted.
+     * One pass of loma_masked_attn_fwd over a prompt laid out this way equals ingesting the prompt
+     * token by token with a compress pass per chunk. */
+    LOMA_FLAG_NO_REP_ZONE = 2u,
     /* Run the plain CUDA-core kernel even where a tensor-core kernel exists
      * (second opinion for tests; always used for LOMA_F32). */
     LOMA_FLAG_FORCE_GENERIC = 1u << 8
@@ -109,11 +115,12 @@ enum { LOMA_ZONE_READ = 0, LOMA_ZONE_MEM = 1, LOMA_ZONE_REP = 2 };
  * Each output is int32[S]; any of them may be NULL (skipped).  on_device != 0:
  * outputs are [device] and filled by a kernel on `stream`; on_device == 0:
  * outputs are [host], filled synchronously, no CUDA call is made.
+ * flags: LOMA_FLAG_NO_REP_ZONE selects the layout without repetition zones (S = n_chunks*t*(c+1) + tail_read).
  * t == 0 requires n_chunks == 0 (the sequence is one reading zone).
  * Errors: INVALID_ARG (negative sizes, c < 1, t == 0 with n_chunks > 0,
  * t > 0 with tail_read > tc, S > INT32_MAX), CUDA.
  * ------------------------------------------------------------------------- */
-LOMA_API int loma_layout_index(int n_chunks, int c, int t, int tail_read,
+LOMA_API int loma_layout_index(int n_chunks, int c, int t, int tail_read, unsigned flags,
                                int32_t* chunk, int32_t* zone, int32_t* offset,
                                int32_t* src_token, int32_t* pos_id,
                                int on_device, void* stream);
@@ -160,6 +167,25 @@ LOMA_API int loma_masked_attn_fwd(const void* q, const void* k, const void* v, v
                                   int n_chunks, int c, int t, int tc, int tail_read,
                                   int64_t stride_b, int64_t stride_h, int64_t stride_s,
                                   loma_dtype dtype, float softmax_scale, unsigned flags, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * loma_prefill_cache -- what the cache holds after a prompt has been ingested (Section 3.1 step 3
+ * applied to every complete chunk; Appendix A, compress_last_chunk's torch.cat lines): the memory-zone
+ * K/V rows of chunks 0..n_chunks-1 in order, followed by the tail_read rows of the unfinished chunk.
+ * Bit-exact gather from the laid-out K and V of a one-pass prefill into the generation cache.
+ *
+ *   k, v             [device, in]   [B, H, S, D] with the strides of loma_masked_attn_fwd
+ *   k_cache, v_cache [device, out]  [B, H, cap, D] contiguous; entries [0, n_chunks*t + tail_read) are
+ *                                   written, nothing else is touched
+ *   flags            LOMA_FLAG_NO_REP_ZONE if k, v are in the layout without repetition zones
+ * Returns the new valid cache length in *cache_len_out ([host], may be NULL).
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CAPACITY (cap < n_chunks*t + tail_read), CUDA.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_prefill_cache(const void* k, const void* v, void* k_cache, void* v_cache,
+                                int B, int H, int D, int cap,
+                                int n_chunks, int c, int t, int tc, int tail_read,
+                                int64_t stride_b, int64_t stride_h, int64_t stride_s,
+                                loma_dtype dtype, unsigned flags, int* cache_len_out, void* stream);
 
 /* ---------------------------------------------------------------------------
  * loma_masked_attn_plan_coverage -- host-only introspection of the tensor-core

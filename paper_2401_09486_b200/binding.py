@@ -18,6 +18,7 @@ import torch
 LOMA_F32 = 0
 LOMA_BF16 = 1
 LOMA_FLAG_MEM_SEES_PRIOR_MEM = 1
+LOMA_FLAG_NO_REP_ZONE = 2
 LOMA_FLAG_FORCE_GENERIC = 1 << 8
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libloma.so")
@@ -28,7 +29,8 @@ _i, _i64, _f, _u, _p, _sz = (ctypes.c_int, ctypes.c_int64, ctypes.c_float, ctype
 
 # name -> (restype, argtypes); mirrors include/loma.h
 SIGNATURES = {
-    "loma_layout_index": (_i, [_i, _i, _i, _i, _p, _p, _p, _p, _p, _i, _p]),
+    "loma_layout_index": (_i, [_i, _i, _i, _i, _u, _p, _p, _p, _p, _p, _i, _p]),
+    "loma_prefill_cache": (_i, [_p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i, _u, _p, _p]),
     "loma_generation_index": (_i, [_i, _i, _i, _p, _p, _p, _i, _p]),
     "loma_masked_attn_fwd": (_i, [_p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i, _f,
                                   _u, _p]),
@@ -120,14 +122,14 @@ def loma_device_status(stream=None) -> int:
     return lib().loma_device_status(_stream(stream))
 
 
-def loma_layout_index(n_chunks: int, c: int, t: int, tail_read: int = 0, device="cpu", stream=None):
+def loma_layout_index(n_chunks: int, c: int, t: int, tail_read: int = 0, device="cpu", stream=None, flags: int = 0):
     """Returns int32 tensors (chunk, zone, offset, src_token, pos_id) on `device`."""
     tc = c * t
-    S = n_chunks * (2 * tc + t) + tail_read
+    S = n_chunks * ((tc + t) if (flags & LOMA_FLAG_NO_REP_ZONE) else (2 * tc + t)) + tail_read
     on_device = torch.device(device).type == "cuda"
     outs = [torch.empty(max(S, 0), dtype=torch.int32, device=device) for _ in range(5)]
     st = _stream(stream) if on_device else None
-    rc = lib().loma_layout_index(n_chunks, c, t, tail_read, *[_ptr(x) for x in outs], int(on_device), st)
+    rc = lib().loma_layout_index(n_chunks, c, t, tail_read, int(flags), *[_ptr(x) for x in outs], int(on_device), st)
     _check(rc, "loma_layout_index")
     return tuple(outs)
 
@@ -162,11 +164,28 @@ def loma_masked_attn_fwd(q, k, v, o, lse, n_chunks: int, c: int, t: int, tail_re
 
 def loma_masked_attn_plan_coverage(n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0) -> torch.Tensor:
     """Host replay of the tensor-core kernel's tile plan: uint8 [S, S] visit counts."""
-    S = n_chunks * (2 * c * t + t) + tail_read
+    S = n_chunks * ((c * t + t) if (flags & LOMA_FLAG_NO_REP_ZONE) else (2 * c * t + t)) + tail_read
     counts = torch.empty((S, S), dtype=torch.uint8)
     rc = lib().loma_masked_attn_plan_coverage(n_chunks, c, t, tail_read, int(flags), _ptr(counts))
     _check(rc, "loma_masked_attn_plan_coverage")
     return counts
+
+
+def loma_prefill_cache(k, v, k_cache, v_cache, n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0,
+                       stream=None) -> int:
+    """Gathers the memory-zone rows and the reading tail of laid-out k, v [B, H, S, D] into the caches
+    [B, H, cap, D]; returns the new cache length."""
+    B, H, S, D = k.shape
+    if v.shape != k.shape or v.stride() != k.stride() or k.stride(3) != 1:
+        raise ValueError("k and v must share shape and strides, head dimension contiguous")
+    if not (k_cache.is_contiguous() and v_cache.is_contiguous()):
+        raise ValueError("caches must be contiguous")
+    n = ctypes.c_int(0)
+    rc = lib().loma_prefill_cache(_ptr(k), _ptr(v), _ptr(k_cache), _ptr(v_cache), B, H, D, k_cache.shape[2], n_chunks, c,
+                                  t, c * t, tail_read, k.stride(0), k.stride(1), k.stride(2), _dtype_code(k), int(flags),
+                                  ctypes.byref(n), _stream(stream))
+    _check(rc, "loma_prefill_cache")
+    return n.value
 
 
 def loma_decode_workspace_bytes(B: int, H: int, D: int, cache_len: int) -> int:

@@ -52,7 +52,7 @@ static int make_layout(int n_chunks, int c, int t, int tail_read, unsigned flags
     if (t == 0 && n_chunks != 0) return LOMA_ERR_INVALID_ARG;
     const int64_t tc = (int64_t)c * t;
     if (t > 0 && tail_read > tc) return LOMA_ERR_INVALID_ARG;
-    const int64_t s = 2 * tc + t;
+    const int64_t s = (flags & LOMA_FLAG_NO_REP_ZONE) ? tc + t : 2 * tc + t;
     const int64_t S = (int64_t)n_chunks * s + tail_read;
     if (tc > INT_MAX / 4 || S > INT_MAX) return LOMA_ERR_INVALID_ARG;
     L->n_chunks = n_chunks; L->c = c; L->t = t; L->tc = (int)tc; L->s = (int)s;
@@ -84,10 +84,10 @@ const char* loma_status_string(int status) {
     }
 }
 
-int loma_layout_index(int n_chunks, int c, int t, int tail_read, int32_t* chunk, int32_t* zone,
+int loma_layout_index(int n_chunks, int c, int t, int tail_read, unsigned flags, int32_t* chunk, int32_t* zone,
                       int32_t* offset, int32_t* src_token, int32_t* pos_id, int on_device, void* stream) {
     Layout L;
-    const int rc = make_layout(n_chunks, c, t, tail_read, 0, &L);
+    const int rc = make_layout(n_chunks, c, t, tail_read, flags, &L);
     if (rc != LOMA_OK) return rc;
     if (!on_device) {
         host_layout_index(L, chunk, zone, offset, src_token, pos_id);
@@ -145,6 +145,33 @@ int loma_masked_attn_fwd(const void* q, const void* k, const void* v, void* o, f
         e = launch_masked_attn_tc(q, k, v, o, lse, B, H, D, L, stride_b, stride_h, stride_s, scale, st);
     if (e == cudaErrorNotSupported)
         e = launch_masked_attn_generic(q, k, v, o, lse, B, H, D, L, stride_b, stride_h, stride_s, dtype, scale, st);
+    return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
+int loma_prefill_cache(const void* k, const void* v, void* k_cache, void* v_cache, int B, int H, int D, int cap,
+                       int n_chunks, int c, int t, int tc, int tail_read, int64_t stride_b, int64_t stride_h,
+                       int64_t stride_s, loma_dtype dtype, unsigned flags, int* cache_len_out, void* stream) {
+    if (B < 0 || H < 0 || cap < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    Layout L;
+    const int rc = make_layout(n_chunks, c, t, tail_read, flags, &L);
+    if (rc != LOMA_OK) return rc;
+    if (tc != L.tc) return LOMA_ERR_INVALID_ARG;
+    const int64_t n_rows = (int64_t)n_chunks * t + tail_read;
+    if (n_rows > cap) return LOMA_ERR_CAPACITY;
+    if (cache_len_out) *cache_len_out = (int)n_rows;
+    if (n_rows == 0 || B == 0 || H == 0) return LOMA_OK;
+    if (!k || !v || !k_cache || !v_cache) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
+    if (stride_s < D || stride_b < 0 || stride_h < 0) return LOMA_ERR_INVALID_ARG;
+    const size_t es = elt_size(dtype);
+    if (!aligned16(k) || !aligned16(v) || !aligned16(k_cache) || !aligned16(v_cache)) return LOMA_ERR_ALIGNMENT;
+    if ((stride_b * es) % 16 || (stride_h * es) % 16 || (stride_s * es) % 16) return LOMA_ERR_ALIGNMENT;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    cudaError_t e = launch_prefill_cache(k, v, k_cache, v_cache, B, H, (int)(D * es), cap, L, stride_b * es, stride_h * es,
+                                         stride_s * es, static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 

@@ -24,6 +24,8 @@ cudaError_t launch_layout_index(const Layout& L, int32_t* chunk, int32_t* zone, 
                                 int32_t* src, int32_t* pos, cudaStream_t st);
 cudaError_t launch_generation_index(int n_tokens, int c, int t, int32_t* slot, int32_t* pos,
                                     int32_t* comp, cudaStream_t st);
+cudaError_t launch_prefill_cache(const void* k, const void* v, void* kc, void* vc, int B, int H, int row_bytes, int cap,
+                                 const Layout& L, int64_t sb_bytes, int64_t sh_bytes, int64_t ss_bytes, cudaStream_t st);
 void host_layout_index(const Layout& L, int32_t* chunk, int32_t* zone, int32_t* offset, int32_t* src,
                        int32_t* pos);
 void host_generation_index(int n_tokens, int c, int t, int32_t* slot, int32_t* pos, int32_t* comp);

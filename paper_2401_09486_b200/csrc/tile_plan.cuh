@@ -137,7 +137,7 @@ inline View make_view(int Z, int nch, int chunk_base, int zone_row0) {
 inline void make_plan(const Layout& L, int B, int H, FwdParams* p) {
     p->view[V_READ] = make_view(L.tc, L.n_chunks, 0, 0);
     p->view[V_MEM] = make_view(L.t, L.n_chunks, 0, L.tc);
-    p->view[V_REP] = make_view(L.tc, L.n_chunks, 0, L.tc + L.t);
+    p->view[V_REP] = make_view(L.tc, (L.flags & LOMA_FLAG_NO_REP_ZONE) ? 0 : L.n_chunks, 0, L.tc + L.t);
     p->view[V_TAIL] = make_view(L.tail_read, L.tail_read > 0 ? 1 : 0, L.n_chunks, 0);
     p->n_chunks = L.n_chunks; p->s = L.s; p->S = L.S; p->H = H; p->BH = B * H;
     p->n_tail = p->view[V_TAIL].ntiles; p->n_read = p->view[V_READ].ntiles;

@@ -60,10 +60,19 @@ def test_host_generation_index_bit_exact(lib, n_tok, c, t):
         assert np.array_equal(g.numpy(), w)
 
 
+@pytest.mark.parametrize("n,c,t,tail", [(3, 2, 2, 0), (2, 4, 4, 3), (32, 4, 16, 5), (5, 3, 7, 21)])
+def test_host_layout_index_inference_layout_bit_exact(lib, n, c, t, tail):
+    f = binding.LOMA_FLAG_NO_REP_ZONE
+    got = binding.loma_layout_index(n, c, t, tail, device="cpu", flags=f)
+    want = oracle.layout_index(n, c, t, tail, oracle.FLAG_NO_REP_ZONE)
+    for g, w in zip(got, want):
+        assert np.array_equal(g.numpy(), w)
+
+
 def test_layout_index_null_outputs_are_skipped(lib):
     S = oracle.seq_len(2, 2, 2)
     pos = (ctypes.c_int32 * S)()
-    assert lib.loma_layout_index(2, 2, 2, 0, None, None, None, None, pos, 0, None) == 0
+    assert lib.loma_layout_index(2, 2, 2, 0, 0, None, None, None, None, pos, 0, None) == 0
     assert list(pos) == oracle.layout_index(2, 2, 2)[4].tolist()
 
 
@@ -72,7 +81,7 @@ def test_layout_index_rejects_bad_geometry(lib):
     bad = [(-1, 2, 2, 0), (1, 0, 2, 0), (1, 2, -1, 0), (1, 2, 0, 0), (1, 2, 2, 5), (1, 2, 2, -1),
            (1 << 20, 64, 64, 0)]
     for n, c, t, tail in bad:
-        assert lib.loma_layout_index(n, c, t, tail, buf, None, None, None, None, 0, None) == INVALID
+        assert lib.loma_layout_index(n, c, t, tail, 0, buf, None, None, None, None, 0, None) == INVALID
 
 
 def _fwd(lib, q=0x1000, k=0x2000, v=0x3000, o=0x4000, lse=None, B=1, H=1, D=64, n=1, c=2, t=2, tc=4, tail=0,
@@ -96,6 +105,21 @@ def test_masked_attn_fwd_validation_precedes_any_cuda_call(lib):
     assert _fwd(lib, tail=5) == INVALID                 # tail longer than a reading zone
     assert _fwd(lib, n=0, t=2, tc=4, tail=0) == 0       # empty sequence: no-op
     assert _fwd(lib, B=0) == 0
+
+
+def test_prefill_cache_validation(lib):
+    def call(k=0x1000, v=0x2000, kc=0x3000, vc=0x4000, B=1, H=1, D=128, cap=64, n=2, c=4, t=16, tc=64, tail=3,
+             sb=100000, sh=100000, ss=128, dt=1, flags=0):
+        n_out = ctypes.c_int(-1)
+        rc = lib.loma_prefill_cache(k, v, kc, vc, B, H, D, cap, n, c, t, tc, tail, sb, sh, ss, dt, flags,
+                                    ctypes.byref(n_out), None)
+        return rc, n_out.value
+    assert call(cap=34)[0] == CAPACITY                  # needs 2*16 + 3 slots
+    assert call(tc=60)[0] == INVALID
+    assert call(k=None)[0] == INVALID
+    assert call(v=0x2004)[0] == ALIGNMENT
+    assert call(D=80)[0] == UNSUPPORTED
+    assert call(B=0) == (0, 35)                         # nothing to do, length still reported
 
 
 def test_decode_validation(lib):
@@ -139,7 +163,7 @@ PLAN_GEOMS = [(3, 2, 2, 0), (2, 4, 4, 3), (5, 4, 16, 37), (9, 4, 16, 0), (3, 8, 
 
 
 @pytest.mark.parametrize("n,c,t,tail", PLAN_GEOMS)
-@pytest.mark.parametrize("flags", [0, 1])
+@pytest.mark.parametrize("flags", [0, 1, 2, 3])
 def test_tensor_core_tile_plan_reproduces_the_mask_exactly(lib, n, c, t, tail, flags):
     """Every allowed (row, key) pair of Eq. 2 is visited exactly once by the
     tensor-core kernel's tile plan, and no blocked pair is visited at all."""

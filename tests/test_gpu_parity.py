@@ -17,6 +17,7 @@ from paper_2401_09486_b200 import build, synthetic
 pytestmark = pytest.mark.gpu
 
 PRIOR = L.LOMA_FLAG_MEM_SEES_PRIOR_MEM
+NOREP = L.LOMA_FLAG_NO_REP_ZONE
 GENERIC = L.LOMA_FLAG_FORCE_GENERIC
 DEV = "cuda:0"
 
@@ -124,6 +125,40 @@ def test_masked_fwd_strided_views_and_explicit_scale():
     L.loma_masked_attn_fwd(q, k, v, o, None, n, c, t, 0, 0, 0.05)
     torch.cuda.synchronize()
     check_close(o, want_o, torch.bfloat16)
+
+
+# ----------------------------------------- inference layout (no repetition zones)
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [NOREP, NOREP | PRIOR, NOREP | GENERIC])
+@pytest.mark.parametrize("B,H,D,n,c,t,tail", [(1, 2, 64, 3, 2, 4, 3), (2, 2, 128, 5, 4, 16, 37), (1, 2, 128, 3, 8, 32, 100),
+                                              (1, 1, 128, 2, 3, 7, 0), (1, 2, 128, 20, 4, 16, 0)])
+def test_prefill_one_pass_matches_oracle_and_fills_the_cache(B, H, D, n, c, t, tail, flags, dtype):
+    """One pass over a prompt laid out as [reading | memory] chunks: outputs match the oracle, and
+    loma_prefill_cache leaves exactly the cache that token-by-token ingestion would (bit for bit)."""
+    of = (flags & PRIOR) | oracle.FLAG_NO_REP_ZONE
+    S = oracle.seq_len(n, c, t, tail, of)
+    q, k, v = synthetic.qkv(B, H, S, D, seed=17, std=1.0, dtype=dtype)
+    want_o, want_lse = oracle.masked_attn_fwd(npf(q), npf(k), npf(v), n, c, t, tail, of)
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    o, lse = run_fwd(qd, kd, vd, n, c, t, tail, flags)
+    check_close(o, want_o, dtype)
+    assert np.abs(npf(lse) - want_lse).max() <= (1e-5 if dtype == torch.float32 else 2e-2)
+    got = L.loma_layout_index(n, c, t, tail, device=DEV, flags=NOREP)
+    torch.cuda.synchronize()
+    for g, w in zip(got, oracle.layout_index(n, c, t, tail, oracle.FLAG_NO_REP_ZONE)):
+        assert np.array_equal(g.cpu().numpy(), w)
+    # cache after the prompt = what the oracle's incremental replay leaves
+    _, ref_k, ref_v, ref_len = oracle.replay_generation(bits(q) * 0.0, bits(k), bits(v), n, c, t, tail, of, scale=0.0)
+    cap = n * t + tail + 5
+    kc = torch.full((B, H, cap, D), 7.0, dtype=dtype, device=DEV)
+    vc = torch.full((B, H, cap, D), 7.0, dtype=dtype, device=DEV)
+    length = L.loma_prefill_cache(kd, vd, kc, vc, n, c, t, tail, NOREP)
+    torch.cuda.synchronize()
+    assert length == ref_len == n * t + tail
+    assert np.array_equal(bits(kc[:, :, :length]), ref_k[:, :, :length])
+    assert np.array_equal(bits(vc[:, :, :length]), ref_v[:, :, :length])
+    assert (kc[:, :, length:] == 7.0).all() and (vc[:, :, length:] == 7.0).all()      # nothing else is touched
 
 
 def replay_on_gpu(q, k, v, n, c, t, tail, flags):
