@@ -9,7 +9,8 @@
 // instruction (mma.sync.m16n8k16); the 128-row tcgen05 tile would idle 7/8 of
 // the array here, so this kernel uses the warp-level path on purpose.
 //
-//   CTA (4 warps) = one key range of one (b,h).  The last range of a (b,h) is
+//   Memory zones longer than 16 take several 16-row query tiles, each its own CTA.
+//   CTA (4 warps) = one key range of one (b,h) (and one query tile).  The last range of a (b,h) is
 //   always [tail (tc rows) ; k_mem (t rows)]; with the prior-memory flag the
 //   earlier ranges cut cache[0, mem_len) into pieces.
 //   K and V rows are staged 64 at a time in shared memory with 16-byte
@@ -18,7 +19,8 @@
 //   softmax in registers, O += P V with P straight from the accumulator
 //   registers.  Warps are merged in shared memory; ranges through the workspace
 //   and a small merge kernel (fixed order: bitwise repeatable).
-//   Compaction: the CTA that owns the tail is the only reader of the slots
+//   Compaction (t <= 16; longer zones compact in a second, stream-ordered launch because several
+//   CTAs then read the same tail): the CTA that owns the tail is the only reader of the slots
 //   [mem_len, mem_len + t) in this launch; after a block barrier it overwrites
 //   them with k_mem / v_mem using 16-byte vector stores.
 #include <math.h>
@@ -44,10 +46,11 @@ int compress_num_prior(int BH, int mem_len, unsigned flags) {
 }
 
 size_t compress_workspace_bytes(int BH, int D, int t, int mem_len, unsigned flags) {
-    if (t > 16) return 0;   // handled by the CUDA-core kernel, which needs none
+    if (t > 128) return 0;   // handled by the CUDA-core kernel, which needs none
     const int np = compress_num_prior(BH, mem_len, flags);
     if (np == 0) return 0;
-    return (size_t)BH * (np + 1) * 16 * (D + 2) * sizeof(float);
+    const int mt = (t + 15) / 16;
+    return (size_t)BH * (np + 1) * mt * 16 * (D + 2) * sizeof(float);
 }
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
@@ -98,15 +101,19 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
                     const __nv_bfloat16* __restrict__ v_mem, __nv_bfloat16* __restrict__ k_cache,
                     __nv_bfloat16* __restrict__ v_cache, __nv_bfloat16* __restrict__ o_mem, float* __restrict__ lse,
                     float* __restrict__ ws, int BH, int cap, int mem_len, int t, int tc, int nprior, int prior_len,
-                    float scale_log2) {
+                    int mtiles, float scale_log2) {
     using SM = CmpSmem<D>;
     constexpr int ROWB = SM::ROWB;
     constexpr int VPR = D / 8;                 // 16-byte vectors per row
     extern __shared__ __align__(16) uint8_t smem[];
     const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(smem);
+    // one CTA per (b,h), key range and tile of 16 query rows (t > 16 memory queries take several tiles)
     const int nsp = nprior + 1;
-    const int bh = blockIdx.x / nsp, split = blockIdx.x - bh * nsp;
+    const int mt = blockIdx.x % mtiles;
+    const int bs = blockIdx.x / mtiles;
+    const int bh = bs / nsp, split = bs - bh * nsp;
     const bool is_tail = split == nprior;
+    const int q0 = mt * 16;                    // first query row of this tile
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;
 
@@ -142,7 +149,7 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
     for (int e = threadIdx.x; e < 16 * VPR; e += CMP_WARPS * 32) {
         const int r = e / VPR, cv = e - r * VPR;
         uint4 val = make_uint4(0, 0, 0, 0);
-        if (r < t) val = __ldg(reinterpret_cast<const uint4*>(q_mem + ((int64_t)bh * t + r) * D) + cv);
+        if (q0 + r < t) val = __ldg(reinterpret_cast<const uint4*>(q_mem + ((int64_t)bh * t + q0 + r) * D) + cv);
         *reinterpret_cast<uint4*>(smem + SM::Q_OFF + r * ROWB + cv * 16) = val;
     }
     __syncthreads();
@@ -264,10 +271,10 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
             f[w] = (mw > -INFINITY) ? ex2f(mw - M) : 0.f;
             lt = fmaf(mg_ml[(w * 16 + r) * 2 + 1], f[w], lt);
         }
-        if (r < t) {
+        if (q0 + r < t) {
             if (nsp == 1) {
                 const float inv = 1.f / lt;
-                __nv_bfloat16* dst = o_mem + ((int64_t)bh * t + r) * D + d0;
+                __nv_bfloat16* dst = o_mem + ((int64_t)bh * t + q0 + r) * D + d0;
 #pragma unroll
                 for (int d = 0; d < SEG; d += 2) {
                     float x0 = 0.f, x1 = 0.f;
@@ -278,9 +285,10 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
                     }
                     *reinterpret_cast<uint32_t*>(dst + d) = pack_bf16(x0 * inv, x1 * inv);
                 }
-                if (lse && d0 == 0) lse[(int64_t)bh * t + r] = (M + log2f(lt)) * 0.6931471805599453f;
+                if (lse && d0 == 0) lse[(int64_t)bh * t + q0 + r] = (M + log2f(lt)) * 0.6931471805599453f;
             } else {
-                float* po = ws + (((int64_t)bh * nsp + split) * 16 + r) * D + d0;
+                const int64_t slot = (((int64_t)bh * nsp + split) * mtiles + mt) * 16 + r;
+                float* po = ws + slot * D + d0;
 #pragma unroll
                 for (int d = 0; d < SEG; ++d) {
                     float x = 0.f;
@@ -289,14 +297,15 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
                     po[d] = x;
                 }
                 if (d0 == 0) {
-                    float* pml = ws + (int64_t)BH * nsp * 16 * D + (((int64_t)bh * nsp + split) * 16 + r) * 2;
+                    float* pml = ws + (int64_t)BH * nsp * mtiles * 16 * D + slot * 2;
                     pml[0] = M; pml[1] = lt;
                 }
             }
         }
     }
     // compaction (Section 3.1 step 3): every read of the tail by this launch happened in this CTA, above
-    if (is_tail) {
+    // (with several query tiles per (b,h) other CTAs read the same tail: a separate launch compacts then)
+    if (is_tail && mtiles == 1) {
         __syncthreads();
         const uint4* ksrc = reinterpret_cast<const uint4*>(km);
         const uint4* vsrc = reinterpret_cast<const uint4*>(vm);
@@ -312,22 +321,42 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
 template <int D>
 __global__ void __launch_bounds__(D)
 compress_merge_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ o_mem, float* __restrict__ lse,
-                      int BH, int t, int nsp) {
+                      int BH, int t, int nsp, int mtiles) {
     const int bh = blockIdx.x / t, r = blockIdx.x - bh * t, d = threadIdx.x;
-    const float* pml = ws + (int64_t)BH * nsp * 16 * D;
+    const int mt = r >> 4, r16 = r & 15;
+    const float* pml = ws + (int64_t)BH * nsp * mtiles * 16 * D;
+    auto slot = [&](int s) { return (((int64_t)bh * nsp + s) * mtiles + mt) * 16 + r16; };
     float M = -INFINITY;
-    for (int s = 0; s < nsp; ++s) M = fmaxf(M, pml[(((int64_t)bh * nsp + s) * 16 + r) * 2]);
+    for (int s = 0; s < nsp; ++s) M = fmaxf(M, pml[slot(s) * 2]);
     float lt = 0.f, ot = 0.f;
     for (int s = 0; s < nsp; ++s) {
-        const float ms = pml[(((int64_t)bh * nsp + s) * 16 + r) * 2];
+        const float ms = pml[slot(s) * 2];
         if (ms > -INFINITY) {
             const float f = exp2f(ms - M);
-            lt = fmaf(pml[(((int64_t)bh * nsp + s) * 16 + r) * 2 + 1], f, lt);
-            ot = fmaf(ws[(((int64_t)bh * nsp + s) * 16 + r) * D + d], f, ot);
+            lt = fmaf(pml[slot(s) * 2 + 1], f, lt);
+            ot = fmaf(ws[slot(s) * D + d], f, ot);
         }
     }
     o_mem[((int64_t)bh * t + r) * D + d] = __float2bfloat16_rn(ot / lt);
     if (lse && d == 0) lse[(int64_t)bh * t + r] = (M + log2f(lt)) * 0.6931471805599453f;
+}
+
+// Compaction on its own (used when the memory queries span several 16-row tiles): runs after the
+// attention kernel in stream order, so every read of the tail has completed.
+template <int D>
+__global__ void compaction_kernel(const __nv_bfloat16* __restrict__ k_mem, const __nv_bfloat16* __restrict__ v_mem,
+                                  __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache, int cap,
+                                  int mem_len, int t) {
+    const int bh = blockIdx.x;
+    constexpr int VPR = D / 8;
+    const uint4* ksrc = reinterpret_cast<const uint4*>(k_mem + (int64_t)bh * t * D);
+    const uint4* vsrc = reinterpret_cast<const uint4*>(v_mem + (int64_t)bh * t * D);
+    uint4* kdst = reinterpret_cast<uint4*>(k_cache + ((int64_t)bh * cap + mem_len) * D);
+    uint4* vdst = reinterpret_cast<uint4*>(v_cache + ((int64_t)bh * cap + mem_len) * D);
+    for (int e = threadIdx.x; e < t * VPR; e += blockDim.x) {
+        kdst[e] = __ldg(ksrc + e);
+        vdst[e] = __ldg(vsrc + e);
+    }
 }
 
 template <int D>
@@ -348,21 +377,33 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    compress_mma_kernel<D><<<BH * nsp, CMP_WARPS * 32, smem, st>>>(
+    const int mtiles = (t + 15) / 16;
+    compress_mma_kernel<D><<<BH * nsp * mtiles, CMP_WARPS * 32, smem, st>>>(
         static_cast<const __nv_bfloat16*>(qm), static_cast<const __nv_bfloat16*>(km),
         static_cast<const __nv_bfloat16*>(vm), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
         static_cast<__nv_bfloat16*>(om), lse, static_cast<float*>(ws), BH, cap, mem_len, t, tc, nprior, prior_len,
-        scale * 1.4426950408889634f);
+        mtiles, scale * 1.4426950408889634f);
     count_launches(1);
     e = cudaGetLastError();
-    if (e != cudaSuccess || nsp == 1) return e;
-    compress_merge_kernel<D><<<BH * t, D, 0, st>>>(static_cast<const float*>(ws), static_cast<__nv_bfloat16*>(om), lse,
-                                                   BH, t, nsp);
-    count_launches(1);
-    return cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (nsp > 1) {
+        compress_merge_kernel<D><<<BH * t, D, 0, st>>>(static_cast<const float*>(ws), static_cast<__nv_bfloat16*>(om),
+                                                       lse, BH, t, nsp, mtiles);
+        count_launches(1);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    if (mtiles > 1) {
+        compaction_kernel<D><<<BH, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(km),
+                                                  static_cast<const __nv_bfloat16*>(vm), static_cast<__nv_bfloat16*>(kc),
+                                                  static_cast<__nv_bfloat16*>(vc), cap, mem_len, t);
+        count_launches(1);
+        e = cudaGetLastError();
+    }
+    return e;
 }
 
-// t <= 16 only; the caller falls back to the CUDA-core kernel otherwise.
+// t <= 128; the caller falls back to the CUDA-core kernel otherwise.
 cudaError_t launch_compress_bf16(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
                                  void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len, int c, int t,
                                  unsigned flags, float scale, void* ws, cudaStream_t st) {

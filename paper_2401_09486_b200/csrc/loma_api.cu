@@ -274,7 +274,7 @@ int loma_compress_step(const void* q_mem, const void* k_mem, const void* v_mem, 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((int64_t)B * H * 256 > INT_MAX) return LOMA_ERR_INVALID_ARG;
     cudaError_t e;
-    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC) && t <= 16)
+    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC) && t <= 128)
         e = launch_compress_bf16(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, mem_len, c, t, flags,
                                  scale, workspace, st);
     else

@@ -279,7 +279,8 @@ def test_decode_matches_oracle(B, H, D, cap, cache_len, flags, dtype):
 @pytest.mark.parametrize("B,H,D,c,t,mem_len,extra", [(1, 1, 64, 4, 4, 0, 0), (2, 2, 128, 4, 16, 48, 5),
                                                      (2, 3, 128, 8, 16, 1024, 0), (1, 2, 128, 3, 5, 35, 2),
                                                      (1, 2, 128, 8, 32, 640, 7), (1, 1, 64, 1, 1, 3, 0),
-                                                     (2, 2, 128, 4, 16, 2000, 1)])
+                                                     (2, 2, 128, 4, 16, 2000, 1), (1, 2, 128, 2, 64, 128, 3),
+                                                     (1, 1, 64, 2, 100, 1300, 0), (2, 1, 128, 1, 17, 51, 0)])
 def test_compress_matches_oracle_and_compacts_bit_exact(B, H, D, c, t, mem_len, extra, flags, dtype):
     tc = c * t
     cap = mem_len + tc + extra
