@@ -280,6 +280,20 @@ struct TcSmem {
     static constexpr int TOTAL = 2 * STREAM_BYTES;
 };
 
+// The visited halves of a tile's first 64 steps, one step per lane and two ballots per 32 steps.
+// Called by whole warps only.
+__device__ __forceinline__ HalfMasks tile_half_masks(const FwdParams& p, const TileDesc& td, int lane) {
+    HalfMasks hm;
+    hm.m[0] = hm.m[1] = 0;
+    for (int base = 0; base < td.nsteps && base < 64; base += 32) {
+        const int j = base + lane;
+        const unsigned v = j < td.nsteps ? visited_halves(p, td, j) : 0u;
+        hm.m[0] |= (unsigned long long)__ballot_sync(0xffffffffu, v & 1u) << base;
+        hm.m[1] |= (unsigned long long)__ballot_sync(0xffffffffu, v & 2u) << base;
+    }
+    return hm;
+}
+
 template <int D>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
@@ -388,66 +402,77 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             const uint64_t qd = smem_desc(smem_base + SM::Q_OFF, 16, 1024);
             const uint64_t kd = smem_desc(smem_base + SM::K_OFF, 16, 1024);
             const uint64_t vd = smem_desc(smem_base + SM::V_OFF, SM::PANEL_BYTES, 1024);
-            // scores of keys [64h, 64h+64) of the staged key tile -> score buffer h (64 columns)
-            auto issue_s = [&](int h, bool last) {
+            // Visited halves ("events") are numbered ge = 0, 1, 2, ... across all tiles of the stream.
+            // Event ge uses score buffer ge & 1 and the barriers B_SF/B_PF/B_OF + (ge & 1), whose
+            // completion number ge >> 1 gives the parity to wait for.  K/V buffers go by step (gs).
+            // scores of keys [64h, 64h+64) of the staged key tile -> score buffer b (64 columns)
+            auto issue_s = [&](int b, int h, bool last_of_step, bool last_of_tile) {
                 if (elect_one()) {
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
                         // descriptor start addresses are in 16-byte units; 64 key rows are 8192 bytes further
                         const uint64_t off = (uint64_t)(((kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32) >> 4);
-                        mma_ss(tmem + h * 64, qd + off, kd + off + (uint64_t)((h * 8192) >> 4), IDESC_S, kk > 0);
+                        mma_ss(tmem + b * 64, qd + off, kd + off + (uint64_t)((h * 8192) >> 4), IDESC_S, kk > 0);
                     }
-                    tc_commit(bar(B_SF + h));
-                    if (last) tc_commit(bar(B_KE));
+                    tc_commit(bar(B_SF + b));
+                    if (last_of_step) tc_commit(bar(B_KE));
+                    if (last_of_tile) tc_commit(bar(B_QE));   // every score product of the tile has been issued
                 }
                 __syncwarp();
             };
-            // O += P_h V[64h .. 64h+63]: four instructions of 16 keys, P read from TMEM over score buffer h
-            auto issue_pv = [&](int h, bool first) {
+            // O += P V[64h .. 64h+63]: four instructions of 16 keys, P read from TMEM over score buffer b
+            auto issue_pv = [&](int b, int h, bool first, bool last_of_step) {
                 if (elect_one()) {
 #pragma unroll
                     for (int k4 = 0; k4 < 4; ++k4)
-                        mma_ts(tmem + 128, tmem + h * 64 + k4 * 8, vd + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_PV,
+                        mma_ts(tmem + 128, tmem + b * 64 + k4 * 8, vd + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_PV,
                                !first || (k4 > 0));
-                    tc_commit(bar(B_OF + h));   // one barrier per half: each completes exactly once per step
-                    if (h == 1) tc_commit(bar(B_VE));
+                    tc_commit(bar(B_OF + b));   // one barrier per buffer: each completes once per event
+                    if (last_of_step) tc_commit(bar(B_VE));
                 }
                 __syncwarp();
             };
+            uint32_t ge_s = 0, ge_p = 0;   // events whose scores / whose P.V have been issued
             for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
                 const int rank = w / p.BH;
                 TileDesc td;
                 decode_tile(p, rank, td);
-                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_QF), tcount & 1, abortp, p.status) &&
-                                                 mbar_wait(bar(B_KF), gs & 1, abortp, p.status));
+                const HalfMasks hm = tile_half_masks(p, td, lane);
+                const int nsteps = td.nsteps;
+                HalfWalk sw, pw;
+                sw.start(hm);
+                pw.start(hm);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_QF), tcount & 1, abortp, p.status));
                 if (!ok) break;
-                tc_fence_after();
-                issue_s(0, false);
-                issue_s(1, true);
-                for (int j = 0; j < td.nsteps && ok; ++j, ++gs) {
-                    const uint32_t ph = gs & 1;
-                    const bool more = j + 1 < td.nsteps;
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_PF), ph, abortp, p.status) &&
-                                                     mbar_wait(bar(B_VF), ph, abortp, p.status));
+                // the score products run two events ahead of the P.V products
+                auto next_scores = [&]() {
+                    if (sw.first_of_step(hm)) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar(B_KF), (gs + sw.j) & 1, abortp, p.status));
+                        if (!ok) return;
+                    }
+                    tc_fence_after();
+                    const bool los = sw.last_of_step(hm);
+                    issue_s(ge_s & 1, sw.h, los, los && sw.j == nsteps - 1);
+                    ++ge_s;
+                    sw.next(hm);
+                };
+                next_scores();
+                if (ok && !sw.done(nsteps)) next_scores();
+                bool first = true;
+                while (ok && !pw.done(nsteps)) {
+                    const int b = ge_p & 1;
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_PF + b), (ge_p >> 1) & 1, abortp, p.status));
+                    if (ok && pw.first_of_step(hm))
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar(B_VF), (gs + pw.j) & 1, abortp, p.status));
                     if (!ok) break;
                     tc_fence_after();
-                    issue_pv(0, j == 0);
-                    if (more) {
-                        ok = __all_sync(0xffffffffu, mbar_wait(bar(B_KF), (gs + 1) & 1, abortp, p.status));
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_s(0, false);
-                    }
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_PF + 1), ph, abortp, p.status));
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_pv(1, false);
-                    if (more) issue_s(1, true);
-                    else {
-                        if (elect_one()) tc_commit(bar(B_QE));
-                        __syncwarp();
-                    }
+                    issue_pv(b, pw.h, first, pw.last_of_step(hm));
+                    first = false;
+                    ++ge_p;
+                    if (!sw.done(nsteps)) next_scores();
+                    pw.next(hm);
                 }
+                gs += td.nsteps;
             }
         }
     } else {
@@ -456,7 +481,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         const int rr = threadIdx.x & 127;
         const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         const uint32_t s_addr = lane_addr, o_addr = lane_addr + 128;
-        uint32_t gs = 0;
+        uint32_t ge = 0;   // visited halves so far (see the MMA issuer)
         bool ok = true;
         bool store_pending = false;
         for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r)) {
@@ -475,21 +500,27 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             // output accumulator in TMEM is rescaled once.  Probabilities stay below 2^8.
             float m_used = -INFINITY, l = 0.f;
 
-            for (int j = 0; j < td.nsteps && ok; ++j, ++gs) {
-                KTile kt;
-                step_ktile(p, td, j, kt);
-                int lo, hi2;
-                row_interval(p.view[kt.view], kt, rc, ro, rr, row_valid, lo, hi2);
-                const uint32_t span = (uint32_t)(hi2 - lo);
-                // the 128 keys of the step are handled as two halves of 64, each with its own score buffer,
-                // so the tensor pipe works on one half while this warpgroup works on the other
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const bool full = __all_sync(0xffffffffu, lo <= 64 * h && hi2 >= 64 * h + 64);
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF + h), gs & 1, abortp, p.status));
+            const HalfMasks hm = tile_half_masks(p, td, lane);
+            HalfWalk hw;
+            bool first = true;
+            int lo = 0, hi2 = 0;
+            for (hw.start(hm); ok && !hw.done(td.nsteps); hw.next(hm), ++ge, first = false) {
+                if (hw.first_of_step(hm)) {
+                    KTile kt;
+                    step_ktile(p, td, hw.j, kt);
+                    row_interval(p.view[kt.view], kt, rc, ro, rr, row_valid, lo, hi2);
+                }
+                // One visited half of a key tile (64 keys) per pass, in score buffer ge & 1: the tensor
+                // pipe works on the other buffer while this warpgroup works on this one.
+                {
+                    const int b = ge & 1;
+                    const int lo_h = lo - 64 * hw.h;                  // allowed columns of this half: [lo_h, lo_h + span)
+                    const uint32_t span = (uint32_t)(hi2 - lo);
+                    const bool full = __all_sync(0xffffffffu, lo_h <= 0 && hi2 - 64 * hw.h >= 64);
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF + b), (ge >> 1) & 1, abortp, p.status));
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t sh_addr = s_addr + h * 64;
+                    const uint32_t sh_addr = s_addr + b * 64;
                     uint32_t s[64];
                     tmem_ld32(sh_addr, s);
                     tmem_ld32(sh_addr + 32, s + 32);
@@ -497,7 +528,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     if (!full) {
 #pragma unroll
                         for (int e = 0; e < 64; ++e)
-                            if ((uint32_t)(64 * h + e - lo) >= span) s[e] = 0xff800000u;   // -inf: blocked for this row
+                            if ((uint32_t)(e - lo_h) >= span) s[e] = 0xff800000u;   // -inf: blocked for this row
                     }
                     float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
@@ -509,11 +540,10 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     }
                     const float mrow = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
                     const bool need = mrow > m_used + 8.f;
-                    if ((j > 0 || h > 0) && __any_sync(0xffffffffu, need)) {
-                        // rescale the accumulated output: wait until the previous P.V has landed in TMEM
-                        // (the other half's product of this step, or the second half's of the step before)
-                        ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + (h ^ 1)), (h == 0 ? gs - 1 : gs) & 1, abortp,
-                                                               p.status));
+                    if (!first && __any_sync(0xffffffffu, need)) {
+                        // rescale the accumulated output: wait until the previous event's P.V has landed in TMEM
+                        ok = __all_sync(0xffffffffu,
+                                        mbar_wait(bar(B_OF + ((ge - 1) & 1)), ((ge - 1) >> 1) & 1, abortp, p.status));
                         if (!ok) break;
                         tc_fence_after();
                         const float alpha = need ? fast_ex2(m_used - mrow) : 1.f;
@@ -556,11 +586,11 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     }
                     tmem_wait_st();
                     tc_fence_before();
-                    mbar_arrive(bar(B_PF + h));
+                    mbar_arrive(bar(B_PF + b));
                 }
             }
-            // the last P.V of the tile is the second half of step gs - 1 (products complete in issue order)
-            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + 1), (gs - 1) & 1, abortp, p.status));
+            // the last P.V of the tile belongs to event ge - 1 (products complete in issue order)
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + ((ge - 1) & 1)), ((ge - 1) >> 1) & 1, abortp, p.status));
             if (ok) tc_fence_after();
 
             // epilogue: normalise, round to bf16, stage 64 output columns at a time in shared

@@ -122,6 +122,55 @@ __host__ __device__ __forceinline__ void row_interval(const View& kv, const KTil
     if (!row_valid) { lo = 0; hi = 0; }
 }
 
+// Halves (64 columns each) of a key tile that hold an allowed column for at least one row of the
+// query tile: bit h set = columns [64h, 64h + 64) are visited.  Computed from the union of the row
+// intervals over the tile's chunks; a superset is harmless (every row still applies its own
+// interval), a missing half would drop allowed entries, which the host-side coverage replay checks.
+__host__ __device__ __forceinline__ unsigned step_halves(const FwdParams& p, const TileDesc& td, const KTile& kt) {
+    const View& kv = p.view[kt.view];
+    const int vcols = plan_min(kv.R, kv.Z - kt.r0);
+    int ulo = 0, uhi = 0;
+    if (kt.mode == M_LT || kt.mode == M_LE) {
+        const int nch = plan_min(plan_max(td.a1 - kt.a0 + (kt.mode == M_LE ? 1 : 0), 0), kv.CH);
+        uhi = nch > 0 ? (nch - 1) * kv.R + vcols : 0;
+    } else if (kt.mode == M_DIAG) {
+        uhi = 128;
+    } else {
+        const int d0 = plan_max(td.a0 - kt.a0, 0), d1 = plan_min(td.a1 - kt.a0, kv.CH - 1);
+        if (d1 >= d0) { ulo = d0 * kv.R; uhi = d1 * kv.R + vcols; }
+    }
+    const unsigned m = ((ulo < 64 && uhi > 0) ? 1u : 0u) | (uhi > 64 ? 2u : 0u);
+    return m ? m : 1u;
+}
+
+// Visited halves of a tile's steps as two bit masks: bit j of m[h] = half h of step j is visited.
+// Steps from 64 on are taken whole, so that two 64-bit words always suffice.
+struct HalfMasks {
+    unsigned long long m[2];
+    __host__ __device__ __forceinline__ bool has(int h, int j) const { return j >= 64 || ((m[h] >> j) & 1ull); }
+};
+__host__ __device__ __forceinline__ unsigned visited_halves(const FwdParams& p, const TileDesc& td, int j) {
+    if (j >= 64) return 3u;
+    KTile kt;
+    step_ktile(p, td, j, kt);
+    return step_halves(p, td, kt);
+}
+
+// Walks the visited halves of a query tile's key tiles in order.  One visited half ("event") is
+// the unit of the kernel's pipeline: one score buffer, one softmax pass, one P.V product.
+struct HalfWalk {
+    int j, h;
+    __host__ __device__ __forceinline__ void start(const HalfMasks& hm) { j = 0; h = hm.has(0, 0) ? 0 : 1; }
+    __host__ __device__ __forceinline__ bool done(int nsteps) const { return j >= nsteps; }
+    __host__ __device__ __forceinline__ void next(const HalfMasks& hm) {
+        if (h == 0 && hm.has(1, j)) { h = 1; return; }
+        ++j;
+        h = hm.has(0, j) ? 0 : 1;
+    }
+    __host__ __device__ __forceinline__ bool first_of_step(const HalfMasks& hm) const { return h == 0 || !hm.has(0, j); }
+    __host__ __device__ __forceinline__ bool last_of_step(const HalfMasks& hm) const { return h == 1 || !hm.has(1, j); }
+};
+
 // Fills the geometry part of FwdParams (views, tile counts) from the layout.
 inline View make_view(int Z, int nch, int chunk_base, int zone_row0) {
     View v{};

@@ -15,9 +15,17 @@ void plan_coverage_host(const Layout& L, uint8_t* counts) {
         TileDesc td;
         decode_tile(p, rank, td);
         const View& qv = p.view[td.view];
-        for (int j = 0; j < td.nsteps; ++j) {
+        // the same walk over visited halves as the kernel's roles take
+        HalfMasks hm{{0, 0}};
+        for (int j = 0; j < td.nsteps && j < 64; ++j) {
+            const unsigned v = visited_halves(p, td, j);
+            hm.m[0] |= (unsigned long long)(v & 1u) << j;
+            hm.m[1] |= (unsigned long long)((v >> 1) & 1u) << j;
+        }
+        HalfWalk hw;
+        for (hw.start(hm); !hw.done(td.nsteps); hw.next(hm)) {
             KTile kt;
-            step_ktile(p, td, j, kt);
+            step_ktile(p, td, hw.j, kt);
             const View& kv = p.view[kt.view];
             for (int rr = 0; rr < 128; ++rr) {
                 const int rsub = rr / qv.R;
@@ -28,7 +36,7 @@ void plan_coverage_host(const Layout& L, uint8_t* counts) {
                 row_interval(kv, kt, rc, ro, rr, row_valid, lo, hi);
                 if (!row_valid || hi <= lo) continue;
                 const int64_t grow = (int64_t)rc * L.s + qv.zone_row0 + ro;
-                for (int col = lo; col < hi; ++col) {
+                for (int col = (lo > 64 * hw.h ? lo : 64 * hw.h); col < hi && col < 64 * hw.h + 64; ++col) {
                     // column of the key tile -> row of the laid-out sequence, the way the TMA box gathers it
                     const int ksub = col / kv.R;
                     const int ko = kt.r0 + (col - ksub * kv.R);
