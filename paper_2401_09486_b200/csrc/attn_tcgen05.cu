@@ -351,8 +351,8 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             uint32_t gs = 0, tcount = 0;
             bool ok = true;
             for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
-                const int rank = w / p.BH, bh = w - rank * p.BH;
-                const int bi = bh / p.H, hi = bh - bi * p.H;
+                const int rank = fdiv(w, p.dBH), bh = w - rank * p.BH;
+                const int bi = fdiv(bh, p.dH), hi = bh - bi * p.H;
                 TileDesc td;
                 decode_tile(p, rank, td);
                 const View& qv = p.view[td.view];
@@ -434,7 +434,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             };
             uint32_t ge_s = 0, ge_p = 0;   // events whose scores / whose P.V have been issued
             for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
-                const int rank = w / p.BH;
+                const int rank = fdiv(w, p.dBH);
                 TileDesc td;
                 decode_tile(p, rank, td);
                 const HalfMasks hm = tile_half_masks(p, td, lane);
@@ -485,12 +485,12 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         bool ok = true;
         bool store_pending = false;
         for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r)) {
-            const int rank = w / p.BH, bh = w - rank * p.BH;
-            const int bi = bh / p.H, hi = bh - bi * p.H;
+            const int rank = fdiv(w, p.dBH), bh = w - rank * p.BH;
+            const int bi = fdiv(bh, p.dH), hi = bh - bi * p.H;
             TileDesc td;
             decode_tile(p, rank, td);
             const View& qv = p.view[td.view];
-            const int rsub = rr / qv.R;
+            const int rsub = fdiv(rr, qv.dR);
             const int ro = td.r0 + (rr - rsub * qv.R);
             const int rc = td.a0 + rsub;
             const bool row_valid = (rr < qv.R * qv.CH) && (rc <= td.a1) && (ro < qv.Z);

@@ -12,6 +12,32 @@ namespace loma {
 __host__ __device__ __forceinline__ int plan_min(int a, int b) { return a < b ? a : b; }
 __host__ __device__ __forceinline__ int plan_max(int a, int b) { return a > b ? a : b; }
 
+// Division by a divisor fixed at launch, as one multiply-high, one subtract, one add and two shifts
+// (Granlund and Montgomery, "Division by invariant integers using multiplication", 1994, the
+// unsigned 32-bit case); exact for every numerator 0 <= n < 2^32.  The kernel decodes a tile with
+// half a dozen dependent divisions, which as emulated hardware divisions cost over a microsecond.
+struct FastDiv {
+    unsigned mul, sh1, sh2;
+};
+inline FastDiv make_fastdiv(int d) {
+    if (d < 1) d = 1;
+    int l = 0;
+    while ((1ull << l) < (unsigned long long)d) ++l;
+    FastDiv f;
+    f.mul = (unsigned)((((1ull << l) - (unsigned long long)d) << 32) / (unsigned long long)d + 1ull);
+    f.sh1 = l < 1 ? l : 1;
+    f.sh2 = l > 1 ? l - 1 : 0;
+    return f;
+}
+__host__ __device__ __forceinline__ int fdiv(int n, const FastDiv& f) {
+#ifdef __CUDA_ARCH__
+    const unsigned t = __umulhi(f.mul, (unsigned)n);
+#else
+    const unsigned t = (unsigned)(((unsigned long long)f.mul * (unsigned)n) >> 32);
+#endif
+    return (int)((t + (((unsigned)n - t) >> f.sh1)) >> f.sh2);
+}
+
 enum { V_READ = 0, V_MEM = 1, V_REP = 2, V_TAIL = 3 };
 enum { M_LT = 0, M_LE = 1, M_EQ = 2, M_CAUSAL = 3, M_DIAG = 4 };
 
@@ -24,6 +50,7 @@ struct View {
     int nch;         // chunks in the view
     int chunk_base;  // absolute chunk number of the view's chunk 0 (n_chunks for the tail)
     int zone_row0;   // first row of the zone inside its chunk
+    FastDiv dR, dCH, dtpc;   // division by R, CH and tpc
 };
 
 struct FwdParams {
@@ -32,6 +59,7 @@ struct FwdParams {
     int total_tiles;
     int n_tail, n_read, n_mem, n_rep;   // tiles per view, in scheduling order
     unsigned flags;
+    FastDiv dBH, dH;
     float scale_log2;
     float* lse;
     int* status;
@@ -52,9 +80,9 @@ struct KTile {
 };
 
 // ------------------------------------------------------------------ tile lists
-__host__ __device__ __forceinline__ int tile_of_chunk(const View& v, int c) { return v.Z >= 128 ? c * v.tpc : c / v.CH; }
+__host__ __device__ __forceinline__ int tile_of_chunk(const View& v, int c) { return v.Z >= 128 ? c * v.tpc : fdiv(c, v.dCH); }
 __host__ __device__ __forceinline__ int tiles_covering(const View& v, int nchunks) {
-    return v.Z >= 128 ? nchunks * v.tpc : (nchunks + v.CH - 1) / v.CH;
+    return v.Z >= 128 ? nchunks * v.tpc : fdiv(nchunks + v.CH - 1, v.dCH);
 }
 
 __host__ __device__ __forceinline__ void decode_tile(const FwdParams& p, int rank, TileDesc& td) {
@@ -66,7 +94,7 @@ __host__ __device__ __forceinline__ void decode_tile(const FwdParams& p, int ran
     const View& g = p.view[view];
     td.view = view; td.qi = qi;
     int c1;
-    if (g.Z >= 128) { td.c0 = qi / g.tpc; td.r0 = (qi - td.c0 * g.tpc) * 128; c1 = td.c0; }
+    if (g.Z >= 128) { td.c0 = fdiv(qi, g.dtpc); td.r0 = (qi - td.c0 * g.tpc) * 128; c1 = td.c0; }
     else { td.c0 = qi * g.CH; td.r0 = 0; c1 = plan_min(td.c0 + g.CH, g.nch) - 1; }
     td.a0 = g.chunk_base + td.c0;
     td.a1 = g.chunk_base + c1;
@@ -99,7 +127,7 @@ __host__ __device__ __forceinline__ void step_ktile(const FwdParams& p, const Ti
     const int t = first ? td.seg[0].first + j : td.seg[1].first + (j - td.seg[0].count);
     const View& g = p.view[view];
     kt.view = view; kt.mode = mode;
-    if (g.Z >= 128) { kt.c0 = t / g.tpc; kt.r0 = (t - kt.c0 * g.tpc) * 128; }
+    if (g.Z >= 128) { kt.c0 = fdiv(t, g.dtpc); kt.r0 = (t - kt.c0 * g.tpc) * 128; }
     else { kt.c0 = t * g.CH; kt.r0 = 0; }
     kt.a0 = g.chunk_base + kt.c0;
 }
@@ -175,11 +203,13 @@ struct HalfWalk {
 inline View make_view(int Z, int nch, int chunk_base, int zone_row0) {
     View v{};
     v.Z = Z; v.nch = nch; v.chunk_base = chunk_base; v.zone_row0 = zone_row0;
+    v.dR = v.dCH = v.dtpc = make_fastdiv(1);
     if (Z <= 0 || nch <= 0) { v.R = 1; v.CH = 1; v.tpc = 0; v.ntiles = 0; v.Z = (Z > 0 ? Z : 1); v.nch = 0; return v; }
     v.R = Z < 128 ? Z : 128;
     v.CH = Z >= 128 ? 1 : 128 / Z;
     v.tpc = Z >= 128 ? (Z + 127) / 128 : 0;
     v.ntiles = Z >= 128 ? nch * v.tpc : (nch + v.CH - 1) / v.CH;
+    v.dR = make_fastdiv(v.R); v.dCH = make_fastdiv(v.CH); v.dtpc = make_fastdiv(v.tpc);
     return v;
 }
 
@@ -193,6 +223,7 @@ inline void make_plan(const Layout& L, int B, int H, FwdParams* p) {
     p->n_mem = p->view[V_MEM].ntiles; p->n_rep = p->view[V_REP].ntiles;
     p->total_tiles = p->n_tail + p->n_read + p->n_mem + p->n_rep;
     p->flags = L.flags;
+    p->dBH = make_fastdiv(p->BH); p->dH = make_fastdiv(H);
 }
 
 }  // namespace loma
