@@ -484,23 +484,42 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         uint32_t ge = 0;   // visited halves so far (see the MMA issuer)
         bool ok = true;
         bool store_pending = false;
-        for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r)) {
-            const int rank = fdiv(w, p.dBH), bh = w - rank * p.BH;
-            const int bi = fdiv(bh, p.dH), hi = bh - bi * p.H;
+        // Everything this thread needs to know about a tile.  The next tile is decoded while the last
+        // product of the current one drains, so the decode's chain of dependent loads and integer
+        // arithmetic stays off the path between two tiles.
+        struct TileCtx {
             TileDesc td;
-            decode_tile(p, rank, td);
-            const View& qv = p.view[td.view];
+            HalfMasks hm;
+            int bh, bi, hi, ro, rc, zone_row0;
+            bool row_valid;
+        };
+        auto decode_ctx = [&](int w, TileCtx& c) {
+            const int rank = fdiv(w, p.dBH);
+            c.bh = w - rank * p.BH;
+            c.bi = fdiv(c.bh, p.dH);
+            c.hi = c.bh - c.bi * p.H;
+            decode_tile(p, rank, c.td);
+            const View& qv = p.view[c.td.view];
             const int rsub = fdiv(rr, qv.dR);
-            const int ro = td.r0 + (rr - rsub * qv.R);
-            const int rc = td.a0 + rsub;
-            const bool row_valid = (rr < qv.R * qv.CH) && (rc <= td.a1) && (ro < qv.Z);
+            c.ro = c.td.r0 + (rr - rsub * qv.R);
+            c.rc = c.td.a0 + rsub;
+            c.zone_row0 = qv.zone_row0;
+            c.row_valid = (rr < qv.R * qv.CH) && (c.rc <= c.td.a1) && (c.ro < qv.Z);
+            c.hm = tile_half_masks(p, c.td, lane);
+        };
+        TileCtx cur, nxt;
+        if (sid < total_work) decode_ctx(sid, cur);
+        for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), cur = nxt) {
+            const TileDesc& td = cur.td;
+            const HalfMasks hm = cur.hm;
+            const int bh = cur.bh, bi = cur.bi, hi = cur.hi, ro = cur.ro, rc = cur.rc;
+            const bool row_valid = cur.row_valid;
 
             // Running reference maximum (exp2 domain) and row sum.  The reference only moves
             // when the row maximum has grown by more than 2^8 since it was set; then the
             // output accumulator in TMEM is rescaled once.  Probabilities stay below 2^8.
             float m_used = -INFINITY, l = 0.f;
 
-            const HalfMasks hm = tile_half_masks(p, td, lane);
             HalfWalk hw;
             bool first = true;
             int lo = 0, hi2 = 0;
@@ -589,6 +608,10 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     mbar_arrive(bar(B_PF + b));
                 }
             }
+            {
+                const int wn = tile_of_round(r + 1);
+                if (wn < total_work) decode_ctx(wn, nxt);
+            }
             // the last P.V of the tile belongs to event ge - 1 (products complete in issue order)
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + ((ge - 1) & 1)), ((ge - 1) >> 1) & 1, abortp, p.status));
             if (ok) tc_fence_after();
@@ -640,7 +663,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             if (give_up) { ok = false; break; }
             tc_fence_before();
             if (p.lse && row_valid) {
-                const int64_t grow = (int64_t)rc * p.s + qv.zone_row0 + ro;
+                const int64_t grow = (int64_t)rc * p.s + cur.zone_row0 + ro;
                 p.lse[(int64_t)bh * p.S + grow] = (m_used + log2f(l)) * 0.6931471805599453f;
             }
         }
