@@ -2,7 +2,7 @@
 
 Everything under this package is a plain, slow, fp64 NumPy restatement of what
 the paper defines: the chunk layout (Section 4.1), the attention mask
-(Eq. 1-3), masked softmax attention (Eq. 6-7), and the generation-time cache
+(Eq. 1-3), masked softmax attention (Eq. 6-7) and its gradients (Section 4.4), and the generation-time cache
 algebra (Section 3.1 and Appendix A).  It exists only so that tests, the smoke
 check and the CPU-baseline leg of the benchmark have something independent to
 compare the CUDA library against.  It shares no code with the CUDA path and the
@@ -27,6 +27,8 @@ from .loma_oracle import (  # noqa: F401
     mask_rows,
     masked_softmax_attention,
     masked_attn_fwd,
+    masked_softmax_attention_bwd,
+    masked_attn_bwd,
     decode_attn,
     compress_step,
     replay_generation,

@@ -321,6 +321,55 @@ def masked_attn_fwd(q, k, v, n_chunks, c, t, tail_read=0, flags=0, scale=None,
 
 
 # --------------------------------------------------------------------------
+# Backward of the masked attention (Section 4.4: gradient propagation, Eq. 10)
+# --------------------------------------------------------------------------
+
+def masked_softmax_attention_bwd(q, k, v, d_o, mask, scale=None):
+    """Gradients of O = Softmax(A) V (Eq. 7), A = scale * Q K^T on the mask.
+
+    Given dO = dLoss/dO this is the chain rule written out term by term:
+      * O is linear in V:                      dV = P^T dO
+      * O is linear in P:                      dP = dO V^T
+      * row i of P is a softmax of row i of A (blocked entries have P = 0 and
+        take no part), whose Jacobian is diag(P_i) - P_i P_i^T:
+                                               dA_ij = P_ij (dP_ij - sum_k P_ik dP_ik)
+      * A = scale * Q K^T:                     dQ = scale * dA K,  dK = scale * dA^T Q
+    Section 4.4 follows exactly these paths when it argues (Eq. 10) that the
+    repetition loss reaches k_m and v_m; here nothing is dropped.
+
+    q [R, D], k [C, D], v [C, Dv], d_o [R, Dv], mask boolean [R, C].
+    Returns (dQ [R, D], dK [C, D], dV [C, Dv]) in float64.
+    """
+    q, k, v, d_o = _f64(q), _f64(k), _f64(v), _f64(d_o)
+    if scale is None:
+        scale = 1.0 / np.sqrt(q.shape[-1])
+    _, P, _ = masked_softmax_attention(q, k, v, mask, scale)
+    dV = P.T @ d_o
+    dP = d_o @ v.T
+    row_dot = (P * dP).sum(axis=1, keepdims=True)
+    dA = P * (dP - row_dot)
+    dQ = scale * (dA @ k)
+    dK = scale * (dA.T @ q)
+    return dQ, dK, dV
+
+
+def masked_attn_bwd(q, k, v, d_o, n_chunks, c, t, tail_read=0, flags=0, scale=None):
+    """Gradients of masked_attn_fwd with respect to q, k and v, all rows.
+
+    q, k, v, d_o: [B, H, S, D].  Returns (dQ, dK, dV), each [B, H, S, D] float64.
+    """
+    q, k, v, d_o = _f64(q), _f64(k), _f64(v), _f64(d_o)
+    B, H, S, D = q.shape
+    assert S == seq_len(n_chunks, c, t, tail_read, flags)
+    M = dense_mask(n_chunks, c, t, tail_read, flags)
+    dQ, dK, dV = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v)
+    for b in range(B):
+        for h in range(H):
+            dQ[b, h], dK[b, h], dV[b, h] = masked_softmax_attention_bwd(q[b, h], k[b, h], v[b, h], d_o[b, h], M, scale)
+    return dQ, dK, dV
+
+
+# --------------------------------------------------------------------------
 # Generation (Section 3.1, Appendix A)
 # --------------------------------------------------------------------------
 
