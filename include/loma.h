@@ -5,6 +5,7 @@
  * Three device operations and two integer index maps:
  *
  *   loma_masked_attn_fwd   zone-masked attention over the training layout
+ *   loma_masked_attn_bwd   its gradients with respect to q, k and v
  *                          (Section 4.3, Eq. 1-3; Section 4.4, Eq. 5-7)
  *   loma_decode_attn       one generated token over the compressed cache
  *                          (Section 3.1 steps 1 and 3; Appendix A, inference_input)
@@ -167,6 +168,35 @@ LOMA_API int loma_masked_attn_fwd(const void* q, const void* k, const void* v, v
                                   int n_chunks, int c, int t, int tc, int tail_read,
                                   int64_t stride_b, int64_t stride_h, int64_t stride_s,
                                   loma_dtype dtype, float softmax_scale, unsigned flags, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * loma_masked_attn_bwd -- gradients of loma_masked_attn_fwd: the chain rule through
+ * O = Softmax(A) V of Eq. 7, the paths Section 4.4 follows to Eq. 10 (a loss on the
+ * repetition rows reaches k_m and v_m).  With P_ij = exp(scale q_i.k_j - lse_i) on the
+ * entries Eq. 2 allows and dA_ij = P_ij (dO_i.v_j - dO_i.O_i):
+ *      dQ = scale dA K      dK = scale dA^T Q      dV = P^T dO
+ * Blocked entries carry no gradient.  Every output row is produced by one owner in a fixed
+ * order (no atomics): results repeat bit for bit.
+ *
+ *   q, k, v, o, d_o [device, in]   [B, H, S, D] with the strides of loma_masked_attn_fwd;
+ *                                  o and lse are the forward's outputs for these q, k, v
+ *   lse             [device, in]   fp32 [B, H, S] contiguous (natural-log normaliser)
+ *   dq, dk, dv      [device, out]  same shape, strides and dtype as q; must not alias an input
+ *   workspace       [device]       at least loma_masked_attn_bwd_workspace_bytes(...) bytes,
+ *                                  256-byte aligned; contents need not be initialised
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, WORKSPACE, CUDA.  S == 0 or B*H == 0 is a no-op.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_masked_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                                  const float* lse, void* dq, void* dk, void* dv,
+                                  int B, int H, int D,
+                                  int n_chunks, int c, int t, int tc, int tail_read,
+                                  int64_t stride_b, int64_t stride_h, int64_t stride_s,
+                                  loma_dtype dtype, float softmax_scale, unsigned flags,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* Workspace size in bytes for loma_masked_attn_bwd (0 for an invalid layout). */
+LOMA_API size_t loma_masked_attn_bwd_workspace_bytes(int B, int H, int D, int n_chunks, int c, int t, int tail_read,
+                                                     unsigned flags);
 
 /* ---------------------------------------------------------------------------
  * loma_prefill_cache -- what the cache holds after a prompt has been ingested (Section 3.1 step 3

@@ -34,6 +34,9 @@ SIGNATURES = {
     "loma_generation_index": (_i, [_i, _i, _i, _p, _p, _p, _i, _p]),
     "loma_masked_attn_fwd": (_i, [_p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i, _f,
                                   _u, _p]),
+    "loma_masked_attn_bwd": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i,
+                                  _f, _u, _p, _sz, _p]),
+    "loma_masked_attn_bwd_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i, _u]),
     "loma_masked_attn_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
@@ -160,6 +163,32 @@ def loma_masked_attn_fwd(q, k, v, o, lse, n_chunks: int, c: int, t: int, tail_re
                                     tail_read, q.stride(0), q.stride(1), q.stride(2), _dtype_code(q),
                                     float(softmax_scale), int(flags), _stream(stream))
     _check(rc, "loma_masked_attn_fwd")
+
+
+def loma_masked_attn_bwd_workspace_bytes(B: int, H: int, D: int, n_chunks: int, c: int, t: int, tail_read: int = 0,
+                                         flags: int = 0) -> int:
+    return int(lib().loma_masked_attn_bwd_workspace_bytes(B, H, D, n_chunks, c, t, tail_read, int(flags)))
+
+
+def loma_masked_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, n_chunks: int, c: int, t: int, tail_read: int = 0,
+                         flags: int = 0, workspace=None, softmax_scale: float = 0.0, stream=None) -> None:
+    """Gradients of loma_masked_attn_fwd.  q, k, v, o, d_o, dq, dk, dv: [B, H, S, D] device tensors with
+    identical strides; lse: the forward's fp32 [B, H, S]; workspace: a device byte buffer of at least
+    loma_masked_attn_bwd_workspace_bytes(...) bytes."""
+    B, H, S, D = q.shape
+    for x in (k, v, o, d_o, dq, dk, dv):
+        if x.shape != q.shape or x.stride() != q.stride() or x.dtype != q.dtype:
+            raise ValueError("all tensors must share shape, strides and dtype")
+    if q.stride(3) != 1:
+        raise ValueError("head dimension must be contiguous")
+    if lse.dtype != torch.float32 or not lse.is_contiguous():
+        raise ValueError("lse must be contiguous fp32")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().loma_masked_attn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq), _ptr(dk),
+                                    _ptr(dv), B, H, D, n_chunks, c, t, c * t, tail_read, q.stride(0), q.stride(1),
+                                    q.stride(2), _dtype_code(q), float(softmax_scale), int(flags), _ptr(workspace),
+                                    ws_bytes, _stream(stream))
+    _check(rc, "loma_masked_attn_bwd")
 
 
 def loma_masked_attn_plan_coverage(n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0) -> torch.Tensor:

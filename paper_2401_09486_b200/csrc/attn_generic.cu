@@ -175,6 +175,39 @@ struct TrainMap {
     __device__ __forceinline__ const T* vptr(int vi) const { return v + row(vi) * ss; }
 };
 
+// (chunk, zone, offset) of row i, as in Section 4.1; the reading tail counts as chunk n_chunks
+__device__ __forceinline__ void decompose_row(const Layout& L, int i, int& y, int& zone, int& off) {
+    if (L.s == 0 || i >= L.n_chunks * L.s) {
+        y = L.n_chunks; zone = LOMA_ZONE_READ; off = i - L.n_chunks * L.s;
+    } else {
+        y = i / L.s;
+        const int r = i - y * L.s;
+        if (r < L.tc) { zone = LOMA_ZONE_READ; off = r; }
+        else if (r < L.tc + L.t) { zone = LOMA_ZONE_MEM; off = r - L.tc; }
+        else { zone = LOMA_ZONE_REP; off = r - L.tc - L.t; }
+    }
+}
+
+// Fills the visible-key map of row i and returns its number of visible keys.
+template <typename T>
+__device__ __forceinline__ int train_row_map(const Layout& L, int i, const T* k, const T* v, int64_t ss, TrainMap<T>& map) {
+    int y, zone, off;
+    decompose_row(L, i, y, zone, off);
+    map.k = k; map.v = v; map.ss = ss; map.s = L.s; map.tc = L.tc; map.t = L.t;
+    map.n_range = 0; map.self = 0;
+    if (zone == LOMA_ZONE_READ) {                 // Eq. 3 reading rows + L of Eq. 1
+        map.kind = 0; map.n_prior = y * L.t; map.lo = y * L.s;
+        return map.n_prior + off + 1;
+    }
+    if (zone == LOMA_ZONE_MEM) {                  // Eq. 1 second block row
+        map.kind = 0; map.lo = y * L.s;
+        map.n_prior = (L.flags & LOMA_FLAG_MEM_SEES_PRIOR_MEM) ? y * L.t : 0;
+        return map.n_prior + L.tc + L.t;
+    }
+    map.kind = 1; map.n_prior = 0; map.lo = y * L.s + L.tc; map.n_range = L.t; map.self = i;   // Eq. 1 third block row
+    return L.t + 1;
+}
+
 constexpr int GENERIC_WARPS = 8;
 
 template <typename T, int D>
@@ -190,33 +223,8 @@ masked_attn_generic_kernel(const T* __restrict__ q, const T* __restrict__ k, con
     const int b = bh / H, h = bh - b * H;
     const int64_t base = (int64_t)b * sb + (int64_t)h * sh;
 
-    // (chunk, zone, offset) of the row, as in Section 4.1
-    int y, zone, off;
-    if (L.s == 0 || i >= L.n_chunks * L.s) {
-        y = L.n_chunks; zone = LOMA_ZONE_READ; off = i - L.n_chunks * L.s;
-    } else {
-        y = i / L.s;
-        const int r = i - y * L.s;
-        if (r < L.tc) { zone = LOMA_ZONE_READ; off = r; }
-        else if (r < L.tc + L.t) { zone = LOMA_ZONE_MEM; off = r - L.tc; }
-        else { zone = LOMA_ZONE_REP; off = r - L.tc - L.t; }
-    }
-
     TrainMap<T> map;
-    map.k = k + base; map.v = v + base; map.ss = ss; map.s = L.s; map.tc = L.tc; map.t = L.t;
-    map.n_range = 0; map.self = 0;
-    int nkeys;
-    if (zone == LOMA_ZONE_READ) {                 // Eq. 3 reading rows + L of Eq. 1
-        map.kind = 0; map.n_prior = y * L.t; map.lo = y * L.s;
-        nkeys = map.n_prior + off + 1;
-    } else if (zone == LOMA_ZONE_MEM) {           // Eq. 1 second block row
-        map.kind = 0; map.lo = y * L.s;
-        map.n_prior = (L.flags & LOMA_FLAG_MEM_SEES_PRIOR_MEM) ? y * L.t : 0;
-        nkeys = map.n_prior + L.tc + L.t;
-    } else {                                      // Eq. 1 third block row
-        map.kind = 1; map.n_prior = 0; map.lo = y * L.s + L.tc; map.n_range = L.t; map.self = i;
-        nkeys = L.t + 1;
-    }
+    const int nkeys = train_row_map(L, i, k + base, v + base, ss, map);
     stage_query<T, D>(q_sh[warp], q + base + (int64_t)i * ss, lane);
     attend_row<T, D>(q_sh[warp], map, nkeys, scale, o + base + (int64_t)i * ss,
                      lse ? lse + (int64_t)bh * L.S + i : nullptr, lane);
@@ -314,6 +322,162 @@ compress_generic_kernel(const T* __restrict__ q_mem, const T* __restrict__ k_mem
     }
 }
 
+// ------------------------------------------------------------ masked backward
+// Gradients of Eq. 7 (Section 4.4).  With P_ij = exp(scale q_i.k_j - lse_i) on the allowed
+// entries, delta_i = dO_i . O_i (= sum_j P_ij dP_ij) and dA_ij = P_ij (dO_i . v_j - delta_i):
+//   dQ_i = scale sum_j dA_ij k_j     one warp per query row, over the keys the row sees
+//   dK_j = scale sum_i dA_ij q_i     one warp per key row, over the rows that see the key
+//   dV_j =       sum_i P_ij dO_i
+// Each output row is owned by one warp: no atomics, results repeat bit for bit.
+template <typename T, int D>
+__global__ void __launch_bounds__(GENERIC_WARPS * 32)
+masked_attn_bwd_dq_generic_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                                  const T* __restrict__ o, const T* __restrict__ d_o, const float* __restrict__ lse,
+                                  T* __restrict__ dq, float* __restrict__ delta, int H, Layout L, int64_t sb, int64_t sh,
+                                  int64_t ss, float scale) {
+    __shared__ __align__(16) float q_sh[GENERIC_WARPS][D];
+    __shared__ __align__(16) float g_sh[GENERIC_WARPS][D];
+    constexpr int DPL = D / 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int i = blockIdx.x * GENERIC_WARPS + warp;
+    if (i >= L.S) return;
+    const int bh = blockIdx.y;
+    const int b = bh / H, h = bh - b * H;
+    const int64_t base = (int64_t)b * sb + (int64_t)h * sh;
+    TrainMap<T> map;
+    const int nkeys = train_row_map(L, i, k + base, v + base, ss, map);
+    stage_query<T, D>(q_sh[warp], q + base + (int64_t)i * ss, lane);
+    stage_query<T, D>(g_sh[warp], d_o + base + (int64_t)i * ss, lane);
+    float dl;
+    {
+        float ov[DPL];
+        Io<T>::template load<DPL>(o + base + (int64_t)i * ss + lane * DPL, ov);
+        float part = 0.f;
+#pragma unroll
+        for (int d = 0; d < DPL; ++d) part = fmaf(g_sh[warp][lane * DPL + d], ov[d], part);
+        dl = warp_sum(part);
+        if (lane == 0) delta[(int64_t)bh * L.S + i] = dl;
+    }
+    const float lse_i = lse[(int64_t)bh * L.S + i];
+    float acc[DPL];
+#pragma unroll
+    for (int d = 0; d < DPL; ++d) acc[d] = 0.f;
+    for (int kb = 0; kb < nkeys; kb += 32) {
+        const int vi = kb + lane;
+        float da = 0.f;
+        if (vi < nkeys) {
+            const float sc = Io<T>::template dot<D>(q_sh[warp], map.kptr(vi)) * scale;
+            const float p = expf(sc - lse_i);
+            const float dp = Io<T>::template dot<D>(g_sh[warp], map.vptr(vi));
+            da = p * (dp - dl);
+        }
+        const int cnt = min(32, nkeys - kb);
+        for (int jj = 0; jj < cnt; ++jj) {
+            const float dj = __shfl_sync(0xffffffffu, da, jj);
+            float kk[DPL];
+            Io<T>::template load<DPL>(map.kptr(kb + jj) + lane * DPL, kk);
+#pragma unroll
+            for (int d = 0; d < DPL; ++d) acc[d] = fmaf(dj, kk[d], acc[d]);
+        }
+    }
+#pragma unroll
+    for (int d = 0; d < DPL; ++d) acc[d] *= scale;
+    Io<T>::template store<DPL>(dq + base + (int64_t)i * ss + lane * DPL, acc);
+}
+
+// Rows that see key j, as a visible index -> row map (the columns of Eq. 2 read downwards):
+//   reading key (y, o):    reading rows o.. of chunk y, then the chunk's memory rows (contiguous)
+//   memory key (y, j):     memory and repetition rows of chunk y (contiguous), then the reading
+//                          rows [and, with the prior-memory flag, memory rows] of every later
+//                          chunk, then the reading tail
+//   repetition key:        its own row
+struct SeenByMap {
+    int lo, n_first;      // first contiguous range
+    int y_next, seg_len;  // later chunks y_next.. contribute rows [y*s, y*s + seg_len)
+    int n_later, s, tail0;
+    __device__ __forceinline__ int row(int vi) const {
+        if (vi < n_first) return lo + vi;
+        vi -= n_first;
+        if (vi < n_later) {
+            const int x = vi / seg_len;
+            return (y_next + x) * s + (vi - x * seg_len);
+        }
+        return tail0 + (vi - n_later);
+    }
+};
+
+__device__ __forceinline__ int seen_by_map(const Layout& L, int j, SeenByMap& m) {
+    int y, zone, off;
+    decompose_row(L, j, y, zone, off);
+    m.s = L.s; m.tail0 = L.n_chunks * L.s; m.n_later = 0; m.seg_len = 1; m.y_next = 0;
+    if (zone == LOMA_ZONE_READ) {
+        m.lo = j;
+        m.n_first = (y == L.n_chunks) ? L.S - j : (L.tc - off) + L.t;
+        return m.n_first;
+    }
+    if (zone == LOMA_ZONE_REP) { m.lo = j; m.n_first = 1; return 1; }
+    m.lo = y * L.s + L.tc;
+    m.n_first = (y + 1) * L.s - m.lo;
+    m.y_next = y + 1;
+    m.seg_len = L.tc + ((L.flags & LOMA_FLAG_MEM_SEES_PRIOR_MEM) ? L.t : 0);
+    m.n_later = (L.n_chunks - 1 - y) * m.seg_len;
+    return m.n_first + m.n_later + L.tail_read;
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(GENERIC_WARPS * 32)
+masked_attn_bwd_dkv_generic_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                                   const T* __restrict__ d_o, const float* __restrict__ lse,
+                                   const float* __restrict__ delta, T* __restrict__ dk, T* __restrict__ dv, int H,
+                                   Layout L, int64_t sb, int64_t sh, int64_t ss, float scale) {
+    __shared__ __align__(16) float k_sh[GENERIC_WARPS][D];
+    __shared__ __align__(16) float v_sh[GENERIC_WARPS][D];
+    constexpr int DPL = D / 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int j = blockIdx.x * GENERIC_WARPS + warp;
+    if (j >= L.S) return;
+    const int bh = blockIdx.y;
+    const int b = bh / H, h = bh - b * H;
+    const int64_t base = (int64_t)b * sb + (int64_t)h * sh;
+    SeenByMap map;
+    const int nrows = seen_by_map(L, j, map);
+    stage_query<T, D>(k_sh[warp], k + base + (int64_t)j * ss, lane);
+    stage_query<T, D>(v_sh[warp], v + base + (int64_t)j * ss, lane);
+    float acc_k[DPL], acc_v[DPL];
+#pragma unroll
+    for (int d = 0; d < DPL; ++d) { acc_k[d] = 0.f; acc_v[d] = 0.f; }
+    for (int rb = 0; rb < nrows; rb += 32) {
+        const int vi = rb + lane;
+        float p = 0.f, da = 0.f;
+        int i = 0;
+        if (vi < nrows) {
+            i = map.row(vi);
+            const float sc = Io<T>::template dot<D>(k_sh[warp], q + base + (int64_t)i * ss) * scale;
+            p = expf(sc - lse[(int64_t)bh * L.S + i]);
+            const float dp = Io<T>::template dot<D>(v_sh[warp], d_o + base + (int64_t)i * ss);
+            da = p * (dp - delta[(int64_t)bh * L.S + i]);
+        }
+        const int cnt = min(32, nrows - rb);
+        for (int jj = 0; jj < cnt; ++jj) {
+            const float pj = __shfl_sync(0xffffffffu, p, jj);
+            const float dj = __shfl_sync(0xffffffffu, da, jj);
+            const int ii = __shfl_sync(0xffffffffu, i, jj);
+            float qq[DPL], gg[DPL];
+            Io<T>::template load<DPL>(q + base + (int64_t)ii * ss + lane * DPL, qq);
+            Io<T>::template load<DPL>(d_o + base + (int64_t)ii * ss + lane * DPL, gg);
+#pragma unroll
+            for (int d = 0; d < DPL; ++d) {
+                acc_k[d] = fmaf(dj, qq[d], acc_k[d]);
+                acc_v[d] = fmaf(pj, gg[d], acc_v[d]);
+            }
+        }
+    }
+#pragma unroll
+    for (int d = 0; d < DPL; ++d) acc_k[d] *= scale;
+    Io<T>::template store<DPL>(dk + base + (int64_t)j * ss + lane * DPL, acc_k);
+    Io<T>::template store<DPL>(dv + base + (int64_t)j * ss + lane * DPL, acc_v);
+}
+
 // ------------------------------------------------------------------ launchers
 template <typename T, int D>
 static cudaError_t masked_generic_t(const void* q, const void* k, const void* v, void* o, float* lse, int B,
@@ -336,6 +500,34 @@ cudaError_t launch_masked_attn_generic(const void* q, const void* k, const void*
     }
     return D == 64 ? masked_generic_t<__nv_bfloat16, 64>(q, k, v, o, lse, B, H, L, sb, sh, ss, scale, st)
                    : masked_generic_t<__nv_bfloat16, 128>(q, k, v, o, lse, B, H, L, sb, sh, ss, scale, st);
+}
+
+template <typename T, int D>
+static cudaError_t masked_bwd_generic_t(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                                        const float* lse, void* dq, void* dk, void* dv, float* delta, int B, int H,
+                                        const Layout& L, int64_t sb, int64_t sh, int64_t ss, float scale,
+                                        cudaStream_t st) {
+    dim3 grid((L.S + GENERIC_WARPS - 1) / GENERIC_WARPS, B * H);
+    masked_attn_bwd_dq_generic_kernel<T, D><<<grid, GENERIC_WARPS * 32, 0, st>>>(
+        static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), static_cast<const T*>(o),
+        static_cast<const T*>(d_o), lse, static_cast<T*>(dq), delta, H, L, sb, sh, ss, scale);
+    masked_attn_bwd_dkv_generic_kernel<T, D><<<grid, GENERIC_WARPS * 32, 0, st>>>(
+        static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), static_cast<const T*>(d_o), lse,
+        delta, static_cast<T*>(dk), static_cast<T*>(dv), H, L, sb, sh, ss, scale);
+    count_launches(2);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_masked_attn_bwd_generic(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                                           const float* lse, void* dq, void* dk, void* dv, float* delta, int B, int H,
+                                           int D, const Layout& L, int64_t sb, int64_t sh, int64_t ss, loma_dtype dt,
+                                           float scale, cudaStream_t st) {
+    if (dt == LOMA_F32) {
+        return D == 64 ? masked_bwd_generic_t<float, 64>(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, L, sb, sh, ss, scale, st)
+                       : masked_bwd_generic_t<float, 128>(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, L, sb, sh, ss, scale, st);
+    }
+    return D == 64 ? masked_bwd_generic_t<__nv_bfloat16, 64>(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, L, sb, sh, ss, scale, st)
+                   : masked_bwd_generic_t<__nv_bfloat16, 128>(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, L, sb, sh, ss, scale, st);
 }
 
 template <typename T, int D>

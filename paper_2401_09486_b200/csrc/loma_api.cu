@@ -148,6 +148,55 @@ int loma_masked_attn_fwd(const void* q, const void* k, const void* v, void* o, f
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 
+size_t loma_masked_attn_bwd_workspace_bytes(int B, int H, int D, int n_chunks, int c, int t, int tail_read,
+                                            unsigned flags) {
+    (void)D;
+    Layout L;
+    if (B < 0 || H < 0 || make_layout(n_chunks, c, t, tail_read, flags, &L) != LOMA_OK) return 0;
+    const size_t bytes = (size_t)B * H * L.S * sizeof(float);   // delta_i = dO_i . O_i
+    return (bytes + 255) & ~(size_t)255;
+}
+
+int loma_masked_attn_bwd(const void* q, const void* k, const void* v, const void* o, const void* d_o, const float* lse,
+                         void* dq, void* dk, void* dv, int B, int H, int D, int n_chunks, int c, int t, int tc,
+                         int tail_read, int64_t stride_b, int64_t stride_h, int64_t stride_s, loma_dtype dtype,
+                         float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes, void* stream) {
+    if (B < 0 || H < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    Layout L;
+    const int rc = make_layout(n_chunks, c, t, tail_read, flags, &L);
+    if (rc != LOMA_OK) return rc;
+    if (tc != L.tc) return LOMA_ERR_INVALID_ARG;
+    if (L.S == 0 || B == 0 || H == 0) return LOMA_OK;
+    const void* ins[5] = {q, k, v, o, d_o};
+    void* outs[3] = {dq, dk, dv};
+    for (const void* p : ins) if (!p) return LOMA_ERR_INVALID_ARG;
+    if (!lse) return LOMA_ERR_INVALID_ARG;
+    for (int a = 0; a < 3; ++a) {
+        if (!outs[a]) return LOMA_ERR_INVALID_ARG;
+        for (const void* p : ins) if (outs[a] == p) return LOMA_ERR_INVALID_ARG;
+        for (int b2 = 0; b2 < a; ++b2) if (outs[a] == outs[b2]) return LOMA_ERR_INVALID_ARG;
+    }
+    if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
+    if (stride_s < D || stride_b < 0 || stride_h < 0) return LOMA_ERR_INVALID_ARG;
+    const size_t es = elt_size(dtype);
+    for (const void* p : ins) if (!aligned16(p)) return LOMA_ERR_ALIGNMENT;
+    for (void* p : outs) if (!aligned16(p)) return LOMA_ERR_ALIGNMENT;
+    if (((uintptr_t)lse & 3u) != 0) return LOMA_ERR_ALIGNMENT;
+    if ((stride_b * es) % 16 || (stride_h * es) % 16 || (stride_s * es) % 16) return LOMA_ERR_ALIGNMENT;
+    const size_t need = loma_masked_attn_bwd_workspace_bytes(B, H, D, n_chunks, c, t, tail_read, flags);
+    if (!workspace || workspace_bytes < need) return LOMA_ERR_WORKSPACE;
+    if (((uintptr_t)workspace & 255u) != 0) return LOMA_ERR_ALIGNMENT;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = launch_masked_attn_bwd_generic(q, k, v, o, d_o, lse, dq, dk, dv, static_cast<float*>(workspace), B, H,
+                                                   D, L, stride_b, stride_h, stride_s, dtype, scale, st);
+    return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
 int loma_prefill_cache(const void* k, const void* v, void* k_cache, void* v_cache, int B, int H, int D, int cap,
                        int n_chunks, int c, int t, int tc, int tail_read, int64_t stride_b, int64_t stride_h,
                        int64_t stride_s, loma_dtype dtype, unsigned flags, int* cache_len_out, void* stream) {

@@ -171,3 +171,25 @@ def test_tensor_core_tile_plan_reproduces_the_mask_exactly(lib, n, c, t, tail, f
     want = oracle.dense_mask(n, c, t, tail, flags).astype(np.uint8)
     assert got.shape == want.shape
     assert np.array_equal(got, want), f"{int((got != want).sum())} entries differ"
+
+
+def test_masked_attn_bwd_validation(lib):
+    def call(q=0x1000, k=0x2000, v=0x3000, o=0x4000, g=0x5000, lse=0x6000, dq=0x7000, dk=0x8000, dv=0x9000, B=1, H=1,
+             D=64, n=1, c=2, t=2, tc=4, tail=0, sb=640, sh=640, ss=64, dt=1, ws=0xa000, wsb=1 << 20):
+        return lib.loma_masked_attn_bwd(q, k, v, o, g, lse, dq, dk, dv, B, H, D, n, c, t, tc, tail, sb, sh, ss, dt, 0.0, 0,
+                                        ws, wsb, None)
+    assert call(tc=5) == INVALID
+    assert call(D=96) == UNSUPPORTED
+    assert call(lse=None) == INVALID
+    assert call(g=None) == INVALID
+    assert call(dk=0x2000) == INVALID                   # dk aliases k
+    assert call(dv=0x8000) == INVALID                   # dv aliases dk
+    assert call(dq=0x7008) == ALIGNMENT
+    assert call(ss=68) == ALIGNMENT
+    assert call(ws=None) == WORKSPACE
+    assert call(wsb=8) == WORKSPACE
+    assert call(ws=0xa010) == ALIGNMENT
+    assert call(B=0) == 0
+    need = lib.loma_masked_attn_bwd_workspace_bytes(4, 32, 128, 32, 4, 16, 0, 0)
+    assert need >= 4 * 32 * 4608 * 4 and need % 256 == 0
+    assert lib.loma_masked_attn_bwd_workspace_bytes(1, 1, 64, 1, 0, 2, 0, 0) == 0     # c < 1: no layout

@@ -1,0 +1,126 @@
+"""Parity of loma_masked_attn_bwd (through the C ABI) with the CPU oracle's
+backward, element by element on the same seeded inputs.
+
+The library is given what a training step has at hand: q, k, v, the output and
+log-sum-exp of its own forward, and dO.  The oracle gets the same stored q, k,
+v, dO and recomputes everything else in fp64.
+
+Tolerances.  Gradients are sums over up to thousands of rows, so their size
+varies with the layout; the bars of the forward (stated for outputs of size
+about one) are scaled by the size of the reference: fp32 max |delta| <= 1e-5 *
+max(1, max |ref|); bf16 max |delta| <= 2e-2 * max(1, max |ref|) and mean
+|delta| <= 2e-3 * max(1, mean |ref|).
+"""
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2401_09486_b200 import binding as L
+from paper_2401_09486_b200 import build, synthetic
+
+pytestmark = pytest.mark.gpu
+
+PRIOR = L.LOMA_FLAG_MEM_SEES_PRIOR_MEM
+NOREP = L.LOMA_FLAG_NO_REP_ZONE
+GENERIC = L.LOMA_FLAG_FORCE_GENERIC
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _library():
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    build.build_library()
+    L.lib()
+    torch.cuda.set_device(0)
+    yield
+    assert L.loma_device_status() == 0
+
+
+def npf(x):
+    return x.detach().to("cpu").to(torch.float64).numpy()
+
+
+def check_grad(got, want, dtype, name):
+    g = npf(got)
+    assert g.shape == want.shape and np.isfinite(g).all(), name
+    d = np.abs(g - want)
+    big, mean = max(1.0, np.abs(want).max()), max(1.0, np.abs(want).mean())
+    if dtype == torch.float32:
+        assert d.max() <= 1e-5 * big, f"{name}: fp32 max |delta| {d.max():.3e} (ref max {big:.3g})"
+    else:
+        assert d.max() <= 2e-2 * big, f"{name}: bf16 max |delta| {d.max():.3e} (ref max {big:.3g})"
+        assert d.mean() <= 2e-3 * mean, f"{name}: bf16 mean |delta| {d.mean():.3e}"
+
+
+def run_fwd_bwd(q, k, v, d_o, n, c, t, tail=0, flags=0, scale=0.0):
+    o = torch.full_like(q, float("nan"))
+    lse = torch.full(q.shape[:3], float("nan"), dtype=torch.float32, device=q.device)
+    L.loma_masked_attn_fwd(q, k, v, o, lse, n, c, t, tail, flags, scale)
+    B, H, S, D = q.shape
+    ws = torch.empty(max(256, L.loma_masked_attn_bwd_workspace_bytes(B, H, D, n, c, t, tail, flags)), dtype=torch.uint8,
+                     device=q.device)
+    dq, dk, dv = (torch.full_like(q, float("nan")) for _ in range(3))
+    L.loma_masked_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, n, c, t, tail, flags, ws, scale)
+    torch.cuda.synchronize()
+    return dq, dk, dv
+
+
+BWD_CASES = [
+    # B, H, D, n, c, t, tail
+    (1, 1, 64, 2, 4, 4, 0),       # the tiny configuration
+    (2, 2, 64, 3, 2, 4, 3),
+    (1, 2, 128, 5, 4, 16, 37),    # tc = 64, several tiles and a ragged tail
+    (1, 1, 128, 3, 8, 32, 200),   # tc = 256 with a tail
+    (1, 2, 64, 4, 1, 5, 2),       # c = 1, odd t
+    (1, 1, 128, 2, 3, 7, 0),      # nothing is a power of two
+    (1, 2, 128, 0, 4, 0, 301),    # t = 0: plain causal attention
+    (1, 1, 128, 9, 2, 8, 16),
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, PRIOR, NOREP, NOREP | PRIOR, GENERIC, GENERIC | PRIOR])
+@pytest.mark.parametrize("B,H,D,n,c,t,tail", BWD_CASES)
+def test_masked_bwd_matches_oracle(B, H, D, n, c, t, tail, flags, dtype):
+    lay = flags & (PRIOR | NOREP)
+    S = oracle.seq_len(n, c, t, tail, lay)
+    q, k, v = synthetic.qkv(B, H, S, D, seed=11, std=1.0, dtype=dtype)
+    d_o = synthetic.normal_tensor((B, H, S, D), 97, 1.0, dtype)
+    want = oracle.masked_attn_bwd(npf(q), npf(k), npf(v), npf(d_o), n, c, t, tail, lay)
+    got = run_fwd_bwd(q.to(DEV), k.to(DEV), v.to(DEV), d_o.to(DEV), n, c, t, tail, flags)
+    for g, w, name in zip(got, want, ("dq", "dk", "dv")):
+        check_grad(g, w, dtype, name)
+
+
+def test_masked_bwd_strided_views_explicit_scale_and_unsupervised_memory_rows():
+    """Views into one packed buffer; dO is zero on the memory rows (the paper puts no loss on <m>
+    outputs), so their queries get exactly zero gradient."""
+    B, H, D, n, c, t = 2, 3, 128, 3, 4, 16
+    S = oracle.seq_len(n, c, t)
+    buf = synthetic.normal_tensor((B, S, 9, H, D), 9, 1.0, torch.bfloat16).to(DEV)
+    q, k, v, o, d_o, dq, dk, dv = (buf[:, :, i].permute(0, 2, 1, 3) for i in range(8))
+    zone = torch.from_numpy(oracle.layout_index(n, c, t)[1]).to(DEV)
+    d_o[:, :, zone == 1] = 0
+    lse = torch.empty((B, H, S), dtype=torch.float32, device=DEV)
+    L.loma_masked_attn_fwd(q, k, v, o, lse, n, c, t, 0, 0, 0.05)
+    ws = torch.empty(L.loma_masked_attn_bwd_workspace_bytes(B, H, D, n, c, t), dtype=torch.uint8, device=DEV)
+    L.loma_masked_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, n, c, t, 0, 0, ws, 0.05)
+    torch.cuda.synchronize()
+    want = oracle.masked_attn_bwd(npf(q), npf(k), npf(v), npf(d_o), n, c, t, scale=0.05)
+    for g, w, name in zip((dq, dk, dv), want, ("dq", "dk", "dv")):
+        check_grad(g, w, torch.bfloat16, name)
+    assert float(dq[:, :, zone == 1].abs().max()) == 0.0
+
+
+def test_masked_bwd_is_bitwise_repeatable():
+    B, H, D, n, c, t, tail = 2, 2, 128, 5, 4, 16, 9
+    S = oracle.seq_len(n, c, t, tail)
+    q, k, v = (x.to(DEV) for x in synthetic.qkv(B, H, S, D, seed=5, dtype=torch.bfloat16))
+    d_o = synthetic.normal_tensor((B, H, S, D), 6, 1.0, torch.bfloat16).to(DEV)
+    a = run_fwd_bwd(q, k, v, d_o, n, c, t, tail)
+    b = run_fwd_bwd(q, k, v, d_o, n, c, t, tail)
+    for x, y in zip(a, b):
+        assert torch.equal(x.view(torch.int16), y.view(torch.int16))
