@@ -506,28 +506,30 @@ template <typename T, int D>
 static cudaError_t masked_bwd_generic_t(const void* q, const void* k, const void* v, const void* o, const void* d_o,
                                         const float* lse, void* dq, void* dk, void* dv, float* delta, int B, int H,
                                         const Layout& L, int64_t sb, int64_t sh, int64_t ss, float scale,
-                                        cudaStream_t st) {
+                                        int parts, cudaStream_t st) {
     dim3 grid((L.S + GENERIC_WARPS - 1) / GENERIC_WARPS, B * H);
-    masked_attn_bwd_dq_generic_kernel<T, D><<<grid, GENERIC_WARPS * 32, 0, st>>>(
-        static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), static_cast<const T*>(o),
-        static_cast<const T*>(d_o), lse, static_cast<T*>(dq), delta, H, L, sb, sh, ss, scale);
-    masked_attn_bwd_dkv_generic_kernel<T, D><<<grid, GENERIC_WARPS * 32, 0, st>>>(
-        static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), static_cast<const T*>(d_o), lse,
-        delta, static_cast<T*>(dk), static_cast<T*>(dv), H, L, sb, sh, ss, scale);
-    count_launches(2);
+    if (parts & 1)
+        masked_attn_bwd_dq_generic_kernel<T, D><<<grid, GENERIC_WARPS * 32, 0, st>>>(
+            static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), static_cast<const T*>(o),
+            static_cast<const T*>(d_o), lse, static_cast<T*>(dq), delta, H, L, sb, sh, ss, scale);
+    if (parts & 2)
+        masked_attn_bwd_dkv_generic_kernel<T, D><<<grid, GENERIC_WARPS * 32, 0, st>>>(
+            static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), static_cast<const T*>(d_o), lse,
+            delta, static_cast<T*>(dk), static_cast<T*>(dv), H, L, sb, sh, ss, scale);
+    count_launches((parts & 1) + ((parts >> 1) & 1));
     return cudaGetLastError();
 }
 
 cudaError_t launch_masked_attn_bwd_generic(const void* q, const void* k, const void* v, const void* o, const void* d_o,
                                            const float* lse, void* dq, void* dk, void* dv, float* delta, int B, int H,
                                            int D, const Layout& L, int64_t sb, int64_t sh, int64_t ss, loma_dtype dt,
-                                           float scale, cudaStream_t st) {
+                                           float scale, int parts, cudaStream_t st) {
     if (dt == LOMA_F32) {
-        return D == 64 ? masked_bwd_generic_t<float, 64>(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, L, sb, sh, ss, scale, st)
-                       : masked_bwd_generic_t<float, 128>(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, L, sb, sh, ss, scale, st);
+        return D == 64 ? masked_bwd_generic_t<float, 64>(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, L, sb, sh, ss, scale, parts, st)
+                       : masked_bwd_generic_t<float, 128>(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, L, sb, sh, ss, scale, parts, st);
     }
-    return D == 64 ? masked_bwd_generic_t<__nv_bfloat16, 64>(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, L, sb, sh, ss, scale, st)
-                   : masked_bwd_generic_t<__nv_bfloat16, 128>(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, L, sb, sh, ss, scale, st);
+    return D == 64 ? masked_bwd_generic_t<__nv_bfloat16, 64>(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, L, sb, sh, ss, scale, parts, st)
+                   : masked_bwd_generic_t<__nv_bfloat16, 128>(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, L, sb, sh, ss, scale, parts, st);
 }
 
 template <typename T, int D>

@@ -42,224 +42,13 @@
 // to the 2*gridDim.x streams round robin from a statically ordered list (longest first, (batch,
 // head) fastest).  Every mbarrier wait is bounded: on expiry the CTA records LOMA_ERR_TIMEOUT, all
 // roles leave their loops, TMEM is freed and the kernel returns.
-#include <cuda.h>
-#include <math.h>
-
-#include <mutex>
-
-#include "loma_internal.cuh"
-#include "tile_plan.cuh"
+#include "tcgen05_common.cuh"
 
 namespace loma {
 
 struct TmaMaps {
     CUtensorMap q[4], k[4], v[4], o[4];
 };
-
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // ~2 s: far beyond any legitimate wait
-
-// Bounded wait.  Returns false if the CTA is aborting (this or another thread's wait expired).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
-                *abort_flag = 1;
-                atomicExch(status, (int)LOMA_ERR_TIMEOUT);
-                return false;
-            }
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2,
-                                            int c3, int c4) {
-    asm volatile(
-        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, "
-        "%7}], [%2];" ::"r"(dst),
-        "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-        : "memory");
-}
-__device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3,
-                                             int c4) {
-    asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];" ::"l"(
-                     reinterpret_cast<uint64_t>(map)),
-                 "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-                 : "memory");
-}
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.u32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
-        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
-        : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
-    asm volatile(
-        "{\n.reg .pred p;\nsetp.ne.u32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
-        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// 32 consecutive 32-bit columns of this thread's TMEM lane -> r[0..31]
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
-        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
-        "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
-        "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-        : "memory");
-}
-// 16 consecutive 32-bit columns of this thread's TMEM lane
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
-        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-        : "memory");
-}
-
-__device__ __forceinline__ float fast_ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-// Packed pairs of fp32 (sm_100 has two-wide fp32 FMA and ADD) and the three-input maximum: the
-// softmax warps are bound by instruction issue, so fewer instructions per score matter.
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-    uint64_t r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-    float r;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
-    return r;
-}
-
-// One lane of a converged warp.  The MMA and TMA roles keep their control flow warp-uniform and
-// predicate only the issuing instruction, so descriptors and addresses can live in uniform registers.
-__device__ __forceinline__ bool elect_one() {
-    uint32_t pred;
-    asm volatile("{\n.reg .pred P;\nelect.sync _|P, 0xffffffff;\nselp.u32 %0, 1, 0, P;\n}" : "=r"(pred)::"memory");
-    return pred != 0;
-}
-
-// Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-    return (uint64_t)((addr >> 4) & 0x3FFFu) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |
-           ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
-}
-
-// ---- softmax helpers on one 64-column half of a score row (registers only) ----
-__device__ __forceinline__ void half_load(uint32_t addr, uint32_t (&a)[64], bool full, int col0, int lo, uint32_t span) {
-    tmem_ld32(addr, a);
-    tmem_ld32(addr + 32, a + 32);
-    tmem_wait_ld();
-    if (!full) {
-#pragma unroll
-        for (int e = 0; e < 64; ++e)
-            if ((uint32_t)(col0 + e - lo) >= span) a[e] = 0xff800000u;   // -inf: the key is blocked for this row
-    }
-}
-__device__ __forceinline__ float half_max(const uint32_t (&a)[64]) {
-    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-    for (int e = 0; e < 64; e += 4) {
-        mx0 = fmaxf(mx0, __uint_as_float(a[e]));
-        mx1 = fmaxf(mx1, __uint_as_float(a[e + 1]));
-        mx2 = fmaxf(mx2, __uint_as_float(a[e + 2]));
-        mx3 = fmaxf(mx3, __uint_as_float(a[e + 3]));
-    }
-    return fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-}
-// p = 2^(s*scale - ref) for 64 scores, packed to bf16 pairs and written to 32 TMEM columns at p_addr
-__device__ __forceinline__ void half_exp(const uint32_t (&a)[64], uint32_t p_addr, float scale_log2, float neg_ref,
-                                         float& ls0, float& ls1) {
-#pragma unroll
-    for (int c = 0; c < 2; ++c) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-            const float p0 = fast_ex2(fmaf(__uint_as_float(a[c * 32 + e]), scale_log2, neg_ref));
-            const float p1 = fast_ex2(fmaf(__uint_as_float(a[c * 32 + e + 1]), scale_log2, neg_ref));
-            ls0 += p0;
-            ls1 += p1;
-            pk[e >> 1] = pack_bf16(p0, p1);
-        }
-        tmem_st16(p_addr + c * 16, pk);
-    }
-}
 
 // ------------------------------------------------------------------ the kernel
 constexpr int TC_THREADS = 384;   // 2 softmax warpgroups + 1 warpgroup with 2 TMA warps and 2 MMA warps
@@ -279,20 +68,6 @@ struct TcSmem {
     static constexpr int STREAM_BYTES = 3 * TILE_BYTES + PANEL_BYTES;
     static constexpr int TOTAL = 2 * STREAM_BYTES;
 };
-
-// The visited halves of a tile's first 64 steps, one step per lane and two ballots per 32 steps.
-// Called by whole warps only.
-__device__ __forceinline__ HalfMasks tile_half_masks(const FwdParams& p, const TileDesc& td, int lane) {
-    HalfMasks hm;
-    hm.m[0] = hm.m[1] = 0;
-    for (int base = 0; base < td.nsteps && base < 64; base += 32) {
-        const int j = base + lane;
-        const unsigned v = j < td.nsteps ? visited_halves(p, td, j) : 0u;
-        hm.m[0] |= (unsigned long long)__ballot_sync(0xffffffffu, v & 1u) << base;
-        hm.m[1] |= (unsigned long long)__ballot_sync(0xffffffffu, v & 2u) << base;
-    }
-    return hm;
-}
 
 template <int D>
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -709,42 +484,6 @@ cudaError_t launch_bounded_wait_selftest(cudaStream_t st) {
 }
 
 // ------------------------------------------------------------------ host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        void* f = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(f);
-    });
-    return fn;
-}
-
-// 5-D map (d, row in zone, chunk, head, batch) over one zone view of one tensor.
-static bool encode_view(CUtensorMap* map, const void* base, const View& v, int D, int B, int H, int64_t row0,
-                        int64_t sb, int64_t sh, int64_t ss, int64_t chunk_stride_rows) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const uint64_t es = 2;
-    cuuint64_t dims[5] = {(cuuint64_t)D, (cuuint64_t)v.Z, (cuuint64_t)v.nch, (cuuint64_t)H, (cuuint64_t)B};
-    cuuint64_t chunk_stride = (v.nch > 1 ? (uint64_t)chunk_stride_rows : (uint64_t)v.Z) * ss * es;
-    cuuint64_t hstride = (uint64_t)(sh > 0 ? sh : ss * v.Z) * es;
-    cuuint64_t bstride = (uint64_t)(sb > 0 ? sb : ss * v.Z) * es;
-    cuuint64_t strides[4] = {(cuuint64_t)ss * es, chunk_stride, hstride, bstride};
-    cuuint32_t box[5] = {64, (cuuint32_t)v.R, (cuuint32_t)v.CH, 1, 1};
-    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
-    void* addr = const_cast<uint8_t*>(static_cast<const uint8_t*>(base)) + row0 * ss * es;
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, addr, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 struct MapCacheKey {
     const void *q, *k, *v, *o;
     int B, H, D, n, c, t, tail;

@@ -192,8 +192,16 @@ int loma_masked_attn_bwd(const void* q, const void* k, const void* v, const void
     if (dc != LOMA_OK) return dc;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = launch_masked_attn_bwd_generic(q, k, v, o, d_o, lse, dq, dk, dv, static_cast<float*>(workspace), B, H,
-                                                   D, L, stride_b, stride_h, stride_s, dtype, scale, st);
+    float* delta = static_cast<float*>(workspace);
+    int generic_parts = 3;
+    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC)) {
+        const cudaError_t e = launch_masked_attn_bwd_dq_tc(q, k, v, o, d_o, lse, dq, delta, B, H, D, L, stride_b, stride_h,
+                                                           stride_s, scale, st);
+        if (e == cudaSuccess) generic_parts = 2;
+        else if (e != cudaErrorNotSupported) return LOMA_ERR_CUDA;
+    }
+    const cudaError_t e = launch_masked_attn_bwd_generic(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, D, L, stride_b,
+                                                         stride_h, stride_s, dtype, scale, generic_parts, st);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 

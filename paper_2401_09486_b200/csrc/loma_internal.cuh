@@ -35,11 +35,16 @@ cudaError_t launch_masked_attn_generic(const void* q, const void* k, const void*
                                        int64_t sb, int64_t sh, int64_t ss,
                                        loma_dtype dt, float scale, cudaStream_t st);
 
-// gradients of the masked forward on CUDA cores; delta: B*H*S floats of scratch (row sums dO.O)
+// gradients of the masked forward on CUDA cores; delta: B*H*S floats of scratch (row sums dO.O).
+// parts: bit 0 = delta and dQ, bit 1 = dK and dV (needs delta)
 cudaError_t launch_masked_attn_bwd_generic(const void* q, const void* k, const void* v, const void* o, const void* d_o,
                                            const float* lse, void* dq, void* dk, void* dv, float* delta, int B, int H,
                                            int D, const Layout& L, int64_t sb, int64_t sh, int64_t ss, loma_dtype dt,
-                                           float scale, cudaStream_t st);
+                                           float scale, int parts, cudaStream_t st);
+// bf16 on tcgen05 (attn_bwd_tcgen05.cu): delta for every row, and dQ; cudaErrorNotSupported = use the generic kernels
+cudaError_t launch_masked_attn_bwd_dq_tc(const void* q, const void* k, const void* v, const void* o, const void* d_o,
+                                         const float* lse, void* dq, float* delta, int B, int H, int D, const Layout& L,
+                                         int64_t sb, int64_t sh, int64_t ss, float scale, cudaStream_t st);
 
 // tcgen05 / TMEM / TMA masked forward (attn_tcgen05.cu); cudaErrorNotSupported = use the generic kernel
 cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int D,
