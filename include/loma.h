@@ -232,6 +232,17 @@ LOMA_API int loma_masked_attn_plan_coverage(int n_chunks, int c, int t, int tail
                                             uint8_t* counts);
 
 /* ---------------------------------------------------------------------------
+ * loma_masked_attn_bwd_plan_coverage -- the same host-only replay for the pass of
+ * loma_masked_attn_bwd that produces dK and dV.  That pass owns one 128-row key tile at a
+ * time and walks the query tiles that may attend to it (the columns of Eq. 2 read
+ * downwards); inside a visited query tile each key lets one interval of rows through.
+ * counts has the layout of loma_masked_attn_plan_coverage and must again equal M of Eq. 2.
+ * No CUDA call is made.  Errors: INVALID_ARG.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_masked_attn_bwd_plan_coverage(int n_chunks, int c, int t, int tail_read, unsigned flags,
+                                                uint8_t* counts);
+
+/* ---------------------------------------------------------------------------
  * loma_decode_attn -- one new token per (batch, head) attends to the cache_len
  * entries already in the cache (all memory entries, then the uncompressed tail)
  * and to itself: the mask row tril(ones(1, 1+k), diagonal=k) of Appendix A with

@@ -38,6 +38,7 @@ SIGNATURES = {
                                   _f, _u, _p, _sz, _p]),
     "loma_masked_attn_bwd_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i, _u]),
     "loma_masked_attn_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
+    "loma_masked_attn_bwd_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "loma_decode_attn_static": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _p]),
@@ -197,6 +198,15 @@ def loma_masked_attn_plan_coverage(n_chunks: int, c: int, t: int, tail_read: int
     counts = torch.empty((S, S), dtype=torch.uint8)
     rc = lib().loma_masked_attn_plan_coverage(n_chunks, c, t, tail_read, int(flags), _ptr(counts))
     _check(rc, "loma_masked_attn_plan_coverage")
+    return counts
+
+
+def loma_masked_attn_bwd_plan_coverage(n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0) -> torch.Tensor:
+    """Host replay of the key-tile side of the plan (the backward's dK/dV pass): uint8 [S, S] visit counts."""
+    S = n_chunks * ((c * t + t) if (flags & LOMA_FLAG_NO_REP_ZONE) else (2 * c * t + t)) + tail_read
+    counts = torch.empty((S, S), dtype=torch.uint8)
+    rc = lib().loma_masked_attn_bwd_plan_coverage(n_chunks, c, t, tail_read, int(flags), _ptr(counts))
+    _check(rc, "loma_masked_attn_bwd_plan_coverage")
     return counts
 
 

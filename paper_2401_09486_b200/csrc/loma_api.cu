@@ -242,6 +242,16 @@ int loma_masked_attn_plan_coverage(int n_chunks, int c, int t, int tail_read, un
     return LOMA_OK;
 }
 
+int loma_masked_attn_bwd_plan_coverage(int n_chunks, int c, int t, int tail_read, unsigned flags, uint8_t* counts) {
+    Layout L;
+    const int rc = make_layout(n_chunks, c, t, tail_read, flags, &L);
+    if (rc != LOMA_OK) return rc;
+    if (L.S > 0 && !counts) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)L.S * L.S > (1ll << 32)) return LOMA_ERR_INVALID_ARG;
+    if (L.S > 0) plan_coverage_by_key_host(L, counts);
+    return LOMA_OK;
+}
+
 size_t loma_decode_workspace_bytes(int B, int H, int D, int cache_len) {
     if (B <= 0 || H <= 0 || D <= 0 || cache_len < 0) return 0;
     return decode_workspace_bytes(B * H, D, cache_len + 1);

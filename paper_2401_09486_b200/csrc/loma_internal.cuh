@@ -50,7 +50,8 @@ cudaError_t launch_masked_attn_bwd_dq_tc(const void* q, const void* k, const voi
 cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int D,
                                   const Layout& L, int64_t sb, int64_t sh, int64_t ss, float scale, cudaStream_t st);
 
-void plan_coverage_host(const Layout& L, uint8_t* counts);   // tile_plan_host.cu
+void plan_coverage_host(const Layout& L, uint8_t* counts);          // tile_plan_host.cu
+void plan_coverage_by_key_host(const Layout& L, uint8_t* counts);   // the plan read by key tile (backward)
 
 cudaError_t launch_bounded_wait_selftest(cudaStream_t st);   // attn_tcgen05.cu
 

@@ -199,6 +199,125 @@ struct HalfWalk {
     __host__ __device__ __forceinline__ bool last_of_step(const HalfMasks& hm) const { return h == 1 || !hm.has(1, j); }
 };
 
+// ------------------------------------------------------------------ the plan read by key tile
+// The backward's dK/dV pass owns one key tile at a time and walks the query tiles that visit it:
+// the lists of decode_tile turned round.  A key tile of a view has the geometry of the query tile
+// with the same index; the query tiles that visit it form at most four runs of consecutive tiles,
+// one per view.  The host replays this side too and compares it with Eq. 2.
+struct KeyTileDesc {
+    int view, ki, c0, r0, a0, a1;
+    Seg seg[4];
+    int nseg, nsteps;
+};
+struct QTile {
+    int view, mode, c0, r0, a0, a1;
+};
+
+__host__ __device__ __forceinline__ int last_tile_of_chunk(const View& v, int c) {
+    return v.Z >= 128 ? (c + 1) * v.tpc - 1 : fdiv(c, v.dCH);
+}
+
+__host__ __device__ __forceinline__ void tile_geometry(const View& g, int ti, int& c0, int& r0, int& a0, int& a1) {
+    int c1;
+    if (g.Z >= 128) { c0 = fdiv(ti, g.dtpc); r0 = (ti - c0 * g.tpc) * 128; c1 = c0; }
+    else { c0 = ti * g.CH; r0 = 0; c1 = plan_min(c0 + g.CH, g.nch) - 1; }
+    a0 = g.chunk_base + c0;
+    a1 = g.chunk_base + c1;
+}
+
+// Key tiles in scheduling order: memory tiles first (tile 0 is visited by the most query tiles),
+// then the tail, reading and repetition tiles.
+__host__ __device__ __forceinline__ void decode_key_tile(const FwdParams& p, int rank, KeyTileDesc& kd) {
+    int view, ki;
+    if (rank < p.n_mem) { view = V_MEM; ki = rank; }
+    else if ((rank -= p.n_mem) < p.n_tail) { view = V_TAIL; ki = rank; }
+    else if ((rank -= p.n_tail) < p.n_read) { view = V_READ; ki = rank; }
+    else { view = V_REP; ki = rank - p.n_read; }
+    const View& g = p.view[view];
+    kd.view = view; kd.ki = ki;
+    tile_geometry(g, ki, kd.c0, kd.r0, kd.a0, kd.a1);
+    const View& vm = p.view[V_MEM];
+    const View& vr = p.view[V_READ];
+    const View& vp = p.view[V_REP];
+    int ns = 0;
+    auto add = [&](int v, int mode, int first, int count) {
+        if (count > 0) kd.seg[ns++] = Seg{v, mode, first, count};
+    };
+    if (view == V_MEM) {
+        // reading rows of every later chunk and of the tail (Eq. 3)
+        if (kd.a0 + 1 < p.n_chunks) { const int f = tile_of_chunk(vr, kd.a0 + 1); add(V_READ, M_LT, f, p.n_read - f); }
+        add(V_TAIL, M_LT, 0, p.n_tail);
+        // memory rows: own chunk (Eq. 1, row 2); with the prior-memory flag every later chunk too
+        const int f = (g.Z >= 128) ? kd.c0 * g.tpc : ki;
+        if (p.flags & LOMA_FLAG_MEM_SEES_PRIOR_MEM) add(V_MEM, M_LE, f, p.n_mem - f);
+        else add(V_MEM, M_EQ, f, (g.Z >= 128) ? g.tpc : 1);
+        // repetition rows of the same chunks (Eq. 1, row 3)
+        if (p.n_rep > 0) { const int fr = tile_of_chunk(vp, kd.a0); add(V_REP, M_EQ, fr, last_tile_of_chunk(vp, kd.a1) - fr + 1); }
+    } else if (view == V_READ) {
+        add(V_READ, M_CAUSAL, ki, (g.Z >= 128) ? (kd.c0 + 1) * g.tpc - ki : 1);
+        const int fm = tile_of_chunk(vm, kd.a0);
+        add(V_MEM, M_EQ, fm, last_tile_of_chunk(vm, kd.a1) - fm + 1);
+    } else if (view == V_TAIL) {
+        add(V_TAIL, M_CAUSAL, ki, p.n_tail - ki);
+    } else {
+        add(V_REP, M_DIAG, ki, 1);
+    }
+    kd.nseg = ns;
+    kd.nsteps = 0;
+    for (int i = 0; i < ns; ++i) kd.nsteps += kd.seg[i].count;
+}
+
+__host__ __device__ __forceinline__ void step_qtile(const FwdParams& p, const KeyTileDesc& kd, int j, QTile& qt) {
+    int i = 0;
+    while (i + 1 < kd.nseg && j >= kd.seg[i].count) { j -= kd.seg[i].count; ++i; }
+    qt.view = kd.seg[i].view; qt.mode = kd.seg[i].mode;
+    tile_geometry(p.view[qt.view], kd.seg[i].first + j, qt.c0, qt.r0, qt.a0, qt.a1);
+}
+
+// Rows of a query tile that hold a row of the sequence: always a prefix [0, n).
+__host__ __device__ __forceinline__ int valid_tile_rows(const View& g, int r0, int a0, int a1) {
+    return g.Z >= 128 ? plan_min(128, g.Z - r0) : (a1 - a0 + 1) * g.R;
+}
+
+// Query rows [lo, hi) of query tile qt that may attend to the key at (chunk kc, offset ko), tile-local key row kr:
+// row_interval read by column.
+__host__ __device__ __forceinline__ void col_interval(const View& qv, const QTile& qt, int kc, int ko, int kr, bool key_valid,
+                                                      int& lo, int& hi) {
+    const int nvalid = valid_tile_rows(qv, qt.r0, qt.a0, qt.a1);
+    const int vrows = plan_min(qv.R, qv.Z - qt.r0);   // valid rows per chunk of this tile
+    const int d = kc - qt.a0;                         // the key's chunk relative to the tile's first chunk
+    lo = 0; hi = 0;
+    if (qt.mode == M_LT || qt.mode == M_LE) {
+        const int first = plan_max(d + (qt.mode == M_LT ? 1 : 0), 0);   // first chunk of the tile that sees the key
+        lo = first * qv.R; hi = nvalid;
+    } else if (qt.mode == M_DIAG) {
+        lo = kr; hi = kr + 1;
+    } else if (d >= 0 && d < qv.CH) {
+        lo = d * qv.R + (qt.mode == M_CAUSAL ? plan_min(plan_max(ko - qt.r0, 0), vrows) : 0);
+        hi = d * qv.R + vrows;
+    }
+    if (hi > nvalid) hi = nvalid;
+    if (!key_valid || hi < lo) { lo = 0; hi = 0; }
+}
+
+// Halves (64 query rows each) of step j that some key row of the tile may be seen from.
+__host__ __device__ __forceinline__ unsigned visited_qhalves(const FwdParams& p, const KeyTileDesc& kd, int j) {
+    if (j >= 64) return 3u;
+    QTile qt;
+    step_qtile(p, kd, j, qt);
+    const View& qv = p.view[qt.view];
+    const int nvalid = valid_tile_rows(qv, qt.r0, qt.a0, qt.a1);
+    int ulo = 0, uhi = nvalid;
+    if (qt.mode == M_LT || qt.mode == M_LE) {
+        ulo = plan_max(kd.a0 - qt.a0 + (qt.mode == M_LT ? 1 : 0), 0) * qv.R;
+    } else if (qt.mode != M_DIAG) {
+        const int d0 = plan_max(kd.a0 - qt.a0, 0), d1 = plan_min(kd.a1 - qt.a0, qv.CH - 1);
+        if (d1 >= d0) { ulo = d0 * qv.R; uhi = plan_min(nvalid, (d1 + 1) * qv.R); } else { uhi = 0; }
+    }
+    const unsigned m = ((ulo < 64 && uhi > 0) ? 1u : 0u) | (uhi > 64 ? 2u : 0u);
+    return m ? m : 1u;
+}
+
 // Fills the geometry part of FwdParams (views, tile counts) from the layout.
 inline View make_view(int Z, int nch, int chunk_base, int zone_row0) {
     View v{};

@@ -52,4 +52,48 @@ void plan_coverage_host(const Layout& L, uint8_t* counts) {
     }
 }
 
+// The same count, taken from the key-tile side of the plan (the backward's dK/dV pass).
+void plan_coverage_by_key_host(const Layout& L, uint8_t* counts) {
+    FwdParams p{};
+    make_plan(L, 1, 1, &p);
+    memset(counts, 0, (size_t)L.S * L.S);
+    for (int rank = 0; rank < p.total_tiles; ++rank) {
+        KeyTileDesc kd;
+        decode_key_tile(p, rank, kd);
+        const View& kv = p.view[kd.view];
+        HalfMasks hm{{0, 0}};
+        for (int j = 0; j < kd.nsteps && j < 64; ++j) {
+            const unsigned v = visited_qhalves(p, kd, j);
+            hm.m[0] |= (unsigned long long)(v & 1u) << j;
+            hm.m[1] |= (unsigned long long)((v >> 1) & 1u) << j;
+        }
+        HalfWalk hw;
+        for (hw.start(hm); !hw.done(kd.nsteps); hw.next(hm)) {
+            QTile qt;
+            step_qtile(p, kd, hw.j, qt);
+            const View& qv = p.view[qt.view];
+            for (int kr = 0; kr < 128; ++kr) {
+                const int ksub = kr / kv.R;
+                const int ko = kd.r0 + (kr - ksub * kv.R);
+                const int kc = kd.a0 + ksub;
+                const bool key_valid = (kr < kv.R * kv.CH) && (kc <= kd.a1) && (ko < kv.Z);
+                int lo, hi;
+                col_interval(qv, qt, kc, ko, kr, key_valid, lo, hi);
+                if (!key_valid || hi <= lo) continue;
+                const int64_t gcol = (int64_t)kc * L.s + kv.zone_row0 + ko;
+                for (int row = (lo > 64 * hw.h ? lo : 64 * hw.h); row < hi && row < 64 * hw.h + 64; ++row) {
+                    const int rsub = row / qv.R;
+                    const int ro = qt.r0 + (row - rsub * qv.R);
+                    const int rc = qt.a0 + rsub;
+                    const int64_t grow = (int64_t)rc * L.s + qv.zone_row0 + ro;
+                    if (gcol < L.S && grow >= 0 && grow < L.S) {
+                        uint8_t& c = counts[grow * L.S + gcol];
+                        if (c < 255) ++c;
+                    }
+                }
+            }
+        }
+    }
+}
+
 }  // namespace loma

@@ -193,3 +193,14 @@ def test_masked_attn_bwd_validation(lib):
     need = lib.loma_masked_attn_bwd_workspace_bytes(4, 32, 128, 32, 4, 16, 0, 0)
     assert need >= 4 * 32 * 4608 * 4 and need % 256 == 0
     assert lib.loma_masked_attn_bwd_workspace_bytes(1, 1, 64, 1, 0, 2, 0, 0) == 0     # c < 1: no layout
+
+
+@pytest.mark.parametrize("n,c,t,tail", PLAN_GEOMS)
+@pytest.mark.parametrize("flags", [0, 1, 2, 3])
+def test_key_tile_side_of_the_plan_reproduces_the_mask_exactly(lib, n, c, t, tail, flags):
+    """The backward's dK/dV pass walks, per key tile, the query tiles that see it: every allowed
+    (row, key) pair of Eq. 2 must again be visited exactly once and no blocked pair at all."""
+    got = binding.loma_masked_attn_bwd_plan_coverage(n, c, t, tail, flags).numpy()
+    want = oracle.dense_mask(n, c, t, tail, flags).astype(np.uint8)
+    assert got.shape == want.shape
+    assert np.array_equal(got, want), f"{int((got != want).sum())} entries differ"
