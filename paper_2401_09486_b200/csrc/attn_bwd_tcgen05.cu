@@ -13,6 +13,13 @@
 // TMEM and K_h as an MN-major shared operand.  Nothing is carried from event to event (lse and
 // delta are inputs), so there is no rescaling.  Epilogue: scale, round to bf16, TMA store.
 //
+// dK/dV kernel.  The same machinery turned round: a CTA owns a key tile (K and V stay in shared
+// memory, dK and dV accumulate in TMEM) and walks the query tiles that visit it (the plan read by
+// key tile); Q and dO stream through the ring.  Per visited half of 64 query rows: S^T = K Q_h^T and
+// dP^T = V dO_h^T; the warpgroup (thread = key row) writes P^T over S^T and dA^T over dP^T in bf16
+// (lse and delta of the 128 query rows of the step are staged in shared memory); then
+// dV += P^T dO_h and dK += dA^T Q_h with Q_h, dO_h as MN-major operands.
+//
 // Roles: warps 0-3 warpgroup, warp 4 TMA producer (one lane), warp 5 MMA issuer (warp-uniform
 // control flow, one elected lane issues).  Every mbarrier wait is bounded; on expiry the CTA
 // records LOMA_ERR_TIMEOUT, every role leaves its loop, TMEM is freed and the kernel returns.
@@ -359,6 +366,334 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
     }
 }
 
+// ------------------------------------------------------------------ dK, dV
+struct BwdKvMaps {
+    CUtensorMap q[4], k[4], v[4], g[4], dk[4], dv[4];
+};
+
+__device__ __forceinline__ HalfMasks key_tile_half_masks(const FwdParams& p, const KeyTileDesc& kd, int lane) {
+    HalfMasks hm;
+    hm.m[0] = hm.m[1] = 0;
+    for (int base = 0; base < kd.nsteps && base < 64; base += 32) {
+        const int j = base + lane;
+        const unsigned v = j < kd.nsteps ? visited_qhalves(p, kd, j) : 0u;
+        hm.m[0] |= (unsigned long long)__ballot_sync(0xffffffffu, v & 1u) << base;
+        hm.m[1] |= (unsigned long long)__ballot_sync(0xffffffffu, v & 2u) << base;
+    }
+    return hm;
+}
+
+template <int D>
+__global__ void __launch_bounds__(BWD_THREADS, 1)
+masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdParams bp) {
+    using SM = BwdDqSmem<D>;   // same footprint: two resident tiles, a two-stage ring of tile pairs, one staging panel
+    constexpr int PANELS = SM::PANELS;
+    constexpr int K_OFF = SM::Q_OFF, V_OFF = SM::G_OFF;
+    const FwdParams& p = bp.f;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bars[BWD_NBAR];
+    __shared__ __align__(16) float lse2_s[2][128];   // -lse * log2(e) and delta of the query rows of a step, by ring stage
+    __shared__ __align__(16) float dl_s[2][128];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+
+    const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+
+    enum { B_KVF = 0, B_DONE = 1, B_QGF = 2, B_QGE = 4, B_SF = 6, B_PF = 8 };
+    auto bar = [&](int i) { return smem_u32(&bars[i]); };
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int i = 0; i < BWD_NBAR; ++i) mbar_init(bar(i), (i == B_PF || i == B_PF + 1) ? 128 : 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = threadIdx.x; i < SM::TOTAL / 16; i += BWD_THREADS) reinterpret_cast<uint4*>(smem_gen)[i] = make_uint4(0, 0, 0, 0);
+    fence_async_smem();
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(512)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    // TMEM columns: S^T buffers at 0 and 64, dP^T buffers at 128 and 192, dK accumulator at 256, dV at 384
+    const uint32_t tmem = tmem_slot;
+    volatile int* abortp = &abort_flag;
+
+    const int total_work = p.total_tiles * p.BH;
+    const int nstreams = gridDim.x;
+    const int sid = blockIdx.x;
+    auto tile_of_round = [&](int r) { return r * nstreams + ((r & 1) ? nstreams - 1 - sid : sid); };
+    auto ring_off = [&](int stage) { return (uint32_t)(SM::KV_OFF + stage * 2 * SM::TILE_BYTES); };   // Q, then dO
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t gs = 0, tcount = 0;
+            bool ok = true;
+            for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
+                const int rank = fdiv(w, p.dBH), bh = w - rank * p.BH;
+                const int bi = fdiv(bh, p.dH), hi = bh - bi * p.H;
+                KeyTileDesc kd;
+                decode_key_tile(p, rank, kd);
+                const View& kv = p.view[kd.view];
+                if (tcount > 0) ok = mbar_wait(bar(B_DONE), (tcount - 1) & 1, abortp, p.status);
+                if (!ok) break;
+                mbar_expect_tx(bar(B_KVF), 2 * kv.R * kv.CH * 128 * PANELS);
+                for (int pn = 0; pn < PANELS; ++pn) {
+                    tma_load_5d(smem_base + K_OFF + pn * SM::PANEL_BYTES, &maps.k[kd.view], bar(B_KVF), pn * 64, kd.r0, kd.c0, hi, bi);
+                    tma_load_5d(smem_base + V_OFF + pn * SM::PANEL_BYTES, &maps.v[kd.view], bar(B_KVF), pn * 64, kd.r0, kd.c0, hi, bi);
+                }
+                for (int j = 0; j < kd.nsteps; ++j, ++gs) {
+                    QTile qt;
+                    step_qtile(p, kd, j, qt);
+                    const View& qv = p.view[qt.view];
+                    const int stage = gs & 1;
+                    ok = mbar_wait(bar(B_QGE + stage), ((gs >> 1) & 1) ^ 1, abortp, p.status);
+                    if (!ok) break;
+                    mbar_expect_tx(bar(B_QGF + stage), 2 * qv.R * qv.CH * 128 * PANELS);
+                    for (int pn = 0; pn < PANELS; ++pn) {
+                        tma_load_5d(smem_base + ring_off(stage) + pn * SM::PANEL_BYTES, &maps.q[qt.view], bar(B_QGF + stage), pn * 64,
+                                    qt.r0, qt.c0, hi, bi);
+                        tma_load_5d(smem_base + ring_off(stage) + SM::TILE_BYTES + pn * SM::PANEL_BYTES, &maps.g[qt.view],
+                                    bar(B_QGF + stage), pn * 64, qt.r0, qt.c0, hi, bi);
+                    }
+                }
+            }
+            if (!ok) {
+                const long long t0 = clock64();
+                while (clock64() - t0 < 2000000ll) {}
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issuer
+        constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+        constexpr uint32_t IDESC_ACC =
+            (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
+        uint32_t gs = 0, tcount = 0, ge_s = 0, ge_p = 0;
+        bool ok = true;
+        const uint64_t kd_ = smem_desc(smem_base + K_OFF, 16, 1024);
+        const uint64_t vd_ = smem_desc(smem_base + V_OFF, 16, 1024);
+        // S^T = K Q_h^T and dP^T = V dO_h^T for query rows [64h, 64h+64) of the staged tiles -> buffers b
+        auto issue_st = [&](int b, int h, int stage) {
+            if (elect_one()) {
+                const uint64_t qd = smem_desc(smem_base + ring_off(stage), 16, 1024);
+                const uint64_t gd = smem_desc(smem_base + ring_off(stage) + SM::TILE_BYTES, 16, 1024);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint64_t off = (uint64_t)(((kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32) >> 4);
+                    mma_ss(tmem + b * 64, kd_ + off, qd + off + (uint64_t)((h * 8192) >> 4), IDESC_S, kk > 0);
+                }
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint64_t off = (uint64_t)(((kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32) >> 4);
+                    mma_ss(tmem + 128 + b * 64, vd_ + off, gd + off + (uint64_t)((h * 8192) >> 4), IDESC_S, kk > 0);
+                }
+                tc_commit(bar(B_SF + b));
+            }
+            __syncwarp();
+        };
+        // dV += P^T dO_h and dK += dA^T Q_h: P^T and dA^T (bf16) read from TMEM, dO_h and Q_h as MN-major operands
+        auto issue_acc = [&](int b, int h, int stage, bool first, bool last_of_step, bool last_of_tile) {
+            if (elect_one()) {
+                const uint64_t qmn = smem_desc(smem_base + ring_off(stage), SM::PANEL_BYTES, 1024);
+                const uint64_t gmn = smem_desc(smem_base + ring_off(stage) + SM::TILE_BYTES, SM::PANEL_BYTES, 1024);
+#pragma unroll
+                for (int k4 = 0; k4 < 4; ++k4)
+                    mma_ts(tmem + 384, tmem + b * 64 + k4 * 8, gmn + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_ACC,
+                           !first || (k4 > 0));
+#pragma unroll
+                for (int k4 = 0; k4 < 4; ++k4)
+                    mma_ts(tmem + 256, tmem + 128 + b * 64 + k4 * 8, qmn + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_ACC,
+                           !first || (k4 > 0));
+                if (last_of_step) tc_commit(bar(B_QGE + stage));
+                if (last_of_tile) tc_commit(bar(B_DONE));
+            }
+            __syncwarp();
+        };
+        for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
+            const int rank = fdiv(w, p.dBH);
+            KeyTileDesc kd;
+            decode_key_tile(p, rank, kd);
+            const HalfMasks hm = key_tile_half_masks(p, kd, lane);
+            const int nsteps = kd.nsteps;
+            HalfWalk sw, pw;
+            sw.start(hm);
+            pw.start(hm);
+            ok = __all_sync(0xffffffffu, mbar_wait(bar(B_KVF), tcount & 1, abortp, p.status));
+            if (!ok) break;
+            auto next_scores = [&]() {
+                const uint32_t step = gs + sw.j;
+                if (sw.first_of_step(hm)) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_QGF + (step & 1)), (step >> 1) & 1, abortp, p.status));
+                    if (!ok) return;
+                }
+                tc_fence_after();
+                issue_st(ge_s & 1, sw.h, step & 1);
+                ++ge_s;
+                sw.next(hm);
+            };
+            next_scores();
+            if (ok && !sw.done(nsteps)) next_scores();
+            bool first = true;
+            while (ok && !pw.done(nsteps)) {
+                const int b = ge_p & 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_PF + b), (ge_p >> 1) & 1, abortp, p.status));
+                if (!ok) break;
+                tc_fence_after();
+                const bool los = pw.last_of_step(hm);
+                issue_acc(b, pw.h, (gs + pw.j) & 1, first, los, los && pw.j == nsteps - 1);
+                first = false;
+                ++ge_p;
+                if (!sw.done(nsteps)) next_scores();
+                pw.next(hm);
+            }
+            gs += kd.nsteps;
+        }
+    } else {
+        // ------------------------------------------------------------ warpgroup: P^T, dA^T, epilogue
+        const int kr = threadIdx.x;
+        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        uint32_t ge = 0, gs = 0, tcount = 0;
+        bool ok = true;
+        bool store_pending = false;
+        for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
+            const int rank = fdiv(w, p.dBH), bh = w - rank * p.BH;
+            const int bi = fdiv(bh, p.dH), hi = bh - bi * p.H;
+            KeyTileDesc kd;
+            decode_key_tile(p, rank, kd);
+            const View& kv = p.view[kd.view];
+            const int ksub = fdiv(kr, kv.dR);
+            const int ko = kd.r0 + (kr - ksub * kv.R);
+            const int kc = kd.a0 + ksub;
+            const bool key_valid = (kr < kv.R * kv.CH) && (kc <= kd.a1) && (ko < kv.Z);
+            const HalfMasks hm = key_tile_half_masks(p, kd, lane);
+            HalfWalk hw;
+            int lo = 0, hi2 = 0, stage = 0;
+            for (hw.start(hm); ok && !hw.done(kd.nsteps); hw.next(hm), ++ge) {
+                if (hw.first_of_step(hm)) {
+                    QTile qt;
+                    step_qtile(p, kd, hw.j, qt);
+                    const View& qv = p.view[qt.view];
+                    col_interval(qv, qt, kc, ko, kr, key_valid, lo, hi2);
+                    // this thread fetches lse and delta of query row `kr` of the step's tile for everybody
+                    stage = (gs + hw.j) & 1;
+                    const int rsub = fdiv(kr, qv.dR);
+                    const int ro = qt.r0 + (kr - rsub * qv.R);
+                    const int rc = qt.a0 + rsub;
+                    float nl = 0.f, dl = 0.f;
+                    if ((kr < qv.R * qv.CH) && (rc <= qt.a1) && (ro < qv.Z)) {
+                        const int64_t idx = (int64_t)bh * p.S + (int64_t)rc * p.s + qv.zone_row0 + ro;
+                        nl = -bp.lse_in[idx] * 1.4426950408889634f;
+                        dl = bp.delta[idx];
+                    }
+                    lse2_s[stage][kr] = nl;
+                    dl_s[stage][kr] = dl;
+                    asm volatile("bar.sync 2, 128;" ::: "memory");
+                }
+                const int b = ge & 1;
+                const int lo_h = lo - 64 * hw.h;
+                const uint32_t span = (uint32_t)(hi2 - lo);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF + b), (ge >> 1) & 1, abortp, p.status));
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t s_addr = lane_addr + b * 64, g_addr = lane_addr + 128 + b * 64;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t s[32], g[32], ppk[16], dpk[16];
+                    tmem_ld32(s_addr + c * 32, s);
+                    tmem_ld32(g_addr + c * 32, g);
+                    tmem_wait_ld();
+                    const float4* nl4 = reinterpret_cast<const float4*>(&lse2_s[stage][64 * hw.h + c * 32]);
+                    const float4* dl4 = reinterpret_cast<const float4*>(&dl_s[stage][64 * hw.h + c * 32]);
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4) {
+                        const float4 nl = nl4[e >> 2], dl = dl4[e >> 2];
+                        const float nlv[4] = {nl.x, nl.y, nl.z, nl.w}, dlv[4] = {dl.x, dl.y, dl.z, dl.w};
+                        float pr[4], da[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const bool allowed = (uint32_t)(c * 32 + e + u - lo_h) < span;
+                            pr[u] = allowed ? fast_ex2(fmaf(__uint_as_float(s[e + u]), p.scale_log2, nlv[u])) : 0.f;
+                            da[u] = pr[u] * (__uint_as_float(g[e + u]) - dlv[u]);
+                        }
+                        ppk[e >> 1] = pack_bf16(pr[0], pr[1]);
+                        ppk[(e >> 1) + 1] = pack_bf16(pr[2], pr[3]);
+                        dpk[e >> 1] = pack_bf16(da[0], da[1]);
+                        dpk[(e >> 1) + 1] = pack_bf16(da[2], da[3]);
+                    }
+                    tmem_st16(s_addr + c * 16, ppk);   // P^T over the scores: 32 query rows -> 16 columns
+                    tmem_st16(g_addr + c * 16, dpk);   // dA^T over dP^T
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(B_PF + b));
+            }
+            gs += kd.nsteps;
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_DONE), tcount & 1, abortp, p.status));
+            if (ok) tc_fence_after();
+
+            // epilogue: dK (scaled) then dV, rounded to bf16, 64 columns at a time through the staging panel
+            uint8_t* orow = smem_gen + SM::O_OFF + kr * 128;
+            bool give_up = false;
+#pragma unroll
+            for (int pass = 0; pass < 2 * PANELS; ++pass) {
+                const int which = pass / PANELS, pn = pass % PANELS;   // 0: dK, 1: dV
+                const float mul = which == 0 ? bp.scale : 1.f;
+                if (kr == 0 && store_pending) tma_store_wait_read();
+                if (pass == 0) {
+                    uint32_t any_bad;
+                    asm volatile(
+                        "{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, 1, 128, p;\nselp.u32 %0, 1, 0, q;\n}"
+                        : "=r"(any_bad)
+                        : "r"((uint32_t)(ok ? 0 : 1))
+                        : "memory");
+                    if (any_bad) { give_up = true; break; }
+                } else {
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                }
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t x[32];
+                    tmem_ld32(lane_addr + 256 + which * 128 + pn * 64 + c * 32, x);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        const int ci = c * 4 + q4;
+                        uint4 u;
+                        u.x = pack_bf16(__uint_as_float(x[q4 * 8 + 0]) * mul, __uint_as_float(x[q4 * 8 + 1]) * mul);
+                        u.y = pack_bf16(__uint_as_float(x[q4 * 8 + 2]) * mul, __uint_as_float(x[q4 * 8 + 3]) * mul);
+                        u.z = pack_bf16(__uint_as_float(x[q4 * 8 + 4]) * mul, __uint_as_float(x[q4 * 8 + 5]) * mul);
+                        u.w = pack_bf16(__uint_as_float(x[q4 * 8 + 6]) * mul, __uint_as_float(x[q4 * 8 + 7]) * mul);
+                        *reinterpret_cast<uint4*>(orow + ((ci ^ (kr & 7)) << 4)) = u;
+                    }
+                }
+                fence_async_smem();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (kr == 0) {
+                    tma_store_5d(which == 0 ? &maps.dk[kd.view] : &maps.dv[kd.view], smem_base + SM::O_OFF, pn * 64, kd.r0, kd.c0,
+                                 hi, bi);
+                    tma_store_commit();
+                    store_pending = true;
+                }
+            }
+            if (give_up) { ok = false; break; }
+            tc_fence_before();
+        }
+        if (kr == 0 && store_pending) tma_store_wait_all();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_slot), "r"(512) : "memory");
+    }
+}
+
 // ------------------------------------------------------------------ host side
 struct BwdMapCacheKey {
     const void *q, *k, *v, *g, *dq;
@@ -450,6 +785,86 @@ cudaError_t launch_masked_attn_bwd_dq_tc(const void* q, const void* k, const voi
     else
         masked_attn_bwd_dq_tc_kernel<64><<<grid, BWD_THREADS, BwdDqSmem<64>::TOTAL + 1024, st>>>(maps, bp);
     count_launches(2);
+    return cudaGetLastError();
+}
+
+struct BwdKvMapCacheKey {
+    const void *q, *k, *v, *g, *dk, *dv;
+    int B, H, D, n, c, t, tail;
+    unsigned flags;
+    int64_t sb, sh, ss;
+    bool operator==(const BwdKvMapCacheKey& r) const {
+        return q == r.q && k == r.k && v == r.v && g == r.g && dk == r.dk && dv == r.dv && B == r.B && H == r.H && D == r.D &&
+               n == r.n && c == r.c && t == r.t && tail == r.tail && flags == r.flags && sb == r.sb && sh == r.sh && ss == r.ss;
+    }
+};
+
+// dK and dV on the tensor cores; delta must already be in place (launch_masked_attn_bwd_dq_tc writes it).
+cudaError_t launch_masked_attn_bwd_dkv_tc(const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+                                          const float* delta, void* dk, void* dv, int B, int H, int D, const Layout& L,
+                                          int64_t sb, int64_t sh, int64_t ss, float scale, cudaStream_t st) {
+    if (!encode_fn()) return cudaErrorNotSupported;
+    if (L.t > 256 * 128 || L.tc > (1 << 24)) return cudaErrorNotSupported;
+    BwdParams bp{};
+    make_plan(L, B, H, &bp.f);
+    bp.f.scale_log2 = scale * 1.4426950408889634f;
+    bp.f.status = device_status_word();
+    if (!bp.f.status) return cudaErrorUnknown;
+    if ((int64_t)bp.f.total_tiles * bp.f.BH > 0x7fffffffll) return cudaErrorNotSupported;
+    bp.lse_in = lse;
+    bp.delta = delta;
+    bp.scale = scale;
+
+    static std::mutex mu;
+    static BwdKvMapCacheKey cached_key{};
+    static BwdKvMaps cached_maps;
+    static bool have_cache = false;
+    BwdKvMaps maps;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        BwdKvMapCacheKey key{q, k, v, d_o, dk, dv, B, H, D, L.n_chunks, L.c, L.t, L.tail_read, L.flags, sb, sh, ss};
+        if (!(have_cache && key == cached_key)) {
+            BwdKvMaps mnew{};
+            const void* bases[6] = {q, k, v, d_o, dk, dv};
+            CUtensorMap* arrs[6] = {mnew.q, mnew.k, mnew.v, mnew.g, mnew.dk, mnew.dv};
+            for (int ti = 0; ti < 6; ++ti) {
+                for (int vi = 0; vi < 4; ++vi) {
+                    const View& vw = bp.f.view[vi];
+                    if (vw.ntiles == 0) continue;
+                    const int64_t row0 = (vi == V_TAIL) ? (int64_t)L.n_chunks * L.s : vw.zone_row0;
+                    if (!encode_view(&arrs[ti][vi], bases[ti], vw, D, B, H, row0, sb, sh, ss, L.s)) return cudaErrorNotSupported;
+                }
+            }
+            cached_maps = mnew;
+            cached_key = key;
+            have_cache = true;
+        }
+        maps = cached_maps;
+    }
+
+    static int sm_count[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (sm_count[dev] == 0) {
+        int sms = 0;
+        cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(masked_attn_bwd_dkv_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 BwdDqSmem<128>::TOTAL + 1024);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(masked_attn_bwd_dkv_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 BwdDqSmem<64>::TOTAL + 1024);
+        if (e != cudaSuccess) return e;
+        sm_count[dev] = sms;
+    }
+    const int sms = sm_count[dev];
+    const int64_t work = (int64_t)bp.f.total_tiles * bp.f.BH;
+    const int grid = (int)(work < sms ? work : sms);
+    if (D == 128)
+        masked_attn_bwd_dkv_tc_kernel<128><<<grid, BWD_THREADS, BwdDqSmem<128>::TOTAL + 1024, st>>>(maps, bp);
+    else
+        masked_attn_bwd_dkv_tc_kernel<64><<<grid, BWD_THREADS, BwdDqSmem<64>::TOTAL + 1024, st>>>(maps, bp);
+    count_launches(1);
     return cudaGetLastError();
 }
 

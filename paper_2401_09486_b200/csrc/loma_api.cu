@@ -197,8 +197,15 @@ int loma_masked_attn_bwd(const void* q, const void* k, const void* v, const void
     if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC)) {
         const cudaError_t e = launch_masked_attn_bwd_dq_tc(q, k, v, o, d_o, lse, dq, delta, B, H, D, L, stride_b, stride_h,
                                                            stride_s, scale, st);
-        if (e == cudaSuccess) generic_parts = 2;
-        else if (e != cudaErrorNotSupported) return LOMA_ERR_CUDA;
+        if (e == cudaSuccess) {
+            generic_parts = 2;
+            const cudaError_t e2 = launch_masked_attn_bwd_dkv_tc(q, k, v, d_o, lse, delta, dk, dv, B, H, D, L, stride_b,
+                                                                 stride_h, stride_s, scale, st);
+            if (e2 == cudaSuccess) return LOMA_OK;
+            if (e2 != cudaErrorNotSupported) return LOMA_ERR_CUDA;
+        } else if (e != cudaErrorNotSupported) {
+            return LOMA_ERR_CUDA;
+        }
     }
     const cudaError_t e = launch_masked_attn_bwd_generic(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, D, L, stride_b,
                                                          stride_h, stride_s, dtype, scale, generic_parts, st);

@@ -45,6 +45,9 @@ cudaError_t launch_masked_attn_bwd_generic(const void* q, const void* k, const v
 cudaError_t launch_masked_attn_bwd_dq_tc(const void* q, const void* k, const void* v, const void* o, const void* d_o,
                                          const float* lse, void* dq, float* delta, int B, int H, int D, const Layout& L,
                                          int64_t sb, int64_t sh, int64_t ss, float scale, cudaStream_t st);
+cudaError_t launch_masked_attn_bwd_dkv_tc(const void* q, const void* k, const void* v, const void* d_o, const float* lse,
+                                          const float* delta, void* dk, void* dv, int B, int H, int D, const Layout& L,
+                                          int64_t sb, int64_t sh, int64_t ss, float scale, cudaStream_t st);
 
 // tcgen05 / TMEM / TMA masked forward (attn_tcgen05.cu); cudaErrorNotSupported = use the generic kernel
 cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int D,
