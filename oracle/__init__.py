@@ -29,6 +29,8 @@ from .loma_oracle import (  # noqa: F401
     masked_attn_fwd,
     masked_softmax_attention_bwd,
     masked_attn_bwd,
+    masked_attn_bwd_dq_rows,
+    masked_attn_bwd_dkv_cols,
     decode_attn,
     compress_step,
     replay_generation,

@@ -369,6 +369,49 @@ def masked_attn_bwd(q, k, v, d_o, n_chunks, c, t, tail_read=0, flags=0, scale=No
     return dQ, dK, dV
 
 
+def masked_attn_bwd_dq_rows(q, k, v, d_o, rows, n_chunks, c, t, tail_read=0, flags=0, scale=None):
+    """dQ of the sampled rows only: a row's dQ depends on that row of the mask and of dO alone.
+    Returns [B, H, len(rows), D]."""
+    q, k, v, d_o = _f64(q), _f64(k), _f64(v), _f64(d_o)
+    rows = np.asarray(rows)
+    B, H, S, D = q.shape
+    M = mask_rows(rows, n_chunks, c, t, tail_read, flags)
+    out = np.zeros((B, H, len(rows), D))
+    for b in range(B):
+        for h in range(H):
+            out[b, h] = masked_softmax_attention_bwd(q[b, h][rows], k[b, h], v[b, h], d_o[b, h][rows], M, scale)[0]
+    return out
+
+
+def masked_attn_bwd_dkv_cols(q, k, v, d_o, cols, n_chunks, c, t, tail_read=0, flags=0, scale=None, block=2048):
+    """dK and dV of the sampled keys only.  A key's gradients sum over the rows that see it, and each
+    such row needs its whole softmax, so: find the rows whose mask row allows one of `cols`
+    (block by block, the mask is never held whole), run those rows in full, keep the sampled columns.
+    Returns (dK [B, H, len(cols), D], dV [B, H, len(cols), D])."""
+    q, k, v, d_o = _f64(q), _f64(k), _f64(v), _f64(d_o)
+    cols = np.asarray(cols)
+    B, H, S, D = q.shape
+    need = []
+    for lo in range(0, S, block):
+        r = np.arange(lo, min(S, lo + block))
+        hit = mask_rows(r, n_chunks, c, t, tail_read, flags)[:, cols].any(axis=1)
+        need.append(r[hit])
+    rows = np.concatenate(need)
+    M = mask_rows(rows, n_chunks, c, t, tail_read, flags)
+    dK = np.zeros((B, H, len(cols), D))
+    dV = np.zeros((B, H, len(cols), D))
+    sc = (1.0 / np.sqrt(D)) if scale is None else scale
+    for b in range(B):
+        for h in range(H):
+            _, P, _ = masked_softmax_attention(q[b, h][rows], k[b, h], v[b, h], M, sc)
+            g = d_o[b, h][rows]
+            dP = g @ v[b, h].T
+            dA = P * (dP - (P * dP).sum(axis=1, keepdims=True))
+            dK[b, h] = sc * (dA[:, cols].T @ q[b, h][rows])
+            dV[b, h] = P[:, cols].T @ g
+    return dK, dV
+
+
 # --------------------------------------------------------------------------
 # Generation (Section 3.1, Appendix A)
 # --------------------------------------------------------------------------

@@ -124,3 +124,65 @@ def test_masked_bwd_is_bitwise_repeatable():
     b = run_fwd_bwd(q, k, v, d_o, n, c, t, tail)
     for x, y in zip(a, b):
         assert torch.equal(x.view(torch.int16), y.view(torch.int16))
+
+
+# ------------------------------------- named workloads at full size (sampled)
+
+def _fwd_bwd_big(B, H, S, D, n, c, t, seed, flags=0):
+    q, k, v, d_o = (synthetic.big_normal_(torch.empty(B, H, S, D, dtype=torch.bfloat16, device=DEV), seed + i) for i in range(4))
+    return (q, k, v, d_o) + tuple(run_fwd_bwd(q, k, v, d_o, n, c, t, 0, flags))
+
+
+def test_training_layout_4608_tokens_backward_sampled_heads():
+    """B4 H32 D128 bf16, c=4, t=16, 4608 rows: the full launch; the oracle runs two (b,h) pairs in full."""
+    B, H, D, n, c, t = 4, 32, 128, 32, 4, 16
+    S = oracle.seq_len(n, c, t)
+    q, k, v, d_o, dq, dk, dv = _fwd_bwd_big(B, H, S, D, n, c, t, 200)
+    for b, h in [(0, 0), (3, 17)]:
+        sl = (slice(b, b + 1), slice(h, h + 1))
+        want = oracle.masked_attn_bwd(npf(q[sl]), npf(k[sl]), npf(v[sl]), npf(d_o[sl]), n, c, t)
+        for g, w, name in zip((dq, dk, dv), want, ("dq", "dk", "dv")):
+            check_grad(g[sl], w, torch.bfloat16, name)
+    for g in (dq, dk, dv):
+        assert torch.isfinite(g.float()).all()
+
+
+def test_training_layout_4608_tokens_backward_agrees_with_the_cuda_core_kernels_everywhere():
+    """Every element of the tensor-core result against the CUDA-core kernels of the same library
+    (an on-GPU second opinion over all 128 (b,h) pairs; the oracle covers two of them above)."""
+    B, H, D, n, c, t = 4, 32, 128, 32, 4, 16
+    S = oracle.seq_len(n, c, t)
+    q, k, v, d_o, dq, dk, dv = _fwd_bwd_big(B, H, S, D, n, c, t, 210)
+    gq, gk, gv = run_fwd_bwd(q, k, v, d_o, n, c, t, 0, GENERIC)
+    for a, b_, name in ((dq, gq, "dq"), (dk, gk, "dk"), (dv, gv, "dv")):
+        ref = b_.float()
+        d = (a.float() - ref).abs()
+        big = max(1.0, float(ref.abs().max()))
+        assert float(d.max()) <= 2e-2 * big, f"{name}: {float(d.max()):.3e} vs scale {big:.3g}"
+
+
+def test_long_training_layout_69632_tokens_backward_sampled_rows_and_keys():
+    """B1 H2 D128 bf16, c=8, t=32, 69632 rows: dQ on a seeded sample of rows of every zone type, dK and dV
+    on sampled keys (reading, repetition and late memory keys: an early memory key is seen by tens of
+    thousands of rows, each needing its whole softmax on the CPU)."""
+    B, H, D, n, c, t = 1, 2, 128, 128, 8, 32
+    S = oracle.seq_len(n, c, t)
+    assert S == 69632
+    q, k, v, d_o, dq, dk, dv = _fwd_bwd_big(B, H, S, D, n, c, t, 220)
+    ch, zone = oracle.layout_index(n, c, t)[:2]
+    rng = np.random.default_rng(1)
+    rows = np.unique(np.concatenate([rng.choice(np.nonzero(zone == z)[0], 48, replace=False) for z in (0, 1, 2)]
+                                    + [np.array([0, 255, 256, 287, 288, 543, S - 1, S - 257, S - 545])]))
+    cols = np.unique(np.concatenate([rng.choice(np.nonzero(zone == 0)[0], 24, replace=False),
+                                     rng.choice(np.nonzero(zone == 2)[0], 8, replace=False),
+                                     rng.choice(np.nonzero((zone == 1) & (ch >= n - 3))[0], 12, replace=False)]))
+    ri, ci = torch.from_numpy(rows).to(DEV), torch.from_numpy(cols).to(DEV)
+    h = 1
+    sl = (slice(0, 1), slice(h, h + 1))
+    want_dq = oracle.masked_attn_bwd_dq_rows(npf(q[sl]), npf(k[sl]), npf(v[sl]), npf(d_o[sl]), rows, n, c, t)
+    check_grad(dq[sl][:, :, ri], want_dq, torch.bfloat16, "dq")
+    want_dk, want_dv = oracle.masked_attn_bwd_dkv_cols(npf(q[sl]), npf(k[sl]), npf(v[sl]), npf(d_o[sl]), cols, n, c, t)
+    check_grad(dk[sl][:, :, ci], want_dk, torch.bfloat16, "dk")
+    check_grad(dv[sl][:, :, ci], want_dv, torch.bfloat16, "dv")
+    for g in (dq, dk, dv):
+        assert torch.isfinite(g.float()).all()

@@ -131,6 +131,19 @@ def test_gradient_support_follows_the_mask_and_reaches_the_memory_zone():
     assert np.abs(dk[0, 0, (zone == 0) & (chunk < 2)]).max() == 0
 
 
+@pytest.mark.parametrize("n,c,t,tail,flags", [(3, 2, 2, 1, 0), (2, 4, 4, 5, 1), (3, 2, 4, 0, 2)])
+def test_sampled_rows_and_keys_equal_the_full_backward(n, c, t, tail, flags):
+    S, D = oracle.seq_len(n, c, t, tail, flags), 8
+    q, k, v, w = (_rand((1, 2, S, D), 60 + i) for i in range(4))
+    dq, dk, dv = oracle.masked_attn_bwd(q, k, v, w, n, c, t, tail, flags)
+    rng = np.random.default_rng(3)
+    rows = np.sort(rng.choice(S, min(S, 11), replace=False))
+    cols = np.sort(rng.choice(S, min(S, 9), replace=False))
+    assert np.abs(oracle.masked_attn_bwd_dq_rows(q, k, v, w, rows, n, c, t, tail, flags) - dq[:, :, rows]).max() < 1e-12
+    gk, gv = oracle.masked_attn_bwd_dkv_cols(q, k, v, w, cols, n, c, t, tail, flags, block=7)
+    assert np.abs(gk - dk[:, :, cols]).max() < 1e-12 and np.abs(gv - dv[:, :, cols]).max() < 1e-12
+
+
 def test_planted_mistakes_in_the_backward_are_caught(monkeypatch):
     orig = lo.masked_softmax_attention_bwd
 
