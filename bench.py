@@ -393,6 +393,32 @@ def other_workloads(L, synthetic, torch, dev, peaks):
                                "useful_tflops": flops / (ms * 1e-3) / 1e12,
                                "frac_of_measured_bf16": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                                "gbs": 4.0 * q.numel() * 2 / (ms * 1e-3) / 1e9}
+
+    def backward(tag, B, H, n, c, t, q, k, v, o):
+        # gradients of the same layout (useful FLOPs: five products of the allowed pairs, 10*D per pair)
+        S = q.shape[2]
+        lse = torch.empty((B, H, S), dtype=torch.float32, device=dev)
+        L.loma_masked_attn_fwd(q, k, v, o, lse, n, c, t, 0, 0, 0.0, stream)
+        d_o = synthetic.big_normal_(torch.empty_like(q), 3050, std)
+        dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+        wsb = torch.empty(L.loma_masked_attn_bwd_workspace_bytes(B, H, D, n, c, t), dtype=torch.uint8, device=dev)
+        ms_b = timed(lambda: L.loma_masked_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, n, c, t, 0, 0, wsb, 0.0, stream))
+        fl = 10.0 * D * allowed_pairs(n, c, t) * B * H
+        nbytes = 8.0 * q.numel() * 2     # q, k, v, o, dO read, dq, dk, dv written, once each
+        res[tag] = {"config": dict(B=B, H=H, D=D, n=n, c=c, t=t, S=S), "ms": ms_b,
+                    "useful_tflops": fl / (ms_b * 1e-3) / 1e12,
+                    "frac_of_measured_bf16": fl / (ms_b * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                    "gbs": nbytes / (ms_b * 1e-3) / 1e9, "frac_of_measured_hbm": nbytes / (ms_b * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                    "kernels": "bwd_delta + masked_attn_bwd_dq_tc + masked_attn_bwd_dkv_tc"}
+
+    backward("masked_bwd_69632", B, H, n, c, t, q, k, v, o)
+    del q, k, v, o
+    torch.cuda.empty_cache()
+    B, H, n, c, t = 4, 32, 32, 4, 16
+    S = n * (2 * c * t + t)
+    q, k, v = (synthetic.big_normal_(torch.empty(B, H, S, D, dtype=bf, device=dev), 3060 + i, std) for i in range(3))
+    o = torch.empty_like(q)
+    backward("masked_bwd_4608", B, H, n, c, t, q, k, v, o)
     del q, k, v, o
     torch.cuda.empty_cache()
     B, H, c, t, mem_len = 64, 32, 8, 16, 16384
