@@ -20,7 +20,8 @@
 // (lse and delta of the 128 query rows of the step are staged in shared memory); then
 // dV += P^T dO_h and dK += dA^T Q_h with Q_h, dO_h as MN-major operands.
 //
-// Roles: warps 0-3 warpgroup, warp 4 TMA producer (one lane), warp 5 MMA issuer (warp-uniform
+// Roles: warps 0-7 two warpgroups (each takes half of the columns of every event, and half of the
+// epilogue), warp 8 TMA producer (one lane), warp 9 MMA issuer (warp-uniform
 // control flow, one elected lane issues).  Every mbarrier wait is bounded; on expiry the CTA
 // records LOMA_ERR_TIMEOUT, every role leaves its loop, TMEM is freed and the kernel returns.
 #include "tcgen05_common.cuh"
@@ -38,7 +39,7 @@ struct BwdParams {
     float scale;
 };
 
-constexpr int BWD_THREADS = 192;
+constexpr int BWD_THREADS = 320;   // two warpgroups, one TMA warp, one MMA warp
 constexpr int BWD_NBAR = 11;
 
 template <int D>
@@ -49,8 +50,8 @@ struct BwdDqSmem {
     static constexpr int Q_OFF = 0;
     static constexpr int G_OFF = TILE_BYTES;
     static constexpr int KV_OFF = 2 * TILE_BYTES;          // stage s: K at KV_OFF + 2*s*TILE, V one tile further
-    static constexpr int O_OFF = 6 * TILE_BYTES;           // 64-column staging panel of the output
-    static constexpr int TOTAL = 6 * TILE_BYTES + PANEL_BYTES;
+    static constexpr int O_OFF = 6 * TILE_BYTES;           // two 64-column staging panels of the output, one per warpgroup
+    static constexpr int TOTAL = 6 * TILE_BYTES + 2 * PANEL_BYTES;
 };
 
 // ------------------------------------------------------------------ delta_i = dO_i . O_i
@@ -97,13 +98,13 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int i = 0; i < BWD_NBAR; ++i) mbar_init(bar(i), (i == B_PF || i == B_PF + 1) ? 128 : 1);
+        for (int i = 0; i < BWD_NBAR; ++i) mbar_init(bar(i), (i == B_PF || i == B_PF + 1) ? 256 : 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // zero the operand buffers once: rows a TMA box does not cover keep finite contents
     for (int i = threadIdx.x; i < SM::TOTAL / 16; i += BWD_THREADS) reinterpret_cast<uint4*>(smem_gen)[i] = make_uint4(0, 0, 0, 0);
     fence_async_smem();
-    if (warp == 5) {
+    if (warp == 9) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(512)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -121,7 +122,7 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
     auto tile_of_round = [&](int r) { return r * nstreams + ((r & 1) ? nstreams - 1 - sid : sid); };
     auto kv_off = [&](int stage) { return (uint32_t)(SM::KV_OFF + stage * 2 * SM::TILE_BYTES); };
 
-    if (warp == 4) {
+    if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t gs = 0, tcount = 0;
@@ -163,7 +164,7 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
                 while (clock64() - t0 < 2000000ll) {}
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer
         constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
         constexpr uint32_t IDESC_DQ =
@@ -192,13 +193,14 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
             }
             __syncwarp();
         };
-        // dQ += dA K[64h .. 64h+63]: dA (bf16) read from TMEM over the S buffer, K as an MN-major operand
+        // dQ += dA K[64h .. 64h+63]: dA (bf16) read from TMEM over the S buffer (16 keys = 8 columns; keys 0-31 at
+        // columns 0-15, keys 32-63 at columns 32-47: each warpgroup writes inside the columns it read), K MN-major
         auto issue_dq = [&](int b, int h, int stage, bool first, bool last_of_step, bool last_of_tile) {
             if (elect_one()) {
                 const uint64_t kmn = smem_desc(smem_base + kv_off(stage), SM::PANEL_BYTES, 1024);
 #pragma unroll
                 for (int k4 = 0; k4 < 4; ++k4)
-                    mma_ts(tmem + 256, tmem + b * 64 + k4 * 8, kmn + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_DQ,
+                    mma_ts(tmem + 256, tmem + b * 64 + (k4 >> 1) * 32 + (k4 & 1) * 8, kmn + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_DQ,
                            !first || (k4 > 0));
                 if (last_of_step) tc_commit(bar(B_KVE + stage));
                 if (last_of_tile) tc_commit(bar(B_DQ));
@@ -245,9 +247,10 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
             gs += td.nsteps;
         }
     } else {
-        // ------------------------------------------------------------ warpgroup: dA, epilogue
-        const int rr = threadIdx.x;
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        // ------------------------------------------------------------ two warpgroups: dA, epilogue
+        // thread = query row = TMEM lane; warpgroup wg takes columns [32 wg, 32 wg + 32) of every event
+        const int rr = threadIdx.x & 127, wg = warp >> 2;
+        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         uint32_t ge = 0, tcount = 0;
         bool ok = true;
         bool store_pending = false;
@@ -283,8 +286,8 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t s_addr = lane_addr + b * 64, g_addr = lane_addr + 128 + b * 64;
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
+                {
+                    const int c = wg;
                     uint32_t s[32], g[32], pk[16];
                     tmem_ld32(s_addr + c * 32, s);
                     tmem_ld32(g_addr + c * 32, g);
@@ -300,7 +303,7 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
                         }
                         pk[e >> 1] = pack_bf16(da[0], da[1]);
                     }
-                    tmem_st16(s_addr + c * 16, pk);   // dA over the scores: 32 keys -> 16 columns
+                    tmem_st16(s_addr + c * 32, pk);   // dA over the scores this warpgroup has just read: 32 keys -> 16 columns
                 }
                 tmem_wait_st();
                 tc_fence_before();
@@ -309,48 +312,49 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_DQ), tcount & 1, abortp, p.status));
             if (ok) tc_fence_after();
 
-            // epilogue: scale, round to bf16, stage 64 columns at a time in shared memory, TMA store.
-            // Every thread of the warpgroup reaches the first barrier for every tile it started; it
+            // epilogue: scale, round to bf16, stage in shared memory, TMA store.  Warpgroup wg takes
+            // the output columns [64 wg, 64 wg + 64) (its own staging panel, its own named barrier).
+            // Every thread of a warpgroup reaches the first barrier for every tile it started; it
             // also makes giving up a uniform decision.
-            uint8_t* orow = smem_gen + SM::O_OFF + rr * 128;
+            uint8_t* orow = smem_gen + SM::O_OFF + wg * SM::PANEL_BYTES + rr * 128;
             bool give_up = false;
-#pragma unroll
-            for (int pn = 0; pn < PANELS; ++pn) {
+            if (wg < PANELS) {
+                const int pn = wg;
                 if (rr == 0 && store_pending) tma_store_wait_read();   // the staging panel is free again
-                if (pn == 0) {
-                    uint32_t any_bad;
-                    asm volatile(
-                        "{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, 1, 128, p;\nselp.u32 %0, 1, 0, q;\n}"
-                        : "=r"(any_bad)
-                        : "r"((uint32_t)(ok ? 0 : 1))
-                        : "memory");
-                    if (any_bad) { give_up = true; break; }
-                } else {
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-                }
+                uint32_t any_bad;
+                asm volatile(
+                    "{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, %2, 128, p;\nselp.u32 %0, 1, 0, q;\n}"
+                    : "=r"(any_bad)
+                    : "r"((uint32_t)(ok ? 0 : 1)), "r"(1 + wg)
+                    : "memory");
+                if (any_bad) give_up = true;
+                if (!give_up) {
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t x[32];
-                    tmem_ld32(lane_addr + 256 + pn * 64 + c * 32, x);
-                    tmem_wait_ld();
+                    for (int c = 0; c < 2; ++c) {
+                        uint32_t x[32];
+                        tmem_ld32(lane_addr + 256 + pn * 64 + c * 32, x);
+                        tmem_wait_ld();
 #pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        const int ci = c * 4 + q4;       // 16-byte chunk of the 128-byte panel row
-                        uint4 u;
-                        u.x = pack_bf16(__uint_as_float(x[q4 * 8 + 0]) * bp.scale, __uint_as_float(x[q4 * 8 + 1]) * bp.scale);
-                        u.y = pack_bf16(__uint_as_float(x[q4 * 8 + 2]) * bp.scale, __uint_as_float(x[q4 * 8 + 3]) * bp.scale);
-                        u.z = pack_bf16(__uint_as_float(x[q4 * 8 + 4]) * bp.scale, __uint_as_float(x[q4 * 8 + 5]) * bp.scale);
-                        u.w = pack_bf16(__uint_as_float(x[q4 * 8 + 6]) * bp.scale, __uint_as_float(x[q4 * 8 + 7]) * bp.scale);
-                        *reinterpret_cast<uint4*>(orow + ((ci ^ (rr & 7)) << 4)) = u;
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            const int ci = c * 4 + q4;       // 16-byte chunk of the 128-byte panel row
+                            uint4 u;
+                            u.x = pack_bf16(__uint_as_float(x[q4 * 8 + 0]) * bp.scale, __uint_as_float(x[q4 * 8 + 1]) * bp.scale);
+                            u.y = pack_bf16(__uint_as_float(x[q4 * 8 + 2]) * bp.scale, __uint_as_float(x[q4 * 8 + 3]) * bp.scale);
+                            u.z = pack_bf16(__uint_as_float(x[q4 * 8 + 4]) * bp.scale, __uint_as_float(x[q4 * 8 + 5]) * bp.scale);
+                            u.w = pack_bf16(__uint_as_float(x[q4 * 8 + 6]) * bp.scale, __uint_as_float(x[q4 * 8 + 7]) * bp.scale);
+                            *reinterpret_cast<uint4*>(orow + ((ci ^ (rr & 7)) << 4)) = u;
+                        }
+                    }
+                    fence_async_smem();
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
+                    if (rr == 0) {
+                        tma_store_5d(&maps.dq[td.view], smem_base + SM::O_OFF + wg * SM::PANEL_BYTES, pn * 64, td.r0, td.c0, hi, bi);
+                        tma_store_commit();
+                        store_pending = true;
                     }
                 }
-                fence_async_smem();
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (rr == 0) {
-                    tma_store_5d(&maps.dq[td.view], smem_base + SM::O_OFF, pn * 64, td.r0, td.c0, hi, bi);
-                    tma_store_commit();
-                    store_pending = true;
-                }
+            } else if (!ok) {
+                give_up = true;
             }
             if (give_up) { ok = false; break; }
             tc_fence_before();
@@ -360,7 +364,7 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == 9) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_slot), "r"(512) : "memory");
     }
@@ -392,8 +396,8 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
     const FwdParams& p = bp.f;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bars[BWD_NBAR];
-    __shared__ __align__(16) float lse2_s[2][128];   // -lse * log2(e) and delta of the query rows of a step, by ring stage
-    __shared__ __align__(16) float dl_s[2][128];
+    __shared__ __align__(16) float lse2_s[128];   // -lse * log2(e) and delta of the 128 query rows of the current step
+    __shared__ __align__(16) float dl_s[128];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
@@ -406,12 +410,12 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int i = 0; i < BWD_NBAR; ++i) mbar_init(bar(i), (i == B_PF || i == B_PF + 1) ? 128 : 1);
+        for (int i = 0; i < BWD_NBAR; ++i) mbar_init(bar(i), (i == B_PF || i == B_PF + 1) ? 256 : 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int i = threadIdx.x; i < SM::TOTAL / 16; i += BWD_THREADS) reinterpret_cast<uint4*>(smem_gen)[i] = make_uint4(0, 0, 0, 0);
     fence_async_smem();
-    if (warp == 5) {
+    if (warp == 9) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(512)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -429,7 +433,7 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
     auto tile_of_round = [&](int r) { return r * nstreams + ((r & 1) ? nstreams - 1 - sid : sid); };
     auto ring_off = [&](int stage) { return (uint32_t)(SM::KV_OFF + stage * 2 * SM::TILE_BYTES); };   // Q, then dO
 
-    if (warp == 4) {
+    if (warp == 8) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t gs = 0, tcount = 0;
@@ -468,7 +472,7 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
                 while (clock64() - t0 < 2000000ll) {}
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == 9) {
         // ------------------------------------------------------------ MMA issuer
         constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
         constexpr uint32_t IDESC_ACC =
@@ -503,11 +507,11 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
                 const uint64_t gmn = smem_desc(smem_base + ring_off(stage) + SM::TILE_BYTES, SM::PANEL_BYTES, 1024);
 #pragma unroll
                 for (int k4 = 0; k4 < 4; ++k4)
-                    mma_ts(tmem + 384, tmem + b * 64 + k4 * 8, gmn + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_ACC,
+                    mma_ts(tmem + 384, tmem + b * 64 + (k4 >> 1) * 32 + (k4 & 1) * 8, gmn + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_ACC,
                            !first || (k4 > 0));
 #pragma unroll
                 for (int k4 = 0; k4 < 4; ++k4)
-                    mma_ts(tmem + 256, tmem + 128 + b * 64 + k4 * 8, qmn + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_ACC,
+                    mma_ts(tmem + 256, tmem + 128 + b * 64 + (k4 >> 1) * 32 + (k4 & 1) * 8, qmn + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_ACC,
                            !first || (k4 > 0));
                 if (last_of_step) tc_commit(bar(B_QGE + stage));
                 if (last_of_tile) tc_commit(bar(B_DONE));
@@ -554,9 +558,10 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
             gs += kd.nsteps;
         }
     } else {
-        // ------------------------------------------------------------ warpgroup: P^T, dA^T, epilogue
-        const int kr = threadIdx.x;
-        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        // ------------------------------------------------------------ two warpgroups: P^T, dA^T, epilogue
+        // thread = key row = TMEM lane; warpgroup wg takes query rows [32 wg, 32 wg + 32) of every event
+        const int kr = threadIdx.x & 127, wg = warp >> 2;
+        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         uint32_t ge = 0, gs = 0, tcount = 0;
         bool ok = true;
         bool store_pending = false;
@@ -572,7 +577,7 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
             const bool key_valid = (kr < kv.R * kv.CH) && (kc <= kd.a1) && (ko < kv.Z);
             const HalfMasks hm = key_tile_half_masks(p, kd, lane);
             HalfWalk hw;
-            int lo = 0, hi2 = 0, stage = 0;
+            int lo = 0, hi2 = 0;
             for (hw.start(hm); ok && !hw.done(kd.nsteps); hw.next(hm), ++ge) {
                 if (hw.first_of_step(hm)) {
                     QTile qt;
@@ -580,7 +585,6 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
                     const View& qv = p.view[qt.view];
                     col_interval(qv, qt, kc, ko, kr, key_valid, lo, hi2);
                     // this thread fetches lse and delta of query row `kr` of the step's tile for everybody
-                    stage = (gs + hw.j) & 1;
                     const int rsub = fdiv(kr, qv.dR);
                     const int ro = qt.r0 + (kr - rsub * qv.R);
                     const int rc = qt.a0 + rsub;
@@ -590,9 +594,12 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
                         nl = -bp.lse_in[idx] * 1.4426950408889634f;
                         dl = bp.delta[idx];
                     }
-                    lse2_s[stage][kr] = nl;
-                    dl_s[stage][kr] = dl;
-                    asm volatile("bar.sync 2, 128;" ::: "memory");
+                    asm volatile("bar.sync 3, 256;" ::: "memory");   // everybody has finished with the previous step's values
+                    if (wg == 0) {
+                        lse2_s[kr] = nl;
+                        dl_s[kr] = dl;
+                    }
+                    asm volatile("bar.sync 3, 256;" ::: "memory");
                 }
                 const int b = ge & 1;
                 const int lo_h = lo - 64 * hw.h;
@@ -601,14 +608,14 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t s_addr = lane_addr + b * 64, g_addr = lane_addr + 128 + b * 64;
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
+                {
+                    const int c = wg;
                     uint32_t s[32], g[32], ppk[16], dpk[16];
                     tmem_ld32(s_addr + c * 32, s);
                     tmem_ld32(g_addr + c * 32, g);
                     tmem_wait_ld();
-                    const float4* nl4 = reinterpret_cast<const float4*>(&lse2_s[stage][64 * hw.h + c * 32]);
-                    const float4* dl4 = reinterpret_cast<const float4*>(&dl_s[stage][64 * hw.h + c * 32]);
+                    const float4* nl4 = reinterpret_cast<const float4*>(&lse2_s[64 * hw.h + c * 32]);
+                    const float4* dl4 = reinterpret_cast<const float4*>(&dl_s[64 * hw.h + c * 32]);
 #pragma unroll
                     for (int e = 0; e < 32; e += 4) {
                         const float4 nl = nl4[e >> 2], dl = dl4[e >> 2];
@@ -625,8 +632,8 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
                         dpk[e >> 1] = pack_bf16(da[0], da[1]);
                         dpk[(e >> 1) + 1] = pack_bf16(da[2], da[3]);
                     }
-                    tmem_st16(s_addr + c * 16, ppk);   // P^T over the scores: 32 query rows -> 16 columns
-                    tmem_st16(g_addr + c * 16, dpk);   // dA^T over dP^T
+                    tmem_st16(s_addr + c * 32, ppk);   // P^T over the scores this warpgroup has just read: 32 query rows -> 16 columns
+                    tmem_st16(g_addr + c * 32, dpk);   // dA^T over dP^T, likewise
                 }
                 tmem_wait_st();
                 tc_fence_before();
@@ -636,29 +643,29 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_DONE), tcount & 1, abortp, p.status));
             if (ok) tc_fence_after();
 
-            // epilogue: dK (scaled) then dV, rounded to bf16, 64 columns at a time through the staging panel
-            uint8_t* orow = smem_gen + SM::O_OFF + kr * 128;
+            // epilogue: warpgroup 0 stores dK (scaled), warpgroup 1 stores dV, each rounded to bf16 and
+            // taken 64 columns at a time through its own staging panel and named barrier
+            uint8_t* orow = smem_gen + SM::O_OFF + wg * SM::PANEL_BYTES + kr * 128;
+            const float mul = wg == 0 ? bp.scale : 1.f;
             bool give_up = false;
 #pragma unroll
-            for (int pass = 0; pass < 2 * PANELS; ++pass) {
-                const int which = pass / PANELS, pn = pass % PANELS;   // 0: dK, 1: dV
-                const float mul = which == 0 ? bp.scale : 1.f;
+            for (int pn = 0; pn < PANELS; ++pn) {
                 if (kr == 0 && store_pending) tma_store_wait_read();
-                if (pass == 0) {
+                if (pn == 0) {
                     uint32_t any_bad;
                     asm volatile(
-                        "{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, 1, 128, p;\nselp.u32 %0, 1, 0, q;\n}"
+                        "{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, %2, 128, p;\nselp.u32 %0, 1, 0, q;\n}"
                         : "=r"(any_bad)
-                        : "r"((uint32_t)(ok ? 0 : 1))
+                        : "r"((uint32_t)(ok ? 0 : 1)), "r"(1 + wg)
                         : "memory");
                     if (any_bad) { give_up = true; break; }
                 } else {
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
                 }
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     uint32_t x[32];
-                    tmem_ld32(lane_addr + 256 + which * 128 + pn * 64 + c * 32, x);
+                    tmem_ld32(lane_addr + 256 + wg * 128 + pn * 64 + c * 32, x);
                     tmem_wait_ld();
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4) {
@@ -672,10 +679,10 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
                     }
                 }
                 fence_async_smem();
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + wg) : "memory");
                 if (kr == 0) {
-                    tma_store_5d(which == 0 ? &maps.dk[kd.view] : &maps.dv[kd.view], smem_base + SM::O_OFF, pn * 64, kd.r0, kd.c0,
-                                 hi, bi);
+                    tma_store_5d(wg == 0 ? &maps.dk[kd.view] : &maps.dv[kd.view], smem_base + SM::O_OFF + wg * SM::PANEL_BYTES, pn * 64,
+                                 kd.r0, kd.c0, hi, bi);
                     tma_store_commit();
                     store_pending = true;
                 }
@@ -688,7 +695,7 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == 9) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_slot), "r"(512) : "memory");
     }
@@ -858,6 +865,7 @@ cudaError_t launch_masked_attn_bwd_dkv_tc(const void* q, const void* k, const vo
         sm_count[dev] = sms;
     }
     const int sms = sm_count[dev];
+    static_assert(BwdDqSmem<128>::TOTAL + 1024 + 1536 <= 227 * 1024, "dynamic + static shared memory of the backward kernels");
     const int64_t work = (int64_t)bp.f.total_tiles * bp.f.BH;
     const int grid = (int)(work < sms ? work : sms);
     if (D == 128)
