@@ -1,6 +1,6 @@
 """Small, self-contained launches of each kernel for profiler captures.
 
-    python -m paper_2401_09486_b200.profile_cases decode|compress|compress_prior|masked|masked_long [--reps N]
+    python -m paper_2401_09486_b200.profile_cases decode|compress|compress_prior|masked|masked_long|bwd|bwd_long [--reps N]
 
 Each case keeps the inputs larger than L2 (126 MB) so DRAM counters mean
 something, but holds at most a few GB on the device and launches the kernel a
@@ -22,7 +22,7 @@ from . import build, synthetic
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["decode", "compress", "compress_prior", "masked", "masked_long"])
+    ap.add_argument("case", choices=["decode", "compress", "compress_prior", "masked", "masked_long", "bwd", "bwd_long"])
     ap.add_argument("--reps", type=int, default=3)
     args = ap.parse_args()
     build.build_library()
@@ -52,15 +52,24 @@ def main():
             for r in range(args.reps):
                 L.loma_compress_step(qm, km, vm, kc, vc, om, None, mem_len, c, t, ws, flags)
     else:
-        if args.case == "masked":
+        if args.case in ("masked", "bwd"):
             B, H, n, c, t = 1, 32, 32, 4, 16               # one batch element of the 4608-token layout: 151 MB per tensor
         else:
             B, H, n, c, t = 1, 8, 128, 8, 32               # 8 heads of the 69632-token layout: 143 MB per tensor
         S = n * (2 * c * t + t)
         q, k, v = (synthetic.big_normal_(torch.empty(B, H, S, D, dtype=bf, device=dev), 10 + i, std) for i in range(3))
         o = torch.empty_like(q)
-        for r in range(args.reps):
-            L.loma_masked_attn_fwd(q, k, v, o, None, n, c, t)
+        if args.case.startswith("bwd"):
+            lse = torch.empty((B, H, S), dtype=torch.float32, device=dev)
+            L.loma_masked_attn_fwd(q, k, v, o, lse, n, c, t)
+            d_o = synthetic.big_normal_(torch.empty_like(q), 20, std)
+            dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+            ws = torch.empty(L.loma_masked_attn_bwd_workspace_bytes(B, H, D, n, c, t), dtype=torch.uint8, device=dev)
+            for r in range(args.reps):
+                L.loma_masked_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, n, c, t, 0, 0, ws)
+        else:
+            for r in range(args.reps):
+                L.loma_masked_attn_fwd(q, k, v, o, None, n, c, t)
     torch.cuda.synchronize()
     assert L.loma_device_status() == 0
     print("ok", args.case)
