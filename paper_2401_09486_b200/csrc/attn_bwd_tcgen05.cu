@@ -292,16 +292,20 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
                     tmem_ld32(s_addr + c * 32, s);
                     tmem_ld32(g_addr + c * 32, g);
                     tmem_wait_ld();
+                    // every row of this warp sees all 32 columns: no compare per entry
+                    const bool full = __all_sync(0xffffffffu, lo_h <= c * 32 && hi2 - 64 * hw.h >= c * 32 + 32);
+                    const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nl2 = pack2(neg_lse2, neg_lse2), ndl2 = pack2(-dl, -dl);
 #pragma unroll
                     for (int e = 0; e < 32; e += 2) {
-                        float da[2];
-#pragma unroll
-                        for (int u = 0; u < 2; ++u) {
-                            const bool allowed = (uint32_t)(c * 32 + e + u - lo_h) < span;
-                            const float pr = allowed ? fast_ex2(fmaf(__uint_as_float(s[e + u]), p.scale_log2, neg_lse2)) : 0.f;
-                            da[u] = pr * (__uint_as_float(g[e + u]) - dl);
+                        float x0, x1, d0, d1;
+                        unpack2(fma2(pack2(__uint_as_float(s[e]), __uint_as_float(s[e + 1])), sc2, nl2), x0, x1);
+                        unpack2(add2(pack2(__uint_as_float(g[e]), __uint_as_float(g[e + 1])), ndl2), d0, d1);
+                        float p0 = fast_ex2(x0), p1 = fast_ex2(x1);
+                        if (!full) {
+                            if ((uint32_t)(c * 32 + e - lo_h) >= span) p0 = 0.f;
+                            if ((uint32_t)(c * 32 + e + 1 - lo_h) >= span) p1 = 0.f;
                         }
-                        pk[e >> 1] = pack_bf16(da[0], da[1]);
+                        pk[e >> 1] = pack_bf16(p0 * d0, p1 * d1);
                     }
                     tmem_st16(s_addr + c * 32, pk);   // dA over the scores this warpgroup has just read: 32 keys -> 16 columns
                 }
@@ -616,21 +620,26 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
                     tmem_wait_ld();
                     const float4* nl4 = reinterpret_cast<const float4*>(&lse2_s[64 * hw.h + c * 32]);
                     const float4* dl4 = reinterpret_cast<const float4*>(&dl_s[64 * hw.h + c * 32]);
+                    const bool full = __all_sync(0xffffffffu, lo_h <= c * 32 && hi2 - 64 * hw.h >= c * 32 + 32);
+                    const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2);
 #pragma unroll
                     for (int e = 0; e < 32; e += 4) {
                         const float4 nl = nl4[e >> 2], dl = dl4[e >> 2];
-                        const float nlv[4] = {nl.x, nl.y, nl.z, nl.w}, dlv[4] = {dl.x, dl.y, dl.z, dl.w};
-                        float pr[4], da[4];
+                        float x[4], d[4];
+                        unpack2(fma2(pack2(__uint_as_float(s[e]), __uint_as_float(s[e + 1])), sc2, pack2(nl.x, nl.y)), x[0], x[1]);
+                        unpack2(fma2(pack2(__uint_as_float(s[e + 2]), __uint_as_float(s[e + 3])), sc2, pack2(nl.z, nl.w)), x[2], x[3]);
+                        d[0] = __uint_as_float(g[e]) - dl.x; d[1] = __uint_as_float(g[e + 1]) - dl.y;
+                        d[2] = __uint_as_float(g[e + 2]) - dl.z; d[3] = __uint_as_float(g[e + 3]) - dl.w;
+                        float pr[4];
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
-                            const bool allowed = (uint32_t)(c * 32 + e + u - lo_h) < span;
-                            pr[u] = allowed ? fast_ex2(fmaf(__uint_as_float(s[e + u]), p.scale_log2, nlv[u])) : 0.f;
-                            da[u] = pr[u] * (__uint_as_float(g[e + u]) - dlv[u]);
+                            pr[u] = fast_ex2(x[u]);
+                            if (!full && (uint32_t)(c * 32 + e + u - lo_h) >= span) pr[u] = 0.f;
                         }
                         ppk[e >> 1] = pack_bf16(pr[0], pr[1]);
                         ppk[(e >> 1) + 1] = pack_bf16(pr[2], pr[3]);
-                        dpk[e >> 1] = pack_bf16(da[0], da[1]);
-                        dpk[(e >> 1) + 1] = pack_bf16(da[2], da[3]);
+                        dpk[e >> 1] = pack_bf16(pr[0] * d[0], pr[1] * d[1]);
+                        dpk[(e >> 1) + 1] = pack_bf16(pr[2] * d[2], pr[3] * d[3]);
                     }
                     tmem_st16(s_addr + c * 32, ppk);   // P^T over the scores this warpgroup has just read: 32 query rows -> 16 columns
                     tmem_st16(g_addr + c * 32, dpk);   // dA^T over dP^T, likewise
