@@ -199,6 +199,27 @@ LOMA_API size_t loma_masked_attn_bwd_workspace_bytes(int B, int H, int D, int n_
                                                      unsigned flags);
 
 /* ---------------------------------------------------------------------------
+ * loma_rope_apply -- rotary position embedding of Q and K, in place, at the position ids of
+ * Section 4.5: reading rows keep their original ids, memory row j of chunk y gets
+ * y*tc + (j+1)c - 1 (Eq. 14; the generator's position_type 'intermittent'), repetition rows the id
+ * of the token they reproduce (the paper does not say).  position_type 1 selects the generator's
+ * other setting (Appendix A): memory row j of chunk y gets y*t + j.  The ids are computed from the
+ * row number; no id tensor is read.  The paper passes its ids to a Llama-2 model and does not write
+ * the rotation out; this is that model's: with half = D/2, theta_d = theta_base^(-2d/D),
+ *     x'[d] = x[d] cos(p theta_d) - x[d+half] sin(p theta_d),
+ *     x'[d+half] = x[d+half] cos(p theta_d) + x[d] sin(p theta_d),      d in [0, half).
+ *
+ *   q, k [device, in/out]  [B, H, S, D] with the strides of loma_masked_attn_fwd; either may be NULL
+ *   theta_base             <= 0 selects 10000
+ *   flags                  LOMA_FLAG_NO_REP_ZONE for the layout without repetition zones
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.  S == 0 or B*H == 0 is a no-op.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_rope_apply(void* q, void* k, int B, int H, int D,
+                             int n_chunks, int c, int t, int tc, int tail_read,
+                             int64_t stride_b, int64_t stride_h, int64_t stride_s,
+                             loma_dtype dtype, float theta_base, int position_type, unsigned flags, void* stream);
+
+/* ---------------------------------------------------------------------------
  * loma_prefill_cache -- what the cache holds after a prompt has been ingested (Section 3.1 step 3
  * applied to every complete chunk; Appendix A, compress_last_chunk's torch.cat lines): the memory-zone
  * K/V rows of chunks 0..n_chunks-1 in order, followed by the tail_read rows of the unfinished chunk.

@@ -31,6 +31,9 @@ from .loma_oracle import (  # noqa: F401
     masked_attn_bwd,
     masked_attn_bwd_dq_rows,
     masked_attn_bwd_dkv_cols,
+    position_ids,
+    rope_rotate,
+    rope_apply,
     decode_attn,
     compress_step,
     replay_generation,

@@ -413,6 +413,44 @@ def masked_attn_bwd_dkv_cols(q, k, v, d_o, cols, n_chunks, c, t, tail_read=0, fl
 
 
 # --------------------------------------------------------------------------
+# Rotary embedding at LoMA's position ids (Section 4.5; the rotation is Llama-2's)
+# --------------------------------------------------------------------------
+
+def position_ids(n_chunks, c, t, tail_read=0, flags=0, position_type="intermittent"):
+    """Position id of every row.  'intermittent' is Eq. 14 (layout_index's pos_id); 'contiguous' is the
+    generator's other setting (Appendix A, compress_last_chunk): memory row j of chunk y gets
+    mem_cursor + j with mem_cursor = y*t, everything else unchanged."""
+    chunk, zone, offset, _, pos = layout_index(n_chunks, c, t, tail_read, flags)
+    if position_type == "intermittent":
+        return pos.astype(np.int64)
+    assert position_type == "contiguous"
+    pos = pos.astype(np.int64).copy()
+    mem = zone == ZONE_MEM
+    pos[mem] = chunk[mem].astype(np.int64) * t + offset[mem]
+    return pos
+
+
+def rope_rotate(x, pos, theta_base=10000.0):
+    """Rotary position embedding as Llama-2 applies it (the model the paper fine-tunes; the paper only
+    supplies the ids).  x [..., S, D], pos [S].  Feature d of the first half is paired with feature
+    d + D/2; the pair is rotated by the angle pos * theta_base**(-2d/D)."""
+    x = _f64(x)
+    D = x.shape[-1]
+    half = D // 2
+    theta = theta_base ** (-2.0 * np.arange(half) / D)
+    ang = np.asarray(pos, dtype=np.float64)[:, None] * theta[None, :]      # [S, half]
+    cs, sn = np.cos(ang), np.sin(ang)
+    a, b = x[..., :half], x[..., half:]
+    return np.concatenate([a * cs - b * sn, b * cs + a * sn], axis=-1)
+
+
+def rope_apply(q, k, n_chunks, c, t, tail_read=0, flags=0, theta_base=10000.0, position_type="intermittent"):
+    """q and k [B, H, S, D] rotated at the layout's position ids.  Returns (q', k') in float64."""
+    pos = position_ids(n_chunks, c, t, tail_read, flags, position_type)
+    return rope_rotate(q, pos, theta_base), rope_rotate(k, pos, theta_base)
+
+
+# --------------------------------------------------------------------------
 # Generation (Section 3.1, Appendix A)
 # --------------------------------------------------------------------------
 

@@ -37,6 +37,7 @@ SIGNATURES = {
     "loma_masked_attn_bwd": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i,
                                   _f, _u, _p, _sz, _p]),
     "loma_masked_attn_bwd_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i, _u]),
+    "loma_rope_apply": (_i, [_p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i, _f, _i, _u, _p]),
     "loma_masked_attn_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
     "loma_masked_attn_bwd_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
@@ -208,6 +209,22 @@ def loma_masked_attn_bwd_plan_coverage(n_chunks: int, c: int, t: int, tail_read:
     rc = lib().loma_masked_attn_bwd_plan_coverage(n_chunks, c, t, tail_read, int(flags), _ptr(counts))
     _check(rc, "loma_masked_attn_bwd_plan_coverage")
     return counts
+
+
+def loma_rope_apply(q, k, n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0, theta_base: float = 0.0,
+                    position_type: int = 0, stream=None) -> None:
+    """Rotates q and k ([B, H, S, D] device tensors with identical strides; either may be None) in place at
+    the layout's position ids.  position_type 0: Eq. 14; 1: the generator's contiguous memory ids."""
+    ref = q if q is not None else k
+    B, H, S, D = ref.shape
+    if q is not None and k is not None and (k.shape != q.shape or k.stride() != q.stride() or k.dtype != q.dtype):
+        raise ValueError("q and k must share shape, strides and dtype")
+    if ref.stride(3) != 1:
+        raise ValueError("head dimension must be contiguous")
+    rc = lib().loma_rope_apply(_ptr(q), _ptr(k), B, H, D, n_chunks, c, t, c * t, tail_read, ref.stride(0), ref.stride(1),
+                               ref.stride(2), _dtype_code(ref), float(theta_base), int(position_type), int(flags),
+                               _stream(stream))
+    _check(rc, "loma_rope_apply")
 
 
 def loma_prefill_cache(k, v, k_cache, v_cache, n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0,

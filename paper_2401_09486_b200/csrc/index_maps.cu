@@ -5,44 +5,6 @@
 
 namespace loma {
 
-struct RowInfo {
-    int chunk, zone, offset, src, pos;
-};
-
-// Row i of the laid-out sequence -> its chunk, zone, offset, source token and
-// position id.  Rows beyond the last complete chunk are reading rows of chunk
-// n_chunks.  Memory position ids follow Eq. 14 with the chunk start at y*tc.
-__host__ __device__ inline RowInfo layout_row(int i, int n_chunks, int c, int t, int s) {
-    const int tc = c * t;   // s: chunk length, 2*tc + t, or tc + t in the layout without repetition zones
-    RowInfo r;
-    if (s == 0 || i >= n_chunks * s) {
-        r.chunk = n_chunks;
-        r.zone = LOMA_ZONE_READ;
-        r.offset = i - n_chunks * s;
-    } else {
-        r.chunk = i / s;
-        const int rem = i - r.chunk * s;
-        if (rem < tc) {
-            r.zone = LOMA_ZONE_READ;
-            r.offset = rem;
-        } else if (rem < tc + t) {
-            r.zone = LOMA_ZONE_MEM;
-            r.offset = rem - tc;
-        } else {
-            r.zone = LOMA_ZONE_REP;
-            r.offset = rem - tc - t;
-        }
-    }
-    if (r.zone == LOMA_ZONE_MEM) {
-        r.src = -1;
-        r.pos = r.chunk * tc + (r.offset + 1) * c - 1;
-    } else {
-        r.src = r.chunk * tc + r.offset;
-        r.pos = r.src;
-    }
-    return r;
-}
-
 struct GenInfo {
     int slot, pos, comp;
 };

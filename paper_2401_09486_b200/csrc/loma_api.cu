@@ -212,6 +212,35 @@ int loma_masked_attn_bwd(const void* q, const void* k, const void* v, const void
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 
+int loma_rope_apply(void* q, void* k, int B, int H, int D, int n_chunks, int c, int t, int tc, int tail_read,
+                    int64_t stride_b, int64_t stride_h, int64_t stride_s, loma_dtype dtype, float theta_base,
+                    int position_type, unsigned flags, void* stream) {
+    if (B < 0 || H < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    if (position_type != 0 && position_type != 1) return LOMA_ERR_INVALID_ARG;
+    Layout L;
+    const int rc = make_layout(n_chunks, c, t, tail_read, flags, &L);
+    if (rc != LOMA_OK) return rc;
+    if (tc != L.tc) return LOMA_ERR_INVALID_ARG;
+    if (L.S == 0 || B == 0 || H == 0 || (!q && !k)) return LOMA_OK;
+    if (q && q == k) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
+    if (stride_s < D || stride_b < 0 || stride_h < 0) return LOMA_ERR_INVALID_ARG;
+    const size_t es = elt_size(dtype);
+    if ((q && !aligned16(q)) || (k && !aligned16(k))) return LOMA_ERR_ALIGNMENT;
+    if ((stride_b * es) % 16 || (stride_h * es) % 16 || (stride_s * es) % 16) return LOMA_ERR_ALIGNMENT;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    const double base = theta_base > 0.f ? (double)theta_base : 10000.0;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the kernel skips a NULL tensor
+    cudaError_t e = cudaSuccess;
+    if (q && k) e = launch_rope(q, k, B, H, D, L, stride_b, stride_h, stride_s, dtype, base, position_type, st);
+    else e = launch_rope(q ? q : k, nullptr, B, H, D, L, stride_b, stride_h, stride_s, dtype, base, position_type, st);
+    return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
 int loma_prefill_cache(const void* k, const void* v, void* k_cache, void* v_cache, int B, int H, int D, int cap,
                        int n_chunks, int c, int t, int tc, int tail_read, int64_t stride_b, int64_t stride_h,
                        int64_t stride_s, loma_dtype dtype, unsigned flags, int* cache_len_out, void* stream) {

@@ -19,6 +19,45 @@ struct Layout {
     unsigned flags;
 };
 
+// ---- one row of the laid-out sequence (shared by the index-map and rotary kernels) ----
+struct RowInfo {
+    int chunk, zone, offset, src, pos;
+};
+
+// Row i of the laid-out sequence -> its chunk, zone, offset, source token and
+// position id.  Rows beyond the last complete chunk are reading rows of chunk
+// n_chunks.  Memory position ids follow Eq. 14 with the chunk start at y*tc.
+__host__ __device__ inline RowInfo layout_row(int i, int n_chunks, int c, int t, int s) {
+    const int tc = c * t;   // s: chunk length, 2*tc + t, or tc + t in the layout without repetition zones
+    RowInfo r;
+    if (s == 0 || i >= n_chunks * s) {
+        r.chunk = n_chunks;
+        r.zone = LOMA_ZONE_READ;
+        r.offset = i - n_chunks * s;
+    } else {
+        r.chunk = i / s;
+        const int rem = i - r.chunk * s;
+        if (rem < tc) {
+            r.zone = LOMA_ZONE_READ;
+            r.offset = rem;
+        } else if (rem < tc + t) {
+            r.zone = LOMA_ZONE_MEM;
+            r.offset = rem - tc;
+        } else {
+            r.zone = LOMA_ZONE_REP;
+            r.offset = rem - tc - t;
+        }
+    }
+    if (r.zone == LOMA_ZONE_MEM) {
+        r.src = -1;
+        r.pos = r.chunk * tc + (r.offset + 1) * c - 1;
+    } else {
+        r.src = r.chunk * tc + r.offset;
+        r.pos = r.src;
+    }
+    return r;
+}
+
 // ---- launchers (each defined in its own .cu) ------------------------------
 cudaError_t launch_layout_index(const Layout& L, int32_t* chunk, int32_t* zone, int32_t* offset,
                                 int32_t* src, int32_t* pos, cudaStream_t st);
@@ -84,6 +123,10 @@ cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const 
                                     void* k_cache, void* v_cache, void* o_mem, float* lse,
                                     int B, int H, int D, int cap, int mem_len, int c, int t,
                                     loma_dtype dt, float scale, unsigned flags, cudaStream_t st);
+
+// rotary embedding of Q and K rows at the layout's position ids (rope.cu)
+cudaError_t launch_rope(void* q, void* k, int B, int H, int D, const Layout& L, int64_t sb, int64_t sh, int64_t ss,
+                        loma_dtype dt, double theta_base, int position_type, cudaStream_t st);
 
 // ---- launch accounting -------------------------------------------------------
 void count_launches(int n);   // called by every launcher with the number of kernels it enqueued
