@@ -420,6 +420,11 @@ def other_workloads(L, synthetic, torch, dev, peaks):
     q, k, v = (synthetic.big_normal_(torch.empty(B, H, S, D, dtype=bf, device=dev), 3060 + i, std) for i in range(3))
     o = torch.empty_like(q)
     backward("masked_bwd_4608", B, H, n, c, t, q, k, v, o)
+    # rotary embedding of Q and K at the layout's position ids: Q and K read and written once
+    ms = timed(lambda: L.loma_rope_apply(q, k, n, c, t, 0, 0, 0.0, 0, stream))
+    nbytes = 4.0 * q.numel() * 2
+    res["rope_4608"] = {"config": dict(B=B, H=H, D=D, n=n, c=c, t=t, S=S), "ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9,
+                        "frac_of_measured_hbm": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "kernel": "rope_kernel"}
     del q, k, v, o
     torch.cuda.empty_cache()
     B, H, c, t, mem_len = 64, 32, 8, 16, 16384
