@@ -217,3 +217,30 @@ def test_rope_validation(lib):
     assert call(ss=68) == ALIGNMENT
     assert call(q=None, k=None) == 0                    # nothing to rotate
     assert call(H=0) == 0
+
+
+def _random_geometries(count, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < count:
+        c = int(rng.integers(1, 9))
+        t = int(rng.choice([1, 2, 3, 5, 8, 16, 17, 32, 48, 64, 100, 128, 130, 200]))
+        tc = c * t
+        n = int(rng.integers(0, 7))
+        tail = int(rng.integers(0, min(tc, 300) + 1))
+        flags = int(rng.integers(0, 4))
+        S = n * ((tc + t) if flags & 2 else (2 * tc + t)) + tail
+        if 0 < S <= 2600:
+            out.append((n, c, t, tail, flags))
+    return out
+
+
+@pytest.mark.parametrize("n,c,t,tail,flags", _random_geometries(40, 2024))
+def test_both_sides_of_the_plan_on_seeded_random_geometries(lib, n, c, t, tail, flags):
+    """Seeded random layouts (zone lengths on both sides of 64 and 128, odd sizes, ragged tails, every flag
+    combination): the plan read by query tile and the plan read by key tile both reproduce Eq. 2 exactly."""
+    want = oracle.dense_mask(n, c, t, tail, flags).astype(np.uint8)
+    by_query = binding.loma_masked_attn_plan_coverage(n, c, t, tail, flags).numpy()
+    by_key = binding.loma_masked_attn_bwd_plan_coverage(n, c, t, tail, flags).numpy()
+    assert np.array_equal(by_query, want), f"query side: {int((by_query != want).sum())} entries differ"
+    assert np.array_equal(by_key, want), f"key side: {int((by_key != want).sum())} entries differ"

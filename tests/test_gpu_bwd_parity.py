@@ -186,3 +186,40 @@ def test_long_training_layout_69632_tokens_backward_sampled_rows_and_keys():
     check_grad(dv[sl][:, :, ci], want_dv, torch.bfloat16, "dv")
     for g in (dq, dk, dv):
         assert torch.isfinite(g.float()).all()
+
+
+def _random_layouts(count, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < count:
+        c = int(rng.integers(1, 7))
+        t = int(rng.choice([1, 3, 5, 8, 16, 17, 32, 48, 64, 100, 130]))
+        tc = c * t
+        n = int(rng.integers(1, 5))
+        tail = int(rng.integers(0, min(tc, 200) + 1))
+        flags = int(rng.integers(0, 4))
+        S = n * ((tc + t) if flags & 2 else (2 * tc + t)) + tail
+        if 64 < S <= 900:
+            out.append((n, c, t, tail, flags, int(rng.choice([64, 128]))))
+    return out
+
+
+@pytest.mark.parametrize("n,c,t,tail,flags,D", _random_layouts(14, 7))
+def test_forward_and_backward_on_seeded_random_layouts(n, c, t, tail, flags, D):
+    """Zone lengths on both sides of 64 and 128, odd sizes, ragged tails, every flag combination, bf16
+    tensor-core kernels: outputs, log-sum-exp and all three gradients against the oracle."""
+    B, H = 1, 2
+    S = oracle.seq_len(n, c, t, tail, flags)
+    q, k, v = synthetic.qkv(B, H, S, D, seed=41, std=1.0, dtype=torch.bfloat16)
+    d_o = synthetic.normal_tensor((B, H, S, D), 43, 1.0, torch.bfloat16)
+    qd, kd, vd, gd = (x.to(DEV) for x in (q, k, v, d_o))
+    o = torch.full_like(qd, float("nan"))
+    lse = torch.full((B, H, S), float("nan"), dtype=torch.float32, device=DEV)
+    L.loma_masked_attn_fwd(qd, kd, vd, o, lse, n, c, t, tail, flags)
+    want_o, want_lse = oracle.masked_attn_fwd(npf(q), npf(k), npf(v), n, c, t, tail, flags)
+    torch.cuda.synchronize()
+    assert np.abs(npf(o) - want_o).max() <= 2e-2 and np.abs(npf(lse) - want_lse).max() <= 2e-2
+    got = run_fwd_bwd(qd, kd, vd, gd, n, c, t, tail, flags)
+    want = oracle.masked_attn_bwd(npf(q), npf(k), npf(v), npf(d_o), n, c, t, tail, flags)
+    for g, w, name in zip(got, want, ("dq", "dk", "dv")):
+        check_grad(g, w, torch.bfloat16, name)
