@@ -295,6 +295,30 @@ LOMA_API int loma_decode_attn(const void* q, const void* k_new, const void* v_ne
 LOMA_API size_t loma_decode_workspace_bytes(int B, int H, int D, int cache_len);
 
 /* ---------------------------------------------------------------------------
+ * loma_decode_attn_ragged -- the same decode step for a batch whose sequences stand at
+ * different points of their chunks.  The generator of Appendix A handles one sequence;
+ * batched, each sequence b has its own count of cache entries (memory entries of its
+ * compressed chunks plus its current tail), so sequence b attends to cache[b][0, len_b) and
+ * to itself, and its K/V are appended at slot len_b.
+ *
+ *   cache_lens     [device, in]  int32 [B]: entries before this token, per sequence;
+ *                                values are clamped to [0, max_cache_len] on the device
+ *   max_cache_len  [host]        an upper bound of cache_lens known to the caller without a
+ *                                device read (e.g. the longest sequence's length); sizes the
+ *                                launch and the workspace: loma_decode_workspace_bytes(B,H,D,max_cache_len);
+ *                                requires 0 <= max_cache_len < cap
+ * Everything else as in loma_decode_attn.  The split of the key range depends on
+ * max_cache_len only, so results repeat bit for bit for fixed arguments.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CAPACITY, WORKSPACE, CUDA.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_decode_attn_ragged(const void* q, const void* k_new, const void* v_new,
+                                     void* k_cache, void* v_cache, void* o, float* lse,
+                                     int B, int H, int D, int cap,
+                                     const int32_t* cache_lens, int max_cache_len,
+                                     loma_dtype dtype, float softmax_scale, unsigned flags,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------
  * loma_decode_attn_static -- the same decode step as loma_decode_attn (bf16
  * only), for callers that cannot hand the library a workspace because they
  * cannot obtain device memory at the point of the call.  (The paper has no

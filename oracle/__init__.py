@@ -35,6 +35,7 @@ from .loma_oracle import (  # noqa: F401
     rope_rotate,
     rope_apply,
     decode_attn,
+    decode_attn_ragged,
     compress_step,
     replay_generation,
 )

@@ -483,6 +483,23 @@ def decode_attn(q, k_new, v_new, k_cache, v_cache, cache_len, scale=None):
     return o, lse, kc, vc
 
 
+def decode_attn_ragged(q, k_new, v_new, k_cache, v_cache, cache_lens, scale=None):
+    """decode_attn for a batch whose sequences have their own cache lengths: sequence b is an
+    independent run of the generator (Appendix A handles one sequence at a time), so this is
+    decode_attn applied to each b with cache_lens[b].  Same return values as decode_attn."""
+    q = _f64(q)
+    B, H, _, D = q.shape
+    o = np.zeros((B, H, 1, D))
+    lse = np.zeros((B, H, 1))
+    kc = np.array(k_cache, copy=True)
+    vc = np.array(v_cache, copy=True)
+    for b in range(B):
+        ob, lb, kb, vb = decode_attn(q[b:b + 1], np.asarray(k_new)[b:b + 1], np.asarray(v_new)[b:b + 1],
+                                     np.asarray(k_cache)[b:b + 1], np.asarray(v_cache)[b:b + 1], int(cache_lens[b]), scale)
+        o[b], lse[b], kc[b], vc[b] = ob[0], lb[0], kb[0], vb[0]
+    return o, lse, kc, vc
+
+
 def compress_step(q_mem, k_mem, v_mem, k_cache, v_cache, mem_len, c, t, flags=0, scale=None):
     """Compress pass + compaction (Section 3.1 steps 2-3; Appendix A
     `compress_last_chunk`).

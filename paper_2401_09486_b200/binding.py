@@ -42,6 +42,7 @@ SIGNATURES = {
     "loma_masked_attn_bwd_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
+    "loma_decode_attn_ragged": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_attn_static": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _p]),
     "loma_decode_static_scratch_bytes": (_sz, []),
     "loma_compress_step": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz,
@@ -260,6 +261,23 @@ def loma_decode_attn(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len: int, 
                                 _ptr(lse), B, H, D, cap, cache_len, _dtype_code(q), float(softmax_scale),
                                 int(flags), _ptr(workspace), ws_bytes, _stream(stream))
     _check(rc, "loma_decode_attn")
+
+
+def loma_decode_attn_ragged(q, k_new, v_new, k_cache, v_cache, o, lse, cache_lens, max_cache_len: int, workspace=None,
+                            flags: int = 0, softmax_scale: float = 0.0, stream=None) -> None:
+    """loma_decode_attn with one cache length per sequence: cache_lens is a device int32 [B] tensor,
+    max_cache_len a host-side upper bound of its entries."""
+    B, H, cap, D = k_cache.shape
+    for x in (q, k_new, v_new, k_cache, v_cache, o, cache_lens):
+        if x is not None and not x.is_contiguous():
+            raise ValueError("decode tensors must be contiguous")
+    if cache_lens.dtype != torch.int32 or cache_lens.numel() != B:
+        raise ValueError("cache_lens must be int32 [B]")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().loma_decode_attn_ragged(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(o),
+                                       _ptr(lse), B, H, D, cap, _ptr(cache_lens), int(max_cache_len), _dtype_code(q),
+                                       float(softmax_scale), int(flags), _ptr(workspace), ws_bytes, _stream(stream))
+    _check(rc, "loma_decode_attn_ragged")
 
 
 def loma_decode_static_scratch_bytes() -> int:

@@ -246,9 +246,11 @@ template <typename T, int D>
 __global__ void __launch_bounds__(32)
 decode_generic_kernel(const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
                       T* __restrict__ k_cache, T* __restrict__ v_cache, T* __restrict__ o,
-                      float* __restrict__ lse, int cap, int cache_len, float scale) {
+                      float* __restrict__ lse, int cap, int cache_len_max, const int32_t* __restrict__ lens, int H,
+                      float scale) {
     __shared__ __align__(16) float q_sh[D];
     const int bh = blockIdx.x, lane = threadIdx.x;
+    const int cache_len = lens ? min(max(lens[bh / H], 0), cache_len_max) : cache_len_max;   // ragged batch
     T* kc = k_cache + (int64_t)bh * cap * D;
     T* vc = v_cache + (int64_t)bh * cap * D;
     DecodeMap<T> map;
@@ -534,30 +536,30 @@ cudaError_t launch_masked_attn_bwd_generic(const void* q, const void* k, const v
 
 template <typename T, int D>
 static cudaError_t decode_generic_t(const void* q, const void* kn, const void* vn, void* kc, void* vc,
-                                    void* o, float* lse, int BH, int cap, int cache_len, float scale,
-                                    cudaStream_t st) {
+                                    void* o, float* lse, int BH, int cap, int cache_len, const int32_t* lens, int H,
+                                    float scale, cudaStream_t st) {
     decode_generic_kernel<T, D><<<BH, 32, 0, st>>>(static_cast<const T*>(q), static_cast<const T*>(kn),
                                                    static_cast<const T*>(vn), static_cast<T*>(kc),
                                                    static_cast<T*>(vc), static_cast<T*>(o), lse, cap,
-                                                   cache_len, scale);
+                                                   cache_len, lens, H, scale);
     count_launches(1);
     return cudaGetLastError();
 }
 
 cudaError_t launch_decode_generic(const void* q, const void* k_new, const void* v_new, void* k_cache,
                                   void* v_cache, void* o, float* lse, int B, int H, int D, int cap,
-                                  int cache_len, loma_dtype dt, float scale, cudaStream_t st) {
+                                  int cache_len, const int32_t* lens, loma_dtype dt, float scale, cudaStream_t st) {
     const int BH = B * H;
     if (dt == LOMA_F32) {
         return D == 64 ? decode_generic_t<float, 64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
-                                                     cache_len, scale, st)
+                                                     cache_len, lens, H, scale, st)
                        : decode_generic_t<float, 128>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
-                                                      cache_len, scale, st);
+                                                      cache_len, lens, H, scale, st);
     }
     return D == 64 ? decode_generic_t<__nv_bfloat16, 64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
-                                                         cache_len, scale, st)
+                                                         cache_len, lens, H, scale, st)
                    : decode_generic_t<__nv_bfloat16, 128>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
-                                                          cache_len, scale, st);
+                                                          cache_len, lens, H, scale, st);
 }
 
 template <typename T, int D>

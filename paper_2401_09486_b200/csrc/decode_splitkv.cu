@@ -80,8 +80,8 @@ __global__ void __launch_bounds__(DEC_WARPS * 32)
 decode_splitkv_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                       const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ k_cache,
                       __nv_bfloat16* __restrict__ v_cache, __nv_bfloat16* __restrict__ o,
-                      float* __restrict__ lse, float* __restrict__ ws, int BH, int cap, int cache_len,
-                      int splits, int split_len, float scale_log2) {
+                      float* __restrict__ lse, float* __restrict__ ws, int BH, int cap, int cache_len_max,
+                      const int32_t* __restrict__ lens, int H, int splits, int split_len, float scale_log2) {
     constexpr int LPK = D / 8;           // lanes per row
     constexpr int KPL = 32 / LPK;        // rows per warp load
     constexpr int BK = DEC_NL * KPL;     // rows per warp iteration
@@ -89,12 +89,15 @@ decode_splitkv_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
     __shared__ __align__(16) float sm_o[DEC_WARPS][D];
 
     const int bh = blockIdx.x / splits, split = blockIdx.x - bh * splits;
+    // ragged batch: every sequence has its own length (clamped to the bound the launch was sized for);
+    // ranges beyond a sequence's end are empty and contribute nothing to the merge
+    const int cache_len = lens ? min(max(__ldg(lens + bh / H), 0), cache_len_max) : cache_len_max;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int sub = lane / LPK;          // which of the KPL rows of a load this lane works on
     const int li = lane % LPK;           // 16-byte column of the row
     const int total = cache_len + 1;
     const int k_begin = split * split_len;
-    const int k_end = min(total, k_begin + split_len);
+    const int k_end = min(total, k_begin + split_len);   // may be <= k_begin in a ragged batch
 
     const uint4* kc = reinterpret_cast<const uint4*>(k_cache + (int64_t)bh * cap * D);
     const uint4* vc = reinterpret_cast<const uint4*>(v_cache + (int64_t)bh * cap * D);
@@ -234,8 +237,8 @@ decode_merge_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ o,
 
 template <int D>
 static cudaError_t decode_bf16_t(const void* q, const void* kn, const void* vn, void* kc, void* vc, void* o,
-                                 float* lse, int BH, int cap, int cache_len, float scale, void* ws,
-                                 cudaStream_t st) {
+                                 float* lse, int BH, int cap, int cache_len, const int32_t* lens, int H, float scale,
+                                 void* ws, cudaStream_t st) {
     const int total = cache_len + 1;
     const int splits = decode_num_splits(BH, total);
     int split_len = (total + splits - 1) / splits;
@@ -244,7 +247,7 @@ static cudaError_t decode_bf16_t(const void* q, const void* kn, const void* vn, 
     decode_splitkv_kernel<D><<<BH * splits, DEC_WARPS * 32, 0, st>>>(
         static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(kn),
         static_cast<const __nv_bfloat16*>(vn), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
-        static_cast<__nv_bfloat16*>(o), lse, static_cast<float*>(ws), BH, cap, cache_len, splits, split_len,
+        static_cast<__nv_bfloat16*>(o), lse, static_cast<float*>(ws), BH, cap, cache_len, lens, H, splits, split_len,
         scale_log2);
     count_launches(1);
     cudaError_t e = cudaGetLastError();
@@ -257,10 +260,10 @@ static cudaError_t decode_bf16_t(const void* q, const void* kn, const void* vn, 
 
 cudaError_t launch_decode_bf16(const void* q, const void* k_new, const void* v_new, void* k_cache,
                                void* v_cache, void* o, float* lse, int B, int H, int D, int cap, int cache_len,
-                               float scale, void* ws, cudaStream_t st) {
+                               const int32_t* lens, float scale, void* ws, cudaStream_t st) {
     const int BH = B * H;
-    return D == 64 ? decode_bf16_t<64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap, cache_len, scale, ws, st)
-                   : decode_bf16_t<128>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap, cache_len, scale, ws,
+    return D == 64 ? decode_bf16_t<64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap, cache_len, lens, H, scale, ws, st)
+                   : decode_bf16_t<128>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap, cache_len, lens, H, scale, ws,
                                         st);
 }
 
@@ -294,7 +297,7 @@ cudaError_t launch_decode_bf16_static(const void* q, const void* k_new, const vo
                                       int cache_len, float scale, cudaStream_t st) {
     void* ws = decode_static_scratch();
     if (!ws) return cudaErrorInvalidSymbol;
-    return launch_decode_bf16(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, scale, ws, st);
+    return launch_decode_bf16(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, nullptr, scale, ws, st);
 }
 
 }  // namespace loma

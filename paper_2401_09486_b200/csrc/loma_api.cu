@@ -316,11 +316,42 @@ int loma_decode_attn(const void* q, const void* k_new, const void* v_new, void* 
     if ((int64_t)B * H * 128 > INT_MAX) return LOMA_ERR_INVALID_ARG;
     cudaError_t e;
     if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC))
-        e = launch_decode_bf16(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, scale,
+        e = launch_decode_bf16(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, nullptr, scale,
                                workspace, st);
     else
-        e = launch_decode_generic(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, dtype,
+        e = launch_decode_generic(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, nullptr, dtype,
                                   scale, st);
+    return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
+int loma_decode_attn_ragged(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
+                            float* lse, int B, int H, int D, int cap, const int32_t* cache_lens, int max_cache_len,
+                            loma_dtype dtype, float softmax_scale, unsigned flags, void* workspace,
+                            size_t workspace_bytes, void* stream) {
+    if (B < 0 || H < 0 || cap < 0 || max_cache_len < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    if ((k_new == nullptr) != (v_new == nullptr)) return LOMA_ERR_INVALID_ARG;
+    if (max_cache_len >= cap) return LOMA_ERR_CAPACITY;
+    if (B == 0 || H == 0) return LOMA_OK;
+    if (!q || !k_cache || !v_cache || !o || !cache_lens) return LOMA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) || !aligned16(k_new) ||
+        !aligned16(v_new) || !aligned16(workspace) || ((uintptr_t)cache_lens & 3u))
+        return LOMA_ERR_ALIGNMENT;
+    const size_t need = loma_decode_workspace_bytes(B, H, D, max_cache_len);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return LOMA_ERR_WORKSPACE;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((int64_t)B * H * 128 > INT_MAX) return LOMA_ERR_INVALID_ARG;
+    cudaError_t e;
+    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC))
+        e = launch_decode_bf16(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, max_cache_len, cache_lens, scale,
+                               workspace, st);
+    else
+        e = launch_decode_generic(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, max_cache_len, cache_lens,
+                                  dtype, scale, st);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 

@@ -99,14 +99,14 @@ cudaError_t launch_bounded_wait_selftest(cudaStream_t st);   // attn_tcgen05.cu
 
 cudaError_t launch_decode_generic(const void* q, const void* k_new, const void* v_new,
                                   void* k_cache, void* v_cache, void* o, float* lse,
-                                  int B, int H, int D, int cap, int cache_len,
+                                  int B, int H, int D, int cap, int cache_len, const int32_t* lens,
                                   loma_dtype dt, float scale, cudaStream_t st);
 
 // bf16 split-KV decode (decode_splitkv.cu)
 size_t decode_workspace_bytes(int BH, int D, int total_keys);
 cudaError_t launch_decode_bf16(const void* q, const void* k_new, const void* v_new, void* k_cache,
                                void* v_cache, void* o, float* lse, int B, int H, int D, int cap, int cache_len,
-                               float scale, void* ws, cudaStream_t st);
+                               const int32_t* lens, float scale, void* ws, cudaStream_t st);   // lens: per-sequence lengths or NULL
 
 size_t decode_static_scratch_bytes();
 cudaError_t launch_decode_bf16_static(const void* q, const void* k_new, const void* v_new, void* k_cache,

@@ -244,3 +244,15 @@ def test_both_sides_of_the_plan_on_seeded_random_geometries(lib, n, c, t, tail, 
     by_key = binding.loma_masked_attn_bwd_plan_coverage(n, c, t, tail, flags).numpy()
     assert np.array_equal(by_query, want), f"query side: {int((by_query != want).sum())} entries differ"
     assert np.array_equal(by_key, want), f"key side: {int((by_key != want).sum())} entries differ"
+
+
+def test_ragged_decode_validation(lib):
+    def call(q=0x1000, kn=0x2000, vn=0x3000, kc=0x4000, vc=0x5000, o=0x6000, B=2, H=1, D=128, cap=8, lens=0x7000, mx=3,
+             dt=1):
+        return lib.loma_decode_attn_ragged(q, kn, vn, kc, vc, o, None, B, H, D, cap, lens, mx, dt, 0.0, 0, None, 0, None)
+    assert call(mx=8) == CAPACITY
+    assert call(mx=-1) == INVALID
+    assert call(lens=None) == INVALID
+    assert call(lens=0x7002) == ALIGNMENT
+    assert call(D=100) == UNSUPPORTED
+    assert call(B=0) == 0

@@ -275,6 +275,41 @@ def test_decode_matches_oracle(B, H, D, cap, cache_len, flags, dtype):
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, GENERIC])
+@pytest.mark.parametrize("H,D,cap,lens", [(2, 64, 40, [0, 1, 39, 17]), (3, 128, 3000, [2999, 0, 1500, 257, 256, 255]),
+                                          (2, 128, 5000, [4133, 4133]), (4, 128, 9000, [8193, 100, 8256, 4097, 1])])
+def test_ragged_decode_matches_oracle(H, D, cap, lens, flags, dtype):
+    """Sequences at different points of their chunks: each attends to its own prefix of its cache."""
+    B = len(lens)
+    kc = synthetic.normal_tensor((B, H, cap, D), 31, 1.0, dtype)
+    vc = synthetic.normal_tensor((B, H, cap, D), 32, 1.0, dtype)
+    q, kn, vn = synthetic.qkv(B, H, 1, D, seed=33, std=1.0, dtype=dtype)
+    want_o, want_lse, _, _ = oracle.decode_attn_ragged(npf(q), npf(kn), npf(vn), npf(kc), npf(vc), lens)
+    kcd, vcd = kc.to(DEV), vc.to(DEV)
+    o = torch.full((B, H, 1, D), float("nan"), dtype=dtype, device=DEV)
+    lse = torch.full((B, H), float("nan"), dtype=torch.float32, device=DEV)
+    max_len = max(lens)
+    ws = workspace(L.loma_decode_workspace_bytes(B, H, D, max_len))
+    lens_d = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    L.loma_decode_attn_ragged(q.to(DEV), kn.to(DEV), vn.to(DEV), kcd, vcd, o, lse, lens_d, max_len, ws, flags)
+    torch.cuda.synchronize()
+    check_close(o, want_o, dtype)
+    assert np.abs(npf(lse) - want_lse[:, :, 0]).max() <= (1e-5 if dtype == torch.float32 else 2e-2)
+    exp_k, exp_v = kc.clone(), vc.clone()
+    for b, n in enumerate(lens):
+        exp_k[b, :, n] = kn[b, :, 0]
+        exp_v[b, :, n] = vn[b, :, 0]
+    assert np.array_equal(bits(kcd), bits(exp_k)) and np.array_equal(bits(vcd), bits(exp_v))
+    # equal lengths reproduce the uniform entry point bit for bit
+    o_u, o_r = torch.empty_like(o), torch.empty_like(o)
+    same = torch.full((B,), max_len, dtype=torch.int32, device=DEV)
+    L.loma_decode_attn(q.to(DEV), None, None, kcd, vcd, o_u, None, max_len, ws, flags)
+    L.loma_decode_attn_ragged(q.to(DEV), None, None, kcd, vcd, o_r, None, same, max_len, ws, flags)
+    torch.cuda.synchronize()
+    assert torch.equal(o_u, o_r)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("flags", [0, PRIOR, GENERIC, GENERIC | PRIOR])
 @pytest.mark.parametrize("B,H,D,c,t,mem_len,extra", [(1, 1, 64, 4, 4, 0, 0), (2, 2, 128, 4, 16, 48, 5),
                                                      (2, 3, 128, 8, 16, 1024, 0), (1, 2, 128, 3, 5, 35, 2),

@@ -589,3 +589,25 @@ def test_planted_mistakes_in_the_oracle_are_caught(monkeypatch, golden_dir):
         m.setattr(oracle, "compress_step", broken_compress)
         with pytest.raises(AssertionError):
             test_compress_is_unmasked_sdpa_and_cat_compaction(0)
+
+
+def test_ragged_decode_is_per_sequence_decode():
+    """Equal lengths give the uniform function; a sequence's result does not depend on its neighbours'
+    lengths or contents; entries at and beyond a sequence's own length (other than the appended slot)
+    are neither read nor written."""
+    B, H, D, cap = 3, 2, 8, 12
+    kc, vc = _rand((B, H, cap, D), 70), _rand((B, H, cap, D), 71)
+    q, kn, vn = _rand((B, H, 1, D), 72), _rand((B, H, 1, D), 73), _rand((B, H, 1, D), 74)
+    o_u, l_u, k_u, v_u = oracle.decode_attn(q, kn, vn, kc, vc, 5)
+    o_r, l_r, k_r, v_r = oracle.decode_attn_ragged(q, kn, vn, kc, vc, [5, 5, 5])
+    assert np.array_equal(o_u, o_r) and np.array_equal(l_u, l_r) and np.array_equal(k_u, k_r) and np.array_equal(v_u, v_r)
+    lens = [0, 7, 3]
+    o_r, _, k_r, v_r = oracle.decode_attn_ragged(q, kn, vn, kc, vc, lens)
+    kc2 = kc.copy(); kc2[0] += 100.0; kc2[2, :, 4:] = np.nan      # other sequences changed, own tail beyond len poisoned
+    o_2, _, _, _ = oracle.decode_attn_ragged(q, kn, vn, kc2, vc, lens)
+    assert np.array_equal(o_r[1], o_2[1]) and np.isfinite(o_2[2]).all()
+    assert np.allclose(o_r[0, :, 0], vn[0, :, 0])                 # empty cache: the token sees only itself
+    for b, n in enumerate(lens):
+        assert np.array_equal(k_r[b, :, n], kn[b, :, 0]) and np.array_equal(v_r[b, :, n], vn[b, :, 0])
+        keep = np.ones(cap, bool); keep[n] = False
+        assert np.array_equal(k_r[b][:, keep], kc[b][:, keep])
