@@ -444,6 +444,14 @@ def other_workloads(L, synthetic, torch, dev, peaks):
     res["decode_B64_16k"] = {"config": dict(B=B, H=H, D=D, c=c, t=t, cache_len=cache_len), "ms": ms,
                              "gbs": nbytes / (ms * 1e-3) / 1e9,
                              "frac_of_measured_hbm": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    # the same decode with one length per sequence, spread over the last chunk's tail positions
+    lens = torch.tensor([mem_len + (7 * b) % tc for b in range(B)], dtype=torch.int32, device=dev)
+    max_len = mem_len + tc - 1
+    ms = timed(lambda: L.loma_decode_attn_ragged(q1, k1, v1, kc, vc, o1, None, lens, max_len, ws, 0, 0.0, stream))
+    nbytes = 2.0 * float((lens.double() + 1).sum()) * H * D * 2
+    res["decode_ragged_B64_16k"] = {"config": dict(B=B, H=H, D=D, c=c, t=t, lens="mem_len + (7 b) mod tc"), "ms": ms,
+                                    "gbs": nbytes / (ms * 1e-3) / 1e9,
+                                    "frac_of_measured_hbm": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
     for name, flags in (("compress_B64_16k", 0), ("compress_B64_16k_prior_mem", 1)):
         def run_decode_then_compress():
             L.loma_compress_step(qm, km, vm, kc, vc, om, None, mem_len, c, t, ws, flags, 0.0, stream)
