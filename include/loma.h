@@ -396,6 +396,27 @@ LOMA_API int loma_compress_step(const void* q_mem, const void* k_mem, const void
 
 LOMA_API size_t loma_compress_workspace_bytes(int B, int H, int D, int t, int mem_len, unsigned flags);
 
+/* ---------------------------------------------------------------------------
+ * loma_compress_step_ragged -- the compress step for a batch whose sequences reach the end
+ * of a chunk at different times (Section 3.1 steps 2-3 once per sequence; Appendix A runs one
+ * sequence).  Sequence b compresses in this call iff mem_lens[b] >= 0: its t memory queries then
+ * attend to its tail cache[b][mem_lens[b], mem_lens[b] + tc) and to their own keys, and
+ * k_mem[b], v_mem[b] are written over slots [mem_lens[b], mem_lens[b] + t).  Sequences with a
+ * negative entry are left alone: their caches and their rows of o_mem and lse are not touched.
+ *
+ *   mem_lens     [device, in]  int32 [B]: memory entries in front of the tail, per sequence,
+ *                              or negative; values above max_mem_len are clamped to it
+ *   max_mem_len  [host]        upper bound of mem_lens; requires max_mem_len + tc <= cap
+ * Only the default mask (memory rows see their own chunk) is offered: with
+ * LOMA_FLAG_MEM_SEES_PRIOR_MEM the call returns UNSUPPORTED.  No workspace is needed.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CAPACITY, CUDA.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_compress_step_ragged(const void* q_mem, const void* k_mem, const void* v_mem,
+                                       void* k_cache, void* v_cache, void* o_mem, float* lse,
+                                       int B, int H, int D, int cap,
+                                       const int32_t* mem_lens, int max_mem_len, int c, int t, int tc,
+                                       loma_dtype dtype, float softmax_scale, unsigned flags, void* stream);
+
 /* Synchronises `stream`, then returns the device status word of the current
  * device: LOMA_OK, or LOMA_ERR_TIMEOUT if a bounded wait inside a kernel has
  * expired since the last call (the word is cleared by the call).

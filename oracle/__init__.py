@@ -37,5 +37,6 @@ from .loma_oracle import (  # noqa: F401
     decode_attn,
     decode_attn_ragged,
     compress_step,
+    compress_step_ragged,
     replay_generation,
 )

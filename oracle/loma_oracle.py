@@ -543,6 +543,29 @@ def compress_step(q_mem, k_mem, v_mem, k_cache, v_cache, mem_len, c, t, flags=0,
     return o, lse, new_k, new_v
 
 
+def compress_step_ragged(q_mem, k_mem, v_mem, k_cache, v_cache, mem_lens, c, t, scale=None):
+    """compress_step for a batch whose sequences finish their chunks at different times: sequence b
+    is compressed with its own mem_lens[b] when that is >= 0 and left alone otherwise (each sequence
+    is its own run of the generator).  Returns (o_mem [B,H,t,D] with NaN rows for untouched
+    sequences, lse likewise, k_cache', v_cache')."""
+    q_mem = _f64(q_mem)
+    B, H, _, D = q_mem.shape
+    o = np.full((B, H, t, D), np.nan)
+    lse = np.full((B, H, t), np.nan)
+    kc = np.array(k_cache, copy=True)
+    vc = np.array(v_cache, copy=True)
+    for b in range(B):
+        n = int(mem_lens[b])
+        if n < 0:
+            continue
+        ob, lb, kb, vb = compress_step(q_mem[b:b + 1], np.asarray(k_mem)[b:b + 1], np.asarray(v_mem)[b:b + 1],
+                                       np.asarray(k_cache)[b:b + 1], np.asarray(v_cache)[b:b + 1], n, c, t, 0, scale)
+        o[b], lse[b] = ob[0], lb[0]
+        kc[b, :, :n + t] = kb[0]
+        vc[b, :, :n + t] = vb[0]
+    return o, lse, kc, vc
+
+
 def replay_generation(q, k, v, n_chunks, c, t, tail_read=0, flags=0, scale=None):
     """Run the laid-out sequence through the generation path chunk by chunk.
 

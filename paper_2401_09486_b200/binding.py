@@ -48,6 +48,7 @@ SIGNATURES = {
     "loma_compress_step": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz,
                                 _p]),
     "loma_compress_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _u]),
+    "loma_compress_step_ragged": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _p, _i, _i, _i, _i, _i, _f, _u, _p]),
     "loma_device_status": (_i, [_p]),
     "loma_selftest_bounded_wait": (_i, [_p]),
     "loma_launch_count": (ctypes.c_uint64, []),
@@ -297,6 +298,22 @@ def loma_decode_attn_static(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len
                                        _ptr(lse), B, H, D, cap, cache_len, _dtype_code(q), float(softmax_scale),
                                        _stream(stream))
     _check(rc, "loma_decode_attn_static")
+
+
+def loma_compress_step_ragged(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, mem_lens, max_mem_len: int, c: int, t: int,
+                              flags: int = 0, softmax_scale: float = 0.0, stream=None) -> None:
+    """loma_compress_step with one count of memory entries per sequence (device int32 [B]; negative = the
+    sequence does not compress in this call)."""
+    B, H, cap, D = k_cache.shape
+    for x in (q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, mem_lens):
+        if not x.is_contiguous():
+            raise ValueError("compress tensors must be contiguous")
+    if mem_lens.dtype != torch.int32 or mem_lens.numel() != B:
+        raise ValueError("mem_lens must be int32 [B]")
+    rc = lib().loma_compress_step_ragged(_ptr(q_mem), _ptr(k_mem), _ptr(v_mem), _ptr(k_cache), _ptr(v_cache), _ptr(o_mem),
+                                         _ptr(lse), B, H, D, cap, _ptr(mem_lens), int(max_mem_len), c, t, c * t,
+                                         _dtype_code(q_mem), float(softmax_scale), int(flags), _stream(stream))
+    _check(rc, "loma_compress_step_ragged")
 
 
 def loma_compress_workspace_bytes(B: int, H: int, D: int, t: int, mem_len: int, flags: int = 0) -> int:

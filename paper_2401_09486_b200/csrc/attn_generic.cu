@@ -292,10 +292,15 @@ template <typename T, int D>
 __global__ void __launch_bounds__(GENERIC_WARPS * 32)
 compress_generic_kernel(const T* __restrict__ q_mem, const T* __restrict__ k_mem,
                         const T* __restrict__ v_mem, T* __restrict__ k_cache, T* __restrict__ v_cache,
-                        T* __restrict__ o_mem, float* __restrict__ lse, int cap, int mem_len, int t, int tc,
-                        unsigned flags, float scale) {
+                        T* __restrict__ o_mem, float* __restrict__ lse, int cap, int mem_len, const int32_t* __restrict__ mem_lens,
+                        int H, int t, int tc, unsigned flags, float scale) {
     __shared__ __align__(16) float q_sh[GENERIC_WARPS][D];
     const int bh = blockIdx.x;
+    if (mem_lens) {                          // ragged batch: own count of memory entries; negative = not compressing now
+        const int own = mem_lens[bh / H];
+        if (own < 0) return;
+        mem_len = min(own, mem_len);
+    }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     T* kc = k_cache + (int64_t)bh * cap * D;
     T* vc = v_cache + (int64_t)bh * cap * D;
@@ -564,30 +569,30 @@ cudaError_t launch_decode_generic(const void* q, const void* k_new, const void* 
 
 template <typename T, int D>
 static cudaError_t compress_generic_t(const void* qm, const void* km, const void* vm, void* kc, void* vc,
-                                      void* om, float* lse, int BH, int cap, int mem_len, int t, int tc,
-                                      unsigned flags, float scale, cudaStream_t st) {
+                                      void* om, float* lse, int BH, int cap, int mem_len, const int32_t* mem_lens, int H, int t,
+                                      int tc, unsigned flags, float scale, cudaStream_t st) {
     compress_generic_kernel<T, D><<<BH, GENERIC_WARPS * 32, 0, st>>>(
         static_cast<const T*>(qm), static_cast<const T*>(km), static_cast<const T*>(vm), static_cast<T*>(kc),
-        static_cast<T*>(vc), static_cast<T*>(om), lse, cap, mem_len, t, tc, flags, scale);
+        static_cast<T*>(vc), static_cast<T*>(om), lse, cap, mem_len, mem_lens, H, t, tc, flags, scale);
     count_launches(1);
     return cudaGetLastError();
 }
 
 cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache,
                                     void* v_cache, void* o_mem, float* lse, int B, int H, int D, int cap,
-                                    int mem_len, int c, int t, loma_dtype dt, float scale, unsigned flags,
-                                    cudaStream_t st) {
+                                    int mem_len, const int32_t* mem_lens, int c, int t, loma_dtype dt, float scale,
+                                    unsigned flags, cudaStream_t st) {
     const int BH = B * H, tc = c * t;
     if (dt == LOMA_F32) {
         return D == 64 ? compress_generic_t<float, 64>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH,
-                                                       cap, mem_len, t, tc, flags, scale, st)
+                                                       cap, mem_len, mem_lens, H, t, tc, flags, scale, st)
                        : compress_generic_t<float, 128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH,
-                                                        cap, mem_len, t, tc, flags, scale, st);
+                                                        cap, mem_len, mem_lens, H, t, tc, flags, scale, st);
     }
     return D == 64 ? compress_generic_t<__nv_bfloat16, 64>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse,
-                                                           BH, cap, mem_len, t, tc, flags, scale, st)
+                                                           BH, cap, mem_len, mem_lens, H, t, tc, flags, scale, st)
                    : compress_generic_t<__nv_bfloat16, 128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse,
-                                                            BH, cap, mem_len, t, tc, flags, scale, st);
+                                                            BH, cap, mem_len, mem_lens, H, t, tc, flags, scale, st);
 }
 
 }  // namespace loma

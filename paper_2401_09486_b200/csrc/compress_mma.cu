@@ -100,8 +100,8 @@ __global__ void __launch_bounds__(CMP_WARPS * 32)
 compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16* __restrict__ k_mem,
                     const __nv_bfloat16* __restrict__ v_mem, __nv_bfloat16* __restrict__ k_cache,
                     __nv_bfloat16* __restrict__ v_cache, __nv_bfloat16* __restrict__ o_mem, float* __restrict__ lse,
-                    float* __restrict__ ws, int BH, int cap, int mem_len, int t, int tc, int nprior, int prior_len,
-                    int mtiles, float scale_log2) {
+                    float* __restrict__ ws, int BH, int cap, int mem_len_all, const int32_t* __restrict__ mem_lens, int H,
+                    int t, int tc, int nprior, int prior_len, int mtiles, float scale_log2) {
     using SM = CmpSmem<D>;
     constexpr int ROWB = SM::ROWB;
     constexpr int VPR = D / 8;                 // 16-byte vectors per row
@@ -113,6 +113,14 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
     const int bs = blockIdx.x / mtiles;
     const int bh = bs / nsp, split = bs - bh * nsp;
     const bool is_tail = split == nprior;
+    // ragged batch (default variant only, nprior == 0): every sequence has its own count of memory entries, clamped
+    // to the bound the caller vouched for; a negative count means the sequence does not compress in this call
+    int mem_len = mem_len_all;
+    if (mem_lens) {
+        mem_len = __ldg(mem_lens + bh / H);
+        if (mem_len < 0) return;
+        mem_len = min(mem_len, mem_len_all);
+    }
     const int q0 = mt * 16;                    // first query row of this tile
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;
@@ -346,8 +354,13 @@ compress_merge_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ 
 template <int D>
 __global__ void compaction_kernel(const __nv_bfloat16* __restrict__ k_mem, const __nv_bfloat16* __restrict__ v_mem,
                                   __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache, int cap,
-                                  int mem_len, int t) {
+                                  int mem_len, const int32_t* __restrict__ mem_lens, int H, int t) {
     const int bh = blockIdx.x;
+    if (mem_lens) {
+        const int own = __ldg(mem_lens + bh / H);
+        if (own < 0) return;
+        mem_len = min(own, mem_len);
+    }
     constexpr int VPR = D / 8;
     const uint4* ksrc = reinterpret_cast<const uint4*>(k_mem + (int64_t)bh * t * D);
     const uint4* vsrc = reinterpret_cast<const uint4*>(v_mem + (int64_t)bh * t * D);
@@ -361,8 +374,8 @@ __global__ void compaction_kernel(const __nv_bfloat16* __restrict__ k_mem, const
 
 template <int D>
 static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* vm, void* kc, void* vc, void* om,
-                                   float* lse, int BH, int cap, int mem_len, int t, int tc, unsigned flags, float scale,
-                                   void* ws, cudaStream_t st) {
+                                   float* lse, int BH, int cap, int mem_len, const int32_t* mem_lens, int H, int t, int tc,
+                                   unsigned flags, float scale, void* ws, cudaStream_t st) {
     const int nprior = compress_num_prior(BH, mem_len, flags);
     int prior_len = 0;
     if (nprior > 0) prior_len = ((mem_len + nprior - 1) / nprior + 15) / 16 * 16;
@@ -381,8 +394,8 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
     compress_mma_kernel<D><<<BH * nsp * mtiles, CMP_WARPS * 32, smem, st>>>(
         static_cast<const __nv_bfloat16*>(qm), static_cast<const __nv_bfloat16*>(km),
         static_cast<const __nv_bfloat16*>(vm), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
-        static_cast<__nv_bfloat16*>(om), lse, static_cast<float*>(ws), BH, cap, mem_len, t, tc, nprior, prior_len,
-        mtiles, scale * 1.4426950408889634f);
+        static_cast<__nv_bfloat16*>(om), lse, static_cast<float*>(ws), BH, cap, mem_len, mem_lens, H, t, tc, nprior,
+        prior_len, mtiles, scale * 1.4426950408889634f);
     count_launches(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -396,7 +409,7 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
     if (mtiles > 1) {
         compaction_kernel<D><<<BH, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(km),
                                                   static_cast<const __nv_bfloat16*>(vm), static_cast<__nv_bfloat16*>(kc),
-                                                  static_cast<__nv_bfloat16*>(vc), cap, mem_len, t);
+                                                  static_cast<__nv_bfloat16*>(vc), cap, mem_len, mem_lens, H, t);
         count_launches(1);
         e = cudaGetLastError();
     }
@@ -405,13 +418,14 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
 
 // t <= 128; the caller falls back to the CUDA-core kernel otherwise.
 cudaError_t launch_compress_bf16(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
-                                 void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len, int c, int t,
-                                 unsigned flags, float scale, void* ws, cudaStream_t st) {
+                                 void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len,
+                                 const int32_t* mem_lens, int c, int t, unsigned flags, float scale, void* ws,
+                                 cudaStream_t st) {
     const int BH = B * H, tc = c * t;
-    return D == 64 ? compress_bf16_t<64>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH, cap, mem_len, t, tc,
-                                         flags, scale, ws, st)
-                   : compress_bf16_t<128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH, cap, mem_len, t, tc,
-                                          flags, scale, ws, st);
+    return D == 64 ? compress_bf16_t<64>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH, cap, mem_len, mem_lens, H, t,
+                                         tc, flags, scale, ws, st)
+                   : compress_bf16_t<128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH, cap, mem_len, mem_lens, H, t,
+                                          tc, flags, scale, ws, st);
 }
 
 }  // namespace loma

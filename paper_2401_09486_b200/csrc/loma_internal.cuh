@@ -116,12 +116,13 @@ cudaError_t launch_decode_bf16_static(const void* q, const void* k_new, const vo
 // bf16 compress step on warp-level tensor cores (compress_mma.cu); t <= 16
 size_t compress_workspace_bytes(int BH, int D, int t, int mem_len, unsigned flags);
 cudaError_t launch_compress_bf16(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
-                                 void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len, int c, int t,
-                                 unsigned flags, float scale, void* ws, cudaStream_t st);
+                                 void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len,
+                                 const int32_t* mem_lens, int c, int t, unsigned flags, float scale, void* ws,
+                                 cudaStream_t st);   // mem_lens: per-sequence counts (default variant only) or NULL
 
 cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const void* v_mem,
                                     void* k_cache, void* v_cache, void* o_mem, float* lse,
-                                    int B, int H, int D, int cap, int mem_len, int c, int t,
+                                    int B, int H, int D, int cap, int mem_len, const int32_t* mem_lens, int c, int t,
                                     loma_dtype dt, float scale, unsigned flags, cudaStream_t st);
 
 // rotary embedding of Q and K rows at the layout's position ids (rope.cu)

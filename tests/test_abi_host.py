@@ -256,3 +256,17 @@ def test_ragged_decode_validation(lib):
     assert call(lens=0x7002) == ALIGNMENT
     assert call(D=100) == UNSUPPORTED
     assert call(B=0) == 0
+
+
+def test_ragged_compress_validation(lib):
+    def call(qm=0x1000, km=0x2000, vm=0x3000, kc=0x4000, vc=0x5000, om=0x6000, B=2, H=1, D=128, cap=100, lens=0x7000,
+             mx=16, c=4, t=16, tc=64, dt=1, flags=0):
+        return lib.loma_compress_step_ragged(qm, km, vm, kc, vc, om, None, B, H, D, cap, lens, mx, c, t, tc, dt, 0.0, flags,
+                                             None)
+    assert call(cap=79) == CAPACITY
+    assert call(tc=63) == INVALID
+    assert call(lens=None) == INVALID
+    assert call(lens=0x7001) == ALIGNMENT
+    assert call(flags=1) == UNSUPPORTED                 # prior-memory variant is not offered ragged
+    assert call(D=32) == UNSUPPORTED
+    assert call(B=0) == 0

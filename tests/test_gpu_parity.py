@@ -342,6 +342,35 @@ def test_compress_matches_oracle_and_compacts_bit_exact(B, H, D, c, t, mem_len, 
 
 # ------------------------------------------------------- failure detection
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, GENERIC])
+@pytest.mark.parametrize("H,D,c,t,lens", [(2, 64, 4, 4, [0, 16, -1, 8]), (2, 128, 4, 16, [48, -1, 1024, 0, 512]),
+                                          (1, 128, 2, 64, [128, 64, -1]), (2, 128, 8, 16, [8192, 4096, -1, 16])])
+def test_ragged_compress_matches_oracle_and_leaves_idle_sequences_alone(H, D, c, t, lens, flags, dtype):
+    B, tc = len(lens), c * t
+    max_len = max(lens)
+    cap = max_len + tc + 3
+    kc = synthetic.normal_tensor((B, H, cap, D), 41, 1.0, dtype)
+    vc = synthetic.normal_tensor((B, H, cap, D), 42, 1.0, dtype)
+    qm, km, vm = synthetic.qkv(B, H, t, D, seed=43, std=1.0, dtype=dtype)
+    want_o, want_lse, want_k, want_v = oracle.compress_step_ragged(npf(qm), npf(km), npf(vm), npf(kc), npf(vc), lens, c, t)
+    kcd, vcd = kc.to(DEV), vc.to(DEV)
+    om = torch.full((B, H, t, D), 7.0, dtype=dtype, device=DEV)
+    lse = torch.full((B, H, t), 7.0, dtype=torch.float32, device=DEV)
+    lens_d = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    L.loma_compress_step_ragged(qm.to(DEV), km.to(DEV), vm.to(DEV), kcd, vcd, om, lse, lens_d, max_len, c, t, flags)
+    torch.cuda.synchronize()
+    for b, n in enumerate(lens):
+        if n < 0:
+            assert float((om[b].float() - 7.0).abs().max()) == 0.0 and float((lse[b] - 7.0).abs().max()) == 0.0
+            assert torch.equal(kcd[b].cpu(), kc[b]) and torch.equal(vcd[b].cpu(), vc[b])
+            continue
+        check_close(om[b:b + 1], want_o[b:b + 1], dtype)
+        assert np.abs(npf(lse[b]) - want_lse[b]).max() <= (1e-5 if dtype == torch.float32 else 2e-2)
+        assert np.array_equal(npf(kcd[b, :, :n + t]), want_k[b, :, :n + t]) and np.array_equal(npf(vcd[b, :, :n + t]), want_v[b, :, :n + t])
+        assert torch.equal(kcd[b, :, n + t:].cpu(), kc[b, :, n + t:])      # slots beyond the rewritten ones keep their contents
+
+
 def test_bounded_wait_times_out_and_leaves_the_context_usable():
     """A device-side wait that can never be satisfied gives up after its limit,
     reports LOMA_ERR_TIMEOUT through the status word, and later launches work."""

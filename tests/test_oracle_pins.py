@@ -611,3 +611,22 @@ def test_ragged_decode_is_per_sequence_decode():
         assert np.array_equal(k_r[b, :, n], kn[b, :, 0]) and np.array_equal(v_r[b, :, n], vn[b, :, 0])
         keep = np.ones(cap, bool); keep[n] = False
         assert np.array_equal(k_r[b][:, keep], kc[b][:, keep])
+
+
+def test_ragged_compress_is_per_sequence_compress():
+    B, H, D, c, t, cap = 3, 2, 8, 2, 2, 20
+    tc = c * t
+    kc, vc = _rand((B, H, cap, D), 80), _rand((B, H, cap, D), 81)
+    qm, km, vm = _rand((B, H, t, D), 82), _rand((B, H, t, D), 83), _rand((B, H, t, D), 84)
+    o_u, l_u, k_u, v_u = oracle.compress_step(qm, km, vm, kc, vc, 6, c, t)
+    o_r, l_r, k_r, v_r = oracle.compress_step_ragged(qm, km, vm, kc, vc, [6, 6, 6], c, t)
+    assert np.array_equal(o_u, o_r) and np.array_equal(l_u, l_r)
+    assert np.array_equal(k_r[:, :, :6 + t], k_u) and np.array_equal(v_r[:, :, :6 + t], v_u)
+    lens = [0, -1, 10]
+    o_r, _, k_r, v_r = oracle.compress_step_ragged(qm, km, vm, kc, vc, lens, c, t)
+    assert np.isnan(o_r[1]).all() and np.array_equal(k_r[1], kc[1]) and np.array_equal(v_r[1], vc[1])
+    for b in (0, 2):
+        n = lens[b]
+        ob, _, kb, _ = oracle.compress_step(qm[b:b + 1], km[b:b + 1], vm[b:b + 1], kc[b:b + 1], vc[b:b + 1], n, c, t)
+        assert np.array_equal(o_r[b], ob[0]) and np.array_equal(k_r[b, :, :n + t], kb[0])
+        assert np.array_equal(k_r[b, :, n + t:], kc[b, :, n + t:])        # nothing beyond the new length is touched
