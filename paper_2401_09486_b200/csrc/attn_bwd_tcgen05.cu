@@ -21,8 +21,8 @@
 // dV += P^T dO_h and dK += dA^T Q_h with Q_h, dO_h as MN-major operands.
 //
 // Roles: warps 0-7 two warpgroups (each takes half of the columns of every event, and half of the
-// epilogue), warp 8 TMA producer (one lane), warp 9 MMA issuer (warp-uniform
-// control flow, one elected lane issues).  Every mbarrier wait is bounded; on expiry the CTA
+// epilogue), warp 8 TMA producer (one lane), warps 9 and 10 MMA issuers (warp-uniform control flow, one
+// elected lane issues; warp 9 the score products, warp 10 the accumulating products).  Every mbarrier wait is bounded; on expiry the CTA
 // records LOMA_ERR_TIMEOUT, every role leaves its loop, TMEM is freed and the kernel returns.
 #include "tcgen05_common.cuh"
 
@@ -39,8 +39,7 @@ struct BwdParams {
     float scale;
 };
 
-constexpr int BWD_THREADS = 320;      // dK/dV kernel: two warpgroups, one TMA warp, one MMA warp
-constexpr int BWD_DQ_THREADS = 352;   // dQ kernel: one more MMA warp
+constexpr int BWD_THREADS = 352;   // two warpgroups, one TMA warp, two MMA warps
 constexpr int BWD_NBAR = 13;
 
 template <int D>
@@ -80,7 +79,7 @@ bwd_delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __res
 
 // ------------------------------------------------------------------ dQ
 template <int D>
-__global__ void __launch_bounds__(BWD_DQ_THREADS, 1)
+__global__ void __launch_bounds__(BWD_THREADS, 1)
 masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdParams bp) {
     using SM = BwdDqSmem<D>;
     constexpr int PANELS = SM::PANELS;
@@ -103,7 +102,7 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // zero the operand buffers once: rows a TMA box does not cover keep finite contents
-    for (int i = threadIdx.x; i < SM::TOTAL / 16; i += BWD_DQ_THREADS) reinterpret_cast<uint4*>(smem_gen)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = threadIdx.x; i < SM::TOTAL / 16; i += BWD_THREADS) reinterpret_cast<uint4*>(smem_gen)[i] = make_uint4(0, 0, 0, 0);
     fence_async_smem();
     if (warp == 9) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(512)
@@ -414,7 +413,7 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
 
-    enum { B_KVF = 0, B_DONE = 1, B_QGF = 2, B_QGE = 4, B_SF = 6, B_PF = 8 };
+    enum { B_KVF = 0, B_DONE = 1, B_QGF = 2, B_QGE = 4, B_SF = 6, B_PF = 8, B_DA = 10 };
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
 
     if (threadIdx.x == 0) {
@@ -482,87 +481,87 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
             }
         }
     } else if (warp == 9) {
-        // ------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------ MMA issuer A: the score products
+        // (two issuing warps, as in the dQ kernel: this one S^T and dP^T, warp 10 the dV and dK accumulation)
         constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-        constexpr uint32_t IDESC_ACC =
-            (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
-        uint32_t gs = 0, tcount = 0, ge_s = 0, ge_p = 0;
+        uint32_t gs = 0, tcount = 0, ge = 0;
         bool ok = true;
         const uint64_t kd_ = smem_desc(smem_base + K_OFF, 16, 1024);
         const uint64_t vd_ = smem_desc(smem_base + V_OFF, 16, 1024);
-        // S^T = K Q_h^T and dP^T = V dO_h^T for query rows [64h, 64h+64) of the staged tiles -> buffers b
-        auto issue_st = [&](int b, int h, int stage) {
-            if (elect_one()) {
-                const uint64_t qd = smem_desc(smem_base + ring_off(stage), 16, 1024);
-                const uint64_t gd = smem_desc(smem_base + ring_off(stage) + SM::TILE_BYTES, 16, 1024);
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint64_t off = (uint64_t)(((kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32) >> 4);
-                    mma_ss(tmem + b * 64, kd_ + off, qd + off + (uint64_t)((h * 8192) >> 4), IDESC_S, kk > 0);
-                }
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint64_t off = (uint64_t)(((kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32) >> 4);
-                    mma_ss(tmem + 128 + b * 64, vd_ + off, gd + off + (uint64_t)((h * 8192) >> 4), IDESC_S, kk > 0);
-                }
-                tc_commit(bar(B_SF + b));
-            }
-            __syncwarp();
-        };
-        // dV += P^T dO_h and dK += dA^T Q_h: P^T and dA^T (bf16) read from TMEM, dO_h and Q_h as MN-major operands
-        auto issue_acc = [&](int b, int h, int stage, bool first, bool last_of_step, bool last_of_tile) {
-            if (elect_one()) {
-                const uint64_t qmn = smem_desc(smem_base + ring_off(stage), SM::PANEL_BYTES, 1024);
-                const uint64_t gmn = smem_desc(smem_base + ring_off(stage) + SM::TILE_BYTES, SM::PANEL_BYTES, 1024);
-#pragma unroll
-                for (int k4 = 0; k4 < 4; ++k4)
-                    mma_ts(tmem + 384, tmem + b * 64 + (k4 >> 1) * 32 + (k4 & 1) * 8, gmn + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_ACC,
-                           !first || (k4 > 0));
-#pragma unroll
-                for (int k4 = 0; k4 < 4; ++k4)
-                    mma_ts(tmem + 256, tmem + 128 + b * 64 + (k4 >> 1) * 32 + (k4 & 1) * 8, qmn + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_ACC,
-                           !first || (k4 > 0));
-                if (last_of_step) tc_commit(bar(B_QGE + stage));
-                if (last_of_tile) tc_commit(bar(B_DONE));
-            }
-            __syncwarp();
-        };
         for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
             const int rank = fdiv(w, p.dBH);
             KeyTileDesc kd;
             decode_key_tile(p, rank, kd);
             const HalfMasks hm = key_tile_half_masks(p, kd, lane);
             const int nsteps = kd.nsteps;
-            HalfWalk sw, pw;
-            sw.start(hm);
-            pw.start(hm);
             ok = __all_sync(0xffffffffu, mbar_wait(bar(B_KVF), tcount & 1, abortp, p.status));
-            if (!ok) break;
-            auto next_scores = [&]() {
+            HalfWalk sw;
+            for (sw.start(hm); ok && !sw.done(nsteps); sw.next(hm), ++ge) {
                 const uint32_t step = gs + sw.j;
-                if (sw.first_of_step(hm)) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_QGF + (step & 1)), (step >> 1) & 1, abortp, p.status));
-                    if (!ok) return;
-                }
-                tc_fence_after();
-                issue_st(ge_s & 1, sw.h, step & 1);
-                ++ge_s;
-                sw.next(hm);
-            };
-            next_scores();
-            if (ok && !sw.done(nsteps)) next_scores();
-            bool first = true;
-            while (ok && !pw.done(nsteps)) {
-                const int b = ge_p & 1;
-                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_PF + b), (ge_p >> 1) & 1, abortp, p.status));
+                const int b = ge & 1, h = sw.h, stage = step & 1;
+                if (sw.first_of_step(hm))
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_QGF + stage), (step >> 1) & 1, abortp, p.status));
+                // buffers b are free once the accumulation of event ge - 2 has read P^T and dA^T out of them
+                if (ok && ge >= 2) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_DA + b), ((ge - 2) >> 1) & 1, abortp, p.status));
                 if (!ok) break;
                 tc_fence_after();
-                const bool los = pw.last_of_step(hm);
-                issue_acc(b, pw.h, (gs + pw.j) & 1, first, los, los && pw.j == nsteps - 1);
-                first = false;
-                ++ge_p;
-                if (!sw.done(nsteps)) next_scores();
-                pw.next(hm);
+                // S^T = K Q_h^T and dP^T = V dO_h^T for query rows [64h, 64h+64) of the staged tiles -> buffers b
+                if (elect_one()) {
+                    const uint64_t qd = smem_desc(smem_base + ring_off(stage), 16, 1024);
+                    const uint64_t gd = smem_desc(smem_base + ring_off(stage) + SM::TILE_BYTES, 16, 1024);
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint64_t off = (uint64_t)(((kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32) >> 4);
+                        mma_ss(tmem + b * 64, kd_ + off, qd + off + (uint64_t)((h * 8192) >> 4), IDESC_S, kk > 0);
+                    }
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint64_t off = (uint64_t)(((kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32) >> 4);
+                        mma_ss(tmem + 128 + b * 64, vd_ + off, gd + off + (uint64_t)((h * 8192) >> 4), IDESC_S, kk > 0);
+                    }
+                    tc_commit(bar(B_SF + b));
+                }
+                __syncwarp();
+            }
+            gs += kd.nsteps;
+        }
+    } else if (warp == 10) {
+        // ------------------------------------------------------------ MMA issuer B: the dV and dK accumulation
+        constexpr uint32_t IDESC_ACC =
+            (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
+        uint32_t gs = 0, ge = 0;
+        bool ok = true;
+        for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r)) {
+            const int rank = fdiv(w, p.dBH);
+            KeyTileDesc kd;
+            decode_key_tile(p, rank, kd);
+            const HalfMasks hm = key_tile_half_masks(p, kd, lane);
+            const int nsteps = kd.nsteps;
+            bool first = true;
+            HalfWalk pw;
+            for (pw.start(hm); ok && !pw.done(nsteps); pw.next(hm), ++ge, first = false) {
+                const int b = ge & 1, h = pw.h, stage = (gs + pw.j) & 1;
+                const bool los = pw.last_of_step(hm), lot = los && pw.j == nsteps - 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_PF + b), (ge >> 1) & 1, abortp, p.status));
+                if (!ok) break;
+                tc_fence_after();
+                // dV += P^T dO_h and dK += dA^T Q_h: P^T and dA^T (bf16) read from TMEM, dO_h and Q_h as MN-major operands
+                if (elect_one()) {
+                    const uint64_t qmn = smem_desc(smem_base + ring_off(stage), SM::PANEL_BYTES, 1024);
+                    const uint64_t gmn = smem_desc(smem_base + ring_off(stage) + SM::TILE_BYTES, SM::PANEL_BYTES, 1024);
+#pragma unroll
+                    for (int k4 = 0; k4 < 4; ++k4)
+                        mma_ts(tmem + 384, tmem + b * 64 + (k4 >> 1) * 32 + (k4 & 1) * 8, gmn + (uint64_t)(((h * 4 + k4) * 2048) >> 4),
+                               IDESC_ACC, !first || (k4 > 0));
+#pragma unroll
+                    for (int k4 = 0; k4 < 4; ++k4)
+                        mma_ts(tmem + 256, tmem + 128 + b * 64 + (k4 >> 1) * 32 + (k4 & 1) * 8,
+                               qmn + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_ACC, !first || (k4 > 0));
+                    tc_commit(bar(B_DA + b));
+                    if (los) tc_commit(bar(B_QGE + stage));
+                    if (lot) tc_commit(bar(B_DONE));
+                }
+                __syncwarp();
             }
             gs += kd.nsteps;
         }
@@ -802,9 +801,9 @@ cudaError_t launch_masked_attn_bwd_dq_tc(const void* q, const void* k, const voi
     const int64_t work = (int64_t)bp.f.total_tiles * bp.f.BH;
     const int grid = (int)(work < sms ? work : sms);
     if (D == 128)
-        masked_attn_bwd_dq_tc_kernel<128><<<grid, BWD_DQ_THREADS, BwdDqSmem<128>::TOTAL + 1024, st>>>(maps, bp);
+        masked_attn_bwd_dq_tc_kernel<128><<<grid, BWD_THREADS, BwdDqSmem<128>::TOTAL + 1024, st>>>(maps, bp);
     else
-        masked_attn_bwd_dq_tc_kernel<64><<<grid, BWD_DQ_THREADS, BwdDqSmem<64>::TOTAL + 1024, st>>>(maps, bp);
+        masked_attn_bwd_dq_tc_kernel<64><<<grid, BWD_THREADS, BwdDqSmem<64>::TOTAL + 1024, st>>>(maps, bp);
     count_launches(2);
     return cudaGetLastError();
 }
