@@ -239,39 +239,45 @@ __host__ __device__ __forceinline__ void decode_key_tile(const FwdParams& p, int
     const View& vm = p.view[V_MEM];
     const View& vr = p.view[V_READ];
     const View& vp = p.view[V_REP];
-    int ns = 0;
-    auto add = [&](int v, int mode, int first, int count) {
-        if (count > 0) kd.seg[ns++] = Seg{v, mode, first, count};
-    };
+    // four fixed slots (an absent run has count 0), written with compile-time indices so that they stay in registers
+    const Seg none = Seg{view, M_EQ, 0, 0};
+    kd.seg[0] = kd.seg[1] = kd.seg[2] = kd.seg[3] = none;
+    auto run = [](int v, int mode, int first, int count) { return Seg{v, mode, first, count > 0 ? count : 0}; };
     if (view == V_MEM) {
         // reading rows of every later chunk and of the tail (Eq. 3)
-        if (kd.a0 + 1 < p.n_chunks) { const int f = tile_of_chunk(vr, kd.a0 + 1); add(V_READ, M_LT, f, p.n_read - f); }
-        add(V_TAIL, M_LT, 0, p.n_tail);
+        if (kd.a0 + 1 < p.n_chunks) { const int f = tile_of_chunk(vr, kd.a0 + 1); kd.seg[0] = run(V_READ, M_LT, f, p.n_read - f); }
+        kd.seg[1] = run(V_TAIL, M_LT, 0, p.n_tail);
         // memory rows: own chunk (Eq. 1, row 2); with the prior-memory flag every later chunk too
         const int f = (g.Z >= 128) ? kd.c0 * g.tpc : ki;
-        if (p.flags & LOMA_FLAG_MEM_SEES_PRIOR_MEM) add(V_MEM, M_LE, f, p.n_mem - f);
-        else add(V_MEM, M_EQ, f, (g.Z >= 128) ? g.tpc : 1);
+        if (p.flags & LOMA_FLAG_MEM_SEES_PRIOR_MEM) kd.seg[2] = run(V_MEM, M_LE, f, p.n_mem - f);
+        else kd.seg[2] = run(V_MEM, M_EQ, f, (g.Z >= 128) ? g.tpc : 1);
         // repetition rows of the same chunks (Eq. 1, row 3)
-        if (p.n_rep > 0) { const int fr = tile_of_chunk(vp, kd.a0); add(V_REP, M_EQ, fr, last_tile_of_chunk(vp, kd.a1) - fr + 1); }
+        if (p.n_rep > 0) { const int fr = tile_of_chunk(vp, kd.a0); kd.seg[3] = run(V_REP, M_EQ, fr, last_tile_of_chunk(vp, kd.a1) - fr + 1); }
     } else if (view == V_READ) {
-        add(V_READ, M_CAUSAL, ki, (g.Z >= 128) ? (kd.c0 + 1) * g.tpc - ki : 1);
+        kd.seg[0] = run(V_READ, M_CAUSAL, ki, (g.Z >= 128) ? (kd.c0 + 1) * g.tpc - ki : 1);
         const int fm = tile_of_chunk(vm, kd.a0);
-        add(V_MEM, M_EQ, fm, last_tile_of_chunk(vm, kd.a1) - fm + 1);
+        kd.seg[1] = run(V_MEM, M_EQ, fm, last_tile_of_chunk(vm, kd.a1) - fm + 1);
     } else if (view == V_TAIL) {
-        add(V_TAIL, M_CAUSAL, ki, p.n_tail - ki);
+        kd.seg[0] = run(V_TAIL, M_CAUSAL, ki, p.n_tail - ki);
     } else {
-        add(V_REP, M_DIAG, ki, 1);
+        kd.seg[0] = run(V_REP, M_DIAG, ki, 1);
     }
-    kd.nseg = ns;
-    kd.nsteps = 0;
-    for (int i = 0; i < ns; ++i) kd.nsteps += kd.seg[i].count;
+    kd.nseg = 4;
+    kd.nsteps = kd.seg[0].count + kd.seg[1].count + kd.seg[2].count + kd.seg[3].count;
 }
 
 __host__ __device__ __forceinline__ void step_qtile(const FwdParams& p, const KeyTileDesc& kd, int j, QTile& qt) {
-    int i = 0;
-    while (i + 1 < kd.nseg && j >= kd.seg[i].count) { j -= kd.seg[i].count; ++i; }
-    qt.view = kd.seg[i].view; qt.mode = kd.seg[i].mode;
-    tile_geometry(p.view[qt.view], kd.seg[i].first + j, qt.c0, qt.r0, qt.a0, qt.a1);
+    // the run that holds step j (compile-time indices; runs with count 0 are stepped over)
+    Seg sg = kd.seg[0];
+#pragma unroll
+    for (int i = 0; i < 3; ++i) {
+        if (j >= sg.count) {
+            j -= sg.count;
+            sg = kd.seg[i + 1];
+        }
+    }
+    qt.view = sg.view; qt.mode = sg.mode;
+    tile_geometry(p.view[qt.view], sg.first + j, qt.c0, qt.r0, qt.a0, qt.a1);
 }
 
 // Rows of a query tile that hold a row of the sequence: always a prefix [0, n).
