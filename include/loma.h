@@ -2,11 +2,18 @@
  * loma.h -- C ABI of the LoMA (Lossless Compressed Memory Attention,
  * arxiv 2401.09486) attention hot path for NVIDIA B200 (sm_100a).
  *
- * Three device operations and two integer index maps:
+ * The device operations and the two integer index maps:
  *
  *   loma_masked_attn_fwd   zone-masked attention over the training layout
- *   loma_masked_attn_bwd   its gradients with respect to q, k and v
  *                          (Section 4.3, Eq. 1-3; Section 4.4, Eq. 5-7)
+ *   loma_masked_attn_bwd   its gradients with respect to q, k and v
+ *                          (Section 4.4, the paths to Eq. 10)
+ *   loma_rope_apply        rotary embedding of q and k at the position ids of
+ *                          Section 4.5 (Eq. 14)
+ *   loma_prefill_cache     the cache a one-pass prompt prefill leaves behind
+ *   loma_decode_attn_ragged, loma_compress_step_ragged
+ *                          the two generation steps for batches whose sequences
+ *                          stand at different points of their chunks
  *   loma_decode_attn       one generated token over the compressed cache
  *                          (Section 3.1 steps 1 and 3; Appendix A, inference_input)
  *   loma_compress_step     the t <m> queries over the uncompressed tail, fused
