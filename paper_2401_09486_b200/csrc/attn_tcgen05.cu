@@ -38,9 +38,9 @@
 //                     O += P_h V_h with P read from TMEM and V as an MN-major shared operand.
 //                     S_h of the next step is issued right after P_h V_h of this one, so the
 //                     tensor pipe works on one half while the warpgroup works on the other.
-// The two streams fill each other's waits (tensor latency, TMEM loads, epilogues).  Tiles are dealt
-// to the 2*gridDim.x streams round robin from a statically ordered list (longest first, (batch,
-// head) fastest).  Every mbarrier wait is bounded: on expiry the CTA records LOMA_ERR_TIMEOUT, all
+// The two streams fill each other's waits (tensor latency, TMEM loads, epilogues).  Tiles are handed
+// out at run time from one counter over a statically ordered list (longest first, (batch, head)
+// fastest): a stream that finishes a tile draws the next.  Every mbarrier wait is bounded: on expiry the CTA records LOMA_ERR_TIMEOUT, all
 // roles leave their loops, TMEM is freed and the kernel returns.
 #include "tcgen05_common.cuh"
 
@@ -53,7 +53,7 @@ struct TmaMaps {
 // ------------------------------------------------------------------ the kernel
 constexpr int TC_THREADS = 384;   // 2 softmax warpgroups + 1 warpgroup with 2 TMA warps and 2 MMA warps
 constexpr int TMEM_COLS = 512;
-constexpr int NBAR = 12;          // mbarriers per stream
+constexpr int NBAR = 14;          // mbarriers per stream
 
 // Shared memory of one stream: Q tile, one K tile, one V tile, and a 64-column output staging panel.
 template <int D>
@@ -78,6 +78,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     __shared__ __align__(8) uint64_t bars[2 * NBAR];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ int tile_ring_s[2][4];
 
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
     // which of the CTA's two independent streams this warp serves
@@ -87,7 +88,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     const uint32_t smem_base = smem_base0 + st * SM::STREAM_BYTES;
     uint8_t* smem_gen = smem_gen0 + st * SM::STREAM_BYTES;
 
-    enum { B_QF = 0, B_QE = 1, B_KF = 2, B_KE = 3, B_VF = 4, B_VE = 5, B_SF = 6, B_PF = 8, B_OF = 10 };
+    enum { B_QF = 0, B_QE = 1, B_KF = 2, B_KE = 3, B_VF = 4, B_VE = 5, B_SF = 6, B_PF = 8, B_OF = 10, B_TF = 12 };
     auto bar = [&](int i) { return smem_u32(&bars[st * NBAR + i]); };
 
     if (threadIdx.x == 0) {
@@ -114,10 +115,17 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
 
     // Tiles (longest first) are dealt to the 2*gridDim.x streams in rounds, forwards in even rounds
     // and backwards in odd ones, so no stream always receives the longest tile of a round.
+    // Tiles are handed out from one counter, longest first ((batch, head) fastest inside a rank): a stream
+    // that finishes early simply takes the next one.  The stream's producer draws the number and posts it
+    // in a four-slot ring (barrier B_TF + (n & 1), completion n >> 1, for the stream's n-th tile); the MMA
+    // issuer and the warpgroup read it there.  A negative number ends the stream.  Which stream computes a
+    // tile has no influence on the tile's result.
     const int total_work = p.total_tiles * p.BH;
-    const int nstreams = 2 * gridDim.x;
-    const int sid = blockIdx.x + st * gridDim.x;
-    auto tile_of_round = [&](int r) { return r * nstreams + ((r & 1) ? nstreams - 1 - sid : sid); };
+    volatile int* tile_ring = tile_ring_s[st];
+    auto next_tile = [&](uint32_t n, bool& ok_) -> int {   // called by whole warps
+        ok_ = __all_sync(0xffffffffu, mbar_wait(bar(B_TF + (n & 1)), (n >> 1) & 1, abortp, p.status));
+        return ok_ ? tile_ring[n & 3] : -1;
+    };
 
     if (warp == 8 || warp == 9) {
         // ------------------------------------------------------------ TMA producer of stream st
@@ -125,7 +133,14 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         if (lane == 0) {
             uint32_t gs = 0, tcount = 0;
             bool ok = true;
-            for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
+            for (;; ++tcount) {
+                // draw the stream's next tile and post it (a number past the end tells the other roles to stop)
+                int w = (int)atomicAdd(p.sched, 1u);
+                if (w >= total_work || !ok) w = -1;
+                tile_ring[tcount & 3] = w;
+                __threadfence_block();
+                mbar_arrive(bar(B_TF + (tcount & 1)));
+                if (w < 0) break;
                 const int rank = fdiv(w, p.dBH), bh = w - rank * p.BH;
                 const int bi = fdiv(bh, p.dH), hi = bh - bi * p.H;
                 TileDesc td;
@@ -208,7 +223,9 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 __syncwarp();
             };
             uint32_t ge_s = 0, ge_p = 0;   // events whose scores / whose P.V have been issued
-            for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
+            for (;; ++tcount) {
+                const int w = next_tile(tcount, ok);
+                if (w < 0) break;
                 const int rank = fdiv(w, p.dBH);
                 TileDesc td;
                 decode_tile(p, rank, td);
@@ -283,8 +300,10 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             c.hm = tile_half_masks(p, c.td, lane);
         };
         TileCtx cur, nxt;
-        if (sid < total_work) decode_ctx(sid, cur);
-        for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), cur = nxt) {
+        uint32_t tcount = 0;
+        int w_cur = next_tile(0, ok), w_next = -1;
+        if (w_cur >= 0) decode_ctx(w_cur, cur);
+        for (; w_cur >= 0 && ok; w_cur = w_next, cur = nxt, ++tcount) {
             const TileDesc& td = cur.td;
             const HalfMasks hm = cur.hm;
             const int bh = cur.bh, bi = cur.bi, hi = cur.hi, ro = cur.ro, rc = cur.rc;
@@ -384,8 +403,10 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 }
             }
             {
-                const int wn = tile_of_round(r + 1);
-                if (wn < total_work) decode_ctx(wn, nxt);
+                bool got = true;
+                w_next = next_tile(tcount + 1, got);
+                if (!got) ok = false;
+                if (w_next >= 0) decode_ctx(w_next, nxt);
             }
             // the last P.V of the tile belongs to event ge - 1 (products complete in issue order)
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + ((ge - 1) & 1)), ((ge - 1) >> 1) & 1, abortp, p.status));
@@ -451,6 +472,15 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_slot), "r"(TMEM_COLS) : "memory");
     }
+    // the last CTA to leave puts the scheduler's counters back to zero for the next launch that uses them
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(p.sched + 1, 1u) == gridDim.x - 1) {
+            p.sched[0] = 0;
+            p.sched[1] = 0;
+            __threadfence();
+        }
+    }
 }
 
 // ------------------------------------------------------------------ bounded-wait self test
@@ -484,6 +514,23 @@ cudaError_t launch_bounded_wait_selftest(cudaStream_t st) {
 }
 
 // ------------------------------------------------------------------ host side
+// Tile counters of the in-kernel scheduler: 64 pairs (next tile, CTAs finished), handed to launches round robin
+// and cleared by the last CTA of the launch that used them.  512 bytes per device, zero at load.
+static __device__ unsigned g_sched_counters[64][2];
+
+static unsigned* sched_counters() {
+    static unsigned* base[64] = {nullptr};
+    static std::atomic<unsigned> seq{0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!base[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_sched_counters) != cudaSuccess) return nullptr;
+        base[dev] = static_cast<unsigned*>(ptr);
+    }
+    return base[dev] + 2 * (seq.fetch_add(1) % 64);
+}
+
 struct MapCacheKey {
     const void *q, *k, *v, *o;
     int B, H, D, n, c, t, tail;
@@ -507,7 +554,9 @@ cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, v
     p.lse = lse;
     p.status = device_status_word();
     if (!p.status) return cudaErrorUnknown;
-    if ((int64_t)p.total_tiles * p.BH > 0x7fffffffll) return cudaErrorNotSupported;
+    if ((int64_t)p.total_tiles * p.BH > 0x7ffffff0ll - 2 * 148) return cudaErrorNotSupported;
+    p.sched = sched_counters();
+    if (!p.sched) return cudaErrorUnknown;
 
     // tensor maps, cached for repeated calls on the same tensors
     static std::mutex mu;

@@ -7,6 +7,7 @@
 #include <cuda.h>
 #include <math.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "loma_internal.cuh"

@@ -63,6 +63,7 @@ struct FwdParams {
     float scale_log2;
     float* lse;
     int* status;
+    unsigned* sched;   // [0] next tile to hand out, [1] CTAs that have finished (the last one clears both)
 };
 
 
