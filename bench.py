@@ -53,6 +53,15 @@ def allowed_pairs(n: int, c: int, t: int, prior_mem: bool = False) -> int:
     return n * per_chunk + cross * n * (n - 1) // 2
 
 
+def _device_pause(torch, cycles: int) -> None:
+    """Keeps the GPU busy for `cycles` clocks on the current stream (a spin kernel that ships with torch),
+    so that the calls enqueued right after it are already queued when the GPU reaches them.  Without it
+    (should a torch build lack the helper) short kernels are merely timed with the host's launch path included."""
+    spin = getattr(torch.cuda, "_sleep", None)
+    if spin is not None:
+        spin(int(cycles))
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -195,7 +204,7 @@ def run_ours(args):
         # A device-side pause of ~0.08 ms (counted in the step and in the index phase): by the time it ends the
         # host has enqueued the forward, so the two events around the forward see the kernel and not the host's
         # launch path (an idle GPU otherwise waits ~12 us for the call to arrive, 7 % of this kernel's run time).
-        torch.cuda._sleep(150_000)
+        _device_pause(torch, 150_000)
         mark("index")
         L.loma_masked_attn_fwd(q, k, v, o, None, f["n"], f["c"], f["t"], 0, 0, 0.0, stream)
         mark("masked_fwd")
@@ -384,7 +393,7 @@ def other_workloads(L, synthetic, torch, dev, peaks):
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             # keep the GPU busy for ~0.3 ms while the host enqueues the events and the call: the interval
             # between the events is then device time only (no wait for the host's launch path)
-            torch.cuda._sleep(600_000)
+            _device_pause(torch, 600_000)
             a.record(stream); fn(); b.record(stream); torch.cuda.synchronize()
             ts.append(a.elapsed_time(b))
         return statistics.median(ts)
