@@ -443,6 +443,20 @@ def other_workloads(L, synthetic, torch, dev, peaks):
                         "frac_of_measured_hbm": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "kernel": "rope_kernel"}
     del q, k, v, o
     torch.cuda.empty_cache()
+    # the compression settings of the paper's Table 1 / Fig. 7 sweeps (c = 2, short memory zones), ~4600 tokens
+    for (n2, c2, t2) in ((230, 2, 4), (115, 2, 8), (29, 2, 32)):
+        B, H = 4, 32
+        S = n2 * (2 * c2 * t2 + t2)
+        q, k, v = (synthetic.big_normal_(torch.empty(B, H, S, D, dtype=bf, device=dev), 3070 + i, std) for i in range(3))
+        o = torch.empty_like(q)
+        ms = timed(lambda: L.loma_masked_attn_fwd(q, k, v, o, None, n2, c2, t2, 0, 0, 0.0, stream))
+        fl = 4.0 * D * allowed_pairs(n2, c2, t2) * B * H
+        res[f"masked_fwd_c{c2}_t{t2}"] = {"config": dict(B=B, H=H, D=D, n=n2, c=c2, t=t2, S=S), "ms": ms,
+                                          "useful_tflops": fl / (ms * 1e-3) / 1e12,
+                                          "gbs": 4.0 * q.numel() * 2 / (ms * 1e-3) / 1e9,
+                                          "frac_of_measured_hbm": 4.0 * q.numel() * 2 / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        del q, k, v, o
+    torch.cuda.empty_cache()
     B, H, c, t, mem_len = 64, 32, 8, 16, 16384
     tc = c * t
     cap = mem_len + tc + t

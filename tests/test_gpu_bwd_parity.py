@@ -223,3 +223,24 @@ def test_forward_and_backward_on_seeded_random_layouts(n, c, t, tail, flags, D):
     want = oracle.masked_attn_bwd(npf(q), npf(k), npf(v), npf(d_o), n, c, t, tail, flags)
     for g, w, name in zip(got, want, ("dq", "dk", "dv")):
         check_grad(g, w, torch.bfloat16, name)
+
+
+@pytest.mark.parametrize("c,t,n", [(2, 4, 40), (2, 8, 24), (2, 32, 6), (4, 8, 12), (8, 8, 6)])
+def test_table1_style_geometries_forward_and_backward(c, t, n):
+    """The compression settings of the paper's Table 1 / Fig. 7 sweeps (short memory zones, c = 2..8): many
+    chunks per 128-row tile.  Forward and all three gradients against the oracle, bf16 tensor-core kernels."""
+    B, H, D = 1, 2, 128
+    S = oracle.seq_len(n, c, t)
+    q, k, v = synthetic.qkv(B, H, S, D, seed=51, std=1.0, dtype=torch.bfloat16)
+    d_o = synthetic.normal_tensor((B, H, S, D), 53, 1.0, torch.bfloat16)
+    qd, kd, vd, gd = (x.to(DEV) for x in (q, k, v, d_o))
+    o = torch.full_like(qd, float("nan"))
+    lse = torch.full((B, H, S), float("nan"), dtype=torch.float32, device=DEV)
+    L.loma_masked_attn_fwd(qd, kd, vd, o, lse, n, c, t)
+    torch.cuda.synchronize()
+    want_o, want_lse = oracle.masked_attn_fwd(npf(q), npf(k), npf(v), n, c, t)
+    assert np.abs(npf(o) - want_o).max() <= 2e-2 and np.abs(npf(lse) - want_lse).max() <= 2e-2
+    got = run_fwd_bwd(qd, kd, vd, gd, n, c, t)
+    want = oracle.masked_attn_bwd(npf(q), npf(k), npf(v), npf(d_o), n, c, t)
+    for g, w, name in zip(got, want, ("dq", "dk", "dv")):
+        check_grad(g, w, torch.bfloat16, name)
