@@ -176,7 +176,10 @@ __host__ __device__ __forceinline__ unsigned step_halves(const FwdParams& p, con
 // Steps from 64 on are taken whole, so that two 64-bit words always suffice.
 struct HalfMasks {
     unsigned long long m[2];
-    __host__ __device__ __forceinline__ bool has(int h, int j) const { return j >= 64 || ((m[h] >> j) & 1ull); }
+    // visited halves of step j as two bits (bit h = half h)
+    __host__ __device__ __forceinline__ unsigned bits(int j) const {
+        return j >= 64 ? 3u : (unsigned)((m[0] >> j) & 1ull) | ((unsigned)((m[1] >> j) & 1ull) << 1);
+    }
 };
 __host__ __device__ __forceinline__ unsigned visited_halves(const FwdParams& p, const TileDesc& td, int j) {
     if (j >= 64) return 3u;
@@ -189,15 +192,17 @@ __host__ __device__ __forceinline__ unsigned visited_halves(const FwdParams& p, 
 // the unit of the kernel's pipeline: one score buffer, one softmax pass, one P.V product.
 struct HalfWalk {
     int j, h;
-    __host__ __device__ __forceinline__ void start(const HalfMasks& hm) { j = 0; h = hm.has(0, 0) ? 0 : 1; }
+    unsigned cur;   // visited halves of step j (looked up once per step)
+    __host__ __device__ __forceinline__ void start(const HalfMasks& hm) { j = 0; cur = hm.bits(0); h = (cur & 1u) ? 0 : 1; }
     __host__ __device__ __forceinline__ bool done(int nsteps) const { return j >= nsteps; }
     __host__ __device__ __forceinline__ void next(const HalfMasks& hm) {
-        if (h == 0 && hm.has(1, j)) { h = 1; return; }
+        if (h == 0 && (cur & 2u)) { h = 1; return; }
         ++j;
-        h = hm.has(0, j) ? 0 : 1;
+        cur = hm.bits(j);
+        h = (cur & 1u) ? 0 : 1;
     }
-    __host__ __device__ __forceinline__ bool first_of_step(const HalfMasks& hm) const { return h == 0 || !hm.has(0, j); }
-    __host__ __device__ __forceinline__ bool last_of_step(const HalfMasks& hm) const { return h == 1 || !hm.has(1, j); }
+    __host__ __device__ __forceinline__ bool first_of_step(const HalfMasks&) const { return h == 0 || !(cur & 1u); }
+    __host__ __device__ __forceinline__ bool last_of_step(const HalfMasks&) const { return h == 1 || !(cur & 2u); }
 };
 
 // ------------------------------------------------------------------ the plan read by key tile
