@@ -270,3 +270,20 @@ def test_ragged_compress_validation(lib):
     assert call(flags=1) == UNSUPPORTED                 # prior-memory variant is not offered ragged
     assert call(D=32) == UNSUPPORTED
     assert call(B=0) == 0
+
+
+def test_header_and_library_are_usable_from_plain_c(lib, tmp_path):
+    """include/loma.h compiles as strict C99 and a C program linked against the library gets the documented
+    answers from the entry points that need no device."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    exe = str(tmp_path / "abi_check")
+    libdir = os.path.dirname(binding.library_path())
+    cmd = ["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+           os.path.join(ROOT, "tests", "c_abi", "abi_check.c"), "-o", exe, "-L", libdir, "-lloma", f"-Wl,-rpath,{libdir}"]
+    subprocess.run(cmd, check=True, capture_output=True, text=True)
+    out = subprocess.run([exe], capture_output=True, text=True)
+    assert out.returncode == 0, out.stderr
+    assert "abi_check ok" in out.stdout
