@@ -244,3 +244,43 @@ def test_table1_style_geometries_forward_and_backward(c, t, n):
     want = oracle.masked_attn_bwd(npf(q), npf(k), npf(v), npf(d_o), n, c, t)
     for g, w, name in zip(got, want, ("dq", "dk", "dv")):
         check_grad(g, w, torch.bfloat16, name)
+
+
+def test_training_calls_replay_from_a_cuda_graph():
+    """Rotary embedding, forward and backward captured once (after an eager warm-up) and replayed twice: the
+    forward's run-time tile counter is cleared by each launch's last CTA, so every replay starts from zero and
+    reproduces the eager results bit for bit."""
+    B, H, D, n, c, t, tail = 2, 2, 128, 5, 4, 16, 9
+    S = oracle.seq_len(n, c, t, tail)
+    q0, k0, v0 = (x.to(DEV) for x in synthetic.qkv(B, H, S, D, seed=71, dtype=torch.bfloat16))
+    d_o = synthetic.normal_tensor((B, H, S, D), 72, 1.0, torch.bfloat16).to(DEV)
+    ws = torch.empty(L.loma_masked_attn_bwd_workspace_bytes(B, H, D, n, c, t, tail), dtype=torch.uint8, device=DEV)
+
+    def run(q, k, v, o, lse, dq, dk, dv, stream=None):
+        L.loma_rope_apply(q, k, n, c, t, tail, 0, 0.0, 0, stream)
+        L.loma_masked_attn_fwd(q, k, v, o, lse, n, c, t, tail, 0, 0.0, stream)
+        L.loma_masked_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, n, c, t, tail, 0, ws, 0.0, stream)
+
+    def buffers():
+        return (q0.clone(), k0.clone(), v0.clone(), torch.zeros_like(q0), torch.zeros((B, H, S), dtype=torch.float32, device=DEV),
+                torch.zeros_like(q0), torch.zeros_like(q0), torch.zeros_like(q0))
+
+    eager = buffers()
+    run(*eager)
+    torch.cuda.synchronize()
+    g = buffers()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            run(*g, side)
+    torch.cuda.synchronize()
+    for _ in range(2):
+        g[0].copy_(q0); g[1].copy_(k0)          # the rotation is in place
+        for x in g[3:]:
+            x.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for a, b in zip(g, eager):
+            assert torch.equal(a, b)

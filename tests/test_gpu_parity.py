@@ -494,3 +494,45 @@ def test_generation_workloads_sampled_heads(B, H, c, t, mem_len, steps):
             assert np.array_equal(npf(kc2[b, h, :mem_len + t]), nk[0, 0])
             assert np.array_equal(npf(vc2[b, h, :mem_len + t]), nv[0, 0])
         del kc2, vc2
+
+
+def test_generation_cycle_replays_from_a_cuda_graph():
+    """After one eager call of each entry point (first calls look up device symbols and set kernel attributes),
+    a tail of decode steps plus the compress step is captured into a CUDA graph and replayed: the replay equals
+    the eager run bit for bit, outputs and caches."""
+    B, H, D, c, t, mem_len = 2, 4, 128, 4, 16, 256
+    tc = c * t
+    cap = mem_len + tc + t
+    dtype = torch.bfloat16
+    kc0 = synthetic.normal_tensor((B, H, cap, D), 61, 1.0, dtype).to(DEV)
+    vc0 = synthetic.normal_tensor((B, H, cap, D), 62, 1.0, dtype).to(DEV)
+    steps = 5
+    qs, ks, vs = (synthetic.normal_tensor((steps, B, H, 1, D), 63 + i, 1.0, dtype).to(DEV) for i in range(3))
+    qm, km, vm = (x.to(DEV) for x in synthetic.qkv(B, H, t, D, seed=66, dtype=dtype))
+    ws = workspace(max(L.loma_decode_workspace_bytes(B, H, D, cap), L.loma_compress_workspace_bytes(B, H, D, t, mem_len, 0)))
+
+    def cycle(kc, vc, outs, om, stream=None):
+        for j in range(steps):
+            L.loma_decode_attn(qs[j], ks[j], vs[j], kc, vc, outs[j], None, mem_len + tc - steps + j, ws, 0, 0.0, stream)
+        L.loma_compress_step(qm, km, vm, kc, vc, om, None, mem_len, c, t, ws, 0, 0.0, stream)
+
+    kc_e, vc_e = kc0.clone(), vc0.clone()
+    outs_e, om_e = torch.zeros((steps, B, H, 1, D), dtype=dtype, device=DEV), torch.zeros((B, H, t, D), dtype=dtype, device=DEV)
+    cycle(kc_e, vc_e, outs_e, om_e)
+    torch.cuda.synchronize()
+
+    kc_g, vc_g = kc0.clone(), vc0.clone()
+    outs_g, om_g = torch.zeros_like(outs_e), torch.zeros_like(om_e)
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            cycle(kc_g, vc_g, outs_g, om_g, side)
+    torch.cuda.synchronize()
+    for _ in range(2):
+        kc_g.copy_(kc0); vc_g.copy_(vc0); outs_g.zero_(); om_g.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(outs_g, outs_e) and torch.equal(om_g, om_e)
+        assert torch.equal(kc_g[:, :, :mem_len + t], kc_e[:, :, :mem_len + t]) and torch.equal(vc_g[:, :, :mem_len + t], vc_e[:, :, :mem_len + t])
