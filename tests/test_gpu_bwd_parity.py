@@ -284,3 +284,26 @@ def test_training_calls_replay_from_a_cuda_graph():
         torch.cuda.synchronize()
         for a, b in zip(g, eager):
             assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_autograd_wrapper_matches_torch_autograd_on_the_dense_mask(dtype):
+    """The differentiable torch op built on the two entry points against torch's own autograd of dense masked
+    softmax attention in fp64 on the same stored inputs (a third opinion next to the oracle)."""
+    from paper_2401_09486_b200.autograd import loma_masked_attention
+    B, H, D, n, c, t, tail = 2, 2, 64, 3, 4, 8, 5
+    S = oracle.seq_len(n, c, t, tail)
+    q, k, v = (x.to(DEV).requires_grad_(True) for x in synthetic.qkv(B, H, S, D, seed=81, dtype=dtype))
+    w = synthetic.normal_tensor((B, H, S, D), 82, 1.0, dtype).to(DEV)
+    o = loma_masked_attention(q, k, v, n, c, t, tail)
+    (o.float() * w.float()).sum().backward()
+    M = torch.from_numpy(oracle.dense_mask(n, c, t, tail)).to(DEV)
+    q2, k2, v2 = (x.detach().double().requires_grad_(True) for x in (q, k, v))
+    A = (q2 @ k2.transpose(-1, -2)) / D ** 0.5
+    o2 = torch.softmax(A.masked_fill(~M, float("-inf")), dim=-1) @ v2
+    (o2 * w.double()).sum().backward()
+    torch.cuda.synchronize()
+    tol = 1e-5 if dtype == torch.float32 else 2e-2
+    assert float((o.detach().double() - o2.detach()).abs().max()) <= tol
+    for g, g2, name in ((q.grad, q2.grad, "dq"), (k.grad, k2.grad, "dk"), (v.grad, v2.grad, "dv")):
+        check_grad(g, g2.cpu().numpy(), dtype, name)
