@@ -307,3 +307,32 @@ def test_autograd_wrapper_matches_torch_autograd_on_the_dense_mask(dtype):
     assert float((o.detach().double() - o2.detach()).abs().max()) <= tol
     for g, g2, name in ((q.grad, q2.grad, "dq"), (k.grad, k2.grad, "dk"), (v.grad, v2.grad, "dv")):
         check_grad(g, g2.cpu().numpy(), dtype, name)
+
+
+def test_tiles_with_more_than_64_steps_forward_and_backward():
+    """c = 1, t = 128, 70 chunks (26880 rows): the last reading tiles visit 70 key tiles and the first memory key
+    tiles are visited by 70+ query tiles, beyond the 64 steps whose visited halves the kernels keep as bit masks
+    (later steps are taken whole).  Sampled rows against the oracle; every element against the CUDA-core kernels."""
+    B, H, D, n, c, t = 1, 2, 64, 70, 1, 128
+    S = oracle.seq_len(n, c, t)
+    q, k, v, d_o = (synthetic.big_normal_(torch.empty(B, H, S, D, dtype=torch.bfloat16, device=DEV), 300 + i) for i in range(4))
+    o = torch.full_like(q, float("nan"))
+    lse = torch.full((B, H, S), float("nan"), dtype=torch.float32, device=DEV)
+    L.loma_masked_attn_fwd(q, k, v, o, lse, n, c, t)
+    dq, dk, dv = run_fwd_bwd(q, k, v, d_o, n, c, t)
+    o_g = torch.empty_like(q)
+    L.loma_masked_attn_fwd(q, k, v, o_g, None, n, c, t, 0, GENERIC)
+    gq, gk, gv = run_fwd_bwd(q, k, v, d_o, n, c, t, 0, GENERIC)
+    torch.cuda.synchronize()
+    assert float((o.float() - o_g.float()).abs().max()) <= 2e-2
+    for a, b_, name in ((dq, gq, "dq"), (dk, gk, "dk"), (dv, gv, "dv")):
+        ref = b_.float()
+        assert float((a.float() - ref).abs().max()) <= 2e-2 * max(1.0, float(ref.abs().max())), name
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([rng.choice(S, 40, replace=False), np.arange(S - 384, S - 380), np.array([0, 127, 128, 255, 256])]))
+    ri = torch.from_numpy(rows).to(DEV)
+    sl = (slice(0, 1), slice(1, 2))
+    want_o, want_lse = oracle.masked_attn_fwd(npf(q[sl]), npf(k[sl]), npf(v[sl]), n, c, t, rows=rows)
+    assert np.abs(npf(o[sl][:, :, ri]) - want_o).max() <= 2e-2 and np.abs(npf(lse[sl][:, :, ri]) - want_lse).max() <= 2e-2
+    want_dq = oracle.masked_attn_bwd_dq_rows(npf(q[sl]), npf(k[sl]), npf(v[sl]), npf(d_o[sl]), rows, n, c, t)
+    check_grad(dq[sl][:, :, ri], want_dq, torch.bfloat16, "dq")
