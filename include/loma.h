@@ -326,6 +326,30 @@ LOMA_API int loma_decode_attn_ragged(const void* q, const void* k_new, const voi
                                      void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * loma_decode_attn_paged -- the ragged decode step over a paged cache: the K and V entries of all
+ * sequences live in one pool of fixed-size pages, and a block table says which page holds which
+ * stretch of which sequence (the paper keeps one contiguous cache per sequence; this is the same
+ * step, Appendix A inference_input, for a serving engine that hands out cache memory page by page).
+ * Slot j of sequence b is row j % page_size of page block_table[b][j / page_size].
+ *
+ *   k_pool, v_pool [device, in/out]  [n_pages, H, page_size, D] contiguous
+ *   block_table    [device, in]      int32 [B, max_pages]; entries are clamped to [0, n_pages) on the device;
+ *                                    only the blocks below a sequence's length (and the one that takes the new
+ *                                    token) are read
+ *   page_size      a power of two
+ *   cache_lens, max_cache_len        as in loma_decode_attn_ragged; max_cache_len < max_pages * page_size
+ * The new token's K/V are written at slot cache_lens[b] of sequence b (its page must be in the table).
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CAPACITY, WORKSPACE, CUDA.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_decode_attn_paged(const void* q, const void* k_new, const void* v_new,
+                                    void* k_pool, void* v_pool, const int32_t* block_table,
+                                    void* o, float* lse, int B, int H, int D,
+                                    int page_size, int max_pages, int n_pages,
+                                    const int32_t* cache_lens, int max_cache_len,
+                                    loma_dtype dtype, float softmax_scale, unsigned flags,
+                                    void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------
  * loma_decode_attn_static -- the same decode step as loma_decode_attn (bf16
  * only), for callers that cannot hand the library a workspace because they
  * cannot obtain device memory at the point of the call.  (The paper has no

@@ -36,6 +36,8 @@ from .loma_oracle import (  # noqa: F401
     rope_apply,
     decode_attn,
     decode_attn_ragged,
+    decode_attn_paged,
+    paged_to_contiguous,
     compress_step,
     compress_step_ragged,
     replay_generation,

@@ -500,6 +500,37 @@ def decode_attn_ragged(q, k_new, v_new, k_cache, v_cache, cache_lens, scale=None
     return o, lse, kc, vc
 
 
+def paged_to_contiguous(pool, block_table, cap):
+    """The logical cache [B, H, cap, D] that a pool [n_pages, H, page_size, D] and a block table [B, max_pages]
+    describe: slot j of sequence b is row j % page_size of page block_table[b][j // page_size]."""
+    pool = np.asarray(pool)
+    n_pages, H, ps, D = pool.shape
+    B = len(block_table)
+    out = np.zeros((B, H, cap, D), dtype=pool.dtype)
+    for b in range(B):
+        for j in range(cap):
+            out[b, :, j] = pool[int(block_table[b][j // ps]), :, j % ps]
+    return out
+
+
+def decode_attn_paged(q, k_new, v_new, k_pool, v_pool, block_table, cache_lens, scale=None):
+    """decode_attn_ragged over a paged cache: read every sequence's logical cache out of the pools, run the
+    per-sequence decode, and write the appended entry back into its page.  Returns (o, lse, k_pool', v_pool')."""
+    k_pool, v_pool = np.asarray(k_pool), np.asarray(v_pool)
+    ps = k_pool.shape[2]
+    cap = max(int(n) for n in cache_lens) + 1
+    kc = paged_to_contiguous(k_pool, block_table, cap)
+    vc = paged_to_contiguous(v_pool, block_table, cap)
+    o, lse, kc2, vc2 = decode_attn_ragged(q, k_new, v_new, kc, vc, cache_lens, scale)
+    kp, vp = k_pool.copy(), v_pool.copy()
+    for b, n in enumerate(cache_lens):
+        n = int(n)
+        page = int(block_table[b][n // ps])
+        kp[page, :, n % ps] = kc2[b, :, n]
+        vp[page, :, n % ps] = vc2[b, :, n]
+    return o, lse, kp, vp
+
+
 def compress_step(q_mem, k_mem, v_mem, k_cache, v_cache, mem_len, c, t, flags=0, scale=None):
     """Compress pass + compaction (Section 3.1 steps 2-3; Appendix A
     `compress_last_chunk`).

@@ -42,6 +42,7 @@ SIGNATURES = {
     "loma_masked_attn_bwd_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
+    "loma_decode_attn_paged": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_attn_ragged": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_attn_static": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _p]),
     "loma_decode_static_scratch_bytes": (_sz, []),
@@ -279,6 +280,25 @@ def loma_decode_attn_ragged(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len
                                        _ptr(lse), B, H, D, cap, _ptr(cache_lens), int(max_cache_len), _dtype_code(q),
                                        float(softmax_scale), int(flags), _ptr(workspace), ws_bytes, _stream(stream))
     _check(rc, "loma_decode_attn_ragged")
+
+
+def loma_decode_attn_paged(q, k_new, v_new, k_pool, v_pool, block_table, o, lse, cache_lens, max_cache_len: int,
+                           workspace=None, flags: int = 0, softmax_scale: float = 0.0, stream=None) -> None:
+    """Ragged decode over a paged cache.  k_pool, v_pool: [n_pages, H, page_size, D]; block_table: device int32
+    [B, max_pages]; cache_lens: device int32 [B]; q, k_new, v_new, o: [B, H, 1, D]."""
+    n_pages, H, page_size, D = k_pool.shape
+    B, max_pages = block_table.shape
+    for x in (q, k_new, v_new, k_pool, v_pool, o, block_table, cache_lens):
+        if x is not None and not x.is_contiguous():
+            raise ValueError("decode tensors must be contiguous")
+    if block_table.dtype != torch.int32 or cache_lens.dtype != torch.int32 or cache_lens.numel() != B:
+        raise ValueError("block_table must be int32 [B, max_pages] and cache_lens int32 [B]")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().loma_decode_attn_paged(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool), _ptr(block_table),
+                                      _ptr(o), _ptr(lse), B, H, D, page_size, max_pages, n_pages, _ptr(cache_lens),
+                                      int(max_cache_len), _dtype_code(q), float(softmax_scale), int(flags),
+                                      _ptr(workspace), ws_bytes, _stream(stream))
+    _check(rc, "loma_decode_attn_paged")
 
 
 def loma_decode_static_scratch_bytes() -> int:

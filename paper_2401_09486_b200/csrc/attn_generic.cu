@@ -238,8 +238,15 @@ struct DecodeMap {
     const T* kn;
     const T* vn;
     int len, D;
-    __device__ __forceinline__ const T* kptr(int vi) const { return vi < len ? kc + (int64_t)vi * D : kn; }
-    __device__ __forceinline__ const T* vptr(int vi) const { return vi < len ? vc + (int64_t)vi * D : vn; }
+    Paging pg;        // pg.table != NULL: kc / vc are the pools and slots go through the block table
+    int b, h, H;
+    __device__ __forceinline__ int64_t slot(int vi) const {
+        if (!pg.table) return (int64_t)vi * D;
+        const int page = min(max(pg.table[(int64_t)b * pg.max_pages + (vi >> pg.log2_ps)], 0), pg.n_pages - 1);
+        return ((((int64_t)page * H + h) << pg.log2_ps) + (vi & ((1 << pg.log2_ps) - 1))) * D;
+    }
+    __device__ __forceinline__ const T* kptr(int vi) const { return vi < len ? kc + slot(vi) : kn; }
+    __device__ __forceinline__ const T* vptr(int vi) const { return vi < len ? vc + slot(vi) : vn; }
 };
 
 template <typename T, int D>
@@ -247,24 +254,26 @@ __global__ void __launch_bounds__(32)
 decode_generic_kernel(const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
                       T* __restrict__ k_cache, T* __restrict__ v_cache, T* __restrict__ o,
                       float* __restrict__ lse, int cap, int cache_len_max, const int32_t* __restrict__ lens, int H,
-                      float scale) {
+                      float scale, Paging pg) {
     __shared__ __align__(16) float q_sh[D];
     const int bh = blockIdx.x, lane = threadIdx.x;
     const int cache_len = lens ? min(max(lens[bh / H], 0), cache_len_max) : cache_len_max;   // ragged batch
-    T* kc = k_cache + (int64_t)bh * cap * D;
-    T* vc = v_cache + (int64_t)bh * cap * D;
+    T* kc = pg.table ? k_cache : k_cache + (int64_t)bh * cap * D;
+    T* vc = pg.table ? v_cache : v_cache + (int64_t)bh * cap * D;
     DecodeMap<T> map;
     map.kc = kc; map.vc = vc; map.len = cache_len; map.D = D;
-    map.kn = k_new ? k_new + (int64_t)bh * D : kc + (int64_t)cache_len * D;
-    map.vn = v_new ? v_new + (int64_t)bh * D : vc + (int64_t)cache_len * D;
+    map.pg = pg; map.b = bh / H; map.h = bh - map.b * H; map.H = H;
+    const int64_t new_off = map.slot(cache_len);
+    map.kn = k_new ? k_new + (int64_t)bh * D : kc + new_off;
+    map.vn = v_new ? v_new + (int64_t)bh * D : vc + new_off;
     stage_query<T, D>(q_sh, q + (int64_t)bh * D, lane);
     attend_row<T, D>(q_sh, map, cache_len + 1, scale, o + (int64_t)bh * D, lse ? lse + bh : nullptr, lane);
     if (k_new) {      // append: the slot is read by nobody in this launch
         constexpr int DPL = D / 32;
 #pragma unroll
         for (int d = 0; d < DPL; ++d) {
-            kc[(int64_t)cache_len * D + lane * DPL + d] = k_new[(int64_t)bh * D + lane * DPL + d];
-            vc[(int64_t)cache_len * D + lane * DPL + d] = v_new[(int64_t)bh * D + lane * DPL + d];
+            kc[new_off + lane * DPL + d] = k_new[(int64_t)bh * D + lane * DPL + d];
+            vc[new_off + lane * DPL + d] = v_new[(int64_t)bh * D + lane * DPL + d];
         }
     }
 }
@@ -542,29 +551,30 @@ cudaError_t launch_masked_attn_bwd_generic(const void* q, const void* k, const v
 template <typename T, int D>
 static cudaError_t decode_generic_t(const void* q, const void* kn, const void* vn, void* kc, void* vc,
                                     void* o, float* lse, int BH, int cap, int cache_len, const int32_t* lens, int H,
-                                    float scale, cudaStream_t st) {
+                                    float scale, const Paging& pg, cudaStream_t st) {
     decode_generic_kernel<T, D><<<BH, 32, 0, st>>>(static_cast<const T*>(q), static_cast<const T*>(kn),
                                                    static_cast<const T*>(vn), static_cast<T*>(kc),
                                                    static_cast<T*>(vc), static_cast<T*>(o), lse, cap,
-                                                   cache_len, lens, H, scale);
+                                                   cache_len, lens, H, scale, pg);
     count_launches(1);
     return cudaGetLastError();
 }
 
 cudaError_t launch_decode_generic(const void* q, const void* k_new, const void* v_new, void* k_cache,
                                   void* v_cache, void* o, float* lse, int B, int H, int D, int cap,
-                                  int cache_len, const int32_t* lens, loma_dtype dt, float scale, cudaStream_t st) {
+                                  int cache_len, const int32_t* lens, loma_dtype dt, float scale, const Paging& pg,
+                                  cudaStream_t st) {
     const int BH = B * H;
     if (dt == LOMA_F32) {
         return D == 64 ? decode_generic_t<float, 64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
-                                                     cache_len, lens, H, scale, st)
+                                                     cache_len, lens, H, scale, pg, st)
                        : decode_generic_t<float, 128>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
-                                                      cache_len, lens, H, scale, st);
+                                                      cache_len, lens, H, scale, pg, st);
     }
     return D == 64 ? decode_generic_t<__nv_bfloat16, 64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
-                                                         cache_len, lens, H, scale, st)
+                                                         cache_len, lens, H, scale, pg, st)
                    : decode_generic_t<__nv_bfloat16, 128>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
-                                                          cache_len, lens, H, scale, st);
+                                                          cache_len, lens, H, scale, pg, st);
 }
 
 template <typename T, int D>

@@ -75,13 +75,15 @@ __device__ __forceinline__ void axpy8(float (&o)[8], float p, const uint4& v) {
 }
 
 // total = cache_len + 1 visible keys; key index cache_len is the new token.
-template <int D>
+// PAGED: the cache is a pool of pages [n_pages, H, page_size, D]; slot j of sequence b lives in page
+// table[b][j / page_size] at row j % page_size (page numbers are clamped to the pool on the device).
+template <int D, bool PAGED>
 __global__ void __launch_bounds__(DEC_WARPS * 32)
 decode_splitkv_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_new,
                       const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ k_cache,
                       __nv_bfloat16* __restrict__ v_cache, __nv_bfloat16* __restrict__ o,
                       float* __restrict__ lse, float* __restrict__ ws, int BH, int cap, int cache_len_max,
-                      const int32_t* __restrict__ lens, int H, int splits, int split_len, float scale_log2) {
+                      const int32_t* __restrict__ lens, int H, int splits, int split_len, float scale_log2, Paging pg) {
     constexpr int LPK = D / 8;           // lanes per row
     constexpr int KPL = 32 / LPK;        // rows per warp load
     constexpr int BK = DEC_NL * KPL;     // rows per warp iteration
@@ -99,10 +101,18 @@ decode_splitkv_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
     const int k_begin = split * split_len;
     const int k_end = min(total, k_begin + split_len);   // may be <= k_begin in a ragged batch
 
-    const uint4* kc = reinterpret_cast<const uint4*>(k_cache + (int64_t)bh * cap * D);
-    const uint4* vc = reinterpret_cast<const uint4*>(v_cache + (int64_t)bh * cap * D);
-    const uint4* kn = k_new ? reinterpret_cast<const uint4*>(k_new + (int64_t)bh * D) : kc + (int64_t)cache_len * LPK;
-    const uint4* vn = v_new ? reinterpret_cast<const uint4*>(v_new + (int64_t)bh * D) : vc + (int64_t)cache_len * LPK;
+    // slot j of this (b,h) -> offset of its row in 16-byte units from kc / vc
+    const int pb = bh / H, phd = bh - pb * H;
+    auto row_off = [&](int j) -> int64_t {
+        if (!PAGED) return (int64_t)j * LPK;
+        const int page = min(max(__ldg(pg.table + (int64_t)pb * pg.max_pages + (j >> pg.log2_ps)), 0), pg.n_pages - 1);
+        return ((((int64_t)page * H + phd) << pg.log2_ps) + (j & ((1 << pg.log2_ps) - 1))) * LPK;
+    };
+    const uint4* kc = reinterpret_cast<const uint4*>(PAGED ? k_cache : k_cache + (int64_t)bh * cap * D);
+    const uint4* vc = reinterpret_cast<const uint4*>(PAGED ? v_cache : v_cache + (int64_t)bh * cap * D);
+    const int64_t new_off = row_off(cache_len);
+    const uint4* kn = k_new ? reinterpret_cast<const uint4*>(k_new + (int64_t)bh * D) : kc + new_off;
+    const uint4* vn = v_new ? reinterpret_cast<const uint4*>(v_new + (int64_t)bh * D) : vc + new_off;
 
     float qf[8];
     {
@@ -126,13 +136,13 @@ decode_splitkv_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
             const int j = j0 + i * KPL + sub;
             valid[i] = j < k_end;
             const int jc = min(j, cache_len);                  // stay inside [0, cache_len]
-            const uint4* kp = (jc < cache_len) ? kc + (int64_t)jc * LPK : kn;
+            const uint4* kp = (jc < cache_len) ? kc + row_off(jc) : kn;
             kr[i] = ld_stream(kp + li);
         }
 #pragma unroll
         for (int i = 0; i < DEC_NL; ++i) {
             const int jc = min(j0 + i * KPL + sub, cache_len);
-            const uint4* vp = (jc < cache_len) ? vc + (int64_t)jc * LPK : vn;
+            const uint4* vp = (jc < cache_len) ? vc + row_off(jc) : vn;
             vr[i] = ld_stream(vp + li);
         }
         float s[DEC_NL];
@@ -206,8 +216,8 @@ decode_splitkv_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
     }
     // append the new token's K/V at slot cache_len (read by nobody in this launch)
     if (k_new && split == splits - 1 && warp == 0 && lane < LPK) {
-        uint4* kd = reinterpret_cast<uint4*>(k_cache + ((int64_t)bh * cap + cache_len) * D);
-        uint4* vd = reinterpret_cast<uint4*>(v_cache + ((int64_t)bh * cap + cache_len) * D);
+        uint4* kd = const_cast<uint4*>(kc) + new_off;
+        uint4* vd = const_cast<uint4*>(vc) + new_off;
         kd[lane] = __ldg(kn + lane);
         vd[lane] = __ldg(vn + lane);
     }
@@ -238,17 +248,24 @@ decode_merge_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ o,
 template <int D>
 static cudaError_t decode_bf16_t(const void* q, const void* kn, const void* vn, void* kc, void* vc, void* o,
                                  float* lse, int BH, int cap, int cache_len, const int32_t* lens, int H, float scale,
-                                 void* ws, cudaStream_t st) {
+                                 void* ws, const Paging& pg, cudaStream_t st) {
     const int total = cache_len + 1;
     const int splits = decode_num_splits(BH, total);
     int split_len = (total + splits - 1) / splits;
     split_len = (split_len + 15) / 16 * 16;
     const float scale_log2 = scale * 1.4426950408889634f;
-    decode_splitkv_kernel<D><<<BH * splits, DEC_WARPS * 32, 0, st>>>(
-        static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(kn),
-        static_cast<const __nv_bfloat16*>(vn), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
-        static_cast<__nv_bfloat16*>(o), lse, static_cast<float*>(ws), BH, cap, cache_len, lens, H, splits, split_len,
-        scale_log2);
+    if (pg.table)
+        decode_splitkv_kernel<D, true><<<BH * splits, DEC_WARPS * 32, 0, st>>>(
+            static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(kn),
+            static_cast<const __nv_bfloat16*>(vn), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
+            static_cast<__nv_bfloat16*>(o), lse, static_cast<float*>(ws), BH, cap, cache_len, lens, H, splits, split_len,
+            scale_log2, pg);
+    else
+        decode_splitkv_kernel<D, false><<<BH * splits, DEC_WARPS * 32, 0, st>>>(
+            static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(kn),
+            static_cast<const __nv_bfloat16*>(vn), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
+            static_cast<__nv_bfloat16*>(o), lse, static_cast<float*>(ws), BH, cap, cache_len, lens, H, splits, split_len,
+            scale_log2, pg);
     count_launches(1);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || splits == 1) return e;
@@ -260,11 +277,11 @@ static cudaError_t decode_bf16_t(const void* q, const void* kn, const void* vn, 
 
 cudaError_t launch_decode_bf16(const void* q, const void* k_new, const void* v_new, void* k_cache,
                                void* v_cache, void* o, float* lse, int B, int H, int D, int cap, int cache_len,
-                               const int32_t* lens, float scale, void* ws, cudaStream_t st) {
+                               const int32_t* lens, float scale, void* ws, const Paging& pg, cudaStream_t st) {
     const int BH = B * H;
-    return D == 64 ? decode_bf16_t<64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap, cache_len, lens, H, scale, ws, st)
+    return D == 64 ? decode_bf16_t<64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap, cache_len, lens, H, scale, ws, pg, st)
                    : decode_bf16_t<128>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap, cache_len, lens, H, scale, ws,
-                                        st);
+                                        pg, st);
 }
 
 // ---------------------------------------------------------------------------
@@ -297,7 +314,7 @@ cudaError_t launch_decode_bf16_static(const void* q, const void* k_new, const vo
                                       int cache_len, float scale, cudaStream_t st) {
     void* ws = decode_static_scratch();
     if (!ws) return cudaErrorInvalidSymbol;
-    return launch_decode_bf16(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, nullptr, scale, ws, st);
+    return launch_decode_bf16(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, nullptr, scale, ws, Paging{}, st);
 }
 
 }  // namespace loma

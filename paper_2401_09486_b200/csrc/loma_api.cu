@@ -317,10 +317,10 @@ int loma_decode_attn(const void* q, const void* k_new, const void* v_new, void* 
     cudaError_t e;
     if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC))
         e = launch_decode_bf16(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, nullptr, scale,
-                               workspace, st);
+                               workspace, Paging{}, st);
     else
         e = launch_decode_generic(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, nullptr, dtype,
-                                  scale, st);
+                                  scale, Paging{}, st);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 
@@ -348,10 +348,53 @@ int loma_decode_attn_ragged(const void* q, const void* k_new, const void* v_new,
     cudaError_t e;
     if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC))
         e = launch_decode_bf16(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, max_cache_len, cache_lens, scale,
-                               workspace, st);
+                               workspace, Paging{}, st);
     else
         e = launch_decode_generic(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, max_cache_len, cache_lens,
-                                  dtype, scale, st);
+                                  dtype, scale, Paging{}, st);
+    return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
+// page_size must be a power of two; returns its log2 or -1
+static int log2_exact(int x) {
+    if (x <= 0 || (x & (x - 1))) return -1;
+    int l = 0;
+    while ((1 << l) < x) ++l;
+    return l;
+}
+
+int loma_decode_attn_paged(const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+                           const int32_t* block_table, void* o, float* lse, int B, int H, int D, int page_size,
+                           int max_pages, int n_pages, const int32_t* cache_lens, int max_cache_len, loma_dtype dtype,
+                           float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes, void* stream) {
+    if (B < 0 || H < 0 || max_pages < 0 || n_pages < 0 || max_cache_len < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    const int l2 = log2_exact(page_size);
+    if (l2 < 0 || page_size > 65536) return LOMA_ERR_INVALID_ARG;
+    if ((k_new == nullptr) != (v_new == nullptr)) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)max_cache_len >= (int64_t)max_pages * page_size) return LOMA_ERR_CAPACITY;   // the new token needs a slot too
+    if (B == 0 || H == 0) return LOMA_OK;
+    if (!q || !k_pool || !v_pool || !o || !block_table || !cache_lens || n_pages < 1) return LOMA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_pool) || !aligned16(v_pool) || !aligned16(o) || !aligned16(k_new) ||
+        !aligned16(v_new) || !aligned16(workspace) || ((uintptr_t)cache_lens & 3u) || ((uintptr_t)block_table & 3u))
+        return LOMA_ERR_ALIGNMENT;
+    const size_t need = loma_decode_workspace_bytes(B, H, D, max_cache_len);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return LOMA_ERR_WORKSPACE;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((int64_t)B * H * 128 > INT_MAX) return LOMA_ERR_INVALID_ARG;
+    Paging pg;
+    pg.table = block_table; pg.max_pages = max_pages; pg.log2_ps = l2; pg.n_pages = n_pages;
+    cudaError_t e;
+    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC))
+        e = launch_decode_bf16(q, k_new, v_new, k_pool, v_pool, o, lse, B, H, D, 0, max_cache_len, cache_lens, scale,
+                               workspace, pg, st);
+    else
+        e = launch_decode_generic(q, k_new, v_new, k_pool, v_pool, o, lse, B, H, D, 0, max_cache_len, cache_lens, dtype,
+                                  scale, pg, st);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 

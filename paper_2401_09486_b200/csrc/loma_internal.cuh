@@ -58,6 +58,13 @@ __host__ __device__ inline RowInfo layout_row(int i, int n_chunks, int c, int t,
     return r;
 }
 
+// ---- paged cache: a pool of pages [n_pages, H, page_size, D]; table[b * max_pages + p] = page of sequence b's p-th block.
+// table == NULL means a contiguous cache [B, H, cap, D].
+struct Paging {
+    const int32_t* table = nullptr;
+    int max_pages = 0, log2_ps = 0, n_pages = 0;
+};
+
 // ---- launchers (each defined in its own .cu) ------------------------------
 cudaError_t launch_layout_index(const Layout& L, int32_t* chunk, int32_t* zone, int32_t* offset,
                                 int32_t* src, int32_t* pos, cudaStream_t st);
@@ -100,13 +107,14 @@ cudaError_t launch_bounded_wait_selftest(cudaStream_t st);   // attn_tcgen05.cu
 cudaError_t launch_decode_generic(const void* q, const void* k_new, const void* v_new,
                                   void* k_cache, void* v_cache, void* o, float* lse,
                                   int B, int H, int D, int cap, int cache_len, const int32_t* lens,
-                                  loma_dtype dt, float scale, cudaStream_t st);
+                                  loma_dtype dt, float scale, const Paging& pg, cudaStream_t st);
 
 // bf16 split-KV decode (decode_splitkv.cu)
 size_t decode_workspace_bytes(int BH, int D, int total_keys);
 cudaError_t launch_decode_bf16(const void* q, const void* k_new, const void* v_new, void* k_cache,
                                void* v_cache, void* o, float* lse, int B, int H, int D, int cap, int cache_len,
-                               const int32_t* lens, float scale, void* ws, cudaStream_t st);   // lens: per-sequence lengths or NULL
+                               const int32_t* lens, float scale, void* ws, const Paging& pg,
+                               cudaStream_t st);   // lens: per-sequence lengths or NULL
 
 size_t decode_static_scratch_bytes();
 cudaError_t launch_decode_bf16_static(const void* q, const void* k_new, const void* v_new, void* k_cache,

@@ -287,3 +287,18 @@ def test_header_and_library_are_usable_from_plain_c(lib, tmp_path):
     out = subprocess.run([exe], capture_output=True, text=True)
     assert out.returncode == 0, out.stderr
     assert "abi_check ok" in out.stdout
+
+
+def test_paged_decode_validation(lib):
+    def call(q=0x1000, kn=0x2000, vn=0x3000, kp=0x4000, vp=0x5000, bt=0x6000, o=0x7000, B=2, H=1, D=128, ps=16, mp=4, npg=8,
+             lens=0x8000, mx=40, dt=1):
+        return lib.loma_decode_attn_paged(q, kn, vn, kp, vp, bt, o, None, B, H, D, ps, mp, npg, lens, mx, dt, 0.0, 0, None, 0,
+                                          None)
+    assert call(ps=24) == INVALID                       # page size must be a power of two
+    assert call(mx=64) == CAPACITY                      # no slot left for the new token
+    assert call(bt=None) == INVALID
+    assert call(lens=None) == INVALID
+    assert call(npg=0) == INVALID
+    assert call(bt=0x6002) == ALIGNMENT
+    assert call(D=100) == UNSUPPORTED
+    assert call(B=0) == 0

@@ -371,6 +371,36 @@ def test_ragged_compress_matches_oracle_and_leaves_idle_sequences_alone(H, D, c,
         assert torch.equal(kcd[b, :, n + t:].cpu(), kc[b, :, n + t:])      # slots beyond the rewritten ones keep their contents
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, GENERIC])
+@pytest.mark.parametrize("H,D,ps,lens", [(2, 64, 16, [0, 1, 39, 17]), (3, 128, 64, [2999, 0, 1500, 257, 256, 255]),
+                                         (4, 128, 256, [8193, 100, 8256, 4097, 1]), (2, 128, 16, [4133, 4133])])
+def test_paged_decode_matches_oracle(H, D, ps, lens, flags, dtype):
+    """Sequences scattered over a shuffled pool of pages: each attends to its own slots through the block table."""
+    B = len(lens)
+    max_len = max(lens)
+    max_pages = max_len // ps + 1
+    n_pages = B * max_pages + 3
+    rng = np.random.default_rng(7)
+    perm = rng.permutation(n_pages)[: B * max_pages].reshape(B, max_pages).astype(np.int32)
+    kp = synthetic.normal_tensor((n_pages, H, ps, D), 51, 1.0, dtype)
+    vp = synthetic.normal_tensor((n_pages, H, ps, D), 52, 1.0, dtype)
+    q, kn, vn = synthetic.qkv(B, H, 1, D, seed=53, std=1.0, dtype=dtype)
+    want_o, want_lse, want_k, want_v = oracle.decode_attn_paged(npf(q), npf(kn), npf(vn), npf(kp), npf(vp), perm, lens)
+    kpd, vpd = kp.to(DEV), vp.to(DEV)
+    o = torch.full((B, H, 1, D), float("nan"), dtype=dtype, device=DEV)
+    lse = torch.full((B, H), float("nan"), dtype=torch.float32, device=DEV)
+    ws = workspace(L.loma_decode_workspace_bytes(B, H, D, max_len))
+    table_d = torch.from_numpy(perm).to(DEV)
+    lens_d = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    L.loma_decode_attn_paged(q.to(DEV), kn.to(DEV), vn.to(DEV), kpd, vpd, table_d, o, lse, lens_d, max_len, ws, flags)
+    torch.cuda.synchronize()
+    check_close(o, want_o, dtype)
+    assert np.abs(npf(lse) - want_lse[:, :, 0]).max() <= (1e-5 if dtype == torch.float32 else 2e-2)
+    # the pools changed in exactly the appended slots
+    assert np.array_equal(npf(kpd), want_k) and np.array_equal(npf(vpd), want_v)
+
+
 def test_bounded_wait_times_out_and_leaves_the_context_usable():
     """A device-side wait that can never be satisfied gives up after its limit,
     reports LOMA_ERR_TIMEOUT through the status word, and later launches work."""

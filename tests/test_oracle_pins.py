@@ -630,3 +630,33 @@ def test_ragged_compress_is_per_sequence_compress():
         ob, _, kb, _ = oracle.compress_step(qm[b:b + 1], km[b:b + 1], vm[b:b + 1], kc[b:b + 1], vc[b:b + 1], n, c, t)
         assert np.array_equal(o_r[b], ob[0]) and np.array_equal(k_r[b, :, :n + t], kb[0])
         assert np.array_equal(k_r[b, :, n + t:], kc[b, :, n + t:])        # nothing beyond the new length is touched
+
+
+def test_paged_decode_is_contiguous_decode_through_the_block_table():
+    """An identity block table reproduces the contiguous (ragged) decode; relabelling the pages (pool and table
+    permuted together) changes nothing; pages no table entry points at are neither read nor written."""
+    B, H, D, ps, max_pages = 3, 2, 8, 4, 3
+    cap = ps * max_pages
+    kc, vc = _rand((B, H, cap, D), 90), _rand((B, H, cap, D), 91)
+    q, kn, vn = _rand((B, H, 1, D), 92), _rand((B, H, 1, D), 93), _rand((B, H, 1, D), 94)
+    lens = [0, 11, 5]
+    # pools whose page b*max_pages + p holds slots [p*ps, (p+1)*ps) of sequence b, plus two unused pages
+    n_pages = B * max_pages + 2
+    kp, vp = np.full((n_pages, H, ps, D), np.nan), np.full((n_pages, H, ps, D), np.nan)
+    table = np.zeros((B, max_pages), np.int32)
+    for b in range(B):
+        for p_ in range(max_pages):
+            table[b, p_] = b * max_pages + p_
+            kp[table[b, p_]] = kc[b, :, p_ * ps:(p_ + 1) * ps]
+            vp[table[b, p_]] = vc[b, :, p_ * ps:(p_ + 1) * ps]
+    o_c, l_c, k_c, v_c = oracle.decode_attn_ragged(q, kn, vn, kc, vc, lens)
+    o_p, l_p, kp2, vp2 = oracle.decode_attn_paged(q, kn, vn, kp, vp, table, lens)
+    assert np.array_equal(o_c, o_p) and np.array_equal(l_c, l_p)
+    for b, n in enumerate(lens):
+        assert np.array_equal(kp2[table[b, n // ps], :, n % ps], kn[b, :, 0])
+    assert np.isnan(kp2[-2:]).all() and np.isnan(vp2[-2:]).all()
+    perm = np.random.default_rng(0).permutation(n_pages)          # new label of page i is perm[i]
+    kq, vq = np.empty_like(kp), np.empty_like(vp)
+    kq[perm], vq[perm] = kp, vp
+    o_q, _, _, _ = oracle.decode_attn_paged(q, kn, vn, kq, vq, perm[table], lens)
+    assert np.array_equal(o_q, o_p)
