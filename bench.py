@@ -459,7 +459,7 @@ def other_workloads(L, synthetic, torch, dev, peaks):
     torch.cuda.empty_cache()
     B, H, c, t, mem_len = 64, 32, 8, 16, 16384
     tc = c * t
-    cap = mem_len + tc + t
+    cap = (mem_len + tc + t + 63) // 64 * 64      # a whole number of 64-row pages (for the paged variant below)
     kc = synthetic.big_normal_(torch.empty(B, H, cap, D, dtype=bf, device=dev), 3100, std)
     vc = synthetic.big_normal_(torch.empty(B, H, cap, D, dtype=bf, device=dev), 3101, std)
     q1, k1, v1 = (synthetic.big_normal_(torch.empty(B, H, 1, D, dtype=bf, device=dev), 3102 + i, std) for i in range(3))
@@ -482,6 +482,20 @@ def other_workloads(L, synthetic, torch, dev, peaks):
     res["decode_ragged_B64_16k"] = {"config": dict(B=B, H=H, D=D, c=c, t=t, lens="mem_len + (7 b) mod tc"), "ms": ms,
                                     "gbs": nbytes / (ms * 1e-3) / 1e9,
                                     "frac_of_measured_hbm": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    # the same ragged decode over a paged cache: the cache tensors re-read as a pool of 64-row pages, scattered by a
+    # seeded permutation of the page numbers (every (b) owns cap/64 pages; the pool holds all heads of a page)
+    ps = 64
+    if cap % ps == 0 and hasattr(L, "loma_decode_attn_paged"):
+        mp = cap // ps
+        g_cpu = torch.Generator().manual_seed(3120)
+        table = torch.randperm(B * mp, generator=g_cpu).to(torch.int32).view(B, mp).to(dev)
+        kpool = kc.view(B, H, mp, ps, D).permute(0, 2, 1, 3, 4).reshape(B * mp, H, ps, D).contiguous()
+        vpool = vc.view(B, H, mp, ps, D).permute(0, 2, 1, 3, 4).reshape(B * mp, H, ps, D).contiguous()
+        ms = timed(lambda: L.loma_decode_attn_paged(q1, k1, v1, kpool, vpool, table, o1, None, lens, max_len, ws, 0, 0.0, stream))
+        res["decode_paged_B64_16k"] = {"config": dict(B=B, H=H, D=D, page_size=ps, pages=B * mp), "ms": ms,
+                                       "gbs": nbytes / (ms * 1e-3) / 1e9,
+                                       "frac_of_measured_hbm": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        del kpool, vpool
     for name, flags in (("compress_B64_16k", 0), ("compress_B64_16k_prior_mem", 1)):
         def run_decode_then_compress():
             L.loma_compress_step(qm, km, vm, kc, vc, om, None, mem_len, c, t, ws, flags, 0.0, stream)
