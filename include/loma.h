@@ -14,6 +14,8 @@
  *   loma_decode_attn_ragged, loma_compress_step_ragged
  *                          the two generation steps for batches whose sequences
  *                          stand at different points of their chunks
+ *   loma_decode_attn_paged, loma_compress_step_paged
+ *                          the same over a pool of cache pages and a block table
  *   loma_decode_attn       one generated token over the compressed cache
  *                          (Section 3.1 steps 1 and 3; Appendix A, inference_input)
  *   loma_compress_step     the t <m> queries over the uncompressed tail, fused
@@ -348,6 +350,24 @@ LOMA_API int loma_decode_attn_paged(const void* q, const void* k_new, const void
                                     const int32_t* cache_lens, int max_cache_len,
                                     loma_dtype dtype, float softmax_scale, unsigned flags,
                                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------
+ * loma_compress_step_paged -- loma_compress_step_ragged over the paged cache of
+ * loma_decode_attn_paged: sequence b (when mem_lens[b] >= 0) reads its tail from slots
+ * [mem_lens[b], mem_lens[b] + tc) through the block table and its t memory keys and values are
+ * written over slots [mem_lens[b], mem_lens[b] + t), wherever their pages lie.  Afterwards the
+ * sequence's valid length is mem_lens[b] + t; pages that hold only slots beyond it can go back to
+ * the caller's allocator (the library never touches the table).
+ * Default mask only (LOMA_FLAG_MEM_SEES_PRIOR_MEM returns UNSUPPORTED).  No workspace.
+ * Requires max_mem_len + tc <= max_pages * page_size.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CAPACITY, CUDA.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_compress_step_paged(const void* q_mem, const void* k_mem, const void* v_mem,
+                                      void* k_pool, void* v_pool, const int32_t* block_table,
+                                      void* o_mem, float* lse, int B, int H, int D,
+                                      int page_size, int max_pages, int n_pages,
+                                      const int32_t* mem_lens, int max_mem_len, int c, int t, int tc,
+                                      loma_dtype dtype, float softmax_scale, unsigned flags, void* stream);
 
 /* ---------------------------------------------------------------------------
  * loma_decode_attn_static -- the same decode step as loma_decode_attn (bf16

@@ -40,5 +40,6 @@ from .loma_oracle import (  # noqa: F401
     paged_to_contiguous,
     compress_step,
     compress_step_ragged,
+    compress_step_paged,
     replay_generation,
 )

@@ -597,6 +597,28 @@ def compress_step_ragged(q_mem, k_mem, v_mem, k_cache, v_cache, mem_lens, c, t, 
     return o, lse, kc, vc
 
 
+def compress_step_paged(q_mem, k_mem, v_mem, k_pool, v_pool, block_table, mem_lens, c, t, scale=None):
+    """compress_step_ragged over a paged cache: read the logical caches out of the pools, compress per sequence,
+    write the t new memory entries of every compressing sequence back into their pages.
+    Returns (o_mem, lse, k_pool', v_pool')."""
+    k_pool, v_pool = np.asarray(k_pool), np.asarray(v_pool)
+    ps = k_pool.shape[2]
+    cap = max(int(n) for n in mem_lens) + c * t
+    kc = paged_to_contiguous(k_pool, block_table, cap)
+    vc = paged_to_contiguous(v_pool, block_table, cap)
+    o, lse, kc2, vc2 = compress_step_ragged(q_mem, k_mem, v_mem, kc, vc, mem_lens, c, t, scale)
+    kp, vp = k_pool.copy(), v_pool.copy()
+    for b, n in enumerate(mem_lens):
+        n = int(n)
+        if n < 0:
+            continue
+        for j in range(n, n + t):
+            page = int(block_table[b][j // ps])
+            kp[page, :, j % ps] = kc2[b, :, j]
+            vp[page, :, j % ps] = vc2[b, :, j]
+    return o, lse, kp, vp
+
+
 def replay_generation(q, k, v, n_chunks, c, t, tail_read=0, flags=0, scale=None):
     """Run the laid-out sequence through the generation path chunk by chunk.
 

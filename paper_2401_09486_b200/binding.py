@@ -49,6 +49,7 @@ SIGNATURES = {
     "loma_compress_step": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz,
                                 _p]),
     "loma_compress_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _u]),
+    "loma_compress_step_paged": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _p, _i, _i, _i, _i, _i, _f, _u, _p]),
     "loma_compress_step_ragged": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _p, _i, _i, _i, _i, _i, _f, _u, _p]),
     "loma_device_status": (_i, [_p]),
     "loma_selftest_bounded_wait": (_i, [_p]),
@@ -334,6 +335,23 @@ def loma_compress_step_ragged(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse,
                                          _ptr(lse), B, H, D, cap, _ptr(mem_lens), int(max_mem_len), c, t, c * t,
                                          _dtype_code(q_mem), float(softmax_scale), int(flags), _stream(stream))
     _check(rc, "loma_compress_step_ragged")
+
+
+def loma_compress_step_paged(q_mem, k_mem, v_mem, k_pool, v_pool, block_table, o_mem, lse, mem_lens, max_mem_len: int,
+                             c: int, t: int, flags: int = 0, softmax_scale: float = 0.0, stream=None) -> None:
+    """Ragged compress over a paged cache (pools [n_pages, H, page_size, D], block_table int32 [B, max_pages])."""
+    n_pages, H, page_size, D = k_pool.shape
+    B, max_pages = block_table.shape
+    for x in (q_mem, k_mem, v_mem, k_pool, v_pool, o_mem, mem_lens, block_table):
+        if not x.is_contiguous():
+            raise ValueError("compress tensors must be contiguous")
+    if block_table.dtype != torch.int32 or mem_lens.dtype != torch.int32 or mem_lens.numel() != B:
+        raise ValueError("block_table must be int32 [B, max_pages] and mem_lens int32 [B]")
+    rc = lib().loma_compress_step_paged(_ptr(q_mem), _ptr(k_mem), _ptr(v_mem), _ptr(k_pool), _ptr(v_pool), _ptr(block_table),
+                                        _ptr(o_mem), _ptr(lse), B, H, D, page_size, max_pages, n_pages, _ptr(mem_lens),
+                                        int(max_mem_len), c, t, c * t, _dtype_code(q_mem), float(softmax_scale), int(flags),
+                                        _stream(stream))
+    _check(rc, "loma_compress_step_paged")
 
 
 def loma_compress_workspace_bytes(B: int, H: int, D: int, t: int, mem_len: int, flags: int = 0) -> int:

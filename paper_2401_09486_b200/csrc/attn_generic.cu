@@ -281,16 +281,23 @@ decode_generic_kernel(const T* __restrict__ q, const T* __restrict__ k_new, cons
 // ------------------------------------------------------------- compress map
 template <typename T>
 struct CompressMap {
-    const T* kc;   // cache row `lo`
+    const T* kc;   // the (b,h)'s cache (contiguous) or the pool (paged)
     const T* vc;
     const T* km;   // this (b,h)'s t memory keys
     const T* vm;
-    int n_cache, D;
+    int lo, n_cache, D;   // visible cache slots [lo, lo + n_cache)
+    Paging pg;
+    int b, h, H;
+    __device__ __forceinline__ int64_t slot(int j) const {
+        if (!pg.table) return (int64_t)j * D;
+        const int page = min(max(pg.table[(int64_t)b * pg.max_pages + (j >> pg.log2_ps)], 0), pg.n_pages - 1);
+        return ((((int64_t)page * H + h) << pg.log2_ps) + (j & ((1 << pg.log2_ps) - 1))) * D;
+    }
     __device__ __forceinline__ const T* kptr(int vi) const {
-        return vi < n_cache ? kc + (int64_t)vi * D : km + (int64_t)(vi - n_cache) * D;
+        return vi < n_cache ? kc + slot(lo + vi) : km + (int64_t)(vi - n_cache) * D;
     }
     __device__ __forceinline__ const T* vptr(int vi) const {
-        return vi < n_cache ? vc + (int64_t)vi * D : vm + (int64_t)(vi - n_cache) * D;
+        return vi < n_cache ? vc + slot(lo + vi) : vm + (int64_t)(vi - n_cache) * D;
     }
 };
 
@@ -302,7 +309,7 @@ __global__ void __launch_bounds__(GENERIC_WARPS * 32)
 compress_generic_kernel(const T* __restrict__ q_mem, const T* __restrict__ k_mem,
                         const T* __restrict__ v_mem, T* __restrict__ k_cache, T* __restrict__ v_cache,
                         T* __restrict__ o_mem, float* __restrict__ lse, int cap, int mem_len, const int32_t* __restrict__ mem_lens,
-                        int H, int t, int tc, unsigned flags, float scale) {
+                        int H, int t, int tc, unsigned flags, float scale, Paging pg) {
     __shared__ __align__(16) float q_sh[GENERIC_WARPS][D];
     const int bh = blockIdx.x;
     if (mem_lens) {                          // ragged batch: own count of memory entries; negative = not compressing now
@@ -311,13 +318,14 @@ compress_generic_kernel(const T* __restrict__ q_mem, const T* __restrict__ k_mem
         mem_len = min(own, mem_len);
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    T* kc = k_cache + (int64_t)bh * cap * D;
-    T* vc = v_cache + (int64_t)bh * cap * D;
+    T* kc = pg.table ? k_cache : k_cache + (int64_t)bh * cap * D;
+    T* vc = pg.table ? v_cache : v_cache + (int64_t)bh * cap * D;
     const int lo = (flags & LOMA_FLAG_MEM_SEES_PRIOR_MEM) ? 0 : mem_len;
     CompressMap<T> map;
-    map.kc = kc + (int64_t)lo * D; map.vc = vc + (int64_t)lo * D;
+    map.kc = kc; map.vc = vc; map.lo = lo;
     map.km = k_mem + (int64_t)bh * t * D; map.vm = v_mem + (int64_t)bh * t * D;
     map.n_cache = mem_len + tc - lo; map.D = D;
+    map.pg = pg; map.b = bh / H; map.h = bh - map.b * H; map.H = H;
     for (int j = warp; j < t; j += GENERIC_WARPS) {
         stage_query<T, D>(q_sh[warp], q_mem + ((int64_t)bh * t + j) * D, lane);
         attend_row<T, D>(q_sh[warp], map, map.n_cache + t, scale, o_mem + ((int64_t)bh * t + j) * D,
@@ -327,14 +335,14 @@ compress_generic_kernel(const T* __restrict__ q_mem, const T* __restrict__ k_mem
     __syncthreads();
     // compaction: 16-byte vector copies, bit for bit
     constexpr int VEC = 16 / sizeof(T);
-    const int nvec = t * D / VEC;
+    constexpr int VPR = D / VEC;             // 16-byte vectors per row
     const uint4* ksrc = reinterpret_cast<const uint4*>(map.km);
     const uint4* vsrc = reinterpret_cast<const uint4*>(map.vm);
-    uint4* kdst = reinterpret_cast<uint4*>(kc + (int64_t)mem_len * D);
-    uint4* vdst = reinterpret_cast<uint4*>(vc + (int64_t)mem_len * D);
-    for (int e = threadIdx.x; e < nvec; e += blockDim.x) {
-        kdst[e] = ksrc[e];
-        vdst[e] = vsrc[e];
+    for (int e = threadIdx.x; e < t * VPR; e += blockDim.x) {
+        const int r = e / VPR, cv = e - r * VPR;
+        const int64_t off = map.slot(mem_len + r) + cv * VEC;
+        *reinterpret_cast<uint4*>(kc + off) = ksrc[e];
+        *reinterpret_cast<uint4*>(vc + off) = vsrc[e];
     }
 }
 
@@ -580,10 +588,10 @@ cudaError_t launch_decode_generic(const void* q, const void* k_new, const void* 
 template <typename T, int D>
 static cudaError_t compress_generic_t(const void* qm, const void* km, const void* vm, void* kc, void* vc,
                                       void* om, float* lse, int BH, int cap, int mem_len, const int32_t* mem_lens, int H, int t,
-                                      int tc, unsigned flags, float scale, cudaStream_t st) {
+                                      int tc, unsigned flags, float scale, const Paging& pg, cudaStream_t st) {
     compress_generic_kernel<T, D><<<BH, GENERIC_WARPS * 32, 0, st>>>(
         static_cast<const T*>(qm), static_cast<const T*>(km), static_cast<const T*>(vm), static_cast<T*>(kc),
-        static_cast<T*>(vc), static_cast<T*>(om), lse, cap, mem_len, mem_lens, H, t, tc, flags, scale);
+        static_cast<T*>(vc), static_cast<T*>(om), lse, cap, mem_len, mem_lens, H, t, tc, flags, scale, pg);
     count_launches(1);
     return cudaGetLastError();
 }
@@ -591,18 +599,18 @@ static cudaError_t compress_generic_t(const void* qm, const void* km, const void
 cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache,
                                     void* v_cache, void* o_mem, float* lse, int B, int H, int D, int cap,
                                     int mem_len, const int32_t* mem_lens, int c, int t, loma_dtype dt, float scale,
-                                    unsigned flags, cudaStream_t st) {
+                                    unsigned flags, const Paging& pg, cudaStream_t st) {
     const int BH = B * H, tc = c * t;
     if (dt == LOMA_F32) {
         return D == 64 ? compress_generic_t<float, 64>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH,
-                                                       cap, mem_len, mem_lens, H, t, tc, flags, scale, st)
+                                                       cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st)
                        : compress_generic_t<float, 128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH,
-                                                        cap, mem_len, mem_lens, H, t, tc, flags, scale, st);
+                                                        cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st);
     }
     return D == 64 ? compress_generic_t<__nv_bfloat16, 64>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse,
-                                                           BH, cap, mem_len, mem_lens, H, t, tc, flags, scale, st)
+                                                           BH, cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st)
                    : compress_generic_t<__nv_bfloat16, 128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse,
-                                                            BH, cap, mem_len, mem_lens, H, t, tc, flags, scale, st);
+                                                            BH, cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st);
 }
 
 }  // namespace loma

@@ -101,7 +101,7 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
                     const __nv_bfloat16* __restrict__ v_mem, __nv_bfloat16* __restrict__ k_cache,
                     __nv_bfloat16* __restrict__ v_cache, __nv_bfloat16* __restrict__ o_mem, float* __restrict__ lse,
                     float* __restrict__ ws, int BH, int cap, int mem_len_all, const int32_t* __restrict__ mem_lens, int H,
-                    int t, int tc, int nprior, int prior_len, int mtiles, float scale_log2) {
+                    int t, int tc, int nprior, int prior_len, int mtiles, float scale_log2, Paging pg) {
     using SM = CmpSmem<D>;
     constexpr int ROWB = SM::ROWB;
     constexpr int VPR = D / 8;                 // 16-byte vectors per row
@@ -125,8 +125,15 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;
 
-    const __nv_bfloat16* kc = k_cache + (int64_t)bh * cap * D;
-    const __nv_bfloat16* vc = v_cache + (int64_t)bh * cap * D;
+    // cache slot j of this (b,h) -> element offset from k_cache / v_cache (through the block table when the cache is paged)
+    const int pb = bh / H, phd = bh - pb * H;
+    auto cache_row = [&](int j) -> int64_t {
+        if (!pg.table) return ((int64_t)bh * cap + j) * D;
+        const int page = min(max(__ldg(pg.table + (int64_t)pb * pg.max_pages + (j >> pg.log2_ps)), 0), pg.n_pages - 1);
+        return ((((int64_t)page * H + phd) << pg.log2_ps) + (j & ((1 << pg.log2_ps) - 1))) * D;
+    };
+    const __nv_bfloat16* kc = k_cache;
+    const __nv_bfloat16* vc = v_cache;
     const __nv_bfloat16* km = k_mem + (int64_t)bh * t * D;
     const __nv_bfloat16* vm = v_mem + (int64_t)bh * t * D;
     // key i of this CTA's range -> source row
@@ -142,7 +149,7 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
             const bool valid = i < nkeys;
             const int ic = valid ? i : 0;
             const __nv_bfloat16 *ksrc, *vsrc;
-            if (ic < n_cache_rows) { ksrc = kc + (int64_t)(k0 + ic) * D; vsrc = vc + (int64_t)(k0 + ic) * D; }
+            if (ic < n_cache_rows) { const int64_t off = cache_row(k0 + ic); ksrc = kc + off; vsrc = vc + off; }
             else { ksrc = km + (int64_t)(ic - n_cache_rows) * D; vsrc = vm + (int64_t)(ic - n_cache_rows) * D; }
             cp_async16(kdst + r * ROWB + cv * 16, ksrc + cv * 8, valid);
             cp_async16(vdst + r * ROWB + cv * 16, vsrc + cv * 8, valid);
@@ -317,11 +324,11 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
         __syncthreads();
         const uint4* ksrc = reinterpret_cast<const uint4*>(km);
         const uint4* vsrc = reinterpret_cast<const uint4*>(vm);
-        uint4* kdst = reinterpret_cast<uint4*>(k_cache + ((int64_t)bh * cap + mem_len) * D);
-        uint4* vdst = reinterpret_cast<uint4*>(v_cache + ((int64_t)bh * cap + mem_len) * D);
         for (int e = threadIdx.x; e < t * VPR; e += CMP_WARPS * 32) {
-            kdst[e] = __ldg(ksrc + e);
-            vdst[e] = __ldg(vsrc + e);
+            const int r = e / VPR, cv = e - r * VPR;
+            const int64_t off = cache_row(mem_len + r) + cv * 8;
+            *reinterpret_cast<uint4*>(k_cache + off) = __ldg(ksrc + e);
+            *reinterpret_cast<uint4*>(v_cache + off) = __ldg(vsrc + e);
         }
     }
 }
@@ -354,7 +361,7 @@ compress_merge_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ 
 template <int D>
 __global__ void compaction_kernel(const __nv_bfloat16* __restrict__ k_mem, const __nv_bfloat16* __restrict__ v_mem,
                                   __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache, int cap,
-                                  int mem_len, const int32_t* __restrict__ mem_lens, int H, int t) {
+                                  int mem_len, const int32_t* __restrict__ mem_lens, int H, int t, Paging pg) {
     const int bh = blockIdx.x;
     if (mem_lens) {
         const int own = __ldg(mem_lens + bh / H);
@@ -364,18 +371,25 @@ __global__ void compaction_kernel(const __nv_bfloat16* __restrict__ k_mem, const
     constexpr int VPR = D / 8;
     const uint4* ksrc = reinterpret_cast<const uint4*>(k_mem + (int64_t)bh * t * D);
     const uint4* vsrc = reinterpret_cast<const uint4*>(v_mem + (int64_t)bh * t * D);
-    uint4* kdst = reinterpret_cast<uint4*>(k_cache + ((int64_t)bh * cap + mem_len) * D);
-    uint4* vdst = reinterpret_cast<uint4*>(v_cache + ((int64_t)bh * cap + mem_len) * D);
+    const int pb = bh / H, phd = bh - pb * H;
     for (int e = threadIdx.x; e < t * VPR; e += blockDim.x) {
-        kdst[e] = __ldg(ksrc + e);
-        vdst[e] = __ldg(vsrc + e);
+        const int r = e / VPR, cv = e - r * VPR, j = mem_len + r;
+        int64_t off;
+        if (!pg.table) {
+            off = ((int64_t)bh * cap + j) * D;
+        } else {
+            const int page = min(max(__ldg(pg.table + (int64_t)pb * pg.max_pages + (j >> pg.log2_ps)), 0), pg.n_pages - 1);
+            off = ((((int64_t)page * H + phd) << pg.log2_ps) + (j & ((1 << pg.log2_ps) - 1))) * D;
+        }
+        *reinterpret_cast<uint4*>(k_cache + off + cv * 8) = __ldg(ksrc + e);
+        *reinterpret_cast<uint4*>(v_cache + off + cv * 8) = __ldg(vsrc + e);
     }
 }
 
 template <int D>
 static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* vm, void* kc, void* vc, void* om,
                                    float* lse, int BH, int cap, int mem_len, const int32_t* mem_lens, int H, int t, int tc,
-                                   unsigned flags, float scale, void* ws, cudaStream_t st) {
+                                   unsigned flags, float scale, void* ws, const Paging& pg, cudaStream_t st) {
     const int nprior = compress_num_prior(BH, mem_len, flags);
     int prior_len = 0;
     if (nprior > 0) prior_len = ((mem_len + nprior - 1) / nprior + 15) / 16 * 16;
@@ -395,7 +409,7 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
         static_cast<const __nv_bfloat16*>(qm), static_cast<const __nv_bfloat16*>(km),
         static_cast<const __nv_bfloat16*>(vm), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
         static_cast<__nv_bfloat16*>(om), lse, static_cast<float*>(ws), BH, cap, mem_len, mem_lens, H, t, tc, nprior,
-        prior_len, mtiles, scale * 1.4426950408889634f);
+        prior_len, mtiles, scale * 1.4426950408889634f, pg);
     count_launches(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -409,7 +423,7 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
     if (mtiles > 1) {
         compaction_kernel<D><<<BH, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(km),
                                                   static_cast<const __nv_bfloat16*>(vm), static_cast<__nv_bfloat16*>(kc),
-                                                  static_cast<__nv_bfloat16*>(vc), cap, mem_len, mem_lens, H, t);
+                                                  static_cast<__nv_bfloat16*>(vc), cap, mem_len, mem_lens, H, t, pg);
         count_launches(1);
         e = cudaGetLastError();
     }
@@ -420,12 +434,12 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
 cudaError_t launch_compress_bf16(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
                                  void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len,
                                  const int32_t* mem_lens, int c, int t, unsigned flags, float scale, void* ws,
-                                 cudaStream_t st) {
+                                 const Paging& pg, cudaStream_t st) {
     const int BH = B * H, tc = c * t;
     return D == 64 ? compress_bf16_t<64>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH, cap, mem_len, mem_lens, H, t,
-                                         tc, flags, scale, ws, st)
+                                         tc, flags, scale, ws, pg, st)
                    : compress_bf16_t<128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH, cap, mem_len, mem_lens, H, t,
-                                          tc, flags, scale, ws, st);
+                                          tc, flags, scale, ws, pg, st);
 }
 
 }  // namespace loma

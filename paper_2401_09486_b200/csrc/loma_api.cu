@@ -398,6 +398,41 @@ int loma_decode_attn_paged(const void* q, const void* k_new, const void* v_new, 
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 
+int loma_compress_step_paged(const void* q_mem, const void* k_mem, const void* v_mem, void* k_pool, void* v_pool,
+                             const int32_t* block_table, void* o_mem, float* lse, int B, int H, int D, int page_size,
+                             int max_pages, int n_pages, const int32_t* mem_lens, int max_mem_len, int c, int t, int tc,
+                             loma_dtype dtype, float softmax_scale, unsigned flags, void* stream) {
+    if (B < 0 || H < 0 || max_pages < 0 || n_pages < 0 || max_mem_len < 0 || c < 1 || t < 1) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)c * t != (int64_t)tc) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    if (flags & LOMA_FLAG_MEM_SEES_PRIOR_MEM) return LOMA_ERR_UNSUPPORTED;
+    const int l2 = log2_exact(page_size);
+    if (l2 < 0 || page_size > 65536) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)max_mem_len + tc > (int64_t)max_pages * page_size) return LOMA_ERR_CAPACITY;
+    if (B == 0 || H == 0) return LOMA_OK;
+    if (!q_mem || !k_mem || !v_mem || !k_pool || !v_pool || !o_mem || !mem_lens || !block_table || n_pages < 1)
+        return LOMA_ERR_INVALID_ARG;
+    if (!aligned16(q_mem) || !aligned16(k_mem) || !aligned16(v_mem) || !aligned16(k_pool) || !aligned16(v_pool) ||
+        !aligned16(o_mem) || ((uintptr_t)mem_lens & 3u) || ((uintptr_t)block_table & 3u))
+        return LOMA_ERR_ALIGNMENT;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if ((int64_t)B * H * 256 > INT_MAX) return LOMA_ERR_INVALID_ARG;
+    Paging pg;
+    pg.table = block_table; pg.max_pages = max_pages; pg.log2_ps = l2; pg.n_pages = n_pages;
+    cudaError_t e;
+    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC) && t <= 128)
+        e = launch_compress_bf16(q_mem, k_mem, v_mem, k_pool, v_pool, o_mem, lse, B, H, D, 0, max_mem_len, mem_lens, c, t, flags,
+                                 scale, nullptr, pg, st);
+    else
+        e = launch_compress_generic(q_mem, k_mem, v_mem, k_pool, v_pool, o_mem, lse, B, H, D, 0, max_mem_len, mem_lens, c, t,
+                                    dtype, scale, flags, pg, st);
+    return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
 size_t loma_decode_static_scratch_bytes(void) { return decode_static_scratch_bytes(); }
 
 int loma_decode_attn_static(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
@@ -453,10 +488,10 @@ int loma_compress_step(const void* q_mem, const void* k_mem, const void* v_mem, 
     cudaError_t e;
     if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC) && t <= 128)
         e = launch_compress_bf16(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, mem_len, nullptr, c, t,
-                                 flags, scale, workspace, st);
+                                 flags, scale, workspace, Paging{}, st);
     else
         e = launch_compress_generic(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, mem_len, nullptr, c,
-                                    t, dtype, scale, flags, st);
+                                    t, dtype, scale, flags, Paging{}, st);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 
@@ -483,10 +518,10 @@ int loma_compress_step_ragged(const void* q_mem, const void* k_mem, const void* 
     cudaError_t e;
     if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC) && t <= 128)
         e = launch_compress_bf16(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, max_mem_len, mem_lens, c, t,
-                                 flags, scale, nullptr, st);
+                                 flags, scale, nullptr, Paging{}, st);
     else
         e = launch_compress_generic(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, max_mem_len, mem_lens,
-                                    c, t, dtype, scale, flags, st);
+                                    c, t, dtype, scale, flags, Paging{}, st);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 

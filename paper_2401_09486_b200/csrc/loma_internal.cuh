@@ -126,12 +126,12 @@ size_t compress_workspace_bytes(int BH, int D, int t, int mem_len, unsigned flag
 cudaError_t launch_compress_bf16(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
                                  void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len,
                                  const int32_t* mem_lens, int c, int t, unsigned flags, float scale, void* ws,
-                                 cudaStream_t st);   // mem_lens: per-sequence counts (default variant only) or NULL
+                                 const Paging& pg, cudaStream_t st);   // mem_lens: per-sequence counts (default variant only) or NULL
 
 cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const void* v_mem,
                                     void* k_cache, void* v_cache, void* o_mem, float* lse,
                                     int B, int H, int D, int cap, int mem_len, const int32_t* mem_lens, int c, int t,
-                                    loma_dtype dt, float scale, unsigned flags, cudaStream_t st);
+                                    loma_dtype dt, float scale, unsigned flags, const Paging& pg, cudaStream_t st);
 
 // rotary embedding of Q and K rows at the layout's position ids (rope.cu)
 cudaError_t launch_rope(void* q, void* k, int B, int H, int D, const Layout& L, int64_t sb, int64_t sh, int64_t ss,

@@ -302,3 +302,17 @@ def test_paged_decode_validation(lib):
     assert call(bt=0x6002) == ALIGNMENT
     assert call(D=100) == UNSUPPORTED
     assert call(B=0) == 0
+
+
+def test_paged_compress_validation(lib):
+    def call(qm=0x1000, km=0x2000, vm=0x3000, kp=0x4000, vp=0x5000, bt=0x6000, om=0x7000, B=2, H=1, D=128, ps=16, mp=8,
+             npg=16, lens=0x8000, mx=16, c=4, t=16, tc=64, dt=1, flags=0):
+        return lib.loma_compress_step_paged(qm, km, vm, kp, vp, bt, om, None, B, H, D, ps, mp, npg, lens, mx, c, t, tc, dt,
+                                            0.0, flags, None)
+    assert call(mx=65) == CAPACITY                      # tail would run past the table
+    assert call(ps=48) == INVALID
+    assert call(tc=63) == INVALID
+    assert call(bt=None) == INVALID
+    assert call(flags=1) == UNSUPPORTED
+    assert call(lens=0x8002) == ALIGNMENT
+    assert call(B=0) == 0

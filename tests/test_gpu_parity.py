@@ -401,6 +401,36 @@ def test_paged_decode_matches_oracle(H, D, ps, lens, flags, dtype):
     assert np.array_equal(npf(kpd), want_k) and np.array_equal(npf(vpd), want_v)
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, GENERIC])
+@pytest.mark.parametrize("H,D,c,t,ps,lens", [(2, 64, 4, 4, 16, [0, 16, -1, 8]), (2, 128, 4, 16, 64, [48, -1, 1024, 0, 500]),
+                                             (1, 128, 2, 64, 32, [128, 70, -1]), (2, 128, 8, 16, 256, [8192, 4090, -1, 16])])
+def test_paged_compress_matches_oracle(H, D, c, t, ps, lens, flags, dtype):
+    """Tails and rewritten slots that straddle pages of a shuffled pool; idle sequences and unused pages untouched."""
+    B, tc = len(lens), c * t
+    max_len = max(lens)
+    max_pages = (max_len + tc + ps - 1) // ps
+    n_pages = B * max_pages + 2
+    table = np.random.default_rng(9).permutation(n_pages)[: B * max_pages].reshape(B, max_pages).astype(np.int32)
+    kp = synthetic.normal_tensor((n_pages, H, ps, D), 61, 1.0, dtype)
+    vp = synthetic.normal_tensor((n_pages, H, ps, D), 62, 1.0, dtype)
+    qm, km, vm = synthetic.qkv(B, H, t, D, seed=63, std=1.0, dtype=dtype)
+    want_o, want_lse, want_k, want_v = oracle.compress_step_paged(npf(qm), npf(km), npf(vm), npf(kp), npf(vp), table, lens, c, t)
+    kpd, vpd = kp.to(DEV), vp.to(DEV)
+    om = torch.full((B, H, t, D), 7.0, dtype=dtype, device=DEV)
+    lse = torch.full((B, H, t), 7.0, dtype=torch.float32, device=DEV)
+    L.loma_compress_step_paged(qm.to(DEV), km.to(DEV), vm.to(DEV), kpd, vpd, torch.from_numpy(table).to(DEV), om, lse,
+                               torch.tensor(lens, dtype=torch.int32, device=DEV), max_len, c, t, flags)
+    torch.cuda.synchronize()
+    for b, n in enumerate(lens):
+        if n < 0:
+            assert float((om[b].float() - 7.0).abs().max()) == 0.0
+            continue
+        check_close(om[b:b + 1], want_o[b:b + 1], dtype)
+        assert np.abs(npf(lse[b]) - want_lse[b]).max() <= (1e-5 if dtype == torch.float32 else 2e-2)
+    assert np.array_equal(npf(kpd), want_k) and np.array_equal(npf(vpd), want_v)      # pools differ in the rewritten slots only
+
+
 def test_bounded_wait_times_out_and_leaves_the_context_usable():
     """A device-side wait that can never be satisfied gives up after its limit,
     reports LOMA_ERR_TIMEOUT through the status word, and later launches work."""

@@ -660,3 +660,28 @@ def test_paged_decode_is_contiguous_decode_through_the_block_table():
     kq[perm], vq[perm] = kp, vp
     o_q, _, _, _ = oracle.decode_attn_paged(q, kn, vn, kq, vq, perm[table], lens)
     assert np.array_equal(o_q, o_p)
+
+
+def test_paged_compress_is_ragged_compress_through_the_block_table():
+    B, H, D, c, t, ps, max_pages = 3, 2, 8, 2, 2, 4, 5
+    tc, cap = c * t, 4 * 5
+    kc, vc = _rand((B, H, cap, D), 95), _rand((B, H, cap, D), 96)
+    qm, km, vm = _rand((B, H, t, D), 97), _rand((B, H, t, D), 98), _rand((B, H, t, D), 99)
+    lens = [3, -1, 14]                                   # slots [3, 5) and [14, 16) straddle no page / end a page
+    n_pages = B * max_pages + 1
+    kp, vp = np.full((n_pages, H, ps, D), np.nan), np.full((n_pages, H, ps, D), np.nan)
+    table = np.random.default_rng(1).permutation(n_pages)[: B * max_pages].reshape(B, max_pages).astype(np.int32)
+    for b in range(B):
+        for p_ in range(max_pages):
+            kp[table[b, p_]] = kc[b, :, p_ * ps:(p_ + 1) * ps]
+            vp[table[b, p_]] = vc[b, :, p_ * ps:(p_ + 1) * ps]
+    o_r, l_r, k_r, v_r = oracle.compress_step_ragged(qm, km, vm, kc, vc, lens, c, t)
+    o_p, l_p, kp2, vp2 = oracle.compress_step_paged(qm, km, vm, kp, vp, table, lens, c, t)
+    assert np.array_equal(o_r[[0, 2]], o_p[[0, 2]]) and np.isnan(o_p[1]).all()
+    back = oracle.paged_to_contiguous(kp2, table, cap)
+    for b, n in enumerate(lens):
+        if n >= 0:
+            assert np.array_equal(back[b, :, :n + t], k_r[b, :, :n + t])
+    unused = np.setdiff1d(np.arange(n_pages), table.ravel())
+    assert np.isnan(kp2[unused]).all()
+    assert np.array_equal(kp2[table[1]], kp[table[1]])   # the idle sequence's pages are untouched
