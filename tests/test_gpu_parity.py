@@ -242,6 +242,66 @@ def test_incremental_generation_equals_one_shot(B, H, D, n, c, t, tail, flags, d
     assert torch.equal(vc[:, :, :length].cpu(), v[:, :, rows])
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_staggered_sequences_over_a_paged_cache_equal_the_one_shot_forward(dtype):
+    """Invariant (c) through the ragged and paged entry points: three sequences that started 0, 5 and 11 tokens
+    apart share one pool of pages; every step decodes one token of every sequence that still has tokens, and a
+    sequence compresses as soon as its tail holds tc tokens, whatever the others are doing.  Every live row of the
+    one-shot forward of each sequence is reproduced."""
+    H, D, n, c, t, tail, ps = 2, 128, 3, 2, 8, 5, 16
+    tc, s = c * t, oracle.chunk_len(c, t)
+    S = oracle.seq_len(n, c, t, tail)
+    B, starts = 3, [0, 5, 11]
+    q, k, v = synthetic.qkv(B, H, S, D, seed=91, std=1.0, dtype=dtype)
+    want_o, _ = oracle.masked_attn_fwd(npf(q), npf(k), npf(v), n, c, t, tail)
+    zone = oracle.layout_index(n, c, t, tail)[1]
+    gen_rows = [i for i in range(S) if zone[i] == oracle.ZONE_READ]          # tokens decoded one at a time, in order
+    max_pages = (n * t + tc + ps - 1) // ps + 1
+    n_pages = B * max_pages
+    table = np.random.default_rng(3).permutation(n_pages).reshape(B, max_pages).astype(np.int32)
+    kpool = torch.zeros((n_pages, H, ps, D), dtype=dtype, device=DEV)
+    vpool = torch.zeros_like(kpool)
+    table_d = torch.from_numpy(table).to(DEV)
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    got = torch.full((B, H, S, D), float("nan"), dtype=dtype, device=DEV)
+    ws = workspace(L.loma_decode_workspace_bytes(B, H, D, n * t + tc))
+    pos = [0] * B            # next entry of gen_rows per sequence
+    lens = [0] * B           # cache entries per sequence
+    chunks = [0] * B
+    step = 0
+    while any(p_ < len(gen_rows) for p_ in pos):
+        active = [step >= starts[b] and pos[b] < len(gen_rows) for b in range(B)]
+        rows = [gen_rows[min(pos[b], len(gen_rows) - 1)] for b in range(B)]
+        take = lambda x: torch.stack([x[b, :, rows[b]:rows[b] + 1] for b in range(B)]).contiguous()
+        o1 = torch.empty((B, H, 1, D), dtype=dtype, device=DEV)
+        # idle sequences decode a throw-away token into a spare slot of their own pages (their length does not advance)
+        lens_d = torch.tensor(lens, dtype=torch.int32, device=DEV)
+        L.loma_decode_attn_paged(take(qd), take(kd), take(vd), kpool, vpool, table_d, o1, None, lens_d, max(lens), ws)
+        for b in range(B):
+            if active[b]:
+                got[b, :, rows[b]] = o1[b, :, 0]
+                pos[b] += 1
+                lens[b] += 1
+        # compress every sequence whose tail is full
+        mem_lens = [chunks[b] * t if (lens[b] == chunks[b] * t + tc and chunks[b] < n) else -1 for b in range(B)]
+        if any(m >= 0 for m in mem_lens):
+            m_rows = [chunks[b] * s + tc for b in range(B)]
+            takem = lambda x: torch.stack([x[b, :, m_rows[b]:m_rows[b] + t] if mem_lens[b] >= 0 else x[b, :, :t]
+                                           for b in range(B)]).contiguous()
+            om = torch.empty((B, H, t, D), dtype=dtype, device=DEV)
+            L.loma_compress_step_paged(takem(qd), takem(kd), takem(vd), kpool, vpool, table_d, om, None,
+                                       torch.tensor(mem_lens, dtype=torch.int32, device=DEV), max(mem_lens), c, t)
+            for b in range(B):
+                if mem_lens[b] >= 0:
+                    got[b, :, m_rows[b]:m_rows[b] + t] = om[b]
+                    chunks[b] += 1
+                    lens[b] = chunks[b] * t
+        step += 1
+    torch.cuda.synchronize()
+    live = torch.from_numpy(zone != oracle.ZONE_REP).to(DEV)
+    check_close(got[:, :, live], want_o[:, :, zone != oracle.ZONE_REP], dtype)
+
+
 # ------------------------------------------------------------- decode, compress
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
