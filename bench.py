@@ -354,8 +354,9 @@ def run_ours(args):
             {"kernel": "masked_attn_tc_kernel<128>", "workload": "4608-token layout", "bound": "hbm",
              "achieved": fwd_bytes / (t_fwd * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
              "frac": fwd_bytes / (t_fwd * 1e-3) / 1e9 / peaks["hbm_gbs"],
-             # dram__bytes.sum of one launch on one batch element of this layout (profiles/masked_attn_tc_small_cases.md) x B
-             "traffic": 151.1e6 * f["B"],
+             # dram__bytes_read.sum + dram__bytes_write.sum of one launch on one batch element of this layout
+             # (profiles/masked_attn_tc_small_cases.md) x B
+             "traffic": 142.2e6 * f["B"],
              "tensor_frac_of_measured_bf16_useful": fwd_tflops / world / peaks["bf16_tflops"]},
             {"kernel": "compress_mma_kernel<128>", "workload": "B32 H32 mem 8192, default variant", "bound": "hbm",
              "achieved": cmp_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": cmp_gbs / peaks["hbm_gbs"],
