@@ -656,3 +656,24 @@ def test_generation_cycle_replays_from_a_cuda_graph():
         torch.cuda.synchronize()
         assert torch.equal(outs_g, outs_e) and torch.equal(om_g, om_e)
         assert torch.equal(kc_g[:, :, :mem_len + t], kc_e[:, :, :mem_len + t]) and torch.equal(vc_g[:, :, :mem_len + t], vc_e[:, :, :mem_len + t])
+
+
+def test_forwards_on_two_streams_at_once_do_not_disturb_each_other():
+    """The forward hands out tiles from a counter; launches get their counters round robin, so two launches in
+    flight on different streams must each produce exactly what they produce alone."""
+    B, H, D, n, c, t = 2, 8, 128, 12, 4, 16
+    S = oracle.seq_len(n, c, t)
+    a = [x.to(DEV) for x in synthetic.qkv(B, H, S, D, seed=101, dtype=torch.bfloat16)]
+    b = [x.to(DEV) for x in synthetic.qkv(B, H, S, D, seed=102, dtype=torch.bfloat16)]
+    alone_a, _ = run_fwd(*a, n, c, t)
+    alone_b, _ = run_fwd(*b, n, c, t)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    oa = [torch.empty_like(a[0]) for _ in range(6)]
+    ob = [torch.empty_like(b[0]) for _ in range(6)]
+    for i in range(6):
+        L.loma_masked_attn_fwd(*a, oa[i], None, n, c, t, 0, 0, 0.0, s1)
+        L.loma_masked_attn_fwd(*b, ob[i], None, n, c, t, 0, 0, 0.0, s2)
+    torch.cuda.synchronize()
+    for i in range(6):
+        assert torch.equal(oa[i], alone_a) and torch.equal(ob[i], alone_b)
