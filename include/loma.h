@@ -218,11 +218,16 @@ LOMA_API size_t loma_masked_attn_bwd_workspace_bytes(int B, int H, int D, int n_
  *     x'[d] = x[d] cos(p theta_d) - x[d+half] sin(p theta_d),
  *     x'[d+half] = x[d+half] cos(p theta_d) + x[d] sin(p theta_d),      d in [0, half).
  *
+ * Adding LOMA_ROPE_INVERSE (2) to position_type rotates by the opposite angle: the inverse, which is also the
+ * transpose, i.e. what the gradients of the rotated q and k need on their way back to the unrotated ones.
+ *
  *   q, k [device, in/out]  [B, H, S, D] with the strides of loma_masked_attn_fwd; either may be NULL
  *   theta_base             <= 0 selects 10000
  *   flags                  LOMA_FLAG_NO_REP_ZONE for the layout without repetition zones
  * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CUDA.  S == 0 or B*H == 0 is a no-op.
  * ------------------------------------------------------------------------- */
+enum { LOMA_ROPE_INVERSE = 2 };
+
 LOMA_API int loma_rope_apply(void* q, void* k, int B, int H, int D,
                              int n_chunks, int c, int t, int tc, int tail_read,
                              int64_t stride_b, int64_t stride_h, int64_t stride_s,

@@ -47,3 +47,26 @@ def loma_masked_attention(q, k, v, n_chunks: int, c: int, t: int, tail_read: int
     Returns O [B, H, S, D]; gradients flow to q, k and v through the library's backward kernels.
     """
     return _MaskedAttention.apply(q, k, v, n_chunks, c, t, tail_read, flags, softmax_scale)
+
+
+class _Rope(torch.autograd.Function):
+    @staticmethod
+    def forward(ctx, q, k, n_chunks, c, t, tail_read, flags, theta_base, position_type):
+        q, k = q.contiguous().clone(), k.contiguous().clone()
+        L.loma_rope_apply(q, k, n_chunks, c, t, tail_read, flags, theta_base, position_type)
+        ctx.layout = (n_chunks, c, t, tail_read, flags, theta_base, position_type)
+        return q, k
+
+    @staticmethod
+    def backward(ctx, dq, dk):
+        n_chunks, c, t, tail_read, flags, theta_base, position_type = ctx.layout
+        dq, dk = dq.contiguous().clone(), dk.contiguous().clone()
+        L.loma_rope_apply(dq, dk, n_chunks, c, t, tail_read, flags, theta_base, position_type | L.LOMA_ROPE_INVERSE)
+        return dq, dk, None, None, None, None, None, None, None
+
+
+def loma_rope(q, k, n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0, theta_base: float = 0.0,
+              position_type: int = 0):
+    """Rotary embedding of q and k at the layout's position ids as a differentiable torch op (out of place;
+    the gradient is the rotation by the opposite angle, run by the same kernel)."""
+    return _Rope.apply(q, k, n_chunks, c, t, tail_read, flags, theta_base, position_type)

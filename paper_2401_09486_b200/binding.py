@@ -215,6 +215,9 @@ def loma_masked_attn_bwd_plan_coverage(n_chunks: int, c: int, t: int, tail_read:
     return counts
 
 
+LOMA_ROPE_INVERSE = 2
+
+
 def loma_rope_apply(q, k, n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0, theta_base: float = 0.0,
                     position_type: int = 0, stream=None) -> None:
     """Rotates q and k ([B, H, S, D] device tensors with identical strides; either may be None) in place at

@@ -218,7 +218,7 @@ int loma_rope_apply(void* q, void* k, int B, int H, int D, int n_chunks, int c, 
     if (B < 0 || H < 0) return LOMA_ERR_INVALID_ARG;
     if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
     if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
-    if (position_type != 0 && position_type != 1) return LOMA_ERR_INVALID_ARG;
+    if (position_type < 0 || position_type > (1 | LOMA_ROPE_INVERSE)) return LOMA_ERR_INVALID_ARG;
     Layout L;
     const int rc = make_layout(n_chunks, c, t, tail_read, flags, &L);
     if (rc != LOMA_OK) return rc;

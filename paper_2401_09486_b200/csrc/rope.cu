@@ -59,7 +59,8 @@ rope_kernel(T* __restrict__ q, T* __restrict__ k, int BH, int H, Layout L, int64
     if (i >= L.S) return;
     const RowInfo r = layout_row(i, L.n_chunks, L.c, L.t, L.s);
     int pos = r.pos;
-    if (position_type == 1 && r.zone == LOMA_ZONE_MEM) pos = r.chunk * L.t + r.offset;
+    if ((position_type & 1) && r.zone == LOMA_ZONE_MEM) pos = r.chunk * L.t + r.offset;
+    if (position_type & LOMA_ROPE_INVERSE) pos = -pos;      // the transposed rotation: what a gradient needs on its way back
     const int d0 = (lane % LPR) * N;
     float cs[N], sn[N];
 #pragma unroll

@@ -210,7 +210,8 @@ def test_rope_validation(lib):
     def call(q=0x1000, k=0x2000, B=1, H=1, D=64, n=1, c=2, t=2, tc=4, tail=0, sb=640, sh=640, ss=64, dt=1, ptype=0):
         return lib.loma_rope_apply(q, k, B, H, D, n, c, t, tc, tail, sb, sh, ss, dt, 0.0, ptype, 0, None)
     assert call(tc=5) == INVALID
-    assert call(ptype=2) == INVALID
+    assert call(ptype=4) == INVALID
+    assert call(ptype=-1) == INVALID
     assert call(D=96) == UNSUPPORTED
     assert call(k=0x1000) == INVALID                    # q aliases k
     assert call(q=0x1004) == ALIGNMENT

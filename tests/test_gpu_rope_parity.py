@@ -82,3 +82,46 @@ def test_rotated_scores_see_positions_only_through_their_difference():
     got = float((gq[0, 0, i].double() * gk[0, 0, j].double()).sum())
     want = float((oracle.rope_rotate(npf(q)[0, 0, i:i + 1], np.array([pos[i] - pos[j]]))[0] * npf(k)[0, 0, j]).sum())
     assert abs(got - want) < 1e-4
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_inverse_rotation_undoes_the_rotation_and_matches_the_oracle_at_negated_positions(dtype):
+    B, H, D, n, c, t, tail = 2, 2, 128, 5, 4, 16, 9
+    S = oracle.seq_len(n, c, t, tail)
+    q, k, _ = synthetic.qkv(B, H, S, D, seed=25, dtype=dtype)
+    gq, gk = q.to(DEV), k.to(DEV)
+    L.loma_rope_apply(gq, gk, n, c, t, tail, 0, 0.0, L.LOMA_ROPE_INVERSE)
+    torch.cuda.synchronize()
+    pos = oracle.position_ids(n, c, t, tail)
+    check(gq, oracle.rope_rotate(npf(q), -pos), dtype)
+    check(gk, oracle.rope_rotate(npf(k), -pos), dtype)
+    L.loma_rope_apply(gq, gk, n, c, t, tail)                       # forward rotation of the inverse: back to the start
+    torch.cuda.synchronize()
+    tol = 1e-5 if dtype == torch.float32 else 3e-2
+    assert float((gq.float().cpu() - q.float()).abs().max()) <= tol * max(1.0, float(q.float().abs().max()))
+
+
+def test_differentiable_rope_then_attention_against_torch_autograd():
+    """rope -> masked attention as torch ops built on the library, against torch's own autograd of the same
+    composition in fp64 (rotation written with cos/sin tables from the oracle's position ids)."""
+    from paper_2401_09486_b200.autograd import loma_masked_attention, loma_rope
+    B, H, D, n, c, t = 1, 2, 64, 3, 2, 8
+    S = oracle.seq_len(n, c, t)
+    q, k, v = (x.to(DEV).requires_grad_(True) for x in synthetic.qkv(B, H, S, D, seed=27, dtype=torch.float32))
+    w = synthetic.normal_tensor((B, H, S, D), 28, 1.0, torch.float32).to(DEV)
+    rq, rk = loma_rope(q, k, n, c, t)
+    (loma_masked_attention(rq, rk, v, n, c, t) * w).sum().backward()
+    pos = torch.from_numpy(oracle.position_ids(n, c, t)).double().to(DEV)
+    theta = 10000.0 ** (-2.0 * torch.arange(D // 2, dtype=torch.float64, device=DEV) / D)
+    ang = pos[:, None] * theta[None, :]
+    cs, sn = torch.cos(ang), torch.sin(ang)
+    def rot(x):
+        a, b = x[..., : D // 2], x[..., D // 2:]
+        return torch.cat([a * cs - b * sn, b * cs + a * sn], dim=-1)
+    q2, k2, v2 = (x.detach().double().requires_grad_(True) for x in (q, k, v))
+    M = torch.from_numpy(oracle.dense_mask(n, c, t)).to(DEV)
+    A = (rot(q2) @ rot(k2).transpose(-1, -2)) / D ** 0.5
+    ((torch.softmax(A.masked_fill(~M, float("-inf")), dim=-1) @ v2) * w.double()).sum().backward()
+    torch.cuda.synchronize()
+    for g, g2 in ((q.grad, q2.grad), (k.grad, k2.grad), (v.grad, v2.grad)):
+        assert float((g.double() - g2).abs().max()) <= 2e-5 * max(1.0, float(g2.abs().max()))
