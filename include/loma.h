@@ -38,8 +38,11 @@
  *     anything is launched; on error nothing has been launched.
  *   - Pointers marked [device] are CUDA device pointers on the current device;
  *     [host] are ordinary host pointers.  The caller owns every buffer before
- *     and after the call; the library allocates no device memory and keeps no
- *     pointer beyond the call.
+ *     and after the call; the library allocates no device memory and reads or
+ *     writes nothing through a pointer after the work enqueued by the call has
+ *     finished (the tensor-core paths remember the last call's addresses, as
+ *     numbers, to reuse its TMA descriptors when the same tensors come again).
+ *   - stride_b / stride_h of 0 are rejected (INVALID_ARG) when B / H exceeds 1.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
  *     work is enqueued on it and the call returns without synchronising.
  *   - Tensors are row-major with the head dimension D contiguous.  D is 64 or
@@ -267,6 +270,20 @@ LOMA_API int loma_masked_attn_plan_coverage(int n_chunks, int c, int t, int tail
                                             uint8_t* counts);
 
 /* ---------------------------------------------------------------------------
+ * loma_masked_attn_pair_plan_check -- host-only check of how the tensor-core kernel
+ * of loma_masked_attn_fwd (Eq. 1-3, Eq. 5-7) schedules its work.  The kernel takes two
+ * neighbouring query tiles at a time, loads the union of their key tiles once, in one
+ * merged order, through a two-stage ring, and issues the two tiles' tensor-core
+ * instructions interleaved.  This routine replays, for every pair of the plan, the
+ * merged order and the order of issue, and returns the number of violations of the
+ * properties the kernel relies on (a step sequence that is not monotone, a shared step
+ * whose two key tiles differ, an instruction whose K/V stage could not have been loaded
+ * from instructions issued before it, a stage released twice or never).  0 = sound.
+ * No CUDA call is made.  Negative return: INVALID_ARG (bad geometry).
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_masked_attn_pair_plan_check(int n_chunks, int c, int t, int tail_read, unsigned flags);
+
+/* ---------------------------------------------------------------------------
  * loma_masked_attn_bwd_plan_coverage -- the same host-only replay for the pass of
  * loma_masked_attn_bwd that produces dK and dV.  That pass owns one 128-row key tile at a
  * time and walks the query tiles that may attend to it (the columns of Eq. 2 read
@@ -489,6 +506,13 @@ LOMA_API int loma_selftest_bounded_wait(void* stream);
 /* Number of kernels this library has enqueued in the calling process since it
  * was loaded (all devices, all streams).  Host-side counter; never fails. */
 LOMA_API uint64_t loma_launch_count(void);
+
+/* Number of bf16 calls (forward or backward of the masked attention) for which the
+ * tensor-core path declined the arguments (TMA descriptor not encodable, zone longer
+ * than the tile plan supports) and the slower CUDA-core kernels ran instead.  The
+ * result of such a call is still correct; a caller that cares about speed can watch
+ * this counter.  Host-side counter; never fails. */
+LOMA_API uint64_t loma_fallback_count(void);
 
 /* Static, human-readable name of a status code. */
 LOMA_API const char* loma_status_string(int status);

@@ -40,6 +40,7 @@ SIGNATURES = {
     "loma_rope_apply": (_i, [_p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i, _f, _i, _u, _p]),
     "loma_masked_attn_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
     "loma_masked_attn_bwd_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
+    "loma_masked_attn_pair_plan_check": (_i, [_i, _i, _i, _i, _u]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "loma_decode_attn_paged": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p, _sz, _p]),
@@ -54,6 +55,7 @@ SIGNATURES = {
     "loma_device_status": (_i, [_p]),
     "loma_selftest_bounded_wait": (_i, [_p]),
     "loma_launch_count": (ctypes.c_uint64, []),
+    "loma_fallback_count": (ctypes.c_uint64, []),
     "loma_status_string": (ctypes.c_char_p, [_i]),
     "loma_version": (_i, []),
 }
@@ -121,6 +123,11 @@ def loma_version() -> int:
 
 def loma_launch_count() -> int:
     return int(lib().loma_launch_count())
+
+
+def loma_fallback_count() -> int:
+    """bf16 calls that ran on the CUDA-core kernels because the tensor-core path declined them."""
+    return int(lib().loma_fallback_count())
 
 
 def loma_selftest_bounded_wait(stream=None) -> None:
@@ -204,6 +211,15 @@ def loma_masked_attn_plan_coverage(n_chunks: int, c: int, t: int, tail_read: int
     rc = lib().loma_masked_attn_plan_coverage(n_chunks, c, t, tail_read, int(flags), _ptr(counts))
     _check(rc, "loma_masked_attn_plan_coverage")
     return counts
+
+
+def loma_masked_attn_pair_plan_check(n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0) -> int:
+    """Host replay of the forward kernel's pair schedule (merged key-tile order, order of issue against
+    the two-stage ring): number of violations, 0 = sound."""
+    rc = lib().loma_masked_attn_pair_plan_check(n_chunks, c, t, tail_read, int(flags))
+    if rc < 0:
+        _check(rc, "loma_masked_attn_pair_plan_check")
+    return rc
 
 
 def loma_masked_attn_bwd_plan_coverage(n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0) -> torch.Tensor:

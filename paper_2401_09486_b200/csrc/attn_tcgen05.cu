@@ -19,29 +19,33 @@
 //   repetition rows x own memory zone                  key chunk == row chunk   (Eq. 1, row 3)
 //   repetition rows x themselves                       diagonal                 (I of Eq. 1)
 //
-// One CTA (384 threads) per SM, persistent.  A CTA runs two independent "streams": each stream
-// owns a query tile at a time and has its own shared-memory buffers (Q, one K tile, one V tile,
-// a 64-column output staging panel), its own quarter of TMEM (two 64-column score buffers and a
-// 128-column output accumulator) and its own warps:
-//   warps 0-3 / 4-7   softmax warpgroup of stream 0 / 1: thread = query row = TMEM lane.  The 128
-//                     keys of a step are taken as two halves of 64: read the scores of a half,
-//                     row maximum (three-input max), probabilities 2^(s*scale - ref) with packed
-//                     two-wide fp32 FMA/ADD, bf16 P written back over the scores.  The output
-//                     accumulates in TMEM; the reference maximum only moves, and the accumulator
-//                     is only rescaled, when a row maximum has grown by more than 2^8.  Epilogue:
-//                     normalise, round to bf16, stage 64 columns at a time, TMA store.
-//   warp 8 / 9        TMA producer of stream 0 / 1 (one lane): Q per tile, K and V per step
-//   warp 10 / 11      MMA issuer of stream 0 / 1: the warp's control flow is uniform and one
-//                     elected lane issues, so descriptors stay in uniform registers (issuing from
-//                     a divergent single-lane branch halved the tensor throughput).  Per step:
-//                     S_h = Q K_h^T for both halves (operands in shared memory, N = 64), and
-//                     O += P_h V_h with P read from TMEM and V as an MN-major shared operand.
-//                     S_h of the next step is issued right after P_h V_h of this one, so the
-//                     tensor pipe works on one half while the warpgroup works on the other.
-// The two streams fill each other's waits (tensor latency, TMEM loads, epilogues).  Tiles are handed
-// out at run time from one counter over a statically ordered list (longest first, (batch, head)
-// fastest): a stream that finishes a tile draws the next.  Every mbarrier wait is bounded: on expiry the CTA records LOMA_ERR_TIMEOUT, all
+// One persistent CTA (384 threads) per SM.  A CTA works on a PAIR of query tiles at a time (tiles 2i and
+// 2i + 1 of one view and one (batch, head): A and B) and feeds both from one stream of key tiles -- two
+// neighbouring tiles visit almost the same keys, so a K/V tile both need crosses into shared memory once
+// (see "pairs of query tiles" in tile_plan.cuh for the merged order).  Shared memory: Q_A, Q_B, a two-stage
+// ring of (K tile, V tile), and one 64-column output staging panel per tile.  TMEM: per tile a 128-column
+// score region (the two 64-key halves of a key tile side by side) and a 128-column output accumulator.
+//   warps 0-3 / 4-7   softmax warpgroup of tile A / B: thread = query row = TMEM lane.  The 128 keys of a
+//                     step are taken as two halves of 64 ("events"): read the scores of a half, row maximum
+//                     (three-input max), probabilities 2^(s*scale - ref) with packed two-wide fp32 FMA/ADD,
+//                     bf16 P written back over the scores.  The output accumulates in TMEM; the reference
+//                     maximum only moves, and the accumulator is only rescaled, when a row maximum has
+//                     grown by more than 2^8.  Epilogue: normalise, round to bf16, stage 64 columns at a
+//                     time, TMA store.
+//   warp 8            TMA producer (one lane): draws the next pair, loads Q_A and Q_B, then K and V of every
+//                     merged step into the ring; it runs ahead of the other roles as far as the ring and the
+//                     Q buffers allow, across pair boundaries too.
+//   warp 9 / 10       MMA issuer of tile A / B: control flow is warp-uniform and one elected lane issues.
+//                     Per step: S = Q K^T with both operands in shared memory (N = 128 when both halves of
+//                     the key tile are visited, N = 64 otherwise), then per visited half O += P_h V_h with P
+//                     read from TMEM and V as an MN-major shared operand.  While one tile's warpgroup turns
+//                     scores into probabilities the tensor pipe works for the other tile; a ring stage is
+//                     refilled once both tiles (or the only one that visits the step) have released it.
+// Pairs are handed out at run time from one counter over a statically ordered list (longest first,
+// (batch, head) fastest).  Every mbarrier wait is bounded: on expiry the CTA records LOMA_ERR_TIMEOUT, all
 // roles leave their loops, TMEM is freed and the kernel returns.
+#include <type_traits>
+
 #include "tcgen05_common.cuh"
 
 namespace loma {
@@ -51,22 +55,36 @@ struct TmaMaps {
 };
 
 // ------------------------------------------------------------------ the kernel
-constexpr int TC_THREADS = 384;   // 2 softmax warpgroups + 1 warpgroup with 2 TMA warps and 2 MMA warps
+constexpr int TC_THREADS = 384;   // 2 softmax warpgroups + 1 warpgroup holding the TMA warp and the two MMA warps
 constexpr int TMEM_COLS = 512;
-constexpr int NBAR = 14;          // mbarriers per stream
 
-// Shared memory of one stream: Q tile, one K tile, one V tile, and a 64-column output staging panel.
+// mbarriers of a CTA
+enum {
+    B_QF = 0,    // +x   Q tile of A / B has landed
+    B_QE = 2,    // +x   every score product of the pair's tile x has completed: Q buffer free
+    B_KF = 4,    // +s   K tile of ring stage s has landed
+    B_KE = 6,    // +s   every score product that reads stage s has completed (two arrivals: one per tile, or both from the only visitor)
+    B_VF = 8,    // +s
+    B_VE = 10,   // +s   every P.V product that reads stage s has completed (two arrivals, as B_KE)
+    B_SF = 12,   // +x   scores of tile x's current step are in TMEM
+    B_PF = 14,   // +2x+(event & 1)   probabilities of an event are in TMEM (128 arrivals)
+    B_OF = 18,   // +2x+(event & 1)   the P.V product of an event of tile x has completed
+    B_TF = 22,   // +(n & 3)  the n-th pair number has been posted in slot n & 3 of the pair ring
+    B_TE = 26,   // +(n & 3)  every reader (8 softmax warps, 2 MMA warps) has taken the n-th pair number
+    NBAR = 30
+};
+
+// Shared memory: Q_A, Q_B, ring of two (K, V) stages, one output staging panel per tile.
 template <int D>
 struct TcSmem {
     static constexpr int PANELS = D / 64;
     static constexpr int PANEL_BYTES = 128 * 128;           // 128 rows x 64 bf16
     static constexpr int TILE_BYTES = PANELS * PANEL_BYTES; // one 128 x D tile
-    static constexpr int Q_OFF = 0;
-    static constexpr int K_OFF = TILE_BYTES;
-    static constexpr int V_OFF = 2 * TILE_BYTES;
-    static constexpr int O_OFF = 3 * TILE_BYTES;
-    static constexpr int STREAM_BYTES = 3 * TILE_BYTES + PANEL_BYTES;
-    static constexpr int TOTAL = 2 * STREAM_BYTES;
+    static constexpr int Q_OFF = 0;                         // + x * TILE_BYTES
+    static constexpr int K_OFF = 2 * TILE_BYTES;            // + s * 2 * TILE_BYTES
+    static constexpr int V_OFF = 3 * TILE_BYTES;            // + s * 2 * TILE_BYTES
+    static constexpr int O_OFF = 6 * TILE_BYTES;            // + x * PANEL_BYTES
+    static constexpr int TOTAL = 6 * TILE_BYTES + 2 * PANEL_BYTES;
 };
 
 template <int D>
@@ -75,33 +93,28 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     using SM = TcSmem<D>;
     constexpr int PANELS = SM::PANELS;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * NBAR];
+    __shared__ __align__(8) uint64_t bars[NBAR];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ int tile_ring_s[2][4];
+    __shared__ int pair_ring_s[4];
 
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;
-    // which of the CTA's two independent streams this warp serves
-    const int st = warp < 8 ? (warp >> 2) : (warp & 1);
-    const uint32_t smem_base0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* smem_gen0 = smem_raw + (smem_base0 - smem_u32(smem_raw));
-    const uint32_t smem_base = smem_base0 + st * SM::STREAM_BYTES;
-    uint8_t* smem_gen = smem_gen0 + st * SM::STREAM_BYTES;
-
-    enum { B_QF = 0, B_QE = 1, B_KF = 2, B_KE = 3, B_VF = 4, B_VE = 5, B_SF = 6, B_PF = 8, B_OF = 10, B_TF = 12 };
-    auto bar = [&](int i) { return smem_u32(&bars[st * NBAR + i]); };
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    auto bar = [&](int i) { return smem_u32(&bars[i]); };
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
-        for (int s2 = 0; s2 < 2; ++s2)
-            for (int i = 0; i < NBAR; ++i) mbar_init(smem_u32(&bars[s2 * NBAR + i]), (i == B_PF || i == B_PF + 1) ? 128 : 1);
+        for (int i = 0; i < NBAR; ++i)
+            mbar_init(bar(i), (i >= B_PF && i < B_PF + 4) ? 128 : (i >= B_TE && i < B_TE + 4) ? 10
+                                  : (i >= B_KE && i < B_KE + 2) || (i >= B_VE && i < B_VE + 2) ? 2 : 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // zero the operand buffers once: rows a TMA box does not cover keep finite contents
     for (int i = threadIdx.x; i < SM::TOTAL / 16; i += TC_THREADS)
-        reinterpret_cast<uint4*>(smem_gen0)[i] = make_uint4(0, 0, 0, 0);
+        reinterpret_cast<uint4*>(smem_gen)[i] = make_uint4(0, 0, 0, 0);
     fence_async_smem();
-    if (warp == 10) {
+    if (warp == 9) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)),
                      "r"(TMEM_COLS)
                      : "memory");
@@ -110,170 +123,189 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = tmem_slot + st * 256;   // this stream's scores at +0, output accumulator at +128
+    const uint32_t tmem0 = tmem_slot;   // tile x: scores at tmem0 + 256 x, output accumulator at + 128
     volatile int* abortp = &abort_flag;
 
-    // Tiles (longest first) are dealt to the 2*gridDim.x streams in rounds, forwards in even rounds
-    // and backwards in odd ones, so no stream always receives the longest tile of a round.
-    // Tiles are handed out from one counter, longest first ((batch, head) fastest inside a rank): a stream
-    // that finishes early simply takes the next one.  The stream's producer draws the number and posts it
-    // in a four-slot ring (barrier B_TF + (n & 1), completion n >> 1, for the stream's n-th tile); the MMA
-    // issuer and the warpgroup read it there.  A negative number ends the stream.  Which stream computes a
-    // tile has no influence on the tile's result.
-    const int total_work = p.total_tiles * p.BH;
-    volatile int* tile_ring = tile_ring_s[st];
-    auto next_tile = [&](uint32_t n, bool& ok_) -> int {   // called by whole warps
-        ok_ = __all_sync(0xffffffffu, mbar_wait(bar(B_TF + (n & 1)), (n >> 1) & 1, abortp, p.status));
-        return ok_ ? tile_ring[n & 3] : -1;
+    // Pairs are handed out from one counter, longest first ((batch, head) fastest inside a rank).  The
+    // producer draws the number and posts it in a four-slot ring (slot n & 3, barrier B_TF + (n & 3),
+    // completion n >> 2, for the CTA's n-th pair); the MMA issuer and the warpgroups read it there and
+    // acknowledge on B_TE, which the producer waits for before it reuses the slot (a warpgroup without a
+    // tile in some pairs may lag behind the others).  A negative number ends the CTA's work.  Which CTA
+    // computes a pair has no influence on the pair's result.  Without a counter (p.sched == NULL) the
+    // pairs are dealt round robin.
+    const int total_work = p.total_pairs * p.BH;
+    volatile int* pair_ring = pair_ring_s;
+    auto next_pair = [&](uint32_t n, bool& ok_) -> int {   // called by whole warps
+        ok_ = __all_sync(0xffffffffu, mbar_wait(bar(B_TF + (n & 3)), (n >> 2) & 1, abortp, p.status));
+        const int w = ok_ ? pair_ring[n & 3] : -1;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(B_TE + (n & 3)));
+        return w;
     };
 
-    if (warp == 8 || warp == 9) {
-        // ------------------------------------------------------------ TMA producer of stream st
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
+    if (warp >= 8) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 88;" ::: "memory");
+    }
+    if (warp == 8) {
+        // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t gs = 0, tcount = 0;
+            uint32_t gl = 0, pcount = 0;      // K/V loads so far (one per merged step), pairs so far
+            uint32_t nq[2] = {0, 0};          // uses of each Q buffer so far
             bool ok = true;
-            for (;; ++tcount) {
-                // draw the stream's next tile and post it (a number past the end tells the other roles to stop)
-                int w = (int)atomicAdd(p.sched, 1u);
+            for (;; ++pcount) {
+                int w = p.sched ? (int)atomicAdd(p.sched, 1u) : (int)(blockIdx.x + pcount * gridDim.x);
                 if (w >= total_work || !ok) w = -1;
-                tile_ring[tcount & 3] = w;
+                if (pcount >= 4 && ok) ok = mbar_wait(bar(B_TE + (pcount & 3)), ((pcount >> 2) - 1) & 1, abortp, p.status);
+                if (!ok) w = -1;
+                pair_ring[pcount & 3] = w;
                 __threadfence_block();
-                mbar_arrive(bar(B_TF + (tcount & 1)));
+                mbar_arrive(bar(B_TF + (pcount & 3)));
                 if (w < 0) break;
                 const int rank = fdiv(w, p.dBH), bh = w - rank * p.BH;
                 const int bi = fdiv(bh, p.dH), hi = bh - bi * p.H;
-                TileDesc td;
-                decode_tile(p, rank, td);
-                const View& qv = p.view[td.view];
-                if (tcount > 0) ok = mbar_wait(bar(B_QE), (tcount - 1) & 1, abortp, p.status);
-                if (!ok) break;
-                mbar_expect_tx(bar(B_QF), qv.R * qv.CH * 128 * PANELS);
-                for (int pn = 0; pn < PANELS; ++pn)
-                    tma_load_5d(smem_base + SM::Q_OFF + pn * SM::PANEL_BYTES, &maps.q[td.view], bar(B_QF), pn * 64, td.r0,
-                                td.c0, hi, bi);
-                for (int j = 0; j < td.nsteps; ++j, ++gs) {
-                    KTile kt;
-                    step_ktile(p, td, j, kt);
-                    const View& kv = p.view[kt.view];
-                    const uint32_t ph = gs & 1;
-                    const uint32_t bytes = kv.R * kv.CH * 128 * PANELS;
-                    ok = mbar_wait(bar(B_KE), ph ^ 1, abortp, p.status);
+                PairDesc pd;
+                decode_pair(p, rank, pd);
+                const View& qv = p.view[pd.td[0].view];
+#pragma unroll
+                for (int x = 0; x < 2; ++x) {
+                    if (x == 1 && !pd.nb) break;
+                    if (nq[x] > 0) ok = mbar_wait(bar(B_QE + x), (nq[x] - 1) & 1, abortp, p.status);
                     if (!ok) break;
-                    mbar_expect_tx(bar(B_KF), bytes);
+                    ++nq[x];
+                    mbar_expect_tx(bar(B_QF + x), qv.R * qv.CH * 128 * PANELS);
                     for (int pn = 0; pn < PANELS; ++pn)
-                        tma_load_5d(smem_base + SM::K_OFF + pn * SM::PANEL_BYTES, &maps.k[kt.view], bar(B_KF), pn * 64,
-                                    kt.r0, kt.c0, hi, bi);
-                    ok = mbar_wait(bar(B_VE), ph ^ 1, abortp, p.status);
-                    if (!ok) break;
-                    mbar_expect_tx(bar(B_VF), bytes);
-                    for (int pn = 0; pn < PANELS; ++pn)
-                        tma_load_5d(smem_base + SM::V_OFF + pn * SM::PANEL_BYTES, &maps.v[kt.view], bar(B_VF), pn * 64,
-                                    kt.r0, kt.c0, hi, bi);
+                        tma_load_5d(smem_base + SM::Q_OFF + x * SM::TILE_BYTES + pn * SM::PANEL_BYTES, &maps.q[pd.td[x].view],
+                                    bar(B_QF + x), pn * 64, pd.td[x].r0, pd.td[x].c0, hi, bi);
                 }
+                if (!ok) break;
+                for (int m = 0; m < pd.pm.nmerged; ++m, ++gl) {
+                    int x, j;
+                    merged_source(pd.pm, m, x, j);
+                    KTile kt;
+                    if (x) step_ktile(p, pd.td[1], j, kt);
+                    else step_ktile(p, pd.td[0], j, kt);
+                    const View& kv = p.view[kt.view];
+                    const uint32_t s = gl & 1, ph = (gl >> 1) & 1;
+                    const uint32_t bytes = kv.R * kv.CH * 128 * PANELS;
+                    ok = mbar_wait(bar(B_KE + s), ph ^ 1, abortp, p.status);
+                    if (!ok) break;
+                    mbar_expect_tx(bar(B_KF + s), bytes);
+                    for (int pn = 0; pn < PANELS; ++pn)
+                        tma_load_5d(smem_base + SM::K_OFF + s * 2 * SM::TILE_BYTES + pn * SM::PANEL_BYTES, &maps.k[kt.view],
+                                    bar(B_KF + s), pn * 64, kt.r0, kt.c0, hi, bi);
+                    ok = mbar_wait(bar(B_VE + s), ph ^ 1, abortp, p.status);
+                    if (!ok) break;
+                    mbar_expect_tx(bar(B_VF + s), bytes);
+                    for (int pn = 0; pn < PANELS; ++pn)
+                        tma_load_5d(smem_base + SM::V_OFF + s * 2 * SM::TILE_BYTES + pn * SM::PANEL_BYTES, &maps.v[kt.view],
+                                    bar(B_VF + s), pn * 64, kt.r0, kt.c0, hi, bi);
+                }
+                if (!ok) break;
             }
             if (!ok) {
-                // leaving early: give copies already in flight a bounded time to land in this CTA's shared memory
+                // leaving early (the abort flag is set): give copies in flight a bounded time to land
                 const long long t0 = clock64();
                 while (clock64() - t0 < 2000000ll) {}
             }
         }
-    } else if (warp >= 10) {
-        // ------------------------------------------------------------ MMA issuer of stream st
-        // All 32 lanes run the loops (warp-uniform); one elected lane issues the instructions.
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
-        {
-            // instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128
-            constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-            constexpr uint32_t IDESC_PV =
-                (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
-            uint32_t gs = 0, tcount = 0;
-            bool ok = true;
-            const uint64_t qd = smem_desc(smem_base + SM::Q_OFF, 16, 1024);
-            const uint64_t kd = smem_desc(smem_base + SM::K_OFF, 16, 1024);
-            const uint64_t vd = smem_desc(smem_base + SM::V_OFF, SM::PANEL_BYTES, 1024);
-            // Visited halves ("events") are numbered ge = 0, 1, 2, ... across all tiles of the stream.
-            // Event ge uses score buffer ge & 1 and the barriers B_SF/B_PF/B_OF + (ge & 1), whose
-            // completion number ge >> 1 gives the parity to wait for.  K/V buffers go by step (gs).
-            // scores of keys [64h, 64h+64) of the staged key tile -> score buffer b (64 columns)
-            auto issue_s = [&](int b, int h, bool last_of_step, bool last_of_tile) {
-                if (elect_one()) {
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        // descriptor start addresses are in 16-byte units; 64 key rows are 8192 bytes further
-                        const uint64_t off = (uint64_t)(((kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32) >> 4);
-                        mma_ss(tmem + b * 64, qd + off, kd + off + (uint64_t)((h * 8192) >> 4), IDESC_S, kk > 0);
-                    }
-                    tc_commit(bar(B_SF + b));
-                    if (last_of_step) tc_commit(bar(B_KE));
-                    if (last_of_tile) tc_commit(bar(B_QE));   // every score product of the tile has been issued
+    } else if (warp == 9 || warp == 10) {
+        // ------------------------------------------------------------ MMA issuer of tile X
+        // All 32 lanes run the loops (warp-uniform); one elected lane issues the instructions.  One warp per
+        // tile: an issuing thread runs in step with the tensor pipe (its queue is short), so the bookkeeping
+        // between two instructions of one warp is covered by the other warp's instructions.
+        const int X = warp - 9;
+        // instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128
+        constexpr uint32_t IDESC_S64 = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+        constexpr uint32_t IDESC_S128 = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+        constexpr uint32_t IDESC_PV =
+            (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
+        const uint32_t tm = tmem0 + X * 256;
+        const uint64_t qd = smem_desc(smem_base + SM::Q_OFF + X * SM::TILE_BYTES, 16, 1024);
+        uint32_t ge = 0;                  // events (visited halves) issued on this tile slot, all pairs
+        uint32_t nq = 0;                  // pairs in which this slot was used
+        uint32_t gbase = 0, pcount = 0;   // merged steps of earlier pairs, pairs so far
+        bool ok = true;
+        for (;; ++pcount) {
+            const int w = next_pair(pcount, ok);
+            if (w < 0) break;
+            const int rank = fdiv(w, p.dBH);
+            PairMap pm;
+            TileIssue ti;
+            bool mine;
+            {
+                PairDesc pd;
+                decode_pair(p, rank, pd);
+                pm = pd.pm;
+                mine = (X == 0) || pd.nb;
+                if (mine) {
+                    if (X) ti.start(tile_half_masks(p, pd.td[1], lane), pd.td[1].nsteps);
+                    else ti.start(tile_half_masks(p, pd.td[0], lane), pd.td[0].nsteps);
                 }
-                __syncwarp();
-            };
-            // O += P V[64h .. 64h+63]: four instructions of 16 keys, P read from TMEM over score buffer b
-            auto issue_pv = [&](int b, int h, bool first, bool last_of_step) {
-                if (elect_one()) {
-#pragma unroll
-                    for (int k4 = 0; k4 < 4; ++k4)
-                        mma_ts(tmem + 128, tmem + b * 64 + k4 * 8, vd + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_PV,
-                               !first || (k4 > 0));
-                    tc_commit(bar(B_OF + b));   // one barrier per buffer: each completes once per event
-                    if (last_of_step) tc_commit(bar(B_VE));
-                }
-                __syncwarp();
-            };
-            uint32_t ge_s = 0, ge_p = 0;   // events whose scores / whose P.V have been issued
-            for (;; ++tcount) {
-                const int w = next_tile(tcount, ok);
-                if (w < 0) break;
-                const int rank = fdiv(w, p.dBH);
-                TileDesc td;
-                decode_tile(p, rank, td);
-                const HalfMasks hm = tile_half_masks(p, td, lane);
-                const int nsteps = td.nsteps;
-                HalfWalk sw, pw;
-                sw.start(hm);
-                pw.start(hm);
-                ok = __all_sync(0xffffffffu, mbar_wait(bar(B_QF), tcount & 1, abortp, p.status));
-                if (!ok) break;
-                // the score products run two events ahead of the P.V products
-                auto next_scores = [&]() {
-                    if (sw.first_of_step(hm)) {
-                        ok = __all_sync(0xffffffffu, mbar_wait(bar(B_KF), (gs + sw.j) & 1, abortp, p.status));
-                        if (!ok) return;
-                    }
-                    tc_fence_after();
-                    const bool los = sw.last_of_step(hm);
-                    issue_s(ge_s & 1, sw.h, los, los && sw.j == nsteps - 1);
-                    ++ge_s;
-                    sw.next(hm);
-                };
-                next_scores();
-                if (ok && !sw.done(nsteps)) next_scores();
-                bool first = true;
-                while (ok && !pw.done(nsteps)) {
-                    const int b = ge_p & 1;
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_PF + b), (ge_p >> 1) & 1, abortp, p.status));
-                    if (ok && pw.first_of_step(hm))
-                        ok = __all_sync(0xffffffffu, mbar_wait(bar(B_VF), (gs + pw.j) & 1, abortp, p.status));
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_pv(b, pw.h, first, pw.last_of_step(hm));
-                    first = false;
-                    ++ge_p;
-                    if (!sw.done(nsteps)) next_scores();
-                    pw.next(hm);
-                }
-                gs += td.nsteps;
             }
+            if (mine) {
+                ++nq;
+                IssueAct act;
+                while (ok && !ti.done()) {
+                    ti.next(pm, X, act);
+                    const uint32_t gl = gbase + (uint32_t)act.m, s = gl & 1, ph = (gl >> 1) & 1;
+                    if (act.is_s) {
+                        if (act.first_event)
+                            ok = __all_sync(0xffffffffu, mbar_wait(bar(B_QF + X), (nq - 1) & 1, abortp, p.status));
+                        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_KF + s), ph, abortp, p.status));
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (elect_one()) {
+                            const uint64_t kd = smem_desc(smem_base + SM::K_OFF + s * 2 * SM::TILE_BYTES, 16, 1024);
+                            const uint32_t half_off = (act.cur == 2u) ? 1u : 0u;   // only the second half: keys 64.., columns 64..
+                            const uint32_t idesc = (act.cur == 3u) ? IDESC_S128 : IDESC_S64;
+#pragma unroll
+                            for (int kk = 0; kk < D / 16; ++kk) {
+                                // descriptor start addresses are in 16-byte units; 64 key rows are 8192 bytes further
+                                const uint64_t off = (uint64_t)(((kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32) >> 4);
+                                mma_ss(tm + half_off * 64, qd + off, kd + off + (uint64_t)((half_off * 8192) >> 4), idesc, kk > 0);
+                            }
+                            tc_commit(bar(B_SF + X));
+                            tc_commit(bar(B_KE + s));
+                            if (act.release == 2) tc_commit(bar(B_KE + s));   // the other tile does not visit this step
+                            if (act.last_s) tc_commit(bar(B_QE + X));
+                        }
+                        __syncwarp();
+                    } else {
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar(B_PF + 2 * X + (ge & 1)), (ge >> 1) & 1, abortp, p.status));
+                        if (ok && act.first_of_step)
+                            ok = __all_sync(0xffffffffu, mbar_wait(bar(B_VF + s), ph, abortp, p.status));
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (elect_one()) {
+                            const uint64_t vd = smem_desc(smem_base + SM::V_OFF + s * 2 * SM::TILE_BYTES, SM::PANEL_BYTES, 1024);
+                            const int h = act.h;
+#pragma unroll
+                            for (int k4 = 0; k4 < 4; ++k4)
+                                mma_ts(tm + 128, tm + h * 64 + k4 * 8, vd + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_PV,
+                                       !act.first_event || (k4 > 0));
+                            tc_commit(bar(B_OF + 2 * X + (ge & 1)));
+                            if (act.release >= 1) tc_commit(bar(B_VE + s));
+                            if (act.release == 2) tc_commit(bar(B_VE + s));
+                        }
+                        __syncwarp();
+                        ++ge;
+                    }
+                }
+            }
+            if (!ok) break;
+            gbase += (uint32_t)pm.nmerged;
         }
-    } else {
-        // ------------------------------------------------------------ softmax + epilogue of stream st (128 threads)
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 232;" ::: "memory");
+    } else if (warp < 8) {
+        // ------------------------------------------------------------ softmax + epilogue of tile X (128 threads)
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;" ::: "memory");
+        const int X = warp >> 2;
         const int rr = threadIdx.x & 127;
-        const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        const uint32_t lane_addr = tmem0 + X * 256 + ((uint32_t)((warp & 3) * 32) << 16);
         const uint32_t s_addr = lane_addr, o_addr = lane_addr + 128;
-        uint32_t ge = 0;   // visited halves so far (see the MMA issuer)
+        const uint32_t o_stage = smem_base + SM::O_OFF + X * SM::PANEL_BYTES;
+        uint8_t* o_stage_gen = smem_gen + SM::O_OFF + X * SM::PANEL_BYTES;
+        uint32_t ge = 0;    // visited halves so far on this tile slot (see the MMA issuer)
+        uint32_t gst = 0;   // visited steps so far on this tile slot
         bool ok = true;
         bool store_pending = false;
         // Everything this thread needs to know about a tile.  The next tile is decoded while the last
@@ -285,12 +317,16 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             int bh, bi, hi, ro, rc, zone_row0;
             bool row_valid;
         };
-        auto decode_ctx = [&](int w, TileCtx& c) {
+        // the pair's tile X, or false when the pair has no tile B
+        auto decode_ctx = [&](int w, TileCtx& c) -> bool {
             const int rank = fdiv(w, p.dBH);
             c.bh = w - rank * p.BH;
             c.bi = fdiv(c.bh, p.dH);
             c.hi = c.bh - c.bi * p.H;
-            decode_tile(p, rank, c.td);
+            int view, qa, nb;
+            pair_tiles(p, rank, view, qa, nb);
+            if (X == 1 && !nb) return false;
+            decode_tile_at(p, view, qa + X, c.td);
             const View& qv = p.view[c.td.view];
             const int rsub = fdiv(rr, qv.dR);
             c.ro = c.td.r0 + (rr - rsub * qv.R);
@@ -298,12 +334,23 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             c.zone_row0 = qv.zone_row0;
             c.row_valid = (rr < qv.R * qv.CH) && (c.rc <= c.td.a1) && (c.ro < qv.Z);
             c.hm = tile_half_masks(p, c.td, lane);
+            return true;
+        };
+        // the next pair (from number n on) in which this warpgroup has a tile; -1 = no more
+        uint32_t pcount = 0;
+        auto next_ctx = [&](TileCtx& c) -> int {
+            for (;;) {
+                bool got = true;
+                const int w = next_pair(pcount, got);
+                if (!got) { ok = false; return -1; }
+                if (w < 0) return -1;
+                ++pcount;
+                if (decode_ctx(w, c)) return w;
+            }
         };
         TileCtx cur, nxt;
-        uint32_t tcount = 0;
-        int w_cur = next_tile(0, ok), w_next = -1;
-        if (w_cur >= 0) decode_ctx(w_cur, cur);
-        for (; w_cur >= 0 && ok; w_cur = w_next, cur = nxt, ++tcount) {
+        int w_cur = next_ctx(cur), w_next = -1;
+        for (; w_cur >= 0 && ok; w_cur = w_next, cur = nxt) {
             const TileDesc& td = cur.td;
             const HalfMasks hm = cur.hm;
             const int bh = cur.bh, bi = cur.bi, hi = cur.hi, ro = cur.ro, rc = cur.rc;
@@ -322,18 +369,18 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     KTile kt;
                     step_ktile(p, td, hw.j, kt);
                     row_interval(p.view[kt.view], kt, rc, ro, rr, row_valid, lo, hi2);
+                    // the scores of both visited halves of the step arrive together
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF + X), gst & 1, abortp, p.status));
+                    if (!ok) break;
+                    ++gst;
+                    tc_fence_after();
                 }
-                // One visited half of a key tile (64 keys) per pass, in score buffer ge & 1: the tensor
-                // pipe works on the other buffer while this warpgroup works on this one.
+                // One visited half of a key tile (64 keys) per pass.
                 {
-                    const int b = ge & 1;
                     const int lo_h = lo - 64 * hw.h;                  // allowed columns of this half: [lo_h, lo_h + span)
                     const uint32_t span = (uint32_t)(hi2 - lo);
                     const bool full = __all_sync(0xffffffffu, lo_h <= 0 && hi2 - 64 * hw.h >= 64);
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF + b), (ge >> 1) & 1, abortp, p.status));
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t sh_addr = s_addr + b * 64;
+                    const uint32_t sh_addr = s_addr + hw.h * 64;
                     uint32_t s[64];
                     tmem_ld32(sh_addr, s);
                     tmem_ld32(sh_addr + 32, s + 32);
@@ -355,8 +402,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     const bool need = mrow > m_used + 8.f;
                     if (!first && __any_sync(0xffffffffu, need)) {
                         // rescale the accumulated output: wait until the previous event's P.V has landed in TMEM
-                        ok = __all_sync(0xffffffffu,
-                                        mbar_wait(bar(B_OF + ((ge - 1) & 1)), ((ge - 1) >> 1) & 1, abortp, p.status));
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + 2 * X + ((ge - 1) & 1)), ((ge - 1) >> 1) & 1, abortp, p.status));
                         if (!ok) break;
                         tc_fence_after();
                         const float alpha = need ? fast_ex2(m_used - mrow) : 1.f;
@@ -399,24 +445,19 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     }
                     tmem_wait_st();
                     tc_fence_before();
-                    mbar_arrive(bar(B_PF + b));
+                    mbar_arrive(bar(B_PF + 2 * X + (ge & 1)));
                 }
             }
-            {
-                bool got = true;
-                w_next = next_tile(tcount + 1, got);
-                if (!got) ok = false;
-                if (w_next >= 0) decode_ctx(w_next, nxt);
-            }
+            if (ok) w_next = next_ctx(nxt);
             // the last P.V of the tile belongs to event ge - 1 (products complete in issue order)
-            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + ((ge - 1) & 1)), ((ge - 1) >> 1) & 1, abortp, p.status));
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + 2 * X + ((ge - 1) & 1)), ((ge - 1) >> 1) & 1, abortp, p.status));
             if (ok) tc_fence_after();
 
             // epilogue: normalise, round to bf16, stage 64 output columns at a time in shared
             // memory, TMA store.  Every thread of the warpgroup reaches the first barrier for
             // every tile it started; it also makes giving up a uniform decision.
             const float inv = 1.f / l;
-            uint8_t* orow = smem_gen + SM::O_OFF + rr * 128;
+            uint8_t* orow = o_stage_gen + rr * 128;
             bool give_up = false;
 #pragma unroll
             for (int pn = 0; pn < PANELS; ++pn) {
@@ -426,11 +467,11 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     asm volatile(
                         "{\n.reg .pred p, q;\nsetp.ne.u32 p, %1, 0;\nbar.red.or.pred q, %2, 128, p;\nselp.u32 %0, 1, 0, q;\n}"
                         : "=r"(any_bad)
-                        : "r"((uint32_t)(ok ? 0 : 1)), "r"(1 + st)
+                        : "r"((uint32_t)(ok ? 0 : 1)), "r"(1 + X)
                         : "memory");
                     if (any_bad) { give_up = true; break; }
                 } else {
-                    asm volatile("bar.sync %0, 128;" ::"r"(1 + st) : "memory");
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + X) : "memory");
                 }
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
@@ -449,9 +490,9 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     }
                 }
                 fence_async_smem();
-                asm volatile("bar.sync %0, 128;" ::"r"(1 + st) : "memory");
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + X) : "memory");
                 if (rr == 0) {
-                    tma_store_5d(&maps.o[td.view], smem_base + SM::O_OFF, pn * 64, td.r0, td.c0, hi, bi);
+                    tma_store_5d(&maps.o[td.view], o_stage, pn * 64, td.r0, td.c0, hi, bi);
                     tma_store_commit();
                     store_pending = true;
                 }
@@ -468,12 +509,12 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 10) {
+    if (warp == 9) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_slot), "r"(TMEM_COLS) : "memory");
     }
     // the last CTA to leave puts the scheduler's counters back to zero for the next launch that uses them
-    if (threadIdx.x == 0) {
+    if (threadIdx.x == 0 && p.sched) {
         __threadfence();
         if (atomicAdd(p.sched + 1, 1u) == gridDim.x - 1) {
             p.sched[0] = 0;
@@ -514,30 +555,50 @@ cudaError_t launch_bounded_wait_selftest(cudaStream_t st) {
 }
 
 // ------------------------------------------------------------------ host side
-// Tile counters of the in-kernel scheduler: 64 pairs (next tile, CTAs finished), handed to launches round robin
-// and cleared by the last CTA of the launch that used them.  512 bytes per device, zero at load.
-static __device__ unsigned g_sched_counters[64][2];
+// Counters of the in-kernel scheduler: pairs of (next pair, CTAs finished), cleared by the last CTA of the
+// launch that used them.  Two launches that may run at the same time must not share a pair, so a pair
+// belongs to a stream (kernels of one stream never overlap): the first SCHED_STREAMS streams that call
+// get one each.  A launch that is being captured into a CUDA graph may later be replayed on any stream,
+// next to anything, so it gets a pair of its own that is never handed out again (SCHED_CAPTURES of them).
+// When a table is full the launch runs without a counter: the kernel then deals the pairs round robin,
+// which is a few percent slower on short layouts and just as correct.
+constexpr int SCHED_STREAMS = 192, SCHED_CAPTURES = 320;
+static __device__ unsigned g_sched_counters[SCHED_STREAMS + SCHED_CAPTURES][2];
 
-static unsigned* sched_counters() {
+static unsigned* sched_counters(cudaStream_t st) {
+    static std::mutex mu;
     static unsigned* base[64] = {nullptr};
-    static std::atomic<unsigned> seq{0};
+    static cudaStream_t owner[64][SCHED_STREAMS];
+    static int n_owner[64] = {0}, n_capture[64] = {0};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
     if (!base[dev]) {
         void* ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, g_sched_counters) != cudaSuccess) return nullptr;
         base[dev] = static_cast<unsigned*>(ptr);
     }
-    return base[dev] + 2 * (seq.fetch_add(1) % 64);
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    if (cs != cudaStreamCaptureStatusNone) {
+        if (n_capture[dev] >= SCHED_CAPTURES) return nullptr;
+        return base[dev] + 2 * (SCHED_STREAMS + n_capture[dev]++);
+    }
+    for (int i = 0; i < n_owner[dev]; ++i)
+        if (owner[dev][i] == st) return base[dev] + 2 * i;
+    if (n_owner[dev] >= SCHED_STREAMS) return nullptr;
+    owner[dev][n_owner[dev]] = st;
+    return base[dev] + 2 * n_owner[dev]++;
 }
 
 struct MapCacheKey {
     const void *q, *k, *v, *o;
     int B, H, D, n, c, t, tail;
+    unsigned flags;
     int64_t sb, sh, ss;
     bool operator==(const MapCacheKey& r) const {
         return q == r.q && k == r.k && v == r.v && o == r.o && B == r.B && H == r.H && D == r.D && n == r.n && c == r.c &&
-               t == r.t && tail == r.tail && sb == r.sb && sh == r.sh && ss == r.ss;
+               t == r.t && tail == r.tail && flags == r.flags && sb == r.sb && sh == r.sh && ss == r.ss;
     }
 };
 
@@ -554,11 +615,11 @@ cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, v
     p.lse = lse;
     p.status = device_status_word();
     if (!p.status) return cudaErrorUnknown;
-    if ((int64_t)p.total_tiles * p.BH > 0x7ffffff0ll - 2 * 148) return cudaErrorNotSupported;
-    p.sched = sched_counters();
-    if (!p.sched) return cudaErrorUnknown;
+    if ((int64_t)p.total_pairs * p.BH > 0x7ffffff0ll - 2 * 148) return cudaErrorNotSupported;
+    p.sched = sched_counters(st);   // NULL: static deal
 
-    // tensor maps, cached for repeated calls on the same tensors
+    // tensor maps, cached for repeated calls on the same tensors with the same layout (the addresses are
+    // part of the key only; nothing is read through them after the call)
     static std::mutex mu;
     static MapCacheKey cached_key{};
     static TmaMaps cached_maps;
@@ -566,7 +627,7 @@ cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, v
     TmaMaps maps;
     {
         std::lock_guard<std::mutex> lock(mu);
-        MapCacheKey key{q, k, v, o, B, H, D, L.n_chunks, L.c, L.t, L.tail_read, sb, sh, ss};
+        MapCacheKey key{q, k, v, o, B, H, D, L.n_chunks, L.c, L.t, L.tail_read, L.flags, sb, sh, ss};
         if (!(have_cache && key == cached_key)) {
             TmaMaps mnew{};
             const void* bases[4] = {q, k, v, o};
@@ -604,9 +665,8 @@ cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, v
         sm_count[dev] = sms;
     }
     const int sms = sm_count[dev];
-    const int64_t work = (int64_t)p.total_tiles * p.BH;
-    const int64_t want = (work + 1) / 2;            // two streams (query tiles in flight) per CTA
-    const int grid = (int)(want < sms ? want : sms);
+    const int64_t work = (int64_t)p.total_pairs * p.BH;
+    const int grid = (int)(work < sms ? work : sms);
     // the shared-memory footprint also keeps one CTA per SM (each allocates all 512 TMEM columns)
     if (D == 128)
         masked_attn_tc_kernel<128><<<grid, TC_THREADS, TcSmem<128>::TOTAL + 1024, st>>>(maps, p);

@@ -11,6 +11,7 @@ namespace loma {
 
 static std::atomic<uint64_t> g_launches{0};
 void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+static std::atomic<uint64_t> g_fallbacks{0};
 
 __device__ int g_status_word = 0;
 
@@ -69,6 +70,8 @@ extern "C" {
 int loma_version(void) { return 100; }
 
 uint64_t loma_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+uint64_t loma_fallback_count(void) { return g_fallbacks.load(std::memory_order_relaxed); }
 
 const char* loma_status_string(int status) {
     switch (status) {
@@ -133,6 +136,7 @@ int loma_masked_attn_fwd(const void* q, const void* k, const void* v, void* o, f
     if (o == q || o == k || o == v) return LOMA_ERR_INVALID_ARG;
     if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
     if (stride_s < D || stride_b < 0 || stride_h < 0) return LOMA_ERR_INVALID_ARG;
+    if ((stride_b == 0 && B > 1) || (stride_h == 0 && H > 1)) return LOMA_ERR_INVALID_ARG;   // rows of two (b, h) would coincide
     const size_t es = elt_size(dtype);
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return LOMA_ERR_ALIGNMENT;
     if ((stride_b * es) % 16 || (stride_h * es) % 16 || (stride_s * es) % 16) return LOMA_ERR_ALIGNMENT;
@@ -143,8 +147,10 @@ int loma_masked_attn_fwd(const void* q, const void* k, const void* v, void* o, f
     cudaError_t e = cudaErrorNotSupported;
     if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC))
         e = launch_masked_attn_tc(q, k, v, o, lse, B, H, D, L, stride_b, stride_h, stride_s, scale, st);
-    if (e == cudaErrorNotSupported)
+    if (e == cudaErrorNotSupported) {
+        if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC)) g_fallbacks.fetch_add(1, std::memory_order_relaxed);
         e = launch_masked_attn_generic(q, k, v, o, lse, B, H, D, L, stride_b, stride_h, stride_s, dtype, scale, st);
+    }
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 
@@ -180,6 +186,7 @@ int loma_masked_attn_bwd(const void* q, const void* k, const void* v, const void
     }
     if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
     if (stride_s < D || stride_b < 0 || stride_h < 0) return LOMA_ERR_INVALID_ARG;
+    if ((stride_b == 0 && B > 1) || (stride_h == 0 && H > 1)) return LOMA_ERR_INVALID_ARG;   // rows of two (b, h) would coincide
     const size_t es = elt_size(dtype);
     for (const void* p : ins) if (!aligned16(p)) return LOMA_ERR_ALIGNMENT;
     for (void* p : outs) if (!aligned16(p)) return LOMA_ERR_ALIGNMENT;
@@ -207,6 +214,7 @@ int loma_masked_attn_bwd(const void* q, const void* k, const void* v, const void
             return LOMA_ERR_CUDA;
         }
     }
+    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC)) g_fallbacks.fetch_add(1, std::memory_order_relaxed);
     const cudaError_t e = launch_masked_attn_bwd_generic(q, k, v, o, d_o, lse, dq, dk, dv, delta, B, H, D, L, stride_b,
                                                          stride_h, stride_s, dtype, scale, generic_parts, st);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
@@ -227,6 +235,7 @@ int loma_rope_apply(void* q, void* k, int B, int H, int D, int n_chunks, int c, 
     if (q && q == k) return LOMA_ERR_INVALID_ARG;
     if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
     if (stride_s < D || stride_b < 0 || stride_h < 0) return LOMA_ERR_INVALID_ARG;
+    if ((stride_b == 0 && B > 1) || (stride_h == 0 && H > 1)) return LOMA_ERR_INVALID_ARG;   // rows of two (b, h) would coincide
     const size_t es = elt_size(dtype);
     if ((q && !aligned16(q)) || (k && !aligned16(k))) return LOMA_ERR_ALIGNMENT;
     if ((stride_b * es) % 16 || (stride_h * es) % 16 || (stride_s * es) % 16) return LOMA_ERR_ALIGNMENT;
@@ -258,6 +267,7 @@ int loma_prefill_cache(const void* k, const void* v, void* k_cache, void* v_cach
     if (!k || !v || !k_cache || !v_cache) return LOMA_ERR_INVALID_ARG;
     if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
     if (stride_s < D || stride_b < 0 || stride_h < 0) return LOMA_ERR_INVALID_ARG;
+    if ((stride_b == 0 && B > 1) || (stride_h == 0 && H > 1)) return LOMA_ERR_INVALID_ARG;   // rows of two (b, h) would coincide
     const size_t es = elt_size(dtype);
     if (!aligned16(k) || !aligned16(v) || !aligned16(k_cache) || !aligned16(v_cache)) return LOMA_ERR_ALIGNMENT;
     if ((stride_b * es) % 16 || (stride_h * es) % 16 || (stride_s * es) % 16) return LOMA_ERR_ALIGNMENT;
@@ -276,6 +286,13 @@ int loma_masked_attn_plan_coverage(int n_chunks, int c, int t, int tail_read, un
     if ((int64_t)L.S * L.S > (1ll << 32)) return LOMA_ERR_INVALID_ARG;
     if (L.S > 0) plan_coverage_host(L, counts);
     return LOMA_OK;
+}
+
+int loma_masked_attn_pair_plan_check(int n_chunks, int c, int t, int tail_read, unsigned flags) {
+    Layout L;
+    const int rc = make_layout(n_chunks, c, t, tail_read, flags, &L);
+    if (rc != LOMA_OK) return rc;
+    return L.S > 0 ? pair_plan_check_host(L) : 0;
 }
 
 int loma_masked_attn_bwd_plan_coverage(int n_chunks, int c, int t, int tail_read, unsigned flags, uint8_t* counts) {

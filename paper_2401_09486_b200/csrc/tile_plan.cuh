@@ -57,13 +57,14 @@ struct FwdParams {
     View view[4];
     int n_chunks, s, S, H, BH;
     int total_tiles;
+    int total_pairs;    // pairs of query tiles (the forward's unit of work), see decode_pair
     int n_tail, n_read, n_mem, n_rep;   // tiles per view, in scheduling order
     unsigned flags;
     FastDiv dBH, dH;
     float scale_log2;
     float* lse;
     int* status;
-    unsigned* sched;   // [0] next tile to hand out, [1] CTAs that have finished (the last one clears both)
+    unsigned* sched;   // [0] next pair to hand out, [1] CTAs that have finished (the last one clears both); NULL = static deal
 };
 
 
@@ -86,12 +87,8 @@ __host__ __device__ __forceinline__ int tiles_covering(const View& v, int nchunk
     return v.Z >= 128 ? nchunks * v.tpc : fdiv(nchunks + v.CH - 1, v.dCH);
 }
 
-__host__ __device__ __forceinline__ void decode_tile(const FwdParams& p, int rank, TileDesc& td) {
-    int view, qi;
-    if (rank < p.n_tail) { view = V_TAIL; qi = p.n_tail - 1 - rank; }
-    else if ((rank -= p.n_tail) < p.n_read) { view = V_READ; qi = p.n_read - 1 - rank; }
-    else if ((rank -= p.n_read) < p.n_mem) { view = V_MEM; qi = p.n_mem - 1 - rank; }
-    else { view = V_REP; qi = rank - p.n_mem; }
+// Tile qi of a view: its geometry and the key tiles it visits (two runs of consecutive tiles).
+__host__ __device__ __forceinline__ void decode_tile_at(const FwdParams& p, int view, int qi, TileDesc& td) {
     const View& g = p.view[view];
     td.view = view; td.qi = qi;
     int c1;
@@ -119,6 +116,16 @@ __host__ __device__ __forceinline__ void decode_tile(const FwdParams& p, int ran
         td.seg[1] = Seg{V_REP, M_DIAG, qi, 1};
     }
     td.nsteps = td.seg[0].count + td.seg[1].count;
+}
+
+// Tiles in scheduling order (longest first): tail, reading (last chunk first), memory, repetition.
+__host__ __device__ __forceinline__ void decode_tile(const FwdParams& p, int rank, TileDesc& td) {
+    int view, qi;
+    if (rank < p.n_tail) { view = V_TAIL; qi = p.n_tail - 1 - rank; }
+    else if ((rank -= p.n_tail) < p.n_read) { view = V_READ; qi = p.n_read - 1 - rank; }
+    else if ((rank -= p.n_read) < p.n_mem) { view = V_MEM; qi = p.n_mem - 1 - rank; }
+    else { view = V_REP; qi = rank - p.n_mem; }
+    decode_tile_at(p, view, qi, td);
 }
 
 __host__ __device__ __forceinline__ void step_ktile(const FwdParams& p, const TileDesc& td, int j, KTile& kt) {
@@ -203,6 +210,142 @@ struct HalfWalk {
     }
     __host__ __device__ __forceinline__ bool first_of_step(const HalfMasks&) const { return h == 0 || !(cur & 1u); }
     __host__ __device__ __forceinline__ bool last_of_step(const HalfMasks&) const { return h == 1 || !(cur & 2u); }
+};
+
+// ------------------------------------------------------------------ pairs of query tiles
+// The forward kernel gives a CTA two query tiles at a time -- tiles 2i and 2i + 1 of one view and one
+// (batch, head) -- and feeds both from ONE stream of key tiles: consecutive tiles of a view visit almost
+// the same keys (two reading tiles see the same earlier memory zones), so a key tile both of them visit
+// is loaded once.  Each tile keeps its own list of steps (decode_tile_at); the pair adds the order in which
+// the union of the two lists is loaded ("merged steps").  Per run of a tile's list (seg[0], seg[1]):
+//   * both runs start at the same key tile  -> merged run = the longer one; step k of either tile is merged
+//     step k (the tiles share every step both have);
+//   * otherwise                             -> the two runs are interleaved (A0 B0 A1 B1 ... then the rest
+//     of the longer one) and no step is shared (a key tile both happen to visit is then loaded twice).
+// A tile's steps keep their order in the merged list, which is all the kernel's roles rely on.
+struct PairMap {
+    int ca0, ca1, cb0, cb1;   // steps of tile A / B in run 0 / 1 (0 for an absent tile)
+    int same0, same1;         // run l starts at the same key tile for both tiles
+    int mc0;                  // merged steps of run 0
+    int nmerged;              // merged steps of the pair
+    // (scalar fields and selects instead of arrays: the kernel's roles keep this in registers)
+    __host__ __device__ __forceinline__ int cnt(int x, int l) const { return x ? (l ? cb1 : cb0) : (l ? ca1 : ca0); }
+    __host__ __device__ __forceinline__ int same(int l) const { return l ? same1 : same0; }
+};
+struct PairDesc {
+    TileDesc td[2];
+    int nb;          // 1 if tile B exists
+    PairMap pm;
+};
+
+__host__ __device__ __forceinline__ void make_pair_map(const TileDesc& a, const TileDesc& b, int nb, PairMap& pm) {
+    pm.ca0 = a.seg[0].count; pm.ca1 = a.seg[1].count;
+    pm.cb0 = nb ? b.seg[0].count : 0; pm.cb1 = nb ? b.seg[1].count : 0;
+    pm.same0 = nb && pm.ca0 > 0 && pm.cb0 > 0 && a.seg[0].view == b.seg[0].view && a.seg[0].first == b.seg[0].first;
+    pm.same1 = nb && pm.ca1 > 0 && pm.cb1 > 0 && a.seg[1].view == b.seg[1].view && a.seg[1].first == b.seg[1].first;
+    pm.mc0 = pm.same0 ? plan_max(pm.ca0, pm.cb0) : pm.ca0 + pm.cb0;
+    pm.nmerged = pm.mc0 + (pm.same1 ? plan_max(pm.ca1, pm.cb1) : pm.ca1 + pm.cb1);
+}
+
+// Pairs in scheduling order (longest first), the order of decode_tile taken two tiles at a time.
+__host__ __device__ __forceinline__ int pairs_of(int ntiles) { return (ntiles + 1) >> 1; }
+__host__ __device__ __forceinline__ void pair_tiles(const FwdParams& p, int rank, int& view, int& qa, int& nb) {
+    int pi, nt;
+    const int pt = pairs_of(p.n_tail), pr = pairs_of(p.n_read), pmm = pairs_of(p.n_mem);
+    if (rank < pt) { view = V_TAIL; nt = p.n_tail; pi = pt - 1 - rank; }
+    else if ((rank -= pt) < pr) { view = V_READ; nt = p.n_read; pi = pr - 1 - rank; }
+    else if ((rank -= pr) < pmm) { view = V_MEM; nt = p.n_mem; pi = pmm - 1 - rank; }
+    else { view = V_REP; nt = p.n_rep; pi = rank - pmm; }
+    qa = 2 * pi;
+    nb = (qa + 1 < nt) ? 1 : 0;
+}
+__host__ __device__ __forceinline__ void decode_pair(const FwdParams& p, int rank, PairDesc& pd) {
+    int view, qa;
+    pair_tiles(p, rank, view, qa, pd.nb);
+    decode_tile_at(p, view, qa, pd.td[0]);
+    if (pd.nb) decode_tile_at(p, view, qa + 1, pd.td[1]);
+    else pd.td[1] = pd.td[0];
+    make_pair_map(pd.td[0], pd.td[1], pd.nb, pd.pm);
+}
+
+// Merged index of step j of tile x.
+__host__ __device__ __forceinline__ int merged_index(const PairMap& pm, int x, int j) {
+    const int c0 = pm.cnt(x, 0);
+    const int l = j >= c0 ? 1 : 0;
+    const int k = l ? j - c0 : j;
+    const int base = l ? pm.mc0 : 0;
+    if (pm.same(l)) return base + k;
+    const int mn = plan_min(pm.cnt(0, l), pm.cnt(1, l));
+    return base + (k < mn ? 2 * k + x : mn + k);
+}
+// Merged step m -> the tile whose list names its key tile (A where both do) and that tile's step.
+__host__ __device__ __forceinline__ void merged_source(const PairMap& pm, int m, int& x, int& j) {
+    const int l = m >= pm.mc0 ? 1 : 0;
+    const int k = l ? m - pm.mc0 : m;
+    const int ca = pm.cnt(0, l), cb = pm.cnt(1, l);
+    int kk;
+    if (pm.same(l)) { x = k < ca ? 0 : 1; kk = k; }
+    else {
+        const int mn = plan_min(ca, cb);
+        if (k < 2 * mn) { x = k & 1; kk = k >> 1; }
+        else { x = ca > cb ? 0 : 1; kk = k - mn; }
+    }
+    j = kk + (l ? pm.cnt(x, 0) : 0);
+}
+// Does tile x visit merged step m?
+__host__ __device__ __forceinline__ bool visits_merged(const PairMap& pm, int x, int m) {
+    const int l = m >= pm.mc0 ? 1 : 0;
+    const int k = l ? m - pm.mc0 : m;
+    const int ca = pm.cnt(0, l), cb = pm.cnt(1, l);
+    if (pm.same(l)) return k < (x ? cb : ca);
+    const int mn = plan_min(ca, cb);
+    if (k < 2 * mn) return (k & 1) == x;
+    return (ca > cb ? 0 : 1) == x;
+}
+
+// The tensor-core instructions of one tile of a pair, in the order its issuing warp gives them:
+// S(step 0), PV(step 0, visited halves), S(step 1), ... (a tile has one score region, so the score product of
+// a step follows the last P.V of the step before).  Each tile of a pair has its own issuing warp; the two
+// meet only at the K/V ring: a stage is refilled after TWO releases, one per tile that visits the step, or
+// both from the only visitor (release = 2).  The host replays both walks against the ring (pair_plan_check)
+// and verifies that neither they nor the loads can block for ever.
+struct IssueAct {
+    int is_s;            // score product (1) or P.V product (0)
+    int m;               // merged step
+    int h;               // P.V: half of the key tile; S: unused
+    unsigned cur;        // S: visited halves of the step (1, 2 or 3)
+    int first_of_step;   // P.V: first visited half of its step (the V tile is first needed here)
+    int first_event;     // first of the tile: S waits for the Q tile, P.V overwrites the accumulator
+    int last_s;          // S: the tile's last score product (its Q buffer is free afterwards)
+    int release;         // releases of the step's K stage (after S) or V stage (after the step's last P.V): 0, 1 or 2
+};
+struct TileIssue {
+    HalfMasks hm;
+    HalfWalk w;      // next step / half to issue for
+    int nsteps;
+    int need_s;      // the next instruction is the score product of step w.j
+    __host__ __device__ __forceinline__ void start(const HalfMasks& hm_, int nsteps_) {
+        hm = hm_; nsteps = nsteps_; need_s = 1; w.start(hm);
+    }
+    __host__ __device__ __forceinline__ bool done() const { return w.done(nsteps); }
+    // the next instruction of tile x; call only while !done()
+    __host__ __device__ __forceinline__ void next(const PairMap& pm, int x, IssueAct& act) {
+        const int m = merged_index(pm, x, w.j);
+        const int rel = visits_merged(pm, 1 - x, m) ? 1 : 2;
+        act.m = m; act.is_s = need_s; act.h = w.h; act.cur = w.cur;
+        act.first_of_step = w.first_of_step(hm);
+        act.first_event = (w.j == 0) && act.first_of_step;
+        act.last_s = w.j == nsteps - 1;
+        if (need_s) {
+            act.release = rel;
+            need_s = 0;
+        } else {
+            const bool los = w.last_of_step(hm);
+            act.release = los ? rel : 0;
+            w.next(hm);
+            if (los) need_s = 1;
+        }
+    }
 };
 
 // ------------------------------------------------------------------ the plan read by key tile
@@ -353,6 +496,7 @@ inline void make_plan(const Layout& L, int B, int H, FwdParams* p) {
     p->n_tail = p->view[V_TAIL].ntiles; p->n_read = p->view[V_READ].ntiles;
     p->n_mem = p->view[V_MEM].ntiles; p->n_rep = p->view[V_REP].ntiles;
     p->total_tiles = p->n_tail + p->n_read + p->n_mem + p->n_rep;
+    p->total_pairs = (p->n_tail + 1) / 2 + (p->n_read + 1) / 2 + (p->n_mem + 1) / 2 + (p->n_rep + 1) / 2;
     p->flags = L.flags;
     p->dBH = make_fastdiv(p->BH); p->dH = make_fastdiv(H);
 }

@@ -101,6 +101,8 @@ def test_masked_attn_fwd_validation_precedes_any_cuda_call(lib):
     assert _fwd(lib, q=0x1008) == ALIGNMENT
     assert _fwd(lib, ss=68, dt=1) == ALIGNMENT          # 136-byte row stride
     assert _fwd(lib, ss=32) == INVALID                  # rows overlap
+    assert _fwd(lib, B=2, sb=0) == INVALID              # two batch elements on the same rows
+    assert _fwd(lib, H=3, sh=0) == INVALID              # two heads on the same rows
     assert _fwd(lib, t=0, tc=0, n=1) == INVALID         # t == 0 needs n_chunks == 0
     assert _fwd(lib, tail=5) == INVALID                 # tail longer than a reading zone
     assert _fwd(lib, n=0, t=2, tc=4, tail=0) == 0       # empty sequence: no-op
@@ -171,6 +173,16 @@ def test_tensor_core_tile_plan_reproduces_the_mask_exactly(lib, n, c, t, tail, f
     want = oracle.dense_mask(n, c, t, tail, flags).astype(np.uint8)
     assert got.shape == want.shape
     assert np.array_equal(got, want), f"{int((got != want).sum())} entries differ"
+
+
+@pytest.mark.parametrize("n,c,t,tail", PLAN_GEOMS + [(32, 4, 16, 0), (128, 8, 32, 0), (40, 2, 4, 3), (7, 3, 12, 20)])
+@pytest.mark.parametrize("flags", [0, 1, 2, 3])
+def test_pair_schedule_of_the_forward_is_sound(lib, n, c, t, tail, flags):
+    """The forward kernel takes two neighbouring query tiles at a time and loads the union of their key
+    tiles once through a two-stage ring.  The host replay of that schedule must find every tile's steps in
+    increasing merged order, shared steps naming one key tile, every instruction's stage loadable from what
+    was issued before it (no wait can block for ever), and every stage released exactly once."""
+    assert binding.loma_masked_attn_pair_plan_check(n, c, t, tail, flags) == 0
 
 
 def test_masked_attn_bwd_validation(lib):
@@ -245,6 +257,7 @@ def test_both_sides_of_the_plan_on_seeded_random_geometries(lib, n, c, t, tail, 
     by_key = binding.loma_masked_attn_bwd_plan_coverage(n, c, t, tail, flags).numpy()
     assert np.array_equal(by_query, want), f"query side: {int((by_query != want).sum())} entries differ"
     assert np.array_equal(by_key, want), f"key side: {int((by_key != want).sum())} entries differ"
+    assert binding.loma_masked_attn_pair_plan_check(n, c, t, tail, flags) == 0
 
 
 def test_ragged_decode_validation(lib):
