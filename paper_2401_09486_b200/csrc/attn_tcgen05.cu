@@ -54,6 +54,31 @@ struct TmaMaps {
     CUtensorMap q[4], k[4], v[4], o[4];
 };
 
+// Optional clock counters of the roles' waits and a time line of the first CTA's events (compiled in with
+// -DLOMA_KERNEL_TIMERS only; a development aid, read back with loma_debug_read_timers / _trace).
+#ifdef LOMA_KERNEL_TIMERS
+__device__ unsigned long long g_timers[160][48];
+__device__ unsigned long long g_trace[8][4096];
+#define TRACE(role, idx) do { if (blockIdx.x == 0 && (idx) < 4096) g_trace[role][idx] = (unsigned long long)clock64(); } while (0)
+#define TIMER_DECL unsigned long long tmr_[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}; long long tmr_t0_ = 0; const long long tmr_begin_ = clock64()
+#define TIMER_START() (tmr_t0_ = clock64())
+#define TIMER_STOP(i) (tmr_[i] += (unsigned long long)(clock64() - tmr_t0_))
+#define TIMER_COUNT(i) (++tmr_[i])
+#define TIMER_FLUSH(base, n)                                                                    \
+    do {                                                                                        \
+        tmr_[(n) - 1] = (unsigned long long)(clock64() - tmr_begin_);                           \
+        if (blockIdx.x < 160)                                                                   \
+            for (int i_ = 0; i_ < (n); ++i_) g_timers[blockIdx.x][(base) + i_] += tmr_[i_];     \
+    } while (0)
+#else
+#define TRACE(role, idx) ((void)0)
+#define TIMER_DECL
+#define TIMER_START() ((void)0)
+#define TIMER_STOP(i) ((void)0)
+#define TIMER_COUNT(i) ((void)0)
+#define TIMER_FLUSH(base, n) ((void)0)
+#endif
+
 // ------------------------------------------------------------------ the kernel
 constexpr int TC_THREADS = 384;   // 2 softmax warpgroups + 1 warpgroup holding the TMA warp and the two MMA warps
 constexpr int TMEM_COLS = 512;
@@ -63,15 +88,15 @@ enum {
     B_QF = 0,    // +x   Q tile of A / B has landed
     B_QE = 2,    // +x   every score product of the pair's tile x has completed: Q buffer free
     B_KF = 4,    // +s   K tile of ring stage s has landed
-    B_KE = 6,    // +s   every score product that reads stage s has completed (two arrivals: one per tile, or both from the only visitor)
+    B_KE = 6,    // +s   every score product that reads stage s has completed (two arrivals: one per tile that visits the step, the missing one from the loader)
     B_VF = 8,    // +s
     B_VE = 10,   // +s   every P.V product that reads stage s has completed (two arrivals, as B_KE)
-    B_SF = 12,   // +x   scores of tile x's current step are in TMEM
-    B_PF = 14,   // +2x+(event & 1)   probabilities of an event are in TMEM (128 arrivals)
-    B_OF = 18,   // +2x+(event & 1)   the P.V product of an event of tile x has completed
-    B_TF = 22,   // +(n & 3)  the n-th pair number has been posted in slot n & 3 of the pair ring
-    B_TE = 26,   // +(n & 3)  every reader (8 softmax warps, 2 MMA warps) has taken the n-th pair number
-    NBAR = 30
+    B_SF = 12,   // +2x+(event & 1)   scores of an event of tile x are in TMEM
+    B_PF = 16,   // +2x+(event & 1)   probabilities of an event are in TMEM (128 arrivals)
+    B_OF = 20,   // +2x+(event & 1)   the P.V product of an event of tile x has completed
+    B_TF = 24,   // +(n & 3)  the n-th pair number has been posted in slot n & 3 of the pair ring
+    B_TE = 28,   // +(n & 3)  every reader (8 softmax warps, 2 MMA warps) has taken the n-th pair number
+    NBAR = 32
 };
 
 // Shared memory: Q_A, Q_B, ring of two (K, V) stages, one output staging panel per tile.
@@ -152,6 +177,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             uint32_t gl = 0, pcount = 0;      // K/V loads so far (one per merged step), pairs so far
             uint32_t nq[2] = {0, 0};          // uses of each Q buffer so far
             bool ok = true;
+            TIMER_DECL;
             for (;; ++pcount) {
                 int w = p.sched ? (int)atomicAdd(p.sched, 1u) : (int)(blockIdx.x + pcount * gridDim.x);
                 if (w >= total_work || !ok) w = -1;
@@ -169,7 +195,9 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
 #pragma unroll
                 for (int x = 0; x < 2; ++x) {
                     if (x == 1 && !pd.nb) break;
+                    TIMER_START();
                     if (nq[x] > 0) ok = mbar_wait(bar(B_QE + x), (nq[x] - 1) & 1, abortp, p.status);
+                    TIMER_STOP(0);
                     if (!ok) break;
                     ++nq[x];
                     mbar_expect_tx(bar(B_QF + x), qv.R * qv.CH * 128 * PANELS);
@@ -187,21 +215,30 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     const View& kv = p.view[kt.view];
                     const uint32_t s = gl & 1, ph = (gl >> 1) & 1;
                     const uint32_t bytes = kv.R * kv.CH * 128 * PANELS;
+                    // a stage is released by two arrivals; where only one tile visits the step, the other one is given here
+                    const bool lone = !visits_merged(pd.pm, 1 - x, m);
+                    TIMER_START();
                     ok = mbar_wait(bar(B_KE + s), ph ^ 1, abortp, p.status);
+                    TIMER_STOP(1);
                     if (!ok) break;
                     mbar_expect_tx(bar(B_KF + s), bytes);
                     for (int pn = 0; pn < PANELS; ++pn)
                         tma_load_5d(smem_base + SM::K_OFF + s * 2 * SM::TILE_BYTES + pn * SM::PANEL_BYTES, &maps.k[kt.view],
                                     bar(B_KF + s), pn * 64, kt.r0, kt.c0, hi, bi);
+                    if (lone) mbar_arrive(bar(B_KE + s));
+                    TIMER_START();
                     ok = mbar_wait(bar(B_VE + s), ph ^ 1, abortp, p.status);
+                    TIMER_STOP(2);
                     if (!ok) break;
                     mbar_expect_tx(bar(B_VF + s), bytes);
                     for (int pn = 0; pn < PANELS; ++pn)
                         tma_load_5d(smem_base + SM::V_OFF + s * 2 * SM::TILE_BYTES + pn * SM::PANEL_BYTES, &maps.v[kt.view],
                                     bar(B_VF + s), pn * 64, kt.r0, kt.c0, hi, bi);
+                    if (lone) mbar_arrive(bar(B_VE + s));
                 }
                 if (!ok) break;
             }
+            TIMER_FLUSH(0, 4);
             if (!ok) {
                 // leaving early (the abort flag is set): give copies in flight a bounded time to land
                 const long long t0 = clock64();
@@ -216,15 +253,15 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         const int X = warp - 9;
         // instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128
         constexpr uint32_t IDESC_S64 = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
-        constexpr uint32_t IDESC_S128 = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
         constexpr uint32_t IDESC_PV =
             (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | (((uint32_t)D >> 3) << 17) | ((128u >> 4) << 24);
         const uint32_t tm = tmem0 + X * 256;
         const uint64_t qd = smem_desc(smem_base + SM::Q_OFF + X * SM::TILE_BYTES, 16, 1024);
-        uint32_t ge = 0;                  // events (visited halves) issued on this tile slot, all pairs
+        uint32_t ge = 0, gse = 0;         // events (visited halves) whose P.V / whose scores have been issued on this slot, all pairs
         uint32_t nq = 0;                  // pairs in which this slot was used
         uint32_t gbase = 0, pcount = 0;   // merged steps of earlier pairs, pairs so far
         bool ok = true;
+        TIMER_DECL;
         for (;; ++pcount) {
             const int w = next_pair(pcount, ok);
             if (w < 0) break;
@@ -238,56 +275,68 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 pm = pd.pm;
                 mine = (X == 0) || pd.nb;
                 if (mine) {
-                    if (X) ti.start(tile_half_masks(p, pd.td[1], lane), pd.td[1].nsteps);
-                    else ti.start(tile_half_masks(p, pd.td[0], lane), pd.td[0].nsteps);
+                    if (X) ti.start(pm, 1, tile_half_masks(p, pd.td[1], lane), pd.td[1].nsteps);
+                    else ti.start(pm, 0, tile_half_masks(p, pd.td[0], lane), pd.td[0].nsteps);
                 }
             }
             if (mine) {
                 ++nq;
                 IssueAct act;
                 while (ok && !ti.done()) {
-                    ti.next(pm, X, act);
+                    TIMER_START();
+                    ti.next(act);
+                    TIMER_STOP(4);
                     const uint32_t gl = gbase + (uint32_t)act.m, s = gl & 1, ph = (gl >> 1) & 1;
                     if (act.is_s) {
+                        TIMER_START();
                         if (act.first_event)
                             ok = __all_sync(0xffffffffu, mbar_wait(bar(B_QF + X), (nq - 1) & 1, abortp, p.status));
-                        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_KF + s), ph, abortp, p.status));
+                        if (ok && act.first_of_step) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_KF + s), ph, abortp, p.status));
+                        TIMER_STOP(0);
                         if (!ok) break;
+                        TIMER_START();
                         tc_fence_after();
                         if (elect_one()) {
                             const uint64_t kd = smem_desc(smem_base + SM::K_OFF + s * 2 * SM::TILE_BYTES, 16, 1024);
-                            const uint32_t half_off = (act.cur == 2u) ? 1u : 0u;   // only the second half: keys 64.., columns 64..
-                            const uint32_t idesc = (act.cur == 3u) ? IDESC_S128 : IDESC_S64;
 #pragma unroll
                             for (int kk = 0; kk < D / 16; ++kk) {
                                 // descriptor start addresses are in 16-byte units; 64 key rows are 8192 bytes further
                                 const uint64_t off = (uint64_t)(((kk >> 2) * SM::PANEL_BYTES + (kk & 3) * 32) >> 4);
-                                mma_ss(tm + half_off * 64, qd + off, kd + off + (uint64_t)((half_off * 8192) >> 4), idesc, kk > 0);
+                                mma_ss(tm + (gse & 1) * 64, qd + off, kd + off + (uint64_t)((act.h * 8192) >> 4), IDESC_S64, kk > 0);
                             }
-                            tc_commit(bar(B_SF + X));
-                            tc_commit(bar(B_KE + s));
-                            if (act.release == 2) tc_commit(bar(B_KE + s));   // the other tile does not visit this step
+                            tc_commit(bar(B_SF + 2 * X + (gse & 1)));
+                            if (act.last_of_step) tc_commit(bar(B_KE + s));
                             if (act.last_s) tc_commit(bar(B_QE + X));
                         }
                         __syncwarp();
+                        TIMER_STOP(5);
+                        if (lane == 0) TRACE(4 * X + 2, gse);
+                        ++gse;
                     } else {
+                        TIMER_START();
                         ok = __all_sync(0xffffffffu, mbar_wait(bar(B_PF + 2 * X + (ge & 1)), (ge >> 1) & 1, abortp, p.status));
+                        TIMER_STOP(1);
+                        TIMER_START();
                         if (ok && act.first_of_step)
                             ok = __all_sync(0xffffffffu, mbar_wait(bar(B_VF + s), ph, abortp, p.status));
+                        TIMER_STOP(2);
+                        TIMER_COUNT(3);
                         if (!ok) break;
+                        TIMER_START();
                         tc_fence_after();
                         if (elect_one()) {
                             const uint64_t vd = smem_desc(smem_base + SM::V_OFF + s * 2 * SM::TILE_BYTES, SM::PANEL_BYTES, 1024);
                             const int h = act.h;
 #pragma unroll
                             for (int k4 = 0; k4 < 4; ++k4)
-                                mma_ts(tm + 128, tm + h * 64 + k4 * 8, vd + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_PV,
+                                mma_ts(tm + 128, tm + (ge & 1) * 64 + k4 * 8, vd + (uint64_t)(((h * 4 + k4) * 2048) >> 4), IDESC_PV,
                                        !act.first_event || (k4 > 0));
                             tc_commit(bar(B_OF + 2 * X + (ge & 1)));
-                            if (act.release >= 1) tc_commit(bar(B_VE + s));
-                            if (act.release == 2) tc_commit(bar(B_VE + s));
+                            if (act.last_of_step) tc_commit(bar(B_VE + s));
                         }
                         __syncwarp();
+                        TIMER_STOP(6);
+                        if (lane == 0) TRACE(4 * X + 3, ge);
                         ++ge;
                     }
                 }
@@ -295,6 +344,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             if (!ok) break;
             gbase += (uint32_t)pm.nmerged;
         }
+        if (lane == 0) TIMER_FLUSH(8 + 8 * X, 8);
     } else if (warp < 8) {
         // ------------------------------------------------------------ softmax + epilogue of tile X (128 threads)
         asm volatile("setmaxnreg.inc.sync.aligned.u32 208;" ::: "memory");
@@ -305,9 +355,9 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         const uint32_t o_stage = smem_base + SM::O_OFF + X * SM::PANEL_BYTES;
         uint8_t* o_stage_gen = smem_gen + SM::O_OFF + X * SM::PANEL_BYTES;
         uint32_t ge = 0;    // visited halves so far on this tile slot (see the MMA issuer)
-        uint32_t gst = 0;   // visited steps so far on this tile slot
         bool ok = true;
         bool store_pending = false;
+        TIMER_DECL;
         // Everything this thread needs to know about a tile.  The next tile is decoded while the last
         // product of the current one drains, so the decode's chain of dependent loads and integer
         // arithmetic stays off the path between two tiles.
@@ -369,19 +419,23 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     KTile kt;
                     step_ktile(p, td, hw.j, kt);
                     row_interval(p.view[kt.view], kt, rc, ro, rr, row_valid, lo, hi2);
-                    // the scores of both visited halves of the step arrive together
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF + X), gst & 1, abortp, p.status));
-                    if (!ok) break;
-                    ++gst;
-                    tc_fence_after();
                 }
-                // One visited half of a key tile (64 keys) per pass.
+                // One visited half of a key tile (64 keys) per pass, in score buffer ge & 1: the tensor
+                // pipe works on the other buffer while this warpgroup works on this one.
                 {
+                    const int b = ge & 1;
+                    TIMER_START();
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF + 2 * X + b), (ge >> 1) & 1, abortp, p.status));
+                    TIMER_STOP(0);
+                    if (!ok) break;
+                    if (rr == 0) TRACE(4 * X + 0, ge);
+                    tc_fence_after();
                     const int lo_h = lo - 64 * hw.h;                  // allowed columns of this half: [lo_h, lo_h + span)
                     const uint32_t span = (uint32_t)(hi2 - lo);
                     const bool full = __all_sync(0xffffffffu, lo_h <= 0 && hi2 - 64 * hw.h >= 64);
-                    const uint32_t sh_addr = s_addr + hw.h * 64;
+                    const uint32_t sh_addr = s_addr + b * 64;
                     uint32_t s[64];
+                    TIMER_START();
                     tmem_ld32(sh_addr, s);
                     tmem_ld32(sh_addr + 32, s + 32);
                     tmem_wait_ld();
@@ -400,7 +454,9 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     }
                     const float mrow = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
                     const bool need = mrow > m_used + 8.f;
+                    TIMER_STOP(1);
                     if (!first && __any_sync(0xffffffffu, need)) {
+                        TIMER_COUNT(6);
                         // rescale the accumulated output: wait until the previous event's P.V has landed in TMEM
                         ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + 2 * X + ((ge - 1) & 1)), ((ge - 1) >> 1) & 1, abortp, p.status));
                         if (!ok) break;
@@ -418,6 +474,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                         l *= alpha;
                     }
                     if (need) m_used = mrow;
+                    TIMER_START();
                     const float neg_ref = (m_used == -INFINITY) ? 0.f : -m_used;
                     const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nr2 = pack2(neg_ref, neg_ref);
                     uint64_t lsa = pack2(0.f, 0.f), lsb = lsa;
@@ -446,12 +503,17 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     tmem_wait_st();
                     tc_fence_before();
                     mbar_arrive(bar(B_PF + 2 * X + (ge & 1)));
+                    TIMER_STOP(2);
+                    if (rr == 0) TRACE(4 * X + 1, ge);
                 }
             }
+            TIMER_START();
             if (ok) w_next = next_ctx(nxt);
+            TIMER_STOP(3);
             // the last P.V of the tile belongs to event ge - 1 (products complete in issue order)
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(B_OF + 2 * X + ((ge - 1) & 1)), ((ge - 1) >> 1) & 1, abortp, p.status));
             if (ok) tc_fence_after();
+            TIMER_START();
 
             // epilogue: normalise, round to bf16, stage 64 output columns at a time in shared
             // memory, TMA store.  Every thread of the warpgroup reaches the first barrier for
@@ -498,6 +560,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 }
             }
             if (give_up) { ok = false; break; }
+            TIMER_STOP(4);
             tc_fence_before();
             if (p.lse && row_valid) {
                 const int64_t grow = (int64_t)rc * p.s + cur.zone_row0 + ro;
@@ -505,6 +568,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             }
         }
         if (rr == 0 && store_pending) tma_store_wait_all();
+        if (rr == 0) TIMER_FLUSH(24 + 8 * X, 8);
     }
 
     tc_fence_before();
@@ -523,6 +587,22 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         }
     }
 }
+
+#ifdef LOMA_KERNEL_TIMERS
+}  // namespace loma
+// development aids: copy the counters to out[160*48] and clear them / copy the time line to out[8*4096]
+extern "C" __attribute__((visibility("default"))) int loma_debug_read_timers(unsigned long long* out) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+    if (cudaMemcpyFromSymbol(out, loma::g_timers, sizeof(unsigned long long) * 160 * 48) != cudaSuccess) return -1;
+    static unsigned long long zeros[160 * 48] = {0};
+    return cudaMemcpyToSymbol(loma::g_timers, zeros, sizeof(zeros)) == cudaSuccess ? 0 : -1;
+}
+extern "C" __attribute__((visibility("default"))) int loma_debug_read_trace(unsigned long long* out) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+    return cudaMemcpyFromSymbol(out, loma::g_trace, sizeof(unsigned long long) * 8 * 4096) == cudaSuccess ? 0 : -1;
+}
+namespace loma {
+#endif
 
 // ------------------------------------------------------------------ bounded-wait self test
 // One thread waits on an mbarrier that nobody ever arrives on, with the same wait routine as the

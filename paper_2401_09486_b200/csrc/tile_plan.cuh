@@ -303,47 +303,87 @@ __host__ __device__ __forceinline__ bool visits_merged(const PairMap& pm, int x,
     return (ca > cb ? 0 : 1) == x;
 }
 
-// The tensor-core instructions of one tile of a pair, in the order its issuing warp gives them:
-// S(step 0), PV(step 0, visited halves), S(step 1), ... (a tile has one score region, so the score product of
-// a step follows the last P.V of the step before).  Each tile of a pair has its own issuing warp; the two
-// meet only at the K/V ring: a stage is refilled after TWO releases, one per tile that visits the step, or
-// both from the only visitor (release = 2).  The host replays both walks against the ring (pair_plan_check)
-// and verifies that neither they nor the loads can block for ever.
+// The tensor-core instructions of one tile of a pair, in the order its issuing warp gives them.  The unit is
+// one visited half of a key tile (an "event": 64 keys): S_e = Q K_h^T into one of two score buffers, and
+// O += P_e V_h once the warpgroup has turned the scores into probabilities.  The score products run two
+// events ahead of the P.V products (S0 S1 PV0 S2 PV1 S3 ... PV PV), so the tensor pipe fills one score
+// buffer while the warpgroup works on the other.  Each tile of a pair has its own issuing warp; the two
+// meet only at the K/V rings: a stage is refilled after TWO releases, one per tile that visits the step;
+// for a step only one tile visits, the loader gives the second one itself right after the load (it knows
+// the visitors).  The host replays both walks against the rings (pair_plan_check) and verifies that
+// neither they nor the loads can block for ever.
 struct IssueAct {
     int is_s;            // score product (1) or P.V product (0)
     int m;               // merged step
-    int h;               // P.V: half of the key tile; S: unused
-    unsigned cur;        // S: visited halves of the step (1, 2 or 3)
-    int first_of_step;   // P.V: first visited half of its step (the V tile is first needed here)
+    int h;               // half of the key tile
+    int first_of_step;   // first visited half of its step: S needs the K tile here, P.V the V tile
+    int last_of_step;    // last visited half of its step: afterwards this tile is done with the K (S) / V (P.V) stage
     int first_event;     // first of the tile: S waits for the Q tile, P.V overwrites the accumulator
     int last_s;          // S: the tile's last score product (its Q buffer is free afterwards)
-    int release;         // releases of the step's K stage (after S) or V stage (after the step's last P.V): 0, 1 or 2
 };
+// Kept small on purpose: the issuing warp runs this between two batches of tensor-core instructions, and
+// whatever it costs is added to the time the other roles wait for the next batch.  The visited-half masks
+// are kept shifted (bit 0 = the cursor's step, ones shifted in from the top: steps past 63 visit both
+// halves), the merged index is recomputed only when a cursor enters a new step.
 struct TileIssue {
-    HalfMasks hm;
-    HalfWalk w;      // next step / half to issue for
+    unsigned long long sm0, sm1, pm0, pm1;   // shifted masks of the S cursor / the P.V cursor
+    int sj, sh, pj, ph;                      // step and half of the two cursors
+    int s_m, p_m;                            // merged index of the cursors' steps
+    int ns, np;                              // events whose S / whose P.V has been issued
     int nsteps;
-    int need_s;      // the next instruction is the score product of step w.j
-    __host__ __device__ __forceinline__ void start(const HalfMasks& hm_, int nsteps_) {
-        hm = hm_; nsteps = nsteps_; need_s = 1; w.start(hm);
+    int x, c0, mc0, same0, same1, mn0, mn1;  // what merged_index needs, unpacked for tile x
+    __host__ __device__ __forceinline__ int midx(int j) const {
+        const int l = j >= c0 ? 1 : 0;
+        const int k = l ? j - c0 : j;
+        const int mn = l ? mn1 : mn0;
+        return (l ? mc0 : 0) + ((l ? same1 : same0) ? k : (k < mn ? 2 * k + x : mn + k));
     }
-    __host__ __device__ __forceinline__ bool done() const { return w.done(nsteps); }
-    // the next instruction of tile x; call only while !done()
-    __host__ __device__ __forceinline__ void next(const PairMap& pm, int x, IssueAct& act) {
-        const int m = merged_index(pm, x, w.j);
-        const int rel = visits_merged(pm, 1 - x, m) ? 1 : 2;
-        act.m = m; act.is_s = need_s; act.h = w.h; act.cur = w.cur;
-        act.first_of_step = w.first_of_step(hm);
-        act.first_event = (w.j == 0) && act.first_of_step;
-        act.last_s = w.j == nsteps - 1;
-        if (need_s) {
-            act.release = rel;
-            need_s = 0;
+    __host__ __device__ __forceinline__ void start(const PairMap& pm, int x_, const HalfMasks& hm, int nsteps_) {
+        x = x_; nsteps = nsteps_;
+        c0 = pm.cnt(x, 0); mc0 = pm.mc0; same0 = pm.same0; same1 = pm.same1;
+        mn0 = plan_min(pm.ca0, pm.cb0); mn1 = plan_min(pm.ca1, pm.cb1);
+        sm0 = pm0 = hm.m[0]; sm1 = pm1 = hm.m[1];
+        sj = pj = 0; ns = np = 0;
+        sh = ph = (hm.m[0] & 1ull) ? 0 : 1;
+        s_m = p_m = midx(0);
+    }
+    __host__ __device__ __forceinline__ bool done() const { return pj >= nsteps; }
+    // the next instruction of the tile; call only while !done()
+    __host__ __device__ __forceinline__ void next(IssueAct& act) {
+        const bool is_s = sj < nsteps && ns < np + 2;
+        act.is_s = is_s;
+        if (is_s) {
+            const unsigned cur = (unsigned)(sm0 & 1ull) | ((unsigned)(sm1 & 1ull) << 1);
+            const bool los = sh == 1 || !(cur & 2u);
+            act.m = s_m; act.h = sh;
+            act.first_of_step = sh == 0 || !(cur & 1u);
+            act.last_of_step = los;
+            act.first_event = ns == 0;
+            act.last_s = los && sj == nsteps - 1;
+            ++ns;
+            if (!los) { sh = 1; }
+            else {
+                ++sj;
+                sm0 = (sm0 >> 1) | (1ull << 63); sm1 = (sm1 >> 1) | (1ull << 63);
+                sh = (sm0 & 1ull) ? 0 : 1;
+                s_m = midx(sj);
+            }
         } else {
-            const bool los = w.last_of_step(hm);
-            act.release = los ? rel : 0;
-            w.next(hm);
-            if (los) need_s = 1;
+            const unsigned cur = (unsigned)(pm0 & 1ull) | ((unsigned)(pm1 & 1ull) << 1);
+            const bool los = ph == 1 || !(cur & 2u);
+            act.m = p_m; act.h = ph;
+            act.first_of_step = ph == 0 || !(cur & 1u);
+            act.last_of_step = los;
+            act.first_event = np == 0;
+            act.last_s = 0;
+            ++np;
+            if (!los) { ph = 1; }
+            else {
+                ++pj;
+                pm0 = (pm0 >> 1) | (1ull << 63); pm1 = (pm1 >> 1) | (1ull << 63);
+                ph = (pm0 & 1ull) ? 0 : 1;
+                p_m = midx(pj);
+            }
         }
     }
 };

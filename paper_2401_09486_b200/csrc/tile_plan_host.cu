@@ -68,8 +68,8 @@ void plan_coverage_host(const Layout& L, uint8_t* counts) {
 //   2. with a two-stage K/V ring that is filled in order (K0 V0 K1 V1 ...) and refilled after two releases,
 //      the loader and the two tiles' issuers, each running as far as the ring lets it, all reach the end
 //      (no wait can block for ever);
-//   3. every K and V stage is released exactly twice, every tile issues one score product per step and
-//      one P.V product per visited half, and the Q buffer is released once per tile.
+//   3. every K and V stage is released exactly twice, every tile issues one score product and one P.V
+//      product per visited half, and the Q buffer is released once per tile.
 int pair_plan_check_host(const Layout& L) {
     FwdParams p{};
     make_plan(L, 1, 1, &p);
@@ -116,25 +116,27 @@ int pair_plan_check_host(const Layout& L) {
         const HalfMasks hma = host_half_masks(p, pd.td[0]);
         const HalfMasks hmb = pd.nb ? host_half_masks(p, pd.td[1]) : hma;
         TileIssue ti[2];
-        ti[0].start(hma, pd.td[0].nsteps);
-        ti[1].start(hmb, pd.nb ? pd.td[1].nsteps : 0);
-        if (!pd.nb) { ti[1].w.j = 0; ti[1].nsteps = 0; }
+        ti[0].start(pm, 0, hma, pd.td[0].nsteps);
+        ti[1].start(pm, 1, hmb, pd.nb ? pd.td[1].nsteps : 0);
         int* rel_k = new int[nm]();
         int* rel_v = new int[nm]();
         int kl = 0, vl = 0;   // K / V tiles loaded so far, in the order K0 V0 K1 V1 ...
         int n_s[2] = {0, 0}, n_pv[2] = {0, 0}, n_q[2] = {0, 0};
         IssueAct pending[2];
         bool have[2] = {false, false};
-        int last_m[2] = {-1, -1};
+        int last_m[2][2] = {{-1, -1}, {-1, -1}};   // per tile: last merged step of a P.V / of a score product
         for (long guard = 0;; ++guard) {
             if (guard > 16l * nm + 64) { ++bad; break; }
             bool moved = false;
             for (;;) {   // the loader
+                // (the loader gives the second release itself where only one tile visits the step)
                 if (kl == vl) {
                     if (kl >= nm || !(kl < 2 || rel_k[kl - 2] == 2)) break;
+                    rel_k[kl] += 2 - (int)visits_merged(pm, 0, kl) - (int)visits_merged(pm, 1, kl);
                     ++kl;
                 } else {
                     if (!(vl < 2 || rel_v[vl - 2] == 2)) break;
+                    rel_v[vl] += 2 - (int)visits_merged(pm, 0, vl) - (int)visits_merged(pm, 1, vl);
                     ++vl;
                 }
                 moved = true;
@@ -143,23 +145,23 @@ int pair_plan_check_host(const Layout& L) {
                 for (;;) {
                     if (!have[x]) {
                         if (ti[x].done()) break;
-                        ti[x].next(pm, x, pending[x]);
+                        ti[x].next(pending[x]);
                         have[x] = true;
-                        if (pending[x].m < last_m[x] || pending[x].m < 0 || pending[x].m >= nm) ++bad;
-                        last_m[x] = pending[x].m;
+                        int& lm = last_m[x][pending[x].is_s ? 1 : 0];
+                        if (pending[x].m < lm || pending[x].m < 0 || pending[x].m >= nm) ++bad;
+                        lm = pending[x].m;
                     }
                     const IssueAct& act = pending[x];
                     if (act.m < 0 || act.m >= nm) { have[x] = false; continue; }
                     if (act.is_s) {
                         if (kl <= act.m) break;   // waits for the K tile
                         ++n_s[x];
-                        rel_k[act.m] += act.release;
-                        if (act.release < 1) ++bad;
+                        rel_k[act.m] += act.last_of_step;
                         if (act.last_s) ++n_q[x];
                     } else {
                         if (vl <= act.m) break;   // waits for the V tile (the probabilities always come)
                         ++n_pv[x];
-                        rel_v[act.m] += act.release;
+                        rel_v[act.m] += act.last_of_step;
                     }
                     have[x] = false;
                     moved = true;
@@ -174,7 +176,7 @@ int pair_plan_check_host(const Layout& L) {
             const HalfMasks& hm = x ? hmb : hma;
             HalfWalk hw;
             for (hw.start(hm); !hw.done(pd.td[x].nsteps); hw.next(hm)) ++events;
-            if (n_s[x] != pd.td[x].nsteps || n_pv[x] != events || n_q[x] != 1) ++bad;
+            if (n_s[x] != events || n_pv[x] != events || n_q[x] != 1) ++bad;
         }
         delete[] rel_k;
         delete[] rel_v;
