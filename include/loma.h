@@ -270,20 +270,6 @@ LOMA_API int loma_masked_attn_plan_coverage(int n_chunks, int c, int t, int tail
                                             uint8_t* counts);
 
 /* ---------------------------------------------------------------------------
- * loma_masked_attn_pair_plan_check -- host-only check of how the tensor-core kernel
- * of loma_masked_attn_fwd (Eq. 1-3, Eq. 5-7) schedules its work.  The kernel takes two
- * neighbouring query tiles at a time, loads the union of their key tiles once, in one
- * merged order, through a two-stage ring, and issues the two tiles' tensor-core
- * instructions interleaved.  This routine replays, for every pair of the plan, the
- * merged order and the order of issue, and returns the number of violations of the
- * properties the kernel relies on (a step sequence that is not monotone, a shared step
- * whose two key tiles differ, an instruction whose K/V stage could not have been loaded
- * from instructions issued before it, a stage released twice or never).  0 = sound.
- * No CUDA call is made.  Negative return: INVALID_ARG (bad geometry).
- * ------------------------------------------------------------------------- */
-LOMA_API int loma_masked_attn_pair_plan_check(int n_chunks, int c, int t, int tail_read, unsigned flags);
-
-/* ---------------------------------------------------------------------------
  * loma_masked_attn_bwd_plan_coverage -- the same host-only replay for the pass of
  * loma_masked_attn_bwd that produces dK and dV.  That pass owns one 128-row key tile at a
  * time and walks the query tiles that may attend to it (the columns of Eq. 2 read

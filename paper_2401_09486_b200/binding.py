@@ -40,7 +40,6 @@ SIGNATURES = {
     "loma_rope_apply": (_i, [_p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i, _f, _i, _u, _p]),
     "loma_masked_attn_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
     "loma_masked_attn_bwd_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
-    "loma_masked_attn_pair_plan_check": (_i, [_i, _i, _i, _i, _u]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "loma_decode_attn_paged": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p, _sz, _p]),
@@ -211,15 +210,6 @@ def loma_masked_attn_plan_coverage(n_chunks: int, c: int, t: int, tail_read: int
     rc = lib().loma_masked_attn_plan_coverage(n_chunks, c, t, tail_read, int(flags), _ptr(counts))
     _check(rc, "loma_masked_attn_plan_coverage")
     return counts
-
-
-def loma_masked_attn_pair_plan_check(n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0) -> int:
-    """Host replay of the forward kernel's pair schedule (merged key-tile order, order of issue against
-    the two-stage ring): number of violations, 0 = sound."""
-    rc = lib().loma_masked_attn_pair_plan_check(n_chunks, c, t, tail_read, int(flags))
-    if rc < 0:
-        _check(rc, "loma_masked_attn_pair_plan_check")
-    return rc
 
 
 def loma_masked_attn_bwd_plan_coverage(n_chunks: int, c: int, t: int, tail_read: int = 0, flags: int = 0) -> torch.Tensor:

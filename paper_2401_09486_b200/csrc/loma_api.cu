@@ -288,13 +288,6 @@ int loma_masked_attn_plan_coverage(int n_chunks, int c, int t, int tail_read, un
     return LOMA_OK;
 }
 
-int loma_masked_attn_pair_plan_check(int n_chunks, int c, int t, int tail_read, unsigned flags) {
-    Layout L;
-    const int rc = make_layout(n_chunks, c, t, tail_read, flags, &L);
-    if (rc != LOMA_OK) return rc;
-    return L.S > 0 ? pair_plan_check_host(L) : 0;
-}
-
 int loma_masked_attn_bwd_plan_coverage(int n_chunks, int c, int t, int tail_read, unsigned flags, uint8_t* counts) {
     Layout L;
     const int rc = make_layout(n_chunks, c, t, tail_read, flags, &L);

@@ -100,7 +100,6 @@ cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, v
                                   const Layout& L, int64_t sb, int64_t sh, int64_t ss, float scale, cudaStream_t st);
 
 void plan_coverage_host(const Layout& L, uint8_t* counts);          // tile_plan_host.cu
-int pair_plan_check_host(const Layout& L);                          // violations of the forward's pair plan (0 = sound)
 void plan_coverage_by_key_host(const Layout& L, uint8_t* counts);   // the plan read by key tile (backward)
 
 cudaError_t launch_bounded_wait_selftest(cudaStream_t st);   // attn_tcgen05.cu

@@ -57,14 +57,13 @@ struct FwdParams {
     View view[4];
     int n_chunks, s, S, H, BH;
     int total_tiles;
-    int total_pairs;    // pairs of query tiles (the forward's unit of work), see decode_pair
     int n_tail, n_read, n_mem, n_rep;   // tiles per view, in scheduling order
     unsigned flags;
     FastDiv dBH, dH;
     float scale_log2;
     float* lse;
     int* status;
-    unsigned* sched;   // [0] next pair to hand out, [1] CTAs that have finished (the last one clears both); NULL = static deal
+    unsigned* sched;   // [0] next tile to hand out, [1] CTAs that have finished (the last one clears both); NULL = static deal
 };
 
 
@@ -87,8 +86,12 @@ __host__ __device__ __forceinline__ int tiles_covering(const View& v, int nchunk
     return v.Z >= 128 ? nchunks * v.tpc : fdiv(nchunks + v.CH - 1, v.dCH);
 }
 
-// Tile qi of a view: its geometry and the key tiles it visits (two runs of consecutive tiles).
-__host__ __device__ __forceinline__ void decode_tile_at(const FwdParams& p, int view, int qi, TileDesc& td) {
+__host__ __device__ __forceinline__ void decode_tile(const FwdParams& p, int rank, TileDesc& td) {
+    int view, qi;
+    if (rank < p.n_tail) { view = V_TAIL; qi = p.n_tail - 1 - rank; }
+    else if ((rank -= p.n_tail) < p.n_read) { view = V_READ; qi = p.n_read - 1 - rank; }
+    else if ((rank -= p.n_read) < p.n_mem) { view = V_MEM; qi = p.n_mem - 1 - rank; }
+    else { view = V_REP; qi = rank - p.n_mem; }
     const View& g = p.view[view];
     td.view = view; td.qi = qi;
     int c1;
@@ -116,16 +119,6 @@ __host__ __device__ __forceinline__ void decode_tile_at(const FwdParams& p, int 
         td.seg[1] = Seg{V_REP, M_DIAG, qi, 1};
     }
     td.nsteps = td.seg[0].count + td.seg[1].count;
-}
-
-// Tiles in scheduling order (longest first): tail, reading (last chunk first), memory, repetition.
-__host__ __device__ __forceinline__ void decode_tile(const FwdParams& p, int rank, TileDesc& td) {
-    int view, qi;
-    if (rank < p.n_tail) { view = V_TAIL; qi = p.n_tail - 1 - rank; }
-    else if ((rank -= p.n_tail) < p.n_read) { view = V_READ; qi = p.n_read - 1 - rank; }
-    else if ((rank -= p.n_read) < p.n_mem) { view = V_MEM; qi = p.n_mem - 1 - rank; }
-    else { view = V_REP; qi = rank - p.n_mem; }
-    decode_tile_at(p, view, qi, td);
 }
 
 __host__ __device__ __forceinline__ void step_ktile(const FwdParams& p, const TileDesc& td, int j, KTile& kt) {
@@ -210,182 +203,6 @@ struct HalfWalk {
     }
     __host__ __device__ __forceinline__ bool first_of_step(const HalfMasks&) const { return h == 0 || !(cur & 1u); }
     __host__ __device__ __forceinline__ bool last_of_step(const HalfMasks&) const { return h == 1 || !(cur & 2u); }
-};
-
-// ------------------------------------------------------------------ pairs of query tiles
-// The forward kernel gives a CTA two query tiles at a time -- tiles 2i and 2i + 1 of one view and one
-// (batch, head) -- and feeds both from ONE stream of key tiles: consecutive tiles of a view visit almost
-// the same keys (two reading tiles see the same earlier memory zones), so a key tile both of them visit
-// is loaded once.  Each tile keeps its own list of steps (decode_tile_at); the pair adds the order in which
-// the union of the two lists is loaded ("merged steps").  Per run of a tile's list (seg[0], seg[1]):
-//   * both runs start at the same key tile  -> merged run = the longer one; step k of either tile is merged
-//     step k (the tiles share every step both have);
-//   * otherwise                             -> the two runs are interleaved (A0 B0 A1 B1 ... then the rest
-//     of the longer one) and no step is shared (a key tile both happen to visit is then loaded twice).
-// A tile's steps keep their order in the merged list, which is all the kernel's roles rely on.
-struct PairMap {
-    int ca0, ca1, cb0, cb1;   // steps of tile A / B in run 0 / 1 (0 for an absent tile)
-    int same0, same1;         // run l starts at the same key tile for both tiles
-    int mc0;                  // merged steps of run 0
-    int nmerged;              // merged steps of the pair
-    // (scalar fields and selects instead of arrays: the kernel's roles keep this in registers)
-    __host__ __device__ __forceinline__ int cnt(int x, int l) const { return x ? (l ? cb1 : cb0) : (l ? ca1 : ca0); }
-    __host__ __device__ __forceinline__ int same(int l) const { return l ? same1 : same0; }
-};
-struct PairDesc {
-    TileDesc td[2];
-    int nb;          // 1 if tile B exists
-    PairMap pm;
-};
-
-__host__ __device__ __forceinline__ void make_pair_map(const TileDesc& a, const TileDesc& b, int nb, PairMap& pm) {
-    pm.ca0 = a.seg[0].count; pm.ca1 = a.seg[1].count;
-    pm.cb0 = nb ? b.seg[0].count : 0; pm.cb1 = nb ? b.seg[1].count : 0;
-    pm.same0 = nb && pm.ca0 > 0 && pm.cb0 > 0 && a.seg[0].view == b.seg[0].view && a.seg[0].first == b.seg[0].first;
-    pm.same1 = nb && pm.ca1 > 0 && pm.cb1 > 0 && a.seg[1].view == b.seg[1].view && a.seg[1].first == b.seg[1].first;
-    pm.mc0 = pm.same0 ? plan_max(pm.ca0, pm.cb0) : pm.ca0 + pm.cb0;
-    pm.nmerged = pm.mc0 + (pm.same1 ? plan_max(pm.ca1, pm.cb1) : pm.ca1 + pm.cb1);
-}
-
-// Pairs in scheduling order (longest first), the order of decode_tile taken two tiles at a time.
-__host__ __device__ __forceinline__ int pairs_of(int ntiles) { return (ntiles + 1) >> 1; }
-__host__ __device__ __forceinline__ void pair_tiles(const FwdParams& p, int rank, int& view, int& qa, int& nb) {
-    int pi, nt;
-    const int pt = pairs_of(p.n_tail), pr = pairs_of(p.n_read), pmm = pairs_of(p.n_mem);
-    if (rank < pt) { view = V_TAIL; nt = p.n_tail; pi = pt - 1 - rank; }
-    else if ((rank -= pt) < pr) { view = V_READ; nt = p.n_read; pi = pr - 1 - rank; }
-    else if ((rank -= pr) < pmm) { view = V_MEM; nt = p.n_mem; pi = pmm - 1 - rank; }
-    else { view = V_REP; nt = p.n_rep; pi = rank - pmm; }
-    qa = 2 * pi;
-    nb = (qa + 1 < nt) ? 1 : 0;
-}
-__host__ __device__ __forceinline__ void decode_pair(const FwdParams& p, int rank, PairDesc& pd) {
-    int view, qa;
-    pair_tiles(p, rank, view, qa, pd.nb);
-    decode_tile_at(p, view, qa, pd.td[0]);
-    if (pd.nb) decode_tile_at(p, view, qa + 1, pd.td[1]);
-    else pd.td[1] = pd.td[0];
-    make_pair_map(pd.td[0], pd.td[1], pd.nb, pd.pm);
-}
-
-// Merged index of step j of tile x.
-__host__ __device__ __forceinline__ int merged_index(const PairMap& pm, int x, int j) {
-    const int c0 = pm.cnt(x, 0);
-    const int l = j >= c0 ? 1 : 0;
-    const int k = l ? j - c0 : j;
-    const int base = l ? pm.mc0 : 0;
-    if (pm.same(l)) return base + k;
-    const int mn = plan_min(pm.cnt(0, l), pm.cnt(1, l));
-    return base + (k < mn ? 2 * k + x : mn + k);
-}
-// Merged step m -> the tile whose list names its key tile (A where both do) and that tile's step.
-__host__ __device__ __forceinline__ void merged_source(const PairMap& pm, int m, int& x, int& j) {
-    const int l = m >= pm.mc0 ? 1 : 0;
-    const int k = l ? m - pm.mc0 : m;
-    const int ca = pm.cnt(0, l), cb = pm.cnt(1, l);
-    int kk;
-    if (pm.same(l)) { x = k < ca ? 0 : 1; kk = k; }
-    else {
-        const int mn = plan_min(ca, cb);
-        if (k < 2 * mn) { x = k & 1; kk = k >> 1; }
-        else { x = ca > cb ? 0 : 1; kk = k - mn; }
-    }
-    j = kk + (l ? pm.cnt(x, 0) : 0);
-}
-// Does tile x visit merged step m?
-__host__ __device__ __forceinline__ bool visits_merged(const PairMap& pm, int x, int m) {
-    const int l = m >= pm.mc0 ? 1 : 0;
-    const int k = l ? m - pm.mc0 : m;
-    const int ca = pm.cnt(0, l), cb = pm.cnt(1, l);
-    if (pm.same(l)) return k < (x ? cb : ca);
-    const int mn = plan_min(ca, cb);
-    if (k < 2 * mn) return (k & 1) == x;
-    return (ca > cb ? 0 : 1) == x;
-}
-
-// The tensor-core instructions of one tile of a pair, in the order its issuing warp gives them.  The unit is
-// one visited half of a key tile (an "event": 64 keys): S_e = Q K_h^T into one of two score buffers, and
-// O += P_e V_h once the warpgroup has turned the scores into probabilities.  The score products run two
-// events ahead of the P.V products (S0 S1 PV0 S2 PV1 S3 ... PV PV), so the tensor pipe fills one score
-// buffer while the warpgroup works on the other.  Each tile of a pair has its own issuing warp; the two
-// meet only at the K/V rings: a stage is refilled after TWO releases, one per tile that visits the step;
-// for a step only one tile visits, the loader gives the second one itself right after the load (it knows
-// the visitors).  The host replays both walks against the rings (pair_plan_check) and verifies that
-// neither they nor the loads can block for ever.
-struct IssueAct {
-    int is_s;            // score product (1) or P.V product (0)
-    int m;               // merged step
-    int h;               // half of the key tile
-    int first_of_step;   // first visited half of its step: S needs the K tile here, P.V the V tile
-    int last_of_step;    // last visited half of its step: afterwards this tile is done with the K (S) / V (P.V) stage
-    int first_event;     // first of the tile: S waits for the Q tile, P.V overwrites the accumulator
-    int last_s;          // S: the tile's last score product (its Q buffer is free afterwards)
-};
-// Kept small on purpose: the issuing warp runs this between two batches of tensor-core instructions, and
-// whatever it costs is added to the time the other roles wait for the next batch.  The visited-half masks
-// are kept shifted (bit 0 = the cursor's step, ones shifted in from the top: steps past 63 visit both
-// halves), the merged index is recomputed only when a cursor enters a new step.
-struct TileIssue {
-    unsigned long long sm0, sm1, pm0, pm1;   // shifted masks of the S cursor / the P.V cursor
-    int sj, sh, pj, ph;                      // step and half of the two cursors
-    int s_m, p_m;                            // merged index of the cursors' steps
-    int ns, np;                              // events whose S / whose P.V has been issued
-    int nsteps;
-    int x, c0, mc0, same0, same1, mn0, mn1;  // what merged_index needs, unpacked for tile x
-    __host__ __device__ __forceinline__ int midx(int j) const {
-        const int l = j >= c0 ? 1 : 0;
-        const int k = l ? j - c0 : j;
-        const int mn = l ? mn1 : mn0;
-        return (l ? mc0 : 0) + ((l ? same1 : same0) ? k : (k < mn ? 2 * k + x : mn + k));
-    }
-    __host__ __device__ __forceinline__ void start(const PairMap& pm, int x_, const HalfMasks& hm, int nsteps_) {
-        x = x_; nsteps = nsteps_;
-        c0 = pm.cnt(x, 0); mc0 = pm.mc0; same0 = pm.same0; same1 = pm.same1;
-        mn0 = plan_min(pm.ca0, pm.cb0); mn1 = plan_min(pm.ca1, pm.cb1);
-        sm0 = pm0 = hm.m[0]; sm1 = pm1 = hm.m[1];
-        sj = pj = 0; ns = np = 0;
-        sh = ph = (hm.m[0] & 1ull) ? 0 : 1;
-        s_m = p_m = midx(0);
-    }
-    __host__ __device__ __forceinline__ bool done() const { return pj >= nsteps; }
-    // the next instruction of the tile; call only while !done()
-    __host__ __device__ __forceinline__ void next(IssueAct& act) {
-        const bool is_s = sj < nsteps && ns < np + 2;
-        act.is_s = is_s;
-        if (is_s) {
-            const unsigned cur = (unsigned)(sm0 & 1ull) | ((unsigned)(sm1 & 1ull) << 1);
-            const bool los = sh == 1 || !(cur & 2u);
-            act.m = s_m; act.h = sh;
-            act.first_of_step = sh == 0 || !(cur & 1u);
-            act.last_of_step = los;
-            act.first_event = ns == 0;
-            act.last_s = los && sj == nsteps - 1;
-            ++ns;
-            if (!los) { sh = 1; }
-            else {
-                ++sj;
-                sm0 = (sm0 >> 1) | (1ull << 63); sm1 = (sm1 >> 1) | (1ull << 63);
-                sh = (sm0 & 1ull) ? 0 : 1;
-                s_m = midx(sj);
-            }
-        } else {
-            const unsigned cur = (unsigned)(pm0 & 1ull) | ((unsigned)(pm1 & 1ull) << 1);
-            const bool los = ph == 1 || !(cur & 2u);
-            act.m = p_m; act.h = ph;
-            act.first_of_step = ph == 0 || !(cur & 1u);
-            act.last_of_step = los;
-            act.first_event = np == 0;
-            act.last_s = 0;
-            ++np;
-            if (!los) { ph = 1; }
-            else {
-                ++pj;
-                pm0 = (pm0 >> 1) | (1ull << 63); pm1 = (pm1 >> 1) | (1ull << 63);
-                ph = (pm0 & 1ull) ? 0 : 1;
-                p_m = midx(pj);
-            }
-        }
-    }
 };
 
 // ------------------------------------------------------------------ the plan read by key tile
@@ -536,7 +353,6 @@ inline void make_plan(const Layout& L, int B, int H, FwdParams* p) {
     p->n_tail = p->view[V_TAIL].ntiles; p->n_read = p->view[V_READ].ntiles;
     p->n_mem = p->view[V_MEM].ntiles; p->n_rep = p->view[V_REP].ntiles;
     p->total_tiles = p->n_tail + p->n_read + p->n_mem + p->n_rep;
-    p->total_pairs = (p->n_tail + 1) / 2 + (p->n_read + 1) / 2 + (p->n_mem + 1) / 2 + (p->n_rep + 1) / 2;
     p->flags = L.flags;
     p->dBH = make_fastdiv(p->BH); p->dH = make_fastdiv(H);
 }
