@@ -14,6 +14,16 @@ One step = one pass of the whole hot path over one batch of synthetic input:
 decode GB/s (the other half of the metric) is in `decode_attn`, and the
 roofline object describes the decode kernel, which dominates the step's time.
 
+At N=1 a second loop with the same --steps/--warmup times the two largest
+workloads as steps of their own: the 69632-token forward (B1 H32 D128, c=8,
+t=32, 128 chunks: the tensor-bound case) and one generation cycle at the
+higher ratio (B64 H32 D128, 16384 memory entries, c=8, t=16: 128 decodes +
+1 compress), reported in `large_workloads` with a roofline object per kernel.
+
+  python bench.py --profile-case NAME [--reps N]   runs a cut-down launch of one
+kernel (same per-(batch, head) shapes, fewer pairs; inputs larger than L2, a few GB
+at most) and exits (what a profiler capture wraps).
+
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
 With --gpus N > 1 (launched under torch.distributed.run, one rank per GPU) every
@@ -339,24 +349,23 @@ def run_ours(args):
         "masked_attn": {"useful_tflops": fwd_tflops, "ms": t_fwd, "useful_flops": fwd_flops,
                         "compulsory_bytes": fwd_bytes, "gbs": fwd_bytes / (t_fwd * 1e-3) / 1e9,
                         "frac_of_measured_hbm": fwd_bytes / (t_fwd * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                        "frac_of_measured_bf16": fwd_tflops / world / peaks["bf16_tflops"]},
+                        "frac_of_measured_bf16": fwd_tflops / world / peaks["bf16_tflops"],
+                        "ms_x_sm_ghz": (t_fwd * clocks["sm_mhz"] / 1e3) if clocks.get("sm_mhz") else None},
         "compress": {"ms": t_cmp, "bytes": cmp_bytes, "gbs": cmp_gbs,
                      "frac_of_measured_hbm": cmp_gbs / peaks["hbm_gbs"],
                      "note": "timed in place after the 64 decodes of the cycle"},
         "roofline": {"kernel": "decode_splitkv_kernel<128> (+ merge), per loma_decode_attn call", "bound": "hbm",
                      "achieved": dec_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": dec_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                     # dram__bytes_read + write of one launch: captured on the B8 case (1.084e9 bytes for 1.0779e9
-                     # algorithmic, profiles/decode_splitkv_B8_H32_L8224.md) and scaled by the (b,h) count, 1024 / 256
-                     "traffic": 1.084e9 * (g["B"] * g["H"]) / 256.0,
+                     # dram__bytes_read + write of one launch: captured on the B8 case and scaled by the (b,h) count, 1024 / 256
+                     "traffic": DECODE_TRAFFIC_B8_L8224 * (g["B"] * g["H"]) / 256.0,
                      "traffic_source": "ncu small case x4"},
         "roofline_other_kernels": [
             {"kernel": "masked_attn_tc_kernel<128>", "workload": "4608-token layout", "bound": "hbm",
              "achieved": fwd_bytes / (t_fwd * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
              "frac": fwd_bytes / (t_fwd * 1e-3) / 1e9 / peaks["hbm_gbs"],
-             # dram__bytes_read.sum + dram__bytes_write.sum of one launch on one batch element of this layout
-             # (profiles/masked_attn_tc_small_cases.md) x B
-             "traffic": 142.2e6 * f["B"],
+             # dram__bytes_read.sum + dram__bytes_write.sum of one launch on one batch element of this layout x B
+             "traffic": FWD_SHORT_TRAFFIC_B1 * f["B"],
              "tensor_frac_of_measured_bf16_useful": fwd_tflops / world / peaks["bf16_tflops"]},
             {"kernel": "compress_mma_kernel<128>", "workload": "B32 H32 mem 8192, default variant", "bound": "hbm",
              "achieved": cmp_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": cmp_gbs / peaks["hbm_gbs"],
@@ -370,7 +379,14 @@ def run_ours(args):
         "clocks": clocks,
     }
     if world == 1 and not args.no_extras:
-        # the two other named workloads, timed once each (context, not the metric)
+        # free the step's tensors, then the two largest workloads as steps of their own (same --steps / --warmup)
+        del q, k, v, o, kc, vc, dq, dk, dv, do, hq, hk, hv, ho, hdq, hdk, hdv, hdo
+        torch.cuda.empty_cache()
+        out["large_workloads"] = large_workloads(L, synthetic, torch, dev, peaks, args.steps, max(args.warmup, 3),
+                                                 clocks.get("sm_mhz"))
+        out["roofline_large"] = [out["large_workloads"]["masked_fwd_69632"]["roofline"],
+                                 out["large_workloads"]["generation_B64_16k"]["roofline"]]
+        # further shapes, timed a few times each (context, not the metric)
         out["other_workloads"] = other_workloads(L, synthetic, torch, dev, peaks)
     if rank == 0:
         out["cpu_baseline"] = cpu_baseline()
@@ -509,6 +525,171 @@ def other_workloads(L, synthetic, torch, dev, peaks):
     return res
 
 
+def large_workloads(L, synthetic, torch, dev, peaks, steps, warmup, clocks_mhz):
+    """The two largest single-GPU workloads, each as a step of its own, `steps` timed repetitions after
+    `warmup`: the 69632-token training-layout forward and one generation cycle at the higher ratio
+    (128 decodes with the tail growing 0..127, then one compress).  CUDA events on the launching stream."""
+    bf = torch.bfloat16
+    stream = torch.cuda.current_stream()
+    D = 128
+    std = 1.0 / math.sqrt(D)
+    ghz = (clocks_mhz or 0.0) / 1e3
+    out = {}
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    # ---- forward on the long layout
+    B, H, n, c, t = 1, 32, 128, 8, 32
+    S = n * (2 * c * t + t)
+    q, k, v = (synthetic.big_normal_(torch.empty(B, H, S, D, dtype=bf, device=dev), 3000 + i, std) for i in range(3))
+    o = torch.empty_like(q)
+    for _ in range(warmup):
+        L.loma_masked_attn_fwd(q, k, v, o, None, n, c, t, 0, 0, 0.0, stream)
+    torch.cuda.synchronize()
+    marks = []
+    for _ in range(steps):
+        _device_pause(torch, 300_000)
+        a, b = ev(), ev()
+        a.record(stream)
+        L.loma_masked_attn_fwd(q, k, v, o, None, n, c, t, 0, 0, 0.0, stream)
+        b.record(stream)
+        marks.append((a, b))
+    torch.cuda.synchronize()
+    ts = [a.elapsed_time(b) for a, b in marks]
+    ms = sum(ts) / len(ts)
+    flops = 4.0 * D * allowed_pairs(n, c, t) * B * H
+    nbytes = 4.0 * q.numel() * 2
+    tf = flops / (ms * 1e-3) / 1e12
+    out["masked_fwd_69632"] = {
+        "config": dict(B=B, H=H, D=D, n=n, c=c, t=t, S=S), "steps": steps, "ms": ms, "ms_min": min(ts),
+        "ms_x_sm_ghz": ms * ghz if ghz else None, "useful_tflops": tf, "useful_flops": flops, "compulsory_bytes": nbytes,
+        "roofline": {"kernel": "masked_attn_tc_kernel<128>", "bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"],
+                     "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst bf16)",
+                     "frac_of_sustained": tf / peaks["bf16_tflops_sustained"],
+                     # dram bytes of one launch on the 8-head case of this layout (ncu), times 4 for 32 heads
+                     "traffic": FWD_LONG_TRAFFIC_8_HEADS * (H / 8.0) if FWD_LONG_TRAFFIC_8_HEADS else None,
+                     "traffic_source": "ncu 8-head case x4"}}
+    del q, k, v, o
+    torch.cuda.empty_cache()
+
+    # ---- generation cycle at the higher ratio
+    B, H, c, t, mem_len = 64, 32, 8, 16, 16384
+    tc = c * t
+    cap = mem_len + tc + t
+    kc = synthetic.big_normal_(torch.empty(B, H, cap, D, dtype=bf, device=dev), 3100, std)
+    vc = synthetic.big_normal_(torch.empty(B, H, cap, D, dtype=bf, device=dev), 3101, std)
+    dq, dk, dv = (synthetic.big_normal_(torch.empty(tc, B, H, 1, D, dtype=bf, device=dev), 3102 + i, std) for i in range(3))
+    do = torch.empty_like(dq)
+    qm, km, vm = (synthetic.big_normal_(torch.empty(B, H, t, D, dtype=bf, device=dev), 3110 + i, std) for i in range(3))
+    om = torch.empty_like(qm)
+    ws = torch.empty(max(16, L.loma_decode_workspace_bytes(B, H, D, cap), L.loma_compress_workspace_bytes(B, H, D, t, mem_len, 0)),
+                     dtype=torch.uint8, device=dev)
+
+    def cycle(marks=None):
+        e0 = ev(); e0.record(stream)
+        for j in range(tc):
+            L.loma_decode_attn(dq[j], dk[j], dv[j], kc, vc, do[j], None, mem_len + j, ws, 0, 0.0, stream)
+        e1 = ev(); e1.record(stream)
+        L.loma_compress_step(qm, km, vm, kc, vc, om, None, mem_len, c, t, ws, 0, 0.0, stream)
+        e2 = ev(); e2.record(stream)
+        if marks is not None:
+            marks.append((e0, e1, e2))
+
+    for _ in range(max(1, min(warmup, 3))):
+        cycle()
+    torch.cuda.synchronize()
+    marks = []
+    for _ in range(steps):
+        cycle(marks)
+    torch.cuda.synchronize()
+    t_dec = sum(a.elapsed_time(b) for a, b, _ in marks) / steps
+    t_cmp = sum(b.elapsed_time(c2) for _, b, c2 in marks) / steps
+    dec_rows = sum(mem_len + j + 1 for j in range(tc))
+    dec_bytes_call = 2.0 * dec_rows * B * H * D * 2 / tc
+    dec_ms_call = t_dec / tc
+    dec_gbs = dec_bytes_call / (dec_ms_call * 1e-3) / 1e9
+    cmp_bytes = float(B * H) * D * 2 * (2 * tc + 6 * t)
+    cmp_gbs = cmp_bytes / (t_cmp * 1e-3) / 1e9
+    out["generation_B64_16k"] = {
+        "config": dict(B=B, H=H, D=D, c=c, t=t, mem_len=mem_len, cap=cap, decode_steps=tc), "steps": steps,
+        "cycle_ms": t_dec + t_cmp, "decode_ms_per_call": dec_ms_call, "decode_ms_x_sm_ghz": dec_ms_call * ghz if ghz else None,
+        "decode_gbs": dec_gbs, "decode_bytes_per_call": dec_bytes_call, "compress_ms": t_cmp, "compress_gbs": cmp_gbs,
+        "roofline": {"kernel": "decode_splitkv_kernel<128> (+ merge), per loma_decode_attn call", "bound": "hbm", "achieved": dec_gbs,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"], "frac_of_8tbs": dec_gbs / 8000.0,
+                     "peak_source": peaks["source"],
+                     # every (b, h) streams its own rows once: the B8 / 8224-row capture scaled by rows and (b, h) pairs
+                     "traffic": DECODE_TRAFFIC_B8_L8224 * (B * H / 256.0) * ((mem_len + tc / 2.0 + 0.5) / 8224.0),
+                     "traffic_source": "ncu small case scaled by (b,h) pairs and rows"},
+        "roofline_compress": {"kernel": "compress_mma_kernel<128>", "bound": "hbm", "achieved": cmp_gbs, "peak": peaks["hbm_gbs"],
+                              "unit": "GB/s", "frac": cmp_gbs / peaks["hbm_gbs"], "traffic": None,
+                              "note": "0.19 GB in one launch right after the decodes of the cycle"}}
+    return out
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch, from ncu captures of the --profile-case launches
+DECODE_TRAFFIC_B8_L8224 = 1.084e9      # decode_splitkv + merge, B8 H32, 8224 rows (1.0779e9 algorithmic)
+FWD_SHORT_TRAFFIC_B1 = 151.1e6         # masked_attn_tc, one batch element of the 4608-token layout
+FWD_LONG_TRAFFIC_8_HEADS = None        # masked_attn_tc, 8 heads of the 69632-token layout: no capture of the current kernel
+
+
+def profile_case(args):
+    """One cut-down launch sequence of a single kernel, for profiler captures."""
+    import torch
+
+    from paper_2401_09486_b200 import binding as L
+    from paper_2401_09486_b200 import build, synthetic
+
+    build.build_library()
+    torch.cuda.set_device(0)
+    dev = "cuda:0"
+    bf = torch.bfloat16
+    D = 128
+    std = 1.0 / math.sqrt(D)
+    case = args.profile_case
+    if case in ("decode", "compress", "compress_prior"):
+        B, H, c, t, mem_len = 8, 32, 4, 16, 8192          # 1/4 of the generation workload's batch: 1.08 GB of cache
+        tc = c * t
+        cap = mem_len + tc + t
+        kc = synthetic.big_normal_(torch.empty(B, H, cap, D, dtype=bf, device=dev), 1, std)
+        vc = synthetic.big_normal_(torch.empty(B, H, cap, D, dtype=bf, device=dev), 2, std)
+        flags = L.LOMA_FLAG_MEM_SEES_PRIOR_MEM if case == "compress_prior" else 0
+        ws = torch.empty(max(16, L.loma_decode_workspace_bytes(B, H, D, cap),
+                             L.loma_compress_workspace_bytes(B, H, D, t, mem_len, flags)), dtype=torch.uint8, device=dev)
+        if case == "decode":
+            q, kn, vn = (x.to(dev) for x in synthetic.qkv(B, H, 1, D, 3, std, bf))
+            o = torch.empty_like(q)
+            for r in range(args.reps):
+                L.loma_decode_attn(q, kn, vn, kc, vc, o, None, mem_len + 31 + r, ws)
+        else:
+            qm, km, vm = (x.to(dev) for x in synthetic.qkv(B, H, t, D, 4, std, bf))
+            om = torch.empty_like(qm)
+            for r in range(args.reps):
+                L.loma_compress_step(qm, km, vm, kc, vc, om, None, mem_len, c, t, ws, flags)
+    else:
+        if case in ("masked", "bwd"):
+            B, H, n, c, t = 1, 32, 32, 4, 16               # one batch element of the 4608-token layout: 151 MB per tensor
+        else:
+            B, H, n, c, t = 1, 8, 128, 8, 32               # 8 heads of the 69632-token layout: 143 MB per tensor
+        S = n * (2 * c * t + t)
+        q, k, v = (synthetic.big_normal_(torch.empty(B, H, S, D, dtype=bf, device=dev), 10 + i, std) for i in range(3))
+        o = torch.empty_like(q)
+        if case.startswith("bwd"):
+            lse = torch.empty((B, H, S), dtype=torch.float32, device=dev)
+            L.loma_masked_attn_fwd(q, k, v, o, lse, n, c, t)
+            d_o = synthetic.big_normal_(torch.empty_like(q), 20, std)
+            dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+            ws = torch.empty(L.loma_masked_attn_bwd_workspace_bytes(B, H, D, n, c, t), dtype=torch.uint8, device=dev)
+            for r in range(args.reps):
+                L.loma_masked_attn_bwd(q, k, v, o, d_o, lse, dq, dk, dv, n, c, t, 0, 0, ws)
+        else:
+            for r in range(args.reps):
+                L.loma_masked_attn_fwd(q, k, v, o, None, n, c, t)
+    torch.cuda.synchronize()
+    assert L.loma_device_status() == 0
+    print("ok", case)
+
+
 # ------------------------------------------------------------------ oracle timing
 
 def _oracle_sample(n_heads_fwd: int, n_heads_dec: int, seed: int = 0):
@@ -592,9 +773,14 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--no-extras", action="store_true", help="skip the two extra workloads timed at N=1")
+    ap.add_argument("--no-extras", action="store_true", help="skip the large and the context workloads timed at N=1")
+    ap.add_argument("--profile-case", choices=["decode", "compress", "compress_prior", "masked", "masked_long", "bwd", "bwd_long"],
+                    help="run one cut-down kernel launch sequence (for profiler captures) and exit")
+    ap.add_argument("--reps", type=int, default=3, help="launches of --profile-case")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.profile_case:
+        profile_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

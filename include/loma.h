@@ -172,6 +172,15 @@ LOMA_API int loma_generation_index(int n_tokens, int c, int t,
  *   flags                  LOMA_FLAG_* bits
  * o must not alias q, k or v.  Rows are independent; every row has at least one
  * allowed key (itself), so no output is undefined.
+ * Concurrency: the bf16 kernel hands out its tiles from a counter inside the library.
+ * Calls on different streams each use their stream's own counter and may overlap freely
+ * (the first 192 streams that call get one; later ones run with a fixed deal of the
+ * tiles, slower by a few percent on short layouts).  A call recorded while its stream is
+ * being captured into a CUDA graph gets a counter of its own for good (320 per device,
+ * then the fixed deal), so replays may overlap eager calls and other graphs; two
+ * replays of the same captured call must not overlap each other (CUDA already orders
+ * launches of one executable graph).  Make one eager bf16 call per device before the
+ * first capture: the first call looks up device symbols and sets kernel attributes.
  * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT (pointers and byte strides must be
  * multiples of 16), CUDA.  S == 0 or B*H == 0 is a successful no-op.
  * ------------------------------------------------------------------------- */

@@ -127,6 +127,26 @@ def test_masked_fwd_strided_views_and_explicit_scale():
     check_close(o, want_o, torch.bfloat16)
 
 
+def test_same_tensors_with_and_without_repetition_zones_do_not_share_descriptors():
+    """Two bf16 calls on the same addresses with the same strides, B, H, D, n, c, t, once in the training
+    layout and once in the layout without repetition zones: the second call must not reuse the TMA
+    descriptors of the first (their chunk stride and zone views differ)."""
+    B, H, D, n, c, t = 2, 3, 128, 3, 4, 16
+    S_full = oracle.seq_len(n, c, t)
+    S_norep = oracle.seq_len(n, c, t, 0, NOREP)
+    buf = synthetic.normal_tensor((B, S_full, 4, H, D), 19, 1.0, torch.bfloat16).to(DEV)
+    q, k, v, o = (buf[:, :, i].permute(0, 2, 1, 3) for i in range(4))      # [B, H, S, D] strided views
+    for _ in range(2):                                                       # full, norep, full, norep
+        for flags, S in ((0, S_full), (NOREP, S_norep)):
+            qs, ks, vs, os_ = (x[:, :, :S] for x in (q, k, v, o))
+            assert qs.data_ptr() == q.data_ptr() and qs.stride() == q.stride()
+            want_o, _ = oracle.masked_attn_fwd(npf(qs), npf(ks), npf(vs), n, c, t, 0, flags)
+            os_.fill_(float("nan"))
+            L.loma_masked_attn_fwd(qs, ks, vs, os_, None, n, c, t, 0, flags, 0.0)
+            torch.cuda.synchronize()
+            check_close(os_, want_o, torch.bfloat16)
+
+
 # ----------------------------------------- inference layout (no repetition zones)
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
@@ -659,21 +679,38 @@ def test_generation_cycle_replays_from_a_cuda_graph():
 
 
 def test_forwards_on_two_streams_at_once_do_not_disturb_each_other():
-    """The forward hands out tiles from a counter; launches get their counters round robin, so two launches in
-    flight on different streams must each produce exactly what they produce alone."""
+    """The forward hands out tiles from a counter that belongs to the launch's stream (a captured launch gets
+    one of its own), so launches in flight on different streams -- many more than there were counters when
+    they were dealt round robin -- and a graph replay next to eager launches must each produce exactly what
+    they produce alone."""
     B, H, D, n, c, t = 2, 8, 128, 12, 4, 16
     S = oracle.seq_len(n, c, t)
     a = [x.to(DEV) for x in synthetic.qkv(B, H, S, D, seed=101, dtype=torch.bfloat16)]
     b = [x.to(DEV) for x in synthetic.qkv(B, H, S, D, seed=102, dtype=torch.bfloat16)]
     alone_a, _ = run_fwd(*a, n, c, t)
     alone_b, _ = run_fwd(*b, n, c, t)
-    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    s1, s2, s3 = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
     torch.cuda.synchronize()
-    oa = [torch.empty_like(a[0]) for _ in range(6)]
-    ob = [torch.empty_like(b[0]) for _ in range(6)]
-    for i in range(6):
-        L.loma_masked_attn_fwd(*a, oa[i], None, n, c, t, 0, 0, 0.0, s1)
-        L.loma_masked_attn_fwd(*b, ob[i], None, n, c, t, 0, 0, 0.0, s2)
+    # a captured forward (replayed below on a third stream while the eager ones run)
+    og = torch.empty_like(a[0])
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s3):
+        L.loma_masked_attn_fwd(*a, og, None, n, c, t, 0, 0, 0.0, s3)      # set-up call before the capture
+        s3.synchronize()
+        with torch.cuda.graph(graph, stream=s3):
+            L.loma_masked_attn_fwd(*a, og, None, n, c, t, 0, 0, 0.0, torch.cuda.current_stream())
+    og.fill_(float("nan"))
     torch.cuda.synchronize()
-    for i in range(6):
+    reps = 70                                        # > 64 launches outstanding per stream
+    oa = [torch.empty_like(a[0]) for _ in range(4)]
+    ob = [torch.empty_like(b[0]) for _ in range(4)]
+    for i in range(reps):
+        L.loma_masked_attn_fwd(*a, oa[i % 4], None, n, c, t, 0, 0, 0.0, s1)
+        L.loma_masked_attn_fwd(*b, ob[i % 4], None, n, c, t, 0, 0, 0.0, s2)
+        if i % 10 == 5:
+            with torch.cuda.stream(s3):
+                graph.replay()
+    torch.cuda.synchronize()
+    for i in range(4):
         assert torch.equal(oa[i], alone_a) and torch.equal(ob[i], alone_b)
+    assert torch.equal(og, alone_a)

@@ -7,7 +7,8 @@ stalls the whole device.  They cannot pass loma_decode_attn a workspace, so the
 library offers the same step with the split partials kept in an 8 MiB array
 inside the library itself.  This test calls that entry point through the C ABI
 twice in a row -- the second call finds the first call's partials still in the
-array -- and checks each result against loma_decode_attn on identical inputs.
+array -- and checks each result against loma_decode_attn on identical inputs
+(bit for bit: the two run the same kernels) and against the CPU oracle.
 It lives in its own file, collected last, and passes on its own in a fresh
 process as well as after the rest of the suite.
 """
@@ -16,6 +17,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2401_09486_b200 import binding as L
 from paper_2401_09486_b200 import build, synthetic
 
@@ -34,6 +36,7 @@ def _one_call(B, H, D, cap, cache_len, seed):
 
     # reference: the existing entry point with a caller-provided workspace
     kc_ref, vc_ref = kc.clone(), vc.clone()
+    want_o, want_lse, _, _ = oracle.decode_attn(_f64(q), _f64(kn), _f64(vn), _f64(kc), _f64(vc), cache_len)
     need = L.loma_decode_workspace_bytes(B, H, D, cache_len)
     assert need > 0, "pick a shape that really uses split partials"
     ws = torch.empty(need, dtype=torch.uint8, device=DEV)
@@ -53,6 +56,12 @@ def _one_call(B, H, D, cap, cache_len, seed):
     assert d.max() <= 2e-2 and d.mean() <= 2e-3          # the suite's bf16 tolerance
     assert np.abs(_f64(lse) - _f64(lse_ref)).max() <= 2e-2
     assert torch.equal(kc, kc_ref) and torch.equal(vc, vc_ref)   # same bit-exact append
+    # both entry points run the same two kernels with the same split of the key range, so they agree bit for bit
+    assert torch.equal(o, o_ref) and torch.equal(lse, lse_ref)
+    # and the new entry point on its own against the CPU oracle (Appendix A, inference_input with one token)
+    d = np.abs(_f64(o) - want_o)
+    assert d.max() <= 2e-2 and d.mean() <= 2e-3
+    assert np.abs(_f64(lse) - want_lse.reshape(_f64(lse).shape)).max() <= 2e-2
 
 
 def test_static_scratch_decode_matches_workspace_decode_twice_in_a_row():
