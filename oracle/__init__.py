@@ -35,6 +35,8 @@ from .loma_oracle import (  # noqa: F401
     rope_rotate,
     rope_apply,
     decode_attn,
+    prefill_attn,
+    replay_prompt_pieces,
     decode_attn_ragged,
     decode_attn_paged,
     paged_to_contiguous,

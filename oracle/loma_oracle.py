@@ -483,6 +483,85 @@ def decode_attn(q, k_new, v_new, k_cache, v_cache, cache_len, scale=None):
     return o, lse, kc, vc
 
 
+def prefill_attn(q, k_new, v_new, k_cache, v_cache, cache_len, scale=None):
+    """Several new tokens at once over an existing cache (Appendix A, `inference_input`).
+
+    The l new tokens see every one of the cache_len cached entries and, among
+    themselves, are causal: the mask is tril(ones(l, l + cache_len), diagonal=cache_len),
+    row i allowing columns 0 .. cache_len + i.  Their K/V are appended to the cache.
+
+    q, k_new, v_new: [B, H, l, D]; k_cache, v_cache: [B, H, cap, D] with the first
+    cache_len entries valid.  Returns (o [B,H,l,D], lse [B,H,l], k_cache', v_cache')
+    where the primed caches are copies with entries cache_len .. cache_len+l-1 filled in.
+    """
+    q = _f64(q)
+    B, H, l, D = q.shape
+    kc = np.array(k_cache, copy=True)
+    vc = np.array(v_cache, copy=True)
+    kc[:, :, cache_len:cache_len + l, :] = np.asarray(k_new)
+    vc[:, :, cache_len:cache_len + l, :] = np.asarray(v_new)
+    mask = np.tril(np.ones((l, l + cache_len), bool), k=cache_len)
+    o = np.zeros((B, H, l, D))
+    lse = np.zeros((B, H, l))
+    for b in range(B):
+        for h in range(H):
+            o[b, h], _, lse[b, h] = masked_softmax_attention(q[b, h], kc[b, h, :cache_len + l], vc[b, h, :cache_len + l],
+                                                            mask, scale)
+    return o, lse, kc, vc
+
+
+def replay_prompt_pieces(q, k, v, pieces, c, t, flags=0, scale=None):
+    """Feed a prompt to the generation path in arbitrary pieces, the way Appendix A's
+    `add_token_ids` does: tokens are buffered; whenever the uncompressed tail can be filled
+    up to tc entries, exactly that many tokens go through `inference_input` (one
+    prefill_attn call) and the chunk is compressed; what is left at the end of a piece goes
+    through `inference_input` as it is.
+
+    q, k, v: [B, H, S, D] in the inference layout (chunks of [tc reading | t memory], no
+    repetition zones, then a reading tail), so that row numbers of the one-shot forward
+    with FLAG_NO_REP_ZONE apply.  pieces: lengths of the token pieces; their sum is the
+    number of reading rows.  Returns (O [B,H,S,D], k_cache, v_cache, length).
+    """
+    q, k, v = np.asarray(q), np.asarray(k), np.asarray(v)
+    B, H, S, D = q.shape
+    tc = t * c
+    s = tc + t
+    n_tokens = int(sum(pieces))
+    n_chunks, tail = (n_tokens // tc, n_tokens % tc) if tc > 0 else (0, n_tokens)
+    assert S == n_chunks * s + tail
+    row_of_token = lambda g: (g // tc) * s + g % tc if tc > 0 else g
+    cap = n_chunks * t + max(tc, tail) + 1
+    kc = np.zeros((B, H, cap, D), dtype=k.dtype)
+    vc = np.zeros((B, H, cap, D), dtype=v.dtype)
+    O = np.full((B, H, S, D), np.nan)
+    length, done, chunks = 0, 0, 0          # cache entries, tokens processed, chunks compressed
+    fed = 0
+    for piece in pieces:
+        fed += int(piece)
+        while done < fed:
+            uncompressed = length - chunks * t
+            take = fed - done
+            fills = tc > 0 and uncompressed + take >= tc
+            if fills:
+                take = tc - uncompressed
+            rows = [row_of_token(g) for g in range(done, done + take)]
+            out, _, kc, vc = prefill_attn(q[:, :, rows], k[:, :, rows], v[:, :, rows], kc, vc, length, scale)
+            O[:, :, rows] = out
+            length += take
+            done += take
+            if fills:
+                m0 = chunks * s + tc
+                mem_len = chunks * t
+                out, _, nk, nv = compress_step(q[:, :, m0:m0 + t], k[:, :, m0:m0 + t], v[:, :, m0:m0 + t],
+                                               kc, vc, mem_len, c, t, flags & FLAG_MEM_SEES_PRIOR_MEM, scale)
+                O[:, :, m0:m0 + t] = out
+                chunks += 1
+                length = mem_len + t
+                kc[:, :, :length] = nk
+                vc[:, :, :length] = nv
+    return O, kc, vc, length
+
+
 def decode_attn_ragged(q, k_new, v_new, k_cache, v_cache, cache_lens, scale=None):
     """decode_attn for a batch whose sequences have their own cache lengths: sequence b is an
     independent run of the generator (Appendix A handles one sequence at a time), so this is

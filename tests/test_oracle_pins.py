@@ -498,6 +498,115 @@ def test_inference_layout_equals_training_layout_on_shared_rows_and_replays(n, c
     assert pos2.tolist() == oracle.layout_index(n, c, t, tail)[4][live].tolist()
 
 
+# ------------------------------------------- several tokens over an existing cache
+
+def test_prefill_with_one_token_is_decode():
+    B, H, L, D = 2, 3, 9, 8
+    q, k, v = (_rand((B, H, 1, D), sd) for sd in (300, 301, 302))
+    kc, vc = _rand((B, H, L + 3, D), 303), _rand((B, H, L + 3, D), 304)
+    a = oracle.prefill_attn(q, k, v, kc, vc, L)
+    b = oracle.decode_attn(q, k, v, kc, vc, L)
+    assert np.allclose(a[0], b[0], atol=1e-14) and np.allclose(a[1], b[1], atol=1e-14)
+    assert np.array_equal(a[2], b[2]) and np.array_equal(a[3], b[3])
+
+
+@pytest.mark.parametrize("l", [1, 2, 7, 33])
+def test_prefill_over_an_empty_cache_is_library_causal_sdpa(l):
+    B, H, D = 2, 2, 16
+    q, k, v = (_rand((B, H, l, D), sd) for sd in (310, 311, 312))
+    kc = np.full((B, H, l + 2, D), 7.0); vc = np.full((B, H, l + 2, D), -7.0)      # stale contents must not matter
+    o, lse, kc2, vc2 = oracle.prefill_attn(q, k, v, kc, vc, 0)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q), torch.from_numpy(k), torch.from_numpy(v), is_causal=True).numpy()
+    assert np.allclose(o, ref, atol=1e-13)
+    assert np.array_equal(kc2[:, :, :l], k) and np.array_equal(vc2[:, :, :l], v)
+    assert np.array_equal(kc2[:, :, l:], kc[:, :, l:])
+
+
+@pytest.mark.parametrize("l,kk", [(2, 5), (17, 3), (5, 40)])
+def test_prefill_rows_are_the_last_rows_of_causal_sdpa_over_cache_plus_new(l, kk):
+    """Listing mask tril(ones(l, l+k), diagonal=k): new token i sees the k cached entries and new tokens 0..i --
+    exactly the last l rows of plain causal attention over the concatenation; written out with the library
+    routine and an explicit boolean mask."""
+    B, H, D = 1, 2, 8
+    q, k, v = (_rand((B, H, l, D), sd) for sd in (320, 321, 322))
+    kc, vc = _rand((B, H, kk + l + 1, D), 323), _rand((B, H, kk + l + 1, D), 324)
+    o, lse, kc2, vc2 = oracle.prefill_attn(q, k, v, kc, vc, kk)
+    K = np.concatenate([kc[:, :, :kk], k], axis=2)
+    V = np.concatenate([vc[:, :, :kk], v], axis=2)
+    mask = torch.tril(torch.ones(l, l + kk, dtype=torch.bool), diagonal=kk)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q), torch.from_numpy(K), torch.from_numpy(V), attn_mask=mask).numpy()
+    assert np.allclose(o, ref, atol=1e-13)
+    # row sums of the implied probabilities: lse is the log of the normaliser of exactly the allowed scores
+    sc = np.einsum("bhid,bhjd->bhij", q, K) / math.sqrt(D)
+    want_lse = np.log(np.where(mask.numpy(), np.exp(sc), 0.0).sum(-1))
+    assert np.allclose(lse, want_lse, atol=1e-12)
+    assert np.array_equal(kc2[:, :, :kk + l], K) and np.array_equal(vc2[:, :, :kk + l], V)
+
+
+@pytest.mark.parametrize("c,t,pieces", [(4, 4, [56]), (4, 4, [5, 51]), (2, 2, [1, 2, 3, 4, 5]), (3, 5, [7, 7, 7, 7, 7, 3]),
+                                        (4, 4, [16, 16, 16, 8]), (2, 8, [40, 1, 15])])
+@pytest.mark.parametrize("prior", [0, 1])
+def test_prompt_fed_in_pieces_equals_the_one_shot_inference_layout(c, t, pieces, prior):
+    """Appendix A `add_token_ids`: however a prompt is cut into pieces (a piece that starts or ends in the middle
+    of a chunk goes through `inference_input` with several tokens over a non-empty cache), every reading and
+    memory row comes out as in the one-pass forward over the inference layout, and the cache ends up holding
+    the memory zones in order followed by the tail."""
+    flags = NOREP | prior
+    tc = c * t
+    n_tok = sum(pieces)
+    n, tail = n_tok // tc, n_tok % tc
+    S = oracle.seq_len(n, c, t, tail, flags)
+    D = 8
+    q, k, v = (_rand((1, 2, S, D), sd) for sd in (330, 331, 332))
+    O, _ = oracle.masked_attn_fwd(q, k, v, n, c, t, tail, flags)
+    Og, kc, vc, length = oracle.replay_prompt_pieces(q, k, v, pieces, c, t, flags)
+    assert not np.isnan(Og).any()
+    assert np.allclose(Og, O, atol=1e-13)
+    zn = oracle.layout_index(n, c, t, tail, flags)[1]
+    mem_rows = np.nonzero(zn == oracle.ZONE_MEM)[0].tolist()
+    tail_rows = list(range(n * (tc + t), S))
+    assert length == len(mem_rows) + tail
+    assert np.array_equal(kc[:, :, :length], k[:, :, mem_rows + tail_rows])
+    assert np.array_equal(vc[:, :, :length], v[:, :, mem_rows + tail_rows])
+    # and one token per piece is the token-by-token replay
+    Og1 = oracle.replay_generation(q, k, v, n, c, t, tail, flags)[0]
+    assert np.allclose(Og1, O, atol=1e-13)
+
+
+def test_planted_mistakes_in_prefill_are_caught(monkeypatch):
+    """A shifted diagonal, a mask that forgets the cache, and an append at the wrong slot must each fail a pin."""
+    good = lo.prefill_attn
+
+    def shifted(q, k_new, v_new, kc, vc, cache_len, scale=None):       # token i does not see itself
+        o, lse, a, b = good(q, k_new, v_new, kc, vc, cache_len, scale)
+        l = np.asarray(q).shape[2]
+        if l > 1 or cache_len > 0:
+            o2 = good(q, k_new, v_new, kc, vc, max(cache_len - 1, 0), scale)[0] if cache_len > 0 else o * 0.5
+            return o2, lse, a, b
+        return o, lse, a, b
+
+    def forgets_cache(q, k_new, v_new, kc, vc, cache_len, scale=None):  # causal among the new tokens only
+        l = np.asarray(q).shape[2]
+        o, lse, _, _ = good(q, k_new, v_new, np.zeros_like(np.asarray(kc)[:, :, :l + 1]), np.zeros_like(np.asarray(vc)[:, :, :l + 1]), 0, scale)
+        _, _, a, b = good(q, k_new, v_new, kc, vc, cache_len, scale)
+        return o, lse, a, b
+
+    def wrong_slot(q, k_new, v_new, kc, vc, cache_len, scale=None):     # appended one slot too far
+        o, lse, a, b = good(q, k_new, v_new, kc, vc, cache_len, scale)
+        return o, lse, np.roll(a, 1, axis=2), b
+
+    for bad in (shifted, forgets_cache, wrong_slot):
+        monkeypatch.setattr(oracle, "prefill_attn", bad)
+        monkeypatch.setattr(lo, "prefill_attn", bad)
+        with pytest.raises(AssertionError):
+            test_prefill_rows_are_the_last_rows_of_causal_sdpa_over_cache_plus_new(5, 40)
+            test_prefill_with_one_token_is_decode()
+    monkeypatch.setattr(oracle, "prefill_attn", good)
+    monkeypatch.setattr(lo, "prefill_attn", good)
+
+
 # ------------------------------------------ planted mistakes must be caught
 
 def _run_core_pins(golden_dir):
