@@ -318,6 +318,40 @@ LOMA_API int loma_decode_attn(const void* q, const void* k_new, const void* v_ne
                               loma_dtype dtype, float softmax_scale, unsigned flags,
                               void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------
+ * loma_prefill_attn -- several new tokens at once over an existing cache: Appendix A,
+ * `inference_input` called with l > 1 tokens, which `add_token_ids` does whenever a
+ * prompt (or a piece of one) arrives while the cache already holds entries: it feeds
+ * exactly as many tokens as fill the uncompressed tail up to tc, then compresses.  The
+ * mask is the listing's tril(ones(l, l + cache_len), diagonal = cache_len): new token i
+ * sees every cached entry and new tokens 0 .. i.  The l new K/V rows are appended to the
+ * cache first (bit-exact), at entries [cache_len, cache_len + l).  With l == 1 this is
+ * loma_decode_attn; with cache_len == 0 plain causal attention.
+ *
+ *   q, k_new, v_new [device, in]      [B, H, l, D] contiguous; k_new and v_new may both be
+ *                                     NULL when the new rows are already in the cache
+ *   k_cache, v_cache [device, in/out] [B, H, cap, D] contiguous; entries [0, cache_len) are
+ *                                     read, [cache_len, cache_len + l) written then read
+ *   o                [device, out]    [B, H, l, D] contiguous
+ *   lse              [device, out]    fp32 [B, H, l] or NULL
+ *   cache_len        entries before this call (memory entries + uncompressed tail), the
+ *                    same for every sequence of the batch
+ * bf16 calls with l >= 64 run on the tensor-core kernel of loma_masked_attn_fwd (its
+ * concurrency notes apply), the rest on CUDA cores.  No workspace.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CAPACITY (cache_len + l > cap), CUDA.
+ * l == 0 or B*H == 0 is a successful no-op.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_prefill_attn(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                               void* o, float* lse, int B, int H, int D, int l, int cap, int cache_len,
+                               loma_dtype dtype, float softmax_scale, unsigned flags, void* stream);
+
+/* Host-only replay of the tile plan the tensor-core kernel follows for loma_prefill_attn
+ * (Appendix A, inference_input mask): counts[i*(cache_len+l) + j] = number of visits in
+ * which new token i attends to key j, into a [host] uint8 buffer of l*(cache_len+l) bytes.
+ * A correct plan gives tril(ones(l, l+cache_len), diagonal=cache_len) exactly.  No CUDA call.
+ * Errors: INVALID_ARG. */
+LOMA_API int loma_prefill_attn_plan_coverage(int l, int cache_len, uint8_t* counts);
+
 LOMA_API size_t loma_decode_workspace_bytes(int B, int H, int D, int cache_len);
 
 /* ---------------------------------------------------------------------------

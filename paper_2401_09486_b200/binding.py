@@ -40,6 +40,8 @@ SIGNATURES = {
     "loma_rope_apply": (_i, [_p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i, _f, _i, _u, _p]),
     "loma_masked_attn_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
     "loma_masked_attn_bwd_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
+    "loma_prefill_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _f, _u, _p]),
+    "loma_prefill_attn_plan_coverage": (_i, [_i, _i, _p]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "loma_decode_attn_paged": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p, _sz, _p]),
@@ -209,6 +211,27 @@ def loma_masked_attn_plan_coverage(n_chunks: int, c: int, t: int, tail_read: int
     counts = torch.empty((S, S), dtype=torch.uint8)
     rc = lib().loma_masked_attn_plan_coverage(n_chunks, c, t, tail_read, int(flags), _ptr(counts))
     _check(rc, "loma_masked_attn_plan_coverage")
+    return counts
+
+
+def loma_prefill_attn(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len: int, flags: int = 0,
+                      softmax_scale: float = 0.0, stream=None) -> None:
+    """q, k_new, v_new, o: [B, H, l, D] contiguous; caches [B, H, cap, D] contiguous; appends then attends."""
+    B, H, l, D = q.shape
+    for x in (q, k_new, v_new, k_cache, v_cache, o):
+        if x is not None and not x.is_contiguous():
+            raise ValueError("loma_prefill_attn takes contiguous tensors")
+    rc = lib().loma_prefill_attn(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse),
+                                 B, H, D, l, k_cache.shape[2], int(cache_len), _dtype_code(q), float(softmax_scale),
+                                 int(flags), _stream(stream))
+    _check(rc, "loma_prefill_attn")
+
+
+def loma_prefill_attn_plan_coverage(l: int, cache_len: int) -> torch.Tensor:
+    """Host replay of the tensor-core kernel's tile plan for loma_prefill_attn: uint8 [l, cache_len + l] visit counts."""
+    counts = torch.empty((l, cache_len + l), dtype=torch.uint8)
+    rc = lib().loma_prefill_attn_plan_coverage(int(l), int(cache_len), _ptr(counts))
+    _check(rc, "loma_prefill_attn_plan_coverage")
     return counts
 
 

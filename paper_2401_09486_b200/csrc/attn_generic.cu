@@ -15,6 +15,8 @@
 //   repetition row (y, o): own memory zone, then itself          (Eq. 1 row 3)
 //   decode:                cache[0, len) then the new token      (Appendix A)
 //   compress:              cache tail (tc) then the t own keys   (Appendix A)
+//   prefill row i:         cache[0, len + i + 1): the cached entries and the new tokens
+//                          up to itself, already appended            (Appendix A)
 #include <math.h>
 
 #include "loma_internal.cuh"
@@ -275,6 +277,50 @@ decode_generic_kernel(const T* __restrict__ q, const T* __restrict__ k_new, cons
             kc[new_off + lane * DPL + d] = k_new[(int64_t)bh * D + lane * DPL + d];
             vc[new_off + lane * DPL + d] = v_new[(int64_t)bh * D + lane * DPL + d];
         }
+    }
+}
+
+// --------------------------------------------- several new tokens over a cache
+// Appendix A, inference_input with l tokens: the mask tril(ones(l, l + len), diagonal = len).  The new
+// tokens' K/V have been appended at [len, len + l) by cache_append_kernel before this launch, so row i simply
+// sees cache rows 0 .. len + i.
+template <typename T>
+struct CacheRangeMap {
+    const T* kc;
+    const T* vc;
+    int D;
+    __device__ __forceinline__ const T* kptr(int vi) const { return kc + (int64_t)vi * D; }
+    __device__ __forceinline__ const T* vptr(int vi) const { return vc + (int64_t)vi * D; }
+};
+
+template <typename T, int D>
+__global__ void __launch_bounds__(GENERIC_WARPS * 32)
+prefill_generic_kernel(const T* __restrict__ q, const T* __restrict__ k_cache, const T* __restrict__ v_cache,
+                       T* __restrict__ o, float* __restrict__ lse, int l, int cap, int cache_len, float scale) {
+    __shared__ __align__(16) float q_sh[GENERIC_WARPS][D];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int i = blockIdx.x * GENERIC_WARPS + warp;
+    if (i >= l) return;
+    const int bh = blockIdx.y;
+    CacheRangeMap<T> map;
+    map.kc = k_cache + (int64_t)bh * cap * D;
+    map.vc = v_cache + (int64_t)bh * cap * D;
+    map.D = D;
+    const int64_t row = ((int64_t)bh * l + i) * D;
+    stage_query<T, D>(q_sh[warp], q + row, lane);
+    attend_row<T, D>(q_sh[warp], map, cache_len + i + 1, scale, o + row, lse ? lse + (int64_t)bh * l + i : nullptr, lane);
+}
+
+// k_new, v_new [B, H, l, D] -> cache rows [cache_len, cache_len + l) of every (b, h): 16-byte vectors, bit-exact.
+__global__ void cache_append_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
+                                    uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, int vec_per_row, int l, int cap,
+                                    int cache_len) {
+    const int bh = blockIdx.y;
+    const int64_t n = (int64_t)l * vec_per_row;
+    const int64_t in = (int64_t)bh * n, out = ((int64_t)bh * cap + cache_len) * vec_per_row;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) {
+        k_cache[out + e] = __ldg(k_new + in + e);
+        v_cache[out + e] = __ldg(v_new + in + e);
     }
 }
 
@@ -611,6 +657,41 @@ cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const 
                                                            BH, cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st)
                    : compress_generic_t<__nv_bfloat16, 128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse,
                                                             BH, cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st);
+}
+
+template <typename T, int D>
+static cudaError_t prefill_generic_t(const void* q, const void* kc, const void* vc, void* o, float* lse, int BH, int l,
+                                     int cap, int cache_len, float scale, cudaStream_t st) {
+    dim3 grid((l + GENERIC_WARPS - 1) / GENERIC_WARPS, BH);
+    prefill_generic_kernel<T, D><<<grid, GENERIC_WARPS * 32, 0, st>>>(static_cast<const T*>(q), static_cast<const T*>(kc),
+                                                                     static_cast<const T*>(vc), static_cast<T*>(o), lse, l, cap,
+                                                                     cache_len, scale);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_prefill_attn_generic(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                                        int B, int H, int D, int l, int cap, int cache_len, loma_dtype dt, float scale,
+                                        cudaStream_t st) {
+    const int BH = B * H;
+    if (dt == LOMA_F32)
+        return D == 64 ? prefill_generic_t<float, 64>(q, k_cache, v_cache, o, lse, BH, l, cap, cache_len, scale, st)
+                       : prefill_generic_t<float, 128>(q, k_cache, v_cache, o, lse, BH, l, cap, cache_len, scale, st);
+    return D == 64 ? prefill_generic_t<__nv_bfloat16, 64>(q, k_cache, v_cache, o, lse, BH, l, cap, cache_len, scale, st)
+                   : prefill_generic_t<__nv_bfloat16, 128>(q, k_cache, v_cache, o, lse, BH, l, cap, cache_len, scale, st);
+}
+
+cudaError_t launch_cache_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache, int B, int H,
+                                int row_bytes, int l, int cap, int cache_len, cudaStream_t st) {
+    const int vec = row_bytes / 16;
+    const int64_t n = (int64_t)l * vec;
+    int gx = (int)((n + 255) / 256);
+    if (gx > 64) gx = 64;
+    dim3 grid(gx, B * H);
+    cache_append_kernel<<<grid, 256, 0, st>>>(static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new),
+                                              static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache), vec, l, cap, cache_len);
+    count_launches(1);
+    return cudaGetLastError();
 }
 
 }  // namespace loma

@@ -551,6 +551,38 @@ static unsigned* sched_counters(cudaStream_t st) {
     return base[dev] + 2 * n_owner[dev]++;
 }
 
+// Launch of the kernel for a finished plan: per-device set-up (done once), grid size.
+static cudaError_t launch_tc_kernel(const TmaMaps& maps, const FwdParams& p, int D, cudaStream_t st) {
+    // SM count and the opt-in to large dynamic shared memory
+    static int sm_count[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (sm_count[dev] == 0) {
+        int sms = 0;
+        cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(masked_attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TcSmem<128>::TOTAL + 1024);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(masked_attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 TcSmem<64>::TOTAL + 1024);
+        if (e != cudaSuccess) return e;
+        sm_count[dev] = sms;
+    }
+    const int sms = sm_count[dev];
+    const int64_t work = (int64_t)p.total_tiles * p.BH;
+    const int64_t want = (work + 1) / 2;            // two streams (query tiles in flight) per CTA
+    const int grid = (int)(want < sms ? want : sms);
+    // the shared-memory footprint also keeps one CTA per SM (each allocates all 512 TMEM columns)
+    if (D == 128)
+        masked_attn_tc_kernel<128><<<grid, TC_THREADS, TcSmem<128>::TOTAL + 1024, st>>>(maps, p);
+    else
+        masked_attn_tc_kernel<64><<<grid, TC_THREADS, TcSmem<64>::TOTAL + 1024, st>>>(maps, p);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+
 struct MapCacheKey {
     const void *q, *k, *v, *o;
     int B, H, D, n, c, t, tail;
@@ -608,33 +640,57 @@ cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, v
         maps = cached_maps;
     }
 
-    // per-device set-up, done once: SM count and the opt-in to large dynamic shared memory
-    static int sm_count[64] = {0};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (sm_count[dev] == 0) {
-        int sms = 0;
-        cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(masked_attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 TcSmem<128>::TOTAL + 1024);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(masked_attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 TcSmem<64>::TOTAL + 1024);
-        if (e != cudaSuccess) return e;
-        sm_count[dev] = sms;
+    return launch_tc_kernel(maps, p, D, st);
+}
+
+// New tokens over an existing cache on the same kernel: the query view is the l new rows, the key view the
+// cache rows 0 .. cache_len + l - 1 (the new rows' K/V have been appended before this launch).
+// q, o: [B, H, l, D] contiguous; k_cache, v_cache: [B, H, cap, D] contiguous.
+cudaError_t launch_prefill_attn_tc(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, int B,
+                                   int H, int D, int l, int cap, int cache_len, float scale, cudaStream_t st) {
+    if (!encode_fn()) return cudaErrorNotSupported;
+    FwdParams p{};
+    make_prefill_plan(l, cache_len, B, H, &p);
+    p.scale_log2 = scale * 1.4426950408889634f;
+    p.lse = lse;
+    p.status = device_status_word();
+    if (!p.status) return cudaErrorUnknown;
+    if ((int64_t)p.total_tiles * p.BH > 0x7ffffff0ll - 2 * 148) return cudaErrorNotSupported;
+    p.sched = sched_counters(st);   // NULL: static deal
+
+    struct Key {
+        const void *q, *k, *v, *o;
+        int B, H, D, l, cap, cache_len;
+        bool operator==(const Key& r) const {
+            return q == r.q && k == r.k && v == r.v && o == r.o && B == r.B && H == r.H && D == r.D && l == r.l &&
+                   cap == r.cap && cache_len == r.cache_len;
+        }
+    };
+    static std::mutex mu;
+    static Key cached_key{};
+    static TmaMaps cached_maps;
+    static bool have_cache = false;
+    TmaMaps maps;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        Key key{q, k_cache, v_cache, o, B, H, D, l, cap, cache_len};
+        if (!(have_cache && key == cached_key)) {
+            TmaMaps mnew{};
+            const int64_t qs_h = (int64_t)l * D, qs_b = qs_h * H, cs_h = (int64_t)cap * D, cs_b = cs_h * H;
+            const View& qv = p.view[V_TAIL];
+            const View& kv = p.view[V_MEM];
+            if (!encode_view(&mnew.q[V_TAIL], q, qv, D, B, H, 0, qs_b, qs_h, D, l) ||
+                !encode_view(&mnew.o[V_TAIL], o, qv, D, B, H, 0, qs_b, qs_h, D, l) ||
+                !encode_view(&mnew.k[V_MEM], k_cache, kv, D, B, H, 0, cs_b, cs_h, D, cache_len + l) ||
+                !encode_view(&mnew.v[V_MEM], v_cache, kv, D, B, H, 0, cs_b, cs_h, D, cache_len + l))
+                return cudaErrorNotSupported;
+            cached_maps = mnew;
+            cached_key = key;
+            have_cache = true;
+        }
+        maps = cached_maps;
     }
-    const int sms = sm_count[dev];
-    const int64_t work = (int64_t)p.total_tiles * p.BH;
-    const int64_t want = (work + 1) / 2;            // two streams (query tiles in flight) per CTA
-    const int grid = (int)(want < sms ? want : sms);
-    // the shared-memory footprint also keeps one CTA per SM (each allocates all 512 TMEM columns)
-    if (D == 128)
-        masked_attn_tc_kernel<128><<<grid, TC_THREADS, TcSmem<128>::TOTAL + 1024, st>>>(maps, p);
-    else
-        masked_attn_tc_kernel<64><<<grid, TC_THREADS, TcSmem<64>::TOTAL + 1024, st>>>(maps, p);
-    count_launches(1);
-    return cudaGetLastError();
+    return launch_tc_kernel(maps, p, D, st);
 }
 
 }  // namespace loma

@@ -334,6 +334,50 @@ int loma_decode_attn(const void* q, const void* k_new, const void* v_new, void* 
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 
+int loma_prefill_attn(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
+                      float* lse, int B, int H, int D, int l, int cap, int cache_len, loma_dtype dtype,
+                      float softmax_scale, unsigned flags, void* stream) {
+    if (B < 0 || H < 0 || l < 0 || cap < 0 || cache_len < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    if ((k_new == nullptr) != (v_new == nullptr)) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)cache_len + l > cap) return LOMA_ERR_CAPACITY;
+    if (B == 0 || H == 0 || l == 0) return LOMA_OK;
+    if (!q || !k_cache || !v_cache || !o) return LOMA_ERR_INVALID_ARG;
+    if (o == q || o == k_new || o == v_new) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) || !aligned16(k_new) ||
+        !aligned16(v_new))
+        return LOMA_ERR_ALIGNMENT;
+    if (lse && ((uintptr_t)lse & 3u)) return LOMA_ERR_ALIGNMENT;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // 1. the new tokens' K/V go into the cache (bit-exact); 2. every new row attends to cache rows 0 .. cache_len + i
+    if (k_new) {
+        if (launch_cache_append(k_new, v_new, k_cache, v_cache, B, H, (int)(D * elt_size(dtype)), l, cap, cache_len, st) !=
+            cudaSuccess)
+            return LOMA_ERR_CUDA;
+    }
+    cudaError_t e = cudaErrorNotSupported;
+    if (dtype == LOMA_BF16 && l >= 64 && !(flags & LOMA_FLAG_FORCE_GENERIC)) {
+        e = launch_prefill_attn_tc(q, k_cache, v_cache, o, lse, B, H, D, l, cap, cache_len, scale, st);
+        if (e == cudaErrorNotSupported) g_fallbacks.fetch_add(1, std::memory_order_relaxed);
+    }
+    if (e == cudaErrorNotSupported)
+        e = launch_prefill_attn_generic(q, k_cache, v_cache, o, lse, B, H, D, l, cap, cache_len, dtype, scale, st);
+    return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
+int loma_prefill_attn_plan_coverage(int l, int cache_len, uint8_t* counts) {
+    if (l < 0 || cache_len < 0) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)l * ((int64_t)l + cache_len) > (1ll << 32)) return LOMA_ERR_INVALID_ARG;
+    if (l > 0 && !counts) return LOMA_ERR_INVALID_ARG;
+    if (l > 0) prefill_plan_coverage_host(l, cache_len, counts);
+    return LOMA_OK;
+}
+
 int loma_decode_attn_ragged(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
                             float* lse, int B, int H, int D, int cap, const int32_t* cache_lens, int max_cache_len,
                             loma_dtype dtype, float softmax_scale, unsigned flags, void* workspace,

@@ -99,7 +99,18 @@ cudaError_t launch_masked_attn_bwd_dkv_tc(const void* q, const void* k, const vo
 cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, void* o, float* lse, int B, int H, int D,
                                   const Layout& L, int64_t sb, int64_t sh, int64_t ss, float scale, cudaStream_t st);
 
+// l new tokens over a cache that already holds their K/V at [cache_len, cache_len + l) (attn_tcgen05.cu)
+cudaError_t launch_prefill_attn_tc(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, int B,
+                                   int H, int D, int l, int cap, int cache_len, float scale, cudaStream_t st);
+// the same on CUDA cores (any l, fp32 or bf16), and the bit-exact append that precedes both (attn_generic.cu)
+cudaError_t launch_prefill_attn_generic(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
+                                        int B, int H, int D, int l, int cap, int cache_len, loma_dtype dt, float scale,
+                                        cudaStream_t st);
+cudaError_t launch_cache_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache, int B, int H,
+                                int row_bytes, int l, int cap, int cache_len, cudaStream_t st);
+
 void plan_coverage_host(const Layout& L, uint8_t* counts);          // tile_plan_host.cu
+void prefill_plan_coverage_host(int l, int cache_len, uint8_t* counts);
 void plan_coverage_by_key_host(const Layout& L, uint8_t* counts);   // the plan read by key tile (backward)
 
 cudaError_t launch_bounded_wait_selftest(cudaStream_t st);   // attn_tcgen05.cu

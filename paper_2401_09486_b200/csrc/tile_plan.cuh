@@ -39,7 +39,7 @@ __host__ __device__ __forceinline__ int fdiv(int n, const FastDiv& f) {
 }
 
 enum { V_READ = 0, V_MEM = 1, V_REP = 2, V_TAIL = 3 };
-enum { M_LT = 0, M_LE = 1, M_EQ = 2, M_CAUSAL = 3, M_DIAG = 4 };
+enum { M_LT = 0, M_LE = 1, M_EQ = 2, M_CAUSAL = 3, M_DIAG = 4, M_CAUSAL_OFF = 5 };   // M_CAUSAL_OFF: causal with the diagonal moved by View::diag
 
 struct View {
     int Z;           // zone length (rows per chunk in this view)
@@ -50,6 +50,7 @@ struct View {
     int nch;         // chunks in the view
     int chunk_base;  // absolute chunk number of the view's chunk 0 (n_chunks for the tail)
     int zone_row0;   // first row of the zone inside its chunk
+    int diag;        // key views of the prefill plan: row o of the query view sees keys 0 .. o + diag (M_CAUSAL_OFF)
     FastDiv dR, dCH, dtpc;   // division by R, CH and tpc
 };
 
@@ -59,6 +60,7 @@ struct FwdParams {
     int total_tiles;
     int n_tail, n_read, n_mem, n_rep;   // tiles per view, in scheduling order
     unsigned flags;
+    int prefill;       // 1: the plan of loma_prefill_attn (query view V_TAIL over the new tokens, key view V_MEM over the cache)
     FastDiv dBH, dH;
     float scale_log2;
     float* lse;
@@ -102,7 +104,13 @@ __host__ __device__ __forceinline__ void decode_tile(const FwdParams& p, int ran
     const View& vm = p.view[V_MEM];
     const View& vr = p.view[V_READ];
     const int sub = (g.Z >= 128) ? qi - td.c0 * g.tpc : 0;   // tile index inside its chunk
-    if (view == V_READ || view == V_TAIL) {
+    if (p.prefill) {
+        // new tokens over the cache (Appendix A, inference_input): key tiles 0 .. the one that holds the
+        // diagonal of the tile's last row (row o sees keys 0 .. o + diag)
+        const int last_row = plan_min(td.r0 + 127, g.Z - 1);
+        td.seg[0] = Seg{V_MEM, M_CAUSAL_OFF, 0, (last_row + vm.diag) / 128 + 1};
+        td.seg[1] = Seg{V_MEM, M_CAUSAL_OFF, 0, 0};
+    } else if (view == V_READ || view == V_TAIL) {
         // memory zones of every earlier chunk, then the own reading zone up to this tile
         td.seg[0] = Seg{V_MEM, M_LT, 0, tiles_covering(vm, td.a1)};
         td.seg[1] = Seg{view, M_CAUSAL, (g.Z >= 128) ? td.c0 * g.tpc : qi, sub + 1};
@@ -144,6 +152,8 @@ __host__ __device__ __forceinline__ void row_interval(const View& kv, const KTil
         hi = nch > 0 ? (nch - 1) * kv.R + vcols : 0;
     } else if (kt.mode == M_DIAG) {
         lo = rr; hi = rr + 1;
+    } else if (kt.mode == M_CAUSAL_OFF) {
+        hi = plan_min(plan_max(ro + kv.diag - kt.r0 + 1, 0), vcols);
     } else if (d >= 0 && d < kv.CH) {
         lo = d * kv.R;
         hi = lo + (kt.mode == M_EQ ? vcols : plan_min(plan_max(ro - kt.r0 + 1, 0), vcols));
@@ -164,6 +174,9 @@ __host__ __device__ __forceinline__ unsigned step_halves(const FwdParams& p, con
         uhi = nch > 0 ? (nch - 1) * kv.R + vcols : 0;
     } else if (kt.mode == M_DIAG) {
         uhi = 128;
+    } else if (kt.mode == M_CAUSAL_OFF) {
+        const int last_row = plan_min(td.r0 + 127, p.view[td.view].Z - 1);
+        uhi = plan_min(plan_max(last_row + kv.diag - kt.r0 + 1, 0), vcols);
     } else {
         const int d0 = plan_max(td.a0 - kt.a0, 0), d1 = plan_min(td.a1 - kt.a0, kv.CH - 1);
         if (d1 >= d0) { ulo = d0 * kv.R; uhi = d1 * kv.R + vcols; }
@@ -353,7 +366,23 @@ inline void make_plan(const Layout& L, int B, int H, FwdParams* p) {
     p->n_tail = p->view[V_TAIL].ntiles; p->n_read = p->view[V_READ].ntiles;
     p->n_mem = p->view[V_MEM].ntiles; p->n_rep = p->view[V_REP].ntiles;
     p->total_tiles = p->n_tail + p->n_read + p->n_mem + p->n_rep;
-    p->flags = L.flags;
+    p->flags = L.flags; p->prefill = 0;
+    p->dBH = make_fastdiv(p->BH); p->dH = make_fastdiv(H);
+}
+
+// The plan of loma_prefill_attn: l new tokens (query view V_TAIL, one "chunk" of l rows) over a cache that holds
+// cache_len earlier entries followed by the l new ones (key view V_MEM, one chunk of cache_len + l rows); row o
+// sees keys 0 .. o + cache_len.
+inline void make_prefill_plan(int l, int cache_len, int B, int H, FwdParams* p) {
+    p->view[V_READ] = make_view(0, 0, 0, 0);
+    p->view[V_MEM] = make_view(cache_len + l, 1, 0, 0);
+    p->view[V_MEM].diag = cache_len;
+    p->view[V_REP] = make_view(0, 0, 0, 0);
+    p->view[V_TAIL] = make_view(l, 1, 0, 0);
+    p->n_chunks = 0; p->s = 0; p->S = l; p->H = H; p->BH = B * H;
+    p->n_tail = p->view[V_TAIL].ntiles; p->n_read = 0; p->n_mem = 0; p->n_rep = 0;
+    p->total_tiles = p->n_tail;
+    p->flags = 0; p->prefill = 1;
     p->dBH = make_fastdiv(p->BH); p->dH = make_fastdiv(H);
 }
 

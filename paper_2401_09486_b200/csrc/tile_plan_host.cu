@@ -52,6 +52,52 @@ void plan_coverage_host(const Layout& L, uint8_t* counts) {
     }
 }
 
+// The plan of loma_prefill_attn replayed the same way: counts[i * (cache_len + l) + j] = visits in which new
+// token i attends to key j (cached entries 0 .. cache_len - 1, then the new tokens).  A correct plan gives
+// tril(ones(l, l + cache_len), diagonal = cache_len).
+void prefill_plan_coverage_host(int l, int cache_len, uint8_t* counts) {
+    FwdParams p{};
+    make_prefill_plan(l, cache_len, 1, 1, &p);
+    const int64_t W = (int64_t)cache_len + l;
+    memset(counts, 0, (size_t)l * W);
+    for (int rank = 0; rank < p.total_tiles; ++rank) {
+        TileDesc td;
+        decode_tile(p, rank, td);
+        const View& qv = p.view[td.view];
+        HalfMasks hm{{0, 0}};
+        for (int j = 0; j < td.nsteps && j < 64; ++j) {
+            const unsigned v = visited_halves(p, td, j);
+            hm.m[0] |= (unsigned long long)(v & 1u) << j;
+            hm.m[1] |= (unsigned long long)((v >> 1) & 1u) << j;
+        }
+        HalfWalk hw;
+        for (hw.start(hm); !hw.done(td.nsteps); hw.next(hm)) {
+            KTile kt;
+            step_ktile(p, td, hw.j, kt);
+            const View& kv = p.view[kt.view];
+            for (int rr = 0; rr < 128; ++rr) {
+                const int rsub = rr / qv.R;
+                const int ro = td.r0 + (rr - rsub * qv.R);
+                const int rc = td.a0 + rsub;
+                const bool row_valid = (rr < qv.R * qv.CH) && (rc <= td.a1) && (ro < qv.Z);
+                int lo, hi;
+                row_interval(kv, kt, rc, ro, rr, row_valid, lo, hi);
+                if (!row_valid || hi <= lo) continue;
+                for (int col = (lo > 64 * hw.h ? lo : 64 * hw.h); col < hi && col < 64 * hw.h + 64; ++col) {
+                    const int ksub = col / kv.R;
+                    const int64_t key = kt.r0 + (col - ksub * kv.R);
+                    if (ksub == 0 && ro < l && key < W) {
+                        uint8_t& c = counts[(int64_t)ro * W + key];
+                        if (c < 255) ++c;
+                    } else {
+                        counts[0] = 255;   // a column outside the cache: never allowed
+                    }
+                }
+            }
+        }
+    }
+}
+
 // The same count, taken from the key-tile side of the plan (the backward's dK/dV pass).
 void plan_coverage_by_key_host(const Layout& L, uint8_t* counts) {
     FwdParams p{};

@@ -109,6 +109,33 @@ def test_masked_attn_fwd_validation_precedes_any_cuda_call(lib):
     assert _fwd(lib, B=0) == 0
 
 
+def test_prefill_attn_validation(lib):
+    def call(q=0x1000, kn=0x2000, vn=0x3000, kc=0x4000, vc=0x5000, o=0x6000, lse=None, B=1, H=1, D=128, l=4, cap=16,
+             cache_len=3, dt=1, flags=0):
+        return lib.loma_prefill_attn(q, kn, vn, kc, vc, o, lse, B, H, D, l, cap, cache_len, dt, 0.0, flags, None)
+    assert call(cache_len=13) == CAPACITY                # 13 + 4 > 16
+    assert call(l=-1) == INVALID
+    assert call(kn=None) == INVALID                      # k_new without v_new
+    assert call(o=0x1000) == INVALID                     # o aliases q
+    assert call(q=None) == INVALID
+    assert call(D=96) == UNSUPPORTED
+    assert call(dt=5) == UNSUPPORTED
+    assert call(vc=0x5004) == ALIGNMENT
+    assert call(lse=0x7002) == ALIGNMENT
+    assert call(l=0) == 0
+    assert call(H=0) == 0
+
+
+@pytest.mark.parametrize("l", [1, 2, 17, 64, 100, 128, 129, 200, 300, 517])
+@pytest.mark.parametrize("cache_len", [0, 1, 16, 63, 64, 100, 127, 128, 500, 8192])
+def test_prefill_tile_plan_reproduces_the_listing_mask(lib, l, cache_len):
+    """The tensor-core kernel's plan for several tokens over a cache visits exactly the entries of
+    tril(ones(l, l + k), diagonal = k) (Appendix A, `inference_input`), each once."""
+    got = binding.loma_prefill_attn_plan_coverage(l, cache_len).numpy()
+    want = np.tril(np.ones((l, l + cache_len), np.uint8), k=cache_len)
+    assert np.array_equal(got, want), f"{int((got != want).sum())} entries differ"
+
+
 def test_prefill_cache_validation(lib):
     def call(k=0x1000, v=0x2000, kc=0x3000, vc=0x4000, B=1, H=1, D=128, cap=64, n=2, c=4, t=16, tc=64, tail=3,
              sb=100000, sh=100000, ss=128, dt=1, flags=0):

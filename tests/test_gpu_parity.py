@@ -262,6 +262,103 @@ def test_incremental_generation_equals_one_shot(B, H, D, n, c, t, tail, flags, d
     assert torch.equal(vc[:, :, :length].cpu(), v[:, :, rows])
 
 
+# ------------------------------------------- several new tokens over an existing cache
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, GENERIC])
+@pytest.mark.parametrize("l", [1, 2, 17, 64, 200, 300])
+@pytest.mark.parametrize("cache_len", [0, 16, 100, 8192])
+def test_prefill_over_a_cache_matches_oracle_and_appends_bit_exact(l, cache_len, flags, dtype):
+    """Appendix A `inference_input` with l tokens: mask tril(ones(l, l + k), diagonal = k), K/V appended."""
+    B, H, D = (1, 2, 128) if cache_len > 1000 else (2, 3, 128 if l != 17 else 64)
+    cap = cache_len + l + 5
+    kc = synthetic.normal_tensor((B, H, cap, D), 41, 1.0, dtype)
+    vc = synthetic.normal_tensor((B, H, cap, D), 42, 1.0, dtype)
+    q, kn, vn = synthetic.qkv(B, H, l, D, seed=43, std=1.0, dtype=dtype)
+    want_o, want_lse, want_kc, want_vc = oracle.prefill_attn(npf(q), npf(kn), npf(vn), npf(kc), npf(vc), cache_len)
+    kcd, vcd = kc.to(DEV), vc.to(DEV)
+    o = torch.full((B, H, l, D), float("nan"), dtype=dtype, device=DEV)
+    lse = torch.full((B, H, l), float("nan"), dtype=torch.float32, device=DEV)
+    L.loma_prefill_attn(q.to(DEV), kn.to(DEV), vn.to(DEV), kcd, vcd, o, lse, cache_len, flags)
+    torch.cuda.synchronize()
+    check_close(o, want_o, dtype)
+    assert np.abs(npf(lse) - want_lse).max() <= (1e-5 if dtype == torch.float32 else 2e-2)
+    # the cache: new rows appended bit for bit, everything else untouched
+    exp_k, exp_v = kc.clone(), vc.clone()
+    exp_k[:, :, cache_len:cache_len + l] = kn
+    exp_v[:, :, cache_len:cache_len + l] = vn
+    assert np.array_equal(bits(kcd), bits(exp_k)) and np.array_equal(bits(vcd), bits(exp_v))
+    assert np.array_equal(npf(kcd), want_kc) and np.array_equal(npf(vcd), want_vc)
+
+
+def test_prefill_with_rows_already_in_the_cache_and_repeatable():
+    """k_new = v_new = NULL: the new rows are read where they already lie; two calls give the same bits."""
+    B, H, D, l, cache_len = 2, 2, 128, 150, 333
+    cap = cache_len + l
+    kc = synthetic.normal_tensor((B, H, cap, D), 51, 1.0, torch.bfloat16).to(DEV)
+    vc = synthetic.normal_tensor((B, H, cap, D), 52, 1.0, torch.bfloat16).to(DEV)
+    q = synthetic.normal_tensor((B, H, l, D), 53, 1.0, torch.bfloat16).to(DEV)
+    want_o, _, _, _ = oracle.prefill_attn(npf(q), npf(kc[:, :, cache_len:]), npf(vc[:, :, cache_len:]), npf(kc), npf(vc), cache_len)
+    o1, o2 = torch.empty_like(q), torch.empty_like(q)
+    L.loma_prefill_attn(q, None, None, kc, vc, o1, None, cache_len)
+    L.loma_prefill_attn(q, None, None, kc, vc, o2, None, cache_len)
+    torch.cuda.synchronize()
+    check_close(o1, want_o, torch.bfloat16)
+    assert torch.equal(o1, o2)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("c,t,pieces", [(4, 16, [150, 74]), (8, 16, [70, 200, 178]), (2, 8, [5, 51])])
+def test_prompt_ingested_in_pieces_equals_the_one_shot_inference_layout(c, t, pieces, dtype):
+    """Appendix A `add_token_ids` on the GPU path: a prompt of 3.5 chunks arrives in pieces that start and end in
+    the middle of chunks; every piece goes through loma_prefill_attn over the cache as it stands (exactly the
+    tokens that fill the tail up to tc, then loma_compress_step), and every reading and memory row equals the
+    one-pass forward over the inference layout; the cache ends as memory zones in order plus the tail."""
+    B, H, D = 1, 2, 128
+    tc = c * t
+    n_tok = sum(pieces)
+    n, tail = n_tok // tc, n_tok % tc
+    s = tc + t
+    S = oracle.seq_len(n, c, t, tail, NOREP)
+    q, k, v = synthetic.qkv(B, H, S, D, seed=61, std=1.0, dtype=dtype)
+    want_o, _ = oracle.masked_attn_fwd(npf(q), npf(k), npf(v), n, c, t, tail, NOREP)
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    cap = n * t + tc + 8
+    kc = torch.zeros((B, H, cap, D), dtype=dtype, device=DEV)
+    vc = torch.zeros_like(kc)
+    got = torch.full_like(qd, float("nan"))
+    ws = workspace(L.loma_compress_workspace_bytes(B, H, D, t, n * t, 0))
+    row_of = lambda g: (g // tc) * s + g % tc
+    length = done = chunks = fed = 0
+    for piece in pieces:
+        fed += piece
+        while done < fed:
+            take = fed - done
+            fills = (length - chunks * t) + take >= tc
+            if fills:
+                take = tc - (length - chunks * t)
+            rows = torch.tensor([row_of(g) for g in range(done, done + take)], device=DEV)
+            o = torch.empty((B, H, take, D), dtype=dtype, device=DEV)
+            L.loma_prefill_attn(qd[:, :, rows].contiguous(), kd[:, :, rows].contiguous(), vd[:, :, rows].contiguous(), kc, vc, o,
+                                None, length)
+            got[:, :, rows] = o
+            length += take
+            done += take
+            if fills:
+                m0 = chunks * s + tc
+                om = torch.empty((B, H, t, D), dtype=dtype, device=DEV)
+                L.loma_compress_step(qd[:, :, m0:m0 + t].contiguous(), kd[:, :, m0:m0 + t].contiguous(),
+                                     vd[:, :, m0:m0 + t].contiguous(), kc, vc, om, None, chunks * t, c, t, ws)
+                got[:, :, m0:m0 + t] = om
+                chunks += 1
+                length = chunks * t
+    torch.cuda.synchronize()
+    check_close(got, want_o, dtype)
+    rows = [y * s + tc + j for y in range(n) for j in range(t)] + list(range(n * s, S))
+    assert length == len(rows)
+    assert torch.equal(kc[:, :, :length].cpu(), k[:, :, rows]) and torch.equal(vc[:, :, :length].cpu(), v[:, :, rows])
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_staggered_sequences_over_a_paged_cache_equal_the_one_shot_forward(dtype):
     """Invariant (c) through the ragged and paged entry points: three sequences that started 0, 5 and 11 tokens
