@@ -319,6 +319,35 @@ LOMA_API int loma_decode_attn(const void* q, const void* k_new, const void* v_ne
                               void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * loma_decode_attn_rope, loma_compress_step_rope -- the two generation steps with the rotary
+ * position embedding of Section 4.5 done inside the step: q and the new key(s) are rotated in
+ * registers / shared memory by their position ids right where the kernels load them, so the
+ * generation loop has no separate rotation pass (the training layout is rotated by
+ * loma_rope_apply).  The rotation is the one loma_rope_apply documents (feature d paired with
+ * d + D/2, angle pos * theta_base^(-2d/D), theta_base <= 0 selects 10000).  The rotated keys,
+ * rounded to the storage type, are what the step attends to and what is written to the cache;
+ * values are not rotated.  Everything else is as in loma_decode_attn / loma_compress_step.
+ *
+ *   decode:    pos = the token's position id -- the generator's `cursor` (Appendix A,
+ *              inference_input: position_ids = arange(cursor, cursor + l)); k_new and v_new
+ *              are required
+ *   compress:  memory row j gets pos0 + j * pos_stride: Eq. 14 ('intermittent') is
+ *              pos0 = y*tc + c - 1, pos_stride = c for chunk y; the generator's other setting
+ *              is pos0 = mem_len (= mem_cursor), pos_stride = 1 (Appendix A, compress_last_chunk)
+ * Errors: as the plain calls, plus INVALID_ARG for a negative position or missing k_new, and
+ * UNSUPPORTED for a memory zone too long to stage (t*D*sizeof(element) > 200 KB).
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_decode_attn_rope(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                                   void* o, float* lse, int B, int H, int D, int cap, int cache_len, int pos,
+                                   float theta_base, loma_dtype dtype, float softmax_scale, unsigned flags,
+                                   void* workspace, size_t workspace_bytes, void* stream);
+LOMA_API int loma_compress_step_rope(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache,
+                                     void* v_cache, void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len,
+                                     int c, int t, int tc, int pos0, int pos_stride, float theta_base, loma_dtype dtype,
+                                     float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes,
+                                     void* stream);
+
+/* ---------------------------------------------------------------------------
  * loma_prefill_attn -- several new tokens at once over an existing cache: Appendix A,
  * `inference_input` called with l > 1 tokens, which `add_token_ids` does whenever a
  * prompt (or a piece of one) arrives while the cache already holds entries: it feeds

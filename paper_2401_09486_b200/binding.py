@@ -43,6 +43,9 @@ SIGNATURES = {
     "loma_prefill_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _f, _u, _p]),
     "loma_prefill_attn_plan_coverage": (_i, [_i, _i, _p]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
+    "loma_decode_attn_rope": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _i, _f, _u, _p, _sz, _p]),
+    "loma_compress_step_rope": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _i, _f, _u, _p,
+                                     _sz, _p]),
     "loma_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "loma_decode_attn_paged": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_attn_ragged": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p, _sz, _p]),
@@ -296,6 +299,38 @@ def loma_decode_attn(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len: int, 
                                 _ptr(lse), B, H, D, cap, cache_len, _dtype_code(q), float(softmax_scale),
                                 int(flags), _ptr(workspace), ws_bytes, _stream(stream))
     _check(rc, "loma_decode_attn")
+
+
+def loma_decode_attn_rope(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len: int, pos: int, workspace=None,
+                          flags: int = 0, softmax_scale: float = 0.0, theta_base: float = 0.0, stream=None) -> None:
+    """loma_decode_attn with q and k_new rotated inside the step by the position id `pos`."""
+    B, H, cap, D = k_cache.shape
+    for x in (q, k_new, v_new, k_cache, v_cache, o):
+        if x is not None and not x.is_contiguous():
+            raise ValueError("decode tensors must be contiguous")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().loma_decode_attn_rope(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(o),
+                                     _ptr(lse), B, H, D, cap, cache_len, int(pos), float(theta_base), _dtype_code(q),
+                                     float(softmax_scale), int(flags), _ptr(workspace), ws_bytes, _stream(stream))
+    _check(rc, "loma_decode_attn_rope")
+
+
+def loma_compress_step_rope(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, mem_len: int, c: int, t: int, pos0: int,
+                            pos_stride: int, workspace=None, flags: int = 0, softmax_scale: float = 0.0,
+                            theta_base: float = 0.0, stream=None) -> None:
+    """loma_compress_step with memory row j's query and key rotated inside the step by the id pos0 + j * pos_stride."""
+    B, H, cap, D = k_cache.shape
+    for x in (q_mem, k_mem, v_mem, k_cache, v_cache, o_mem):
+        if not x.is_contiguous():
+            raise ValueError("compress tensors must be contiguous")
+    if q_mem.shape[2] != t:
+        raise ValueError("q_mem must have t rows")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().loma_compress_step_rope(_ptr(q_mem), _ptr(k_mem), _ptr(v_mem), _ptr(k_cache), _ptr(v_cache), _ptr(o_mem),
+                                       _ptr(lse), B, H, D, cap, mem_len, c, t, c * t, int(pos0), int(pos_stride),
+                                       float(theta_base), _dtype_code(q_mem), float(softmax_scale), int(flags),
+                                       _ptr(workspace), ws_bytes, _stream(stream))
+    _check(rc, "loma_compress_step_rope")
 
 
 def loma_decode_attn_ragged(q, k_new, v_new, k_cache, v_cache, o, lse, cache_lens, max_cache_len: int, workspace=None,

@@ -31,13 +31,13 @@ template <>
 struct Io<float> {
     // dot of a D-float row in shared memory with a D-element global row
     template <int D>
-    static __device__ __forceinline__ float dot(const float* __restrict__ qs, const float* __restrict__ kp) {
+    static __device__ __forceinline__ float dot(const float* __restrict__ qs, const float* kp) {
         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
         const float4* k4 = reinterpret_cast<const float4*>(kp);
         const float4* q4 = reinterpret_cast<const float4*>(qs);
 #pragma unroll
         for (int i = 0; i < D / 4; ++i) {
-            const float4 kv = __ldg(k4 + i);
+            const float4 kv = k4[i];   // (plain loads: a key row may also sit in shared memory, see the fused rotary embedding)
             const float4 qv = q4[i];
             a0 = fmaf(qv.x, kv.x, a0);
             a1 = fmaf(qv.y, kv.y, a1);
@@ -49,7 +49,7 @@ struct Io<float> {
     template <int N>
     static __device__ __forceinline__ void load(const float* p, float (&x)[N]) {
 #pragma unroll
-        for (int i = 0; i < N; ++i) x[i] = __ldg(p + i);
+        for (int i = 0; i < N; ++i) x[i] = p[i];
     }
     template <int N>
     static __device__ __forceinline__ void store(float* p, const float (&x)[N]) {
@@ -62,13 +62,13 @@ template <>
 struct Io<__nv_bfloat16> {
     template <int D>
     static __device__ __forceinline__ float dot(const float* __restrict__ qs,
-                                                const __nv_bfloat16* __restrict__ kp) {
+                                                const __nv_bfloat16* kp) {
         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
         const uint4* k8 = reinterpret_cast<const uint4*>(kp);
         const float4* q4 = reinterpret_cast<const float4*>(qs);
 #pragma unroll
         for (int i = 0; i < D / 8; ++i) {
-            const uint4 kv = __ldg(k8 + i);
+            const uint4 kv = k8[i];
             const float4 qa = q4[2 * i], qb = q4[2 * i + 1];
             a0 = fmaf(qa.x, bf16lo(kv.x), a0);
             a1 = fmaf(qa.y, bf16hi(kv.x), a1);
@@ -87,7 +87,7 @@ struct Io<__nv_bfloat16> {
         const uint32_t* u = reinterpret_cast<const uint32_t*>(p);
 #pragma unroll
         for (int i = 0; i < N / 2; ++i) {
-            const uint32_t w = __ldg(u + i);
+            const uint32_t w = u[i];
             x[2 * i] = bf16lo(w);
             x[2 * i + 1] = bf16hi(w);
         }
@@ -251,13 +251,21 @@ struct DecodeMap {
     __device__ __forceinline__ const T* vptr(int vi) const { return vi < len ? vc + slot(vi) : vn; }
 };
 
+// to / from the storage type, round to nearest even
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
 template <typename T, int D>
 __global__ void __launch_bounds__(32)
 decode_generic_kernel(const T* __restrict__ q, const T* __restrict__ k_new, const T* __restrict__ v_new,
                       T* __restrict__ k_cache, T* __restrict__ v_cache, T* __restrict__ o,
                       float* __restrict__ lse, int cap, int cache_len_max, const int32_t* __restrict__ lens, int H,
-                      float scale, Paging pg) {
+                      float scale, Paging pg, RopeArgs rope) {
     __shared__ __align__(16) float q_sh[D];
+    __shared__ __align__(16) T kn_sh[D];       // the new key, rotated (fused rotary embedding only)
     const int bh = blockIdx.x, lane = threadIdx.x;
     const int cache_len = lens ? min(max(lens[bh / H], 0), cache_len_max) : cache_len_max;   // ragged batch
     T* kc = pg.table ? k_cache : k_cache + (int64_t)bh * cap * D;
@@ -269,12 +277,28 @@ decode_generic_kernel(const T* __restrict__ q, const T* __restrict__ k_new, cons
     map.kn = k_new ? k_new + (int64_t)bh * D : kc + new_off;
     map.vn = v_new ? v_new + (int64_t)bh * D : vc + new_off;
     stage_query<T, D>(q_sh, q + (int64_t)bh * D, lane);
+    if (rope.on) {
+        // Section 4.5: q and the new key rotated by the step's position id, here instead of in a pass of their own;
+        // the rotated key, rounded to the storage type, is what the step attends to and appends
+        for (int d = lane; d < D / 2; d += 32) {
+            float c, sn;
+            rope_cos_sin(rope.pos0, d, D, rope.log2_base, c, sn);
+            const float qa = q_sh[d], qb = q_sh[d + D / 2];
+            q_sh[d] = qa * c - qb * sn;
+            q_sh[d + D / 2] = qb * c + qa * sn;
+            const float ka = to_f32(map.kn[d]), kb = to_f32(map.kn[d + D / 2]);
+            kn_sh[d] = from_f32<T>(ka * c - kb * sn);
+            kn_sh[d + D / 2] = from_f32<T>(kb * c + ka * sn);
+        }
+        __syncwarp();
+        map.kn = kn_sh;
+    }
     attend_row<T, D>(q_sh, map, cache_len + 1, scale, o + (int64_t)bh * D, lse ? lse + bh : nullptr, lane);
     if (k_new) {      // append: the slot is read by nobody in this launch
         constexpr int DPL = D / 32;
 #pragma unroll
         for (int d = 0; d < DPL; ++d) {
-            kc[new_off + lane * DPL + d] = k_new[(int64_t)bh * D + lane * DPL + d];
+            kc[new_off + lane * DPL + d] = map.kn[lane * DPL + d];
             vc[new_off + lane * DPL + d] = v_new[(int64_t)bh * D + lane * DPL + d];
         }
     }
@@ -355,8 +379,9 @@ __global__ void __launch_bounds__(GENERIC_WARPS * 32)
 compress_generic_kernel(const T* __restrict__ q_mem, const T* __restrict__ k_mem,
                         const T* __restrict__ v_mem, T* __restrict__ k_cache, T* __restrict__ v_cache,
                         T* __restrict__ o_mem, float* __restrict__ lse, int cap, int mem_len, const int32_t* __restrict__ mem_lens,
-                        int H, int t, int tc, unsigned flags, float scale, Paging pg) {
+                        int H, int t, int tc, unsigned flags, float scale, Paging pg, RopeArgs rope) {
     __shared__ __align__(16) float q_sh[GENERIC_WARPS][D];
+    extern __shared__ __align__(16) uint8_t km_rot_raw[];   // t x D rotated memory keys (fused rotary embedding only)
     const int bh = blockIdx.x;
     if (mem_lens) {                          // ragged batch: own count of memory entries; negative = not compressing now
         const int own = mem_lens[bh / H];
@@ -372,8 +397,33 @@ compress_generic_kernel(const T* __restrict__ q_mem, const T* __restrict__ k_mem
     map.km = k_mem + (int64_t)bh * t * D; map.vm = v_mem + (int64_t)bh * t * D;
     map.n_cache = mem_len + tc - lo; map.D = D;
     map.pg = pg; map.b = bh / H; map.h = bh - map.b * H; map.H = H;
+    if (rope.on) {
+        // Section 4.5: memory row j is rotated by the id pos0 + j * stride; its key, rounded to the storage type,
+        // is what every memory query attends to and what goes into the cache
+        T* km_rot = reinterpret_cast<T*>(km_rot_raw);
+        for (int e = threadIdx.x; e < t * (D / 2); e += blockDim.x) {
+            const int j = e / (D / 2), d = e - j * (D / 2);
+            float c, sn;
+            rope_cos_sin(rope.pos0 + j * rope.stride, d, D, rope.log2_base, c, sn);
+            const float a = to_f32(map.km[(int64_t)j * D + d]), b = to_f32(map.km[(int64_t)j * D + d + D / 2]);
+            km_rot[j * D + d] = from_f32<T>(a * c - b * sn);
+            km_rot[j * D + d + D / 2] = from_f32<T>(b * c + a * sn);
+        }
+        __syncthreads();
+        map.km = km_rot;
+    }
     for (int j = warp; j < t; j += GENERIC_WARPS) {
         stage_query<T, D>(q_sh[warp], q_mem + ((int64_t)bh * t + j) * D, lane);
+        if (rope.on) {
+            for (int d = lane; d < D / 2; d += 32) {
+                float c, sn;
+                rope_cos_sin(rope.pos0 + j * rope.stride, d, D, rope.log2_base, c, sn);
+                const float a = q_sh[warp][d], b = q_sh[warp][d + D / 2];
+                q_sh[warp][d] = a * c - b * sn;
+                q_sh[warp][d + D / 2] = b * c + a * sn;
+            }
+            __syncwarp();
+        }
         attend_row<T, D>(q_sh[warp], map, map.n_cache + t, scale, o_mem + ((int64_t)bh * t + j) * D,
                          lse ? lse + (int64_t)bh * t + j : nullptr, lane);
         __syncwarp();
@@ -605,11 +655,11 @@ cudaError_t launch_masked_attn_bwd_generic(const void* q, const void* k, const v
 template <typename T, int D>
 static cudaError_t decode_generic_t(const void* q, const void* kn, const void* vn, void* kc, void* vc,
                                     void* o, float* lse, int BH, int cap, int cache_len, const int32_t* lens, int H,
-                                    float scale, const Paging& pg, cudaStream_t st) {
+                                    float scale, const Paging& pg, cudaStream_t st, const RopeArgs& rope) {
     decode_generic_kernel<T, D><<<BH, 32, 0, st>>>(static_cast<const T*>(q), static_cast<const T*>(kn),
                                                    static_cast<const T*>(vn), static_cast<T*>(kc),
                                                    static_cast<T*>(vc), static_cast<T*>(o), lse, cap,
-                                                   cache_len, lens, H, scale, pg);
+                                                   cache_len, lens, H, scale, pg, rope);
     count_launches(1);
     return cudaGetLastError();
 }
@@ -617,27 +667,34 @@ static cudaError_t decode_generic_t(const void* q, const void* kn, const void* v
 cudaError_t launch_decode_generic(const void* q, const void* k_new, const void* v_new, void* k_cache,
                                   void* v_cache, void* o, float* lse, int B, int H, int D, int cap,
                                   int cache_len, const int32_t* lens, loma_dtype dt, float scale, const Paging& pg,
-                                  cudaStream_t st) {
+                                  cudaStream_t st, const RopeArgs& rope) {
     const int BH = B * H;
     if (dt == LOMA_F32) {
         return D == 64 ? decode_generic_t<float, 64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
-                                                     cache_len, lens, H, scale, pg, st)
+                                                     cache_len, lens, H, scale, pg, st, rope)
                        : decode_generic_t<float, 128>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
-                                                      cache_len, lens, H, scale, pg, st);
+                                                      cache_len, lens, H, scale, pg, st, rope);
     }
     return D == 64 ? decode_generic_t<__nv_bfloat16, 64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
-                                                         cache_len, lens, H, scale, pg, st)
+                                                         cache_len, lens, H, scale, pg, st, rope)
                    : decode_generic_t<__nv_bfloat16, 128>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap,
-                                                          cache_len, lens, H, scale, pg, st);
+                                                          cache_len, lens, H, scale, pg, st, rope);
 }
 
 template <typename T, int D>
 static cudaError_t compress_generic_t(const void* qm, const void* km, const void* vm, void* kc, void* vc,
                                       void* om, float* lse, int BH, int cap, int mem_len, const int32_t* mem_lens, int H, int t,
-                                      int tc, unsigned flags, float scale, const Paging& pg, cudaStream_t st) {
-    compress_generic_kernel<T, D><<<BH, GENERIC_WARPS * 32, 0, st>>>(
+                                      int tc, unsigned flags, float scale, const Paging& pg, cudaStream_t st,
+                                      const RopeArgs& rope) {
+    const size_t dyn = rope.on ? (size_t)t * D * sizeof(T) : 0;
+    if (dyn > 48 * 1024) {
+        if (dyn > 200 * 1024) return cudaErrorNotSupported;
+        const cudaError_t ea = cudaFuncSetAttribute(compress_generic_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+        if (ea != cudaSuccess) return ea;
+    }
+    compress_generic_kernel<T, D><<<BH, GENERIC_WARPS * 32, dyn, st>>>(
         static_cast<const T*>(qm), static_cast<const T*>(km), static_cast<const T*>(vm), static_cast<T*>(kc),
-        static_cast<T*>(vc), static_cast<T*>(om), lse, cap, mem_len, mem_lens, H, t, tc, flags, scale, pg);
+        static_cast<T*>(vc), static_cast<T*>(om), lse, cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, rope);
     count_launches(1);
     return cudaGetLastError();
 }
@@ -645,18 +702,18 @@ static cudaError_t compress_generic_t(const void* qm, const void* km, const void
 cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache,
                                     void* v_cache, void* o_mem, float* lse, int B, int H, int D, int cap,
                                     int mem_len, const int32_t* mem_lens, int c, int t, loma_dtype dt, float scale,
-                                    unsigned flags, const Paging& pg, cudaStream_t st) {
+                                    unsigned flags, const Paging& pg, cudaStream_t st, const RopeArgs& rope) {
     const int BH = B * H, tc = c * t;
     if (dt == LOMA_F32) {
         return D == 64 ? compress_generic_t<float, 64>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH,
-                                                       cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st)
+                                                       cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st, rope)
                        : compress_generic_t<float, 128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH,
-                                                        cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st);
+                                                        cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st, rope);
     }
     return D == 64 ? compress_generic_t<__nv_bfloat16, 64>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse,
-                                                           BH, cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st)
+                                                           BH, cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st, rope)
                    : compress_generic_t<__nv_bfloat16, 128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse,
-                                                            BH, cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st);
+                                                            BH, cap, mem_len, mem_lens, H, t, tc, flags, scale, pg, st, rope);
 }
 
 template <typename T, int D>

@@ -90,7 +90,8 @@ struct CmpSmem {
     static constexpr int ROWB = D * 2 + 16;                  // padded row: conflict-free ldmatrix
     static constexpr int STAGE = 2 * CMP_CHUNK * ROWB;       // K then V
     static constexpr int Q_OFF = 2 * STAGE;
-    static constexpr int TOTAL = Q_OFF + 16 * ROWB;
+    static constexpr int ROPE_OFF = Q_OFF + 16 * ROWB;       // cos/sin of 16 rows x D/2 feature pairs (fused rotary embedding)
+    static constexpr int TOTAL = ROPE_OFF + 16 * (D / 2) * 8;
     static constexpr int MERGE_BYTES = CMP_WARPS * 16 * (D + 2) * 4;   // reuses the stages
     static_assert(MERGE_BYTES <= 2 * STAGE, "merge buffer must fit in the stage buffers");
 };
@@ -101,7 +102,7 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
                     const __nv_bfloat16* __restrict__ v_mem, __nv_bfloat16* __restrict__ k_cache,
                     __nv_bfloat16* __restrict__ v_cache, __nv_bfloat16* __restrict__ o_mem, float* __restrict__ lse,
                     float* __restrict__ ws, int BH, int cap, int mem_len_all, const int32_t* __restrict__ mem_lens, int H,
-                    int t, int tc, int nprior, int prior_len, int mtiles, float scale_log2, Paging pg) {
+                    int t, int tc, int nprior, int prior_len, int mtiles, float scale_log2, Paging pg, RopeArgs rope) {
     using SM = CmpSmem<D>;
     constexpr int ROWB = SM::ROWB;
     constexpr int VPR = D / 8;                 // 16-byte vectors per row
@@ -167,6 +168,30 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
         if (q0 + r < t) val = __ldg(reinterpret_cast<const uint4*>(q_mem + ((int64_t)bh * t + q0 + r) * D) + cv);
         *reinterpret_cast<uint4*>(smem + SM::Q_OFF + r * ROWB + cv * 16) = val;
     }
+    // Fused rotary embedding (Section 4.5): memory row j is rotated by the id pos0 + j * stride -- its query here,
+    // its key where it is staged below and where it is written into the cache.  cos/sin per (row, feature pair)
+    // are tabulated once per CTA.
+    float2* rope_tab = reinterpret_cast<float2*>(smem + SM::ROPE_OFF);
+    auto rotate_row_in_smem = [&](uint8_t* row, int j16, int d) {   // features d and d + D/2 of a staged bf16 row
+        __nv_bfloat16* x = reinterpret_cast<__nv_bfloat16*>(row);
+        const float2 cs = rope_tab[j16 * (D / 2) + d];
+        const float a = __bfloat162float(x[d]), b = __bfloat162float(x[d + D / 2]);
+        x[d] = __float2bfloat16_rn(a * cs.x - b * cs.y);
+        x[d + D / 2] = __float2bfloat16_rn(b * cs.x + a * cs.y);
+    };
+    if (rope.on) {
+        for (int e = threadIdx.x; e < 16 * (D / 2); e += CMP_WARPS * 32) {
+            const int r = e / (D / 2), d = e - r * (D / 2);
+            float c, sn;
+            rope_cos_sin(rope.pos0 + (q0 + r) * rope.stride, d, D, rope.log2_base, c, sn);
+            rope_tab[e] = make_float2(c, sn);
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < 16 * (D / 2); e += CMP_WARPS * 32) {
+            const int r = e / (D / 2), d = e - r * (D / 2);
+            if (q0 + r < t) rotate_row_in_smem(smem + SM::Q_OFF + r * ROWB, r, d);
+        }
+    }
     __syncthreads();
     uint32_t qa[D / 16][4];
     {
@@ -186,6 +211,16 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
         cp_async_commit();
         cp_async_wait<1>();
         __syncthreads();
+        if (rope.on && is_tail && (ci + 1) * CMP_CHUNK > n_cache_rows) {
+            // the memory rows' own keys (rows n_cache_rows .. nkeys - 1 of the range) are rotated where they were staged
+            uint8_t* kst_gen = smem + (ci & 1) * SM::STAGE;
+            for (int e = threadIdx.x; e < CMP_CHUNK * (D / 2); e += CMP_WARPS * 32) {
+                const int r = e / (D / 2), d = e - r * (D / 2);
+                const int j = ci * CMP_CHUNK + r - n_cache_rows;     // memory row
+                if (j >= 0 && j < t) rotate_row_in_smem(kst_gen + r * ROWB, j - q0, d);
+            }
+            __syncthreads();
+        }
         const int kb = ci * CMP_CHUNK + warp * 16;        // this warp's 16 keys
         if (kb < nkeys) {
             const uint32_t kst = sbase + (ci & 1) * SM::STAGE + warp * 16 * ROWB;
@@ -327,8 +362,18 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
         for (int e = threadIdx.x; e < t * VPR; e += CMP_WARPS * 32) {
             const int r = e / VPR, cv = e - r * VPR;
             const int64_t off = cache_row(mem_len + r) + cv * 8;
-            *reinterpret_cast<uint4*>(k_cache + off) = __ldg(ksrc + e);
+            if (!rope.on) *reinterpret_cast<uint4*>(k_cache + off) = __ldg(ksrc + e);
             *reinterpret_cast<uint4*>(v_cache + off) = __ldg(vsrc + e);
+        }
+        if (rope.on) {   // the keys go into the cache rotated (the same arithmetic as for the staged copies)
+            for (int e = threadIdx.x; e < t * (D / 2); e += CMP_WARPS * 32) {
+                const int r = e / (D / 2), d = e - r * (D / 2);
+                const float2 cs = rope_tab[r * (D / 2) + d];
+                const float a = __bfloat162float(km[(int64_t)r * D + d]), b = __bfloat162float(km[(int64_t)r * D + d + D / 2]);
+                const int64_t off = cache_row(mem_len + r);
+                k_cache[off + d] = __float2bfloat16_rn(a * cs.x - b * cs.y);
+                k_cache[off + d + D / 2] = __float2bfloat16_rn(b * cs.x + a * cs.y);
+            }
         }
     }
 }
@@ -389,7 +434,8 @@ __global__ void compaction_kernel(const __nv_bfloat16* __restrict__ k_mem, const
 template <int D>
 static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* vm, void* kc, void* vc, void* om,
                                    float* lse, int BH, int cap, int mem_len, const int32_t* mem_lens, int H, int t, int tc,
-                                   unsigned flags, float scale, void* ws, const Paging& pg, cudaStream_t st) {
+                                   unsigned flags, float scale, void* ws, const Paging& pg, cudaStream_t st,
+                                   const RopeArgs& rope) {
     const int nprior = compress_num_prior(BH, mem_len, flags);
     int prior_len = 0;
     if (nprior > 0) prior_len = ((mem_len + nprior - 1) / nprior + 15) / 16 * 16;
@@ -409,7 +455,7 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
         static_cast<const __nv_bfloat16*>(qm), static_cast<const __nv_bfloat16*>(km),
         static_cast<const __nv_bfloat16*>(vm), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
         static_cast<__nv_bfloat16*>(om), lse, static_cast<float*>(ws), BH, cap, mem_len, mem_lens, H, t, tc, nprior,
-        prior_len, mtiles, scale * 1.4426950408889634f, pg);
+        prior_len, mtiles, scale * 1.4426950408889634f, pg, rope);
     count_launches(1);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -430,16 +476,17 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
     return e;
 }
 
-// t <= 128; the caller falls back to the CUDA-core kernel otherwise.
+// t <= 128 (with the fused rotary embedding: t <= 16); the caller falls back to the CUDA-core kernel otherwise.
 cudaError_t launch_compress_bf16(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
                                  void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len,
                                  const int32_t* mem_lens, int c, int t, unsigned flags, float scale, void* ws,
-                                 const Paging& pg, cudaStream_t st) {
+                                 const Paging& pg, cudaStream_t st, const RopeArgs& rope) {
     const int BH = B * H, tc = c * t;
+    if (rope.on && t > 16) return cudaErrorNotSupported;
     return D == 64 ? compress_bf16_t<64>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH, cap, mem_len, mem_lens, H, t,
-                                         tc, flags, scale, ws, pg, st)
+                                         tc, flags, scale, ws, pg, st, rope)
                    : compress_bf16_t<128>(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, BH, cap, mem_len, mem_lens, H, t,
-                                          tc, flags, scale, ws, pg, st);
+                                          tc, flags, scale, ws, pg, st, rope);
 }
 
 }  // namespace loma

@@ -83,12 +83,16 @@ decode_splitkv_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
                       const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ k_cache,
                       __nv_bfloat16* __restrict__ v_cache, __nv_bfloat16* __restrict__ o,
                       float* __restrict__ lse, float* __restrict__ ws, int BH, int cap, int cache_len_max,
-                      const int32_t* __restrict__ lens, int H, int splits, int split_len, float scale_log2, Paging pg) {
+                      const int32_t* __restrict__ lens, int H, int splits, int split_len, float scale_log2, Paging pg,
+                      RopeArgs rope) {
     constexpr int LPK = D / 8;           // lanes per row
     constexpr int KPL = 32 / LPK;        // rows per warp load
     constexpr int BK = DEC_NL * KPL;     // rows per warp iteration
     __shared__ float sm_m[DEC_WARPS], sm_l[DEC_WARPS];
     __shared__ __align__(16) float sm_o[DEC_WARPS][D];
+    // fused rotary embedding (Section 4.5): cos/sin of the step's position per feature pair, and the rotated new key
+    __shared__ float sm_cs[D / 2], sm_sn[D / 2];
+    __shared__ __align__(16) __nv_bfloat16 sm_kn[D];
 
     const int bh = blockIdx.x / splits, split = blockIdx.x - bh * splits;
     // ragged batch: every sequence has its own length (clamped to the bound the launch was sized for);
@@ -117,11 +121,35 @@ decode_splitkv_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
     float qf[8];
     {
         const uint4 qv = __ldg(reinterpret_cast<const uint4*>(q + (int64_t)bh * D) + li);
-        qf[0] = bf16lo(qv.x) * scale_log2; qf[1] = bf16hi(qv.x) * scale_log2;
-        qf[2] = bf16lo(qv.y) * scale_log2; qf[3] = bf16hi(qv.y) * scale_log2;
-        qf[4] = bf16lo(qv.z) * scale_log2; qf[5] = bf16hi(qv.z) * scale_log2;
-        qf[6] = bf16lo(qv.w) * scale_log2; qf[7] = bf16hi(qv.w) * scale_log2;
+        qf[0] = bf16lo(qv.x); qf[1] = bf16hi(qv.x); qf[2] = bf16lo(qv.y); qf[3] = bf16hi(qv.y);
+        qf[4] = bf16lo(qv.z); qf[5] = bf16hi(qv.z); qf[6] = bf16lo(qv.w); qf[7] = bf16hi(qv.w);
     }
+    // does this CTA read the new key (index cache_len) or write it to the cache?
+    const bool needs_new_key = (k_begin <= cache_len && cache_len < k_end) || split == splits - 1;
+    if (rope.on) {
+        // q and the new key are rotated here, in registers / shared memory, by the step's position id: no
+        // separate pass over them.  The rotated key, rounded to bf16, is what the step attends to and appends.
+        if (threadIdx.x < D / 2) rope_cos_sin(rope.pos0, threadIdx.x, D, rope.log2_base, sm_cs[threadIdx.x], sm_sn[threadIdx.x]);
+        __syncthreads();
+        if (needs_new_key && threadIdx.x < D / 2) {
+            const __nv_bfloat16* kp = reinterpret_cast<const __nv_bfloat16*>(kn);
+            const float a = __bfloat162float(kp[threadIdx.x]), b = __bfloat162float(kp[threadIdx.x + D / 2]);
+            const float c = sm_cs[threadIdx.x], sn = sm_sn[threadIdx.x];
+            sm_kn[threadIdx.x] = __float2bfloat16_rn(a * c - b * sn);
+            sm_kn[threadIdx.x + D / 2] = __float2bfloat16_rn(b * c + a * sn);
+        }
+        const bool second = li >= LPK / 2;                 // this lane holds features of the second half
+        const int dh = (li % (LPK / 2)) * 8;               // its first feature pair
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const float other = __shfl_xor_sync(0xffffffffu, qf[e], LPK / 2);
+            const float c = sm_cs[dh + e], sn = sm_sn[dh + e];
+            qf[e] = second ? qf[e] * c + other * sn : qf[e] * c - other * sn;
+        }
+        __syncthreads();                                   // sm_kn is read below
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) qf[e] *= scale_log2;
 
     float m = -INFINITY, l = 0.f;
     float acc[8];
@@ -137,7 +165,8 @@ decode_splitkv_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
             valid[i] = j < k_end;
             const int jc = min(j, cache_len);                  // stay inside [0, cache_len]
             const uint4* kp = (jc < cache_len) ? kc + row_off(jc) : kn;
-            kr[i] = ld_stream(kp + li);
+            if (rope.on && jc >= cache_len) kr[i] = *(reinterpret_cast<const uint4*>(sm_kn) + li);   // the rotated new key
+            else kr[i] = ld_stream(kp + li);
         }
 #pragma unroll
         for (int i = 0; i < DEC_NL; ++i) {
@@ -218,7 +247,7 @@ decode_splitkv_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
     if (k_new && split == splits - 1 && warp == 0 && lane < LPK) {
         uint4* kd = const_cast<uint4*>(kc) + new_off;
         uint4* vd = const_cast<uint4*>(vc) + new_off;
-        kd[lane] = __ldg(kn + lane);
+        kd[lane] = rope.on ? *(reinterpret_cast<const uint4*>(sm_kn) + lane) : __ldg(kn + lane);
         vd[lane] = __ldg(vn + lane);
     }
 }
@@ -248,7 +277,7 @@ decode_merge_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ o,
 template <int D>
 static cudaError_t decode_bf16_t(const void* q, const void* kn, const void* vn, void* kc, void* vc, void* o,
                                  float* lse, int BH, int cap, int cache_len, const int32_t* lens, int H, float scale,
-                                 void* ws, const Paging& pg, cudaStream_t st) {
+                                 void* ws, const Paging& pg, cudaStream_t st, const RopeArgs& rope) {
     const int total = cache_len + 1;
     const int splits = decode_num_splits(BH, total);
     int split_len = (total + splits - 1) / splits;
@@ -259,13 +288,13 @@ static cudaError_t decode_bf16_t(const void* q, const void* kn, const void* vn, 
             static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(kn),
             static_cast<const __nv_bfloat16*>(vn), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
             static_cast<__nv_bfloat16*>(o), lse, static_cast<float*>(ws), BH, cap, cache_len, lens, H, splits, split_len,
-            scale_log2, pg);
+            scale_log2, pg, rope);
     else
         decode_splitkv_kernel<D, false><<<BH * splits, DEC_WARPS * 32, 0, st>>>(
             static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(kn),
             static_cast<const __nv_bfloat16*>(vn), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
             static_cast<__nv_bfloat16*>(o), lse, static_cast<float*>(ws), BH, cap, cache_len, lens, H, splits, split_len,
-            scale_log2, pg);
+            scale_log2, pg, rope);
     count_launches(1);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess || splits == 1) return e;
@@ -277,11 +306,12 @@ static cudaError_t decode_bf16_t(const void* q, const void* kn, const void* vn, 
 
 cudaError_t launch_decode_bf16(const void* q, const void* k_new, const void* v_new, void* k_cache,
                                void* v_cache, void* o, float* lse, int B, int H, int D, int cap, int cache_len,
-                               const int32_t* lens, float scale, void* ws, const Paging& pg, cudaStream_t st) {
+                               const int32_t* lens, float scale, void* ws, const Paging& pg, cudaStream_t st,
+                               const RopeArgs& rope) {
     const int BH = B * H;
-    return D == 64 ? decode_bf16_t<64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap, cache_len, lens, H, scale, ws, pg, st)
+    return D == 64 ? decode_bf16_t<64>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap, cache_len, lens, H, scale, ws, pg, st, rope)
                    : decode_bf16_t<128>(q, k_new, v_new, k_cache, v_cache, o, lse, BH, cap, cache_len, lens, H, scale, ws,
-                                        pg, st);
+                                        pg, st, rope);
 }
 
 // ---------------------------------------------------------------------------

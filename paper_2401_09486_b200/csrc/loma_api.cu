@@ -303,10 +303,10 @@ size_t loma_decode_workspace_bytes(int B, int H, int D, int cache_len) {
     return decode_workspace_bytes(B * H, D, cache_len + 1);
 }
 
-int loma_decode_attn(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
-                     float* lse, int B, int H, int D, int cap, int cache_len, loma_dtype dtype,
-                     float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes,
-                     void* stream) {
+static int decode_attn_impl(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
+                            float* lse, int B, int H, int D, int cap, int cache_len, loma_dtype dtype,
+                            float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes,
+                            void* stream, const RopeArgs& rope) {
     if (B < 0 || H < 0 || cap < 0 || cache_len < 0) return LOMA_ERR_INVALID_ARG;
     if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
     if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
@@ -327,11 +327,32 @@ int loma_decode_attn(const void* q, const void* k_new, const void* v_new, void* 
     cudaError_t e;
     if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC))
         e = launch_decode_bf16(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, nullptr, scale,
-                               workspace, Paging{}, st);
+                               workspace, Paging{}, st, rope);
     else
         e = launch_decode_generic(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, nullptr, dtype,
-                                  scale, Paging{}, st);
+                                  scale, Paging{}, st, rope);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
+int loma_decode_attn(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
+                     float* lse, int B, int H, int D, int cap, int cache_len, loma_dtype dtype,
+                     float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes,
+                     void* stream) {
+    return decode_attn_impl(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, dtype, softmax_scale, flags,
+                            workspace, workspace_bytes, stream, RopeArgs{});
+}
+
+int loma_decode_attn_rope(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
+                          float* lse, int B, int H, int D, int cap, int cache_len, int pos, float theta_base,
+                          loma_dtype dtype, float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes,
+                          void* stream) {
+    if (pos < 0) return LOMA_ERR_INVALID_ARG;
+    if (B > 0 && H > 0 && (!k_new || !v_new)) return LOMA_ERR_INVALID_ARG;   // the key to rotate has to be given
+    RopeArgs rope;
+    rope.on = 1; rope.pos0 = pos; rope.stride = 0;
+    rope.log2_base = log2(theta_base > 0.f ? (double)theta_base : 10000.0);
+    return decode_attn_impl(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_len, dtype, softmax_scale, flags,
+                            workspace, workspace_bytes, stream, rope);
 }
 
 int loma_prefill_attn(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
@@ -518,10 +539,10 @@ size_t loma_compress_workspace_bytes(int B, int H, int D, int t, int mem_len, un
     return compress_workspace_bytes(B * H, D, t, mem_len, flags);
 }
 
-int loma_compress_step(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
-                       void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len, int c, int t, int tc,
-                       loma_dtype dtype, float softmax_scale, unsigned flags, void* workspace,
-                       size_t workspace_bytes, void* stream) {
+static int compress_step_impl(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
+                              void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len, int c, int t, int tc,
+                              loma_dtype dtype, float softmax_scale, unsigned flags, void* workspace,
+                              size_t workspace_bytes, void* stream, const RopeArgs& rope) {
     if (B < 0 || H < 0 || cap < 0 || mem_len < 0 || c < 1 || t < 1) return LOMA_ERR_INVALID_ARG;
     if ((int64_t)c * t != (int64_t)tc) return LOMA_ERR_INVALID_ARG;
     if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
@@ -539,14 +560,36 @@ int loma_compress_step(const void* q_mem, const void* k_mem, const void* v_mem, 
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((int64_t)B * H * 256 > INT_MAX) return LOMA_ERR_INVALID_ARG;
-    cudaError_t e;
-    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC) && t <= 128)
+    cudaError_t e = cudaErrorNotSupported;
+    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC) && t <= (rope.on ? 16 : 128))
         e = launch_compress_bf16(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, mem_len, nullptr, c, t,
-                                 flags, scale, workspace, Paging{}, st);
-    else
+                                 flags, scale, workspace, Paging{}, st, rope);
+    if (e == cudaErrorNotSupported)
         e = launch_compress_generic(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, mem_len, nullptr, c,
-                                    t, dtype, scale, flags, Paging{}, st);
+                                    t, dtype, scale, flags, Paging{}, st, rope);
+    if (e == cudaErrorNotSupported) return LOMA_ERR_UNSUPPORTED;
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
+int loma_compress_step(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
+                       void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len, int c, int t, int tc,
+                       loma_dtype dtype, float softmax_scale, unsigned flags, void* workspace,
+                       size_t workspace_bytes, void* stream) {
+    return compress_step_impl(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, mem_len, c, t, tc, dtype,
+                              softmax_scale, flags, workspace, workspace_bytes, stream, RopeArgs{});
+}
+
+int loma_compress_step_rope(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
+                            void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len, int c, int t, int tc,
+                            int pos0, int pos_stride, float theta_base, loma_dtype dtype, float softmax_scale,
+                            unsigned flags, void* workspace, size_t workspace_bytes, void* stream) {
+    if (pos0 < 0 || pos_stride < 0) return LOMA_ERR_INVALID_ARG;
+    if (t > 0 && (int64_t)pos0 + (int64_t)(t - 1) * pos_stride > INT_MAX) return LOMA_ERR_INVALID_ARG;
+    RopeArgs rope;
+    rope.on = 1; rope.pos0 = pos0; rope.stride = pos_stride;
+    rope.log2_base = log2(theta_base > 0.f ? (double)theta_base : 10000.0);
+    return compress_step_impl(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, mem_len, c, t, tc, dtype,
+                              softmax_scale, flags, workspace, workspace_bytes, stream, rope);
 }
 
 int loma_compress_step_ragged(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,

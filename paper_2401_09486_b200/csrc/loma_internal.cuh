@@ -65,6 +65,27 @@ struct Paging {
     int max_pages = 0, log2_ps = 0, n_pages = 0;
 };
 
+// ---- rotary embedding fused into the generation steps (Section 4.5; Appendix A position ids) -------------
+// pos0 + j * stride is the position id of row j of the call (decode: one row; compress: the t memory rows,
+// Eq. 14 with pos0 = y*tc + c - 1, stride = c, or the contiguous ids with pos0 = mem_len, stride = 1).
+struct RopeArgs {
+    int on = 0;
+    int pos0 = 0, stride = 0;
+    double log2_base = 0.0;   // log2 of the base (10000 by default)
+};
+
+#ifdef __CUDACC__
+// cos and sin of the rotation angle of feature pair (d, d + D/2) at position pos: pos * base^(-2d/D).  The angle
+// is formed and reduced to [-pi, pi] in double (ids reach tens of thousands, where a float angle has lost the
+// digits the fp32 bar needs); cos/sin of the reduced angle in float are good to ~2e-7.
+__device__ __forceinline__ void rope_cos_sin(int pos, int d, int D, double log2_base, float& c, float& s) {
+    const double theta = exp2(-log2_base * (2.0 * d / D));
+    double a = (double)pos * theta;
+    a -= 6.283185307179586476925 * rint(a * 0.15915494309189533577);
+    sincosf((float)a, &s, &c);
+}
+#endif
+
 // ---- launchers (each defined in its own .cu) ------------------------------
 cudaError_t launch_layout_index(const Layout& L, int32_t* chunk, int32_t* zone, int32_t* offset,
                                 int32_t* src, int32_t* pos, cudaStream_t st);
@@ -118,14 +139,15 @@ cudaError_t launch_bounded_wait_selftest(cudaStream_t st);   // attn_tcgen05.cu
 cudaError_t launch_decode_generic(const void* q, const void* k_new, const void* v_new,
                                   void* k_cache, void* v_cache, void* o, float* lse,
                                   int B, int H, int D, int cap, int cache_len, const int32_t* lens,
-                                  loma_dtype dt, float scale, const Paging& pg, cudaStream_t st);
+                                  loma_dtype dt, float scale, const Paging& pg, cudaStream_t st,
+                                  const RopeArgs& rope = RopeArgs{});
 
 // bf16 split-KV decode (decode_splitkv.cu)
 size_t decode_workspace_bytes(int BH, int D, int total_keys);
 cudaError_t launch_decode_bf16(const void* q, const void* k_new, const void* v_new, void* k_cache,
                                void* v_cache, void* o, float* lse, int B, int H, int D, int cap, int cache_len,
                                const int32_t* lens, float scale, void* ws, const Paging& pg,
-                               cudaStream_t st);   // lens: per-sequence lengths or NULL
+                               cudaStream_t st, const RopeArgs& rope = RopeArgs{});   // lens: per-sequence lengths or NULL
 
 size_t decode_static_scratch_bytes();
 cudaError_t launch_decode_bf16_static(const void* q, const void* k_new, const void* v_new, void* k_cache,
@@ -137,12 +159,14 @@ size_t compress_workspace_bytes(int BH, int D, int t, int mem_len, unsigned flag
 cudaError_t launch_compress_bf16(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
                                  void* o_mem, float* lse, int B, int H, int D, int cap, int mem_len,
                                  const int32_t* mem_lens, int c, int t, unsigned flags, float scale, void* ws,
-                                 const Paging& pg, cudaStream_t st);   // mem_lens: per-sequence counts (default variant only) or NULL
+                                 const Paging& pg, cudaStream_t st,
+                                 const RopeArgs& rope = RopeArgs{});   // mem_lens: per-sequence counts (default variant only) or NULL
 
 cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const void* v_mem,
                                     void* k_cache, void* v_cache, void* o_mem, float* lse,
                                     int B, int H, int D, int cap, int mem_len, const int32_t* mem_lens, int c, int t,
-                                    loma_dtype dt, float scale, unsigned flags, const Paging& pg, cudaStream_t st);
+                                    loma_dtype dt, float scale, unsigned flags, const Paging& pg, cudaStream_t st,
+                                    const RopeArgs& rope = RopeArgs{});
 
 // rotary embedding of Q and K rows at the layout's position ids (rope.cu)
 cudaError_t launch_rope(void* q, void* k, int B, int H, int D, const Layout& L, int64_t sb, int64_t sh, int64_t ss,

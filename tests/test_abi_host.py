@@ -109,6 +109,29 @@ def test_masked_attn_fwd_validation_precedes_any_cuda_call(lib):
     assert _fwd(lib, B=0) == 0
 
 
+def test_rope_fused_steps_validation(lib):
+    def dec(q=0x1000, kn=0x2000, vn=0x3000, kc=0x4000, vc=0x5000, o=0x6000, B=1, H=1, D=128, cap=8, cache_len=3, pos=3, dt=1):
+        return lib.loma_decode_attn_rope(q, kn, vn, kc, vc, o, None, B, H, D, cap, cache_len, pos, 0.0, dt, 0.0, 0, None, 0, None)
+    assert dec(pos=-1) == INVALID
+    assert dec(kn=None, vn=None) == INVALID             # the key to rotate has to be given
+    assert dec(cache_len=8) == CAPACITY
+    assert dec(D=96) == UNSUPPORTED
+    assert dec(q=0x1004) == ALIGNMENT
+    assert dec(H=0) == 0
+
+    def cmp_(qm=0x1000, km=0x2000, vm=0x3000, kc=0x4000, vc=0x5000, om=0x6000, B=1, H=1, D=128, cap=96, mem_len=16, c=4, t=16,
+             tc=64, pos0=67, stride=4, dt=1):
+        return lib.loma_compress_step_rope(qm, km, vm, kc, vc, om, None, B, H, D, cap, mem_len, c, t, tc, pos0, stride, 0.0, dt,
+                                           0.0, 0, None, 0, None)
+    assert cmp_(pos0=-1) == INVALID
+    assert cmp_(stride=-2) == INVALID
+    assert cmp_(pos0=2**31 - 10, stride=4) == INVALID    # the last id would overflow
+    assert cmp_(tc=63) == INVALID
+    assert cmp_(cap=79) == CAPACITY
+    assert cmp_(km=None) == INVALID
+    assert cmp_(B=0) == 0
+
+
 def test_prefill_attn_validation(lib):
     def call(q=0x1000, kn=0x2000, vn=0x3000, kc=0x4000, vc=0x5000, o=0x6000, lse=None, B=1, H=1, D=128, l=4, cap=16,
              cache_len=3, dt=1, flags=0):

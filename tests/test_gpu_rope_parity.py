@@ -125,3 +125,118 @@ def test_differentiable_rope_then_attention_against_torch_autograd():
     torch.cuda.synchronize()
     for g, g2 in ((q.grad, q2.grad), (k.grad, k2.grad), (v.grad, v2.grad)):
         assert float((g.double() - g2).abs().max()) <= 2e-5 * max(1.0, float(g2.abs().max()))
+
+
+# ------------------------------------------------- rotation fused into the generation steps
+
+def _round_to(x64, dtype):
+    """fp64 array -> rounded once to the storage type -> fp64."""
+    return torch.from_numpy(x64).to(dtype).to(torch.float64).numpy()
+
+
+def _ulp_close(got, want64, dtype):
+    """The appended keys are rotated in fp32 on the device and rounded to the storage type: equal to the fp64
+    rotation rounded the same way, up to one unit in the last place where a rounding tie falls differently."""
+    g = npf(got)
+    if dtype == torch.float32:
+        assert np.abs(g - want64).max() <= 2e-6          # fp32 arithmetic on values of size about one
+    else:
+        tol = 2.0 ** -7 * np.maximum(np.abs(want64), 2.0 ** -6)
+        assert (np.abs(g - _round_to(want64, dtype)) <= tol).all()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, L.LOMA_FLAG_FORCE_GENERIC])
+@pytest.mark.parametrize("B,H,D,cap,cache_len,pos", [(1, 1, 64, 4, 0, 0), (2, 3, 128, 40, 17, 5), (2, 2, 128, 700, 613, 2500),
+                                                      (1, 4, 64, 9000, 8300, 32767), (3, 2, 128, 5000, 4999, 20001)])
+def test_decode_with_fused_rotation_matches_oracle(B, H, D, cap, cache_len, pos, flags, dtype):
+    kc = synthetic.normal_tensor((B, H, cap, D), 71, 1.0, dtype)
+    vc = synthetic.normal_tensor((B, H, cap, D), 72, 1.0, dtype)
+    q, kn, vn = synthetic.qkv(B, H, 1, D, seed=73, std=1.0, dtype=dtype)
+    q_rot = oracle.rope_rotate(npf(q), [pos])
+    k_rot = oracle.rope_rotate(npf(kn), [pos])
+    want_o, want_lse, _, _ = oracle.decode_attn(q_rot, _round_to(k_rot, dtype), npf(vn), npf(kc), npf(vc), cache_len)
+    kcd, vcd = kc.to(DEV), vc.to(DEV)
+    o = torch.full((B, H, 1, D), float("nan"), dtype=dtype, device=DEV)
+    lse = torch.full((B, H), float("nan"), dtype=torch.float32, device=DEV)
+    ws = torch.empty(max(16, L.loma_decode_workspace_bytes(B, H, D, cache_len)), dtype=torch.uint8, device=DEV)
+    L.loma_decode_attn_rope(q.to(DEV), kn.to(DEV), vn.to(DEV), kcd, vcd, o, lse, cache_len, pos, ws, flags)
+    torch.cuda.synchronize()
+    check(o, want_o, dtype)
+    assert np.abs(npf(lse) - want_lse.reshape(B, H)).max() <= (1e-5 if dtype == torch.float32 else 2e-2)
+    # the cache: the rotated key and the value appended at cache_len, nothing else touched
+    keep = [j for j in range(cap) if j != cache_len]
+    assert torch.equal(kcd[:, :, keep].cpu(), kc[:, :, keep]) and torch.equal(vcd[:, :, keep].cpu(), vc[:, :, keep])
+    assert torch.equal(vcd[:, :, cache_len].cpu(), vn[:, :, 0])
+    _ulp_close(kcd[:, :, cache_len], k_rot[:, :, 0], dtype)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, L.LOMA_FLAG_MEM_SEES_PRIOR_MEM, L.LOMA_FLAG_FORCE_GENERIC])
+@pytest.mark.parametrize("B,H,D,c,t,mem_len,pos0,stride", [(1, 1, 64, 4, 4, 0, 3, 4), (2, 2, 128, 4, 16, 48, 3 * 64 + 3, 4),
+                                                            (2, 3, 128, 8, 16, 1024, 64 * 128 + 7, 8), (1, 2, 128, 4, 16, 512, 512, 1),
+                                                            (1, 2, 64, 2, 40, 80, 2 * 80 + 1, 2)])
+def test_compress_with_fused_rotation_matches_oracle(B, H, D, c, t, mem_len, pos0, stride, flags, dtype):
+    tc = c * t
+    cap = mem_len + tc + 3
+    kc = synthetic.normal_tensor((B, H, cap, D), 81, 1.0, dtype)
+    vc = synthetic.normal_tensor((B, H, cap, D), 82, 1.0, dtype)
+    qm, km, vm = synthetic.qkv(B, H, t, D, seed=83, std=1.0, dtype=dtype)
+    pos = [pos0 + j * stride for j in range(t)]
+    q_rot = oracle.rope_rotate(npf(qm), pos)
+    k_rot = oracle.rope_rotate(npf(km), pos)
+    prior = flags & L.LOMA_FLAG_MEM_SEES_PRIOR_MEM
+    want_o, _, want_k, want_v = oracle.compress_step(q_rot, _round_to(k_rot, dtype), npf(vm), npf(kc), npf(vc), mem_len, c, t, prior)
+    kcd, vcd = kc.to(DEV), vc.to(DEV)
+    om = torch.full((B, H, t, D), float("nan"), dtype=dtype, device=DEV)
+    ws = torch.empty(max(16, L.loma_compress_workspace_bytes(B, H, D, t, mem_len, prior)), dtype=torch.uint8, device=DEV)
+    L.loma_compress_step_rope(qm.to(DEV), km.to(DEV), vm.to(DEV), kcd, vcd, om, None, mem_len, c, t, pos0, stride, ws, flags)
+    torch.cuda.synchronize()
+    check(om, want_o, dtype)
+    assert torch.equal(kcd[:, :, :mem_len].cpu(), kc[:, :, :mem_len]) and torch.equal(vcd[:, :, :mem_len].cpu(), vc[:, :, :mem_len])
+    assert torch.equal(vcd[:, :, mem_len:mem_len + t].cpu(), vm)
+    _ulp_close(kcd[:, :, mem_len:mem_len + t], k_rot, dtype)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("ptype", [0, 1])
+def test_generation_with_fused_rotation_equals_rotated_one_shot_forward(ptype, dtype):
+    """Decode every reading token at its id and compress every chunk at the memory ids (Eq. 14, or the
+    generator's contiguous ids) with the rotation fused into the steps: every reading and memory row equals the
+    one-shot forward over Q and K rotated at the layout's position ids."""
+    B, H, D, n, c, t, tail = 1, 2, 128, 3, 4, 16, 9
+    tc, s = c * t, oracle.chunk_len(c, t)
+    S = oracle.seq_len(n, c, t, tail)
+    q, k, v = synthetic.qkv(B, H, S, D, seed=91, std=1.0, dtype=dtype)
+    wq, wk = oracle.rope_apply(npf(q), npf(k), n, c, t, tail, 0, 10000.0, "contiguous" if ptype else "intermittent")
+    want_o, _ = oracle.masked_attn_fwd(wq, wk, npf(v), n, c, t, tail)
+    pos = oracle.position_ids(n, c, t, tail, 0, "contiguous" if ptype else "intermittent")
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    cap = n * t + tc + 4
+    kc = torch.zeros((B, H, cap, D), dtype=dtype, device=DEV)
+    vc = torch.zeros_like(kc)
+    got = torch.full_like(qd, float("nan"))
+    ws = torch.empty(max(16, L.loma_decode_workspace_bytes(B, H, D, cap)), dtype=torch.uint8, device=DEV)
+    length = 0
+    rows = lambda a, b: slice(a, b)
+    for y in range(n + 1):
+        nread = tc if y < n else tail
+        for o_ in range(nread):
+            i = y * s + o_
+            o1 = torch.empty((B, H, 1, D), dtype=dtype, device=DEV)
+            L.loma_decode_attn_rope(qd[:, :, i:i + 1].contiguous(), kd[:, :, i:i + 1].contiguous(), vd[:, :, i:i + 1].contiguous(),
+                                    kc, vc, o1, None, length, int(pos[i]), ws)
+            got[:, :, i] = o1[:, :, 0]
+            length += 1
+        if y < n:
+            m0 = y * s + tc
+            om = torch.empty((B, H, t, D), dtype=dtype, device=DEV)
+            p0 = int(pos[m0]); st = int(pos[m0 + 1] - pos[m0])
+            L.loma_compress_step_rope(qd[:, :, m0:m0 + t].contiguous(), kd[:, :, m0:m0 + t].contiguous(),
+                                      vd[:, :, m0:m0 + t].contiguous(), kc, vc, om, None, y * t, c, t, p0, st, None)
+            got[:, :, m0:m0 + t] = om
+            length = (y + 1) * t
+    torch.cuda.synchronize()
+    zone = oracle.layout_index(n, c, t, tail)[1]
+    live = zone != oracle.ZONE_REP
+    check(got[:, :, torch.from_numpy(live).to(DEV)], want_o[:, :, live], dtype)
