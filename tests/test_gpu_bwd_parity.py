@@ -43,7 +43,17 @@ def npf(x):
     return x.detach().to("cpu").to(torch.float64).numpy()
 
 
-def check_grad(got, want, dtype, name):
+def check_grad(got, want, dtype, name, zones=None):
+    """Whole-tensor bars scaled by the size of the reference (a gradient is a sum over up to tens of thousands
+    of rows), and, where the rows' zones are given, a bar per element: the forward's bar (2e-2, stated for
+    values of size about one) scaled by the element itself plus the root-mean-square of its own zone type where
+    that exceeds one.  Reading, memory and repetition rows have gradients of very different sizes (an early
+    memory key collects from every later reading row), and an error on the small ones must not hide behind the
+    largest element of the tensor.  The arithmetic: every output is rounded to bf16 (2^-9 of itself); P and dA
+    enter the second products rounded to bf16, 2^-9 of each of ~N terms of random sign, i.e. about 2^-9 of the
+    sum's typical size (the zone's rms); and delta = dO.O is formed from the bf16-rounded forward output, an
+    absolute error of about 2^-9 sqrt(D) |dO| |O| in every dA, which is what keeps the bar from going below the
+    forward's 2e-2 for gradients smaller than one."""
     g = npf(got)
     assert g.shape == want.shape and np.isfinite(g).all(), name
     d = np.abs(g - want)
@@ -53,6 +63,17 @@ def check_grad(got, want, dtype, name):
     else:
         assert d.max() <= 2e-2 * big, f"{name}: bf16 max |delta| {d.max():.3e} (ref max {big:.3g})"
         assert d.mean() <= 2e-3 * mean, f"{name}: bf16 mean |delta| {d.mean():.3e}"
+    if zones is not None:
+        zones = np.asarray(zones)
+        assert zones.shape[0] == want.shape[2]
+        rel = 1e-5 if dtype == torch.float32 else 2e-2
+        for z in np.unique(zones):
+            sel = zones == z
+            w, dz = want[:, :, sel], d[:, :, sel]
+            rms = max(float(np.sqrt((w ** 2).mean())), 1e-3)
+            bad = dz > rel * np.maximum(1.0, np.abs(w) + rms)
+            assert not bad.any(), (f"{name}, zone {int(z)}: {int(bad.sum())} elements beyond {rel:g} * max(1, |ref| + rms {rms:.3g}); "
+                                   f"worst |delta| {float(dz.max()):.3e}")
 
 
 def run_fwd_bwd(q, k, v, d_o, n, c, t, tail=0, flags=0, scale=0.0):
@@ -91,8 +112,9 @@ def test_masked_bwd_matches_oracle(B, H, D, n, c, t, tail, flags, dtype):
     d_o = synthetic.normal_tensor((B, H, S, D), 97, 1.0, dtype)
     want = oracle.masked_attn_bwd(npf(q), npf(k), npf(v), npf(d_o), n, c, t, tail, lay)
     got = run_fwd_bwd(q.to(DEV), k.to(DEV), v.to(DEV), d_o.to(DEV), n, c, t, tail, flags)
+    zone = oracle.layout_index(n, c, t, tail, lay)[1]
     for g, w, name in zip(got, want, ("dq", "dk", "dv")):
-        check_grad(g, w, dtype, name)
+        check_grad(g, w, dtype, name, zone)
 
 
 def test_masked_bwd_strided_views_explicit_scale_and_unsupervised_memory_rows():
@@ -141,8 +163,9 @@ def test_training_layout_4608_tokens_backward_sampled_heads():
     for b, h in [(0, 0), (3, 17)]:
         sl = (slice(b, b + 1), slice(h, h + 1))
         want = oracle.masked_attn_bwd(npf(q[sl]), npf(k[sl]), npf(v[sl]), npf(d_o[sl]), n, c, t)
+        zone = oracle.layout_index(n, c, t)[1]
         for g, w, name in zip((dq, dk, dv), want, ("dq", "dk", "dv")):
-            check_grad(g[sl], w, torch.bfloat16, name)
+            check_grad(g[sl], w, torch.bfloat16, name, zone)
     for g in (dq, dk, dv):
         assert torch.isfinite(g.float()).all()
 
@@ -180,10 +203,10 @@ def test_long_training_layout_69632_tokens_backward_sampled_rows_and_keys():
     h = 1
     sl = (slice(0, 1), slice(h, h + 1))
     want_dq = oracle.masked_attn_bwd_dq_rows(npf(q[sl]), npf(k[sl]), npf(v[sl]), npf(d_o[sl]), rows, n, c, t)
-    check_grad(dq[sl][:, :, ri], want_dq, torch.bfloat16, "dq")
+    check_grad(dq[sl][:, :, ri], want_dq, torch.bfloat16, "dq", zone[rows])
     want_dk, want_dv = oracle.masked_attn_bwd_dkv_cols(npf(q[sl]), npf(k[sl]), npf(v[sl]), npf(d_o[sl]), cols, n, c, t)
-    check_grad(dk[sl][:, :, ci], want_dk, torch.bfloat16, "dk")
-    check_grad(dv[sl][:, :, ci], want_dv, torch.bfloat16, "dv")
+    check_grad(dk[sl][:, :, ci], want_dk, torch.bfloat16, "dk", zone[cols])
+    check_grad(dv[sl][:, :, ci], want_dv, torch.bfloat16, "dv", zone[cols])
     for g in (dq, dk, dv):
         assert torch.isfinite(g.float()).all()
 
@@ -334,5 +357,17 @@ def test_tiles_with_more_than_64_steps_forward_and_backward():
     sl = (slice(0, 1), slice(1, 2))
     want_o, want_lse = oracle.masked_attn_fwd(npf(q[sl]), npf(k[sl]), npf(v[sl]), n, c, t, rows=rows)
     assert np.abs(npf(o[sl][:, :, ri]) - want_o).max() <= 2e-2 and np.abs(npf(lse[sl][:, :, ri]) - want_lse).max() <= 2e-2
+    zone = oracle.layout_index(n, c, t)[1]
     want_dq = oracle.masked_attn_bwd_dq_rows(npf(q[sl]), npf(k[sl]), npf(v[sl]), npf(d_o[sl]), rows, n, c, t)
-    check_grad(dq[sl][:, :, ri], want_dq, torch.bfloat16, "dq")
+    check_grad(dq[sl][:, :, ri], want_dq, torch.bfloat16, "dq", zone[rows])
+    # dK and dV against the oracle too: reading, repetition and late memory keys (a key tile that more than 64 query
+    # tiles visit is covered by the late-chunk reading keys: each is seen by its own zone's later rows and memory rows)
+    ch = oracle.layout_index(n, c, t)[0]
+    cols = np.unique(np.concatenate([rng.choice(np.nonzero(zone == 0)[0], 12, replace=False),
+                                     rng.choice(np.nonzero(zone == 2)[0], 6, replace=False),
+                                     rng.choice(np.nonzero((zone == 1) & (ch >= n - 2))[0], 8, replace=False),
+                                     rng.choice(np.nonzero((zone == 1) & (ch == 2))[0], 2, replace=False)]))
+    ci = torch.from_numpy(cols).to(DEV)
+    want_dk, want_dv = oracle.masked_attn_bwd_dkv_cols(npf(q[sl]), npf(k[sl]), npf(v[sl]), npf(d_o[sl]), cols, n, c, t)
+    check_grad(dk[sl][:, :, ci], want_dk, torch.bfloat16, "dk", zone[cols])
+    check_grad(dv[sl][:, :, ci], want_dv, torch.bfloat16, "dv", zone[cols])

@@ -689,7 +689,7 @@ def test_long_training_layout_69632_tokens_sampled_rows():
 
 
 @pytest.mark.parametrize("B,H,c,t,mem_len,steps", [(32, 32, 4, 16, 8192, (0, 1, 37, 63)),
-                                                   (8, 32, 8, 16, 16384, (0, 127))])
+                                                   (64, 32, 8, 16, 16384, (0, 127))])
 def test_generation_workloads_sampled_heads(B, H, c, t, mem_len, steps):
     """Generation shapes (D128 bf16): a cache of mem_len memory entries plus a
     growing tail; decode at several tail lengths, then the compress step.  The
