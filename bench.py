@@ -513,6 +513,29 @@ def other_workloads(L, synthetic, torch, dev, peaks):
                                        "gbs": nbytes / (ms * 1e-3) / 1e9,
                                        "frac_of_measured_hbm": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
         del kpool, vpool
+    # the generator's loop over layers: 8 layers' caches of the B32 / 8192 shape decoded in one call, per layer
+    del kc, vc
+    torch.cuda.empty_cache()
+    nl, Bl, memL, cl, tl = 8, 32, 8192, 4, 16
+    capL = memL + cl * tl + tl
+    kcs = [synthetic.big_normal_(torch.empty(Bl, H, capL, D, dtype=bf, device=dev), 3200 + i, std) for i in range(nl)]
+    vcs = [synthetic.big_normal_(torch.empty(Bl, H, capL, D, dtype=bf, device=dev), 3300 + i, std) for i in range(nl)]
+    qs, kns, vns = ([synthetic.big_normal_(torch.empty(Bl, H, 1, D, dtype=bf, device=dev), 3400 + 10 * j + i, std) for i in range(nl)]
+                    for j in range(3))
+    outs = [torch.empty_like(x) for x in qs]
+    wsl = torch.empty(max(16, L.loma_decode_workspace_bytes(Bl, H, D, capL)), dtype=torch.uint8, device=dev)
+    lenL = memL + 32
+    ms_layers = timed(lambda: L.loma_decode_attn_layers(qs, kns, vns, kcs, vcs, outs, None, lenL, wsl, 0, 0.0, stream))
+    ms_single = timed(lambda: L.loma_decode_attn(qs[0], kns[0], vns[0], kcs[0], vcs[0], outs[0], None, lenL, wsl, 0, 0.0, stream))
+    nbl = 2.0 * (lenL + 1) * Bl * H * D * 2
+    res["decode_8_layers_B32_8k"] = {"config": dict(layers=nl, B=Bl, H=H, D=D, cache_len=lenL), "ms": ms_layers,
+                                     "ms_per_layer": ms_layers / nl, "ms_single_layer_call": ms_single,
+                                     "gbs": nl * nbl / (ms_layers * 1e-3) / 1e9,
+                                     "frac_of_measured_hbm": nl * nbl / (ms_layers * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    del kcs, vcs
+    torch.cuda.empty_cache()
+    kc = synthetic.big_normal_(torch.empty(B, H, cap, D, dtype=bf, device=dev), 3100, std)
+    vc = synthetic.big_normal_(torch.empty(B, H, cap, D, dtype=bf, device=dev), 3101, std)
     for name, flags in (("compress_B64_16k", 0), ("compress_B64_16k_prior_mem", 1)):
         def run_decode_then_compress():
             L.loma_compress_step(qm, km, vm, kc, vc, om, None, mem_len, c, t, ws, flags, 0.0, stream)

@@ -319,6 +319,28 @@ LOMA_API int loma_decode_attn(const void* q, const void* k_new, const void* v_ne
                               void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * loma_decode_attn_layers, loma_compress_step_layers -- the generator's loop over the layers of the
+ * model (Appendix A: inference_input hands every layer's cache to the model, compress_last_chunk
+ * slices and re-concatenates `for i in range(len(self.kv_cache))`): the same step for n_layers
+ * independent (q, k, v, cache, output) sets of one shape, enqueued back to back on the stream.
+ * Every pointer argument is a [host] array of n_layers [device] pointers with the meaning the
+ * single-layer call gives them (k_new / v_new / lse may be NULL as a whole, or hold NULL entries
+ * where the single-layer call allows NULL).  The layers share one workspace of the single-layer
+ * size: they run one after the other.  Caches and outputs of different layers must be distinct.
+ * All layers are validated before the first is enqueued.  Errors: those of the single-layer call.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_decode_attn_layers(int n_layers, const void* const* q, const void* const* k_new,
+                                     const void* const* v_new, void* const* k_cache, void* const* v_cache,
+                                     void* const* o, float* const* lse, int B, int H, int D, int cap, int cache_len,
+                                     loma_dtype dtype, float softmax_scale, unsigned flags, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+LOMA_API int loma_compress_step_layers(int n_layers, const void* const* q_mem, const void* const* k_mem,
+                                       const void* const* v_mem, void* const* k_cache, void* const* v_cache,
+                                       void* const* o_mem, float* const* lse, int B, int H, int D, int cap, int mem_len,
+                                       int c, int t, int tc, loma_dtype dtype, float softmax_scale, unsigned flags,
+                                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------
  * loma_decode_attn_rope, loma_compress_step_rope -- the two generation steps with the rotary
  * position embedding of Section 4.5 done inside the step: q and the new key(s) are rotated in
  * registers / shared memory by their position ids right where the kernels load them, so the

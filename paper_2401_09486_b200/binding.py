@@ -43,6 +43,9 @@ SIGNATURES = {
     "loma_prefill_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _f, _u, _p]),
     "loma_prefill_attn_plan_coverage": (_i, [_i, _i, _p]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
+    "loma_decode_attn_layers": (_i, [_i, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
+    "loma_compress_step_layers": (_i, [_i, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz,
+                                       _p]),
     "loma_decode_attn_rope": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _i, _f, _u, _p, _sz, _p]),
     "loma_compress_step_rope": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _i, _f, _u, _p,
                                      _sz, _p]),
@@ -299,6 +302,48 @@ def loma_decode_attn(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len: int, 
                                 _ptr(lse), B, H, D, cap, cache_len, _dtype_code(q), float(softmax_scale),
                                 int(flags), _ptr(workspace), ws_bytes, _stream(stream))
     _check(rc, "loma_decode_attn")
+
+
+def _ptr_array(tensors):
+    """[host] array of device pointers, one per layer (None stays NULL)."""
+    if tensors is None:
+        return None
+    arr = (ctypes.c_void_p * len(tensors))()
+    for i, x in enumerate(tensors):
+        arr[i] = None if x is None else x.data_ptr()
+    return arr
+
+
+def loma_decode_attn_layers(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len: int, workspace=None, flags: int = 0,
+                            softmax_scale: float = 0.0, stream=None) -> None:
+    """Lists of per-layer tensors (shapes of loma_decode_attn); k_new, v_new, lse may be None."""
+    n = len(q)
+    B, H, cap, D = k_cache[0].shape
+    for group in (q, k_new, v_new, k_cache, v_cache, o):
+        for x in (group or []):
+            if x is not None and not x.is_contiguous():
+                raise ValueError("decode tensors must be contiguous")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    arrays = [_ptr_array(x) for x in (q, k_new, v_new, k_cache, v_cache, o, lse)]
+    rc = lib().loma_decode_attn_layers(n, *arrays, B, H, D, cap, cache_len, _dtype_code(q[0]), float(softmax_scale), int(flags),
+                                       _ptr(workspace), ws_bytes, _stream(stream))
+    _check(rc, "loma_decode_attn_layers")
+
+
+def loma_compress_step_layers(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, mem_len: int, c: int, t: int, workspace=None,
+                              flags: int = 0, softmax_scale: float = 0.0, stream=None) -> None:
+    """Lists of per-layer tensors (shapes of loma_compress_step); lse may be None."""
+    n = len(q_mem)
+    B, H, cap, D = k_cache[0].shape
+    for group in (q_mem, k_mem, v_mem, k_cache, v_cache, o_mem):
+        for x in group:
+            if not x.is_contiguous():
+                raise ValueError("compress tensors must be contiguous")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    arrays = [_ptr_array(x) for x in (q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse)]
+    rc = lib().loma_compress_step_layers(n, *arrays, B, H, D, cap, mem_len, c, t, c * t, _dtype_code(q_mem[0]),
+                                         float(softmax_scale), int(flags), _ptr(workspace), ws_bytes, _stream(stream))
+    _check(rc, "loma_compress_step_layers")
 
 
 def loma_decode_attn_rope(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len: int, pos: int, workspace=None,

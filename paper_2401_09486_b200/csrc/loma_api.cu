@@ -355,6 +355,82 @@ int loma_decode_attn_rope(const void* q, const void* k_new, const void* v_new, v
                             workspace, workspace_bytes, stream, rope);
 }
 
+// ---- the generator's loop over layers (Appendix A: `for i in range(len(self.kv_cache))`) ------------------
+int loma_decode_attn_layers(int n_layers, const void* const* q, const void* const* k_new, const void* const* v_new,
+                            void* const* k_cache, void* const* v_cache, void* const* o, float* const* lse, int B, int H,
+                            int D, int cap, int cache_len, loma_dtype dtype, float softmax_scale, unsigned flags,
+                            void* workspace, size_t workspace_bytes, void* stream) {
+    if (n_layers < 0) return LOMA_ERR_INVALID_ARG;
+    if (n_layers > 0 && (!q || !k_cache || !v_cache || !o)) return LOMA_ERR_INVALID_ARG;
+    // every layer is validated before the first one is enqueued (nothing runs on an error)
+    for (int pass = 0; pass < 2; ++pass) {
+        for (int i = 0; i < n_layers; ++i) {
+            const void* kn = k_new ? k_new[i] : nullptr;
+            const void* vn = v_new ? v_new[i] : nullptr;
+            float* ls = lse ? lse[i] : nullptr;
+            if (pass == 0) {
+                if ((kn == nullptr) != (vn == nullptr)) return LOMA_ERR_INVALID_ARG;
+                if (B > 0 && H > 0 && (!q[i] || !k_cache[i] || !v_cache[i] || !o[i])) return LOMA_ERR_INVALID_ARG;
+                if (!aligned16(q[i]) || !aligned16(k_cache[i]) || !aligned16(v_cache[i]) || !aligned16(o[i]) || !aligned16(kn) ||
+                    !aligned16(vn))
+                    return LOMA_ERR_ALIGNMENT;
+                for (int j = 0; j < i; ++j)
+                    if (k_cache[j] == k_cache[i] || v_cache[j] == v_cache[i] || o[j] == o[i]) return LOMA_ERR_INVALID_ARG;
+            } else {
+                // the layers share the workspace: they run one after the other on the stream
+                const int rc = loma_decode_attn(q[i], kn, vn, k_cache[i], v_cache[i], o[i], ls, B, H, D, cap, cache_len, dtype,
+                                                softmax_scale, flags, workspace, workspace_bytes, stream);
+                if (rc != LOMA_OK) return rc;
+            }
+        }
+        if (pass == 0 && n_layers > 0) {
+            // the scalar arguments: checked once through a call that launches nothing (B = 0 is a no-op after validation)
+            if (B < 0 || H < 0 || cap < 0 || cache_len < 0) return LOMA_ERR_INVALID_ARG;
+            if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+            if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+            if (cache_len >= cap) return LOMA_ERR_CAPACITY;
+            if (!aligned16(workspace)) return LOMA_ERR_ALIGNMENT;
+            const size_t need = loma_decode_workspace_bytes(B, H, D, cache_len);
+            if (B > 0 && H > 0 && need > 0 && (!workspace || workspace_bytes < need)) return LOMA_ERR_WORKSPACE;
+        }
+    }
+    return LOMA_OK;
+}
+
+int loma_compress_step_layers(int n_layers, const void* const* q_mem, const void* const* k_mem, const void* const* v_mem,
+                              void* const* k_cache, void* const* v_cache, void* const* o_mem, float* const* lse, int B,
+                              int H, int D, int cap, int mem_len, int c, int t, int tc, loma_dtype dtype,
+                              float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes, void* stream) {
+    if (n_layers < 0) return LOMA_ERR_INVALID_ARG;
+    if (n_layers > 0 && (!q_mem || !k_mem || !v_mem || !k_cache || !v_cache || !o_mem)) return LOMA_ERR_INVALID_ARG;
+    if (n_layers > 0) {
+        if (B < 0 || H < 0 || cap < 0 || mem_len < 0 || c < 1 || t < 1) return LOMA_ERR_INVALID_ARG;
+        if ((int64_t)c * t != (int64_t)tc) return LOMA_ERR_INVALID_ARG;
+        if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+        if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+        if ((int64_t)mem_len + tc > (int64_t)cap) return LOMA_ERR_CAPACITY;
+        if (!aligned16(workspace)) return LOMA_ERR_ALIGNMENT;
+        const size_t need = loma_compress_workspace_bytes(B, H, D, t, mem_len, flags);
+        if (B > 0 && H > 0 && need > 0 && (!workspace || workspace_bytes < need)) return LOMA_ERR_WORKSPACE;
+    }
+    for (int i = 0; i < n_layers; ++i) {
+        if (B > 0 && H > 0 && (!q_mem[i] || !k_mem[i] || !v_mem[i] || !k_cache[i] || !v_cache[i] || !o_mem[i]))
+            return LOMA_ERR_INVALID_ARG;
+        if (!aligned16(q_mem[i]) || !aligned16(k_mem[i]) || !aligned16(v_mem[i]) || !aligned16(k_cache[i]) ||
+            !aligned16(v_cache[i]) || !aligned16(o_mem[i]))
+            return LOMA_ERR_ALIGNMENT;
+        for (int j = 0; j < i; ++j)
+            if (k_cache[j] == k_cache[i] || v_cache[j] == v_cache[i] || o_mem[j] == o_mem[i]) return LOMA_ERR_INVALID_ARG;
+    }
+    for (int i = 0; i < n_layers; ++i) {
+        const int rc = loma_compress_step(q_mem[i], k_mem[i], v_mem[i], k_cache[i], v_cache[i], o_mem[i], lse ? lse[i] : nullptr,
+                                          B, H, D, cap, mem_len, c, t, tc, dtype, softmax_scale, flags, workspace,
+                                          workspace_bytes, stream);
+        if (rc != LOMA_OK) return rc;
+    }
+    return LOMA_OK;
+}
+
 int loma_prefill_attn(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
                       float* lse, int B, int H, int D, int l, int cap, int cache_len, loma_dtype dtype,
                       float softmax_scale, unsigned flags, void* stream) {

@@ -132,6 +132,35 @@ def test_rope_fused_steps_validation(lib):
     assert cmp_(B=0) == 0
 
 
+def test_layer_loop_validation(lib):
+    import ctypes
+    arr = lambda *xs: (ctypes.c_void_p * len(xs))(*xs)
+    def dec(n=2, q=arr(0x1000, 0x1100), kn=arr(0x2000, 0x2100), vn=arr(0x3000, 0x3100), kc=arr(0x4000, 0x4100),
+            vc=arr(0x5000, 0x5100), o=arr(0x6000, 0x6100), B=1, H=1, D=128, cap=8, cache_len=3, dt=1):
+        return lib.loma_decode_attn_layers(n, q, kn, vn, kc, vc, o, None, B, H, D, cap, cache_len, dt, 0.0, 0, None, 0, None)
+    assert dec(n=-1) == INVALID
+    assert dec(q=None) == INVALID
+    assert dec(kc=arr(0x4000, 0x4000)) == INVALID        # two layers on one cache
+    assert dec(q=arr(0x1000, 0x1104)) == ALIGNMENT       # the second layer is checked before the first is enqueued
+    assert dec(kn=arr(0x2000, None)) == INVALID          # k_new without v_new in layer 1
+    assert dec(cache_len=8) == CAPACITY
+    assert dec(D=96) == UNSUPPORTED
+    assert dec(n=0) == 0
+    assert dec(H=0) == 0
+
+    def cmp_(n=2, qm=arr(0x1000, 0x1100), km=arr(0x2000, 0x2100), vm=arr(0x3000, 0x3100), kc=arr(0x4000, 0x4100),
+             vc=arr(0x5000, 0x5100), om=arr(0x6000, 0x6100), B=1, H=1, D=128, cap=96, mem_len=16, c=4, t=16, tc=64, dt=1):
+        return lib.loma_compress_step_layers(n, qm, km, vm, kc, vc, om, None, B, H, D, cap, mem_len, c, t, tc, dt, 0.0, 0,
+                                             None, 0, None)
+    assert cmp_(tc=63) == INVALID
+    assert cmp_(cap=79) == CAPACITY
+    assert cmp_(km=arr(0x2000, None)) == INVALID
+    assert cmp_(om=arr(0x6000, 0x6000)) == INVALID
+    assert cmp_(vm=arr(0x3000, 0x3108)) == ALIGNMENT
+    assert cmp_(n=0) == 0
+    assert cmp_(B=0) == 0
+
+
 def test_prefill_attn_validation(lib):
     def call(q=0x1000, kn=0x2000, vn=0x3000, kc=0x4000, vc=0x5000, o=0x6000, lse=None, B=1, H=1, D=128, l=4, cap=16,
              cache_len=3, dt=1, flags=0):

@@ -733,6 +733,45 @@ def test_generation_workloads_sampled_heads(B, H, c, t, mem_len, steps):
         del kc2, vc2
 
 
+def test_layer_loop_equals_layer_by_layer_calls_and_the_oracle():
+    """Appendix A loops over the layers' caches; the *_layers entry points do that loop inside one call: same bits
+    as one call per layer, the oracle checked on one layer."""
+    B, H, D, c, t, mem_len, nl = 2, 3, 128, 4, 16, 320, 3
+    tc = c * t
+    cap = mem_len + tc + 4
+    dt = torch.bfloat16
+    mk = lambda shape, seed: [synthetic.normal_tensor(shape, seed + 10 * i, 1.0, dt).to(DEV) for i in range(nl)]
+    kc, vc = mk((B, H, cap, D), 400), mk((B, H, cap, D), 401)
+    kc2, vc2 = [x.clone() for x in kc], [x.clone() for x in vc]
+    ws = workspace(max(L.loma_decode_workspace_bytes(B, H, D, cap), L.loma_compress_workspace_bytes(B, H, D, t, mem_len, 0)))
+    for j in range(tc):                                   # a whole chunk: tc decodes ...
+        q, kn, vn = mk((B, H, 1, D), 500 + j), mk((B, H, 1, D), 600 + j), mk((B, H, 1, D), 700 + j)
+        o = [torch.empty((B, H, 1, D), dtype=dt, device=DEV) for _ in range(nl)]
+        o2 = [torch.empty_like(x) for x in o]
+        if j == tc - 1:
+            want_o, _, _, _ = oracle.decode_attn(npf(q[1]), npf(kn[1]), npf(vn[1]), npf(kc[1]), npf(vc[1]), mem_len + j)
+        L.loma_decode_attn_layers(q, kn, vn, kc, vc, o, None, mem_len + j, ws)
+        for i in range(nl):
+            L.loma_decode_attn(q[i], kn[i], vn[i], kc2[i], vc2[i], o2[i], None, mem_len + j, ws)
+        torch.cuda.synchronize()
+        for i in range(nl):
+            assert torch.equal(o[i], o2[i])
+    check_close(o[1], want_o, dt)
+    qm, km, vm = mk((B, H, t, D), 800), mk((B, H, t, D), 801), mk((B, H, t, D), 802)
+    om = [torch.empty((B, H, t, D), dtype=dt, device=DEV) for _ in range(nl)]
+    om2 = [torch.empty_like(x) for x in om]
+    want_om, _, nk, nv = oracle.compress_step(npf(qm[2]), npf(km[2]), npf(vm[2]), npf(kc[2]), npf(vc[2]), mem_len, c, t)
+    L.loma_compress_step_layers(qm, km, vm, kc, vc, om, None, mem_len, c, t, ws)     # ... then the compress step
+    for i in range(nl):
+        L.loma_compress_step(qm[i], km[i], vm[i], kc2[i], vc2[i], om2[i], None, mem_len, c, t, ws)
+    torch.cuda.synchronize()
+    for i in range(nl):
+        assert torch.equal(om[i], om2[i])
+        assert torch.equal(kc[i][:, :, :mem_len + t], kc2[i][:, :, :mem_len + t]) and torch.equal(vc[i][:, :, :mem_len + t], vc2[i][:, :, :mem_len + t])
+    check_close(om[2], want_om, dt)
+    assert np.array_equal(npf(kc[2][:, :, :mem_len + t]), nk) and np.array_equal(npf(vc[2][:, :, :mem_len + t]), nv)
+
+
 def test_generation_cycle_replays_from_a_cuda_graph():
     """After one eager call of each entry point (first calls look up device symbols and set kernel attributes),
     a tail of decode steps plus the compress step is captured into a CUDA graph and replayed: the replay equals
