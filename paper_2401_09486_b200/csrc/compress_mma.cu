@@ -440,13 +440,14 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
     int prior_len = 0;
     if (nprior > 0) prior_len = ((mem_len + nprior - 1) / nprior + 15) / 16 * 16;
     const int nsp = nprior + 1;
-    const int smem = CmpSmem<D>::TOTAL;
+    // (the cos/sin table of the fused rotary embedding is only allocated when it is used: without it three CTAs fit an SM)
+    const int smem = rope.on ? CmpSmem<D>::TOTAL : CmpSmem<D>::ROPE_OFF;
     cudaError_t e;
     static bool attr_set[64] = {false};   // per device, per template instance
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
     if (!attr_set[dev]) {
-        e = cudaFuncSetAttribute(compress_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        e = cudaFuncSetAttribute(compress_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, CmpSmem<D>::TOTAL);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
