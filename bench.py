@@ -536,6 +536,22 @@ def other_workloads(L, synthetic, torch, dev, peaks):
     torch.cuda.empty_cache()
     kc = synthetic.big_normal_(torch.empty(B, H, cap, D, dtype=bf, device=dev), 3100, std)
     vc = synthetic.big_normal_(torch.empty(B, H, cap, D, dtype=bf, device=dev), 3101, std)
+    # several new tokens over an existing cache (a prompt piece arriving mid-generation): 512 tokens over 8192 entries
+    Bp, lp, kp = 32, 512, 8192
+    kcp = synthetic.big_normal_(torch.empty(Bp, H, kp + lp, D, dtype=bf, device=dev), 3500, std)
+    vcp = synthetic.big_normal_(torch.empty(Bp, H, kp + lp, D, dtype=bf, device=dev), 3501, std)
+    qp, knp, vnp = (synthetic.big_normal_(torch.empty(Bp, H, lp, D, dtype=bf, device=dev), 3502 + i, std) for i in range(3))
+    op = torch.empty_like(qp)
+    ms = timed(lambda: L.loma_prefill_attn(qp, knp, vnp, kcp, vcp, op, None, kp, 0, 0.0, stream))
+    fl = 4.0 * D * Bp * H * (lp * kp + lp * (lp + 1) // 2)
+    nbytes = float(Bp * H) * D * 2 * (2 * (kp + lp) + 4 * lp)      # cache K, V read once; q, k_new, v_new read, o written
+    res["prefill_512_over_8192_B32"] = {"config": dict(B=Bp, H=H, D=D, l=lp, cache_len=kp), "ms": ms,
+                                        "useful_tflops": fl / (ms * 1e-3) / 1e12,
+                                        "frac_of_measured_bf16": fl / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                                        "gbs": nbytes / (ms * 1e-3) / 1e9,
+                                        "kernels": "cache_append_kernel + masked_attn_tc_kernel (prefill plan)"}
+    del kcp, vcp, qp, knp, vnp, op
+    torch.cuda.empty_cache()
     for name, flags in (("compress_B64_16k", 0), ("compress_B64_16k_prior_mem", 1)):
         def run_decode_then_compress():
             L.loma_compress_step(qm, km, vm, kc, vc, om, None, mem_len, c, t, ws, flags, 0.0, stream)
