@@ -387,7 +387,7 @@ LOMA_API int loma_compress_step_rope(const void* q_mem, const void* k_mem, const
  *   lse              [device, out]    fp32 [B, H, l] or NULL
  *   cache_len        entries before this call (memory entries + uncompressed tail), the
  *                    same for every sequence of the batch
- * bf16 calls with l >= 64 run on the tensor-core kernel of loma_masked_attn_fwd (its
+ * bf16 calls with l >= 8 run on the tensor-core kernel of loma_masked_attn_fwd (its
  * concurrency notes apply), the rest on CUDA cores.  No workspace.
  * Errors: INVALID_ARG, UNSUPPORTED, ALIGNMENT, CAPACITY (cache_len + l > cap), CUDA.
  * l == 0 or B*H == 0 is a successful no-op.

@@ -458,7 +458,9 @@ int loma_prefill_attn(const void* q, const void* k_new, const void* v_new, void*
             return LOMA_ERR_CUDA;
     }
     cudaError_t e = cudaErrorNotSupported;
-    if (dtype == LOMA_BF16 && l >= 64 && !(flags & LOMA_FLAG_FORCE_GENERIC)) {
+    // (a handful of rows is cheaper on CUDA cores, one warp per row; from 8 rows on one pass of the cache through the
+    // tensor-core kernel wins over l passes)
+    if (dtype == LOMA_BF16 && l >= 8 && !(flags & LOMA_FLAG_FORCE_GENERIC)) {
         e = launch_prefill_attn_tc(q, k_cache, v_cache, o, lse, B, H, D, l, cap, cache_len, scale, st);
         if (e == cudaErrorNotSupported) g_fallbacks.fetch_add(1, std::memory_order_relaxed);
     }

@@ -266,7 +266,7 @@ def test_incremental_generation_equals_one_shot(B, H, D, n, c, t, tail, flags, d
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("flags", [0, GENERIC])
-@pytest.mark.parametrize("l", [1, 2, 17, 64, 200, 300])
+@pytest.mark.parametrize("l", [1, 2, 8, 17, 64, 200, 300])
 @pytest.mark.parametrize("cache_len", [0, 16, 100, 8192])
 def test_prefill_over_a_cache_matches_oracle_and_appends_bit_exact(l, cache_len, flags, dtype):
     """Appendix A `inference_input` with l tokens: mask tril(ones(l, l + k), diagonal = k), K/V appended."""
