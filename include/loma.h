@@ -319,6 +319,43 @@ LOMA_API int loma_decode_attn(const void* q, const void* k_new, const void* v_ne
                               void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------
+ * The rope-fused steps for ragged batches and the paged cache: loma_decode_attn_rope /
+ * loma_compress_step_rope (Section 4.5; Appendix A position ids) with one position per
+ * sequence, since every sequence of a ragged batch has its own `cursor`.
+ *
+ *   positions [device, in]  int32 [B]: the position id of sequence b's new token
+ *   pos0s     [device, in]  int32 [B]: the id of sequence b's memory row 0; row j gets
+ *                           pos0s[b] + j * pos_stride (entries of sequences that do not compress
+ *                           in this call, mem_lens[b] < 0, are ignored)
+ * Every other argument, and every rule, is that of the entry point without `_rope`; k_new and
+ * v_new are required.  Errors: those of that entry point, plus INVALID_ARG (NULL positions,
+ * negative stride), ALIGNMENT (positions not 4-byte aligned), UNSUPPORTED (memory zone too long
+ * to stage, t*D*sizeof(element) > 200 KB).
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_decode_attn_ragged_rope(const void* q, const void* k_new, const void* v_new, void* k_cache,
+                                          void* v_cache, void* o, float* lse, int B, int H, int D, int cap,
+                                          const int32_t* cache_lens, int max_cache_len, const int32_t* positions,
+                                          float theta_base, loma_dtype dtype, float softmax_scale, unsigned flags,
+                                          void* workspace, size_t workspace_bytes, void* stream);
+LOMA_API int loma_decode_attn_paged_rope(const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+                                         const int32_t* block_table, void* o, float* lse, int B, int H, int D,
+                                         int page_size, int max_pages, int n_pages, const int32_t* cache_lens,
+                                         int max_cache_len, const int32_t* positions, float theta_base, loma_dtype dtype,
+                                         float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes,
+                                         void* stream);
+LOMA_API int loma_compress_step_ragged_rope(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache,
+                                            void* v_cache, void* o_mem, float* lse, int B, int H, int D, int cap,
+                                            const int32_t* mem_lens, int max_mem_len, int c, int t, int tc,
+                                            const int32_t* pos0s, int pos_stride, float theta_base, loma_dtype dtype,
+                                            float softmax_scale, unsigned flags, void* stream);
+LOMA_API int loma_compress_step_paged_rope(const void* q_mem, const void* k_mem, const void* v_mem, void* k_pool,
+                                           void* v_pool, const int32_t* block_table, void* o_mem, float* lse, int B, int H,
+                                           int D, int page_size, int max_pages, int n_pages, const int32_t* mem_lens,
+                                           int max_mem_len, int c, int t, int tc, const int32_t* pos0s, int pos_stride,
+                                           float theta_base, loma_dtype dtype, float softmax_scale, unsigned flags,
+                                           void* stream);
+
+/* ---------------------------------------------------------------------------
  * loma_decode_attn_layers, loma_compress_step_layers -- the generator's loop over the layers of the
  * model (Appendix A: inference_input hands every layer's cache to the model, compress_last_chunk
  * slices and re-concatenates `for i in range(len(self.kv_cache))`): the same step for n_layers

@@ -52,6 +52,12 @@ SIGNATURES = {
     "loma_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "loma_decode_attn_paged": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_attn_ragged": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p, _sz, _p]),
+    "loma_decode_attn_ragged_rope": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _p, _i, _p, _f, _i, _f, _u, _p, _sz, _p]),
+    "loma_decode_attn_paged_rope": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _p, _i, _p, _f, _i, _f, _u, _p, _sz,
+                                         _p]),
+    "loma_compress_step_ragged_rope": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _p, _i, _i, _i, _i, _p, _i, _f, _i, _f, _u, _p]),
+    "loma_compress_step_paged_rope": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _p, _i, _i, _i, _i, _p, _i, _f, _i,
+                                           _f, _u, _p]),
     "loma_decode_attn_static": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _p]),
     "loma_decode_static_scratch_bytes": (_sz, []),
     "loma_compress_step": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz,
@@ -412,6 +418,88 @@ def loma_decode_attn_paged(q, k_new, v_new, k_pool, v_pool, block_table, o, lse,
                                       int(max_cache_len), _dtype_code(q), float(softmax_scale), int(flags),
                                       _ptr(workspace), ws_bytes, _stream(stream))
     _check(rc, "loma_decode_attn_paged")
+
+
+def _check_positions(positions, B, what):
+    if positions.dtype != torch.int32 or positions.numel() != B or not positions.is_contiguous():
+        raise ValueError(f"{what} must be a contiguous int32 [B] tensor")
+
+
+def loma_decode_attn_ragged_rope(q, k_new, v_new, k_cache, v_cache, o, lse, cache_lens, max_cache_len: int, positions,
+                                 workspace=None, flags: int = 0, softmax_scale: float = 0.0, theta_base: float = 0.0,
+                                 stream=None) -> None:
+    """loma_decode_attn_ragged with q and k_new of sequence b rotated inside the step by positions[b] (device int32 [B])."""
+    B, H, cap, D = k_cache.shape
+    for x in (q, k_new, v_new, k_cache, v_cache, o, cache_lens):
+        if x is not None and not x.is_contiguous():
+            raise ValueError("decode tensors must be contiguous")
+    if cache_lens.dtype != torch.int32 or cache_lens.numel() != B:
+        raise ValueError("cache_lens must be int32 [B]")
+    _check_positions(positions, B, "positions")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().loma_decode_attn_ragged_rope(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse),
+                                            B, H, D, cap, _ptr(cache_lens), int(max_cache_len), _ptr(positions),
+                                            float(theta_base), _dtype_code(q), float(softmax_scale), int(flags),
+                                            _ptr(workspace), ws_bytes, _stream(stream))
+    _check(rc, "loma_decode_attn_ragged_rope")
+
+
+def loma_decode_attn_paged_rope(q, k_new, v_new, k_pool, v_pool, block_table, o, lse, cache_lens, max_cache_len: int, positions,
+                                workspace=None, flags: int = 0, softmax_scale: float = 0.0, theta_base: float = 0.0,
+                                stream=None) -> None:
+    """loma_decode_attn_paged with the rotation fused in (positions: device int32 [B])."""
+    n_pages, H, page_size, D = k_pool.shape
+    B, max_pages = block_table.shape
+    for x in (q, k_new, v_new, k_pool, v_pool, o, block_table, cache_lens):
+        if x is not None and not x.is_contiguous():
+            raise ValueError("decode tensors must be contiguous")
+    if block_table.dtype != torch.int32 or cache_lens.dtype != torch.int32 or cache_lens.numel() != B:
+        raise ValueError("block_table must be int32 [B, max_pages] and cache_lens int32 [B]")
+    _check_positions(positions, B, "positions")
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().loma_decode_attn_paged_rope(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool), _ptr(block_table),
+                                           _ptr(o), _ptr(lse), B, H, D, page_size, max_pages, n_pages, _ptr(cache_lens),
+                                           int(max_cache_len), _ptr(positions), float(theta_base), _dtype_code(q),
+                                           float(softmax_scale), int(flags), _ptr(workspace), ws_bytes, _stream(stream))
+    _check(rc, "loma_decode_attn_paged_rope")
+
+
+def loma_compress_step_ragged_rope(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, mem_lens, max_mem_len: int, c: int, t: int,
+                                   pos0s, pos_stride: int, flags: int = 0, softmax_scale: float = 0.0, theta_base: float = 0.0,
+                                   stream=None) -> None:
+    """loma_compress_step_ragged with memory row j of sequence b rotated by pos0s[b] + j * pos_stride inside the step."""
+    B, H, cap, D = k_cache.shape
+    for x in (q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, mem_lens):
+        if not x.is_contiguous():
+            raise ValueError("compress tensors must be contiguous")
+    if mem_lens.dtype != torch.int32 or mem_lens.numel() != B:
+        raise ValueError("mem_lens must be int32 [B]")
+    _check_positions(pos0s, B, "pos0s")
+    rc = lib().loma_compress_step_ragged_rope(_ptr(q_mem), _ptr(k_mem), _ptr(v_mem), _ptr(k_cache), _ptr(v_cache), _ptr(o_mem),
+                                              _ptr(lse), B, H, D, cap, _ptr(mem_lens), int(max_mem_len), c, t, c * t,
+                                              _ptr(pos0s), int(pos_stride), float(theta_base), _dtype_code(q_mem),
+                                              float(softmax_scale), int(flags), _stream(stream))
+    _check(rc, "loma_compress_step_ragged_rope")
+
+
+def loma_compress_step_paged_rope(q_mem, k_mem, v_mem, k_pool, v_pool, block_table, o_mem, lse, mem_lens, max_mem_len: int,
+                                  c: int, t: int, pos0s, pos_stride: int, flags: int = 0, softmax_scale: float = 0.0,
+                                  theta_base: float = 0.0, stream=None) -> None:
+    """loma_compress_step_paged with the rotation fused in (pos0s: device int32 [B])."""
+    n_pages, H, page_size, D = k_pool.shape
+    B, max_pages = block_table.shape
+    for x in (q_mem, k_mem, v_mem, k_pool, v_pool, o_mem, mem_lens, block_table):
+        if not x.is_contiguous():
+            raise ValueError("compress tensors must be contiguous")
+    if block_table.dtype != torch.int32 or mem_lens.dtype != torch.int32 or mem_lens.numel() != B:
+        raise ValueError("block_table must be int32 [B, max_pages] and mem_lens int32 [B]")
+    _check_positions(pos0s, B, "pos0s")
+    rc = lib().loma_compress_step_paged_rope(_ptr(q_mem), _ptr(k_mem), _ptr(v_mem), _ptr(k_pool), _ptr(v_pool),
+                                             _ptr(block_table), _ptr(o_mem), _ptr(lse), B, H, D, page_size, max_pages, n_pages,
+                                             _ptr(mem_lens), int(max_mem_len), c, t, c * t, _ptr(pos0s), int(pos_stride),
+                                             float(theta_base), _dtype_code(q_mem), float(softmax_scale), int(flags),
+                                             _stream(stream))
+    _check(rc, "loma_compress_step_paged_rope")
 
 
 def loma_decode_static_scratch_bytes() -> int:

@@ -280,9 +280,10 @@ decode_generic_kernel(const T* __restrict__ q, const T* __restrict__ k_new, cons
     if (rope.on) {
         // Section 4.5: q and the new key rotated by the step's position id, here instead of in a pass of their own;
         // the rotated key, rounded to the storage type, is what the step attends to and appends
+        const int pos = rope.pos_seq ? rope.pos_seq[bh / H] : rope.pos0;
         for (int d = lane; d < D / 2; d += 32) {
             float c, sn;
-            rope_cos_sin(rope.pos0, d, D, rope.log2_base, c, sn);
+            rope_cos_sin(pos, d, D, rope.log2_base, c, sn);
             const float qa = q_sh[d], qb = q_sh[d + D / 2];
             q_sh[d] = qa * c - qb * sn;
             q_sh[d + D / 2] = qb * c + qa * sn;
@@ -397,6 +398,7 @@ compress_generic_kernel(const T* __restrict__ q_mem, const T* __restrict__ k_mem
     map.km = k_mem + (int64_t)bh * t * D; map.vm = v_mem + (int64_t)bh * t * D;
     map.n_cache = mem_len + tc - lo; map.D = D;
     map.pg = pg; map.b = bh / H; map.h = bh - map.b * H; map.H = H;
+    const int rope_pos0 = rope.pos_seq ? rope.pos_seq[bh / H] : rope.pos0;
     if (rope.on) {
         // Section 4.5: memory row j is rotated by the id pos0 + j * stride; its key, rounded to the storage type,
         // is what every memory query attends to and what goes into the cache
@@ -404,7 +406,7 @@ compress_generic_kernel(const T* __restrict__ q_mem, const T* __restrict__ k_mem
         for (int e = threadIdx.x; e < t * (D / 2); e += blockDim.x) {
             const int j = e / (D / 2), d = e - j * (D / 2);
             float c, sn;
-            rope_cos_sin(rope.pos0 + j * rope.stride, d, D, rope.log2_base, c, sn);
+            rope_cos_sin(rope_pos0 + j * rope.stride, d, D, rope.log2_base, c, sn);
             const float a = to_f32(map.km[(int64_t)j * D + d]), b = to_f32(map.km[(int64_t)j * D + d + D / 2]);
             km_rot[j * D + d] = from_f32<T>(a * c - b * sn);
             km_rot[j * D + d + D / 2] = from_f32<T>(b * c + a * sn);
@@ -417,7 +419,7 @@ compress_generic_kernel(const T* __restrict__ q_mem, const T* __restrict__ k_mem
         if (rope.on) {
             for (int d = lane; d < D / 2; d += 32) {
                 float c, sn;
-                rope_cos_sin(rope.pos0 + j * rope.stride, d, D, rope.log2_base, c, sn);
+                rope_cos_sin(rope_pos0 + j * rope.stride, d, D, rope.log2_base, c, sn);
                 const float a = q_sh[warp][d], b = q_sh[warp][d + D / 2];
                 q_sh[warp][d] = a * c - b * sn;
                 q_sh[warp][d + D / 2] = b * c + a * sn;

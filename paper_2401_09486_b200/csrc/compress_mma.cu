@@ -183,7 +183,7 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
         for (int e = threadIdx.x; e < 16 * (D / 2); e += CMP_WARPS * 32) {
             const int r = e / (D / 2), d = e - r * (D / 2);
             float c, sn;
-            rope_cos_sin(rope.pos0 + (q0 + r) * rope.stride, d, D, rope.log2_base, c, sn);
+            rope_cos_sin((rope.pos_seq ? __ldg(rope.pos_seq + bh / H) : rope.pos0) + (q0 + r) * rope.stride, d, D, rope.log2_base, c, sn);
             rope_tab[e] = make_float2(c, sn);
         }
         __syncthreads();

@@ -129,7 +129,8 @@ decode_splitkv_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
     if (rope.on) {
         // q and the new key are rotated here, in registers / shared memory, by the step's position id: no
         // separate pass over them.  The rotated key, rounded to bf16, is what the step attends to and appends.
-        if (threadIdx.x < D / 2) rope_cos_sin(rope.pos0, threadIdx.x, D, rope.log2_base, sm_cs[threadIdx.x], sm_sn[threadIdx.x]);
+        const int pos = rope.pos_seq ? __ldg(rope.pos_seq + bh / H) : rope.pos0;
+        if (threadIdx.x < D / 2) rope_cos_sin(pos, threadIdx.x, D, rope.log2_base, sm_cs[threadIdx.x], sm_sn[threadIdx.x]);
         __syncthreads();
         if (needs_new_key && threadIdx.x < D / 2) {
             const __nv_bfloat16* kp = reinterpret_cast<const __nv_bfloat16*>(kn);

@@ -477,10 +477,11 @@ int loma_prefill_attn_plan_coverage(int l, int cache_len, uint8_t* counts) {
     return LOMA_OK;
 }
 
-int loma_decode_attn_ragged(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
+static int loma_decode_attn_ragged_impl(const void* q, const void* k_new, const void* v_new, void* k_cache,
+                                        void* v_cache, void* o,
                             float* lse, int B, int H, int D, int cap, const int32_t* cache_lens, int max_cache_len,
                             loma_dtype dtype, float softmax_scale, unsigned flags, void* workspace,
-                            size_t workspace_bytes, void* stream) {
+                            size_t workspace_bytes, void* stream, const RopeArgs& rope) {
     if (B < 0 || H < 0 || cap < 0 || max_cache_len < 0) return LOMA_ERR_INVALID_ARG;
     if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
     if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
@@ -501,11 +502,35 @@ int loma_decode_attn_ragged(const void* q, const void* k_new, const void* v_new,
     cudaError_t e;
     if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC))
         e = launch_decode_bf16(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, max_cache_len, cache_lens, scale,
-                               workspace, Paging{}, st);
+                               workspace, Paging{}, st, rope);
     else
         e = launch_decode_generic(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, max_cache_len, cache_lens,
-                                  dtype, scale, Paging{}, st);
+                                  dtype, scale, Paging{}, st, rope);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
+int loma_decode_attn_ragged(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
+                            float* lse, int B, int H, int D, int cap, const int32_t* cache_lens, int max_cache_len,
+                            loma_dtype dtype, float softmax_scale, unsigned flags, void* workspace,
+                            size_t workspace_bytes, void* stream) {
+    return loma_decode_attn_ragged_impl(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_lens,
+                                        max_cache_len, dtype, softmax_scale, flags, workspace, workspace_bytes,
+                                        stream, RopeArgs{});
+}
+
+int loma_decode_attn_ragged_rope(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                                 void* o, float* lse, int B, int H, int D, int cap, const int32_t* cache_lens,
+                                 int max_cache_len, const int32_t* positions, float theta_base, loma_dtype dtype,
+                                 float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
+    if (B > 0 && H > 0 && (!positions || !k_new || !v_new)) return LOMA_ERR_INVALID_ARG;
+    if ((uintptr_t)positions & 3u) return LOMA_ERR_ALIGNMENT;
+    RopeArgs rope;
+    rope.on = 1; rope.pos_seq = positions; rope.stride = 0;
+    rope.log2_base = log2(theta_base > 0.f ? (double)theta_base : 10000.0);
+    return loma_decode_attn_ragged_impl(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, cap, cache_lens,
+                                        max_cache_len, dtype, softmax_scale, flags, workspace, workspace_bytes,
+                                        stream, rope);
 }
 
 // page_size must be a power of two; returns its log2 or -1
@@ -516,10 +541,11 @@ static int log2_exact(int x) {
     return l;
 }
 
-int loma_decode_attn_paged(const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+static int loma_decode_attn_paged_impl(const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
                            const int32_t* block_table, void* o, float* lse, int B, int H, int D, int page_size,
                            int max_pages, int n_pages, const int32_t* cache_lens, int max_cache_len, loma_dtype dtype,
-                           float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes, void* stream) {
+                           float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes, void* stream,
+                                   const RopeArgs& rope) {
     if (B < 0 || H < 0 || max_pages < 0 || n_pages < 0 || max_cache_len < 0) return LOMA_ERR_INVALID_ARG;
     if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
     if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
@@ -544,17 +570,41 @@ int loma_decode_attn_paged(const void* q, const void* k_new, const void* v_new, 
     cudaError_t e;
     if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC))
         e = launch_decode_bf16(q, k_new, v_new, k_pool, v_pool, o, lse, B, H, D, 0, max_cache_len, cache_lens, scale,
-                               workspace, pg, st);
+                               workspace, pg, st, rope);
     else
         e = launch_decode_generic(q, k_new, v_new, k_pool, v_pool, o, lse, B, H, D, 0, max_cache_len, cache_lens, dtype,
-                                  scale, pg, st);
+                                  scale, pg, st, rope);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
 }
 
-int loma_compress_step_paged(const void* q_mem, const void* k_mem, const void* v_mem, void* k_pool, void* v_pool,
+int loma_decode_attn_paged(const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+                           const int32_t* block_table, void* o, float* lse, int B, int H, int D, int page_size,
+                           int max_pages, int n_pages, const int32_t* cache_lens, int max_cache_len, loma_dtype dtype,
+                           float softmax_scale, unsigned flags, void* workspace, size_t workspace_bytes, void* stream) {
+    return loma_decode_attn_paged_impl(q, k_new, v_new, k_pool, v_pool, block_table, o, lse, B, H, D, page_size,
+                                       max_pages, n_pages, cache_lens, max_cache_len, dtype, softmax_scale, flags,
+                                       workspace, workspace_bytes, stream, RopeArgs{});
+}
+
+int loma_decode_attn_paged_rope(const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+                                const int32_t* block_table, void* o, float* lse, int B, int H, int D, int page_size,
+                                int max_pages, int n_pages, const int32_t* cache_lens, int max_cache_len,
+                                const int32_t* positions, float theta_base, loma_dtype dtype, float softmax_scale,
+                                unsigned flags, void* workspace, size_t workspace_bytes, void* stream) {
+    if (B > 0 && H > 0 && (!positions || !k_new || !v_new)) return LOMA_ERR_INVALID_ARG;
+    if ((uintptr_t)positions & 3u) return LOMA_ERR_ALIGNMENT;
+    RopeArgs rope;
+    rope.on = 1; rope.pos_seq = positions; rope.stride = 0;
+    rope.log2_base = log2(theta_base > 0.f ? (double)theta_base : 10000.0);
+    return loma_decode_attn_paged_impl(q, k_new, v_new, k_pool, v_pool, block_table, o, lse, B, H, D, page_size,
+                                       max_pages, n_pages, cache_lens, max_cache_len, dtype, softmax_scale, flags,
+                                       workspace, workspace_bytes, stream, rope);
+}
+
+static int loma_compress_step_paged_impl(const void* q_mem, const void* k_mem, const void* v_mem, void* k_pool, void* v_pool,
                              const int32_t* block_table, void* o_mem, float* lse, int B, int H, int D, int page_size,
                              int max_pages, int n_pages, const int32_t* mem_lens, int max_mem_len, int c, int t, int tc,
-                             loma_dtype dtype, float softmax_scale, unsigned flags, void* stream) {
+                             loma_dtype dtype, float softmax_scale, unsigned flags, void* stream, const RopeArgs& rope) {
     if (B < 0 || H < 0 || max_pages < 0 || n_pages < 0 || max_mem_len < 0 || c < 1 || t < 1) return LOMA_ERR_INVALID_ARG;
     if ((int64_t)c * t != (int64_t)tc) return LOMA_ERR_INVALID_ARG;
     if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
@@ -577,13 +627,39 @@ int loma_compress_step_paged(const void* q_mem, const void* k_mem, const void* v
     Paging pg;
     pg.table = block_table; pg.max_pages = max_pages; pg.log2_ps = l2; pg.n_pages = n_pages;
     cudaError_t e;
-    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC) && t <= 128)
+    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC) && t <= (rope.on ? 16 : 128))
         e = launch_compress_bf16(q_mem, k_mem, v_mem, k_pool, v_pool, o_mem, lse, B, H, D, 0, max_mem_len, mem_lens, c, t, flags,
-                                 scale, nullptr, pg, st);
+                                 scale, nullptr, pg, st, rope);
     else
         e = launch_compress_generic(q_mem, k_mem, v_mem, k_pool, v_pool, o_mem, lse, B, H, D, 0, max_mem_len, mem_lens, c, t,
-                                    dtype, scale, flags, pg, st);
+                                    dtype, scale, flags, pg, st, rope);
+    if (e == cudaErrorNotSupported) return LOMA_ERR_UNSUPPORTED;
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
+int loma_compress_step_paged(const void* q_mem, const void* k_mem, const void* v_mem, void* k_pool, void* v_pool,
+                             const int32_t* block_table, void* o_mem, float* lse, int B, int H, int D, int page_size,
+                             int max_pages, int n_pages, const int32_t* mem_lens, int max_mem_len, int c, int t, int tc,
+                             loma_dtype dtype, float softmax_scale, unsigned flags, void* stream) {
+    return loma_compress_step_paged_impl(q_mem, k_mem, v_mem, k_pool, v_pool, block_table, o_mem, lse, B, H, D,
+                                         page_size, max_pages, n_pages, mem_lens, max_mem_len, c, t, tc, dtype,
+                                         softmax_scale, flags, stream, RopeArgs{});
+}
+
+int loma_compress_step_paged_rope(const void* q_mem, const void* k_mem, const void* v_mem, void* k_pool, void* v_pool,
+                                  const int32_t* block_table, void* o_mem, float* lse, int B, int H, int D,
+                                  int page_size, int max_pages, int n_pages, const int32_t* mem_lens, int max_mem_len,
+                                  int c, int t, int tc, const int32_t* pos0s, int pos_stride, float theta_base,
+                                  loma_dtype dtype, float softmax_scale, unsigned flags, void* stream) {
+    if (pos_stride < 0) return LOMA_ERR_INVALID_ARG;
+    if (B > 0 && H > 0 && !pos0s) return LOMA_ERR_INVALID_ARG;
+    if ((uintptr_t)pos0s & 3u) return LOMA_ERR_ALIGNMENT;
+    RopeArgs rope;
+    rope.on = 1; rope.pos_seq = pos0s; rope.stride = pos_stride;
+    rope.log2_base = log2(theta_base > 0.f ? (double)theta_base : 10000.0);
+    return loma_compress_step_paged_impl(q_mem, k_mem, v_mem, k_pool, v_pool, block_table, o_mem, lse, B, H, D,
+                                         page_size, max_pages, n_pages, mem_lens, max_mem_len, c, t, tc, dtype,
+                                         softmax_scale, flags, stream, rope);
 }
 
 size_t loma_decode_static_scratch_bytes(void) { return decode_static_scratch_bytes(); }
@@ -670,10 +746,10 @@ int loma_compress_step_rope(const void* q_mem, const void* k_mem, const void* v_
                               softmax_scale, flags, workspace, workspace_bytes, stream, rope);
 }
 
-int loma_compress_step_ragged(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
+static int loma_compress_step_ragged_impl(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
                               void* o_mem, float* lse, int B, int H, int D, int cap, const int32_t* mem_lens,
                               int max_mem_len, int c, int t, int tc, loma_dtype dtype, float softmax_scale, unsigned flags,
-                              void* stream) {
+                              void* stream, const RopeArgs& rope) {
     if (B < 0 || H < 0 || cap < 0 || max_mem_len < 0 || c < 1 || t < 1) return LOMA_ERR_INVALID_ARG;
     if ((int64_t)c * t != (int64_t)tc) return LOMA_ERR_INVALID_ARG;
     if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
@@ -691,13 +767,36 @@ int loma_compress_step_ragged(const void* q_mem, const void* k_mem, const void* 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if ((int64_t)B * H * 256 > INT_MAX) return LOMA_ERR_INVALID_ARG;
     cudaError_t e;
-    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC) && t <= 128)
+    if (dtype == LOMA_BF16 && !(flags & LOMA_FLAG_FORCE_GENERIC) && t <= (rope.on ? 16 : 128))
         e = launch_compress_bf16(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, max_mem_len, mem_lens, c, t,
-                                 flags, scale, nullptr, Paging{}, st);
+                                 flags, scale, nullptr, Paging{}, st, rope);
     else
         e = launch_compress_generic(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, max_mem_len, mem_lens,
-                                    c, t, dtype, scale, flags, Paging{}, st);
+                                    c, t, dtype, scale, flags, Paging{}, st, rope);
     return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
+int loma_compress_step_ragged(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache, void* v_cache,
+                              void* o_mem, float* lse, int B, int H, int D, int cap, const int32_t* mem_lens,
+                              int max_mem_len, int c, int t, int tc, loma_dtype dtype, float softmax_scale, unsigned flags,
+                              void* stream) {
+    return loma_compress_step_ragged_impl(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, mem_lens,
+                                          max_mem_len, c, t, tc, dtype, softmax_scale, flags, stream, RopeArgs{});
+}
+
+int loma_compress_step_ragged_rope(const void* q_mem, const void* k_mem, const void* v_mem, void* k_cache,
+                                   void* v_cache, void* o_mem, float* lse, int B, int H, int D, int cap,
+                                   const int32_t* mem_lens, int max_mem_len, int c, int t, int tc,
+                                   const int32_t* pos0s, int pos_stride, float theta_base, loma_dtype dtype,
+                                   float softmax_scale, unsigned flags, void* stream) {
+    if (pos_stride < 0) return LOMA_ERR_INVALID_ARG;
+    if (B > 0 && H > 0 && !pos0s) return LOMA_ERR_INVALID_ARG;
+    if ((uintptr_t)pos0s & 3u) return LOMA_ERR_ALIGNMENT;
+    RopeArgs rope;
+    rope.on = 1; rope.pos_seq = pos0s; rope.stride = pos_stride;
+    rope.log2_base = log2(theta_base > 0.f ? (double)theta_base : 10000.0);
+    return loma_compress_step_ragged_impl(q_mem, k_mem, v_mem, k_cache, v_cache, o_mem, lse, B, H, D, cap, mem_lens,
+                                          max_mem_len, c, t, tc, dtype, softmax_scale, flags, stream, rope);
 }
 
 int loma_selftest_bounded_wait(void* stream) {

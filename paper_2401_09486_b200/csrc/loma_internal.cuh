@@ -71,6 +71,7 @@ struct Paging {
 struct RopeArgs {
     int on = 0;
     int pos0 = 0, stride = 0;
+    const int32_t* pos_seq = nullptr;   // [device] one pos0 per sequence of the batch (ragged batches), or NULL: pos0 for all
     double log2_base = 0.0;   // log2 of the base (10000 by default)
 };
 

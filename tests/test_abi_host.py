@@ -398,3 +398,53 @@ def test_paged_compress_validation(lib):
     assert call(flags=1) == UNSUPPORTED
     assert call(lens=0x8002) == ALIGNMENT
     assert call(B=0) == 0
+
+
+def test_ragged_and_paged_rope_fused_steps_validation(lib):
+    """The per-sequence position arrays are checked on the host like every other pointer, after which the
+    plain step's own checks apply unchanged."""
+    def dec_r(q=0x1000, kn=0x2000, vn=0x3000, kc=0x4000, vc=0x5000, o=0x6000, B=2, H=1, D=128, cap=8, lens=0x7000, mx=3,
+              pos=0x9000, dt=1):
+        return lib.loma_decode_attn_ragged_rope(q, kn, vn, kc, vc, o, None, B, H, D, cap, lens, mx, pos, 0.0, dt, 0.0, 0, None,
+                                                0, None)
+    assert dec_r(pos=None) == INVALID
+    assert dec_r(pos=0x9002) == ALIGNMENT
+    assert dec_r(kn=None, vn=None) == INVALID           # the key to rotate has to be given
+    assert dec_r(mx=8) == CAPACITY
+    assert dec_r(lens=None) == INVALID
+    assert dec_r(D=100) == UNSUPPORTED
+    assert dec_r(B=0) == 0
+
+    def dec_p(q=0x1000, kn=0x2000, vn=0x3000, kp=0x4000, vp=0x5000, bt=0x6000, o=0x7000, B=2, H=1, D=128, ps=16, mp=4, npg=8,
+              lens=0x8000, mx=40, pos=0x9000, dt=1):
+        return lib.loma_decode_attn_paged_rope(q, kn, vn, kp, vp, bt, o, None, B, H, D, ps, mp, npg, lens, mx, pos, 0.0, dt,
+                                               0.0, 0, None, 0, None)
+    assert dec_p(pos=None) == INVALID
+    assert dec_p(pos=0x9001) == ALIGNMENT
+    assert dec_p(kn=None, vn=None) == INVALID
+    assert dec_p(ps=24) == INVALID
+    assert dec_p(mx=64) == CAPACITY
+    assert dec_p(B=0) == 0
+
+    def cmp_r(qm=0x1000, km=0x2000, vm=0x3000, kc=0x4000, vc=0x5000, om=0x6000, B=2, H=1, D=128, cap=100, lens=0x7000,
+              mx=16, c=4, t=16, tc=64, pos0s=0x9000, stride=4, dt=1, flags=0):
+        return lib.loma_compress_step_ragged_rope(qm, km, vm, kc, vc, om, None, B, H, D, cap, lens, mx, c, t, tc, pos0s, stride,
+                                                  0.0, dt, 0.0, flags, None)
+    assert cmp_r(pos0s=None) == INVALID
+    assert cmp_r(pos0s=0x9002) == ALIGNMENT
+    assert cmp_r(stride=-1) == INVALID
+    assert cmp_r(cap=79) == CAPACITY
+    assert cmp_r(tc=63) == INVALID
+    assert cmp_r(flags=1) == UNSUPPORTED
+    assert cmp_r(B=0) == 0
+
+    def cmp_p(qm=0x1000, km=0x2000, vm=0x3000, kp=0x4000, vp=0x5000, bt=0x6000, om=0x7000, B=2, H=1, D=128, ps=16, mp=8,
+              npg=16, lens=0x8000, mx=16, c=4, t=16, tc=64, pos0s=0x9000, stride=4, dt=1, flags=0):
+        return lib.loma_compress_step_paged_rope(qm, km, vm, kp, vp, bt, om, None, B, H, D, ps, mp, npg, lens, mx, c, t, tc,
+                                                 pos0s, stride, 0.0, dt, 0.0, flags, None)
+    assert cmp_p(pos0s=None) == INVALID
+    assert cmp_p(pos0s=0x9003) == ALIGNMENT
+    assert cmp_p(stride=-3) == INVALID
+    assert cmp_p(mx=65) == CAPACITY
+    assert cmp_p(ps=48) == INVALID
+    assert cmp_p(B=0) == 0

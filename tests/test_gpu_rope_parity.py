@@ -240,3 +240,114 @@ def test_generation_with_fused_rotation_equals_rotated_one_shot_forward(ptype, d
     zone = oracle.layout_index(n, c, t, tail)[1]
     live = zone != oracle.ZONE_REP
     check(got[:, :, torch.from_numpy(live).to(DEV)], want_o[:, :, live], dtype)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, L.LOMA_FLAG_FORCE_GENERIC])
+def test_ragged_steps_with_fused_rotation_match_the_oracle_per_sequence(flags, dtype):
+    """One cache length, one position (decode) or one first memory id (compress) per sequence."""
+    B, H, D, c, t = 4, 2, 128, 4, 16
+    tc = c * t
+    cap = 700
+    lens = [0, 17, 613, 250]
+    poss = [0, 90, 20001, 1234]
+    kc = synthetic.normal_tensor((B, H, cap, D), 101, 1.0, dtype)
+    vc = synthetic.normal_tensor((B, H, cap, D), 102, 1.0, dtype)
+    q, kn, vn = synthetic.qkv(B, H, 1, D, seed=103, std=1.0, dtype=dtype)
+    kcd, vcd = kc.to(DEV), vc.to(DEV)
+    o = torch.full((B, H, 1, D), float("nan"), dtype=dtype, device=DEV)
+    ws = torch.empty(max(16, L.loma_decode_workspace_bytes(B, H, D, max(lens))), dtype=torch.uint8, device=DEV)
+    L.loma_decode_attn_ragged_rope(q.to(DEV), kn.to(DEV), vn.to(DEV), kcd, vcd, o, None,
+                                   torch.tensor(lens, dtype=torch.int32, device=DEV), max(lens),
+                                   torch.tensor(poss, dtype=torch.int32, device=DEV), ws, flags)
+    torch.cuda.synchronize()
+    for b in range(B):
+        sl = slice(b, b + 1)
+        q_rot = oracle.rope_rotate(npf(q[sl]), [poss[b]])
+        k_rot = oracle.rope_rotate(npf(kn[sl]), [poss[b]])
+        want, _, _, _ = oracle.decode_attn(q_rot, _round_to(k_rot, dtype), npf(vn[sl]), npf(kc[sl]), npf(vc[sl]), lens[b])
+        check(o[sl], want, dtype)
+        _ulp_close(kcd[sl, :, lens[b]], k_rot[:, :, 0], dtype)
+        assert torch.equal(vcd[b, :, lens[b]].cpu(), vn[b, :, 0])
+    # compress: sequences 0 and 2 compress now, 1 and 3 do not
+    mem_lens = [32, -1, 160, -1]
+    pos0s = [2 * tc + c - 1, 0, 10 * tc + c - 1, 0]
+    kc2 = synthetic.normal_tensor((B, H, cap, D), 104, 1.0, dtype)
+    vc2 = synthetic.normal_tensor((B, H, cap, D), 105, 1.0, dtype)
+    qm, km, vm = synthetic.qkv(B, H, t, D, seed=106, std=1.0, dtype=dtype)
+    kcd, vcd = kc2.to(DEV), vc2.to(DEV)
+    om = torch.full((B, H, t, D), float("nan"), dtype=dtype, device=DEV)
+    L.loma_compress_step_ragged_rope(qm.to(DEV), km.to(DEV), vm.to(DEV), kcd, vcd, om, None,
+                                     torch.tensor(mem_lens, dtype=torch.int32, device=DEV), max(mem_lens), c, t,
+                                     torch.tensor(pos0s, dtype=torch.int32, device=DEV), c, flags)
+    torch.cuda.synchronize()
+    for b in range(B):
+        sl = slice(b, b + 1)
+        if mem_lens[b] < 0:
+            assert torch.equal(kcd[sl].cpu(), kc2[sl]) and torch.equal(vcd[sl].cpu(), vc2[sl])     # left alone
+            continue
+        pos = [pos0s[b] + j * c for j in range(t)]
+        q_rot, k_rot = oracle.rope_rotate(npf(qm[sl]), pos), oracle.rope_rotate(npf(km[sl]), pos)
+        want, _, _, _ = oracle.compress_step(q_rot, _round_to(k_rot, dtype), npf(vm[sl]), npf(kc2[sl]), npf(vc2[sl]), mem_lens[b], c, t)
+        check(om[sl], want, dtype)
+        _ulp_close(kcd[sl, :, mem_lens[b]:mem_lens[b] + t], k_rot, dtype)
+        assert torch.equal(vcd[sl, :, mem_lens[b]:mem_lens[b] + t].cpu(), vm[sl])
+        assert torch.equal(kcd[sl, :, :mem_lens[b]].cpu(), kc2[sl, :, :mem_lens[b]])
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_staggered_sequences_over_a_paged_cache_with_fused_rotation(dtype):
+    """Three sequences that started 0, 5 and 11 tokens apart share one pool of pages; every step decodes one token of
+    every sequence at that sequence's own position id and a sequence compresses (memory ids of Eq. 14) as soon as its
+    tail is full: every reading and memory row equals the one-shot forward over Q and K rotated at the layout's ids."""
+    H, D, n, c, t, tail, ps = 2, 128, 3, 2, 8, 5, 16
+    tc, s = c * t, oracle.chunk_len(c, t)
+    S = oracle.seq_len(n, c, t, tail)
+    B, starts = 3, [0, 5, 11]
+    q, k, v = synthetic.qkv(B, H, S, D, seed=111, std=1.0, dtype=dtype)
+    wq, wk = oracle.rope_apply(npf(q), npf(k), n, c, t, tail)
+    want_o, _ = oracle.masked_attn_fwd(wq, wk, npf(v), n, c, t, tail)
+    ids = oracle.position_ids(n, c, t, tail)
+    zone = oracle.layout_index(n, c, t, tail)[1]
+    gen_rows = [i for i in range(S) if zone[i] == oracle.ZONE_READ]
+    max_pages = (n * t + tc + ps - 1) // ps + 1
+    n_pages = B * max_pages
+    table = np.random.default_rng(4).permutation(n_pages).reshape(B, max_pages).astype(np.int32)
+    kpool = torch.zeros((n_pages, H, ps, D), dtype=dtype, device=DEV)
+    vpool = torch.zeros_like(kpool)
+    table_d = torch.from_numpy(table).to(DEV)
+    qd, kd, vd = q.to(DEV), k.to(DEV), v.to(DEV)
+    got = torch.full((B, H, S, D), float("nan"), dtype=dtype, device=DEV)
+    ws = torch.empty(max(16, L.loma_decode_workspace_bytes(B, H, D, n * t + tc)), dtype=torch.uint8, device=DEV)
+    i32 = lambda xs: torch.tensor(xs, dtype=torch.int32, device=DEV)
+    nxt, lens, chunks, step = [0] * B, [0] * B, [0] * B, 0
+    while any(p_ < len(gen_rows) for p_ in nxt):
+        active = [step >= starts[b] and nxt[b] < len(gen_rows) for b in range(B)]
+        rows = [gen_rows[min(nxt[b], len(gen_rows) - 1)] for b in range(B)]
+        take = lambda x: torch.stack([x[b, :, rows[b]:rows[b] + 1] for b in range(B)]).contiguous()
+        o1 = torch.empty((B, H, 1, D), dtype=dtype, device=DEV)
+        # idle sequences decode a throw-away token into a spare slot of their own pages (their length does not advance)
+        L.loma_decode_attn_paged_rope(take(qd), take(kd), take(vd), kpool, vpool, table_d, o1, None, i32(lens), max(lens),
+                                      i32([int(ids[r]) for r in rows]), ws)
+        for b in range(B):
+            if active[b]:
+                got[b, :, rows[b]] = o1[b, :, 0]
+                nxt[b] += 1
+                lens[b] += 1
+        mem_lens = [chunks[b] * t if (lens[b] == chunks[b] * t + tc and chunks[b] < n) else -1 for b in range(B)]
+        if any(m >= 0 for m in mem_lens):
+            m_rows = [chunks[b] * s + tc for b in range(B)]
+            takem = lambda x: torch.stack([x[b, :, m_rows[b]:m_rows[b] + t] if mem_lens[b] >= 0 else x[b, :, :t]
+                                           for b in range(B)]).contiguous()
+            om = torch.empty((B, H, t, D), dtype=dtype, device=DEV)
+            L.loma_compress_step_paged_rope(takem(qd), takem(kd), takem(vd), kpool, vpool, table_d, om, None, i32(mem_lens),
+                                            max(mem_lens), c, t, i32([int(ids[min(m_rows[b], S - 1)]) for b in range(B)]), c)
+            for b in range(B):
+                if mem_lens[b] >= 0:
+                    got[b, :, m_rows[b]:m_rows[b] + t] = om[b]
+                    chunks[b] += 1
+                    lens[b] = chunks[b] * t
+        step += 1
+    torch.cuda.synchronize()
+    live = zone != oracle.ZONE_REP
+    check(got[:, :, torch.from_numpy(live).to(DEV)], want_o[:, :, live], dtype)
