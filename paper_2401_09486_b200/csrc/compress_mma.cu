@@ -378,6 +378,215 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
     }
 }
 
+// ------------------------------------------------------------------ default mask, short ranges: the range in one stage
+// Default mask and t <= 16: the key range of a (b,h) is the tc tail rows plus the t memory rows' own keys
+// (80 keys for c = 4, t = 16).  A range that short fits one stage: the CTA (one per (b,h)) issues every load
+// at once and walks no pipeline.  The warps split the scores by key (8 keys per tensor-core tile), the softmax
+// runs over full rows held in shared memory (8 threads per row), and each warp then owns D/4 output columns
+// over all keys: nothing is merged across warps.  The compaction writes the staged (with the fused rotary
+// embedding: rotated) copies of the memory rows, so k_mem / v_mem are read once.  56 KB of shared memory at
+// 80 keys: four CTAs (16 warps) per SM.  (A persistent CTA that loads the next (b,h) while it computes the
+// current one was measured slower: its two buffers leave two CTAs per SM, too few warps to cover the
+// latencies of the arithmetic.)
+struct CmpOneStageLayout {
+    int rowb;       // padded K / V / Q row in bytes: conflict-free ldmatrix
+    int srow;       // fp32 scores per row
+    int prowb;      // bf16 probabilities per row, padded like the operand rows
+    int kv_bytes;   // K rows, V rows, Q rows
+    int s_off, p_off, ml_off, rope_off, total;
+};
+__host__ __device__ inline CmpOneStageLayout cmp_one_stage_layout(int D, int nk16, bool rope) {
+    CmpOneStageLayout l;
+    l.rowb = D * 2 + 16;
+    l.srow = nk16 + 4;
+    l.prowb = nk16 * 2 + 16;
+    l.kv_bytes = (2 * nk16 + 16) * l.rowb;
+    l.s_off = l.kv_bytes;
+    l.p_off = l.s_off + 16 * l.srow * 4;
+    l.ml_off = l.p_off + 16 * l.prowb;
+    l.rope_off = l.ml_off + 32 * 4;
+    l.total = l.rope_off + (rope ? 16 * (D / 2) * 8 : 0);
+    return l;
+}
+constexpr int CMP_ONE_STAGE_MAX_SMEM = 72 * 1024;   // at least three CTAs per SM; longer ranges take the pipelined kernel
+
+template <int D>
+__global__ void __launch_bounds__(CMP_WARPS * 32)
+compress_one_stage_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16* __restrict__ k_mem,
+                      const __nv_bfloat16* __restrict__ v_mem, __nv_bfloat16* __restrict__ k_cache,
+                      __nv_bfloat16* __restrict__ v_cache, __nv_bfloat16* __restrict__ o_mem, float* __restrict__ lse,
+                      int cap, int mem_len_all, const int32_t* __restrict__ mem_lens, int H, int t, int tc,
+                      float scale_log2, Paging pg, RopeArgs rope) {
+    constexpr int VPR = D / 8;                 // 16-byte vectors per row
+    constexpr int NTH = CMP_WARPS * 32;
+    extern __shared__ __align__(16) uint8_t smem[];
+    const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(smem);
+    const int nkeys = tc + t;
+    const int nk16 = (nkeys + 15) & ~15;           // rows past nkeys are zero: their probabilities are zero too
+    const CmpOneStageLayout lay = cmp_one_stage_layout(D, nk16, rope.on != 0);
+    const int ROWB = lay.rowb;
+    const int K_OFF = 0, V_OFF = nk16 * ROWB, Q_OFF = 2 * nk16 * ROWB;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3, mi = lane >> 3;
+
+    // ragged batch: every sequence has its own count of memory entries, clamped to the bound the caller vouched
+    // for; a negative count means the sequence does not compress in this call
+    auto own_mem_len = [&](int bh) -> int {
+        if (!mem_lens) return mem_len_all;
+        const int m = __ldg(mem_lens + bh / H);
+        return m < 0 ? -1 : min(m, mem_len_all);
+    };
+    // cache slot j of (b,h) -> element offset from k_cache / v_cache (through the block table when the cache is paged)
+    auto cache_row = [&](int bh, int j) -> int64_t {
+        if (!pg.table) return ((int64_t)bh * cap + j) * D;
+        const int pb = bh / H, phd = bh - pb * H;
+        const int page = min(max(__ldg(pg.table + (int64_t)pb * pg.max_pages + (j >> pg.log2_ps)), 0), pg.n_pages - 1);
+        return ((((int64_t)page * H + phd) << pg.log2_ps) + (j & ((1 << pg.log2_ps) - 1))) * D;
+    };
+    const int bh = blockIdx.x;
+    const int mem_len = own_mem_len(bh);
+    if (mem_len < 0) return;
+    // every load at once: the tail rows of the cache, the memory rows' own keys and values, the queries
+    const uint32_t base = sbase;
+    const __nv_bfloat16* km = k_mem + (int64_t)bh * t * D;
+    const __nv_bfloat16* vm = v_mem + (int64_t)bh * t * D;
+    for (int e = threadIdx.x; e < nk16 * VPR; e += NTH) {
+        const int r = e / VPR, cv = e - r * VPR;
+        const bool valid = r < nkeys;
+        const __nv_bfloat16 *ksrc = km, *vsrc = vm;
+        if (valid) {
+            if (r < tc) { const int64_t off = cache_row(bh, mem_len + r); ksrc = k_cache + off; vsrc = v_cache + off; }
+            else { ksrc = km + (int64_t)(r - tc) * D; vsrc = vm + (int64_t)(r - tc) * D; }
+        }
+        cp_async16(base + K_OFF + r * ROWB + cv * 16, ksrc + cv * 8, valid);
+        cp_async16(base + V_OFF + r * ROWB + cv * 16, vsrc + cv * 8, valid);
+    }
+    for (int e = threadIdx.x; e < 16 * VPR; e += NTH) {
+        const int r = e / VPR, cv = e - r * VPR;
+        const bool valid = r < t;          // query rows >= t are zero
+        cp_async16(base + Q_OFF + r * ROWB + cv * 16, q_mem + ((int64_t)bh * t + (valid ? r : 0)) * D + cv * 8, valid);
+    }
+    cp_async_commit();
+
+    float* S = reinterpret_cast<float*>(smem + lay.s_off);
+    float* ml = reinterpret_cast<float*>(smem + lay.ml_off);
+    float2* rope_tab = reinterpret_cast<float2*>(smem + lay.rope_off);
+
+    // Fused rotary embedding (Section 4.5), as in compress_mma_kernel: memory row j turns by the id
+    // pos0 + j * stride; the table is computed while the loads are in flight.
+    if (rope.on) {
+        const int pos0 = rope.pos_seq ? __ldg(rope.pos_seq + bh / H) : rope.pos0;
+        for (int e = threadIdx.x; e < t * (D / 2); e += NTH) {
+            const int r = e / (D / 2), d = e - r * (D / 2);
+            float c, sn;
+            rope_cos_sin(pos0 + r * rope.stride, d, D, rope.log2_base, c, sn);
+            rope_tab[e] = make_float2(c, sn);
+        }
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+    if (rope.on) {
+        // the queries and the staged copies of the memory rows' own keys, each pair of features once
+        for (int e = threadIdx.x; e < 2 * t * (D / 2); e += NTH) {
+            const int which = e / (t * (D / 2)), e2 = e - which * t * (D / 2);
+            const int r = e2 / (D / 2), d = e2 - r * (D / 2);
+            __nv_bfloat16* x = reinterpret_cast<__nv_bfloat16*>(smem + (which ? K_OFF + (tc + r) * ROWB : Q_OFF + r * ROWB));
+            const float2 cs = rope_tab[r * (D / 2) + d];
+            const float a = __bfloat162float(x[d]), b = __bfloat162float(x[d + D / 2]);
+            x[d] = __float2bfloat16_rn(a * cs.x - b * cs.y);
+            x[d + D / 2] = __float2bfloat16_rn(b * cs.x + a * cs.y);
+        }
+        __syncthreads();
+    }
+    // Compaction (Section 3.1 step 3): this CTA is the only reader of cache slots [mem_len, mem_len + t) of
+    // this (b,h) in the launch and its copies of them have landed; the slots now take the staged memory rows.
+    for (int e = threadIdx.x; e < t * VPR; e += NTH) {
+        const int r = e / VPR, cv = e - r * VPR;
+        const int64_t off = cache_row(bh, mem_len + r) + cv * 8;
+        *reinterpret_cast<uint4*>(k_cache + off) = *reinterpret_cast<const uint4*>(smem + K_OFF + (tc + r) * ROWB + cv * 16);
+        *reinterpret_cast<uint4*>(v_cache + off) = *reinterpret_cast<const uint4*>(smem + V_OFF + (tc + r) * ROWB + cv * 16);
+    }
+
+    // scores: tensor-core tiles of 8 keys, dealt to the warps round robin
+    {
+        uint32_t qa[D / 16][4];
+        const uint32_t qrow = base + Q_OFF + ((mi & 1) * 8 + (lane & 7)) * ROWB + (mi >> 1) * 16;
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) ldsm_x4(qrow + kk * 32, qa[kk]);
+        for (int nt = warp; nt < nk16 / 8; nt += CMP_WARPS) {
+            float sc[4] = {0.f, 0.f, 0.f, 0.f};
+            const uint32_t krow = base + K_OFF + (nt * 8 + (lane & 7)) * ROWB + mi * 16;
+#pragma unroll
+            for (int k2 = 0; k2 < D / 32; ++k2) {
+                uint32_t kf[4];   // 8 keys x 32 features: the B fragments of two k-steps
+                ldsm_x4(krow + k2 * 64, kf);
+                mma_bf16_16816(sc, qa[2 * k2], kf[0], kf[1]);
+                mma_bf16_16816(sc, qa[2 * k2 + 1], kf[2], kf[3]);
+            }
+            const int col = nt * 8 + 2 * tq;
+            const bool v0 = col < nkeys, v1 = col + 1 < nkeys;
+            *reinterpret_cast<float2*>(S + g * lay.srow + col) =
+                make_float2(v0 ? sc[0] * scale_log2 : -INFINITY, v1 ? sc[1] * scale_log2 : -INFINITY);
+            *reinterpret_cast<float2*>(S + (g + 8) * lay.srow + col) =
+                make_float2(v0 ? sc[2] * scale_log2 : -INFINITY, v1 ? sc[3] * scale_log2 : -INFINITY);
+        }
+    }
+    __syncthreads();
+    // softmax over full rows (exp2 domain): 8 threads per row, two passes over the row in shared memory;
+    // key 0 is valid for every row, so the maximum is finite
+    {
+        const int r = threadIdx.x >> 3, sub = threadIdx.x & 7;
+        const float* srow = S + r * lay.srow;
+        __nv_bfloat16* prow = reinterpret_cast<__nv_bfloat16*>(smem + lay.p_off + r * lay.prowb);
+        float mx = -INFINITY;
+        for (int j = sub; j < nk16; j += 8) mx = fmaxf(mx, srow[j]);
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+        float sum = 0.f;
+        for (int j = sub; j < nk16; j += 8) {
+            const float pr = ex2f(srow[j] - mx);
+            sum += pr;
+            prow[j] = __float2bfloat16_rn(pr);
+        }
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+        if (sub == 0) { ml[r] = mx; ml[16 + r] = sum; }
+    }
+    __syncthreads();
+    // O = P V: each warp owns D/4 output columns over every key
+    {
+        constexpr int NT = D / 32;             // 8-column tiles per warp
+        float oacc[NT][4];
+#pragma unroll
+        for (int j = 0; j < NT; ++j) { oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f; }
+        const uint32_t prow = sbase + lay.p_off + ((mi & 1) * 8 + (lane & 7)) * lay.prowb + (mi >> 1) * 16;
+        const uint32_t vrow = base + V_OFF + ((mi & 1) * 8 + (lane & 7)) * ROWB + (mi >> 1) * 16 + warp * (D / 4) * 2;
+        for (int ks = 0; ks < nk16 / 16; ++ks) {
+            uint32_t pa[4];
+            ldsm_x4(prow + ks * 32, pa);
+#pragma unroll
+            for (int jd = 0; jd < NT; jd += 2) {
+                uint32_t vf[4];
+                ldsm_x4_trans(vrow + ks * 16 * ROWB + jd * 16, vf);
+                mma_bf16_16816(oacc[jd], pa, vf[0], vf[1]);
+                mma_bf16_16816(oacc[jd + 1], pa, vf[2], vf[3]);
+            }
+        }
+        const float inv0 = 1.f / ml[16 + g], inv1 = 1.f / ml[16 + g + 8];
+        __nv_bfloat16* o0 = o_mem + ((int64_t)bh * t + g) * D + warp * (D / 4) + 2 * tq;
+        __nv_bfloat16* o1 = o0 + 8 * D;
+#pragma unroll
+        for (int jd = 0; jd < NT; ++jd) {
+            if (g < t) *reinterpret_cast<uint32_t*>(o0 + jd * 8) = pack_bf16(oacc[jd][0] * inv0, oacc[jd][1] * inv0);
+            if (g + 8 < t) *reinterpret_cast<uint32_t*>(o1 + jd * 8) = pack_bf16(oacc[jd][2] * inv1, oacc[jd][3] * inv1);
+        }
+    }
+    if (lse && threadIdx.x < t)
+        lse[(int64_t)bh * t + threadIdx.x] = (ml[threadIdx.x] + log2f(ml[16 + threadIdx.x])) * 0.6931471805599453f;
+}
+
 template <int D>
 __global__ void __launch_bounds__(D)
 compress_merge_kernel(const float* __restrict__ ws, __nv_bfloat16* __restrict__ o_mem, float* __restrict__ lse,
@@ -440,6 +649,25 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
     int prior_len = 0;
     if (nprior > 0) prior_len = ((mem_len + nprior - 1) / nprior + 15) / 16 * 16;
     const int nsp = nprior + 1;
+    const CmpOneStageLayout wl = cmp_one_stage_layout(D, (tc + t + 15) & ~15, rope.on != 0);
+    if (nprior == 0 && t <= 16 && wl.total <= CMP_ONE_STAGE_MAX_SMEM) {
+        // default mask, short range: the whole range in one stage
+        static bool attr1_set[64] = {false};   // per device, per template instance
+        int dev1 = 0;
+        if (cudaGetDevice(&dev1) != cudaSuccess || dev1 < 0 || dev1 >= 64) return cudaErrorInvalidDevice;
+        if (!attr1_set[dev1]) {
+            cudaError_t e1 = cudaFuncSetAttribute(compress_one_stage_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                  CMP_ONE_STAGE_MAX_SMEM);
+            if (e1 != cudaSuccess) return e1;
+            attr1_set[dev1] = true;
+        }
+        compress_one_stage_kernel<D><<<BH, CMP_WARPS * 32, wl.total, st>>>(
+            static_cast<const __nv_bfloat16*>(qm), static_cast<const __nv_bfloat16*>(km),
+            static_cast<const __nv_bfloat16*>(vm), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
+            static_cast<__nv_bfloat16*>(om), lse, cap, mem_len, mem_lens, H, t, tc, scale * 1.4426950408889634f, pg, rope);
+        count_launches(1);
+        return cudaGetLastError();
+    }
     // (the cos/sin table of the fused rotary embedding is only allocated when it is used: without it three CTAs fit an SM)
     const int smem = rope.on ? CmpSmem<D>::TOTAL : CmpSmem<D>::ROPE_OFF;
     cudaError_t e;
