@@ -408,17 +408,20 @@ __host__ __device__ inline CmpOneStageLayout cmp_one_stage_layout(int D, int nk1
     l.total = l.rope_off + (rope ? 16 * (D / 2) * 8 : 0);
     return l;
 }
-constexpr int CMP_ONE_STAGE_MAX_SMEM = 72 * 1024;   // at least three CTAs per SM; longer ranges take the pipelined kernel
+constexpr int CMP_ONE_STAGE_MAX_SMEM = 72 * 1024;       // three CTAs of four warps per SM
+constexpr int CMP_ONE_STAGE_MAX_SMEM_8W = 110 * 1024;   // two CTAs of eight warps per SM; longer ranges take the pipelined kernel
 
-template <int D>
-__global__ void __launch_bounds__(CMP_WARPS * 32)
+template <int D, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32)
 compress_one_stage_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16* __restrict__ k_mem,
                       const __nv_bfloat16* __restrict__ v_mem, __nv_bfloat16* __restrict__ k_cache,
                       __nv_bfloat16* __restrict__ v_cache, __nv_bfloat16* __restrict__ o_mem, float* __restrict__ lse,
                       int cap, int mem_len_all, const int32_t* __restrict__ mem_lens, int H, int t, int tc,
                       float scale_log2, Paging pg, RopeArgs rope) {
     constexpr int VPR = D / 8;                 // 16-byte vectors per row
-    constexpr int NTH = CMP_WARPS * 32;
+    constexpr int NTH = WARPS * 32;
+    constexpr int TPR = NTH / 16;              // threads per row in the softmax
+    static_assert(D % (8 * WARPS) == 0 && (D / (8 * WARPS)) % 2 == 0, "a warp owns an even number of 8-column tiles");
     extern __shared__ __align__(16) uint8_t smem[];
     const uint32_t sbase = (uint32_t)__cvta_generic_to_shared(smem);
     const int nkeys = tc + t;
@@ -513,7 +516,7 @@ compress_one_stage_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bf
         const uint32_t qrow = base + Q_OFF + ((mi & 1) * 8 + (lane & 7)) * ROWB + (mi >> 1) * 16;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) ldsm_x4(qrow + kk * 32, qa[kk]);
-        for (int nt = warp; nt < nk16 / 8; nt += CMP_WARPS) {
+        for (int nt = warp; nt < nk16 / 8; nt += WARPS) {
             float sc[4] = {0.f, 0.f, 0.f, 0.f};
             const uint32_t krow = base + K_OFF + (nt * 8 + (lane & 7)) * ROWB + mi * 16;
 #pragma unroll
@@ -532,19 +535,20 @@ compress_one_stage_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bf
         }
     }
     __syncthreads();
-    // softmax over full rows (exp2 domain): 8 threads per row, two passes over the row in shared memory;
+    // softmax over full rows (exp2 domain): TPR threads per row, two passes over the row in shared memory;
     // key 0 is valid for every row, so the maximum is finite
     {
-        const int r = threadIdx.x >> 3, sub = threadIdx.x & 7;
+        const int r = threadIdx.x / TPR, sub = threadIdx.x % TPR;
         const float* srow = S + r * lay.srow;
         __nv_bfloat16* prow = reinterpret_cast<__nv_bfloat16*>(smem + lay.p_off + r * lay.prowb);
         float mx = -INFINITY;
-        for (int j = sub; j < nk16; j += 8) mx = fmaxf(mx, srow[j]);
+        for (int j = sub; j < nk16; j += TPR) mx = fmaxf(mx, srow[j]);
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+        if (TPR == 16) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
         float sum = 0.f;
-        for (int j = sub; j < nk16; j += 8) {
+        for (int j = sub; j < nk16; j += TPR) {
             const float pr = ex2f(srow[j] - mx);
             sum += pr;
             prow[j] = __float2bfloat16_rn(pr);
@@ -552,17 +556,18 @@ compress_one_stage_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bf
         sum += __shfl_xor_sync(0xffffffffu, sum, 1);
         sum += __shfl_xor_sync(0xffffffffu, sum, 2);
         sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+        if (TPR == 16) sum += __shfl_xor_sync(0xffffffffu, sum, 8);
         if (sub == 0) { ml[r] = mx; ml[16 + r] = sum; }
     }
     __syncthreads();
-    // O = P V: each warp owns D/4 output columns over every key
+    // O = P V: each warp owns D / WARPS output columns over every key
     {
-        constexpr int NT = D / 32;             // 8-column tiles per warp
+        constexpr int NT = D / (8 * WARPS);     // 8-column tiles per warp
         float oacc[NT][4];
 #pragma unroll
         for (int j = 0; j < NT; ++j) { oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f; }
         const uint32_t prow = sbase + lay.p_off + ((mi & 1) * 8 + (lane & 7)) * lay.prowb + (mi >> 1) * 16;
-        const uint32_t vrow = base + V_OFF + ((mi & 1) * 8 + (lane & 7)) * ROWB + (mi >> 1) * 16 + warp * (D / 4) * 2;
+        const uint32_t vrow = base + V_OFF + ((mi & 1) * 8 + (lane & 7)) * ROWB + (mi >> 1) * 16 + warp * (D / WARPS) * 2;
         for (int ks = 0; ks < nk16 / 16; ++ks) {
             uint32_t pa[4];
             ldsm_x4(prow + ks * 32, pa);
@@ -575,7 +580,7 @@ compress_one_stage_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bf
             }
         }
         const float inv0 = 1.f / ml[16 + g], inv1 = 1.f / ml[16 + g + 8];
-        __nv_bfloat16* o0 = o_mem + ((int64_t)bh * t + g) * D + warp * (D / 4) + 2 * tq;
+        __nv_bfloat16* o0 = o_mem + ((int64_t)bh * t + g) * D + warp * (D / WARPS) + 2 * tq;
         __nv_bfloat16* o1 = o0 + 8 * D;
 #pragma unroll
         for (int jd = 0; jd < NT; ++jd) {
@@ -650,18 +655,25 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
     if (nprior > 0) prior_len = ((mem_len + nprior - 1) / nprior + 15) / 16 * 16;
     const int nsp = nprior + 1;
     const CmpOneStageLayout wl = cmp_one_stage_layout(D, (tc + t + 15) & ~15, rope.on != 0);
-    if (nprior == 0 && t <= 16 && wl.total <= CMP_ONE_STAGE_MAX_SMEM) {
-        // default mask, short range: the whole range in one stage
+    if (nprior == 0 && t <= 16 && wl.total <= (D == 128 ? CMP_ONE_STAGE_MAX_SMEM_8W : CMP_ONE_STAGE_MAX_SMEM)) {
+        // default mask, short range: the whole range in one stage; four warps while three CTAs fit an SM, eight
+        // (D = 128 only: a warp owns at least 16 output columns) while two do
+        constexpr int W8 = D == 128 ? 8 : 4;
+        const bool wide = wl.total > CMP_ONE_STAGE_MAX_SMEM;
         static bool attr1_set[64] = {false};   // per device, per template instance
         int dev1 = 0;
         if (cudaGetDevice(&dev1) != cudaSuccess || dev1 < 0 || dev1 >= 64) return cudaErrorInvalidDevice;
         if (!attr1_set[dev1]) {
-            cudaError_t e1 = cudaFuncSetAttribute(compress_one_stage_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            cudaError_t e1 = cudaFuncSetAttribute(compress_one_stage_kernel<D, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                   CMP_ONE_STAGE_MAX_SMEM);
+            if (e1 == cudaSuccess)
+                e1 = cudaFuncSetAttribute(compress_one_stage_kernel<D, W8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          CMP_ONE_STAGE_MAX_SMEM_8W);
             if (e1 != cudaSuccess) return e1;
             attr1_set[dev1] = true;
         }
-        compress_one_stage_kernel<D><<<BH, CMP_WARPS * 32, wl.total, st>>>(
+        auto kern = wide ? compress_one_stage_kernel<D, W8> : compress_one_stage_kernel<D, 4>;
+        kern<<<BH, (wide ? W8 : 4) * 32, wl.total, st>>>(
             static_cast<const __nv_bfloat16*>(qm), static_cast<const __nv_bfloat16*>(km),
             static_cast<const __nv_bfloat16*>(vm), static_cast<__nv_bfloat16*>(kc), static_cast<__nv_bfloat16*>(vc),
             static_cast<__nv_bfloat16*>(om), lse, cap, mem_len, mem_lens, H, t, tc, scale * 1.4426950408889634f, pg, rope);
