@@ -367,9 +367,10 @@ def run_ours(args):
              # dram__bytes_read.sum + dram__bytes_write.sum of one launch on one batch element of this layout x B
              "traffic": FWD_SHORT_TRAFFIC_B1 * f["B"],
              "tensor_frac_of_measured_bf16_useful": fwd_tflops / world / peaks["bf16_tflops"]},
-            {"kernel": "compress_mma_kernel<128>", "workload": "B32 H32 mem 8192, default variant", "bound": "hbm",
+            {"kernel": "compress_one_stage_kernel<128, 4>", "workload": "B32 H32 mem 8192, default variant", "bound": "hbm",
              "achieved": cmp_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": cmp_gbs / peaks["hbm_gbs"],
-             "traffic": None, "note": "launch-latency bound: 59 MB in one ~35 us launch"},
+             # dram__bytes_read.sum + dram__bytes_write.sum of one launch at this very size (the 12.6 MB it writes stay in L2)
+             "traffic": COMPRESS_TRAFFIC_B32, "note": "59 MB in one launch of 1024 CTAs, four resident per SM: two waves"},
         ],
         "e2e": {"value": world * fwd_flops / (e2e_fwd * 1e-3) / 1e12, "unit": "TFLOP/s",
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_tot,
@@ -660,13 +661,14 @@ def large_workloads(L, synthetic, torch, dev, peaks, steps, warmup, clocks_mhz):
                      # every (b, h) streams its own rows once: the B8 / 8224-row capture scaled by rows and (b, h) pairs
                      "traffic": DECODE_TRAFFIC_B8_L8224 * (B * H / 256.0) * ((mem_len + tc / 2.0 + 0.5) / 8224.0),
                      "traffic_source": "ncu small case scaled by (b,h) pairs and rows"},
-        "roofline_compress": {"kernel": "compress_mma_kernel<128>", "bound": "hbm", "achieved": cmp_gbs, "peak": peaks["hbm_gbs"],
+        "roofline_compress": {"kernel": "compress_one_stage_kernel<128, 8>", "bound": "hbm", "achieved": cmp_gbs, "peak": peaks["hbm_gbs"],
                               "unit": "GB/s", "frac": cmp_gbs / peaks["hbm_gbs"], "traffic": None,
                               "note": "0.19 GB in one launch right after the decodes of the cycle"}}
     return out
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from ncu captures of the --profile-case launches
+COMPRESS_TRAFFIC_B32 = 46.28e6         # compress_one_stage_kernel<128, 4>, B32 H32, c4 t16 (58.7e6 algorithmic, 46.1e6 of them reads)
 DECODE_TRAFFIC_B8_L8224 = 1.0824e9     # decode_splitkv + merge, B8 H32, 8224 rows (1.0779e9 algorithmic)
 FWD_SHORT_TRAFFIC_B1 = 141.5e6         # masked_attn_tc, one batch element of the 4608-token layout (151.0e6 algorithmic)
 FWD_LONG_TRAFFIC_8_HEADS = 706.2e6     # masked_attn_tc, 8 heads of the 69632-token layout (570.4e6 algorithmic)
@@ -686,8 +688,10 @@ def profile_case(args):
     D = 128
     std = 1.0 / math.sqrt(D)
     case = args.profile_case
-    if case in ("decode", "compress", "compress_prior"):
+    if case in ("decode", "compress", "compress_prior", "compress_b32"):
         B, H, c, t, mem_len = 8, 32, 4, 16, 8192          # 1/4 of the generation workload's batch: 1.08 GB of cache
+        if case == "compress_b32":
+            B = 32                                         # the generation workload's own batch (1024 CTAs: two waves), 4.3 GB
         tc = c * t
         cap = mem_len + tc + t
         kc = synthetic.big_normal_(torch.empty(B, H, cap, D, dtype=bf, device=dev), 1, std)
@@ -813,7 +817,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-extras", action="store_true", help="skip the large and the context workloads timed at N=1")
-    ap.add_argument("--profile-case", choices=["decode", "compress", "compress_prior", "masked", "masked_long", "bwd", "bwd_long"],
+    ap.add_argument("--profile-case", choices=["decode", "compress", "compress_prior", "compress_b32", "masked", "masked_long", "bwd", "bwd_long"],
                     help="run one cut-down kernel launch sequence (for profiler captures) and exit")
     ap.add_argument("--reps", type=int, default=3, help="launches of --profile-case")
     args = ap.parse_args()
