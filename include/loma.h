@@ -534,7 +534,7 @@ LOMA_API int loma_compress_step_paged(const void* q_mem, const void* k_mem, cons
  *     allocating routine is reached from it.
  *   - The first call on each device looks up the array's device address
  *     (cudaGetSymbolAddress, with that device current) and caches it.  Make
- *     that first call during set-up, before any stream capture begins.
+ *     that first call during set-up.
  *   - All calls share the one array.  Nothing in it has to be cleared between
  *     calls (every partial that is read has been written by the same call),
  *     but two calls that can overlap on the GPU -- different streams without an

@@ -76,6 +76,31 @@ def test_static_scratch_decode_matches_workspace_decode_twice_in_a_row():
     assert L.loma_device_status() == 0
 
 
+def test_static_scratch_decode_leaves_the_device_memory_as_it_found_it():
+    """After the set-up call a further call changes neither the driver's count of free device memory nor
+    the caching allocator's: everything it touches was there before."""
+    if not torch.cuda.is_available():
+        pytest.fail("GPU tests need a CUDA device")
+    build.build_library()
+    torch.cuda.set_device(0)
+    B, H, D, cap, cache_len = 4, 8, 128, 6000, 5555
+    kc = synthetic.normal_tensor((B, H, cap, D), 920, 1.0, torch.bfloat16).to(DEV)
+    vc = synthetic.normal_tensor((B, H, cap, D), 921, 1.0, torch.bfloat16).to(DEV)
+    q, kn, vn = (x.to(DEV) for x in synthetic.qkv(B, H, 1, D, seed=922, dtype=torch.bfloat16))
+    o = torch.empty(B, H, 1, D, dtype=torch.bfloat16, device=DEV)
+    L.loma_decode_attn_static(q, kn, vn, kc, vc, o, None, cache_len)        # set-up call on this device
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for step in range(3):
+        L.loma_decode_attn_static(q, kn, vn, kc, vc, o, None, cache_len + 1 + step)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == (alloc0, reserved0)
+    assert L.loma_device_status() == 0
+
+
 def test_static_scratch_decode_rejects_requests_beyond_its_array():
     if not torch.cuda.is_available():
         pytest.fail("GPU tests need a CUDA device")
