@@ -27,6 +27,20 @@
 #include "tcgen05_common.cuh"
 
 namespace loma {
+// Work item -> key tile rank and (batch, head) in the dK/dV kernel, whose tiles are dealt statically.  Pair by
+// pair, as in the other kernels, while a pair has fewer key tiles than there are CTAs (several pairs are then in
+// flight and each pair's Q / dO stay in L2: 3 % on the 4608-token layout); one rank for every pair before the
+// next rank otherwise: with 544 key tiles per pair of which 32 are a hundred times longer than the rest, the
+// static deal is only even when those come first for all pairs (2 % on the 69632-token layout).
+__device__ __forceinline__ void split_key_work(const FwdParams& p, int w, int& rank, int& bh) {
+    if (p.total_tiles <= (int)gridDim.x) { split_work(p, w, rank, bh); return; }
+    rank = fdiv(w, p.dBH);
+    bh = w - rank * p.BH;
+}
+}  // namespace loma
+
+
+namespace loma {
 
 struct BwdMaps {
     CUtensorMap q[4], k[4], v[4], g[4], dq[4];   // g = dO
@@ -128,7 +142,8 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
             uint32_t gs = 0, tcount = 0;
             bool ok = true;
             for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
-                const int rank = fdiv(w, p.dBH), bh = w - rank * p.BH;
+                int rank, bh;
+                split_work(p, w, rank, bh);
                 const int bi = fdiv(bh, p.dH), hi = bh - bi * p.H;
                 TileDesc td;
                 decode_tile(p, rank, td);
@@ -175,7 +190,8 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
         const uint64_t qd = smem_desc(smem_base + SM::Q_OFF, 16, 1024);
         const uint64_t gd = smem_desc(smem_base + SM::G_OFF, 16, 1024);
         for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
-            const int rank = fdiv(w, p.dBH);
+            int rank, bh_;
+            split_work(p, w, rank, bh_);
             TileDesc td;
             decode_tile(p, rank, td);
             const HalfMasks hm = tile_half_masks(p, td, lane);
@@ -220,7 +236,8 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
         uint32_t gs = 0, ge = 0;
         bool ok = true;
         for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r)) {
-            const int rank = fdiv(w, p.dBH);
+            int rank, bh_;
+            split_work(p, w, rank, bh_);
             TileDesc td;
             decode_tile(p, rank, td);
             const HalfMasks hm = tile_half_masks(p, td, lane);
@@ -259,7 +276,8 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
         bool ok = true;
         bool store_pending = false;
         for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
-            const int rank = fdiv(w, p.dBH), bh = w - rank * p.BH;
+            int rank, bh;
+            split_work(p, w, rank, bh);
             const int bi = fdiv(bh, p.dH), hi = bh - bi * p.H;
             TileDesc td;
             decode_tile(p, rank, td);
@@ -447,7 +465,8 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
             uint32_t gs = 0, tcount = 0;
             bool ok = true;
             for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
-                const int rank = fdiv(w, p.dBH), bh = w - rank * p.BH;
+                int rank, bh;
+                split_key_work(p, w, rank, bh);
                 const int bi = fdiv(bh, p.dH), hi = bh - bi * p.H;
                 KeyTileDesc kd;
                 decode_key_tile(p, rank, kd);
@@ -489,7 +508,8 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
         const uint64_t kd_ = smem_desc(smem_base + K_OFF, 16, 1024);
         const uint64_t vd_ = smem_desc(smem_base + V_OFF, 16, 1024);
         for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
-            const int rank = fdiv(w, p.dBH);
+            int rank, bh_;
+            split_key_work(p, w, rank, bh_);
             KeyTileDesc kd;
             decode_key_tile(p, rank, kd);
             const HalfMasks hm = key_tile_half_masks(p, kd, lane);
@@ -532,7 +552,8 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
         uint32_t gs = 0, ge = 0;
         bool ok = true;
         for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r)) {
-            const int rank = fdiv(w, p.dBH);
+            int rank, bh_;
+            split_key_work(p, w, rank, bh_);
             KeyTileDesc kd;
             decode_key_tile(p, rank, kd);
             const HalfMasks hm = key_tile_half_masks(p, kd, lane);
@@ -574,7 +595,8 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
         bool ok = true;
         bool store_pending = false;
         for (int r = 0, w = sid; w < total_work && ok; w = tile_of_round(++r), ++tcount) {
-            const int rank = fdiv(w, p.dBH), bh = w - rank * p.BH;
+            int rank, bh;
+            split_key_work(p, w, rank, bh);
             const int bi = fdiv(bh, p.dH), hi = bh - bi * p.H;
             KeyTileDesc kd;
             decode_key_tile(p, rank, kd);

@@ -39,8 +39,8 @@
 //                     S_h of the next step is issued right after P_h V_h of this one, so the
 //                     tensor pipe works on one half while the warpgroup works on the other.
 // The two streams fill each other's waits (tensor latency, TMEM loads, epilogues).  Tiles are handed
-// out at run time from one counter over a statically ordered list (longest first, (batch, head)
-// fastest): a stream that finishes a tile draws the next (without a counter, see the host side, the tiles are
+// out at run time from one counter over a statically ordered list ((batch, head) by (batch, head), each
+// pair's tiles longest first): a stream that finishes a tile draws the next (without a counter, see the host side, the tiles are
 // dealt round robin).  Every mbarrier wait is bounded: on expiry the CTA records LOMA_ERR_TIMEOUT, all
 // roles leave their loops, TMEM is freed and the kernel returns.
 #include "tcgen05_common.cuh"
@@ -114,9 +114,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     const uint32_t tmem = tmem_slot + st * 256;   // this stream's scores at +0, output accumulator at +128
     volatile int* abortp = &abort_flag;
 
-    // Tiles (longest first) are dealt to the 2*gridDim.x streams in rounds, forwards in even rounds
-    // and backwards in odd ones, so no stream always receives the longest tile of a round.
-    // Tiles are handed out from one counter, longest first ((batch, head) fastest inside a rank): a stream
+    // Tiles are handed out from one counter, pair by pair and longest first inside a (batch, head): a stream
     // that finishes early simply takes the next one.  The stream's producer draws the number and posts it
     // in a four-slot ring (barrier B_TF + (n & 1), completion n >> 1, for the stream's n-th tile); the MMA
     // issuer and the warpgroup read it there.  A negative number ends the stream.  Which stream computes a
@@ -142,7 +140,8 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 __threadfence_block();
                 mbar_arrive(bar(B_TF + (tcount & 1)));
                 if (w < 0) break;
-                const int rank = fdiv(w, p.dBH), bh = w - rank * p.BH;
+                int rank, bh;
+                split_work(p, w, rank, bh);
                 const int bi = fdiv(bh, p.dH), hi = bh - bi * p.H;
                 TileDesc td;
                 decode_tile(p, rank, td);
@@ -227,7 +226,8 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             for (;; ++tcount) {
                 const int w = next_tile(tcount, ok);
                 if (w < 0) break;
-                const int rank = fdiv(w, p.dBH);
+                int rank, bh_unused;
+                split_work(p, w, rank, bh_unused);
                 TileDesc td;
                 decode_tile(p, rank, td);
                 const HalfMasks hm = tile_half_masks(p, td, lane);
@@ -287,8 +287,8 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             bool row_valid;
         };
         auto decode_ctx = [&](int w, TileCtx& c) {
-            const int rank = fdiv(w, p.dBH);
-            c.bh = w - rank * p.BH;
+            int rank;
+            split_work(p, w, rank, c.bh);
             c.bi = fdiv(c.bh, p.dH);
             c.hi = c.bh - c.bi * p.H;
             decode_tile(p, rank, c.td);

@@ -61,12 +61,24 @@ struct FwdParams {
     int n_tail, n_read, n_mem, n_rep;   // tiles per view, in scheduling order
     unsigned flags;
     int prefill;       // 1: the plan of loma_prefill_attn (query view V_TAIL over the new tokens, key view V_MEM over the cache)
-    FastDiv dBH, dH;
+    FastDiv dBH, dH, dTT;   // division by BH, H and total_tiles
     float scale_log2;
     float* lse;
     int* status;
     unsigned* sched;   // [0] next tile to hand out, [1] CTAs that have finished (the last one clears both); NULL = static deal
 };
+
+// Work item w of a launch -> tile rank and (batch, head): the tiles of one (b,h) are handed out together,
+// longest first, before the next pair's.  The streams of the whole GPU then work on one or two pairs at a
+// time, whose K and V (35 MB per head on the 69632-token layout, 4.4 MB per pair for a prompt piece over
+// 8192 cache rows) stay in L2 while every tile of the pair streams them: each row is fetched from HBM once.
+// (Handing out one rank for every (b,h) before the next rank -- longest tiles first over the whole launch --
+// kept all pairs in flight at once: the prompt piece then read its cache four times and was bound by that,
+// 2.82 ms against 2.22 ms, and the 69632-token layout took 1.40 ms against 1.32 ms.)
+__host__ __device__ __forceinline__ void split_work(const FwdParams& p, int w, int& rank, int& bh) {
+    bh = fdiv(w, p.dTT);
+    rank = w - bh * p.total_tiles;
+}
 
 
 struct Seg {
@@ -367,7 +379,7 @@ inline void make_plan(const Layout& L, int B, int H, FwdParams* p) {
     p->n_mem = p->view[V_MEM].ntiles; p->n_rep = p->view[V_REP].ntiles;
     p->total_tiles = p->n_tail + p->n_read + p->n_mem + p->n_rep;
     p->flags = L.flags; p->prefill = 0;
-    p->dBH = make_fastdiv(p->BH); p->dH = make_fastdiv(H);
+    p->dBH = make_fastdiv(p->BH); p->dH = make_fastdiv(H); p->dTT = make_fastdiv(p->total_tiles);
 }
 
 // The plan of loma_prefill_attn: l new tokens (query view V_TAIL, one "chunk" of l rows) over a cache that holds
@@ -383,7 +395,7 @@ inline void make_prefill_plan(int l, int cache_len, int B, int H, FwdParams* p) 
     p->n_tail = p->view[V_TAIL].ntiles; p->n_read = 0; p->n_mem = 0; p->n_rep = 0;
     p->total_tiles = p->n_tail;
     p->flags = 0; p->prefill = 1;
-    p->dBH = make_fastdiv(p->BH); p->dH = make_fastdiv(H);
+    p->dBH = make_fastdiv(p->BH); p->dH = make_fastdiv(H); p->dTT = make_fastdiv(p->total_tiles);
 }
 
 }  // namespace loma
