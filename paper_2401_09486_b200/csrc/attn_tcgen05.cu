@@ -414,13 +414,26 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             if (ok) tc_fence_after();
 
             // epilogue: normalise, round to bf16, stage 64 output columns at a time in shared
-            // memory, TMA store.  Every thread of the warpgroup reaches the first barrier for
-            // every tile it started; it also makes giving up a uniform decision.
+            // memory, TMA store.  A panel's 64 columns are fetched from TMEM with one wait and packed
+            // before the thread that issued the previous panel's store waits for that store to have
+            // read the staging panel, so the wait is covered by the fetch.  Every thread of the
+            // warpgroup reaches the first barrier for every tile it started; it also makes giving up
+            // a uniform decision.
             const float inv = 1.f / l;
             uint8_t* orow = smem_gen + SM::O_OFF + rr * 128;
             bool give_up = false;
 #pragma unroll
             for (int pn = 0; pn < PANELS; ++pn) {
+                uint32_t pk[32];
+                {
+                    uint32_t r[64];
+                    tmem_ld32(o_addr + pn * 64, r);
+                    tmem_ld32(o_addr + pn * 64 + 32, r + 32);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        pk[e] = pack_bf16(__uint_as_float(r[2 * e]) * inv, __uint_as_float(r[2 * e + 1]) * inv);
+                }
                 if (rr == 0 && store_pending) tma_store_wait_read();   // the staging panel is free again
                 if (pn == 0) {
                     uint32_t any_bad;
@@ -434,21 +447,9 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     asm volatile("bar.sync %0, 128;" ::"r"(1 + st) : "memory");
                 }
 #pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(o_addr + pn * 64 + c * 32, r);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int q4 = 0; q4 < 4; ++q4) {
-                        const int ci = c * 4 + q4;       // 16-byte chunk of the 128-byte panel row
-                        uint4 u;
-                        u.x = pack_bf16(__uint_as_float(r[q4 * 8 + 0]) * inv, __uint_as_float(r[q4 * 8 + 1]) * inv);
-                        u.y = pack_bf16(__uint_as_float(r[q4 * 8 + 2]) * inv, __uint_as_float(r[q4 * 8 + 3]) * inv);
-                        u.z = pack_bf16(__uint_as_float(r[q4 * 8 + 4]) * inv, __uint_as_float(r[q4 * 8 + 5]) * inv);
-                        u.w = pack_bf16(__uint_as_float(r[q4 * 8 + 6]) * inv, __uint_as_float(r[q4 * 8 + 7]) * inv);
-                        *reinterpret_cast<uint4*>(orow + ((ci ^ (rr & 7)) << 4)) = u;
-                    }
-                }
+                for (int ci = 0; ci < 8; ++ci)           // 16-byte chunk of the 128-byte panel row
+                    *reinterpret_cast<uint4*>(orow + ((ci ^ (rr & 7)) << 4)) =
+                        make_uint4(pk[ci * 4], pk[ci * 4 + 1], pk[ci * 4 + 2], pk[ci * 4 + 3]);
                 fence_async_smem();
                 asm volatile("bar.sync %0, 128;" ::"r"(1 + st) : "memory");
                 if (rr == 0) {
