@@ -330,19 +330,42 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     const int b = ge & 1;
                     const int lo_h = lo - 64 * hw.h;                  // allowed columns of this half: [lo_h, lo_h + span)
                     const uint32_t span = (uint32_t)(hi2 - lo);
-                    const bool full = __all_sync(0xffffffffu, lo_h <= 0 && hi2 - 64 * hw.h >= 64);
+                    const int hi_h = hi2 - 64 * hw.h;
+                    const bool full = __all_sync(0xffffffffu, lo_h <= 0 && hi_h >= 64);
+                    // no row of this warp has an allowed column in this half (the other warps of the tile do):
+                    // e.g. three of the four warps of a memory-zone tile at every reading half it visits
+                    const bool none = __all_sync(0xffffffffu, hi_h <= 0 || lo_h >= 64 || hi2 <= lo);
                     ok = __all_sync(0xffffffffu, mbar_wait(bar(B_SF + b), (ge >> 1) & 1, abortp, p.status));
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t sh_addr = s_addr + b * 64;
+                    if (none) {
+                        // probabilities of zero for the warp's rows; the running maximum and sum stay as they are
+                        uint32_t z[16];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) z[e] = 0u;
+                        tmem_st16(sh_addr, z);
+                        tmem_st16(sh_addr + 16, z);
+                        tmem_wait_st();
+                        tc_fence_before();
+                        mbar_arrive(bar(B_PF + b));
+                        continue;
+                    }
                     uint32_t s[64];
                     tmem_ld32(sh_addr, s);
                     tmem_ld32(sh_addr + 32, s + 32);
                     tmem_wait_ld();
                     if (!full) {
+                        if (__all_sync(0xffffffffu, lo_h <= 0)) {
+                            // only an upper bound in this warp (causal and chunk-prefix masks): one compare per score
 #pragma unroll
-                        for (int e = 0; e < 64; ++e)
-                            if ((uint32_t)(e - lo_h) >= span) s[e] = 0xff800000u;   // -inf: blocked for this row
+                            for (int e = 0; e < 64; ++e)
+                                if (e >= hi_h) s[e] = 0xff800000u;   // -inf: blocked for this row
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 64; ++e)
+                                if ((uint32_t)(e - lo_h) >= span) s[e] = 0xff800000u;
+                        }
                     }
                     float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
