@@ -427,7 +427,9 @@ def other_workloads(L, synthetic, torch, dev, peaks):
     res["masked_fwd_69632"] = {"config": dict(B=B, H=H, D=D, n=n, c=c, t=t, S=S), "ms": ms,
                                "useful_tflops": flops / (ms * 1e-3) / 1e12,
                                "frac_of_measured_bf16": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                               "gbs": 4.0 * q.numel() * 2 / (ms * 1e-3) / 1e9}
+                               "gbs": 4.0 * q.numel() * 2 / (ms * 1e-3) / 1e9,
+                               "note": "single calls, each after an idle gap (the GPU's clock may not have ramped up): "
+                                       "the steady-state figure of this workload is large_workloads.masked_fwd_69632"}
 
     def backward(tag, B, H, n, c, t, q, k, v, o):
         # gradients of the same layout (useful FLOPs: five products of the allowed pairs, 10*D per pair)
