@@ -308,7 +308,13 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t s_addr = lane_addr + b * 64, g_addr = lane_addr + 128 + b * 64;
-                {
+                // no row of this warp sees any of its 32 columns of this half: dA = 0, nothing to read
+                if (__all_sync(0xffffffffu, hi2 - 64 * hw.h <= wg * 32 || lo_h >= wg * 32 + 32 || hi2 <= lo)) {
+                    uint32_t z[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) z[e] = 0u;
+                    tmem_st16(s_addr + wg * 32, z);
+                } else {
                     const int c = wg;
                     uint32_t s[32], g[32], pk[16];
                     tmem_ld32(s_addr + c * 32, s);
@@ -638,7 +644,14 @@ masked_attn_bwd_dkv_tc_kernel(const __grid_constant__ BwdKvMaps maps, const BwdP
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t s_addr = lane_addr + b * 64, g_addr = lane_addr + 128 + b * 64;
-                {
+                // no key row of this warp is seen by any of its 32 query rows of this half: P^T = dA^T = 0
+                if (__all_sync(0xffffffffu, hi2 - 64 * hw.h <= wg * 32 || lo_h >= wg * 32 + 32 || hi2 <= lo)) {
+                    uint32_t z[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) z[e] = 0u;
+                    tmem_st16(s_addr + wg * 32, z);
+                    tmem_st16(g_addr + wg * 32, z);
+                } else {
                     const int c = wg;
                     uint32_t s[32], g[32], ppk[16], dpk[16];
                     tmem_ld32(s_addr + c * 32, s);
