@@ -3,8 +3,9 @@
 // Appendix A), fused with the in-place compaction of the cache (step 3).
 //
 // With t = 16 query rows per key row the step has ~16 flop per byte: it is bound
-// by HBM (or, for the short default variant, by launch latency), but too heavy
-// for the CUDA cores when the prior-memory variant streams the whole cache.  The
+// by HBM (the short default variant by the latency of one CTA's chain of loads
+// and phases: it has a kernel of its own further down, compress_one_stage_kernel),
+// but too heavy for the CUDA cores when the prior-memory variant streams the whole cache.  The
 // 16 queries are exactly one M = 16 tile of the warp-level tensor-core
 // instruction (mma.sync.m16n8k16); the 128-row tcgen05 tile would idle 7/8 of
 // the array here, so this kernel uses the warp-level path on purpose.
