@@ -157,23 +157,36 @@ decode_splitkv_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
 
+    // Paged cache: a row's address hangs on a block-table entry.  The entries of the next iteration's rows are
+    // fetched while this iteration's rows stream in, so no data load waits for a table load issued just before it.
+    int64_t off_cur[DEC_NL], off_nxt[DEC_NL];
+    auto row_offs = [&](int j0, int64_t* o) {
+#pragma unroll
+        for (int i = 0; i < DEC_NL; ++i) o[i] = row_off(min(min(j0 + i * KPL + sub, cache_len), max(cache_len - 1, 0)));
+    };
+    if (PAGED) row_offs(k_begin + warp * BK, off_cur);
     for (int j0 = k_begin + warp * BK; j0 < k_end; j0 += DEC_WARPS * BK) {
         uint4 kr[DEC_NL], vr[DEC_NL];
         bool valid[DEC_NL];
+        if (PAGED) row_offs(j0 + DEC_WARPS * BK, off_nxt);
 #pragma unroll
         for (int i = 0; i < DEC_NL; ++i) {
             const int j = j0 + i * KPL + sub;
             valid[i] = j < k_end;
             const int jc = min(j, cache_len);                  // stay inside [0, cache_len]
-            const uint4* kp = (jc < cache_len) ? kc + row_off(jc) : kn;
+            const uint4* kp = (jc < cache_len) ? kc + (PAGED ? off_cur[i] : row_off(jc)) : kn;
             if (rope.on && jc >= cache_len) kr[i] = *(reinterpret_cast<const uint4*>(sm_kn) + li);   // the rotated new key
             else kr[i] = ld_stream(kp + li);
         }
 #pragma unroll
         for (int i = 0; i < DEC_NL; ++i) {
             const int jc = min(j0 + i * KPL + sub, cache_len);
-            const uint4* vp = (jc < cache_len) ? vc + row_off(jc) : vn;
+            const uint4* vp = (jc < cache_len) ? vc + (PAGED ? off_cur[i] : row_off(jc)) : vn;
             vr[i] = ld_stream(vp + li);
+        }
+        if (PAGED) {
+#pragma unroll
+            for (int i = 0; i < DEC_NL; ++i) off_cur[i] = off_nxt[i];
         }
         float s[DEC_NL];
 #pragma unroll
