@@ -361,7 +361,7 @@ def run_ours(args):
                      "traffic": DECODE_TRAFFIC_B8_L8224 * (g["B"] * g["H"]) / 256.0,
                      "traffic_source": "ncu small case x4"},
         "roofline_other_kernels": [
-            {"kernel": "masked_attn_tc_kernel<128>", "workload": "4608-token layout", "bound": "hbm",
+            {"kernel": "masked_attn_tc_kernel<128, false>", "workload": "4608-token layout", "bound": "hbm",
              "achieved": fwd_bytes / (t_fwd * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
              "frac": fwd_bytes / (t_fwd * 1e-3) / 1e9 / peaks["hbm_gbs"],
              # dram__bytes_read.sum + dram__bytes_write.sum of one launch on one batch element of this layout x B
@@ -553,6 +553,15 @@ def other_workloads(L, synthetic, torch, dev, peaks):
                                         "frac_of_measured_bf16": fl / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                                         "gbs": nbytes / (ms * 1e-3) / 1e9,
                                         "kernels": "cache_append_kernel + masked_attn_tc_kernel (prefill plan)"}
+    if hasattr(L, "loma_prefill_attn_ragged"):
+        # the same piece with one cache length per sequence (8192 minus up to 1023 entries)
+        lens_p = torch.tensor([kp - (37 * b) % 1024 for b in range(Bp)], dtype=torch.int32, device=dev)
+        ms = timed(lambda: L.loma_prefill_attn_ragged(qp, knp, vnp, kcp, vcp, op, None, lens_p, kp, 0, 0.0, stream))
+        fl = 4.0 * D * H * float(sum(lp * int(n) + lp * (lp + 1) // 2 for n in lens_p.tolist()))
+        res["prefill_ragged_512_over_8192_B32"] = {"config": dict(B=Bp, H=H, D=D, l=lp, cache_lens="8192 - (37 b) mod 1024"),
+                                                   "ms": ms, "useful_tflops": fl / (ms * 1e-3) / 1e12,
+                                                   "frac_of_measured_bf16": fl / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                                                   "kernels": "cache_append_kernel + masked_attn_tc_kernel<128, true>"}
     del kcp, vcp, qp, knp, vnp, op
     torch.cuda.empty_cache()
     for name, flags in (("compress_B64_16k", 0), ("compress_B64_16k_prior_mem", 1)):
@@ -606,7 +615,7 @@ def large_workloads(L, synthetic, torch, dev, peaks, steps, warmup, clocks_mhz):
     out["masked_fwd_69632"] = {
         "config": dict(B=B, H=H, D=D, n=n, c=c, t=t, S=S), "steps": steps, "ms": ms, "ms_min": min(ts),
         "ms_x_sm_ghz": ms * ghz if ghz else None, "useful_tflops": tf, "useful_flops": flops, "compulsory_bytes": nbytes,
-        "roofline": {"kernel": "masked_attn_tc_kernel<128>", "bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"],
+        "roofline": {"kernel": "masked_attn_tc_kernel<128, false>", "bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"],
                      "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst bf16)",
                      "frac_of_sustained": tf / peaks["bf16_tflops_sustained"],
                      # dram bytes of one launch on the 8-head case of this layout (ncu), times 4 for 32 heads

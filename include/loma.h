@@ -433,6 +433,38 @@ LOMA_API int loma_prefill_attn(const void* q, const void* k_new, const void* v_n
                                void* o, float* lse, int B, int H, int D, int l, int cap, int cache_len,
                                loma_dtype dtype, float softmax_scale, unsigned flags, void* stream);
 
+/* ---------------------------------------------------------------------------
+ * loma_prefill_attn_ragged, loma_prefill_attn_paged -- the same step (Appendix A,
+ * `inference_input` with l > 1 tokens) for a batch whose sequences hold different numbers
+ * of entries, over a contiguous or a paged cache: one run of the generator per sequence,
+ * each feeding l tokens.  Sequence b appends its l rows at entries
+ * [cache_lens[b], cache_lens[b] + l) and its new token i sees entries 0 .. cache_lens[b] + i.
+ *
+ *   cache_lens [device, in]  int32 [B]: entries of every sequence before the call; values are
+ *                            clamped to [0, max_cache_len] on the device
+ *   max_cache_len            a bound on cache_lens that the caller vouches for (work is sized by it)
+ *   ragged: k_cache, v_cache [B, H, cap, D] as in loma_prefill_attn.  bf16 calls with l >= 8 run on
+ *           the tensor-core kernel; for them the call also sets the entries from each
+ *           sequence's new end up to the next multiple of 128 (at most cap) to zero: that
+ *           kernel reads them (with weight zero), and the contents of the cache past a
+ *           sequence's valid length are unspecified anyway.
+ *   paged:  k_pool, v_pool [n_pages, H, page_size, D] and block_table int32 [B, max_pages] as in
+ *           loma_decode_attn_paged (page numbers clamped to the pool); CUDA cores, one warp per
+ *           new row, for every dtype.
+ * Other arguments, outputs and errors as loma_prefill_attn; CAPACITY when max_cache_len + l
+ * exceeds cap (ragged) or max_pages * page_size (paged); INVALID_ARG for a missing table or
+ * length array or a page size that is not a power of two.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_prefill_attn_ragged(const void* q, const void* k_new, const void* v_new, void* k_cache,
+                                      void* v_cache, void* o, float* lse, int B, int H, int D, int l, int cap,
+                                      const int32_t* cache_lens, int max_cache_len, loma_dtype dtype,
+                                      float softmax_scale, unsigned flags, void* stream);
+LOMA_API int loma_prefill_attn_paged(const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+                                     const int32_t* block_table, void* o, float* lse, int B, int H, int D, int l,
+                                     int page_size, int max_pages, int n_pages, const int32_t* cache_lens,
+                                     int max_cache_len, loma_dtype dtype, float softmax_scale, unsigned flags,
+                                     void* stream);
+
 /* Host-only replay of the tile plan the tensor-core kernel follows for loma_prefill_attn
  * (Appendix A, inference_input mask): counts[i*(cache_len+l) + j] = number of visits in
  * which new token i attends to key j, into a [host] uint8 buffer of l*(cache_len+l) bytes.

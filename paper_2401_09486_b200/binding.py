@@ -41,6 +41,8 @@ SIGNATURES = {
     "loma_masked_attn_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
     "loma_masked_attn_bwd_plan_coverage": (_i, [_i, _i, _i, _i, _u, _p]),
     "loma_prefill_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _f, _u, _p]),
+    "loma_prefill_attn_ragged": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p]),
+    "loma_prefill_attn_paged": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p]),
     "loma_prefill_attn_plan_coverage": (_i, [_i, _i, _p]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_attn_layers": (_i, [_i, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
@@ -237,6 +239,38 @@ def loma_prefill_attn(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len: int,
                                  B, H, D, l, k_cache.shape[2], int(cache_len), _dtype_code(q), float(softmax_scale),
                                  int(flags), _stream(stream))
     _check(rc, "loma_prefill_attn")
+
+
+def loma_prefill_attn_ragged(q, k_new, v_new, k_cache, v_cache, o, lse, cache_lens, max_cache_len: int, flags: int = 0,
+                             softmax_scale: float = 0.0, stream=None) -> None:
+    """loma_prefill_attn with one cache length per sequence (cache_lens: int32 [B] on the device)."""
+    B, H, l, D = q.shape
+    for x in (q, k_new, v_new, k_cache, v_cache, o):
+        if x is not None and not x.is_contiguous():
+            raise ValueError("loma_prefill_attn_ragged takes contiguous tensors")
+    if cache_lens.dtype != torch.int32 or cache_lens.numel() != B or not cache_lens.is_contiguous():
+        raise ValueError("cache_lens must be a contiguous int32 tensor of B entries")
+    rc = lib().loma_prefill_attn_ragged(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse),
+                                        B, H, D, l, k_cache.shape[2], _ptr(cache_lens), int(max_cache_len), _dtype_code(q),
+                                        float(softmax_scale), int(flags), _stream(stream))
+    _check(rc, "loma_prefill_attn_ragged")
+
+
+def loma_prefill_attn_paged(q, k_new, v_new, k_pool, v_pool, block_table, o, lse, cache_lens, max_cache_len: int,
+                            flags: int = 0, softmax_scale: float = 0.0, stream=None) -> None:
+    """loma_prefill_attn over a paged cache: pools [n_pages, H, page_size, D], block_table int32 [B, max_pages]."""
+    B, H, l, D = q.shape
+    for x in (q, k_new, v_new, k_pool, v_pool, o, block_table):
+        if x is not None and not x.is_contiguous():
+            raise ValueError("loma_prefill_attn_paged takes contiguous tensors")
+    if cache_lens.dtype != torch.int32 or cache_lens.numel() != B or block_table.dtype != torch.int32:
+        raise ValueError("cache_lens and block_table must be int32")
+    n_pages, _, page_size, _ = k_pool.shape
+    rc = lib().loma_prefill_attn_paged(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool), _ptr(block_table),
+                                       _ptr(o), _ptr(lse), B, H, D, l, page_size, block_table.shape[1], n_pages,
+                                       _ptr(cache_lens), int(max_cache_len), _dtype_code(q), float(softmax_scale),
+                                       int(flags), _stream(stream))
+    _check(rc, "loma_prefill_attn_paged")
 
 
 def loma_prefill_attn_plan_coverage(l: int, cache_len: int) -> torch.Tensor:

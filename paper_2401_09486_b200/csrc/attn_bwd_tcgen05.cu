@@ -299,7 +299,7 @@ masked_attn_bwd_dq_tc_kernel(const __grid_constant__ BwdMaps maps, const BwdPara
                 if (hw.first_of_step(hm)) {
                     KTile kt;
                     step_ktile(p, td, hw.j, kt);
-                    row_interval(p.view[kt.view], kt, rc, ro, rr, row_valid, lo, hi2);
+                    row_interval(p.view[kt.view], kt, rc, ro, rr, row_valid, lo, hi2, p.view[kt.view].diag);
                 }
                 const int b = ge & 1;
                 const int lo_h = lo - 64 * hw.h;

@@ -311,41 +311,69 @@ decode_generic_kernel(const T* __restrict__ q, const T* __restrict__ k_new, cons
 // sees cache rows 0 .. len + i.
 template <typename T>
 struct CacheRangeMap {
-    const T* kc;
+    const T* kc;   // the (b,h)'s cache (contiguous) or the pool (paged)
     const T* vc;
     int D;
-    __device__ __forceinline__ const T* kptr(int vi) const { return kc + (int64_t)vi * D; }
-    __device__ __forceinline__ const T* vptr(int vi) const { return vc + (int64_t)vi * D; }
+    Paging pg;
+    int b, h, H;
+    __device__ __forceinline__ int64_t slot(int j) const {
+        if (!pg.table) return (int64_t)j * D;
+        const int page = min(max(pg.table[(int64_t)b * pg.max_pages + (j >> pg.log2_ps)], 0), pg.n_pages - 1);
+        return ((((int64_t)page * H + h) << pg.log2_ps) + (j & ((1 << pg.log2_ps) - 1))) * D;
+    }
+    __device__ __forceinline__ const T* kptr(int vi) const { return kc + slot(vi); }
+    __device__ __forceinline__ const T* vptr(int vi) const { return vc + slot(vi); }
 };
 
+// lens (device, [B], or NULL): every sequence's own number of earlier entries, clamped to [0, cache_len]
 template <typename T, int D>
 __global__ void __launch_bounds__(GENERIC_WARPS * 32)
 prefill_generic_kernel(const T* __restrict__ q, const T* __restrict__ k_cache, const T* __restrict__ v_cache,
-                       T* __restrict__ o, float* __restrict__ lse, int l, int cap, int cache_len, float scale) {
+                       T* __restrict__ o, float* __restrict__ lse, int l, int cap, int cache_len,
+                       const int32_t* __restrict__ lens, int H, Paging pg, float scale) {
     __shared__ __align__(16) float q_sh[GENERIC_WARPS][D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int i = blockIdx.x * GENERIC_WARPS + warp;
     if (i >= l) return;
     const int bh = blockIdx.y;
     CacheRangeMap<T> map;
-    map.kc = k_cache + (int64_t)bh * cap * D;
-    map.vc = v_cache + (int64_t)bh * cap * D;
-    map.D = D;
+    map.b = bh / H; map.h = bh - map.b * H; map.H = H; map.pg = pg; map.D = D;
+    map.kc = pg.table ? k_cache : k_cache + (int64_t)bh * cap * D;
+    map.vc = pg.table ? v_cache : v_cache + (int64_t)bh * cap * D;
+    const int own = lens ? min(max(__ldg(lens + map.b), 0), cache_len) : cache_len;
     const int64_t row = ((int64_t)bh * l + i) * D;
     stage_query<T, D>(q_sh[warp], q + row, lane);
-    attend_row<T, D>(q_sh[warp], map, cache_len + i + 1, scale, o + row, lse ? lse + (int64_t)bh * l + i : nullptr, lane);
+    attend_row<T, D>(q_sh[warp], map, own + i + 1, scale, o + row, lse ? lse + (int64_t)bh * l + i : nullptr, lane);
 }
 
-// k_new, v_new [B, H, l, D] -> cache rows [cache_len, cache_len + l) of every (b, h): 16-byte vectors, bit-exact.
+// k_new, v_new [B, H, l, D] -> cache rows [len, len + l) of every (b, h): 16-byte vectors, bit-exact.  With per-sequence
+// lengths (pad_to > 1) the rows from the sequence's new end up to the next multiple of pad_to (and at most cap) are
+// set to zero as well: the tensor-core kernel multiplies them by probabilities of zero, so they have to be finite, and
+// the contents of the cache past the valid length are unspecified anyway.  k_new == NULL: only that.
 __global__ void cache_append_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
                                     uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, int vec_per_row, int l, int cap,
-                                    int cache_len) {
+                                    int cache_len, const int32_t* __restrict__ lens, int H, Paging pg, int pad_to) {
     const int bh = blockIdx.y;
-    const int64_t n = (int64_t)l * vec_per_row;
-    const int64_t in = (int64_t)bh * n, out = ((int64_t)bh * cap + cache_len) * vec_per_row;
+    const int b = bh / H, h = bh - b * H;
+    const int own = lens ? min(max(__ldg(lens + b), 0), cache_len) : cache_len;
+    auto slot = [&](int j) -> int64_t {   // row j of this (b,h) in 16-byte units
+        if (!pg.table) return ((int64_t)bh * cap + j) * vec_per_row;
+        const int page = min(max(__ldg(pg.table + (int64_t)b * pg.max_pages + (j >> pg.log2_ps)), 0), pg.n_pages - 1);
+        return ((((int64_t)page * H + h) << pg.log2_ps) + (j & ((1 << pg.log2_ps) - 1))) * vec_per_row;
+    };
+    const int end = own + l;
+    const int pad_end = pad_to > 1 ? min((end + pad_to - 1) / pad_to * pad_to, cap) : end;
+    const int64_t n = (int64_t)(pad_end - own) * vec_per_row, n_new = (int64_t)l * vec_per_row;
+    const int64_t in = (int64_t)bh * n_new;
     for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) {
-        k_cache[out + e] = __ldg(k_new + in + e);
-        v_cache[out + e] = __ldg(v_new + in + e);
+        const int r = (int)(e / vec_per_row), cv = (int)(e - (int64_t)r * vec_per_row);
+        const int64_t out = slot(own + r) + cv;
+        if (e < n_new) {
+            if (k_new) { k_cache[out] = __ldg(k_new + in + e); v_cache[out] = __ldg(v_new + in + e); }
+        } else {
+            k_cache[out] = make_uint4(0, 0, 0, 0);
+            v_cache[out] = make_uint4(0, 0, 0, 0);
+        }
     }
 }
 
@@ -720,35 +748,41 @@ cudaError_t launch_compress_generic(const void* q_mem, const void* k_mem, const 
 
 template <typename T, int D>
 static cudaError_t prefill_generic_t(const void* q, const void* kc, const void* vc, void* o, float* lse, int BH, int l,
-                                     int cap, int cache_len, float scale, cudaStream_t st) {
+                                     int cap, int cache_len, const int32_t* lens, int H, const Paging& pg, float scale,
+                                     cudaStream_t st) {
     dim3 grid((l + GENERIC_WARPS - 1) / GENERIC_WARPS, BH);
     prefill_generic_kernel<T, D><<<grid, GENERIC_WARPS * 32, 0, st>>>(static_cast<const T*>(q), static_cast<const T*>(kc),
                                                                      static_cast<const T*>(vc), static_cast<T*>(o), lse, l, cap,
-                                                                     cache_len, scale);
+                                                                     cache_len, lens, H, pg, scale);
     count_launches(1);
     return cudaGetLastError();
 }
 
 cudaError_t launch_prefill_attn_generic(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
-                                        int B, int H, int D, int l, int cap, int cache_len, loma_dtype dt, float scale,
-                                        cudaStream_t st) {
+                                        int B, int H, int D, int l, int cap, int cache_len, const int32_t* lens,
+                                        const Paging& pg, loma_dtype dt, float scale, cudaStream_t st) {
     const int BH = B * H;
     if (dt == LOMA_F32)
-        return D == 64 ? prefill_generic_t<float, 64>(q, k_cache, v_cache, o, lse, BH, l, cap, cache_len, scale, st)
-                       : prefill_generic_t<float, 128>(q, k_cache, v_cache, o, lse, BH, l, cap, cache_len, scale, st);
-    return D == 64 ? prefill_generic_t<__nv_bfloat16, 64>(q, k_cache, v_cache, o, lse, BH, l, cap, cache_len, scale, st)
-                   : prefill_generic_t<__nv_bfloat16, 128>(q, k_cache, v_cache, o, lse, BH, l, cap, cache_len, scale, st);
+        return D == 64 ? prefill_generic_t<float, 64>(q, k_cache, v_cache, o, lse, BH, l, cap, cache_len, lens, H, pg, scale, st)
+                       : prefill_generic_t<float, 128>(q, k_cache, v_cache, o, lse, BH, l, cap, cache_len, lens, H, pg, scale, st);
+    return D == 64 ? prefill_generic_t<__nv_bfloat16, 64>(q, k_cache, v_cache, o, lse, BH, l, cap, cache_len, lens, H, pg, scale, st)
+                   : prefill_generic_t<__nv_bfloat16, 128>(q, k_cache, v_cache, o, lse, BH, l, cap, cache_len, lens, H, pg, scale,
+                                                           st);
 }
 
+// pad_to: see cache_append_kernel (1: plain append)
 cudaError_t launch_cache_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache, int B, int H,
-                                int row_bytes, int l, int cap, int cache_len, cudaStream_t st) {
+                                int row_bytes, int l, int cap, int cache_len, const int32_t* lens, const Paging& pg,
+                                int pad_to, cudaStream_t st) {
     const int vec = row_bytes / 16;
-    const int64_t n = (int64_t)l * vec;
+    const int64_t n = (int64_t)(l + (pad_to > 1 ? pad_to : 0)) * vec;
     int gx = (int)((n + 255) / 256);
     if (gx > 64) gx = 64;
+    if (gx < 1) gx = 1;
     dim3 grid(gx, B * H);
     cache_append_kernel<<<grid, 256, 0, st>>>(static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new),
-                                              static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache), vec, l, cap, cache_len);
+                                              static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache), vec, l, cap, cache_len,
+                                              lens, H, pg, pad_to);
     count_launches(1);
     return cudaGetLastError();
 }

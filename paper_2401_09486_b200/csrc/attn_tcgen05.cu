@@ -70,7 +70,9 @@ struct TcSmem {
     static constexpr int TOTAL = 2 * STREAM_BYTES;
 };
 
-template <int D>
+// RAGGED: the prefill plan of a batch whose sequences have their own cache lengths (p.prefill_lens); a kernel of
+// its own so that the other plans carry none of it.
+template <int D, bool RAGGED>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
     using SM = TcSmem<D>;
@@ -125,6 +127,11 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         ok_ = __all_sync(0xffffffffu, mbar_wait(bar(B_TF + (n & 1)), (n >> 1) & 1, abortp, p.status));
         return ok_ ? tile_ring[n & 3] : -1;
     };
+    // ragged prompt pieces: batch element bi's own cache length (clamped to the length the plan was sized for)
+    auto own_diag = [&](int bi) -> int {
+        if (!RAGGED) return -1;
+        return min(max(__ldg(p.prefill_lens + bi), 0), p.view[V_MEM].diag);
+    };
 
     if (warp == 8 || warp == 9) {
         // ------------------------------------------------------------ TMA producer of stream st
@@ -144,7 +151,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 split_work(p, w, rank, bh);
                 const int bi = fdiv(bh, p.dH), hi = bh - bi * p.H;
                 TileDesc td;
-                decode_tile(p, rank, td);
+                decode_tile(p, rank, td, own_diag(bi));
                 const View& qv = p.view[td.view];
                 if (tcount > 0) ok = mbar_wait(bar(B_QE), (tcount - 1) & 1, abortp, p.status);
                 if (!ok) break;
@@ -226,11 +233,12 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             for (;; ++tcount) {
                 const int w = next_tile(tcount, ok);
                 if (w < 0) break;
-                int rank, bh_unused;
-                split_work(p, w, rank, bh_unused);
+                int rank, bh_m;
+                split_work(p, w, rank, bh_m);
                 TileDesc td;
-                decode_tile(p, rank, td);
-                const HalfMasks hm = tile_half_masks(p, td, lane);
+                const int dg = own_diag(fdiv(bh_m, p.dH));
+                decode_tile(p, rank, td, dg);
+                const HalfMasks hm = tile_half_masks(p, td, lane, dg);
                 const int nsteps = td.nsteps;
                 HalfWalk sw, pw;
                 sw.start(hm);
@@ -283,7 +291,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
         struct TileCtx {
             TileDesc td;
             HalfMasks hm;
-            int bh, bi, hi, ro, rc, zone_row0;
+            int bh, bi, hi, ro, rc, zone_row0, diag;
             bool row_valid;
         };
         auto decode_ctx = [&](int w, TileCtx& c) {
@@ -291,14 +299,15 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
             split_work(p, w, rank, c.bh);
             c.bi = fdiv(c.bh, p.dH);
             c.hi = c.bh - c.bi * p.H;
-            decode_tile(p, rank, c.td);
+            c.diag = own_diag(c.bi);
+            decode_tile(p, rank, c.td, c.diag);
             const View& qv = p.view[c.td.view];
             const int rsub = fdiv(rr, qv.dR);
             c.ro = c.td.r0 + (rr - rsub * qv.R);
             c.rc = c.td.a0 + rsub;
             c.zone_row0 = qv.zone_row0;
             c.row_valid = (rr < qv.R * qv.CH) && (c.rc <= c.td.a1) && (c.ro < qv.Z);
-            c.hm = tile_half_masks(p, c.td, lane);
+            c.hm = tile_half_masks(p, c.td, lane, c.diag);
         };
         TileCtx cur, nxt;
         uint32_t tcount = 0;
@@ -322,7 +331,7 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                 if (hw.first_of_step(hm)) {
                     KTile kt;
                     step_ktile(p, td, hw.j, kt);
-                    row_interval(p.view[kt.view], kt, rc, ro, rr, row_valid, lo, hi2);
+                    row_interval(p.view[kt.view], kt, rc, ro, rr, row_valid, lo, hi2, RAGGED ? cur.diag : p.view[kt.view].diag);
                 }
                 // One visited half of a key tile (64 keys) per pass, in score buffer ge & 1: the tensor
                 // pipe works on the other buffer while this warpgroup works on this one.
@@ -585,11 +594,17 @@ static cudaError_t launch_tc_kernel(const TmaMaps& maps, const FwdParams& p, int
         int sms = 0;
         cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(masked_attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(masked_attn_tc_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  TcSmem<128>::TOTAL + 1024);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(masked_attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 TcSmem<64>::TOTAL + 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(masked_attn_tc_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     TcSmem<128>::TOTAL + 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(masked_attn_tc_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     TcSmem<64>::TOTAL + 1024);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(masked_attn_tc_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     TcSmem<64>::TOTAL + 1024);
         if (e != cudaSuccess) return e;
         sm_count[dev] = sms;
     }
@@ -598,10 +613,14 @@ static cudaError_t launch_tc_kernel(const TmaMaps& maps, const FwdParams& p, int
     const int64_t want = (work + 1) / 2;            // two streams (query tiles in flight) per CTA
     const int grid = (int)(want < sms ? want : sms);
     // the shared-memory footprint also keeps one CTA per SM (each allocates all 512 TMEM columns)
-    if (D == 128)
-        masked_attn_tc_kernel<128><<<grid, TC_THREADS, TcSmem<128>::TOTAL + 1024, st>>>(maps, p);
-    else
-        masked_attn_tc_kernel<64><<<grid, TC_THREADS, TcSmem<64>::TOTAL + 1024, st>>>(maps, p);
+    const bool ragged = p.prefill && p.prefill_lens;
+    if (D == 128) {
+        if (ragged) masked_attn_tc_kernel<128, true><<<grid, TC_THREADS, TcSmem<128>::TOTAL + 1024, st>>>(maps, p);
+        else masked_attn_tc_kernel<128, false><<<grid, TC_THREADS, TcSmem<128>::TOTAL + 1024, st>>>(maps, p);
+    } else {
+        if (ragged) masked_attn_tc_kernel<64, true><<<grid, TC_THREADS, TcSmem<64>::TOTAL + 1024, st>>>(maps, p);
+        else masked_attn_tc_kernel<64, false><<<grid, TC_THREADS, TcSmem<64>::TOTAL + 1024, st>>>(maps, p);
+    }
     count_launches(1);
     return cudaGetLastError();
 }
@@ -669,12 +688,16 @@ cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, v
 
 // New tokens over an existing cache on the same kernel: the query view is the l new rows, the key view the
 // cache rows 0 .. cache_len + l - 1 (the new rows' K/V have been appended before this launch).
-// q, o: [B, H, l, D] contiguous; k_cache, v_cache: [B, H, cap, D] contiguous.
+// q, o: [B, H, l, D] contiguous; k_cache, v_cache: [B, H, cap, D] contiguous.  cache_lens (device, [B], or NULL): every
+// sequence's own number of earlier entries; its tiles then stop at its own last key tile, whose rows past the
+// sequence's end the caller has made finite (they are multiplied by probabilities of zero).
 cudaError_t launch_prefill_attn_tc(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, int B,
-                                   int H, int D, int l, int cap, int cache_len, float scale, cudaStream_t st) {
+                                   int H, int D, int l, int cap, int cache_len, const int32_t* cache_lens, float scale,
+                                   cudaStream_t st) {
     if (!encode_fn()) return cudaErrorNotSupported;
     FwdParams p{};
-    make_prefill_plan(l, cache_len, B, H, &p);
+    make_prefill_plan(l, cache_len, B, H, &p);   // ragged batch: cache_len is the bound the per-sequence lengths are clamped to
+    p.prefill_lens = cache_lens;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.lse = lse;
     p.status = device_status_word();

@@ -431,6 +431,37 @@ int loma_compress_step_layers(int n_layers, const void* const* q_mem, const void
     return LOMA_OK;
 }
 
+static int log2_exact(int x);   // defined with the paged entry points below
+
+// The three forms of the prompt piece over a cache.  cache_len: the uniform length, or (cache_lens given) the bound the
+// per-sequence lengths are clamped to; pg.table given: the cache is the paged pool and cap = max_pages * page_size.
+static int prefill_attn_impl(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
+                             float* lse, int B, int H, int D, int l, int cap, int cache_len, const int32_t* cache_lens,
+                             const Paging& pg, loma_dtype dtype, float softmax_scale, unsigned flags, void* stream) {
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the tensor-core kernel (bf16, contiguous cache; a handful of rows is cheaper on CUDA cores, one warp per row:
+    // from 8 rows on one pass of the cache through the tensor-core kernel wins over l passes)
+    const bool tc = dtype == LOMA_BF16 && l >= 8 && !pg.table && !(flags & LOMA_FLAG_FORCE_GENERIC);
+    // 1. the new tokens' K/V go into the cache (bit-exact); 2. every new row attends to cache rows 0 .. len + i.
+    // With per-sequence lengths the tensor-core kernel also wants the rest of each sequence's last 128-row key tile finite.
+    const int pad_to = (tc && cache_lens) ? 128 : 1;
+    if (k_new || pad_to > 1) {
+        if (launch_cache_append(k_new, v_new, k_cache, v_cache, B, H, (int)(D * elt_size(dtype)), l, cap, cache_len,
+                                cache_lens, pg, pad_to, st) != cudaSuccess)
+            return LOMA_ERR_CUDA;
+    }
+    cudaError_t e = cudaErrorNotSupported;
+    if (tc) {
+        e = launch_prefill_attn_tc(q, k_cache, v_cache, o, lse, B, H, D, l, cap, cache_len, cache_lens, scale, st);
+        if (e == cudaErrorNotSupported) g_fallbacks.fetch_add(1, std::memory_order_relaxed);
+    }
+    if (e == cudaErrorNotSupported)
+        e = launch_prefill_attn_generic(q, k_cache, v_cache, o, lse, B, H, D, l, cap, cache_len, cache_lens, pg, dtype,
+                                        scale, st);
+    return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+}
+
 int loma_prefill_attn(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
                       float* lse, int B, int H, int D, int l, int cap, int cache_len, loma_dtype dtype,
                       float softmax_scale, unsigned flags, void* stream) {
@@ -449,24 +480,58 @@ int loma_prefill_attn(const void* q, const void* k_new, const void* v_new, void*
     if (lse && ((uintptr_t)lse & 3u)) return LOMA_ERR_ALIGNMENT;
     const int dc = check_device();
     if (dc != LOMA_OK) return dc;
-    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // 1. the new tokens' K/V go into the cache (bit-exact); 2. every new row attends to cache rows 0 .. cache_len + i
-    if (k_new) {
-        if (launch_cache_append(k_new, v_new, k_cache, v_cache, B, H, (int)(D * elt_size(dtype)), l, cap, cache_len, st) !=
-            cudaSuccess)
-            return LOMA_ERR_CUDA;
-    }
-    cudaError_t e = cudaErrorNotSupported;
-    // (a handful of rows is cheaper on CUDA cores, one warp per row; from 8 rows on one pass of the cache through the
-    // tensor-core kernel wins over l passes)
-    if (dtype == LOMA_BF16 && l >= 8 && !(flags & LOMA_FLAG_FORCE_GENERIC)) {
-        e = launch_prefill_attn_tc(q, k_cache, v_cache, o, lse, B, H, D, l, cap, cache_len, scale, st);
-        if (e == cudaErrorNotSupported) g_fallbacks.fetch_add(1, std::memory_order_relaxed);
-    }
-    if (e == cudaErrorNotSupported)
-        e = launch_prefill_attn_generic(q, k_cache, v_cache, o, lse, B, H, D, l, cap, cache_len, dtype, scale, st);
-    return e == cudaSuccess ? LOMA_OK : LOMA_ERR_CUDA;
+    return prefill_attn_impl(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, l, cap, cache_len, nullptr, Paging{}, dtype,
+                             softmax_scale, flags, stream);
+}
+
+int loma_prefill_attn_ragged(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
+                             float* lse, int B, int H, int D, int l, int cap, const int32_t* cache_lens,
+                             int max_cache_len, loma_dtype dtype, float softmax_scale, unsigned flags, void* stream) {
+    if (B < 0 || H < 0 || l < 0 || cap < 0 || max_cache_len < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    if ((k_new == nullptr) != (v_new == nullptr)) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)max_cache_len + l > cap) return LOMA_ERR_CAPACITY;
+    if (B == 0 || H == 0 || l == 0) return LOMA_OK;
+    if (!q || !k_cache || !v_cache || !o || !cache_lens) return LOMA_ERR_INVALID_ARG;
+    if (o == q || o == k_new || o == v_new) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) || !aligned16(k_new) ||
+        !aligned16(v_new) || ((uintptr_t)cache_lens & 3u))
+        return LOMA_ERR_ALIGNMENT;
+    if (lse && ((uintptr_t)lse & 3u)) return LOMA_ERR_ALIGNMENT;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    return prefill_attn_impl(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, l, cap, max_cache_len, cache_lens, Paging{},
+                             dtype, softmax_scale, flags, stream);
+}
+
+int loma_prefill_attn_paged(const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+                            const int32_t* block_table, void* o, float* lse, int B, int H, int D, int l, int page_size,
+                            int max_pages, int n_pages, const int32_t* cache_lens, int max_cache_len, loma_dtype dtype,
+                            float softmax_scale, unsigned flags, void* stream) {
+    if (B < 0 || H < 0 || l < 0 || max_pages < 0 || n_pages < 0 || max_cache_len < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    const int l2 = log2_exact(page_size);
+    if (l2 < 0 || page_size > 65536) return LOMA_ERR_INVALID_ARG;
+    if ((k_new == nullptr) != (v_new == nullptr)) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)max_cache_len + l > (int64_t)max_pages * page_size) return LOMA_ERR_CAPACITY;
+    if ((int64_t)max_pages * page_size > INT_MAX) return LOMA_ERR_INVALID_ARG;
+    if (B == 0 || H == 0 || l == 0) return LOMA_OK;
+    if (!q || !k_pool || !v_pool || !o || !block_table || !cache_lens || n_pages < 1) return LOMA_ERR_INVALID_ARG;
+    if (o == q || o == k_new || o == v_new) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_pool) || !aligned16(v_pool) || !aligned16(o) || !aligned16(k_new) ||
+        !aligned16(v_new) || ((uintptr_t)cache_lens & 3u) || ((uintptr_t)block_table & 3u))
+        return LOMA_ERR_ALIGNMENT;
+    if (lse && ((uintptr_t)lse & 3u)) return LOMA_ERR_ALIGNMENT;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    Paging pg;
+    pg.table = block_table; pg.max_pages = max_pages; pg.log2_ps = l2; pg.n_pages = n_pages;
+    return prefill_attn_impl(q, k_new, v_new, k_pool, v_pool, o, lse, B, H, D, l, max_pages * page_size, max_cache_len,
+                             cache_lens, pg, dtype, softmax_scale, flags, stream);
 }
 
 int loma_prefill_attn_plan_coverage(int l, int cache_len, uint8_t* counts) {

@@ -123,13 +123,15 @@ cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, v
 
 // l new tokens over a cache that already holds their K/V at [cache_len, cache_len + l) (attn_tcgen05.cu)
 cudaError_t launch_prefill_attn_tc(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, int B,
-                                   int H, int D, int l, int cap, int cache_len, float scale, cudaStream_t st);
+                                   int H, int D, int l, int cap, int cache_len, const int32_t* cache_lens, float scale,
+                                   cudaStream_t st);
 // the same on CUDA cores (any l, fp32 or bf16), and the bit-exact append that precedes both (attn_generic.cu)
 cudaError_t launch_prefill_attn_generic(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
-                                        int B, int H, int D, int l, int cap, int cache_len, loma_dtype dt, float scale,
-                                        cudaStream_t st);
+                                        int B, int H, int D, int l, int cap, int cache_len, const int32_t* lens,
+                                        const Paging& pg, loma_dtype dt, float scale, cudaStream_t st);
 cudaError_t launch_cache_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache, int B, int H,
-                                int row_bytes, int l, int cap, int cache_len, cudaStream_t st);
+                                int row_bytes, int l, int cap, int cache_len, const int32_t* lens, const Paging& pg,
+                                int pad_to, cudaStream_t st);
 
 void plan_coverage_host(const Layout& L, uint8_t* counts);          // tile_plan_host.cu
 void prefill_plan_coverage_host(int l, int cache_len, uint8_t* counts);

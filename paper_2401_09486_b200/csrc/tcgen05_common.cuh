@@ -182,12 +182,12 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 
 // The visited halves of a tile's first 64 steps, one step per lane and two ballots per 32 steps.
 // Called by whole warps only.
-__device__ __forceinline__ HalfMasks tile_half_masks(const FwdParams& p, const TileDesc& td, int lane) {
+__device__ __forceinline__ HalfMasks tile_half_masks(const FwdParams& p, const TileDesc& td, int lane, int own_diag = -1) {
     HalfMasks hm;
     hm.m[0] = hm.m[1] = 0;
     for (int base = 0; base < td.nsteps && base < 64; base += 32) {
         const int j = base + lane;
-        const unsigned v = j < td.nsteps ? visited_halves(p, td, j) : 0u;
+        const unsigned v = j < td.nsteps ? visited_halves(p, td, j, own_diag) : 0u;
         hm.m[0] |= (unsigned long long)__ballot_sync(0xffffffffu, v & 1u) << base;
         hm.m[1] |= (unsigned long long)__ballot_sync(0xffffffffu, v & 2u) << base;
     }

@@ -61,6 +61,7 @@ struct FwdParams {
     int n_tail, n_read, n_mem, n_rep;   // tiles per view, in scheduling order
     unsigned flags;
     int prefill;       // 1: the plan of loma_prefill_attn (query view V_TAIL over the new tokens, key view V_MEM over the cache)
+    const int* prefill_lens;   // prefill plan of a ragged batch: [B] cache lengths on the device (NULL: uniform)
     FastDiv dBH, dH, dTT;   // division by BH, H and total_tiles
     float scale_log2;
     float* lse;
@@ -100,7 +101,9 @@ __host__ __device__ __forceinline__ int tiles_covering(const View& v, int nchunk
     return v.Z >= 128 ? nchunks * v.tpc : fdiv(nchunks + v.CH - 1, v.dCH);
 }
 
-__host__ __device__ __forceinline__ void decode_tile(const FwdParams& p, int rank, TileDesc& td) {
+// own_diag >= 0: the prefill plan of a ragged batch, where every sequence has its own cache length (at most the key
+// view's diag, for which the plan was sized)
+__host__ __device__ __forceinline__ void decode_tile(const FwdParams& p, int rank, TileDesc& td, int own_diag = -1) {
     int view, qi;
     if (rank < p.n_tail) { view = V_TAIL; qi = p.n_tail - 1 - rank; }
     else if ((rank -= p.n_tail) < p.n_read) { view = V_READ; qi = p.n_read - 1 - rank; }
@@ -120,7 +123,7 @@ __host__ __device__ __forceinline__ void decode_tile(const FwdParams& p, int ran
         // new tokens over the cache (Appendix A, inference_input): key tiles 0 .. the one that holds the
         // diagonal of the tile's last row (row o sees keys 0 .. o + diag)
         const int last_row = plan_min(td.r0 + 127, g.Z - 1);
-        td.seg[0] = Seg{V_MEM, M_CAUSAL_OFF, 0, (last_row + vm.diag) / 128 + 1};
+        td.seg[0] = Seg{V_MEM, M_CAUSAL_OFF, 0, (last_row + (own_diag >= 0 ? own_diag : vm.diag)) / 128 + 1};
         td.seg[1] = Seg{V_MEM, M_CAUSAL_OFF, 0, 0};
     } else if (view == V_READ || view == V_TAIL) {
         // memory zones of every earlier chunk, then the own reading zone up to this tile
@@ -154,8 +157,9 @@ __host__ __device__ __forceinline__ void step_ktile(const FwdParams& p, const Ti
 }
 
 // Allowed columns [lo, hi) of a key tile for a row at (chunk rc, offset ro), tile-local row rr.
+// diag (mode M_CAUSAL_OFF only): the key view's diag, or the sequence's own cache length in a ragged batch.
 __host__ __device__ __forceinline__ void row_interval(const View& kv, const KTile& kt, int rc, int ro, int rr, bool row_valid,
-                                             int& lo, int& hi) {
+                                             int& lo, int& hi, int diag) {
     const int vcols = plan_min(kv.R, kv.Z - kt.r0);   // valid columns per chunk of this tile
     const int d = rc - kt.a0;
     lo = 0; hi = 0;
@@ -165,7 +169,7 @@ __host__ __device__ __forceinline__ void row_interval(const View& kv, const KTil
     } else if (kt.mode == M_DIAG) {
         lo = rr; hi = rr + 1;
     } else if (kt.mode == M_CAUSAL_OFF) {
-        hi = plan_min(plan_max(ro + kv.diag - kt.r0 + 1, 0), vcols);
+        hi = plan_min(plan_max(ro + diag - kt.r0 + 1, 0), vcols);
     } else if (d >= 0 && d < kv.CH) {
         lo = d * kv.R;
         hi = lo + (kt.mode == M_EQ ? vcols : plan_min(plan_max(ro - kt.r0 + 1, 0), vcols));
@@ -177,7 +181,7 @@ __host__ __device__ __forceinline__ void row_interval(const View& kv, const KTil
 // query tile: bit h set = columns [64h, 64h + 64) are visited.  Computed from the union of the row
 // intervals over the tile's chunks; a superset is harmless (every row still applies its own
 // interval), a missing half would drop allowed entries, which the host-side coverage replay checks.
-__host__ __device__ __forceinline__ unsigned step_halves(const FwdParams& p, const TileDesc& td, const KTile& kt) {
+__host__ __device__ __forceinline__ unsigned step_halves(const FwdParams& p, const TileDesc& td, const KTile& kt, int own_diag = -1) {
     const View& kv = p.view[kt.view];
     const int vcols = plan_min(kv.R, kv.Z - kt.r0);
     int ulo = 0, uhi = 0;
@@ -188,7 +192,7 @@ __host__ __device__ __forceinline__ unsigned step_halves(const FwdParams& p, con
         uhi = 128;
     } else if (kt.mode == M_CAUSAL_OFF) {
         const int last_row = plan_min(td.r0 + 127, p.view[td.view].Z - 1);
-        uhi = plan_min(plan_max(last_row + kv.diag - kt.r0 + 1, 0), vcols);
+        uhi = plan_min(plan_max(last_row + (own_diag >= 0 ? own_diag : kv.diag) - kt.r0 + 1, 0), vcols);
     } else {
         const int d0 = plan_max(td.a0 - kt.a0, 0), d1 = plan_min(td.a1 - kt.a0, kv.CH - 1);
         if (d1 >= d0) { ulo = d0 * kv.R; uhi = d1 * kv.R + vcols; }
@@ -206,11 +210,11 @@ struct HalfMasks {
         return j >= 64 ? 3u : (unsigned)((m[0] >> j) & 1ull) | ((unsigned)((m[1] >> j) & 1ull) << 1);
     }
 };
-__host__ __device__ __forceinline__ unsigned visited_halves(const FwdParams& p, const TileDesc& td, int j) {
+__host__ __device__ __forceinline__ unsigned visited_halves(const FwdParams& p, const TileDesc& td, int j, int own_diag = -1) {
     if (j >= 64) return 3u;
     KTile kt;
     step_ktile(p, td, j, kt);
-    return step_halves(p, td, kt);
+    return step_halves(p, td, kt, own_diag);
 }
 
 // Walks the visited halves of a query tile's key tiles in order.  One visited half ("event") is
@@ -378,7 +382,7 @@ inline void make_plan(const Layout& L, int B, int H, FwdParams* p) {
     p->n_tail = p->view[V_TAIL].ntiles; p->n_read = p->view[V_READ].ntiles;
     p->n_mem = p->view[V_MEM].ntiles; p->n_rep = p->view[V_REP].ntiles;
     p->total_tiles = p->n_tail + p->n_read + p->n_mem + p->n_rep;
-    p->flags = L.flags; p->prefill = 0;
+    p->flags = L.flags; p->prefill = 0; p->prefill_lens = nullptr;
     p->dBH = make_fastdiv(p->BH); p->dH = make_fastdiv(H); p->dTT = make_fastdiv(p->total_tiles);
 }
 
@@ -394,7 +398,7 @@ inline void make_prefill_plan(int l, int cache_len, int B, int H, FwdParams* p) 
     p->n_chunks = 0; p->s = 0; p->S = l; p->H = H; p->BH = B * H;
     p->n_tail = p->view[V_TAIL].ntiles; p->n_read = 0; p->n_mem = 0; p->n_rep = 0;
     p->total_tiles = p->n_tail;
-    p->flags = 0; p->prefill = 1;
+    p->flags = 0; p->prefill = 1; p->prefill_lens = nullptr;
     p->dBH = make_fastdiv(p->BH); p->dH = make_fastdiv(H); p->dTT = make_fastdiv(p->total_tiles);
 }
 

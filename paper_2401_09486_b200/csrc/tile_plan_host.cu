@@ -33,7 +33,7 @@ void plan_coverage_host(const Layout& L, uint8_t* counts) {
                 const int rc = td.a0 + rsub;
                 const bool row_valid = (rr < qv.R * qv.CH) && (rc <= td.a1) && (ro < qv.Z);
                 int lo, hi;
-                row_interval(kv, kt, rc, ro, rr, row_valid, lo, hi);
+                row_interval(kv, kt, rc, ro, rr, row_valid, lo, hi, kv.diag);
                 if (!row_valid || hi <= lo) continue;
                 const int64_t grow = (int64_t)rc * L.s + qv.zone_row0 + ro;
                 for (int col = (lo > 64 * hw.h ? lo : 64 * hw.h); col < hi && col < 64 * hw.h + 64; ++col) {
@@ -81,7 +81,7 @@ void prefill_plan_coverage_host(int l, int cache_len, uint8_t* counts) {
                 const int rc = td.a0 + rsub;
                 const bool row_valid = (rr < qv.R * qv.CH) && (rc <= td.a1) && (ro < qv.Z);
                 int lo, hi;
-                row_interval(kv, kt, rc, ro, rr, row_valid, lo, hi);
+                row_interval(kv, kt, rc, ro, rr, row_valid, lo, hi, kv.diag);
                 if (!row_valid || hi <= lo) continue;
                 for (int col = (lo > 64 * hw.h ? lo : 64 * hw.h); col < hi && col < 64 * hw.h + 64; ++col) {
                     const int ksub = col / kv.R;

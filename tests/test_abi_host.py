@@ -448,3 +448,29 @@ def test_ragged_and_paged_rope_fused_steps_validation(lib):
     assert cmp_p(mx=65) == CAPACITY
     assert cmp_p(ps=48) == INVALID
     assert cmp_p(B=0) == 0
+
+
+def test_ragged_and_paged_prefill_validation(lib):
+    def rag(q=0x1000, kn=0x2000, vn=0x3000, kc=0x4000, vc=0x5000, o=0x6000, B=2, H=1, D=128, l=4, cap=20, lens=0x7000, mx=16,
+            dt=1):
+        return lib.loma_prefill_attn_ragged(q, kn, vn, kc, vc, o, None, B, H, D, l, cap, lens, mx, dt, 0.0, 0, None)
+    assert rag(mx=17) == CAPACITY
+    assert rag(mx=-1) == INVALID
+    assert rag(lens=None) == INVALID
+    assert rag(lens=0x7002) == ALIGNMENT
+    assert rag(kn=None) == INVALID                       # k_new without v_new
+    assert rag(o=0x1000) == INVALID                      # o aliases q
+    assert rag(D=96) == UNSUPPORTED
+    assert rag(l=0) == 0 and rag(B=0) == 0
+
+    def pag(q=0x1000, kn=0x2000, vn=0x3000, kp=0x4000, vp=0x5000, bt=0x6000, o=0x7000, B=2, H=1, D=128, l=4, ps=16, mp=2,
+            npg=8, lens=0x8000, mx=28, dt=1):
+        return lib.loma_prefill_attn_paged(q, kn, vn, kp, vp, bt, o, None, B, H, D, l, ps, mp, npg, lens, mx, dt, 0.0, 0, None)
+    assert pag(mx=29) == CAPACITY                        # the new rows would run past the table
+    assert pag(ps=24) == INVALID
+    assert pag(bt=None) == INVALID
+    assert pag(lens=None) == INVALID
+    assert pag(npg=0) == INVALID
+    assert pag(bt=0x6002) == ALIGNMENT
+    assert pag(dt=7) == UNSUPPORTED
+    assert pag(l=0) == 0

@@ -291,6 +291,92 @@ def test_prefill_over_a_cache_matches_oracle_and_appends_bit_exact(l, cache_len,
     assert np.array_equal(npf(kcd), want_kc) and np.array_equal(npf(vcd), want_vc)
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, GENERIC])
+@pytest.mark.parametrize("l,lens", [(1, [0, 5, 130]), (17, [16, 0, 300, 129]), (64, [100, 1000, 0]), (200, [513, 37, 1024, 256])])
+def test_ragged_prefill_matches_the_oracle_per_sequence(l, lens, flags, dtype):
+    """One run of Appendix A `inference_input` with l tokens per sequence, every sequence over its own number of
+    cached entries.  The cache rows past every sequence's end start out as NaN: nothing of them may reach an
+    output, and the entries below each sequence's own length stay untouched."""
+    B, H, D = len(lens), 2, 128
+    max_len = max(lens)
+    cap = max_len + l + 130
+    kc = synthetic.normal_tensor((B, H, cap, D), 71, 1.0, dtype)
+    vc = synthetic.normal_tensor((B, H, cap, D), 72, 1.0, dtype)
+    for b, n in enumerate(lens):
+        kc[b, :, n:] = float("nan")
+        vc[b, :, n:] = float("nan")
+    q, kn, vn = synthetic.qkv(B, H, l, D, seed=73, std=1.0, dtype=dtype)
+    kcd, vcd = kc.to(DEV), vc.to(DEV)
+    o = torch.full((B, H, l, D), float("nan"), dtype=dtype, device=DEV)
+    lse = torch.full((B, H, l), float("nan"), dtype=torch.float32, device=DEV)
+    lens_d = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    L.loma_prefill_attn_ragged(q.to(DEV), kn.to(DEV), vn.to(DEV), kcd, vcd, o, lse, lens_d, max_len, flags)
+    torch.cuda.synchronize()
+    for b, n in enumerate(lens):
+        sl = slice(b, b + 1)
+        want_o, want_lse, _, _ = oracle.prefill_attn(npf(q[sl]), npf(kn[sl]), npf(vn[sl]), npf(kc[sl, :, :n + l].nan_to_num()),
+                                                     npf(vc[sl, :, :n + l].nan_to_num()), n)
+        check_close(o[sl], want_o, dtype)
+        assert np.abs(npf(lse[sl]) - want_lse).max() <= (1e-5 if dtype == torch.float32 else 2e-2)
+        assert np.array_equal(bits(kcd[b, :, :n]), bits(kc[b, :, :n])) and np.array_equal(bits(vcd[b, :, :n]), bits(vc[b, :, :n]))
+        assert np.array_equal(bits(kcd[b, :, n:n + l]), bits(kn[b])) and np.array_equal(bits(vcd[b, :, n:n + l]), bits(vn[b]))
+    assert L.loma_device_status() == 0
+
+
+def test_ragged_prefill_with_equal_lengths_equals_the_uniform_call_bit_for_bit():
+    B, H, D, l, n = 3, 2, 128, 150, 333
+    cap = n + l + 7
+    kc = synthetic.normal_tensor((B, H, cap, D), 75, 1.0, torch.bfloat16).to(DEV)
+    vc = synthetic.normal_tensor((B, H, cap, D), 76, 1.0, torch.bfloat16).to(DEV)
+    q, kn, vn = (x.to(DEV) for x in synthetic.qkv(B, H, l, D, seed=77, std=1.0, dtype=torch.bfloat16))
+    o_u, o_r = torch.empty_like(q), torch.empty_like(q)
+    kc2, vc2 = kc.clone(), vc.clone()
+    L.loma_prefill_attn(q, kn, vn, kc, vc, o_u, None, n)
+    L.loma_prefill_attn_ragged(q, kn, vn, kc2, vc2, o_r, None, torch.full((B,), n, dtype=torch.int32, device=DEV), n)
+    torch.cuda.synchronize()
+    assert torch.equal(o_u, o_r)
+    assert torch.equal(kc[:, :, :n + l], kc2[:, :, :n + l]) and torch.equal(vc[:, :, :n + l], vc2[:, :, :n + l])
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("l,ps,lens", [(1, 16, [0, 5, 130]), (17, 16, [16, 0, 300]), (70, 64, [100, 513, 0, 64])])
+def test_paged_prefill_matches_the_oracle_per_sequence(l, ps, lens, dtype):
+    """The same step over a paged cache: pages scattered over the pool by a seeded permutation; the new rows
+    land in the pages the block table names, bit for bit."""
+    B, H, D = len(lens), 2, 128
+    max_len = max(lens)
+    mp = (max_len + l + ps - 1) // ps + 1
+    n_pages = B * mp + 3
+    g = torch.Generator().manual_seed(79)
+    table = torch.randperm(n_pages, generator=g)[:B * mp].to(torch.int32).view(B, mp)
+    kpool = synthetic.normal_tensor((n_pages, H, ps, D), 81, 1.0, dtype)
+    vpool = synthetic.normal_tensor((n_pages, H, ps, D), 82, 1.0, dtype)
+    q, kn, vn = synthetic.qkv(B, H, l, D, seed=83, std=1.0, dtype=dtype)
+
+    def gather(pool, b, n):   # the first n entries of sequence b as [1, H, n, D]
+        rows = [pool[int(table[b, j // ps]), :, j % ps] for j in range(n)]
+        return torch.stack(rows, dim=1).unsqueeze(0) if rows else pool.new_zeros((1, H, 0, D))
+
+    kpd, vpd = kpool.to(DEV), vpool.to(DEV)
+    o = torch.full((B, H, l, D), float("nan"), dtype=dtype, device=DEV)
+    lse = torch.full((B, H, l), float("nan"), dtype=torch.float32, device=DEV)
+    L.loma_prefill_attn_paged(q.to(DEV), kn.to(DEV), vn.to(DEV), kpd, vpd, table.to(DEV), o, lse,
+                              torch.tensor(lens, dtype=torch.int32, device=DEV), max_len)
+    torch.cuda.synchronize()
+    kp_after, vp_after = kpd.cpu(), vpd.cpu()
+    for b, n in enumerate(lens):
+        sl = slice(b, b + 1)
+        kc_b = torch.cat([gather(kpool, b, n), torch.zeros((1, H, l, D), dtype=dtype)], dim=2)
+        vc_b = torch.cat([gather(vpool, b, n), torch.zeros((1, H, l, D), dtype=dtype)], dim=2)
+        want_o, want_lse, _, _ = oracle.prefill_attn(npf(q[sl]), npf(kn[sl]), npf(vn[sl]), npf(kc_b), npf(vc_b), n)
+        check_close(o[sl], want_o, dtype)
+        assert np.abs(npf(lse[sl]) - want_lse).max() <= (1e-5 if dtype == torch.float32 else 2e-2)
+        assert np.array_equal(bits(gather(kp_after, b, n + l)[0, :, n:]), bits(kn[b]))
+        assert np.array_equal(bits(gather(vp_after, b, n + l)[0, :, n:]), bits(vn[b]))
+        assert np.array_equal(bits(gather(kp_after, b, n)), bits(gather(kpool, b, n)))
+
+
 def test_prefill_with_rows_already_in_the_cache_and_repeatable():
     """k_new = v_new = NULL: the new rows are read where they already lie; two calls give the same bits."""
     B, H, D, l, cache_len = 2, 2, 128, 150, 333
