@@ -562,6 +562,21 @@ def other_workloads(L, synthetic, torch, dev, peaks):
                                                    "ms": ms, "useful_tflops": fl / (ms * 1e-3) / 1e12,
                                                    "frac_of_measured_bf16": fl / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                                                    "kernels": "cache_append_kernel + masked_attn_tc_kernel<128, true>"}
+    if hasattr(L, "loma_prefill_attn_paged"):
+        # and over a paged cache: 128-row pages scattered over the pool by a seeded permutation
+        psp = 128
+        mpp = (kp + lp) // psp
+        g_cpu = torch.Generator().manual_seed(3520)
+        table_p = torch.randperm(Bp * mpp, generator=g_cpu).to(torch.int32).view(Bp, mpp).to(dev)
+        kpool = kcp.view(Bp, H, mpp, psp, D).permute(0, 2, 1, 3, 4).reshape(Bp * mpp, H, psp, D).contiguous()
+        vpool = vcp.view(Bp, H, mpp, psp, D).permute(0, 2, 1, 3, 4).reshape(Bp * mpp, H, psp, D).contiguous()
+        ms = timed(lambda: L.loma_prefill_attn_paged(qp, knp, vnp, kpool, vpool, table_p, op, None, lens_p, kp, 0, 0.0, stream))
+        res["prefill_paged_512_over_8192_B32"] = {"config": dict(B=Bp, H=H, D=D, l=lp, page_size=psp, pages=Bp * mpp,
+                                                              cache_lens="8192 - (37 b) mod 1024"),
+                                                  "ms": ms, "useful_tflops": fl / (ms * 1e-3) / 1e12,
+                                                  "frac_of_measured_bf16": fl / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                                                  "kernels": "cache_append_kernel + masked_attn_tc_kernel<128, true> (paged key tiles)"}
+        del kpool, vpool
     del kcp, vcp, qp, knp, vnp, op
     torch.cuda.empty_cache()
     for name, flags in (("compress_B64_16k", 0), ("compress_B64_16k_prior_mem", 1)):

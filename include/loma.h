@@ -449,8 +449,10 @@ LOMA_API int loma_prefill_attn(const void* q, const void* k_new, const void* v_n
  *           kernel reads them (with weight zero), and the contents of the cache past a
  *           sequence's valid length are unspecified anyway.
  *   paged:  k_pool, v_pool [n_pages, H, page_size, D] and block_table int32 [B, max_pages] as in
- *           loma_decode_attn_paged (page numbers clamped to the pool); CUDA cores, one warp per
- *           new row, for every dtype.
+ *           loma_decode_attn_paged (page numbers clamped to the pool).  bf16 calls with l >= 8 over
+ *           pages of a multiple of 128 rows run on the tensor-core kernel (a 128-key tile then lies
+ *           in one page; the zeroing described above applies, inside the sequence's last page);
+ *           every other call on CUDA cores, one warp per new row.
  * Other arguments, outputs and errors as loma_prefill_attn; CAPACITY when max_cache_len + l
  * exceeds cap (ragged) or max_pages * page_size (paged); INVALID_ARG for a missing table or
  * length array or a page size that is not a power of two.

@@ -165,18 +165,26 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     const View& kv = p.view[kt.view];
                     const uint32_t ph = gs & 1;
                     const uint32_t bytes = kv.R * kv.CH * 128 * PANELS;
+                    // where the key tile lies: (row, chunk, batch) of the caller's tensor, or, over a paged cache, (row in
+                    // page, 0, page) of the pool -- pages hold a multiple of 128 rows, so a tile never straddles two
+                    int kr = kt.r0, kc_ = kt.c0, kb = bi;
+                    if (RAGGED && p.page_table) {
+                        kb = min(max(__ldg(p.page_table + (int64_t)bi * p.pt_stride + (kt.r0 >> p.log2_ps)), 0), p.n_pages - 1);
+                        kr = kt.r0 & ((1 << p.log2_ps) - 1);
+                        kc_ = 0;
+                    }
                     ok = mbar_wait(bar(B_KE), ph ^ 1, abortp, p.status);
                     if (!ok) break;
                     mbar_expect_tx(bar(B_KF), bytes);
                     for (int pn = 0; pn < PANELS; ++pn)
                         tma_load_5d(smem_base + SM::K_OFF + pn * SM::PANEL_BYTES, &maps.k[kt.view], bar(B_KF), pn * 64,
-                                    kt.r0, kt.c0, hi, bi);
+                                    kr, kc_, hi, kb);
                     ok = mbar_wait(bar(B_VE), ph ^ 1, abortp, p.status);
                     if (!ok) break;
                     mbar_expect_tx(bar(B_VF), bytes);
                     for (int pn = 0; pn < PANELS; ++pn)
                         tma_load_5d(smem_base + SM::V_OFF + pn * SM::PANEL_BYTES, &maps.v[kt.view], bar(B_VF), pn * 64,
-                                    kt.r0, kt.c0, hi, bi);
+                                    kr, kc_, hi, kb);
                 }
             }
             if (!ok) {
@@ -692,12 +700,14 @@ cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, v
 // sequence's own number of earlier entries; its tiles then stop at its own last key tile, whose rows past the
 // sequence's end the caller has made finite (they are multiplied by probabilities of zero).
 cudaError_t launch_prefill_attn_tc(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, int B,
-                                   int H, int D, int l, int cap, int cache_len, const int32_t* cache_lens, float scale,
-                                   cudaStream_t st) {
+                                   int H, int D, int l, int cap, int cache_len, const int32_t* cache_lens,
+                                   const Paging& pg, float scale, cudaStream_t st) {
     if (!encode_fn()) return cudaErrorNotSupported;
+    if (pg.table && (!cache_lens || pg.log2_ps < 7)) return cudaErrorNotSupported;   // pages of a multiple of 128 rows
     FwdParams p{};
     make_prefill_plan(l, cache_len, B, H, &p);   // ragged batch: cache_len is the bound the per-sequence lengths are clamped to
     p.prefill_lens = cache_lens;
+    p.page_table = pg.table; p.pt_stride = pg.max_pages; p.log2_ps = pg.log2_ps; p.n_pages = pg.n_pages;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.lse = lse;
     p.status = device_status_word();
@@ -707,10 +717,11 @@ cudaError_t launch_prefill_attn_tc(const void* q, const void* k_cache, const voi
 
     struct Key {
         const void *q, *k, *v, *o;
-        int B, H, D, l, cap, cache_len;
+        int B, H, D, l, cap, cache_len, paged, log2_ps, n_pages;
         bool operator==(const Key& r) const {
             return q == r.q && k == r.k && v == r.v && o == r.o && B == r.B && H == r.H && D == r.D && l == r.l &&
-                   cap == r.cap && cache_len == r.cache_len;
+                   cap == r.cap && cache_len == r.cache_len && paged == r.paged && log2_ps == r.log2_ps &&
+                   n_pages == r.n_pages;
         }
     };
     static std::mutex mu;
@@ -720,17 +731,27 @@ cudaError_t launch_prefill_attn_tc(const void* q, const void* k_cache, const voi
     TmaMaps maps;
     {
         std::lock_guard<std::mutex> lock(mu);
-        Key key{q, k_cache, v_cache, o, B, H, D, l, cap, cache_len};
+        Key key{q, k_cache, v_cache, o, B, H, D, l, cap, cache_len, pg.table ? 1 : 0, pg.log2_ps, pg.n_pages};
         if (!(have_cache && key == cached_key)) {
             TmaMaps mnew{};
             const int64_t qs_h = (int64_t)l * D, qs_b = qs_h * H, cs_h = (int64_t)cap * D, cs_b = cs_h * H;
             const View& qv = p.view[V_TAIL];
             const View& kv = p.view[V_MEM];
             if (!encode_view(&mnew.q[V_TAIL], q, qv, D, B, H, 0, qs_b, qs_h, D, l) ||
-                !encode_view(&mnew.o[V_TAIL], o, qv, D, B, H, 0, qs_b, qs_h, D, l) ||
-                !encode_view(&mnew.k[V_MEM], k_cache, kv, D, B, H, 0, cs_b, cs_h, D, cache_len + l) ||
-                !encode_view(&mnew.v[V_MEM], v_cache, kv, D, B, H, 0, cs_b, cs_h, D, cache_len + l))
+                !encode_view(&mnew.o[V_TAIL], o, qv, D, B, H, 0, qs_b, qs_h, D, l))
                 return cudaErrorNotSupported;
+            if (pg.table) {
+                // the pool [n_pages, H, page_size, D] seen as n_pages "batch elements" of one zone of page_size rows
+                const int ps = 1 << pg.log2_ps;
+                const View pv = make_view(ps, 1, 0, 0);
+                const int64_t ps_h = (int64_t)ps * D, ps_b = ps_h * H;
+                if (!encode_view(&mnew.k[V_MEM], k_cache, pv, D, pg.n_pages, H, 0, ps_b, ps_h, D, ps) ||
+                    !encode_view(&mnew.v[V_MEM], v_cache, pv, D, pg.n_pages, H, 0, ps_b, ps_h, D, ps))
+                    return cudaErrorNotSupported;
+            } else if (!encode_view(&mnew.k[V_MEM], k_cache, kv, D, B, H, 0, cs_b, cs_h, D, cache_len + l) ||
+                       !encode_view(&mnew.v[V_MEM], v_cache, kv, D, B, H, 0, cs_b, cs_h, D, cache_len + l)) {
+                return cudaErrorNotSupported;
+            }
             cached_maps = mnew;
             cached_key = key;
             have_cache = true;

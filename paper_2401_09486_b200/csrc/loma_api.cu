@@ -440,9 +440,10 @@ static int prefill_attn_impl(const void* q, const void* k_new, const void* v_new
                              const Paging& pg, loma_dtype dtype, float softmax_scale, unsigned flags, void* stream) {
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // the tensor-core kernel (bf16, contiguous cache; a handful of rows is cheaper on CUDA cores, one warp per row:
+    // the tensor-core kernel (bf16; a handful of rows is cheaper on CUDA cores, one warp per row:
     // from 8 rows on one pass of the cache through the tensor-core kernel wins over l passes)
-    const bool tc = dtype == LOMA_BF16 && l >= 8 && !pg.table && !(flags & LOMA_FLAG_FORCE_GENERIC);
+    // (over a paged cache only when a page holds a multiple of 128 rows: a 128-key tile then lies in one page)
+    const bool tc = dtype == LOMA_BF16 && l >= 8 && (!pg.table || pg.log2_ps >= 7) && !(flags & LOMA_FLAG_FORCE_GENERIC);
     // 1. the new tokens' K/V go into the cache (bit-exact); 2. every new row attends to cache rows 0 .. len + i.
     // With per-sequence lengths the tensor-core kernel also wants the rest of each sequence's last 128-row key tile finite.
     const int pad_to = (tc && cache_lens) ? 128 : 1;
@@ -453,7 +454,7 @@ static int prefill_attn_impl(const void* q, const void* k_new, const void* v_new
     }
     cudaError_t e = cudaErrorNotSupported;
     if (tc) {
-        e = launch_prefill_attn_tc(q, k_cache, v_cache, o, lse, B, H, D, l, cap, cache_len, cache_lens, scale, st);
+        e = launch_prefill_attn_tc(q, k_cache, v_cache, o, lse, B, H, D, l, cap, cache_len, cache_lens, pg, scale, st);
         if (e == cudaErrorNotSupported) g_fallbacks.fetch_add(1, std::memory_order_relaxed);
     }
     if (e == cudaErrorNotSupported)

@@ -123,8 +123,8 @@ cudaError_t launch_masked_attn_tc(const void* q, const void* k, const void* v, v
 
 // l new tokens over a cache that already holds their K/V at [cache_len, cache_len + l) (attn_tcgen05.cu)
 cudaError_t launch_prefill_attn_tc(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse, int B,
-                                   int H, int D, int l, int cap, int cache_len, const int32_t* cache_lens, float scale,
-                                   cudaStream_t st);
+                                   int H, int D, int l, int cap, int cache_len, const int32_t* cache_lens,
+                                   const Paging& pg, float scale, cudaStream_t st);
 // the same on CUDA cores (any l, fp32 or bf16), and the bit-exact append that precedes both (attn_generic.cu)
 cudaError_t launch_prefill_attn_generic(const void* q, const void* k_cache, const void* v_cache, void* o, float* lse,
                                         int B, int H, int D, int l, int cap, int cache_len, const int32_t* lens,

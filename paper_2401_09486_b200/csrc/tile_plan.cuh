@@ -62,6 +62,8 @@ struct FwdParams {
     unsigned flags;
     int prefill;       // 1: the plan of loma_prefill_attn (query view V_TAIL over the new tokens, key view V_MEM over the cache)
     const int* prefill_lens;   // prefill plan of a ragged batch: [B] cache lengths on the device (NULL: uniform)
+    const int* page_table;     // ... over a paged cache: block table [B, pt_stride] (pages of 2^log2_ps >= 128 rows)
+    int pt_stride, log2_ps, n_pages;
     FastDiv dBH, dH, dTT;   // division by BH, H and total_tiles
     float scale_log2;
     float* lse;
@@ -382,7 +384,7 @@ inline void make_plan(const Layout& L, int B, int H, FwdParams* p) {
     p->n_tail = p->view[V_TAIL].ntiles; p->n_read = p->view[V_READ].ntiles;
     p->n_mem = p->view[V_MEM].ntiles; p->n_rep = p->view[V_REP].ntiles;
     p->total_tiles = p->n_tail + p->n_read + p->n_mem + p->n_rep;
-    p->flags = L.flags; p->prefill = 0; p->prefill_lens = nullptr;
+    p->flags = L.flags; p->prefill = 0; p->prefill_lens = nullptr; p->page_table = nullptr;
     p->dBH = make_fastdiv(p->BH); p->dH = make_fastdiv(H); p->dTT = make_fastdiv(p->total_tiles);
 }
 
@@ -398,7 +400,7 @@ inline void make_prefill_plan(int l, int cache_len, int B, int H, FwdParams* p) 
     p->n_chunks = 0; p->s = 0; p->S = l; p->H = H; p->BH = B * H;
     p->n_tail = p->view[V_TAIL].ntiles; p->n_read = 0; p->n_mem = 0; p->n_rep = 0;
     p->total_tiles = p->n_tail;
-    p->flags = 0; p->prefill = 1; p->prefill_lens = nullptr;
+    p->flags = 0; p->prefill = 1; p->prefill_lens = nullptr; p->page_table = nullptr;
     p->dBH = make_fastdiv(p->BH); p->dH = make_fastdiv(H); p->dTT = make_fastdiv(p->total_tiles);
 }
 

@@ -340,10 +340,13 @@ def test_ragged_prefill_with_equal_lengths_equals_the_uniform_call_bit_for_bit()
 
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("l,ps,lens", [(1, 16, [0, 5, 130]), (17, 16, [16, 0, 300]), (70, 64, [100, 513, 0, 64])])
+@pytest.mark.parametrize("l,ps,lens", [(1, 16, [0, 5, 130]), (17, 16, [16, 0, 300]), (70, 64, [100, 513, 0, 64]),
+                                       (70, 128, [100, 513, 0, 64]), (200, 256, [300, 5, 1000]), (8, 128, [127, 128, 121])])
 def test_paged_prefill_matches_the_oracle_per_sequence(l, ps, lens, dtype):
     """The same step over a paged cache: pages scattered over the pool by a seeded permutation; the new rows
-    land in the pages the block table names, bit for bit."""
+    land in the pages the block table names, bit for bit.  (bf16 with pages of 128 rows or more runs on the
+    tensor-core kernel.)  Every pool row that is not one of a sequence's first cache_lens[b] entries starts out as
+    NaN: none of them may reach an output."""
     B, H, D = len(lens), 2, 128
     max_len = max(lens)
     mp = (max_len + l + ps - 1) // ps + 1
@@ -353,6 +356,12 @@ def test_paged_prefill_matches_the_oracle_per_sequence(l, ps, lens, dtype):
     kpool = synthetic.normal_tensor((n_pages, H, ps, D), 81, 1.0, dtype)
     vpool = synthetic.normal_tensor((n_pages, H, ps, D), 82, 1.0, dtype)
     q, kn, vn = synthetic.qkv(B, H, l, D, seed=83, std=1.0, dtype=dtype)
+    owned = torch.zeros((n_pages, ps), dtype=torch.bool)
+    for b, n in enumerate(lens):
+        for j in range(n):
+            owned[int(table[b, j // ps]), j % ps] = True
+    kpool[~owned[:, None, :].expand(n_pages, H, ps)] = float("nan")
+    vpool[~owned[:, None, :].expand(n_pages, H, ps)] = float("nan")
 
     def gather(pool, b, n):   # the first n entries of sequence b as [1, H, n, D]
         rows = [pool[int(table[b, j // ps]), :, j % ps] for j in range(n)]
@@ -361,9 +370,12 @@ def test_paged_prefill_matches_the_oracle_per_sequence(l, ps, lens, dtype):
     kpd, vpd = kpool.to(DEV), vpool.to(DEV)
     o = torch.full((B, H, l, D), float("nan"), dtype=dtype, device=DEV)
     lse = torch.full((B, H, l), float("nan"), dtype=torch.float32, device=DEV)
+    fallbacks = L.loma_fallback_count()
     L.loma_prefill_attn_paged(q.to(DEV), kn.to(DEV), vn.to(DEV), kpd, vpd, table.to(DEV), o, lse,
                               torch.tensor(lens, dtype=torch.int32, device=DEV), max_len)
     torch.cuda.synchronize()
+    assert L.loma_fallback_count() == fallbacks       # a tensor-core call did not end up on CUDA cores
+    assert L.loma_device_status() == 0
     kp_after, vp_after = kpd.cpu(), vpd.cpu()
     for b, n in enumerate(lens):
         sl = slice(b, b + 1)
