@@ -467,6 +467,39 @@ LOMA_API int loma_prefill_attn_paged(const void* q, const void* k_new, const voi
                                      int max_cache_len, loma_dtype dtype, float softmax_scale, unsigned flags,
                                      void* stream);
 
+/* ---------------------------------------------------------------------------
+ * loma_prefill_attn_rope, loma_prefill_attn_ragged_rope, loma_prefill_attn_paged_rope -- the
+ * prompt piece with the rotary embedding of Section 4.5 fused in (rotation as in
+ * loma_rope_apply): new token i of a sequence is rotated by the id pos0 + i -- Appendix A,
+ * `inference_input`: position_ids = cursor .. cursor + l - 1, the count of tokens seen so
+ * far, not the cache length.  q is rotated on its way into the step (the caller's q is
+ * left as it is; o serves as the scratch for the rotated queries before it receives the
+ * output); k_new is rotated, rounded to the storage type and appended -- the cache holds
+ * rotated keys, as after loma_decode_attn_rope; v_new is appended as it is.
+ *
+ *   pos0                   id of the piece's first token, the same for every sequence
+ *   positions [device, in] ragged / paged: int32 [B], the id of every sequence's first new token
+ *   theta_base             <= 0 selects 10000
+ * k_new and v_new are required.  Everything else, and the errors, as the entry point
+ * without the suffix; INVALID_ARG also for a negative pos0, an id that would pass
+ * INT_MAX, or a missing positions array.
+ * ------------------------------------------------------------------------- */
+LOMA_API int loma_prefill_attn_rope(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                                    void* o, float* lse, int B, int H, int D, int l, int cap, int cache_len, int pos0,
+                                    float theta_base, loma_dtype dtype, float softmax_scale, unsigned flags,
+                                    void* stream);
+LOMA_API int loma_prefill_attn_ragged_rope(const void* q, const void* k_new, const void* v_new, void* k_cache,
+                                           void* v_cache, void* o, float* lse, int B, int H, int D, int l, int cap,
+                                           const int32_t* cache_lens, int max_cache_len, const int32_t* positions,
+                                           float theta_base, loma_dtype dtype, float softmax_scale, unsigned flags,
+                                           void* stream);
+LOMA_API int loma_prefill_attn_paged_rope(const void* q, const void* k_new, const void* v_new, void* k_pool,
+                                          void* v_pool, const int32_t* block_table, void* o, float* lse, int B, int H,
+                                          int D, int l, int page_size, int max_pages, int n_pages,
+                                          const int32_t* cache_lens, int max_cache_len, const int32_t* positions,
+                                          float theta_base, loma_dtype dtype, float softmax_scale, unsigned flags,
+                                          void* stream);
+
 /* Host-only replay of the tile plan the tensor-core kernel follows for loma_prefill_attn
  * (Appendix A, inference_input mask): counts[i*(cache_len+l) + j] = number of visits in
  * which new token i attends to key j, into a [host] uint8 buffer of l*(cache_len+l) bytes.

@@ -43,6 +43,10 @@ SIGNATURES = {
     "loma_prefill_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _f, _u, _p]),
     "loma_prefill_attn_ragged": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p]),
     "loma_prefill_attn_paged": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _p, _i, _i, _f, _u, _p]),
+    "loma_prefill_attn_rope": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _f, _i, _f, _u, _p]),
+    "loma_prefill_attn_ragged_rope": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _p, _i, _p, _f, _i, _f, _u, _p]),
+    "loma_prefill_attn_paged_rope": (_i, [_p, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _i, _p, _i, _p, _f, _i, _f,
+                                          _u, _p]),
     "loma_prefill_attn_plan_coverage": (_i, [_i, _i, _p]),
     "loma_decode_attn": (_i, [_p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
     "loma_decode_attn_layers": (_i, [_i, _p, _p, _p, _p, _p, _p, _p, _i, _i, _i, _i, _i, _i, _f, _u, _p, _sz, _p]),
@@ -271,6 +275,48 @@ def loma_prefill_attn_paged(q, k_new, v_new, k_pool, v_pool, block_table, o, lse
                                        _ptr(cache_lens), int(max_cache_len), _dtype_code(q), float(softmax_scale),
                                        int(flags), _stream(stream))
     _check(rc, "loma_prefill_attn_paged")
+
+
+def loma_prefill_attn_rope(q, k_new, v_new, k_cache, v_cache, o, lse, cache_len: int, pos0: int, flags: int = 0,
+                           softmax_scale: float = 0.0, theta_base: float = 0.0, stream=None) -> None:
+    """loma_prefill_attn with q and k_new rotated at the ids pos0 .. pos0 + l - 1 on the way in."""
+    B, H, l, D = q.shape
+    for x in (q, k_new, v_new, k_cache, v_cache, o):
+        if x is not None and not x.is_contiguous():
+            raise ValueError("loma_prefill_attn_rope takes contiguous tensors")
+    rc = lib().loma_prefill_attn_rope(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(o), _ptr(lse),
+                                      B, H, D, l, k_cache.shape[2], int(cache_len), int(pos0), float(theta_base),
+                                      _dtype_code(q), float(softmax_scale), int(flags), _stream(stream))
+    _check(rc, "loma_prefill_attn_rope")
+
+
+def loma_prefill_attn_ragged_rope(q, k_new, v_new, k_cache, v_cache, o, lse, cache_lens, max_cache_len: int, positions,
+                                  flags: int = 0, softmax_scale: float = 0.0, theta_base: float = 0.0, stream=None) -> None:
+    """loma_prefill_attn_ragged with the rotation fused in; positions: int32 [B], id of every sequence's first new token."""
+    B, H, l, D = q.shape
+    for x in (q, k_new, v_new, k_cache, v_cache, o):
+        if x is not None and not x.is_contiguous():
+            raise ValueError("loma_prefill_attn_ragged_rope takes contiguous tensors")
+    _check_positions(positions, B, "positions")
+    rc = lib().loma_prefill_attn_ragged_rope(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_cache), _ptr(v_cache), _ptr(o),
+                                             _ptr(lse), B, H, D, l, k_cache.shape[2], _ptr(cache_lens), int(max_cache_len),
+                                             _ptr(positions), float(theta_base), _dtype_code(q), float(softmax_scale),
+                                             int(flags), _stream(stream))
+    _check(rc, "loma_prefill_attn_ragged_rope")
+
+
+def loma_prefill_attn_paged_rope(q, k_new, v_new, k_pool, v_pool, block_table, o, lse, cache_lens, max_cache_len: int,
+                                 positions, flags: int = 0, softmax_scale: float = 0.0, theta_base: float = 0.0,
+                                 stream=None) -> None:
+    """loma_prefill_attn_paged with the rotation fused in."""
+    B, H, l, D = q.shape
+    _check_positions(positions, B, "positions")
+    n_pages, _, page_size, _ = k_pool.shape
+    rc = lib().loma_prefill_attn_paged_rope(_ptr(q), _ptr(k_new), _ptr(v_new), _ptr(k_pool), _ptr(v_pool), _ptr(block_table),
+                                            _ptr(o), _ptr(lse), B, H, D, l, page_size, block_table.shape[1], n_pages,
+                                            _ptr(cache_lens), int(max_cache_len), _ptr(positions), float(theta_base),
+                                            _dtype_code(q), float(softmax_scale), int(flags), _stream(stream))
+    _check(rc, "loma_prefill_attn_paged_rope")
 
 
 def loma_prefill_attn_plan_coverage(l: int, cache_len: int) -> torch.Tensor:

@@ -352,7 +352,8 @@ prefill_generic_kernel(const T* __restrict__ q, const T* __restrict__ k_cache, c
 // the contents of the cache past the valid length are unspecified anyway.  k_new == NULL: only that.
 __global__ void cache_append_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
                                     uint4* __restrict__ k_cache, uint4* __restrict__ v_cache, int vec_per_row, int l, int cap,
-                                    int cache_len, const int32_t* __restrict__ lens, int H, Paging pg, int pad_to) {
+                                    int cache_len, const int32_t* __restrict__ lens, int H, Paging pg, int pad_to,
+                                    int copy_k) {
     const int bh = blockIdx.y;
     const int b = bh / H, h = bh - b * H;
     const int own = lens ? min(max(__ldg(lens + b), 0), cache_len) : cache_len;
@@ -369,12 +370,48 @@ __global__ void cache_append_kernel(const uint4* __restrict__ k_new, const uint4
         const int r = (int)(e / vec_per_row), cv = (int)(e - (int64_t)r * vec_per_row);
         const int64_t out = slot(own + r) + cv;
         if (e < n_new) {
-            if (k_new) { k_cache[out] = __ldg(k_new + in + e); v_cache[out] = __ldg(v_new + in + e); }
+            if (k_new && copy_k) k_cache[out] = __ldg(k_new + in + e);   // (copy_k == 0: the keys arrive rotated, from another kernel)
+            if (v_new) v_cache[out] = __ldg(v_new + in + e);
         } else {
             k_cache[out] = make_uint4(0, 0, 0, 0);
             v_cache[out] = make_uint4(0, 0, 0, 0);
         }
     }
+}
+
+// Rotary embedding of a prompt piece (Section 4.5; Appendix A, inference_input: new token i of a sequence has the id
+// cursor + i): q rotated into q_rot (the caller's output buffer, which the attention kernels then read as their
+// query), k_new rotated, rounded to the storage type and written to the cache rows [len, len + l).  One thread per
+// feature pair (d, d + D/2).
+template <typename T, int D>
+__global__ void __launch_bounds__(128)
+prefill_rope_kernel(const T* __restrict__ q, const T* __restrict__ k_new, T* __restrict__ q_rot, T* __restrict__ k_cache,
+                    int l, int cap, int cache_len, const int32_t* __restrict__ lens, int H, Paging pg, RopeArgs rope) {
+    constexpr int HALF = D / 2, RPB = 128 / HALF;      // rows per block
+    const int i = blockIdx.x * RPB + threadIdx.x / HALF, d = threadIdx.x % HALF;
+    if (i >= l) return;
+    const int bh = blockIdx.y, b = bh / H, h = bh - b * H;
+    const int own = lens ? min(max(__ldg(lens + b), 0), cache_len) : cache_len;
+    const int pos = (rope.pos_seq ? __ldg(rope.pos_seq + b) : rope.pos0) + i * rope.stride;
+    float c, sn;
+    rope_cos_sin(pos, d, D, rope.log2_base, c, sn);
+    const int64_t row = ((int64_t)bh * l + i) * D;
+    {
+        const float a = to_f32(q[row + d]), bb = to_f32(q[row + d + HALF]);
+        q_rot[row + d] = from_f32<T>(a * c - bb * sn);
+        q_rot[row + d + HALF] = from_f32<T>(bb * c + a * sn);
+    }
+    const int j = own + i;
+    int64_t out;
+    if (!pg.table) {
+        out = ((int64_t)bh * cap + j) * D;
+    } else {
+        const int page = min(max(__ldg(pg.table + (int64_t)b * pg.max_pages + (j >> pg.log2_ps)), 0), pg.n_pages - 1);
+        out = ((((int64_t)page * H + h) << pg.log2_ps) + (j & ((1 << pg.log2_ps) - 1))) * D;
+    }
+    const float a = to_f32(k_new[row + d]), bb = to_f32(k_new[row + d + HALF]);
+    k_cache[out + d] = from_f32<T>(a * c - bb * sn);
+    k_cache[out + d + HALF] = from_f32<T>(bb * c + a * sn);
 }
 
 // ------------------------------------------------------------- compress map
@@ -773,7 +810,7 @@ cudaError_t launch_prefill_attn_generic(const void* q, const void* k_cache, cons
 // pad_to: see cache_append_kernel (1: plain append)
 cudaError_t launch_cache_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache, int B, int H,
                                 int row_bytes, int l, int cap, int cache_len, const int32_t* lens, const Paging& pg,
-                                int pad_to, cudaStream_t st) {
+                                int pad_to, bool copy_k, cudaStream_t st) {
     const int vec = row_bytes / 16;
     const int64_t n = (int64_t)(l + (pad_to > 1 ? pad_to : 0)) * vec;
     int gx = (int)((n + 255) / 256);
@@ -782,9 +819,33 @@ cudaError_t launch_cache_append(const void* k_new, const void* v_new, void* k_ca
     dim3 grid(gx, B * H);
     cache_append_kernel<<<grid, 256, 0, st>>>(static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new),
                                               static_cast<uint4*>(k_cache), static_cast<uint4*>(v_cache), vec, l, cap, cache_len,
-                                              lens, H, pg, pad_to);
+                                              lens, H, pg, pad_to, copy_k ? 1 : 0);
     count_launches(1);
     return cudaGetLastError();
+}
+
+template <typename T, int D>
+static cudaError_t prefill_rope_t(const void* q, const void* k_new, void* q_rot, void* k_cache, int BH, int l, int cap,
+                                  int cache_len, const int32_t* lens, int H, const Paging& pg, const RopeArgs& rope,
+                                  cudaStream_t st) {
+    constexpr int RPB = 128 / (D / 2);
+    dim3 grid((l + RPB - 1) / RPB, BH);
+    prefill_rope_kernel<T, D><<<grid, 128, 0, st>>>(static_cast<const T*>(q), static_cast<const T*>(k_new),
+                                                    static_cast<T*>(q_rot), static_cast<T*>(k_cache), l, cap, cache_len, lens,
+                                                    H, pg, rope);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_prefill_rope(const void* q, const void* k_new, void* q_rot, void* k_cache, int B, int H, int D, int l,
+                                int cap, int cache_len, const int32_t* lens, const Paging& pg, const RopeArgs& rope,
+                                loma_dtype dt, cudaStream_t st) {
+    const int BH = B * H;
+    if (dt == LOMA_F32)
+        return D == 64 ? prefill_rope_t<float, 64>(q, k_new, q_rot, k_cache, BH, l, cap, cache_len, lens, H, pg, rope, st)
+                       : prefill_rope_t<float, 128>(q, k_new, q_rot, k_cache, BH, l, cap, cache_len, lens, H, pg, rope, st);
+    return D == 64 ? prefill_rope_t<__nv_bfloat16, 64>(q, k_new, q_rot, k_cache, BH, l, cap, cache_len, lens, H, pg, rope, st)
+                   : prefill_rope_t<__nv_bfloat16, 128>(q, k_new, q_rot, k_cache, BH, l, cap, cache_len, lens, H, pg, rope, st);
 }
 
 }  // namespace loma

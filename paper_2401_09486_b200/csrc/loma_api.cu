@@ -437,7 +437,8 @@ static int log2_exact(int x);   // defined with the paged entry points below
 // per-sequence lengths are clamped to; pg.table given: the cache is the paged pool and cap = max_pages * page_size.
 static int prefill_attn_impl(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
                              float* lse, int B, int H, int D, int l, int cap, int cache_len, const int32_t* cache_lens,
-                             const Paging& pg, loma_dtype dtype, float softmax_scale, unsigned flags, void* stream) {
+                             const Paging& pg, loma_dtype dtype, float softmax_scale, unsigned flags, void* stream,
+                             const RopeArgs& rope = RopeArgs{}) {
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)D);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // the tensor-core kernel (bf16; a handful of rows is cheaper on CUDA cores, one warp per row:
@@ -449,8 +450,17 @@ static int prefill_attn_impl(const void* q, const void* k_new, const void* v_new
     const int pad_to = (tc && cache_lens) ? 128 : 1;
     if (k_new || pad_to > 1) {
         if (launch_cache_append(k_new, v_new, k_cache, v_cache, B, H, (int)(D * elt_size(dtype)), l, cap, cache_len,
-                                cache_lens, pg, pad_to, st) != cudaSuccess)
+                                cache_lens, pg, pad_to, !rope.on, st) != cudaSuccess)
             return LOMA_ERR_CUDA;
+    }
+    if (rope.on) {
+        // Section 4.5: q and the new keys are rotated at the ids cursor + i.  The rotated keys go straight into the
+        // cache; the rotated queries into o, which the attention kernels below then read as their query (every
+        // tile or row reads its own query rows before it writes the same rows of the output).
+        if (launch_prefill_rope(q, k_new, o, k_cache, B, H, D, l, cap, cache_len, cache_lens, pg, rope, dtype, st) !=
+            cudaSuccess)
+            return LOMA_ERR_CUDA;
+        q = o;
     }
     cudaError_t e = cudaErrorNotSupported;
     if (tc) {
@@ -533,6 +543,101 @@ int loma_prefill_attn_paged(const void* q, const void* k_new, const void* v_new,
     pg.table = block_table; pg.max_pages = max_pages; pg.log2_ps = l2; pg.n_pages = n_pages;
     return prefill_attn_impl(q, k_new, v_new, k_pool, v_pool, o, lse, B, H, D, l, max_pages * page_size, max_cache_len,
                              cache_lens, pg, dtype, softmax_scale, flags, stream);
+}
+
+// The prompt piece with the rotation fused in.  Shared checks of the three forms; then the plain entry point's own.
+static int prefill_rope_args(int B, int H, int l, const void* k_new, const void* v_new, int pos0, const int32_t* positions,
+                             bool per_sequence, float theta_base, RopeArgs* rope) {
+    if (B > 0 && H > 0 && l > 0 && (!k_new || !v_new)) return LOMA_ERR_INVALID_ARG;   // the keys to rotate have to be given
+    if (per_sequence) {
+        if (B > 0 && H > 0 && l > 0 && !positions) return LOMA_ERR_INVALID_ARG;
+        if ((uintptr_t)positions & 3u) return LOMA_ERR_ALIGNMENT;
+    } else if (pos0 < 0 || (l > 0 && (int64_t)pos0 + l - 1 > INT_MAX)) {
+        return LOMA_ERR_INVALID_ARG;
+    }
+    rope->on = 1; rope->pos0 = pos0; rope->stride = 1; rope->pos_seq = per_sequence ? positions : nullptr;
+    rope->log2_base = log2(theta_base > 0.f ? (double)theta_base : 10000.0);
+    return LOMA_OK;
+}
+
+int loma_prefill_attn_rope(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache, void* o,
+                           float* lse, int B, int H, int D, int l, int cap, int cache_len, int pos0, float theta_base,
+                           loma_dtype dtype, float softmax_scale, unsigned flags, void* stream) {
+    RopeArgs rope;
+    const int rc = prefill_rope_args(B, H, l, k_new, v_new, pos0, nullptr, false, theta_base, &rope);
+    if (rc != LOMA_OK) return rc;
+    if (B < 0 || H < 0 || l < 0 || cap < 0 || cache_len < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    if ((int64_t)cache_len + l > cap) return LOMA_ERR_CAPACITY;
+    if (B == 0 || H == 0 || l == 0) return LOMA_OK;
+    if (!q || !k_cache || !v_cache || !o) return LOMA_ERR_INVALID_ARG;
+    if (o == q || o == k_new || o == v_new) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) || !aligned16(k_new) ||
+        !aligned16(v_new))
+        return LOMA_ERR_ALIGNMENT;
+    if (lse && ((uintptr_t)lse & 3u)) return LOMA_ERR_ALIGNMENT;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    return prefill_attn_impl(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, l, cap, cache_len, nullptr, Paging{}, dtype,
+                             softmax_scale, flags, stream, rope);
+}
+
+int loma_prefill_attn_ragged_rope(const void* q, const void* k_new, const void* v_new, void* k_cache, void* v_cache,
+                                  void* o, float* lse, int B, int H, int D, int l, int cap, const int32_t* cache_lens,
+                                  int max_cache_len, const int32_t* positions, float theta_base, loma_dtype dtype,
+                                  float softmax_scale, unsigned flags, void* stream) {
+    RopeArgs rope;
+    const int rc = prefill_rope_args(B, H, l, k_new, v_new, 0, positions, true, theta_base, &rope);
+    if (rc != LOMA_OK) return rc;
+    if (B < 0 || H < 0 || l < 0 || cap < 0 || max_cache_len < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    if ((int64_t)max_cache_len + l > cap) return LOMA_ERR_CAPACITY;
+    if (B == 0 || H == 0 || l == 0) return LOMA_OK;
+    if (!q || !k_cache || !v_cache || !o || !cache_lens) return LOMA_ERR_INVALID_ARG;
+    if (o == q || o == k_new || o == v_new) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(o) || !aligned16(k_new) ||
+        !aligned16(v_new) || ((uintptr_t)cache_lens & 3u))
+        return LOMA_ERR_ALIGNMENT;
+    if (lse && ((uintptr_t)lse & 3u)) return LOMA_ERR_ALIGNMENT;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    return prefill_attn_impl(q, k_new, v_new, k_cache, v_cache, o, lse, B, H, D, l, cap, max_cache_len, cache_lens, Paging{},
+                             dtype, softmax_scale, flags, stream, rope);
+}
+
+int loma_prefill_attn_paged_rope(const void* q, const void* k_new, const void* v_new, void* k_pool, void* v_pool,
+                                 const int32_t* block_table, void* o, float* lse, int B, int H, int D, int l,
+                                 int page_size, int max_pages, int n_pages, const int32_t* cache_lens, int max_cache_len,
+                                 const int32_t* positions, float theta_base, loma_dtype dtype, float softmax_scale,
+                                 unsigned flags, void* stream) {
+    RopeArgs rope;
+    const int rc = prefill_rope_args(B, H, l, k_new, v_new, 0, positions, true, theta_base, &rope);
+    if (rc != LOMA_OK) return rc;
+    if (B < 0 || H < 0 || l < 0 || max_pages < 0 || n_pages < 0 || max_cache_len < 0) return LOMA_ERR_INVALID_ARG;
+    if (dtype != LOMA_F32 && dtype != LOMA_BF16) return LOMA_ERR_UNSUPPORTED;
+    if (D != 64 && D != 128) return LOMA_ERR_UNSUPPORTED;
+    const int l2 = log2_exact(page_size);
+    if (l2 < 0 || page_size > 65536) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)max_cache_len + l > (int64_t)max_pages * page_size) return LOMA_ERR_CAPACITY;
+    if ((int64_t)max_pages * page_size > INT_MAX) return LOMA_ERR_INVALID_ARG;
+    if (B == 0 || H == 0 || l == 0) return LOMA_OK;
+    if (!q || !k_pool || !v_pool || !o || !block_table || !cache_lens || n_pages < 1) return LOMA_ERR_INVALID_ARG;
+    if (o == q || o == k_new || o == v_new) return LOMA_ERR_INVALID_ARG;
+    if ((int64_t)B * H > 65535) return LOMA_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_pool) || !aligned16(v_pool) || !aligned16(o) || !aligned16(k_new) ||
+        !aligned16(v_new) || ((uintptr_t)cache_lens & 3u) || ((uintptr_t)block_table & 3u))
+        return LOMA_ERR_ALIGNMENT;
+    if (lse && ((uintptr_t)lse & 3u)) return LOMA_ERR_ALIGNMENT;
+    const int dc = check_device();
+    if (dc != LOMA_OK) return dc;
+    Paging pg;
+    pg.table = block_table; pg.max_pages = max_pages; pg.log2_ps = l2; pg.n_pages = n_pages;
+    return prefill_attn_impl(q, k_new, v_new, k_pool, v_pool, o, lse, B, H, D, l, max_pages * page_size, max_cache_len,
+                             cache_lens, pg, dtype, softmax_scale, flags, stream, rope);
 }
 
 int loma_prefill_attn_plan_coverage(int l, int cache_len, uint8_t* counts) {

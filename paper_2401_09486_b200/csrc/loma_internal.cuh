@@ -131,7 +131,10 @@ cudaError_t launch_prefill_attn_generic(const void* q, const void* k_cache, cons
                                         const Paging& pg, loma_dtype dt, float scale, cudaStream_t st);
 cudaError_t launch_cache_append(const void* k_new, const void* v_new, void* k_cache, void* v_cache, int B, int H,
                                 int row_bytes, int l, int cap, int cache_len, const int32_t* lens, const Paging& pg,
-                                int pad_to, cudaStream_t st);
+                                int pad_to, bool copy_k, cudaStream_t st);
+cudaError_t launch_prefill_rope(const void* q, const void* k_new, void* q_rot, void* k_cache, int B, int H, int D, int l,
+                                int cap, int cache_len, const int32_t* lens, const Paging& pg, const RopeArgs& rope,
+                                loma_dtype dt, cudaStream_t st);
 
 void plan_coverage_host(const Layout& L, uint8_t* counts);          // tile_plan_host.cu
 void prefill_plan_coverage_host(int l, int cache_len, uint8_t* counts);

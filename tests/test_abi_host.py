@@ -474,3 +474,36 @@ def test_ragged_and_paged_prefill_validation(lib):
     assert pag(bt=0x6002) == ALIGNMENT
     assert pag(dt=7) == UNSUPPORTED
     assert pag(l=0) == 0
+
+
+def test_rope_fused_prompt_piece_validation(lib):
+    def uni(q=0x1000, kn=0x2000, vn=0x3000, kc=0x4000, vc=0x5000, o=0x6000, B=2, H=1, D=128, l=4, cap=20, cache_len=16,
+            pos0=100, dt=1):
+        return lib.loma_prefill_attn_rope(q, kn, vn, kc, vc, o, None, B, H, D, l, cap, cache_len, pos0, 0.0, dt, 0.0, 0, None)
+    assert uni(pos0=-1) == INVALID
+    assert uni(pos0=2**31 - 2) == INVALID                # the last id would overflow
+    assert uni(kn=None, vn=None) == INVALID              # the keys to rotate have to be given
+    assert uni(cache_len=17) == CAPACITY
+    assert uni(D=96) == UNSUPPORTED
+    assert uni(o=0x1000) == INVALID
+    assert uni(l=0) == 0
+
+    def rag(q=0x1000, kn=0x2000, vn=0x3000, kc=0x4000, vc=0x5000, o=0x6000, B=2, H=1, D=128, l=4, cap=20, lens=0x7000, mx=16,
+            pos=0x9000, dt=1):
+        return lib.loma_prefill_attn_ragged_rope(q, kn, vn, kc, vc, o, None, B, H, D, l, cap, lens, mx, pos, 0.0, dt, 0.0, 0,
+                                                 None)
+    assert rag(pos=None) == INVALID
+    assert rag(pos=0x9002) == ALIGNMENT
+    assert rag(lens=None) == INVALID
+    assert rag(mx=17) == CAPACITY
+    assert rag(B=0) == 0
+
+    def pag(q=0x1000, kn=0x2000, vn=0x3000, kp=0x4000, vp=0x5000, bt=0x6000, o=0x7000, B=2, H=1, D=128, l=4, ps=16, mp=2,
+            npg=8, lens=0x8000, mx=28, pos=0x9000, dt=1):
+        return lib.loma_prefill_attn_paged_rope(q, kn, vn, kp, vp, bt, o, None, B, H, D, l, ps, mp, npg, lens, mx, pos, 0.0,
+                                                dt, 0.0, 0, None)
+    assert pag(pos=None) == INVALID
+    assert pag(mx=29) == CAPACITY
+    assert pag(ps=24) == INVALID
+    assert pag(bt=None) == INVALID
+    assert pag(l=0) == 0

@@ -351,3 +351,77 @@ def test_staggered_sequences_over_a_paged_cache_with_fused_rotation(dtype):
     torch.cuda.synchronize()
     live = zone != oracle.ZONE_REP
     check(got[:, :, torch.from_numpy(live).to(DEV)], want_o[:, :, live], dtype)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("flags", [0, L.LOMA_FLAG_FORCE_GENERIC])
+@pytest.mark.parametrize("l,cache_len,pos0", [(1, 5, 5), (17, 100, 4000), (200, 333, 30000), (64, 0, 0)])
+def test_prompt_piece_with_fused_rotation_matches_oracle(l, cache_len, pos0, flags, dtype):
+    """Appendix A `inference_input` with l tokens and position_ids cursor .. cursor + l - 1: the step equals
+    rotate-then-attend in the oracle, the cache receives the rotated keys (rounded once), the caller's q is untouched."""
+    B, H, D = 2, 2, 128
+    cap = cache_len + l + 3
+    kc = synthetic.normal_tensor((B, H, cap, D), 171, 1.0, dtype)
+    vc = synthetic.normal_tensor((B, H, cap, D), 172, 1.0, dtype)
+    q, kn, vn = synthetic.qkv(B, H, l, D, seed=173, std=1.0, dtype=dtype)
+    pos = [pos0 + i for i in range(l)]
+    q_rot = oracle.rope_rotate(npf(q), pos)
+    k_rot = oracle.rope_rotate(npf(kn), pos)
+    want_o, want_lse, _, _ = oracle.prefill_attn(q_rot, _round_to(k_rot, dtype), npf(vn), npf(kc), npf(vc), cache_len)
+    kcd, vcd, qd = kc.to(DEV), vc.to(DEV), q.to(DEV)
+    o = torch.full((B, H, l, D), float("nan"), dtype=dtype, device=DEV)
+    lse = torch.full((B, H, l), float("nan"), dtype=torch.float32, device=DEV)
+    L.loma_prefill_attn_rope(qd, kn.to(DEV), vn.to(DEV), kcd, vcd, o, lse, cache_len, pos0, flags)
+    torch.cuda.synchronize()
+    check(o, want_o, dtype)
+    assert np.abs(npf(lse) - want_lse).max() <= (1e-5 if dtype == torch.float32 else 2e-2)
+    assert torch.equal(qd.cpu(), q)
+    assert torch.equal(kcd[:, :, :cache_len].cpu(), kc[:, :, :cache_len]) and torch.equal(vcd[:, :, :cache_len].cpu(), vc[:, :, :cache_len])
+    assert torch.equal(vcd[:, :, cache_len:cache_len + l].cpu(), vn)
+    _ulp_close(kcd[:, :, cache_len:cache_len + l], k_rot, dtype)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("paged", [False, True])
+def test_ragged_and_paged_prompt_pieces_with_fused_rotation(paged, dtype):
+    """One position and one cache length per sequence; contiguous cache and 128-row pages."""
+    B, H, D, l, ps = 3, 2, 128, 40, 128
+    lens, poss = [100, 0, 300], [1000, 0, 20000]
+    max_len = max(lens)
+    q, kn, vn = synthetic.qkv(B, H, l, D, seed=181, std=1.0, dtype=dtype)
+    mp = (max_len + l + ps - 1) // ps
+    cap = mp * ps
+    kc = synthetic.normal_tensor((B, H, cap, D), 182, 1.0, dtype)
+    vc = synthetic.normal_tensor((B, H, cap, D), 183, 1.0, dtype)
+    o = torch.full((B, H, l, D), float("nan"), dtype=dtype, device=DEV)
+    lens_d = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    pos_d = torch.tensor(poss, dtype=torch.int32, device=DEV)
+    if paged:
+        g = torch.Generator().manual_seed(184)
+        table = torch.randperm(B * mp, generator=g).to(torch.int32).view(B, mp)
+        kpool = torch.empty((B * mp, H, ps, D), dtype=dtype)
+        vpool = torch.empty_like(kpool)
+        for b in range(B):
+            for pi in range(mp):
+                kpool[int(table[b, pi])] = kc[b, :, pi * ps:(pi + 1) * ps]
+                vpool[int(table[b, pi])] = vc[b, :, pi * ps:(pi + 1) * ps]
+        kpd, vpd = kpool.to(DEV), vpool.to(DEV)
+        L.loma_prefill_attn_paged_rope(q.to(DEV), kn.to(DEV), vn.to(DEV), kpd, vpd, table.to(DEV), o, None, lens_d, max_len, pos_d)
+        torch.cuda.synchronize()
+        kc_after = torch.stack([torch.cat([kpd[int(table[b, pi])].cpu() for pi in range(mp)], dim=1) for b in range(B)])
+    else:
+        kcd, vcd = kc.to(DEV), vc.to(DEV)
+        L.loma_prefill_attn_ragged_rope(q.to(DEV), kn.to(DEV), vn.to(DEV), kcd, vcd, o, None, lens_d, max_len, pos_d)
+        torch.cuda.synchronize()
+        kc_after = kcd.cpu()
+    for b, (n, p0) in enumerate(zip(lens, poss)):
+        sl = slice(b, b + 1)
+        pos = [p0 + i for i in range(l)]
+        q_rot = oracle.rope_rotate(npf(q[sl]), pos)
+        k_rot = oracle.rope_rotate(npf(kn[sl]), pos)
+        want_o, _, _, _ = oracle.prefill_attn(q_rot, _round_to(k_rot, dtype), npf(vn[sl]), npf(kc[sl, :, :n + l]),
+                                              npf(vc[sl, :, :n + l]), n)
+        check(o[sl], want_o, dtype)
+        _ulp_close(kc_after[sl, :, n:n + l], k_rot, dtype)
+        assert torch.equal(kc_after[b, :, :n], kc[b, :, :n])
+    assert L.loma_device_status() == 0
