@@ -696,8 +696,8 @@ def large_workloads(L, synthetic, torch, dev, peaks, steps, warmup, clocks_mhz):
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from ncu captures of the --profile-case launches
 COMPRESS_TRAFFIC_B32 = 46.28e6         # compress_one_stage_kernel<128, 4>, B32 H32, c4 t16 (58.7e6 algorithmic, 46.1e6 of them reads)
 DECODE_TRAFFIC_B8_L8224 = 1.0824e9     # decode_splitkv + merge, B8 H32, 8224 rows (1.0779e9 algorithmic)
-FWD_SHORT_TRAFFIC_B1 = 128.2e6         # masked_attn_tc, one batch element of the 4608-token layout (151.0e6 algorithmic; part of O still in L2)
-FWD_LONG_TRAFFIC_8_HEADS = 552.7e6     # masked_attn_tc, 8 heads of the 69632-token layout (570.4e6 algorithmic)
+FWD_SHORT_TRAFFIC_B1 = 128.1e6         # masked_attn_tc, one batch element of the 4608-token layout (151.0e6 algorithmic; part of O still in L2)
+FWD_LONG_TRAFFIC_8_HEADS = 552.6e6     # masked_attn_tc, 8 heads of the 69632-token layout (570.4e6 algorithmic)
 
 
 def profile_case(args):
