@@ -164,11 +164,12 @@ masked_attn_tc_kernel(const __grid_constant__ TmaMaps maps, const FwdParams p) {
                     step_ktile(p, td, j, kt);
                     const View& kv = p.view[kt.view];
                     const uint32_t ph = gs & 1;
-                    const uint32_t bytes = kv.R * kv.CH * 128 * PANELS;
+                    uint32_t bytes = kv.R * kv.CH * 128 * PANELS;
                     // where the key tile lies: (row, chunk, batch) of the caller's tensor, or, over a paged cache, (row in
                     // page, 0, page) of the pool -- pages hold a multiple of 128 rows, so a tile never straddles two
                     int kr = kt.r0, kc_ = kt.c0, kb = bi;
                     if (RAGGED && p.page_table) {
+                        bytes = 128 * 128 * PANELS;   // the pool's box is always 128 rows, whatever the key view's length
                         kb = min(max(__ldg(p.page_table + (int64_t)bi * p.pt_stride + (kt.r0 >> p.log2_ps)), 0), p.n_pages - 1);
                         kr = kt.r0 & ((1 << p.log2_ps) - 1);
                         kc_ = 0;

@@ -341,7 +341,8 @@ def test_ragged_prefill_with_equal_lengths_equals_the_uniform_call_bit_for_bit()
 
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("l,ps,lens", [(1, 16, [0, 5, 130]), (17, 16, [16, 0, 300]), (70, 64, [100, 513, 0, 64]),
-                                       (70, 128, [100, 513, 0, 64]), (200, 256, [300, 5, 1000]), (8, 128, [127, 128, 121])])
+                                       (70, 128, [100, 513, 0, 64]), (200, 256, [300, 5, 1000]), (8, 128, [127, 128, 121]),
+                                       (43, 128, [0]), (81, 128, [1])])      # key view shorter than one 128-row tile
 def test_paged_prefill_matches_the_oracle_per_sequence(l, ps, lens, dtype):
     """The same step over a paged cache: pages scattered over the pool by a seeded permutation; the new rows
     land in the pages the block table names, bit for bit.  (bf16 with pages of 128 rows or more runs on the
