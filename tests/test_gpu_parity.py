@@ -390,6 +390,50 @@ def test_paged_prefill_matches_the_oracle_per_sequence(l, ps, lens, dtype):
         assert np.array_equal(bits(gather(kp_after, b, n)), bits(gather(kpool, b, n)))
 
 
+@pytest.mark.parametrize("seed", range(16))
+def test_ragged_and_paged_prompt_pieces_on_seeded_random_shapes(seed):
+    """Shapes nobody picked by hand (batch, heads, head size, piece length, cache lengths around the tile and page
+    boundaries, page size; odd seeds paged): bf16 tensor-core path against the oracle, sequence by sequence."""
+    import random
+    rnd = random.Random(1000 + seed)
+    B, H, D = rnd.randint(1, 4), rnd.randint(1, 2), rnd.choice([64, 128])
+    l = rnd.randint(8, 200)
+    lens = [rnd.choice([0, 1, 127, 128, 129, rnd.randint(0, 700)]) for _ in range(B)]
+    max_len = max(lens) + rnd.randint(0, 3)
+    paged = seed % 2 == 1
+    ps = rnd.choice([128, 256])
+    mp = (max_len + l + ps - 1) // ps + 1
+    cap = mp * ps
+    dtype = torch.bfloat16
+    kc = synthetic.normal_tensor((B, H, cap, D), 2000 + seed, 1.0, dtype)
+    vc = synthetic.normal_tensor((B, H, cap, D), 2100 + seed, 1.0, dtype)
+    q, kn, vn = synthetic.qkv(B, H, l, D, seed=2200 + seed, std=1.0, dtype=dtype)
+    o = torch.full((B, H, l, D), float("nan"), dtype=dtype, device=DEV)
+    lse = torch.full((B, H, l), float("nan"), dtype=torch.float32, device=DEV)
+    lens_d = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    if paged:
+        g = torch.Generator().manual_seed(2300 + seed)
+        table = torch.randperm(B * mp, generator=g).to(torch.int32).view(B, mp)
+        kpool = torch.empty((B * mp, H, ps, D), dtype=dtype)
+        vpool = torch.empty_like(kpool)
+        for b in range(B):
+            for pi in range(mp):
+                kpool[int(table[b, pi])] = kc[b, :, pi * ps:(pi + 1) * ps]
+                vpool[int(table[b, pi])] = vc[b, :, pi * ps:(pi + 1) * ps]
+        L.loma_prefill_attn_paged(q.to(DEV), kn.to(DEV), vn.to(DEV), kpool.to(DEV), vpool.to(DEV), table.to(DEV), o, lse,
+                                  lens_d, max_len)
+    else:
+        L.loma_prefill_attn_ragged(q.to(DEV), kn.to(DEV), vn.to(DEV), kc.to(DEV), vc.to(DEV), o, lse, lens_d, max_len)
+    torch.cuda.synchronize()
+    assert L.loma_device_status() == 0
+    for b, n in enumerate(lens):
+        sl = slice(b, b + 1)
+        want_o, want_lse, _, _ = oracle.prefill_attn(npf(q[sl]), npf(kn[sl]), npf(vn[sl]), npf(kc[sl, :, :n + l]),
+                                                     npf(vc[sl, :, :n + l]), n)
+        check_close(o[sl], want_o, dtype)
+        assert np.abs(npf(lse[sl]) - want_lse).max() <= 2e-2
+
+
 def test_prefill_with_rows_already_in_the_cache_and_repeatable():
     """k_new = v_new = NULL: the new rows are read where they already lie; two calls give the same bits."""
     B, H, D, l, cache_len = 2, 2, 128, 150, 333
