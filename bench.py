@@ -735,6 +735,19 @@ def profile_case(args):
             om = torch.empty_like(qm)
             for r in range(args.reps):
                 L.loma_compress_step(qm, km, vm, kc, vc, om, None, mem_len, c, t, ws, flags)
+    elif case in ("prefill", "prefill_ragged"):
+        # a quarter of the context workload's batch: 512 new tokens over 8192 cached entries, B8 H32 (1.1 GB of cache)
+        B, H, l, k_len = 8, 32, 512, 8192
+        kc = synthetic.big_normal_(torch.empty(B, H, k_len + l, D, dtype=bf, device=dev), 1, std)
+        vc = synthetic.big_normal_(torch.empty(B, H, k_len + l, D, dtype=bf, device=dev), 2, std)
+        q, kn, vn = (synthetic.big_normal_(torch.empty(B, H, l, D, dtype=bf, device=dev), 3 + i, std) for i in range(3))
+        o = torch.empty_like(q)
+        lens = torch.tensor([k_len - (37 * b) % 1024 for b in range(B)], dtype=torch.int32, device=dev)
+        for r in range(args.reps):
+            if case == "prefill":
+                L.loma_prefill_attn(q, kn, vn, kc, vc, o, None, k_len)
+            else:
+                L.loma_prefill_attn_ragged(q, kn, vn, kc, vc, o, None, lens, k_len)
     else:
         if case in ("masked", "bwd"):
             B, H, n, c, t = 1, 32, 32, 4, 16               # one batch element of the 4608-token layout: 151 MB per tensor
@@ -843,7 +856,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-extras", action="store_true", help="skip the large and the context workloads timed at N=1")
-    ap.add_argument("--profile-case", choices=["decode", "compress", "compress_prior", "compress_b32", "masked", "masked_long", "bwd", "bwd_long"],
+    ap.add_argument("--profile-case", choices=["decode", "compress", "compress_prior", "compress_b32", "masked", "masked_long", "bwd", "bwd_long", "prefill",
+                                                     "prefill_ragged"],
                     help="run one cut-down kernel launch sequence (for profiler captures) and exit")
     ap.add_argument("--reps", type=int, default=3, help="launches of --profile-case")
     args = ap.parse_args()
