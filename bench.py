@@ -714,7 +714,21 @@ def profile_case(args):
     D = 128
     std = 1.0 / math.sqrt(D)
     case = args.profile_case
-    if case in ("decode", "compress", "compress_prior", "compress_b32"):
+    if case == "decode_paged":
+        # the decode case below over a paged cache: 64-row pages scattered over the pool by a seeded permutation
+        B, H, mem_len, ps = 8, 32, 8192, 64
+        mp = (mem_len + 64 + ps) // ps
+        g_cpu = torch.Generator().manual_seed(5)
+        table = torch.randperm(B * mp, generator=g_cpu).to(torch.int32).view(B, mp).to(dev)
+        kpool = synthetic.big_normal_(torch.empty(B * mp, H, ps, D, dtype=bf, device=dev), 1, std)
+        vpool = synthetic.big_normal_(torch.empty(B * mp, H, ps, D, dtype=bf, device=dev), 2, std)
+        q, kn, vn = (x.to(dev) for x in synthetic.qkv(B, H, 1, D, 3, std, bf))
+        o = torch.empty_like(q)
+        ws = torch.empty(max(16, L.loma_decode_workspace_bytes(B, H, D, mem_len + 64)), dtype=torch.uint8, device=dev)
+        for r in range(args.reps):
+            lens = torch.full((B,), mem_len + 31 + r, dtype=torch.int32, device=dev)
+            L.loma_decode_attn_paged(q, kn, vn, kpool, vpool, table, o, None, lens, mem_len + 63, ws)
+    elif case in ("decode", "compress", "compress_prior", "compress_b32"):
         B, H, c, t, mem_len = 8, 32, 4, 16, 8192          # 1/4 of the generation workload's batch: 1.08 GB of cache
         if case == "compress_b32":
             B = 32                                         # the generation workload's own batch (1024 CTAs: two waves), 4.3 GB
@@ -856,7 +870,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-extras", action="store_true", help="skip the large and the context workloads timed at N=1")
-    ap.add_argument("--profile-case", choices=["decode", "compress", "compress_prior", "compress_b32", "masked", "masked_long", "bwd", "bwd_long", "prefill",
+    ap.add_argument("--profile-case", choices=["decode", "decode_paged", "compress", "compress_prior", "compress_b32", "masked", "masked_long", "bwd", "bwd_long", "prefill",
                                                      "prefill_ragged"],
                     help="run one cut-down kernel launch sequence (for profiler captures) and exit")
     ap.add_argument("--reps", type=int, default=3, help="launches of --profile-case")
