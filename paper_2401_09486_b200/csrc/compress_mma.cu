@@ -390,26 +390,27 @@ compress_mma_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bfloat16
 // current one was measured slower: its two buffers leave two CTAs per SM, too few warps to cover the
 // latencies of the arithmetic.)
 struct CmpOneStageLayout {
-    int rowb;       // padded K / V / Q row in bytes: conflict-free ldmatrix
+    int rowb;       // K / V / Q row in bytes, unpadded: 16-byte chunk c of row r lies at chunk c ^ (r & 7), which keeps
+                    // ldmatrix free of bank conflicts without the padding (five CTAs per SM at 80 keys instead of four)
     int srow;       // fp32 scores per row
-    int prowb;      // bf16 probabilities per row, padded like the operand rows
+    int prowb;      // bf16 probabilities per row, padded
     int kv_bytes;   // K rows, V rows, Q rows
-    int s_off, p_off, ml_off, rope_off, total;
+    int s_off, p_off, ml_off, rope_off, total;   // scores and probabilities lie over the K rows, which are dead by then
 };
 __host__ __device__ inline CmpOneStageLayout cmp_one_stage_layout(int D, int nk16, bool rope) {
     CmpOneStageLayout l;
-    l.rowb = D * 2 + 16;
+    l.rowb = D * 2;
     l.srow = nk16 + 4;
     l.prowb = nk16 * 2 + 16;
     l.kv_bytes = (2 * nk16 + 16) * l.rowb;
-    l.s_off = l.kv_bytes;
+    l.s_off = 0;                               // 16 * (nk16 + 4) * 4 + 16 * (2 nk16 + 16) <= nk16 * rowb for nk16 >= 16
     l.p_off = l.s_off + 16 * l.srow * 4;
-    l.ml_off = l.p_off + 16 * l.prowb;
+    l.ml_off = l.kv_bytes;
     l.rope_off = l.ml_off + 32 * 4;
     l.total = l.rope_off + (rope ? 16 * (D / 2) * 8 : 0);
     return l;
 }
-constexpr int CMP_ONE_STAGE_MAX_SMEM = 72 * 1024;       // three CTAs of four warps per SM
+constexpr int CMP_ONE_STAGE_MAX_SMEM = 72 * 1024;       // three CTAs of four warps per SM (nk16 <= 96: three 8-key tiles a warp)
 constexpr int CMP_ONE_STAGE_MAX_SMEM_8W = 110 * 1024;   // two CTAs of eight warps per SM; longer ranges take the pipelined kernel
 
 template <int D, int WARPS>
@@ -430,6 +431,7 @@ compress_one_stage_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bf
     const CmpOneStageLayout lay = cmp_one_stage_layout(D, nk16, rope.on != 0);
     const int ROWB = lay.rowb;
     const int K_OFF = 0, V_OFF = nk16 * ROWB, Q_OFF = 2 * nk16 * ROWB;
+    auto sw = [&](int row, int chunk) -> int { return row * ROWB + ((chunk ^ (row & 7)) << 4); };   // byte offset of a 16-byte chunk
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3, mi = lane >> 3;
 
@@ -462,13 +464,13 @@ compress_one_stage_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bf
             if (r < tc) { const int64_t off = cache_row(bh, mem_len + r); ksrc = k_cache + off; vsrc = v_cache + off; }
             else { ksrc = km + (int64_t)(r - tc) * D; vsrc = vm + (int64_t)(r - tc) * D; }
         }
-        cp_async16(base + K_OFF + r * ROWB + cv * 16, ksrc + cv * 8, valid);
-        cp_async16(base + V_OFF + r * ROWB + cv * 16, vsrc + cv * 8, valid);
+        cp_async16(base + K_OFF + sw(r, cv), ksrc + cv * 8, valid);
+        cp_async16(base + V_OFF + sw(r, cv), vsrc + cv * 8, valid);
     }
     for (int e = threadIdx.x; e < 16 * VPR; e += NTH) {
         const int r = e / VPR, cv = e - r * VPR;
         const bool valid = r < t;          // query rows >= t are zero
-        cp_async16(base + Q_OFF + r * ROWB + cv * 16, q_mem + ((int64_t)bh * t + (valid ? r : 0)) * D + cv * 8, valid);
+        cp_async16(base + Q_OFF + sw(r, cv), q_mem + ((int64_t)bh * t + (valid ? r : 0)) * D + cv * 8, valid);
     }
     cp_async_commit();
 
@@ -494,11 +496,14 @@ compress_one_stage_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bf
         for (int e = threadIdx.x; e < 2 * t * (D / 2); e += NTH) {
             const int which = e / (t * (D / 2)), e2 = e - which * t * (D / 2);
             const int r = e2 / (D / 2), d = e2 - r * (D / 2);
-            __nv_bfloat16* x = reinterpret_cast<__nv_bfloat16*>(smem + (which ? K_OFF + (tc + r) * ROWB : Q_OFF + r * ROWB));
+            const int row = which ? tc + r : r;
+            uint8_t* rowp = smem + (which ? K_OFF : Q_OFF);
+            __nv_bfloat16* xa = reinterpret_cast<__nv_bfloat16*>(rowp + sw(row, d >> 3)) + (d & 7);
+            __nv_bfloat16* xb = reinterpret_cast<__nv_bfloat16*>(rowp + sw(row, (d + D / 2) >> 3)) + (d & 7);
             const float2 cs = rope_tab[r * (D / 2) + d];
-            const float a = __bfloat162float(x[d]), b = __bfloat162float(x[d + D / 2]);
-            x[d] = __float2bfloat16_rn(a * cs.x - b * cs.y);
-            x[d + D / 2] = __float2bfloat16_rn(b * cs.x + a * cs.y);
+            const float a = __bfloat162float(*xa), b = __bfloat162float(*xb);
+            *xa = __float2bfloat16_rn(a * cs.x - b * cs.y);
+            *xb = __float2bfloat16_rn(b * cs.x + a * cs.y);
         }
         __syncthreads();
     }
@@ -507,32 +512,45 @@ compress_one_stage_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bf
     for (int e = threadIdx.x; e < t * VPR; e += NTH) {
         const int r = e / VPR, cv = e - r * VPR;
         const int64_t off = cache_row(bh, mem_len + r) + cv * 8;
-        *reinterpret_cast<uint4*>(k_cache + off) = *reinterpret_cast<const uint4*>(smem + K_OFF + (tc + r) * ROWB + cv * 16);
-        *reinterpret_cast<uint4*>(v_cache + off) = *reinterpret_cast<const uint4*>(smem + V_OFF + (tc + r) * ROWB + cv * 16);
+        *reinterpret_cast<uint4*>(k_cache + off) = *reinterpret_cast<const uint4*>(smem + K_OFF + sw(tc + r, cv));
+        *reinterpret_cast<uint4*>(v_cache + off) = *reinterpret_cast<const uint4*>(smem + V_OFF + sw(tc + r, cv));
     }
 
     // scores: tensor-core tiles of 8 keys, dealt to the warps round robin
     {
+        constexpr int MAXT = 3;                    // 8-key tiles per warp (the launcher keeps nk16 / 8 <= MAXT * WARPS)
         uint32_t qa[D / 16][4];
-        const uint32_t qrow = base + Q_OFF + ((mi & 1) * 8 + (lane & 7)) * ROWB + (mi >> 1) * 16;
+        const int qr = (mi & 1) * 8 + (lane & 7);
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) ldsm_x4(qrow + kk * 32, qa[kk]);
-        for (int nt = warp; nt < nk16 / 8; nt += WARPS) {
-            float sc[4] = {0.f, 0.f, 0.f, 0.f};
-            const uint32_t krow = base + K_OFF + (nt * 8 + (lane & 7)) * ROWB + mi * 16;
+        for (int kk = 0; kk < D / 16; ++kk) ldsm_x4(base + Q_OFF + sw(qr, 2 * kk + (mi >> 1)), qa[kk]);
+        float sc[MAXT][4];
 #pragma unroll
-            for (int k2 = 0; k2 < D / 32; ++k2) {
-                uint32_t kf[4];   // 8 keys x 32 features: the B fragments of two k-steps
-                ldsm_x4(krow + k2 * 64, kf);
-                mma_bf16_16816(sc, qa[2 * k2], kf[0], kf[1]);
-                mma_bf16_16816(sc, qa[2 * k2 + 1], kf[2], kf[3]);
+        for (int i = 0; i < MAXT; ++i) {
+            sc[i][0] = sc[i][1] = sc[i][2] = sc[i][3] = 0.f;
+            const int nt = warp + i * WARPS;
+            if (nt < nk16 / 8) {
+                const int kr = nt * 8 + (lane & 7);
+#pragma unroll
+                for (int k2 = 0; k2 < D / 32; ++k2) {
+                    uint32_t kf[4];   // 8 keys x 32 features: the B fragments of two k-steps
+                    ldsm_x4(base + K_OFF + sw(kr, 4 * k2 + mi), kf);
+                    mma_bf16_16816(sc[i], qa[2 * k2], kf[0], kf[1]);
+                    mma_bf16_16816(sc[i], qa[2 * k2 + 1], kf[2], kf[3]);
+                }
             }
-            const int col = nt * 8 + 2 * tq;
-            const bool v0 = col < nkeys, v1 = col + 1 < nkeys;
-            *reinterpret_cast<float2*>(S + g * lay.srow + col) =
-                make_float2(v0 ? sc[0] * scale_log2 : -INFINITY, v1 ? sc[1] * scale_log2 : -INFINITY);
-            *reinterpret_cast<float2*>(S + (g + 8) * lay.srow + col) =
-                make_float2(v0 ? sc[2] * scale_log2 : -INFINITY, v1 ? sc[3] * scale_log2 : -INFINITY);
+        }
+        __syncthreads();   // every read of the K rows (score products, compaction) is done: the scores go over them
+#pragma unroll
+        for (int i = 0; i < MAXT; ++i) {
+            const int nt = warp + i * WARPS;
+            if (nt < nk16 / 8) {
+                const int col = nt * 8 + 2 * tq;
+                const bool v0 = col < nkeys, v1 = col + 1 < nkeys;
+                *reinterpret_cast<float2*>(S + g * lay.srow + col) =
+                    make_float2(v0 ? sc[i][0] * scale_log2 : -INFINITY, v1 ? sc[i][1] * scale_log2 : -INFINITY);
+                *reinterpret_cast<float2*>(S + (g + 8) * lay.srow + col) =
+                    make_float2(v0 ? sc[i][2] * scale_log2 : -INFINITY, v1 ? sc[i][3] * scale_log2 : -INFINITY);
+            }
         }
     }
     __syncthreads();
@@ -568,14 +586,14 @@ compress_one_stage_kernel(const __nv_bfloat16* __restrict__ q_mem, const __nv_bf
 #pragma unroll
         for (int j = 0; j < NT; ++j) { oacc[j][0] = oacc[j][1] = oacc[j][2] = oacc[j][3] = 0.f; }
         const uint32_t prow = sbase + lay.p_off + ((mi & 1) * 8 + (lane & 7)) * lay.prowb + (mi >> 1) * 16;
-        const uint32_t vrow = base + V_OFF + ((mi & 1) * 8 + (lane & 7)) * ROWB + (mi >> 1) * 16 + warp * (D / WARPS) * 2;
+        const int vr = (mi & 1) * 8 + (lane & 7), vchunk = (mi >> 1) + warp * (D / WARPS) / 8;
         for (int ks = 0; ks < nk16 / 16; ++ks) {
             uint32_t pa[4];
             ldsm_x4(prow + ks * 32, pa);
 #pragma unroll
             for (int jd = 0; jd < NT; jd += 2) {
                 uint32_t vf[4];
-                ldsm_x4_trans(vrow + ks * 16 * ROWB + jd * 16, vf);
+                ldsm_x4_trans(base + V_OFF + sw(ks * 16 + vr, vchunk + jd), vf);
                 mma_bf16_16816(oacc[jd], pa, vf[0], vf[1]);
                 mma_bf16_16816(oacc[jd + 1], pa, vf[2], vf[3]);
             }
@@ -655,12 +673,15 @@ static cudaError_t compress_bf16_t(const void* qm, const void* km, const void* v
     int prior_len = 0;
     if (nprior > 0) prior_len = ((mem_len + nprior - 1) / nprior + 15) / 16 * 16;
     const int nsp = nprior + 1;
-    const CmpOneStageLayout wl = cmp_one_stage_layout(D, (tc + t + 15) & ~15, rope.on != 0);
-    if (nprior == 0 && t <= 16 && wl.total <= (D == 128 ? CMP_ONE_STAGE_MAX_SMEM_8W : CMP_ONE_STAGE_MAX_SMEM)) {
-        // default mask, short range: the whole range in one stage; four warps while three CTAs fit an SM, eight
-        // (D = 128 only: a warp owns at least 16 output columns) while two do
+    const int nk16 = (tc + t + 15) & ~15;
+    const CmpOneStageLayout wl = cmp_one_stage_layout(D, nk16, rope.on != 0);
+    // default mask, short range: the whole range in one stage.  A warp holds the scores of at most three 8-key tiles:
+    // four warps up to 96 keys, eight (D = 128 only: a warp owns at least 16 output columns) up to 192, and two CTAs an SM
+    const bool narrow = nk16 <= 96 && wl.total <= CMP_ONE_STAGE_MAX_SMEM;
+    const bool wide8 = !narrow && D == 128 && nk16 <= 192 && wl.total <= CMP_ONE_STAGE_MAX_SMEM_8W;
+    if (nprior == 0 && t <= 16 && (narrow || wide8)) {
         constexpr int W8 = D == 128 ? 8 : 4;
-        const bool wide = wl.total > CMP_ONE_STAGE_MAX_SMEM;
+        const bool wide = wide8;
         static bool attr1_set[64] = {false};   // per device, per template instance
         int dev1 = 0;
         if (cudaGetDevice(&dev1) != cudaSuccess || dev1 < 0 || dev1 >= 64) return cudaErrorInvalidDevice;
