@@ -354,7 +354,7 @@ def run_ours(args):
         "compress": {"ms": t_cmp, "bytes": cmp_bytes, "gbs": cmp_gbs,
                      "frac_of_measured_hbm": cmp_gbs / peaks["hbm_gbs"],
                      "note": "timed in place after the 64 decodes of the cycle"},
-        "roofline": {"kernel": "decode_splitkv_kernel<128> (+ merge), per loma_decode_attn call", "bound": "hbm",
+        "roofline": {"kernel": "decode_splitkv_kernel<128, false> (+ decode_merge_kernel<128>), per loma_decode_attn call", "bound": "hbm",
                      "achieved": dec_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                      "frac": dec_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
                      # dram__bytes_read + write of one launch: captured on the B8 case and scaled by the (b,h) count, 1024 / 256
@@ -681,7 +681,7 @@ def large_workloads(L, synthetic, torch, dev, peaks, steps, warmup, clocks_mhz):
         "config": dict(B=B, H=H, D=D, c=c, t=t, mem_len=mem_len, cap=cap, decode_steps=tc), "steps": steps,
         "cycle_ms": t_dec + t_cmp, "decode_ms_per_call": dec_ms_call, "decode_ms_x_sm_ghz": dec_ms_call * ghz if ghz else None,
         "decode_gbs": dec_gbs, "decode_bytes_per_call": dec_bytes_call, "compress_ms": t_cmp, "compress_gbs": cmp_gbs,
-        "roofline": {"kernel": "decode_splitkv_kernel<128> (+ merge), per loma_decode_attn call", "bound": "hbm", "achieved": dec_gbs,
+        "roofline": {"kernel": "decode_splitkv_kernel<128, false> (+ decode_merge_kernel<128>), per loma_decode_attn call", "bound": "hbm", "achieved": dec_gbs,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": dec_gbs / peaks["hbm_gbs"], "frac_of_8tbs": dec_gbs / 8000.0,
                      "peak_source": peaks["source"],
                      # every (b, h) streams its own rows once: the B8 / 8224-row capture scaled by rows and (b, h) pairs
